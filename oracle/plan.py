@@ -1,0 +1,106 @@
+"""Index construction for a compaction event, restated in plain Python.
+
+TEST INFRASTRUCTURE ONLY.  Follows the paper's Section 4 ("Snapshot &
+partition": a history of |X| tokens becomes N = ceil(|X| / B) contiguous blocks,
+the last one possibly short; "Dispatch": one sequence per block) and the paged
+KV bookkeeping a serving engine keeps underneath (Section 4.2 names the engine;
+the paper gives no detail, so the rules below are this library's own and are
+stated in full):
+
+* cu_seqlens      prefix sums of the block lengths
+* pages           block b owns ceil((L_b + T) / P) pages, T = reserved summary
+                  tokens; pages are dealt block by block, in order, from the
+                  caller's free list
+* slot of token p of block b:  page_indices[page_indptr[b] + p // P] * P + p % P
+* prefill items   (block, q_tile) for q_tile < ceil(L_b / q_tile_rows); cost is
+                  the number of keys its last row sees; order: descending cost,
+                  ties by ascending block, then tile
+* decode items    (block, kv_head, split): split s covers pages
+                  [s*C, min((s+1)*C, pages_b)); order: descending page count,
+                  ties by ascending block, kv head, split
+* split_indptr    prefix sums of ceil(pages_b / C)
+"""
+from __future__ import annotations
+
+from typing import Dict, Sequence
+
+
+def partition(history_len: int, block_size: int):
+    """Section 4, step 1: N = ceil(|X| / B) contiguous blocks of B tokens."""
+    if history_len < 1 or block_size < 1:
+        raise ValueError("lengths must be positive")
+    n = -(-history_len // block_size)
+    lens = [block_size] * (n - 1)
+    lens.append(history_len - block_size * (n - 1))
+    return lens
+
+
+def build_plan(block_lens: Sequence[int], max_new_tokens: int, page_size: int,
+               free_pages: Sequence[int], num_kv_heads: int,
+               q_tile_rows: int, pages_per_split: int) -> Dict[str, list]:
+    B = len(block_lens)
+    if B < 1:
+        raise ValueError("need at least one block")
+    if any(int(L) < 1 for L in block_lens):
+        raise ValueError("block lengths must be >= 1")
+    if max_new_tokens < 0 or page_size < 1 or q_tile_rows < 1 or pages_per_split < 1:
+        raise ValueError("bad parameter")
+
+    cu = [0]
+    for L in block_lens:
+        cu.append(cu[-1] + int(L))
+
+    pages_per_block = []
+    for L in block_lens:
+        tokens = int(L) + max_new_tokens
+        pages_per_block.append((tokens + page_size - 1) // page_size)
+    indptr = [0]
+    for n in pages_per_block:
+        indptr.append(indptr[-1] + n)
+    if indptr[-1] > len(free_pages):
+        raise MemoryError("not enough free pages")
+    page_indices = [int(free_pages[i]) for i in range(indptr[-1])]
+
+    slot_mapping = []
+    for b, L in enumerate(block_lens):
+        for p in range(int(L)):
+            page = page_indices[indptr[b] + p // page_size]
+            slot_mapping.append(page * page_size + p % page_size)
+
+    prefill = []
+    for b, L in enumerate(block_lens):
+        n_tiles = (int(L) + q_tile_rows - 1) // q_tile_rows
+        for t in range(n_tiles):
+            cost = min((t + 1) * q_tile_rows, int(L))
+            prefill.append((-cost, b, t))
+    prefill.sort()
+    prefill_items = [[b, t] for (_, b, t) in prefill]
+
+    split_indptr = [0]
+    decode = []
+    for b, n in enumerate(pages_per_block):
+        n_splits = (n + pages_per_split - 1) // pages_per_split
+        split_indptr.append(split_indptr[-1] + n_splits)
+        for g in range(num_kv_heads):
+            for s in range(n_splits):
+                size = min(pages_per_split, n - s * pages_per_split)
+                decode.append((-size, b, g, s))
+    decode.sort()
+    decode_items = [[b, g, s] for (_, b, g, s) in decode]
+
+    return {
+        "cu_seqlens": cu,
+        "page_indptr": indptr,
+        "page_indices": page_indices,
+        "seq_lens": [0] * B,
+        "slot_mapping": slot_mapping,
+        "prefill_items": prefill_items,
+        "decode_items": decode_items,
+        "split_indptr": split_indptr,
+    }
+
+
+def slot_of(plan: Dict[str, list], page_size: int, block: int, pos: int) -> int:
+    """Pool slot (page * P + offset) of position `pos` of `block`."""
+    page = plan["page_indices"][plan["page_indptr"][block] + pos // page_size]
+    return page * page_size + pos % page_size
