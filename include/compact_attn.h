@@ -1,0 +1,192 @@
+/*
+ * libcompact_attn -- attention for parallel context compaction on one B200 (sm_100a).
+ *
+ * Problem statement (paper, Section 4 "Parallel Compaction"): when a history
+ * exceeds the threshold it is snapshotted and cut into N contiguous blocks
+ * ("Snapshot & partition", N = ceil(|X| / B), last block possibly short); every
+ * block is handed to its own summarisation sequence and all N run concurrently
+ * ("Dispatch"); the N summaries are concatenated in block order ("Merge").  This
+ * library runs the attention of those N concurrent sequences in the
+ * "independent chunks" layout of Section 4: a sequence sees its own block only,
+ * so attention is block-diagonal and causal inside each block.  Sequential
+ * compaction (Section 2.2, Eq. 1) is the N = 1 case of the same calls.
+ *
+ * The paper does not spell out attention; it is the textbook operation
+ *     O[i,h,:] = sum_{j<=i} softmax_j(scale * q[i,h,:].k[j,g,:]) v[j,g,:],  g = h div G,
+ * with G = num_q_heads / num_kv_heads (contiguous head groups), keys restricted
+ * to the query's own block.
+ *
+ * Conventions for every call
+ *   - "host" pointers are ordinary CPU memory, "device" pointers are CUDA global
+ *     memory of the current device.  The library allocates NO device memory: all
+ *     device buffers belong to the caller, with sizes taken from cpa_plan_param.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default
+ *     stream).  Device work is enqueued asynchronously on it.
+ *   - Tensors are bf16.  Packed token-major layout [tokens, heads, head_dim] for
+ *     Q/K/V/O, blocks back to back in block order (offsets = cu_seqlens).
+ *     KV pools are [num_pages, num_kv_heads, page_size, head_dim], one pool for K
+ *     and one for V; a (page, head) chunk is contiguous.
+ *   - Every call returns 0 (CPA_OK) or a negative cpa_status.  Nothing throws,
+ *     exits, or traps the device.  Device-side waits are bounded; if one gives up
+ *     the kernel records it in the plan's device status word, which
+ *     cpa_plan_status reads back.
+ *   - There is no CPU fallback: without a CUDA device the compute calls return
+ *     CPA_ECUDA.
+ */
+#ifndef COMPACT_ATTN_H_
+#define COMPACT_ATTN_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#if defined(__GNUC__)
+#define CPA_API __attribute__((visibility("default")))
+#else
+#define CPA_API
+#endif
+
+typedef enum cpa_status {
+    CPA_OK = 0,
+    CPA_EINVAL = -1,       /* bad argument: null/misaligned pointer, length < 1, heads not divisible ... */
+    CPA_ENOSPC = -2,       /* free list too short, caller buffer too small, or append beyond the reservation */
+    CPA_EUNSUPPORTED = -3, /* head_dim not in {64,128}, page_size != 16, group size > 8 ... */
+    CPA_ECUDA = -4,        /* a CUDA runtime/driver call failed (no device, launch error) */
+    CPA_ETIMEOUT = -5,     /* a bounded device-side wait gave up (read from the status word) */
+    CPA_ESTATE = -6        /* call order violated (e.g. compute before cpa_plan_upload) */
+} cpa_status;
+
+typedef struct cpa_config {
+    int32_t num_q_heads;
+    int32_t num_kv_heads;    /* must divide num_q_heads; group size G <= 8 */
+    int32_t head_dim;        /* 64 or 128 */
+    int32_t page_size;       /* 16 */
+    float   scale;           /* softmax scale, normally 1/sqrt(head_dim) */
+    int32_t q_tile_rows;     /* query rows per prefill work item; 0 = default (128) */
+    int32_t pages_per_split; /* KV pages per decode work item; 0 = chosen from the batch */
+    int32_t num_sms;         /* SM count the split heuristic aims at; 0 = 148 */
+} cpa_config;
+
+typedef struct cpa_plan cpa_plan; /* opaque; host memory owned by the library */
+
+/* Index arrays a plan holds (all int32), for cpa_plan_export. */
+enum {
+    CPA_ARR_CU_SEQLENS = 0,    /* [B+1] prefix sums of block lengths */
+    CPA_ARR_PAGE_INDPTR = 1,   /* [B+1] prefix sums of pages per block */
+    CPA_ARR_PAGE_INDICES = 2,  /* [page_indptr[B]] pool page ids, block-major */
+    CPA_ARR_SEQ_LENS = 3,      /* [B] tokens cached per block (host mirror) */
+    CPA_ARR_SLOT_MAPPING = 4,  /* [tokens] pool slot (page*P + offset) of every prefill token */
+    CPA_ARR_PREFILL_ITEMS = 5, /* [n,2] (block, q_tile) in launch order */
+    CPA_ARR_DECODE_ITEMS = 6,  /* [n,3] (block, kv_head, split) in launch order */
+    CPA_ARR_SPLIT_INDPTR = 7   /* [B+1] prefix sums of decode splits per block */
+};
+
+/* Scalars of a plan, for cpa_plan_param. */
+enum {
+    CPA_PARAM_NUM_BLOCKS = 0,
+    CPA_PARAM_TOTAL_TOKENS = 1,
+    CPA_PARAM_Q_TILE_ROWS = 2,
+    CPA_PARAM_PAGES_PER_SPLIT = 3,
+    CPA_PARAM_PAGES_USED = 4,            /* page_indptr[B] */
+    CPA_PARAM_INDEX_BYTES = 5,           /* size of the device index buffer for cpa_plan_upload */
+    CPA_PARAM_DECODE_WORKSPACE_BYTES = 6,/* size of cpa_decode's device workspace */
+    CPA_PARAM_TOTAL_SPLITS = 7,          /* split_indptr[B] */
+    CPA_PARAM_MAX_NEW_TOKENS = 8
+};
+
+/*
+ * cpa_plan -- "Snapshot & partition" + "Dispatch" bookkeeping (Section 4).
+ * Builds, on the host, everything the kernels index with:
+ *   cu_seqlens; per block ceil((L_b + max_new_tokens) / page_size) pages taken in
+ *   order from `free_pages` (block 0 first); seq_lens (0: nothing cached yet);
+ *   the slot of every prefill token; the prefill work list of (block, q_tile)
+ *   ordered by descending cost (keys seen by the tile's last row), ties by
+ *   ascending block then tile; the decode work list of (block, kv_head, split),
+ *   split s = pages [s*C, (s+1)*C) of the block, ordered by descending page
+ *   count, ties by ascending block, kv head, split.
+ * block_lens, free_pages: host int32 arrays (copied; caller keeps ownership).
+ * Page ids must be >= 0 and distinct (distinctness is the caller's contract).
+ * Errors: CPA_EINVAL (null pointer, num_blocks < 1, a length < 1,
+ * max_new_tokens < 0, negative page id, heads not divisible), CPA_EUNSUPPORTED,
+ * CPA_ENOSPC (num_free too small).  On error *out is NULL.
+ */
+CPA_API int cpa_plan_create(const cpa_config* cfg, int32_t num_blocks, const int32_t* block_lens,
+                    int32_t max_new_tokens, const int32_t* free_pages, int32_t num_free,
+                    cpa_plan** out);
+
+/* Borrow a host view of one index array (valid until the plan is destroyed or,
+ * for CPA_ARR_SEQ_LENS, until the next cpa_kv_append).  Errors: CPA_EINVAL. */
+CPA_API int cpa_plan_export(const cpa_plan* plan, int which, const int32_t** ptr, int64_t* count);
+
+/* One scalar of the plan, or a negative cpa_status for an unknown `which`. */
+CPA_API int64_t cpa_plan_param(const cpa_plan* plan, int which);
+
+/*
+ * Copy the index arrays into the caller's device buffer (>= CPA_PARAM_INDEX_BYTES
+ * bytes, 16-byte aligned) on `stream` and bind the plan to that buffer; device
+ * seq_lens and the status word start at 0.  The buffer must stay alive and
+ * untouched by the caller until the plan is destroyed.  Errors: CPA_EINVAL,
+ * CPA_ENOSPC (bytes too small), CPA_ECUDA.
+ */
+CPA_API int cpa_plan_upload(cpa_plan* plan, void* d_index_buf, int64_t bytes, void* stream);
+
+/* Synchronise `stream`, read the device status word: CPA_OK, CPA_ETIMEOUT, or
+ * CPA_ECUDA if the stream reports an error.  CPA_ESTATE before upload. */
+CPA_API int cpa_plan_status(cpa_plan* plan, void* stream);
+
+CPA_API void cpa_plan_destroy(cpa_plan* plan);
+
+/*
+ * cpa_prefill -- causal attention of every block over itself (the prefill each
+ * concurrent summarisation sequence runs over its block, Section 4 "Dispatch";
+ * block-diagonal because of the independent-chunks layout).
+ *   q, o : device bf16 [total_tokens, num_q_heads, head_dim]
+ *   k, v : device bf16 [total_tokens, num_kv_heads, head_dim]
+ * All four 16-byte aligned; o must not alias the inputs.  One launch covers all
+ * (block, q_tile, head) work items.  d_workspace is unused (may be NULL).
+ * Errors: CPA_EINVAL, CPA_ESTATE (plan not uploaded), CPA_ECUDA.
+ */
+CPA_API int cpa_prefill(const cpa_plan* plan, const void* q, const void* k, const void* v, void* o,
+                void* d_workspace, void* stream);
+
+/*
+ * cpa_kv_append -- write new K/V rows into the blocks' pages and advance
+ * seq_lens (the KV cache each sequence keeps while it decodes its summary).
+ *   k_new, v_new : device bf16 [sum(new_lens), num_kv_heads, head_dim], block-major
+ *   new_lens     : host int32 [B] tokens to add per block, or NULL = one token
+ *                  per block (a decode step; then k_new is [B, kv_heads, head_dim]).
+ * Token i of block b goes to position seq_lens[b] + i, i.e. pool slot
+ * page_indices[page_indptr[b] + pos / P] * P + pos % P.  With new_lens == NULL,
+ * or new_lens == block_lens on an empty cache, nothing is copied from the host,
+ * so the call can be recorded in a CUDA graph; otherwise B+1 offsets are copied
+ * to the device first.  Errors: CPA_EINVAL, CPA_ESTATE, CPA_ENOSPC (a block would
+ * outgrow L_b + max_new_tokens; nothing is launched), CPA_ECUDA.
+ */
+CPA_API int cpa_kv_append(cpa_plan* plan, const void* k_new, const void* v_new, const int32_t* new_lens,
+                  void* k_pool, void* v_pool, void* stream);
+
+/*
+ * cpa_decode -- one batched decode step: the newest token of every block
+ * attends over that block's whole cache, the token itself included (call
+ * cpa_kv_append for the step first).  Split-K over the block's pages, then a
+ * log-sum-exp merge of the split partials
+ *     m = max_s m_s,  l = sum_s l_s e^(m_s - m),  O = sum_s acc_s e^(m_s - m) / l.
+ *   q, o        : device bf16 [B, num_q_heads, head_dim]
+ *   k_pool/v_pool: device bf16 pools (read only)
+ *   d_workspace : device scratch, >= CPA_PARAM_DECODE_WORKSPACE_BYTES, 16-byte aligned;
+ *                 contents are overwritten; calls sharing one workspace must not overlap.
+ * Lengths are read from the device seq_lens, so T steps can be enqueued back to
+ * back without host synchronisation.  Errors: CPA_EINVAL, CPA_ESTATE, CPA_ECUDA.
+ */
+CPA_API int cpa_decode(const cpa_plan* plan, const void* q, const void* k_pool, const void* v_pool,
+               void* o, void* d_workspace, void* stream);
+
+/* Static text for a cpa_status value. */
+CPA_API const char* cpa_strerror(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* COMPACT_ATTN_H_ */

@@ -1,0 +1,150 @@
+"""ctypes binding of libcompact_attn: argument marshalling only.
+
+Every function has the name and argument order of its C entry point in
+``include/compact_attn.h``; device buffers are passed as torch tensors (their
+``data_ptr()`` is taken) or as raw integer addresses.  There is no fallback:
+if the shared library is missing, importing this module raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional, Sequence
+
+import numpy as np
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG, "libcompact_attn.so")
+
+CPA_OK, CPA_EINVAL, CPA_ENOSPC, CPA_EUNSUPPORTED, CPA_ECUDA, CPA_ETIMEOUT, CPA_ESTATE = 0, -1, -2, -3, -4, -5, -6
+
+ARR_CU_SEQLENS, ARR_PAGE_INDPTR, ARR_PAGE_INDICES, ARR_SEQ_LENS = 0, 1, 2, 3
+ARR_SLOT_MAPPING, ARR_PREFILL_ITEMS, ARR_DECODE_ITEMS, ARR_SPLIT_INDPTR = 4, 5, 6, 7
+_ARR_WIDTH = {ARR_PREFILL_ITEMS: 2, ARR_DECODE_ITEMS: 3}
+
+PARAM_NUM_BLOCKS, PARAM_TOTAL_TOKENS, PARAM_Q_TILE_ROWS, PARAM_PAGES_PER_SPLIT = 0, 1, 2, 3
+PARAM_PAGES_USED, PARAM_INDEX_BYTES, PARAM_DECODE_WORKSPACE_BYTES, PARAM_TOTAL_SPLITS = 4, 5, 6, 7
+PARAM_MAX_NEW_TOKENS = 8
+
+
+class cpa_config(ctypes.Structure):
+    _fields_ = [("num_q_heads", ctypes.c_int32), ("num_kv_heads", ctypes.c_int32),
+                ("head_dim", ctypes.c_int32), ("page_size", ctypes.c_int32),
+                ("scale", ctypes.c_float), ("q_tile_rows", ctypes.c_int32),
+                ("pages_per_split", ctypes.c_int32), ("num_sms", ctypes.c_int32)]
+
+
+class CpaError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {cpa_strerror(status)} ({status})")
+
+
+if not os.path.exists(LIB_PATH):
+    raise ImportError(
+        f"{LIB_PATH} is missing: build it with `python -m paper_2605_23296_b200.build` "
+        "(there is no fallback implementation)")
+_lib = ctypes.CDLL(LIB_PATH)
+
+_vp, _i32p = ctypes.c_void_p, ctypes.POINTER(ctypes.c_int32)
+_lib.cpa_plan_create.argtypes = [ctypes.POINTER(cpa_config), ctypes.c_int32, _i32p, ctypes.c_int32,
+                                 _i32p, ctypes.c_int32, ctypes.POINTER(_vp)]
+_lib.cpa_plan_create.restype = ctypes.c_int
+_lib.cpa_plan_export.argtypes = [_vp, ctypes.c_int, ctypes.POINTER(_i32p), ctypes.POINTER(ctypes.c_int64)]
+_lib.cpa_plan_export.restype = ctypes.c_int
+_lib.cpa_plan_param.argtypes = [_vp, ctypes.c_int]
+_lib.cpa_plan_param.restype = ctypes.c_int64
+_lib.cpa_plan_upload.argtypes = [_vp, _vp, ctypes.c_int64, _vp]
+_lib.cpa_plan_upload.restype = ctypes.c_int
+_lib.cpa_plan_status.argtypes = [_vp, _vp]
+_lib.cpa_plan_status.restype = ctypes.c_int
+_lib.cpa_plan_destroy.argtypes = [_vp]
+_lib.cpa_plan_destroy.restype = None
+_lib.cpa_prefill.argtypes = [_vp, _vp, _vp, _vp, _vp, _vp, _vp]
+_lib.cpa_prefill.restype = ctypes.c_int
+_lib.cpa_kv_append.argtypes = [_vp, _vp, _vp, _i32p, _vp, _vp, _vp]
+_lib.cpa_kv_append.restype = ctypes.c_int
+_lib.cpa_decode.argtypes = [_vp, _vp, _vp, _vp, _vp, _vp, _vp]
+_lib.cpa_decode.restype = ctypes.c_int
+_lib.cpa_strerror.argtypes = [ctypes.c_int]
+_lib.cpa_strerror.restype = ctypes.c_char_p
+
+
+def _ptr(x) -> Optional[int]:
+    """Device/host address of a tensor-like, or the integer itself."""
+    if x is None:
+        return None
+    if isinstance(x, int):
+        return x
+    return int(x.data_ptr())
+
+
+def _i32(a) -> np.ndarray:
+    return np.ascontiguousarray(a, dtype=np.int32)
+
+
+def cpa_strerror(status: int) -> str:
+    return _lib.cpa_strerror(int(status)).decode()
+
+
+def cpa_plan_create(cfg: cpa_config, block_lens: Sequence[int], max_new_tokens: int,
+                    free_pages: Sequence[int], check: bool = True):
+    """Returns the plan handle (int); raises CpaError unless check=False, then (status, handle)."""
+    lens, free = _i32(block_lens), _i32(free_pages)
+    out = _vp()
+    rc = _lib.cpa_plan_create(ctypes.byref(cfg), lens.shape[0], lens.ctypes.data_as(_i32p),
+                              int(max_new_tokens), free.ctypes.data_as(_i32p), free.shape[0],
+                              ctypes.byref(out))
+    if not check:
+        return rc, out.value
+    if rc != CPA_OK:
+        raise CpaError(rc, "cpa_plan_create")
+    return out.value
+
+
+def cpa_plan_export(plan: int, which: int) -> np.ndarray:
+    """Copy of one host index array; item lists come back as [n, width]."""
+    ptr, n = _i32p(), ctypes.c_int64()
+    rc = _lib.cpa_plan_export(plan, which, ctypes.byref(ptr), ctypes.byref(n))
+    if rc != CPA_OK:
+        raise CpaError(rc, "cpa_plan_export")
+    w = _ARR_WIDTH.get(which, 1)
+    if n.value == 0:
+        return np.zeros((0, w) if w > 1 else (0,), dtype=np.int32)
+    a = np.ctypeslib.as_array(ptr, shape=(n.value * w,)).copy()
+    return a.reshape(n.value, w) if w > 1 else a
+
+
+def cpa_plan_param(plan: int, which: int) -> int:
+    return int(_lib.cpa_plan_param(plan, which))
+
+
+def cpa_plan_upload(plan: int, d_index_buf, nbytes: int, stream: int = 0) -> int:
+    return _lib.cpa_plan_upload(plan, _ptr(d_index_buf), int(nbytes), stream or None)
+
+
+def cpa_plan_status(plan: int, stream: int = 0) -> int:
+    return _lib.cpa_plan_status(plan, stream or None)
+
+
+def cpa_plan_destroy(plan: int) -> None:
+    _lib.cpa_plan_destroy(plan)
+
+
+def cpa_prefill(plan: int, q, k, v, o, d_workspace=None, stream: int = 0) -> int:
+    return _lib.cpa_prefill(plan, _ptr(q), _ptr(k), _ptr(v), _ptr(o), _ptr(d_workspace), stream or None)
+
+
+def cpa_kv_append(plan: int, k_new, v_new, new_lens, k_pool, v_pool, stream: int = 0) -> int:
+    if new_lens is None:
+        lens_p = None
+    else:
+        lens = _i32(new_lens)
+        lens_p = lens.ctypes.data_as(_i32p)
+    return _lib.cpa_kv_append(plan, _ptr(k_new), _ptr(v_new), lens_p, _ptr(k_pool), _ptr(v_pool),
+                              stream or None)
+
+
+def cpa_decode(plan: int, q, k_pool, v_pool, o, d_workspace, stream: int = 0) -> int:
+    return _lib.cpa_decode(plan, _ptr(q), _ptr(k_pool), _ptr(v_pool), _ptr(o), _ptr(d_workspace),
+                           stream or None)

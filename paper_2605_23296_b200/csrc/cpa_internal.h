@@ -1,0 +1,62 @@
+// Internal definitions shared by the host planner and the kernel launchers.
+#pragma once
+
+#include <cstdint>
+#include <vector>
+
+#include "compact_attn.h"
+
+// Device-side view of the uploaded index buffer.
+struct cpa_dev_index {
+    int32_t* status;               // [4]  word 0: first timeout/error code recorded by a kernel
+    const int32_t* cu_seqlens;     // [B+1]
+    const int32_t* page_indptr;    // [B+1]
+    const int32_t* split_indptr;   // [B+1]
+    int32_t* seq_lens;             // [B]   tokens cached per block (advanced by the append kernels)
+    int32_t* append_indptr;        // [B+1] source-row offsets of a general append
+    const int32_t* page_indices;   // [pages_used]
+    const int32_t* prefill_items;  // [n_prefill, 2]
+    const int32_t* decode_items;   // [n_decode, 4]  (block, kv_head, split, pages) padded to 16 bytes
+};
+
+struct cpa_plan {
+    cpa_config cfg;
+    int32_t B = 0;
+    int32_t T = 0;          // max_new_tokens
+    int32_t q_tile = 0;     // query rows per prefill item
+    int32_t C = 0;          // pages per decode split
+    int64_t total_tokens = 0;
+    std::vector<int32_t> block_lens, cu_seqlens, page_indptr, page_indices, seq_lens, slot_mapping,
+        prefill_items, decode_items, split_indptr;
+    int32_t n_prefill = 0, n_decode = 0;
+
+    // packed image of the device index buffer (int32 words) and offsets into it
+    std::vector<int32_t> image;
+    int64_t off_status = 0, off_cu = 0, off_pindptr = 0, off_sindptr = 0, off_seqlens = 0,
+            off_append = 0, off_pidx = 0, off_pitems = 0, off_ditems = 0, words = 0;
+    int32_t* d_base = nullptr;   // caller's device buffer after cpa_plan_upload
+    std::vector<int32_t> append_stage;  // host staging for general appends
+
+    int64_t index_bytes() const { return words * 4; }
+    int64_t decode_workspace_bytes() const {
+        // [rows, 2] (max, sum) padded to 16 bytes, then [rows, head_dim] accumulators, fp32
+        int64_t rows = (int64_t)split_indptr[B] * cfg.num_q_heads;
+        int64_t bytes = ((rows * 2 + 3) / 4 * 4 + rows * cfg.head_dim) * 4;
+        return (bytes + 255) / 256 * 256;
+    }
+    cpa_dev_index dev() const {
+        cpa_dev_index d;
+        d.status = d_base + off_status;
+        d.cu_seqlens = d_base + off_cu;
+        d.page_indptr = d_base + off_pindptr;
+        d.split_indptr = d_base + off_sindptr;
+        d.seq_lens = d_base + off_seqlens;
+        d.append_indptr = d_base + off_append;
+        d.page_indices = d_base + off_pidx;
+        d.prefill_items = d_base + off_pitems;
+        d.decode_items = d_base + off_ditems;
+        return d;
+    }
+};
+
+static inline bool cpa_aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }

@@ -1,0 +1,297 @@
+// Batched paged-KV decode attention: one query token per block over that block's
+// pages, split over the KV length, then a log-sum-exp merge of the split partials.
+//
+// The step is a streaming scan of the KV pool and is bound by HBM bandwidth: every
+// K and V element is read once per kv head, with 128-bit loads straight into
+// registers; the G query heads of a kv-head group share those registers.  The
+// per-key arithmetic runs on the legacy warp-level MMA (m16n8k16, bf16 in, fp32
+// accumulate), which costs nothing next to the memory stream and keeps the fp32
+// ALU free at G = 8:
+//   S  [heads(16, G used) x keys(8)]   = Q [heads x dims] . K^T      (A = Q, B = K rows)
+//   O^T[dims(16) x heads(8, G used)]  += V^T[dims x keys(16)] . P^T  (A = V^T, B = P)
+// Both contractions are invariant under a permutation of the contracted index, so
+// a thread loads whole 16-byte chunks and pairs registers up as the MMA fragments
+// need them; no shared-memory staging, no transposes.
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+
+#include "cpa_internal.h"
+
+namespace {
+
+constexpr int kDecodeWarps = 4;
+constexpr int kDecodeThreads = kDecodeWarps * 32;
+
+__device__ __forceinline__ void mma_bf16_16816(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                               uint32_t b0, uint32_t b1) {
+    asm volatile(
+        "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};\n"
+        : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+        : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
+    __nv_bfloat162 t = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<uint32_t*>(&t);
+}
+
+__device__ __forceinline__ uint4 ldg128(const void* p) {
+    uint4 r;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];\n"
+                 : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w)
+                 : "l"(p));
+    return r;
+}
+
+__device__ __forceinline__ uint32_t sel(const uint4& v, int i) {
+    return i == 0 ? v.x : i == 1 ? v.y : i == 2 ? v.z : v.w;
+}
+
+// One work item = (block, kv head, split of up to C pages).  Four warps take the
+// split's pages round-robin, each keeps its own running (max, sum, acc); the CTA
+// merges them in shared memory and writes one partial per query head.
+//   part_ml : [total_splits, Hq, 2]  (max in log2 units, sum), fp32
+//   part_o  : [total_splits, Hq, D]  unnormalised accumulators, fp32
+template <int D>
+__global__ void __launch_bounds__(kDecodeThreads, 4)
+decode_split_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ k_pool,
+                    const __nv_bfloat16* __restrict__ v_pool, float* __restrict__ part_ml,
+                    float* __restrict__ part_o, cpa_dev_index ix, int Hq, int Hkv, int G, int C,
+                    float scale_log2) {
+    constexpr int P = 16;
+    constexpr int KC = D / 32;  // 16-byte K chunks per thread per 8-key group
+    constexpr int VC = D / 64;  // 16-byte V chunks per thread per key row
+    const int4 item = reinterpret_cast<const int4*>(ix.decode_items)[blockIdx.x];
+    const int b = item.x, g = item.y, s = item.z;
+    const int len = ix.seq_lens[b];
+    const int pages_active = (len + P - 1) / P;
+    const int first = s * C;
+    if (first >= pages_active) return;  // split lies beyond the cached length (uniform per CTA)
+    const int last = min(first + C, pages_active);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int gid = lane >> 2, tig = lane & 3;
+
+    // Q fragments: row gid of the A tile is query head g*G + gid (zero rows beyond G)
+    uint4 qf[KC];
+#pragma unroll
+    for (int c = 0; c < KC; ++c) qf[c] = make_uint4(0, 0, 0, 0);
+    if (gid < G) {
+        const __nv_bfloat16* qrow = q + ((int64_t)b * Hq + g * G + gid) * D;
+#pragma unroll
+        for (int c = 0; c < KC; ++c) qf[c] = *reinterpret_cast<const uint4*>(qrow + (c * 4 + tig) * 8);
+    }
+
+    const int32_t* pages = ix.page_indices + ix.page_indptr[b];
+    uint4 kreg[2][KC];
+    uint4 vreg[4][VC];
+    auto load_k = [&](int pg) {
+        const __nv_bfloat16* base = k_pool + ((int64_t)pages[pg] * Hkv + g) * (P * D);
+#pragma unroll
+        for (int t = 0; t < 2; ++t)
+#pragma unroll
+            for (int c = 0; c < KC; ++c) kreg[t][c] = ldg128(base + (gid + 8 * t) * D + (c * 4 + tig) * 8);
+    };
+    auto load_v = [&](int pg) {
+        const __nv_bfloat16* base = v_pool + ((int64_t)pages[pg] * Hkv + g) * (P * D);
+#pragma unroll
+        for (int r = 0; r < 4; ++r) {
+            const int row = 2 * tig + (r & 1) + 8 * (r >> 1);
+#pragma unroll
+            for (int c = 0; c < VC; ++c) vreg[r][c] = ldg128(base + row * D + (c * 8 + gid) * 8);
+        }
+    };
+
+    float acc[VC][4][4];
+#pragma unroll
+    for (int c = 0; c < VC; ++c)
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+#pragma unroll
+            for (int e = 0; e < 4; ++e) acc[c][i][e] = 0.f;
+    float m_run = -INFINITY;  // running max of raw scores, row gid
+    float l_run = 0.f;        // this thread's share of the running sum, row gid
+
+    int pg = first + warp;
+    if (pg < last) { load_k(pg); load_v(pg); }
+    while (pg < last) {
+        // ---- S = Q K^T for the 16 keys of this page
+        float sc[2][4];
+#pragma unroll
+        for (int t = 0; t < 2; ++t) {
+            sc[t][0] = sc[t][1] = sc[t][2] = sc[t][3] = 0.f;
+#pragma unroll
+            for (int c = 0; c < KC; ++c) {
+                mma_bf16_16816(sc[t], qf[c].x, 0u, qf[c].y, 0u, kreg[t][c].x, kreg[t][c].y);
+                mma_bf16_16816(sc[t], qf[c].z, 0u, qf[c].w, 0u, kreg[t][c].z, kreg[t][c].w);
+            }
+        }
+        const int next = pg + kDecodeWarps;
+        if (next < last) load_k(next);
+
+        // ---- mask the tail of the last page by index, then online softmax (row gid)
+        const int key0 = pg * P + tig * 2;
+        const bool partial = (pg + 1) * P > len;
+        if (partial) {
+#pragma unroll
+            for (int t = 0; t < 2; ++t)
+#pragma unroll
+                for (int e = 0; e < 2; ++e)
+                    if (key0 + 8 * t + e >= len) sc[t][e] = -INFINITY;
+        }
+        float mx = fmaxf(fmaxf(sc[0][0], sc[0][1]), fmaxf(sc[1][0], sc[1][1]));
+        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
+        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
+        const float m_new = fmaxf(m_run, mx);  // finite: every visited page holds a valid key
+        const float alpha = (m_run == -INFINITY) ? 0.f : exp2f((m_run - m_new) * scale_log2);
+        const float mb = m_new * scale_log2;
+        float p[2][2];
+#pragma unroll
+        for (int t = 0; t < 2; ++t)
+#pragma unroll
+            for (int e = 0; e < 2; ++e) p[t][e] = exp2f(fmaf(sc[t][e], scale_log2, -mb));
+        // the row sum is taken over the bf16-rounded weights the MMA will multiply with
+        const uint32_t pb0 = pack_bf16x2(p[0][0], p[0][1]);
+        const uint32_t pb1 = pack_bf16x2(p[1][0], p[1][1]);
+        l_run = l_run * alpha + (__uint_as_float(pb0 << 16) + __uint_as_float(pb0 & 0xffff0000u)) +
+                (__uint_as_float(pb1 << 16) + __uint_as_float(pb1 & 0xffff0000u));
+        m_run = m_new;
+
+        // accumulator columns are heads 2*tig, 2*tig+1; their factors live in lanes of row = head
+        const float a0 = __shfl_sync(0xffffffffu, alpha, (2 * tig) * 4);
+        const float a1 = __shfl_sync(0xffffffffu, alpha, (2 * tig + 1) * 4);
+
+        if (partial) {  // unused slots may hold anything (even NaN): select them away
+#pragma unroll
+            for (int r = 0; r < 4; ++r) {
+                const int row = 2 * tig + (r & 1) + 8 * (r >> 1);
+                if (pg * P + row >= len) {
+#pragma unroll
+                    for (int c = 0; c < VC; ++c) vreg[r][c] = make_uint4(0, 0, 0, 0);
+                }
+            }
+        }
+        // ---- O^T += V^T P^T
+#pragma unroll
+        for (int c = 0; c < VC; ++c)
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                acc[c][i][0] *= a0; acc[c][i][1] *= a1; acc[c][i][2] *= a0; acc[c][i][3] *= a1;
+                const uint32_t r0 = sel(vreg[0][c], i), r1 = sel(vreg[1][c], i);
+                const uint32_t r2 = sel(vreg[2][c], i), r3 = sel(vreg[3][c], i);
+                mma_bf16_16816(acc[c][i], __byte_perm(r0, r1, 0x5410), __byte_perm(r0, r1, 0x7632),
+                               __byte_perm(r2, r3, 0x5410), __byte_perm(r2, r3, 0x7632), pb0, pb1);
+            }
+        if (next < last) load_v(next);
+        pg = next;
+    }
+    l_run += __shfl_xor_sync(0xffffffffu, l_run, 1);
+    l_run += __shfl_xor_sync(0xffffffffu, l_run, 2);
+
+    // ---- merge the four warps
+    __shared__ float sm_m[kDecodeWarps][8];
+    __shared__ float sm_l[kDecodeWarps][8];
+    __shared__ float sm_o[kDecodeWarps][8][D + 4];
+    if (tig == 0) { sm_m[warp][gid] = m_run * scale_log2; sm_l[warp][gid] = l_run; }
+#pragma unroll
+    for (int c = 0; c < VC; ++c)
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+#pragma unroll
+            for (int e = 0; e < 4; ++e)
+                sm_o[warp][2 * tig + (e & 1)][8 * (8 * c + gid) + 2 * i + (e >> 1)] = acc[c][i][e];
+    __syncthreads();
+
+    const int64_t prow = ((int64_t)(ix.split_indptr[b] + s) * Hq + g * G);
+    for (int idx = threadIdx.x; idx < G * D; idx += kDecodeThreads) {
+        const int h = idx / D, dim = idx - h * D;
+        float m = sm_m[0][h];
+#pragma unroll
+        for (int w = 1; w < kDecodeWarps; ++w) m = fmaxf(m, sm_m[w][h]);
+        float o = 0.f, l = 0.f;
+#pragma unroll
+        for (int w = 0; w < kDecodeWarps; ++w) {
+            const float mw = sm_m[w][h];
+            const float f = (mw == -INFINITY) ? 0.f : exp2f(mw - m);
+            o = fmaf(f, sm_o[w][h][dim], o);
+            l = fmaf(f, sm_l[w][h], l);
+        }
+        part_o[(prow + h) * D + dim] = o;
+        if (dim == 0) { part_ml[(prow + h) * 2] = m; part_ml[(prow + h) * 2 + 1] = l; }
+    }
+}
+
+// Merge of the split partials; one warp per (block, query head).
+template <int D>
+__global__ void __launch_bounds__(128)
+decode_combine_kernel(const float* __restrict__ part_ml, const float* __restrict__ part_o,
+                      __nv_bfloat16* __restrict__ out, cpa_dev_index ix, int B, int Hq, int C) {
+    constexpr int P = 16;
+    constexpr int E = D / 32;  // dims per lane
+    const int row = blockIdx.x * 4 + (threadIdx.x >> 5);
+    if (row >= B * Hq) return;
+    const int lane = threadIdx.x & 31;
+    const int b = row / Hq, h = row - b * Hq;
+    const int len = ix.seq_lens[b];
+    const int n_splits = ((len + P - 1) / P + C - 1) / C;
+    const int64_t base = (int64_t)ix.split_indptr[b] * Hq + h;
+    float m = -INFINITY;
+    for (int s = lane; s < n_splits; s += 32) m = fmaxf(m, part_ml[(base + (int64_t)s * Hq) * 2]);
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, off));
+    float o[E];
+#pragma unroll
+    for (int e = 0; e < E; ++e) o[e] = 0.f;
+    float l = 0.f;
+    for (int s = 0; s < n_splits; ++s) {
+        const int64_t r = base + (int64_t)s * Hq;
+        const float2 ml = *reinterpret_cast<const float2*>(part_ml + r * 2);
+        const float f = exp2f(ml.x - m);
+        l = fmaf(f, ml.y, l);
+        const float* po = part_o + r * D + lane * E;
+        if constexpr (E == 4) {
+            const float4 t = *reinterpret_cast<const float4*>(po);
+            o[0] = fmaf(f, t.x, o[0]); o[1] = fmaf(f, t.y, o[1]); o[2] = fmaf(f, t.z, o[2]); o[3] = fmaf(f, t.w, o[3]);
+        } else {
+            const float2 t = *reinterpret_cast<const float2*>(po);
+            o[0] = fmaf(f, t.x, o[0]); o[1] = fmaf(f, t.y, o[1]);
+        }
+    }
+    const float inv = n_splits > 0 ? 1.f / l : 0.f;
+    __nv_bfloat16* dst = out + (int64_t)row * D + lane * E;
+#pragma unroll
+    for (int e = 0; e < E; e += 2)
+        *reinterpret_cast<__nv_bfloat162*>(dst + e) = __floats2bfloat162_rn(o[e] * inv, o[e + 1] * inv);
+}
+
+template <int D>
+int launch_decode(const cpa_plan* plan, const void* q, const void* k_pool, const void* v_pool, void* o,
+                  void* ws, cudaStream_t st) {
+    const cpa_config& c = plan->cfg;
+    const int G = c.num_q_heads / c.num_kv_heads;
+    const cpa_dev_index ix = plan->dev();
+    float* part_ml = static_cast<float*>(ws);
+    float* part_o = part_ml + ((int64_t)plan->split_indptr[plan->B] * c.num_q_heads * 2 + 3) / 4 * 4;
+    const float scale_log2 = c.scale * 1.4426950408889634f;
+    decode_split_kernel<D><<<plan->n_decode, kDecodeThreads, 0, st>>>(
+        (const __nv_bfloat16*)q, (const __nv_bfloat16*)k_pool, (const __nv_bfloat16*)v_pool, part_ml, part_o, ix,
+        c.num_q_heads, c.num_kv_heads, G, plan->C, scale_log2);
+    const int rows = plan->B * c.num_q_heads;
+    decode_combine_kernel<D><<<(rows + 3) / 4, 128, 0, st>>>(part_ml, part_o, (__nv_bfloat16*)o, ix, plan->B,
+                                                            c.num_q_heads, plan->C);
+    return cudaGetLastError() == cudaSuccess ? CPA_OK : CPA_ECUDA;
+}
+
+}  // namespace
+
+extern "C" int cpa_decode(const cpa_plan* plan, const void* q, const void* k_pool, const void* v_pool, void* o,
+                          void* d_workspace, void* stream) {
+    if (!plan || !q || !k_pool || !v_pool || !o || !d_workspace) return CPA_EINVAL;
+    if (!cpa_aligned16(q) || !cpa_aligned16(k_pool) || !cpa_aligned16(v_pool) || !cpa_aligned16(o) ||
+        !cpa_aligned16(d_workspace))
+        return CPA_EINVAL;
+    if (!plan->d_base) return CPA_ESTATE;
+    cudaStream_t st = (cudaStream_t)stream;
+    return plan->cfg.head_dim == 128 ? launch_decode<128>(plan, q, k_pool, v_pool, o, d_workspace, st)
+                                     : launch_decode<64>(plan, q, k_pool, v_pool, o, d_workspace, st);
+}

@@ -1,0 +1,117 @@
+// Paged KV append: scatter new K/V rows into the pages each block owns and advance
+// the per-block cached length.  Pure data movement (bit-exact), bound by HBM.
+#include <cuda_runtime.h>
+
+#include "cpa_internal.h"
+
+namespace {
+
+// One 16-byte chunk of one (token, kv head) row.
+__device__ __forceinline__ void copy_row_chunks(const uint4* __restrict__ k_src, const uint4* __restrict__ v_src,
+                                                uint4* __restrict__ k_pool, uint4* __restrict__ v_pool,
+                                                int64_t page, int off, int Hkv, int chunks_per_head, int P) {
+    const int chunks = Hkv * chunks_per_head;
+    for (int c = threadIdx.x; c < chunks; c += blockDim.x) {
+        const int g = c / chunks_per_head;
+        const int j = c - g * chunks_per_head;
+        const int64_t dst = ((page * Hkv + g) * P + off) * chunks_per_head + j;
+        k_pool[dst] = k_src[c];
+        v_pool[dst] = v_src[c];
+    }
+}
+
+// Decode step: one new token per block.  CTA b is the only reader and writer of
+// seq_lens[b], so the length can be advanced in the same launch.
+__global__ void kv_append_step_kernel(const uint4* __restrict__ k_new, const uint4* __restrict__ v_new,
+                                      uint4* __restrict__ k_pool, uint4* __restrict__ v_pool,
+                                      cpa_dev_index ix, int Hkv, int chunks_per_head, int P) {
+    const int b = blockIdx.x;
+    const int pos = ix.seq_lens[b];
+    const int capacity = (ix.page_indptr[b + 1] - ix.page_indptr[b]) * P;
+    __syncthreads();  // every thread has read the length before thread 0 advances it
+    if (pos >= capacity) {  // host checks make this unreachable; never write outside the block's pages
+        if (threadIdx.x == 0) atomicCAS(ix.status, 0, 2);
+        return;
+    }
+    const int64_t page = ix.page_indices[ix.page_indptr[b] + pos / P];
+    const int64_t row = (int64_t)b * Hkv * chunks_per_head;
+    copy_row_chunks(k_new + row, v_new + row, k_pool, v_pool, page, pos % P, Hkv, chunks_per_head, P);
+    if (threadIdx.x == 0) ix.seq_lens[b] = pos + 1;
+}
+
+// Bulk append: `rows` new tokens, block-major; src_indptr[b] is the first row of block b.
+__global__ void kv_append_bulk_kernel(const uint4* __restrict__ k_new, const uint4* __restrict__ v_new,
+                                      uint4* __restrict__ k_pool, uint4* __restrict__ v_pool,
+                                      cpa_dev_index ix, const int32_t* __restrict__ src_indptr, int B,
+                                      int64_t rows, int Hkv, int chunks_per_head, int P) {
+    for (int64_t r = blockIdx.x; r < rows; r += gridDim.x) {
+        // block that owns row r: last b with src_indptr[b] <= r
+        int lo = 0, hi = B - 1;
+        while (lo < hi) {
+            const int mid = (lo + hi + 1) >> 1;
+            if ((int64_t)src_indptr[mid] <= r) lo = mid; else hi = mid - 1;
+        }
+        const int b = lo;
+        const int pos = ix.seq_lens[b] + (int)(r - src_indptr[b]);
+        const int64_t page = ix.page_indices[ix.page_indptr[b] + pos / P];
+        const int64_t row = r * Hkv * chunks_per_head;
+        copy_row_chunks(k_new + row, v_new + row, k_pool, v_pool, page, pos % P, Hkv, chunks_per_head, P);
+    }
+}
+
+__global__ void seq_lens_advance_kernel(cpa_dev_index ix, const int32_t* __restrict__ src_indptr, int B) {
+    const int b = blockIdx.x * blockDim.x + threadIdx.x;
+    if (b < B) ix.seq_lens[b] += src_indptr[b + 1] - src_indptr[b];
+}
+
+}  // namespace
+
+extern "C" int cpa_kv_append(cpa_plan* plan, const void* k_new, const void* v_new, const int32_t* new_lens,
+                             void* k_pool, void* v_pool, void* stream) {
+    if (!plan || !k_new || !v_new || !k_pool || !v_pool) return CPA_EINVAL;
+    if (!cpa_aligned16(k_new) || !cpa_aligned16(v_new) || !cpa_aligned16(k_pool) || !cpa_aligned16(v_pool))
+        return CPA_EINVAL;
+    if (!plan->d_base) return CPA_ESTATE;
+    const int B = plan->B, P = plan->cfg.page_size, Hkv = plan->cfg.num_kv_heads;
+    const int chunks_per_head = plan->cfg.head_dim / 8;
+    cudaStream_t st = (cudaStream_t)stream;
+    const cpa_dev_index ix = plan->dev();
+
+    // capacity check on the host mirror before anything is enqueued
+    bool is_prefill_bulk = new_lens != nullptr;
+    int64_t rows = 0;
+    for (int b = 0; b < B; ++b) {
+        const int n = new_lens ? new_lens[b] : 1;
+        if (n < 0) return CPA_EINVAL;
+        if ((int64_t)plan->seq_lens[b] + n > (int64_t)plan->block_lens[b] + plan->T) return CPA_ENOSPC;
+        if (new_lens && (plan->seq_lens[b] != 0 || n != plan->block_lens[b])) is_prefill_bulk = false;
+        rows += n;
+    }
+    if (rows == 0) return CPA_OK;
+
+    const int threads = std::min(256, std::max(32, (Hkv * chunks_per_head + 31) / 32 * 32));
+    if (!new_lens) {
+        kv_append_step_kernel<<<B, threads, 0, st>>>((const uint4*)k_new, (const uint4*)v_new, (uint4*)k_pool,
+                                                     (uint4*)v_pool, ix, Hkv, chunks_per_head, P);
+    } else {
+        const int32_t* src_indptr = ix.cu_seqlens;
+        if (!is_prefill_bulk) {
+            plan->append_stage[0] = 0;
+            for (int b = 0; b < B; ++b) plan->append_stage[b + 1] = plan->append_stage[b] + new_lens[b];
+            if (cudaMemcpyAsync(ix.append_indptr, plan->append_stage.data(), sizeof(int32_t) * (B + 1),
+                                cudaMemcpyHostToDevice, st) != cudaSuccess) {
+                (void)cudaGetLastError();
+                return CPA_ECUDA;
+            }
+            src_indptr = ix.append_indptr;
+        }
+        const int grid = (int)std::min<int64_t>(rows, 148 * 32);
+        kv_append_bulk_kernel<<<grid, threads, 0, st>>>((const uint4*)k_new, (const uint4*)v_new, (uint4*)k_pool,
+                                                        (uint4*)v_pool, ix, src_indptr, B, rows, Hkv,
+                                                        chunks_per_head, P);
+        seq_lens_advance_kernel<<<(B + 127) / 128, 128, 0, st>>>(ix, src_indptr, B);
+    }
+    if (cudaGetLastError() != cudaSuccess) return CPA_ECUDA;
+    for (int b = 0; b < B; ++b) plan->seq_lens[b] += new_lens ? new_lens[b] : 1;
+    return CPA_OK;
+}

@@ -1,0 +1,231 @@
+// Host planner: partition bookkeeping for one compaction event (Section 4,
+// "Snapshot & partition" and "Dispatch"): block offsets, page table, token slots
+// and the CTA work lists for the prefill and decode kernels.
+#include <cuda_runtime.h>
+
+#include <algorithm>
+#include <cstring>
+#include <new>
+
+#include "cpa_internal.h"
+
+namespace {
+
+int64_t align4(int64_t words) { return (words + 3) / 4 * 4; }  // 16-byte alignment of every array
+
+int64_t decode_item_count(const std::vector<int32_t>& pages_per_block, int32_t hkv, int32_t C) {
+    int64_t n = 0;
+    for (int32_t p : pages_per_block) n += (int64_t)hkv * ((p + C - 1) / C);
+    return n;
+}
+
+}  // namespace
+
+extern "C" int cpa_plan_create(const cpa_config* cfg, int32_t num_blocks, const int32_t* block_lens,
+                               int32_t max_new_tokens, const int32_t* free_pages, int32_t num_free,
+                               cpa_plan** out) {
+    if (out) *out = nullptr;
+    if (!cfg || !block_lens || !out || num_blocks < 1 || max_new_tokens < 0 || num_free < 0 ||
+        (num_free > 0 && !free_pages))
+        return CPA_EINVAL;
+    if (cfg->num_q_heads < 1 || cfg->num_kv_heads < 1 || cfg->num_q_heads % cfg->num_kv_heads != 0 ||
+        cfg->q_tile_rows < 0 || cfg->pages_per_split < 0 || cfg->num_sms < 0 || !(cfg->scale > 0.f))
+        return CPA_EINVAL;
+    if ((cfg->head_dim != 64 && cfg->head_dim != 128) || cfg->page_size != 16 ||
+        cfg->num_q_heads / cfg->num_kv_heads > 8)
+        return CPA_EUNSUPPORTED;
+    if (cfg->q_tile_rows != 0 && cfg->q_tile_rows != 128) return CPA_EUNSUPPORTED;
+
+    cpa_plan* p = new (std::nothrow) cpa_plan();
+    if (!p) return CPA_ENOSPC;
+    p->cfg = *cfg;
+    p->B = num_blocks;
+    p->T = max_new_tokens;
+    p->q_tile = cfg->q_tile_rows ? cfg->q_tile_rows : 128;
+    const int32_t P = cfg->page_size;
+    const int32_t B = num_blocks;
+
+    p->block_lens.assign(block_lens, block_lens + B);
+    p->cu_seqlens.assign(B + 1, 0);
+    p->page_indptr.assign(B + 1, 0);
+    std::vector<int32_t> pages_per_block(B);
+    for (int32_t b = 0; b < B; ++b) {
+        if (block_lens[b] < 1) { delete p; return CPA_EINVAL; }
+        int64_t cu = (int64_t)p->cu_seqlens[b] + block_lens[b];
+        int64_t pages = ((int64_t)block_lens[b] + max_new_tokens + P - 1) / P;
+        int64_t ip = (int64_t)p->page_indptr[b] + pages;
+        if (cu > INT32_MAX / 2 || ip > INT32_MAX / 64) { delete p; return CPA_EUNSUPPORTED; }
+        p->cu_seqlens[b + 1] = (int32_t)cu;
+        p->page_indptr[b + 1] = (int32_t)ip;
+        pages_per_block[b] = (int32_t)pages;
+    }
+    p->total_tokens = p->cu_seqlens[B];
+    const int32_t pages_used = p->page_indptr[B];
+    if (pages_used > num_free) { delete p; return CPA_ENOSPC; }
+    p->page_indices.assign(free_pages, free_pages + pages_used);
+    for (int32_t id : p->page_indices)
+        if (id < 0 || id > INT32_MAX / 64) { delete p; return CPA_EINVAL; }
+    p->seq_lens.assign(B, 0);
+
+    // slot of every prefill token
+    p->slot_mapping.resize((size_t)p->total_tokens);
+    for (int32_t b = 0; b < B; ++b) {
+        const int32_t* pages = p->page_indices.data() + p->page_indptr[b];
+        int32_t* slots = p->slot_mapping.data() + p->cu_seqlens[b];
+        for (int32_t pos = 0; pos < block_lens[b]; ++pos) slots[pos] = pages[pos / P] * P + pos % P;
+    }
+
+    // prefill work list: longest tiles first (later q tiles of a causal block see more keys)
+    struct PItem { int32_t cost, block, tile; };
+    std::vector<PItem> pit;
+    for (int32_t b = 0; b < B; ++b) {
+        int32_t n_tiles = (block_lens[b] + p->q_tile - 1) / p->q_tile;
+        for (int32_t t = 0; t < n_tiles; ++t)
+            pit.push_back({std::min((t + 1) * p->q_tile, block_lens[b]), b, t});
+    }
+    std::stable_sort(pit.begin(), pit.end(), [](const PItem& a, const PItem& c) {
+        if (a.cost != c.cost) return a.cost > c.cost;
+        if (a.block != c.block) return a.block < c.block;
+        return a.tile < c.tile;
+    });
+    p->n_prefill = (int32_t)pit.size();
+    p->prefill_items.reserve(pit.size() * 2);
+    for (const PItem& it : pit) { p->prefill_items.push_back(it.block); p->prefill_items.push_back(it.tile); }
+
+    // pages per decode split: the largest power of two (<= 64) that still yields
+    // about eight work items per SM; never below 4 pages unless asked for
+    if (cfg->pages_per_split > 0) {
+        p->C = cfg->pages_per_split;
+    } else {
+        const int64_t target = 8LL * (cfg->num_sms ? cfg->num_sms : 148);
+        int32_t C = 64;
+        while (C > 4 && decode_item_count(pages_per_block, cfg->num_kv_heads, C) < target) C /= 2;
+        p->C = C;
+    }
+    struct DItem { int32_t pages, block, head, split; };
+    std::vector<DItem> dit;
+    p->split_indptr.assign(B + 1, 0);
+    for (int32_t b = 0; b < B; ++b) {
+        int32_t n_splits = (pages_per_block[b] + p->C - 1) / p->C;
+        p->split_indptr[b + 1] = p->split_indptr[b] + n_splits;
+        for (int32_t g = 0; g < cfg->num_kv_heads; ++g)
+            for (int32_t s = 0; s < n_splits; ++s)
+                dit.push_back({std::min(p->C, pages_per_block[b] - s * p->C), b, g, s});
+    }
+    std::stable_sort(dit.begin(), dit.end(), [](const DItem& a, const DItem& c) {
+        if (a.pages != c.pages) return a.pages > c.pages;
+        if (a.block != c.block) return a.block < c.block;
+        if (a.head != c.head) return a.head < c.head;
+        return a.split < c.split;
+    });
+    p->n_decode = (int32_t)dit.size();
+    p->decode_items.reserve(dit.size() * 3);
+    for (const DItem& it : dit) {
+        p->decode_items.push_back(it.block);
+        p->decode_items.push_back(it.head);
+        p->decode_items.push_back(it.split);
+    }
+
+    // device image
+    int64_t w = 0;
+    p->off_status = w;  w = align4(w + 4);
+    p->off_cu = w;      w = align4(w + B + 1);
+    p->off_pindptr = w; w = align4(w + B + 1);
+    p->off_sindptr = w; w = align4(w + B + 1);
+    p->off_seqlens = w; w = align4(w + B);
+    p->off_append = w;  w = align4(w + B + 1);
+    p->off_pidx = w;    w = align4(w + pages_used);
+    p->off_pitems = w;  w = align4(w + 2LL * p->n_prefill);
+    p->off_ditems = w;  w = align4(w + 4LL * p->n_decode);
+    p->words = w;
+    p->image.assign((size_t)w, 0);
+    int32_t* im = p->image.data();
+    std::memcpy(im + p->off_cu, p->cu_seqlens.data(), sizeof(int32_t) * (B + 1));
+    std::memcpy(im + p->off_pindptr, p->page_indptr.data(), sizeof(int32_t) * (B + 1));
+    std::memcpy(im + p->off_sindptr, p->split_indptr.data(), sizeof(int32_t) * (B + 1));
+    std::memcpy(im + p->off_pidx, p->page_indices.data(), sizeof(int32_t) * pages_used);
+    std::memcpy(im + p->off_pitems, p->prefill_items.data(), sizeof(int32_t) * 2 * p->n_prefill);
+    for (int32_t i = 0; i < p->n_decode; ++i) {
+        im[p->off_ditems + 4 * i + 0] = dit[i].block;
+        im[p->off_ditems + 4 * i + 1] = dit[i].head;
+        im[p->off_ditems + 4 * i + 2] = dit[i].split;
+        im[p->off_ditems + 4 * i + 3] = dit[i].pages;
+    }
+    p->append_stage.assign(B + 1, 0);
+    *out = p;
+    return CPA_OK;
+}
+
+extern "C" int cpa_plan_export(const cpa_plan* plan, int which, const int32_t** ptr, int64_t* count) {
+    if (!plan || !ptr || !count) return CPA_EINVAL;
+    const std::vector<int32_t>* v = nullptr;
+    int64_t div = 1;
+    switch (which) {
+        case CPA_ARR_CU_SEQLENS: v = &plan->cu_seqlens; break;
+        case CPA_ARR_PAGE_INDPTR: v = &plan->page_indptr; break;
+        case CPA_ARR_PAGE_INDICES: v = &plan->page_indices; break;
+        case CPA_ARR_SEQ_LENS: v = &plan->seq_lens; break;
+        case CPA_ARR_SLOT_MAPPING: v = &plan->slot_mapping; break;
+        case CPA_ARR_PREFILL_ITEMS: v = &plan->prefill_items; div = 2; break;
+        case CPA_ARR_DECODE_ITEMS: v = &plan->decode_items; div = 3; break;
+        case CPA_ARR_SPLIT_INDPTR: v = &plan->split_indptr; break;
+        default: return CPA_EINVAL;
+    }
+    *ptr = v->data();
+    *count = (int64_t)v->size() / div;
+    return CPA_OK;
+}
+
+extern "C" int64_t cpa_plan_param(const cpa_plan* plan, int which) {
+    if (!plan) return CPA_EINVAL;
+    switch (which) {
+        case CPA_PARAM_NUM_BLOCKS: return plan->B;
+        case CPA_PARAM_TOTAL_TOKENS: return plan->total_tokens;
+        case CPA_PARAM_Q_TILE_ROWS: return plan->q_tile;
+        case CPA_PARAM_PAGES_PER_SPLIT: return plan->C;
+        case CPA_PARAM_PAGES_USED: return plan->page_indptr[plan->B];
+        case CPA_PARAM_INDEX_BYTES: return plan->index_bytes();
+        case CPA_PARAM_DECODE_WORKSPACE_BYTES: return plan->decode_workspace_bytes();
+        case CPA_PARAM_TOTAL_SPLITS: return plan->split_indptr[plan->B];
+        case CPA_PARAM_MAX_NEW_TOKENS: return plan->T;
+        default: return CPA_EINVAL;
+    }
+}
+
+extern "C" int cpa_plan_upload(cpa_plan* plan, void* d_index_buf, int64_t bytes, void* stream) {
+    if (!plan || !d_index_buf || !cpa_aligned16(d_index_buf)) return CPA_EINVAL;
+    if (bytes < plan->index_bytes()) return CPA_ENOSPC;
+    // the device copy starts from an empty cache, so the host mirror does too
+    std::fill(plan->seq_lens.begin(), plan->seq_lens.end(), 0);
+    cudaError_t e = cudaMemcpyAsync(d_index_buf, plan->image.data(), (size_t)plan->index_bytes(),
+                                    cudaMemcpyHostToDevice, (cudaStream_t)stream);
+    if (e != cudaSuccess) { (void)cudaGetLastError(); return CPA_ECUDA; }
+    plan->d_base = static_cast<int32_t*>(d_index_buf);
+    return CPA_OK;
+}
+
+extern "C" int cpa_plan_status(cpa_plan* plan, void* stream) {
+    if (!plan) return CPA_EINVAL;
+    if (!plan->d_base) return CPA_ESTATE;
+    int32_t word = 0;
+    cudaError_t e = cudaMemcpyAsync(&word, plan->d_base + plan->off_status, sizeof(word),
+                                    cudaMemcpyDeviceToHost, (cudaStream_t)stream);
+    if (e == cudaSuccess) e = cudaStreamSynchronize((cudaStream_t)stream);
+    if (e != cudaSuccess) { (void)cudaGetLastError(); return CPA_ECUDA; }
+    return word == 0 ? CPA_OK : CPA_ETIMEOUT;
+}
+
+extern "C" void cpa_plan_destroy(cpa_plan* plan) { delete plan; }
+
+extern "C" const char* cpa_strerror(int status) {
+    switch (status) {
+        case CPA_OK: return "ok";
+        case CPA_EINVAL: return "invalid argument";
+        case CPA_ENOSPC: return "not enough pages or buffer space";
+        case CPA_EUNSUPPORTED: return "unsupported configuration";
+        case CPA_ECUDA: return "CUDA call failed";
+        case CPA_ETIMEOUT: return "a bounded device-side wait gave up";
+        case CPA_ESTATE: return "call order violated";
+        default: return "unknown status";
+    }
+}

@@ -1,0 +1,119 @@
+"""Device-buffer bookkeeping around the C-ABI calls for one compaction event.
+
+PyTorch is used for device memory and streams only; every step of the path
+(planning, prefill, append, decode, merge) runs inside libcompact_attn.
+"""
+from __future__ import annotations
+
+from typing import Optional, Sequence
+
+import numpy as np
+import torch
+
+from . import binding as B
+
+
+def bits_to_tensor(bits: np.ndarray, device=None, pin: bool = False) -> torch.Tensor:
+    """uint16 bf16 bit patterns -> torch.bfloat16 tensor (same bits)."""
+    t = torch.from_numpy(np.ascontiguousarray(bits).view(np.int16)).view(torch.bfloat16)
+    if pin:
+        t = t.pin_memory()
+    return t.to(device, non_blocking=pin) if device is not None else t
+
+
+def tensor_to_bits(t: torch.Tensor) -> np.ndarray:
+    """torch.bfloat16 tensor -> uint16 bit patterns on the host."""
+    return t.detach().contiguous().view(torch.int16).cpu().numpy().view(np.uint16)
+
+
+class CompactionSession:
+    """One history cut into blocks, one summary sequence per block (paper, Section 4).
+
+    Owns the plan handle, the device index buffer, the K/V page pools and the
+    decode workspace.  All calls are enqueued on the current torch stream of
+    `device` unless a stream is given.
+    """
+
+    def __init__(self, block_lens: Sequence[int], max_new_tokens: int, num_q_heads: int,
+                 num_kv_heads: int, head_dim: int, free_pages: Sequence[int], num_pages: int,
+                 scale: Optional[float] = None, device: str = "cuda:0", pages_per_split: int = 0,
+                 poison_pools: bool = False, page_size: int = 16):
+        self.device = torch.device(device)
+        self.Hq, self.Hkv, self.d, self.P = num_q_heads, num_kv_heads, head_dim, page_size
+        self.B = len(block_lens)
+        self.block_lens = np.asarray(block_lens, dtype=np.int32)
+        self.scale = float(scale if scale is not None else head_dim ** -0.5)
+        props = torch.cuda.get_device_properties(self.device)
+        self.cfg = B.cpa_config(num_q_heads, num_kv_heads, head_dim, page_size, self.scale, 0,
+                                pages_per_split, props.multi_processor_count)
+        self.plan = B.cpa_plan_create(self.cfg, self.block_lens, max_new_tokens, free_pages)
+        self.total_tokens = B.cpa_plan_param(self.plan, B.PARAM_TOTAL_TOKENS)
+        nbytes = B.cpa_plan_param(self.plan, B.PARAM_INDEX_BYTES)
+        self.index_buf = torch.empty(nbytes, dtype=torch.uint8, device=self.device)
+        pool_shape = (num_pages, num_kv_heads, page_size, head_dim)
+        if poison_pools:   # unused slots hold NaN: the kernels must mask by index, not by value
+            self.k_pool = torch.full(pool_shape, float("nan"), dtype=torch.bfloat16, device=self.device)
+            self.v_pool = torch.full(pool_shape, float("nan"), dtype=torch.bfloat16, device=self.device)
+        else:  # no initialisation needed: slots are masked by index until they are written
+            self.k_pool = torch.empty(pool_shape, dtype=torch.bfloat16, device=self.device)
+            self.v_pool = torch.empty(pool_shape, dtype=torch.bfloat16, device=self.device)
+        ws = B.cpa_plan_param(self.plan, B.PARAM_DECODE_WORKSPACE_BYTES)
+        self.workspace = torch.empty(max(ws, 256), dtype=torch.uint8, device=self.device)
+        self._check(B.cpa_plan_upload(self.plan, self.index_buf, nbytes, self._stream()), "cpa_plan_upload")
+
+    # -- helpers ------------------------------------------------------------
+    def _stream(self) -> int:
+        return int(torch.cuda.current_stream(self.device).cuda_stream)
+
+    @staticmethod
+    def _check(rc: int, where: str) -> None:
+        if rc != B.CPA_OK:
+            raise B.CpaError(rc, where)
+
+    def export(self, which: int) -> np.ndarray:
+        return B.cpa_plan_export(self.plan, which)
+
+    def param(self, which: int) -> int:
+        return B.cpa_plan_param(self.plan, which)
+
+    # -- the hot path -------------------------------------------------------
+    def prefill(self, q: torch.Tensor, k: torch.Tensor, v: torch.Tensor,
+                out: Optional[torch.Tensor] = None) -> torch.Tensor:
+        """Causal attention of every block over itself; q/out [tokens,Hq,d], k/v [tokens,Hkv,d]."""
+        if out is None:
+            out = torch.empty_like(q)
+        self._check(B.cpa_prefill(self.plan, q, k, v, out, None, self._stream()), "cpa_prefill")
+        return out
+
+    def append_prefill(self, k: torch.Tensor, v: torch.Tensor) -> None:
+        """Store the prefill K/V of every block in its pages."""
+        self._check(B.cpa_kv_append(self.plan, k, v, self.block_lens, self.k_pool, self.v_pool,
+                                    self._stream()), "cpa_kv_append")
+
+    def append(self, k_new: torch.Tensor, v_new: torch.Tensor, new_lens=None) -> None:
+        """One token per block (new_lens None) or new_lens[b] tokens per block."""
+        self._check(B.cpa_kv_append(self.plan, k_new, v_new, new_lens, self.k_pool, self.v_pool,
+                                    self._stream()), "cpa_kv_append")
+
+    def decode(self, q: torch.Tensor, out: Optional[torch.Tensor] = None) -> torch.Tensor:
+        """q/out [B,Hq,d]: newest token of every block over that block's cache."""
+        if out is None:
+            out = torch.empty_like(q)
+        self._check(B.cpa_decode(self.plan, q, self.k_pool, self.v_pool, out, self.workspace,
+                                 self._stream()), "cpa_decode")
+        return out
+
+    def status(self) -> int:
+        return B.cpa_plan_status(self.plan, self._stream())
+
+    def close(self) -> None:
+        if self.plan:
+            torch.cuda.synchronize(self.device)
+            B.cpa_plan_destroy(self.plan)
+            self.plan = None
+
+    def __del__(self):  # pragma: no cover
+        try:
+            self.close()
+        except Exception:
+            pass

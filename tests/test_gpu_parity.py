@@ -1,0 +1,301 @@
+"""Parity of the CUDA path (through the C-ABI) with the CPU oracle on the same
+seeded inputs: indices and pool bytes bit-exact, attention within max-abs 1e-2 /
+mean-abs 1e-3 of the unrounded fp64 result."""
+import numpy as np
+import pytest
+
+from _util import assert_attention_close
+from oracle import attention as oa
+from oracle import plan as op
+from paper_2605_23296_b200 import workloads as wl
+
+pytestmark = pytest.mark.gpu
+
+
+def _session(w, poison=False, pages_per_split=0):
+    from paper_2605_23296_b200.session import CompactionSession
+    return CompactionSession(w.block_lens, w.decode_steps, w.num_q_heads, w.num_kv_heads,
+                             w.head_dim, w.free_pages, w.num_pages, scale=w.scale,
+                             poison_pools=poison, pages_per_split=pages_per_split)
+
+
+def _dev(bits):
+    from paper_2605_23296_b200.session import bits_to_tensor
+    return bits_to_tensor(bits, "cuda:0")
+
+
+def _bits(t):
+    from paper_2605_23296_b200.session import tensor_to_bits
+    return tensor_to_bits(t)
+
+
+def _cu(w):
+    return np.concatenate([[0], np.cumsum(w.block_lens.astype(np.int64))])
+
+
+def sample_rows(w, per_block=16, seed=0, tile=128):
+    """First/last rows, rows around tile boundaries, and random rows of every block."""
+    rng = np.random.default_rng(seed)
+    cu = _cu(w)
+    rows = []
+    for b, L in enumerate(int(x) for x in w.block_lens):
+        cand = {0, 1, L - 2, L - 1}
+        for t in (tile, 2 * tile, (L // tile) * tile, (L // 2 // tile) * tile):
+            cand |= {t - 1, t, t + 1}
+        cand |= set(int(x) for x in rng.integers(0, L, per_block))
+        if w.outlier_pos is not None:
+            cand |= {int(w.outlier_pos[b]), int(w.outlier_pos[b]) + 1}
+        rows += [cu[b] + r for r in sorted(cand) if 0 <= r < L]
+    return np.asarray(rows, dtype=np.int64)
+
+
+# ----------------------------------------------------------------------------
+# append: bit-exact pool contents
+# ----------------------------------------------------------------------------
+
+@pytest.mark.parametrize("make", [lambda: wl.tiny(5), lambda: wl.custom([1, 15, 16, 17, 300], 8, 2, 128, 6)])
+def test_append_bit_exact(make):
+    import torch
+    w = make().materialise()
+    s = _session(w, poison=True)
+    k, v = _dev(w.k), _dev(w.v)
+    s.append_prefill(k, v)
+    T = w.decode_steps
+    for t in range(T):
+        s.append(_dev(w.k_dec[t]), _dev(w.v_dec[t]))
+    assert s.status() == 0
+    # expected contents from the oracle's own slot arithmetic
+    plan = op.build_plan(w.block_lens.tolist(), T, w.page_size, w.free_pages.tolist(),
+                         w.num_kv_heads, 128, 1)
+    slots = list(plan["slot_mapping"])
+    ks, vs = [w.k], [w.v]
+    for t in range(T):
+        for b in range(w.num_blocks):
+            slots.append(op.slot_of(plan, w.page_size, b, int(w.block_lens[b]) + t))
+        ks.append(w.k_dec[t])
+        vs.append(w.v_dec[t])
+    kp, vp, written = oa.expected_pool(slots, np.concatenate(ks), np.concatenate(vs), w.num_pages, w.page_size)
+    got_k, got_v = _bits(s.k_pool), _bits(s.v_pool)
+    mask = np.broadcast_to(written[:, None, :, None], got_k.shape)
+    assert np.array_equal(got_k[mask], kp[mask]) and np.array_equal(got_v[mask], vp[mask])
+    # slots nobody owns still hold the poison pattern
+    nan_bits = _bits(torch.full((1,), float("nan"), dtype=torch.bfloat16))[0]
+    assert (got_k[~mask] == nan_bits).all() and (got_v[~mask] == nan_bits).all()
+    assert np.array_equal(s.export(3), w.block_lens + T)       # host mirror of seq_lens
+    s.close()
+
+
+def test_append_general_lengths_and_capacity_error():
+    from paper_2605_23296_b200 import binding as B
+    w = wl.custom([40, 7, 100], 4, 2, 64, steps=20, seed=3).materialise()
+    s = _session(w)
+    k, v = _dev(w.k), _dev(w.v)
+    # two uneven bulk appends instead of one: 3 rows of every block first, then the rest
+    cu = _cu(w)
+    first = np.array([3, 3, 3], dtype=np.int32)
+    idx1 = np.concatenate([np.arange(cu[b], cu[b] + 3) for b in range(3)])
+    idx2 = np.concatenate([np.arange(cu[b] + 3, cu[b + 1]) for b in range(3)])
+    s.append(_dev(w.k[idx1]), _dev(w.v[idx1]), first)
+    s.append(_dev(w.k[idx2]), _dev(w.v[idx2]), w.block_lens - 3)
+    assert s.status() == 0
+    plan = op.build_plan(w.block_lens.tolist(), 20, 16, w.free_pages.tolist(), 2, 128, 1)
+    kp, vp, written = oa.expected_pool(plan["slot_mapping"], w.k, w.v, w.num_pages, 16)
+    mask = np.broadcast_to(written[:, None, :, None], kp.shape)
+    assert np.array_equal(_bits(s.k_pool)[mask], kp[mask])
+    assert np.array_equal(_bits(s.v_pool)[mask], vp[mask])
+    # growing a block past L_b + T is refused on the host, nothing is launched
+    too_many = np.array([21, 0, 0], dtype=np.int32)
+    junk = _dev(w.k[:21])
+    assert B.cpa_kv_append(s.plan, junk, junk, too_many, s.k_pool, s.v_pool) == B.CPA_ENOSPC
+    assert np.array_equal(s.export(3), w.block_lens)
+    s.close()
+
+
+# ----------------------------------------------------------------------------
+# prefill
+# ----------------------------------------------------------------------------
+
+def _check_prefill(w, rows=None, what=""):
+    w.materialise()
+    s = _session(w)
+    o = s.prefill(_dev(w.q), _dev(w.k), _dev(w.v))
+    assert s.status() == 0
+    got = _bits(o)
+    want = oa.prefill(w.q, w.k, w.v, _cu(w), w.scale, rows=rows)
+    assert_attention_close(got if rows is None else got[rows], want, what)
+    s.close()
+    return got
+
+
+def test_prefill_tiny_config():
+    _check_prefill(wl.tiny(0), what="tiny")
+
+
+@pytest.mark.parametrize("hq,hkv,d", [(4, 4, 64), (8, 2, 64), (8, 1, 128), (6, 2, 128), (8, 8, 128)])
+def test_prefill_edge_lengths(hq, hkv, d):
+    lens = [1, 2, 63, 64, 65, 127, 128, 129, 191, 192, 193, 255, 256, 257, 500, 16, 1]
+    _check_prefill(wl.custom(lens, hq, hkv, d, steps=0, seed=hq * 100 + d), what=f"edge {hq}/{hkv}/{d}")
+
+
+def test_prefill_single_block_is_sequential_compaction():
+    # B = 1: the whole history in one block (Eq. 1 of the paper)
+    _check_prefill(wl.custom([1500], 8, 2, 128, steps=0, seed=9), what="B=1")
+
+
+def test_prefill_does_not_write_outside_its_rows():
+    import torch
+    w = wl.custom([130, 3, 129], 4, 2, 64, steps=0, seed=4).materialise()
+    s = _session(w)
+    q = _dev(w.q)
+    guard = torch.full((w.total_tokens + 64, 4, 64), 7.0, dtype=torch.bfloat16, device="cuda:0")
+    out = guard[32:32 + w.total_tokens]
+    s.prefill(q, _dev(w.k), _dev(w.v), out=out)
+    assert s.status() == 0
+    assert (guard[:32] == 7.0).all() and (guard[32 + w.total_tokens:] == 7.0).all()
+    assert_attention_close(_bits(out), oa.prefill(w.q, w.k, w.v, _cu(w), w.scale), "guarded")
+    s.close()
+
+
+def test_prefill_outlier_keys():
+    w = wl.dense8b(seed=21, num_blocks=3, block_len=700, steps=0)
+    _check_prefill(w, what="outlier")
+
+
+# ----------------------------------------------------------------------------
+# decode
+# ----------------------------------------------------------------------------
+
+def _check_decode(w, steps=None, poison=True, pages_per_split=0, check_steps=None, what=""):
+    w.materialise()
+    T = w.decode_steps if steps is None else steps
+    s = _session(w, poison=poison, pages_per_split=pages_per_split)
+    s.append_prefill(_dev(w.k), _dev(w.v))
+    st = oa.DecodeState(w.k, w.v, _cu(w), w.decode_steps)
+    kd, vd, qd = _dev(w.k_dec), _dev(w.v_dec), _dev(w.q_dec)
+    outs = []
+    for t in range(T):
+        s.append(kd[t], vd[t])
+        outs.append(s.decode(qd[t]))
+    assert s.status() == 0
+    for t in range(T):
+        st.append(w.k_dec[t], w.v_dec[t])
+        if check_steps is not None and t not in check_steps:
+            continue
+        assert_attention_close(_bits(outs[t]), st.decode(w.q_dec[t], w.scale), f"{what} step {t}")
+    s.close()
+
+
+def test_decode_tiny_config_all_steps():
+    _check_decode(wl.tiny(0), what="tiny")
+
+
+@pytest.mark.parametrize("pps", [1, 2, 5])
+def test_decode_tiny_any_split_size(pps):
+    _check_decode(wl.tiny(1), pages_per_split=pps, what=f"tiny pps={pps}")
+
+
+@pytest.mark.parametrize("hq,hkv,d", [(4, 4, 64), (8, 1, 64), (8, 2, 128), (16, 2, 128), (3, 3, 128)])
+def test_decode_edge_lengths_cross_page_boundaries(hq, hkv, d):
+    # lengths right before / at / after page boundaries; 20 steps cross at least one more
+    lens = [1, 14, 15, 16, 17, 31, 32, 33, 255, 256, 257, 1000]
+    _check_decode(wl.custom(lens, hq, hkv, d, steps=20, seed=hq + d), what=f"edge {hq}/{hkv}/{d}")
+
+
+def test_decode_step_equals_prefill_last_row_on_gpu():
+    # the same identity the oracle is pinned with, now across the two CUDA kernels
+    w = wl.custom([200, 77], 8, 2, 128, steps=1, seed=12).materialise()
+    s = _session(w)
+    s.append_prefill(_dev(w.k), _dev(w.v))
+    s.append(_dev(w.k_dec[0]), _dev(w.v_dec[0]))
+    dec = _bits(s.decode(_dev(w.q_dec[0])))
+    s.close()
+    cu = _cu(w)
+    ext = wl.custom([201, 78], 8, 2, 128, steps=0, seed=12)
+    ext.q = np.concatenate([w.q[:200], w.q_dec[0, :1], w.q[200:], w.q_dec[0, 1:]])
+    ext.k = np.concatenate([w.k[:200], w.k_dec[0, :1], w.k[200:], w.k_dec[0, 1:]])
+    ext.v = np.concatenate([w.v[:200], w.v_dec[0, :1], w.v[200:], w.v_dec[0, 1:]])
+    ext.free_pages = np.arange(ext.num_pages, dtype=np.int32)
+    s2 = _session(ext)
+    pre = _bits(s2.prefill(_dev(ext.q), _dev(ext.k), _dev(ext.v)))
+    s2.close()
+    from _util import bits_to_f64
+    a = bits_to_f64(dec)
+    b = bits_to_f64(pre[[200, 278]])
+    assert np.abs(a - b).max() <= 2e-2
+
+
+def test_decode_independent_of_page_permutation():
+    w1 = wl.custom([300, 45, 129], 8, 2, 128, steps=4, seed=31, permute_pages=False).materialise()
+    w2 = wl.custom([300, 45, 129], 8, 2, 128, steps=4, seed=31, permute_pages=True).materialise()
+    # same tensors (the permutation draw shifts the stream), so copy them over
+    for name in ("q", "k", "v", "q_dec", "k_dec", "v_dec"):
+        setattr(w2, name, getattr(w1, name))
+    outs = []
+    for w in (w1, w2):
+        s = _session(w, poison=True)
+        s.append_prefill(_dev(w.k), _dev(w.v))
+        res = []
+        for t in range(4):
+            s.append(_dev(w.k_dec[t]), _dev(w.v_dec[t]))
+            res.append(_bits(s.decode(_dev(w.q_dec[t]))))
+        outs.append(np.stack(res))
+        s.close()
+    assert np.array_equal(outs[0], outs[1])
+
+
+# ----------------------------------------------------------------------------
+# full-size configurations, sampled rows / steps
+# ----------------------------------------------------------------------------
+
+def _full_config(w, decode_checks, per_block=12):
+    w.materialise()
+    rows = sample_rows(w, per_block=per_block, seed=w.seed)
+    s = _session(w)
+    q, k, v = _dev(w.q), _dev(w.k), _dev(w.v)
+    o = s.prefill(q, k, v)
+    assert s.status() == 0
+    import torch
+    got = _bits(o[torch.from_numpy(rows).to("cuda:0")])
+    want = oa.prefill(w.q, w.k, w.v, _cu(w), w.scale, rows=rows)
+    assert_attention_close(got, want, f"{w.name} prefill")
+    del q, o
+    # decode: run every step on the GPU, check selected steps on a few blocks
+    s.append_prefill(k, v)
+    del k, v
+    kd, vd, qd = _dev(w.k_dec), _dev(w.v_dec), _dev(w.q_dec)
+    keep = {}
+    for t in range(w.decode_steps):
+        s.append(kd[t], vd[t])
+        out = s.decode(qd[t])
+        if t in decode_checks:
+            keep[t] = _bits(out)
+    assert s.status() == 0
+    s.close()
+    blocks = sorted({0, w.num_blocks - 1, int(np.argmax(w.block_lens)), int(np.argmin(w.block_lens))})
+    st = oa.DecodeState(w.k, w.v, _cu(w), w.decode_steps)
+    for t in range(max(decode_checks) + 1):
+        st.append(w.k_dec[t], w.v_dec[t])
+        if t in keep:
+            want = st.decode(w.q_dec[t], w.scale, blocks=blocks)
+            assert_attention_close(keep[t][blocks], want[blocks], f"{w.name} decode step {t}")
+
+
+def test_full_dense8b():
+    w = wl.dense8b()
+    _full_config(w, {0, 1, 15, 16, 17, 100, w.decode_steps - 1})
+
+
+def test_full_ragged():
+    w = wl.ragged()
+    _full_config(w, {0, 1, 15, 16, 17, 300, w.decode_steps - 1}, per_block=6)
+
+
+def test_full_moe120b():
+    w = wl.moe120b()
+    _full_config(w, {0, 1, 15, 16, 17, 300, w.decode_steps - 1}, per_block=6)
+
+
+@pytest.mark.parametrize("nb", [1, 64])
+def test_full_split_sweep_ends(nb):
+    w = wl.split_sweep(nb, steps=32)
+    _full_config(w, {0, 1, 15, 16, 17, 31}, per_block=4 if nb == 1 else 1)

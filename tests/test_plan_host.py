@@ -1,0 +1,149 @@
+"""Host-side checks that need no GPU: the planner against the independent Python
+restatement (bit-exact), error codes, and the exported C symbols."""
+import os
+import re
+
+import numpy as np
+import pytest
+
+from oracle import plan as op
+from paper_2605_23296_b200 import binding as B
+from paper_2605_23296_b200 import workloads as wl
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def make_plan(w, pages_per_split=0, free=None, num_sms=0):
+    cfg = B.cpa_config(w.num_q_heads, w.num_kv_heads, w.head_dim, w.page_size, w.scale, 0,
+                       pages_per_split, num_sms)
+    if free is None:
+        free = np.arange(w.num_pages, dtype=np.int32)
+    return B.cpa_plan_create(cfg, w.block_lens, w.decode_steps, free), free
+
+
+def check_against_oracle(w, pages_per_split=0, permute=False):
+    free = None
+    if permute:
+        free = np.random.default_rng(w.seed).permutation(w.num_pages).astype(np.int32)
+    plan, free = make_plan(w, pages_per_split, free)
+    try:
+        C = B.cpa_plan_param(plan, B.PARAM_PAGES_PER_SPLIT)
+        M = B.cpa_plan_param(plan, B.PARAM_Q_TILE_ROWS)
+        ref = op.build_plan(w.block_lens.tolist(), w.decode_steps, w.page_size, free.tolist(),
+                            w.num_kv_heads, M, C)
+        pairs = [(B.ARR_CU_SEQLENS, "cu_seqlens"), (B.ARR_PAGE_INDPTR, "page_indptr"),
+                 (B.ARR_PAGE_INDICES, "page_indices"), (B.ARR_SEQ_LENS, "seq_lens"),
+                 (B.ARR_SLOT_MAPPING, "slot_mapping"), (B.ARR_PREFILL_ITEMS, "prefill_items"),
+                 (B.ARR_DECODE_ITEMS, "decode_items"), (B.ARR_SPLIT_INDPTR, "split_indptr")]
+        for which, key in pairs:
+            got = B.cpa_plan_export(plan, which)
+            want = np.asarray(ref[key], dtype=np.int32).reshape(got.shape)
+            assert np.array_equal(got, want), key
+        assert B.cpa_plan_param(plan, B.PARAM_NUM_BLOCKS) == w.num_blocks
+        assert B.cpa_plan_param(plan, B.PARAM_TOTAL_TOKENS) == w.total_tokens
+        assert B.cpa_plan_param(plan, B.PARAM_PAGES_USED) == w.pages_needed
+        assert B.cpa_plan_param(plan, B.PARAM_TOTAL_SPLITS) == ref["split_indptr"][-1]
+        assert B.cpa_plan_param(plan, B.PARAM_MAX_NEW_TOKENS) == w.decode_steps
+        rows = ref["split_indptr"][-1] * w.num_q_heads
+        assert B.cpa_plan_param(plan, B.PARAM_DECODE_WORKSPACE_BYTES) >= rows * (w.head_dim + 2) * 4
+        return C
+    finally:
+        B.cpa_plan_destroy(plan)
+
+
+@pytest.mark.parametrize("pps", [0, 1, 3, 8])
+def test_plan_bit_exact_tiny(pps):
+    check_against_oracle(wl.tiny(), pps, permute=True)
+
+
+def test_plan_bit_exact_edge_lengths():
+    w = wl.custom([1, 15, 16, 17, 127, 128, 129, 1000], 8, 2, 64, steps=5)
+    check_against_oracle(w, 0, permute=True)
+    w = wl.custom([4097], 4, 4, 128, steps=0)
+    check_against_oracle(w, 2)
+
+
+@pytest.mark.parametrize("name", ["dense8b", "ragged", "moe120b"])
+def test_plan_bit_exact_full_configs(name):
+    w = wl.CONFIGS[name]()
+    C = check_against_oracle(w, 0, permute=(name == "ragged"))
+    assert C in (4, 8, 16, 32, 64)
+
+
+@pytest.mark.parametrize("nb", [1, 2, 8, 64])
+def test_plan_bit_exact_split_sweep(nb):
+    check_against_oracle(wl.split_sweep(nb), 0)
+
+
+def test_auto_split_aims_at_the_sm_count():
+    w = wl.dense8b()
+    plan_a, _ = make_plan(w, 0, num_sms=148)
+    plan_b, _ = make_plan(w, 0, num_sms=16)
+    try:
+        ca = B.cpa_plan_param(plan_a, B.PARAM_PAGES_PER_SPLIT)
+        cb = B.cpa_plan_param(plan_b, B.PARAM_PAGES_PER_SPLIT)
+        assert cb >= ca
+        items = B.cpa_plan_export(plan_a, B.ARR_DECODE_ITEMS).shape[0]
+        assert items >= 8 * 148 or ca == 4
+    finally:
+        B.cpa_plan_destroy(plan_a)
+        B.cpa_plan_destroy(plan_b)
+
+
+def test_plan_errors():
+    ok = B.cpa_config(8, 2, 64, 16, 0.125, 0, 0, 0)
+    free = np.arange(100, dtype=np.int32)
+
+    def rc(cfg=ok, lens=(40, 50), T=4, fr=free):
+        status, handle = B.cpa_plan_create(cfg, lens, T, fr, check=False)
+        assert status != 0 and not handle
+        return status
+
+    assert rc(lens=(40, 0)) == B.CPA_EINVAL                      # zero-length block
+    assert rc(lens=(40, -3)) == B.CPA_EINVAL
+    assert rc(T=-1) == B.CPA_EINVAL
+    assert rc(fr=np.arange(5, dtype=np.int32)) == B.CPA_ENOSPC   # too few pages
+    assert rc(fr=np.array([0, 1, 2, -4, 5, 6, 7, 8], dtype=np.int32)) == B.CPA_EINVAL
+    assert rc(cfg=B.cpa_config(8, 3, 64, 16, 0.125, 0, 0, 0)) == B.CPA_EINVAL        # 8 % 3
+    assert rc(cfg=B.cpa_config(8, 2, 96, 16, 0.125, 0, 0, 0)) == B.CPA_EUNSUPPORTED  # head_dim
+    assert rc(cfg=B.cpa_config(8, 2, 64, 32, 0.125, 0, 0, 0)) == B.CPA_EUNSUPPORTED  # page size
+    assert rc(cfg=B.cpa_config(16, 1, 64, 16, 0.125, 0, 0, 0)) == B.CPA_EUNSUPPORTED # G = 16
+    assert rc(cfg=B.cpa_config(8, 2, 64, 16, 0.0, 0, 0, 0)) == B.CPA_EINVAL          # scale
+    with pytest.raises(B.CpaError):
+        B.cpa_plan_create(ok, (40, 0), 4, free)
+    # T = 0 is allowed (prefill only)
+    plan = B.cpa_plan_create(ok, (40, 50), 0, free)
+    B.cpa_plan_destroy(plan)
+
+
+def test_compute_calls_before_upload_report_state_error():
+    plan = B.cpa_plan_create(B.cpa_config(8, 2, 64, 16, 0.125, 0, 0, 0), (40, 50), 4,
+                             np.arange(100, dtype=np.int32))
+    try:
+        fake = 4096  # a 16-byte aligned non-null address; never dereferenced before the state check
+        assert B.cpa_prefill(plan, fake, fake, fake, fake + 16) == B.CPA_ESTATE
+        assert B.cpa_kv_append(plan, fake, fake, None, fake, fake) == B.CPA_ESTATE
+        assert B.cpa_decode(plan, fake, fake, fake, fake, fake) == B.CPA_ESTATE
+        assert B.cpa_plan_status(plan) == B.CPA_ESTATE
+        assert B.cpa_prefill(plan, None, fake, fake, fake) == B.CPA_EINVAL
+        assert B.cpa_prefill(plan, fake + 2, fake, fake, fake + 16) == B.CPA_EINVAL   # misaligned
+        assert B.cpa_decode(plan, fake, fake, fake, fake, None) == B.CPA_EINVAL
+    finally:
+        B.cpa_plan_destroy(plan)
+    for code in range(0, -7, -1):
+        assert B.cpa_strerror(code) and B.cpa_strerror(code) != "unknown status"
+    assert B.cpa_strerror(-99) == "unknown status"
+
+
+def test_library_exports_every_declared_symbol():
+    import ctypes
+    names = set()
+    inc = os.path.join(ROOT, "include")
+    for fn in os.listdir(inc):
+        if fn.endswith(".h"):
+            text = open(os.path.join(inc, fn)).read()
+            names |= set(re.findall(r"CPA_API\s+[\w\s\*]*?\b(cpa_\w+)\s*\(", text))
+    assert {"cpa_plan_create", "cpa_prefill", "cpa_kv_append", "cpa_decode"} <= names
+    lib = ctypes.CDLL(B.LIB_PATH)
+    for n in sorted(names):
+        assert hasattr(lib, n), n
