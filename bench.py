@@ -41,10 +41,13 @@ def load_peaks():
         return dict(FALLBACK_PEAKS), "fallback"
 
 
-def make_workload(name: str, seed_offset: int = 0):
-    w = wl.CONFIGS[name]()
+def make_workload(name: str, seed_offset: int = 0, overrides=None):
+    """The named configuration; `overrides` (blocks / block length / decode steps) shrink it for
+    profiler captures, which must stay small."""
+    kw = {k: v for k, v in (overrides or {}).items() if v}
+    w = wl.CONFIGS[name](**kw)
     if seed_offset:
-        w = wl.CONFIGS[name](seed=w.seed + 1000 * seed_offset)
+        w = wl.CONFIGS[name](seed=w.seed + 1000 * seed_offset, **kw)
     return w
 
 
@@ -114,7 +117,7 @@ def run_reference(args) -> None:
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
-    w = make_workload(args.config).materialise()
+    w = make_workload(args.config, overrides=args.overrides).materialise()
     tokens = w.num_blocks * w.decode_steps
     times, info = [], None
     for i in range(args.warmup + args.steps):
@@ -154,7 +157,7 @@ class ClockSampler:
             os.close(fd)
             self.proc = subprocess.Popen(
                 ["nvidia-smi", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits",
-                 "-i", str(self.gpu_index), "-lms", "100"],
+                 "-i", str(self.gpu_index), "-lms", "50"],
                 stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
         except Exception:
             self.proc = None
@@ -212,7 +215,7 @@ def run_gpu(args) -> None:
     peaks, peak_kind = load_peaks()
     # weak scaling: every rank runs its own compaction event of the same shape (own seed);
     # blocks are independent, so there is no data-path collective
-    w = make_workload(args.config, seed_offset=rank).materialise()
+    w = make_workload(args.config, seed_offset=rank, overrides=args.overrides).materialise()
     T, Bn = w.decode_steps, w.num_blocks
     stream = torch.cuda.current_stream(dev)
 
@@ -304,7 +307,7 @@ def run_gpu(args) -> None:
     e2e_ms = []
     h2d = sum(t.numel() * 2 for t in (h_q, h_k, h_v, h_qd, h_kd, h_vd))
     d2h = (h_o.numel() + h_od.numel()) * 2
-    for i in range(1 + args.steps):
+    for i in range(0 if args.skip_e2e else 1 + args.steps):
         flush.fill_(1)
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         torch.cuda.synchronize(dev)
@@ -329,7 +332,7 @@ def run_gpu(args) -> None:
         return float(t.item())
 
     ms = max_over_ranks(statistics.mean(step_ms))
-    e2e = max_over_ranks(statistics.mean(e2e_ms))
+    e2e = max_over_ranks(statistics.mean(e2e_ms)) if e2e_ms else float("nan")
     if rank != 0:
         if world > 1:
             dist.destroy_process_group()
@@ -351,7 +354,10 @@ def run_gpu(args) -> None:
                 "launch_us": samp_ms * 1e3, "bytes_per_launch": samp_bytes,
                 "launches_sampled": len(dec_samples), "traffic": None}
 
-    cpu = oracle_sample_seconds(w, rows_per_block=32, decode_samples=8)
+    if args.skip_cpu:
+        cpu = {"estimated_step_s": float("nan"), "cores": 0, "sample": "skipped", "measured_s": 0.0}
+    else:
+        cpu = oracle_sample_seconds(w, rows_per_block=32, decode_samples=8)
     out = {
         "metric": METRIC, "value": tokens / (ms * 1e-3), "unit": UNIT, "n_gpus": world,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
@@ -382,11 +388,19 @@ def run_gpu(args) -> None:
 def main() -> None:
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", default="dense8b", choices=sorted(wl.CONFIGS))
+    ap.add_argument("--blocks", type=int, default=0, help="override the number of blocks (profiling)")
+    ap.add_argument("--block-len", type=int, default=0, help="override the block length (profiling)")
+    ap.add_argument("--decode-steps", type=int, default=0, help="override the decode steps (profiling)")
+    ap.add_argument("--skip-e2e", action="store_true", help="skip the host-buffer leg (profiling)")
+    ap.add_argument("--skip-cpu", action="store_true", help="skip the CPU oracle leg (profiling)")
     args = ap.parse_args()
+    args.overrides = {"num_blocks": args.blocks, "block_len": args.block_len, "steps": args.decode_steps}
+    if args.config == "ragged" and args.block_len:
+        ap.error("--block-len does not apply to the ragged configuration")
     if args.impl == "reference":
         run_reference(args)
     else:
