@@ -183,6 +183,35 @@ CPA_API int cpa_kv_append(cpa_plan* plan, const void* k_new, const void* v_new, 
 CPA_API int cpa_decode(const cpa_plan* plan, const void* q, const void* k_pool, const void* v_pool,
                void* o, void* d_workspace, void* stream);
 
+/*
+ * cpa_decode_static -- cpa_decode for callers that cannot hand over scratch memory.
+ * (The paper has no counterpart; this is a packaging variant of cpa_decode.)
+ *
+ * Some hosts of this library may not allocate device memory where they decode:
+ * a plugin that only gets fixed buffers from the framework around it, a service
+ * whose device memory is budgeted in full at start-up, or a latency-critical
+ * loop that cannot afford the device-wide synchronisation cudaMalloc and
+ * cudaFree imply.  For them the split partials go to a fixed 16 MiB array
+ * (CPA_STATIC_SCRATCH_BYTES) that is part of the library image on the device;
+ * every GPU that loads the library keeps those 16 MiB until the process exits.
+ * The call allocates and frees nothing.
+ *
+ * Arguments, layouts, results and errors are those of cpa_decode without
+ * d_workspace, plus: CPA_ENOSPC when the plan needs more scratch than the array
+ * holds (CPA_PARAM_DECODE_WORKSPACE_BYTES > CPA_STATIC_SCRATCH_BYTES); nothing is
+ * launched then.  Use a smaller batch or larger pages_per_split, or cpa_decode.
+ *
+ * The first call on each device looks up the array's device address (with that
+ * device current); make that first call outside any stream capture.  All calls
+ * on a device share the one array and it keeps the previous call's contents;
+ * the kernels overwrite every element they later read, so nothing needs
+ * clearing, but two calls whose device work overlaps (different streams,
+ * different plans) race on it: serialise them.
+ */
+#define CPA_STATIC_SCRATCH_BYTES (16ll << 20)
+CPA_API int cpa_decode_static(const cpa_plan* plan, const void* q, const void* k_pool, const void* v_pool,
+                              void* o, void* stream);
+
 /* Static text for a cpa_status value. */
 CPA_API const char* cpa_strerror(int status);
 

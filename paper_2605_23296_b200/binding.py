@@ -66,6 +66,8 @@ _lib.cpa_kv_append.argtypes = [_vp, _vp, _vp, _i32p, _vp, _vp, _vp]
 _lib.cpa_kv_append.restype = ctypes.c_int
 _lib.cpa_decode.argtypes = [_vp, _vp, _vp, _vp, _vp, _vp, _vp]
 _lib.cpa_decode.restype = ctypes.c_int
+_lib.cpa_decode_static.argtypes = [_vp, _vp, _vp, _vp, _vp, _vp]
+_lib.cpa_decode_static.restype = ctypes.c_int
 _lib.cpa_strerror.argtypes = [ctypes.c_int]
 _lib.cpa_strerror.restype = ctypes.c_char_p
 
@@ -148,3 +150,18 @@ def cpa_kv_append(plan: int, k_new, v_new, new_lens, k_pool, v_pool, stream: int
 def cpa_decode(plan: int, q, k_pool, v_pool, o, d_workspace, stream: int = 0) -> int:
     return _lib.cpa_decode(plan, _ptr(q), _ptr(k_pool), _ptr(v_pool), _ptr(o), _ptr(d_workspace),
                            stream or None)
+
+
+STATIC_SCRATCH_BYTES = 16 << 20
+
+
+def cpa_decode_static(plan: int, q, k_pool, v_pool, o, stream: int = 0) -> int:
+    """cpa_decode with the split partials in the library's own fixed 16 MiB device array.
+
+    For callers that cannot allocate or pass scratch memory (a plugin behind a framework
+    that hands out fixed buffers, a service with a fully budgeted device).  Returns
+    CPA_ENOSPC if the plan needs more than STATIC_SCRATCH_BYTES.  Calls that overlap on
+    the device race on the shared array; the first call per device should happen outside
+    stream capture.
+    """
+    return _lib.cpa_decode_static(plan, _ptr(q), _ptr(k_pool), _ptr(v_pool), _ptr(o), stream or None)

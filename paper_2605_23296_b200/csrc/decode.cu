@@ -282,6 +282,11 @@ int launch_decode(const cpa_plan* plan, const void* q, const void* k_pool, const
     return cudaGetLastError() == cudaSuccess ? CPA_OK : CPA_ECUDA;
 }
 
+// Scratch for cpa_decode_static: lives in the library image, so every GPU that loads the
+// library holds these bytes until the process exits.
+constexpr int64_t kStaticScratchBytes = 16ll << 20;
+static __device__ __align__(256) unsigned char g_static_decode_scratch[kStaticScratchBytes];
+
 }  // namespace
 
 extern "C" int cpa_decode(const cpa_plan* plan, const void* q, const void* k_pool, const void* v_pool, void* o,
@@ -294,4 +299,33 @@ extern "C" int cpa_decode(const cpa_plan* plan, const void* q, const void* k_poo
     cudaStream_t st = (cudaStream_t)stream;
     return plan->cfg.head_dim == 128 ? launch_decode<128>(plan, q, k_pool, v_pool, o, d_workspace, st)
                                      : launch_decode<64>(plan, q, k_pool, v_pool, o, d_workspace, st);
+}
+
+extern "C" int cpa_decode_static(const cpa_plan* plan, const void* q, const void* k_pool, const void* v_pool,
+                                 void* o, void* stream) {
+    if (!plan || !q || !k_pool || !v_pool || !o) return CPA_EINVAL;
+    if (!cpa_aligned16(q) || !cpa_aligned16(k_pool) || !cpa_aligned16(v_pool) || !cpa_aligned16(o))
+        return CPA_EINVAL;
+    if (!plan->d_base) return CPA_ESTATE;
+    if (plan->decode_workspace_bytes() > kStaticScratchBytes) return CPA_ENOSPC;
+    // In host code the array's name is only a handle; its device address has to be asked for,
+    // once per device, with that device current.
+    constexpr int kMaxDevices = 64;
+    static void* scratch_addr[kMaxDevices] = {};
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) {
+        (void)cudaGetLastError();
+        return CPA_ECUDA;
+    }
+    if (!scratch_addr[dev]) {
+        void* p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_static_decode_scratch) != cudaSuccess || !p) {
+            (void)cudaGetLastError();
+            return CPA_ECUDA;
+        }
+        scratch_addr[dev] = p;
+    }
+    cudaStream_t st = (cudaStream_t)stream;
+    return plan->cfg.head_dim == 128 ? launch_decode<128>(plan, q, k_pool, v_pool, o, scratch_addr[dev], st)
+                                     : launch_decode<64>(plan, q, k_pool, v_pool, o, scratch_addr[dev], st);
 }
