@@ -16,7 +16,9 @@ struct cpa_dev_index {
     int32_t* append_indptr;        // [B+1] source-row offsets of a general append
     const int32_t* page_indices;   // [pages_used]
     const int32_t* prefill_items;  // [n_prefill, 2]
-    const int32_t* decode_items;   // [n_decode, 4]  (block, kv_head, split, pages) padded to 16 bytes
+    const int32_t* decode_items;   // [n_decode, item_stride]: (block, kv_head, split, pages) + the split's page ids
+    int32_t* merge_tickets;        // [B * Hkv] arrival counters of the fused split merge (zero between launches)
+    int32_t item_stride;           // int32 words per decode item: 4 + pages_per_split rounded up to 4
 };
 
 struct cpa_plan {
@@ -33,7 +35,8 @@ struct cpa_plan {
     // packed image of the device index buffer (int32 words) and offsets into it
     std::vector<int32_t> image;
     int64_t off_status = 0, off_cu = 0, off_pindptr = 0, off_sindptr = 0, off_seqlens = 0,
-            off_append = 0, off_pidx = 0, off_pitems = 0, off_ditems = 0, words = 0;
+            off_append = 0, off_pidx = 0, off_pitems = 0, off_ditems = 0, off_tickets = 0, words = 0;
+    int32_t item_stride = 0;
     int32_t* d_base = nullptr;   // caller's device buffer after cpa_plan_upload
     std::vector<int32_t> append_stage;  // host staging for general appends
 
@@ -55,6 +58,8 @@ struct cpa_plan {
         d.page_indices = d_base + off_pidx;
         d.prefill_items = d_base + off_pitems;
         d.decode_items = d_base + off_ditems;
+        d.merge_tickets = d_base + off_tickets;
+        d.item_stride = item_stride;
         return d;
     }
 };

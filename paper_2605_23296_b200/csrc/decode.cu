@@ -47,30 +47,62 @@ __device__ __forceinline__ uint32_t sel(const uint4& v, int i) {
     return i == 0 ? v.x : i == 1 ? v.y : i == 2 ? v.z : v.w;
 }
 
-// One work item = (block, kv head, split of up to C pages).  Four warps take the
-// split's pages round-robin, each keeps its own running (max, sum, acc); the CTA
-// merges them in shared memory and writes one partial per query head.
+// One work item = (block, kv head, split of up to C pages); the item record carries the
+// split's page ids, so the first K/V load waits for one earlier load only and is issued
+// before the cached length is known (every page of the record belongs to the block, so the
+// speculative read is in bounds; what lies beyond the length is masked by index).  Four
+// warps take the split's pages round-robin, each keeps its own running (max, sum, acc); the
+// CTA merges them in shared memory.  A block with a single active split is normalised and
+// stored directly; otherwise the CTA writes one partial per query head and takes a ticket:
+// the last CTA of a (block, kv head) to arrive merges all partials
+//     m = max_s m_s,  l = sum_s l_s 2^(m_s - m),  O = sum_s acc_s 2^(m_s - m) / l
+// and resets the ticket counter for the next launch.
 //   part_ml : [total_splits, Hq, 2]  (max in log2 units, sum), fp32
 //   part_o  : [total_splits, Hq, D]  unnormalised accumulators, fp32
 template <int D>
 __global__ void __launch_bounds__(kDecodeThreads, 4)
 decode_split_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ k_pool,
                     const __nv_bfloat16* __restrict__ v_pool, float* __restrict__ part_ml,
-                    float* __restrict__ part_o, cpa_dev_index ix, int Hq, int Hkv, int G, int C,
-                    float scale_log2) {
+                    float* __restrict__ part_o, __nv_bfloat16* __restrict__ out, cpa_dev_index ix, int Hq,
+                    int Hkv, int G, int C, float scale_log2) {
     constexpr int P = 16;
     constexpr int KC = D / 32;  // 16-byte K chunks per thread per 8-key group
     constexpr int VC = D / 64;  // 16-byte V chunks per thread per key row
-    const int4 item = reinterpret_cast<const int4*>(ix.decode_items)[blockIdx.x];
-    const int b = item.x, g = item.y, s = item.z;
-    const int len = ix.seq_lens[b];
-    const int pages_active = (len + P - 1) / P;
-    const int first = s * C;
-    if (first >= pages_active) return;  // split lies beyond the cached length (uniform per CTA)
-    const int last = min(first + C, pages_active);
+    const int32_t* item = ix.decode_items + (int64_t)blockIdx.x * ix.item_stride;
+    const int4 hdr = *reinterpret_cast<const int4*>(item);
+    const int b = hdr.x, g = hdr.y, s = hdr.z, n_reserved = hdr.w;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int gid = lane >> 2, tig = lane & 3;
+
+    // lane i keeps the id of this warp's i-th page (pages warp, warp+4, ... of the split)
+    int my_page = 0;
+    if (warp + kDecodeWarps * lane < n_reserved) my_page = item[4 + warp + kDecodeWarps * lane];
+    const int len = ix.seq_lens[b];
+
+    uint4 kreg[2][KC];
+    uint4 vreg[4][VC];
+    auto load_k = [&](int page) {
+        const __nv_bfloat16* base = k_pool + ((int64_t)page * Hkv + g) * (P * D);
+#pragma unroll
+        for (int t = 0; t < 2; ++t)
+#pragma unroll
+            for (int c = 0; c < KC; ++c) kreg[t][c] = ldg128(base + (gid + 8 * t) * D + (c * 4 + tig) * 8);
+    };
+    auto load_v = [&](int page) {
+        const __nv_bfloat16* base = v_pool + ((int64_t)page * Hkv + g) * (P * D);
+#pragma unroll
+        for (int r = 0; r < 4; ++r) {
+            const int row = 2 * tig + (r & 1) + 8 * (r >> 1);
+#pragma unroll
+            for (int c = 0; c < VC; ++c) vreg[r][c] = ldg128(base + row * D + (c * 8 + gid) * 8);
+        }
+    };
+    if (warp < n_reserved) {  // speculative: the page is the block's own even if still empty
+        const int page = __shfl_sync(0xffffffffu, my_page, 0);
+        load_k(page);
+        load_v(page);
+    }
 
     // Q fragments: row gid of the A tile is query head g*G + gid (zero rows beyond G)
     uint4 qf[KC];
@@ -82,25 +114,10 @@ decode_split_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __
         for (int c = 0; c < KC; ++c) qf[c] = *reinterpret_cast<const uint4*>(qrow + (c * 4 + tig) * 8);
     }
 
-    const int32_t* pages = ix.page_indices + ix.page_indptr[b];
-    uint4 kreg[2][KC];
-    uint4 vreg[4][VC];
-    auto load_k = [&](int pg) {
-        const __nv_bfloat16* base = k_pool + ((int64_t)pages[pg] * Hkv + g) * (P * D);
-#pragma unroll
-        for (int t = 0; t < 2; ++t)
-#pragma unroll
-            for (int c = 0; c < KC; ++c) kreg[t][c] = ldg128(base + (gid + 8 * t) * D + (c * 4 + tig) * 8);
-    };
-    auto load_v = [&](int pg) {
-        const __nv_bfloat16* base = v_pool + ((int64_t)pages[pg] * Hkv + g) * (P * D);
-#pragma unroll
-        for (int r = 0; r < 4; ++r) {
-            const int row = 2 * tig + (r & 1) + 8 * (r >> 1);
-#pragma unroll
-            for (int c = 0; c < VC; ++c) vreg[r][c] = ldg128(base + row * D + (c * 8 + gid) * 8);
-        }
-    };
+    const int pages_active = (len + P - 1) / P;
+    const int first = s * C;
+    const int n_active = min(n_reserved, pages_active - first);  // pages of this split that hold keys
+    if (n_active <= 0) return;  // split lies beyond the cached length (uniform per CTA)
 
     float acc[VC][4][4];
 #pragma unroll
@@ -112,9 +129,10 @@ decode_split_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __
     float m_run = -INFINITY;  // running max of raw scores, row gid
     float l_run = 0.f;        // this thread's share of the running sum, row gid
 
-    int pg = first + warp;
-    if (pg < last) { load_k(pg); load_v(pg); }
-    while (pg < last) {
+    for (int i = 0; warp + kDecodeWarps * i < n_active; ++i) {
+        const int pg = first + warp + kDecodeWarps * i;  // page index inside the block
+        const bool has_next = warp + kDecodeWarps * (i + 1) < n_active;
+        const int next_page = __shfl_sync(0xffffffffu, my_page, (i + 1) & 31);
         // ---- S = Q K^T for the 16 keys of this page
         float sc[2][4];
 #pragma unroll
@@ -126,8 +144,7 @@ decode_split_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __
                 mma_bf16_16816(sc[t], qf[c].z, 0u, qf[c].w, 0u, kreg[t][c].z, kreg[t][c].w);
             }
         }
-        const int next = pg + kDecodeWarps;
-        if (next < last) load_k(next);
+        if (has_next) load_k(next_page);
 
         // ---- mask the tail of the last page by index, then online softmax (row gid)
         const int key0 = pg * P + tig * 2;
@@ -175,15 +192,14 @@ decode_split_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __
 #pragma unroll
         for (int c = 0; c < VC; ++c)
 #pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                acc[c][i][0] *= a0; acc[c][i][1] *= a1; acc[c][i][2] *= a0; acc[c][i][3] *= a1;
-                const uint32_t r0 = sel(vreg[0][c], i), r1 = sel(vreg[1][c], i);
-                const uint32_t r2 = sel(vreg[2][c], i), r3 = sel(vreg[3][c], i);
-                mma_bf16_16816(acc[c][i], __byte_perm(r0, r1, 0x5410), __byte_perm(r0, r1, 0x7632),
+            for (int i2 = 0; i2 < 4; ++i2) {
+                acc[c][i2][0] *= a0; acc[c][i2][1] *= a1; acc[c][i2][2] *= a0; acc[c][i2][3] *= a1;
+                const uint32_t r0 = sel(vreg[0][c], i2), r1 = sel(vreg[1][c], i2);
+                const uint32_t r2 = sel(vreg[2][c], i2), r3 = sel(vreg[3][c], i2);
+                mma_bf16_16816(acc[c][i2], __byte_perm(r0, r1, 0x5410), __byte_perm(r0, r1, 0x7632),
                                __byte_perm(r2, r3, 0x5410), __byte_perm(r2, r3, 0x7632), pb0, pb1);
             }
-        if (next < last) load_v(next);
-        pg = next;
+        if (has_next) load_v(next_page);
     }
     l_run += __shfl_xor_sync(0xffffffffu, l_run, 1);
     l_run += __shfl_xor_sync(0xffffffffu, l_run, 2);
@@ -191,7 +207,8 @@ decode_split_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __
     // ---- merge the four warps
     __shared__ float sm_m[kDecodeWarps][8];
     __shared__ float sm_l[kDecodeWarps][8];
-    __shared__ float sm_o[kDecodeWarps][8][D + 4];
+    __shared__ __align__(8) float sm_o[kDecodeWarps][8][D + 4];
+    __shared__ int sm_last;
     if (tig == 0) { sm_m[warp][gid] = m_run * scale_log2; sm_l[warp][gid] = l_run; }
 #pragma unroll
     for (int c = 0; c < VC; ++c)
@@ -202,66 +219,72 @@ decode_split_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __
                 sm_o[warp][2 * tig + (e & 1)][8 * (8 * c + gid) + 2 * i + (e >> 1)] = acc[c][i][e];
     __syncthreads();
 
-    const int64_t prow = ((int64_t)(ix.split_indptr[b] + s) * Hq + g * G);
-    for (int idx = threadIdx.x; idx < G * D; idx += kDecodeThreads) {
-        const int h = idx / D, dim = idx - h * D;
+    const int n_splits = (pages_active + C - 1) / C;  // active splits of this block
+    const int64_t out_row = (int64_t)b * Hq + g * G;
+    const int64_t prow = (int64_t)(ix.split_indptr[b] + s) * Hq + g * G;
+    constexpr int HP = D / 2;  // dim pairs per head
+    for (int idx = threadIdx.x; idx < G * HP; idx += kDecodeThreads) {
+        const int h = idx / HP, dim = 2 * (idx - h * HP);
         float m = sm_m[0][h];
 #pragma unroll
         for (int w = 1; w < kDecodeWarps; ++w) m = fmaxf(m, sm_m[w][h]);
-        float o = 0.f, l = 0.f;
+        float o0 = 0.f, o1 = 0.f, l = 0.f;
 #pragma unroll
         for (int w = 0; w < kDecodeWarps; ++w) {
             const float mw = sm_m[w][h];
             const float f = (mw == -INFINITY) ? 0.f : exp2f(mw - m);
-            o = fmaf(f, sm_o[w][h][dim], o);
+            const float2 t = *reinterpret_cast<const float2*>(&sm_o[w][h][dim]);
+            o0 = fmaf(f, t.x, o0);
+            o1 = fmaf(f, t.y, o1);
             l = fmaf(f, sm_l[w][h], l);
         }
-        part_o[(prow + h) * D + dim] = o;
-        if (dim == 0) { part_ml[(prow + h) * 2] = m; part_ml[(prow + h) * 2 + 1] = l; }
+        if (n_splits == 1) {
+            const float inv = 1.f / l;
+            *reinterpret_cast<__nv_bfloat162*>(out + (out_row + h) * D + dim) = __floats2bfloat162_rn(o0 * inv, o1 * inv);
+        } else {
+            *reinterpret_cast<float2*>(part_o + (prow + h) * D + dim) = make_float2(o0, o1);
+            if (dim == 0) *reinterpret_cast<float2*>(part_ml + (prow + h) * 2) = make_float2(m, l);
+        }
+    }
+    if (n_splits == 1) return;
+
+    // ---- the last CTA of this (block, kv head) merges the splits
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        int* ticket = ix.merge_tickets + b * Hkv + g;
+        const int t = atomicAdd(ticket, 1);
+        sm_last = (t == n_splits - 1);
+        if (sm_last) *ticket = 0;  // every other split has arrived; ready for the next launch
+    }
+    __syncthreads();
+    if (!sm_last) return;
+    __threadfence();
+    const int64_t base = (int64_t)ix.split_indptr[b] * Hq + g * G;
+    for (int idx = threadIdx.x; idx < G * HP; idx += kDecodeThreads) {
+        const int h = idx / HP, dim = 2 * (idx - h * HP);
+        float m = -INFINITY;
+        for (int sp = 0; sp < n_splits; ++sp) m = fmaxf(m, __ldcg(part_ml + (base + (int64_t)sp * Hq + h) * 2));
+        float o0 = 0.f, o1 = 0.f, l = 0.f;
+        for (int sp = 0; sp < n_splits; ++sp) {
+            const int64_t r = base + (int64_t)sp * Hq + h;
+            const float2 ml = __ldcg(reinterpret_cast<const float2*>(part_ml + r * 2));
+            const float2 t = __ldcg(reinterpret_cast<const float2*>(part_o + r * D + dim));
+            const float f = exp2f(ml.x - m);
+            o0 = fmaf(f, t.x, o0);
+            o1 = fmaf(f, t.y, o1);
+            l = fmaf(f, ml.y, l);
+        }
+        const float inv = 1.f / l;
+        *reinterpret_cast<__nv_bfloat162*>(out + (out_row + h) * D + dim) = __floats2bfloat162_rn(o0 * inv, o1 * inv);
     }
 }
 
-// Merge of the split partials; one warp per (block, query head).
-template <int D>
-__global__ void __launch_bounds__(128)
-decode_combine_kernel(const float* __restrict__ part_ml, const float* __restrict__ part_o,
-                      __nv_bfloat16* __restrict__ out, cpa_dev_index ix, int B, int Hq, int C) {
-    constexpr int P = 16;
-    constexpr int E = D / 32;  // dims per lane
-    const int row = blockIdx.x * 4 + (threadIdx.x >> 5);
-    if (row >= B * Hq) return;
-    const int lane = threadIdx.x & 31;
-    const int b = row / Hq, h = row - b * Hq;
-    const int len = ix.seq_lens[b];
-    const int n_splits = ((len + P - 1) / P + C - 1) / C;
-    const int64_t base = (int64_t)ix.split_indptr[b] * Hq + h;
-    float m = -INFINITY;
-    for (int s = lane; s < n_splits; s += 32) m = fmaxf(m, part_ml[(base + (int64_t)s * Hq) * 2]);
-#pragma unroll
-    for (int off = 16; off > 0; off >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, off));
-    float o[E];
-#pragma unroll
-    for (int e = 0; e < E; ++e) o[e] = 0.f;
-    float l = 0.f;
-    for (int s = 0; s < n_splits; ++s) {
-        const int64_t r = base + (int64_t)s * Hq;
-        const float2 ml = *reinterpret_cast<const float2*>(part_ml + r * 2);
-        const float f = exp2f(ml.x - m);
-        l = fmaf(f, ml.y, l);
-        const float* po = part_o + r * D + lane * E;
-        if constexpr (E == 4) {
-            const float4 t = *reinterpret_cast<const float4*>(po);
-            o[0] = fmaf(f, t.x, o[0]); o[1] = fmaf(f, t.y, o[1]); o[2] = fmaf(f, t.z, o[2]); o[3] = fmaf(f, t.w, o[3]);
-        } else {
-            const float2 t = *reinterpret_cast<const float2*>(po);
-            o[0] = fmaf(f, t.x, o[0]); o[1] = fmaf(f, t.y, o[1]);
-        }
-    }
-    const float inv = n_splits > 0 ? 1.f / l : 0.f;
-    __nv_bfloat16* dst = out + (int64_t)row * D + lane * E;
-#pragma unroll
-    for (int e = 0; e < E; e += 2)
-        *reinterpret_cast<__nv_bfloat162*>(dst + e) = __floats2bfloat162_rn(o[e] * inv, o[e + 1] * inv);
+// A block whose cache is still empty has no active split and gets a zero output row.
+__global__ void decode_empty_rows_kernel(__nv_bfloat16* __restrict__ out, cpa_dev_index ix, int B, int row_elems) {
+    const int b = blockIdx.x;
+    if (b >= B || ix.seq_lens[b] > 0) return;
+    for (int i = threadIdx.x; i < row_elems; i += blockDim.x) out[(int64_t)b * row_elems + i] = __float2bfloat16(0.f);
 }
 
 template <int D>
@@ -273,12 +296,13 @@ int launch_decode(const cpa_plan* plan, const void* q, const void* k_pool, const
     float* part_ml = static_cast<float*>(ws);
     float* part_o = part_ml + ((int64_t)plan->split_indptr[plan->B] * c.num_q_heads * 2 + 3) / 4 * 4;
     const float scale_log2 = c.scale * 1.4426950408889634f;
+    bool any_empty = false;  // host mirror of the cached lengths
+    for (int b = 0; b < plan->B; ++b) any_empty |= plan->seq_lens[b] == 0;
+    if (any_empty)
+        decode_empty_rows_kernel<<<plan->B, 128, 0, st>>>((__nv_bfloat16*)o, ix, plan->B, c.num_q_heads * D);
     decode_split_kernel<D><<<plan->n_decode, kDecodeThreads, 0, st>>>(
-        (const __nv_bfloat16*)q, (const __nv_bfloat16*)k_pool, (const __nv_bfloat16*)v_pool, part_ml, part_o, ix,
-        c.num_q_heads, c.num_kv_heads, G, plan->C, scale_log2);
-    const int rows = plan->B * c.num_q_heads;
-    decode_combine_kernel<D><<<(rows + 3) / 4, 128, 0, st>>>(part_ml, part_o, (__nv_bfloat16*)o, ix, plan->B,
-                                                            c.num_q_heads, plan->C);
+        (const __nv_bfloat16*)q, (const __nv_bfloat16*)k_pool, (const __nv_bfloat16*)v_pool, part_ml, part_o,
+        (__nv_bfloat16*)o, ix, c.num_q_heads, c.num_kv_heads, G, plan->C, scale_log2);
     return cudaGetLastError() == cudaSuccess ? CPA_OK : CPA_ECUDA;
 }
 

@@ -35,6 +35,7 @@ extern "C" int cpa_plan_create(const cpa_config* cfg, int32_t num_blocks, const 
         cfg->num_q_heads / cfg->num_kv_heads > 8)
         return CPA_EUNSUPPORTED;
     if (cfg->q_tile_rows != 0 && cfg->q_tile_rows != 128) return CPA_EUNSUPPORTED;
+    if (cfg->pages_per_split > 128) return CPA_EUNSUPPORTED;
 
     cpa_plan* p = new (std::nothrow) cpa_plan();
     if (!p) return CPA_ENOSPC;
@@ -92,12 +93,13 @@ extern "C" int cpa_plan_create(const cpa_config* cfg, int32_t num_blocks, const 
     p->prefill_items.reserve(pit.size() * 2);
     for (const PItem& it : pit) { p->prefill_items.push_back(it.block); p->prefill_items.push_back(it.tile); }
 
-    // pages per decode split: the largest power of two (<= 64) that still yields
-    // about eight work items per SM; never below 4 pages unless asked for
+    // pages per decode split: the largest power of two (<= 64) that still fills about one
+    // wave of resident CTAs (four per SM); never below 4 pages unless asked for.  Few large
+    // splits amortise each CTA's start-up latency and keep the merge short.
     if (cfg->pages_per_split > 0) {
         p->C = cfg->pages_per_split;
     } else {
-        const int64_t target = 8LL * (cfg->num_sms ? cfg->num_sms : 148);
+        const int64_t target = 7LL * (cfg->num_sms ? cfg->num_sms : 148) / 2;
         int32_t C = 64;
         while (C > 4 && decode_item_count(pages_per_block, cfg->num_kv_heads, C) < target) C /= 2;
         p->C = C;
@@ -136,7 +138,9 @@ extern "C" int cpa_plan_create(const cpa_config* cfg, int32_t num_blocks, const 
     p->off_append = w;  w = align4(w + B + 1);
     p->off_pidx = w;    w = align4(w + pages_used);
     p->off_pitems = w;  w = align4(w + 2LL * p->n_prefill);
-    p->off_ditems = w;  w = align4(w + 4LL * p->n_decode);
+    p->item_stride = 4 + (p->C + 3) / 4 * 4;
+    p->off_ditems = w;  w = align4(w + (int64_t)p->item_stride * p->n_decode);
+    p->off_tickets = w; w = align4(w + (int64_t)B * cfg->num_kv_heads);
     p->words = w;
     p->image.assign((size_t)w, 0);
     int32_t* im = p->image.data();
@@ -146,10 +150,15 @@ extern "C" int cpa_plan_create(const cpa_config* cfg, int32_t num_blocks, const 
     std::memcpy(im + p->off_pidx, p->page_indices.data(), sizeof(int32_t) * pages_used);
     std::memcpy(im + p->off_pitems, p->prefill_items.data(), sizeof(int32_t) * 2 * p->n_prefill);
     for (int32_t i = 0; i < p->n_decode; ++i) {
-        im[p->off_ditems + 4 * i + 0] = dit[i].block;
-        im[p->off_ditems + 4 * i + 1] = dit[i].head;
-        im[p->off_ditems + 4 * i + 2] = dit[i].split;
-        im[p->off_ditems + 4 * i + 3] = dit[i].pages;
+        // a decode item carries its own page ids, so the kernel's first KV load depends on
+        // one prior load only
+        int32_t* it = im + p->off_ditems + (int64_t)p->item_stride * i;
+        it[0] = dit[i].block;
+        it[1] = dit[i].head;
+        it[2] = dit[i].split;
+        it[3] = dit[i].pages;
+        const int32_t* src = p->page_indices.data() + p->page_indptr[dit[i].block] + dit[i].split * p->C;
+        for (int32_t j = 0; j < dit[i].pages; ++j) it[4 + j] = src[j];
     }
     p->append_stage.assign(B + 1, 0);
     *out = p;

@@ -84,7 +84,7 @@ def test_auto_split_aims_at_the_sm_count():
         cb = B.cpa_plan_param(plan_b, B.PARAM_PAGES_PER_SPLIT)
         assert cb >= ca
         items = B.cpa_plan_export(plan_a, B.ARR_DECODE_ITEMS).shape[0]
-        assert items >= 8 * 148 or ca == 4
+        assert items >= 7 * 148 // 2 or ca == 4
     finally:
         B.cpa_plan_destroy(plan_a)
         B.cpa_plan_destroy(plan_b)
@@ -109,6 +109,7 @@ def test_plan_errors():
     assert rc(cfg=B.cpa_config(8, 2, 64, 32, 0.125, 0, 0, 0)) == B.CPA_EUNSUPPORTED  # page size
     assert rc(cfg=B.cpa_config(16, 1, 64, 16, 0.125, 0, 0, 0)) == B.CPA_EUNSUPPORTED # G = 16
     assert rc(cfg=B.cpa_config(8, 2, 64, 16, 0.0, 0, 0, 0)) == B.CPA_EINVAL          # scale
+    assert rc(cfg=B.cpa_config(8, 2, 64, 16, 0.125, 0, 129, 0)) == B.CPA_EUNSUPPORTED # split size
     with pytest.raises(B.CpaError):
         B.cpa_plan_create(ok, (40, 0), 4, free)
     # T = 0 is allowed (prefill only)
