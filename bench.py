@@ -239,7 +239,8 @@ def run_gpu(args) -> None:
     def one_pass(q, k, v, qd, kd, vd, o, od, ev=None, dec_events=None):
         """plan -> prefill -> bulk append -> T x (append, decode); all through the C-ABI."""
         s = CompactionSession(w.block_lens, T, w.num_q_heads, w.num_kv_heads, w.head_dim,
-                              w.free_pages, w.num_pages, scale=w.scale, device=str(dev))
+                              w.free_pages, w.num_pages, scale=w.scale, device=str(dev),
+                              pages_per_split=args.pages_per_split)
         if ev:
             ev["planned"].record(stream)
         s.prefill(q, k, v, out=o)
@@ -395,6 +396,7 @@ def main() -> None:
     ap.add_argument("--blocks", type=int, default=0, help="override the number of blocks (profiling)")
     ap.add_argument("--block-len", type=int, default=0, help="override the block length (profiling)")
     ap.add_argument("--decode-steps", type=int, default=0, help="override the decode steps (profiling)")
+    ap.add_argument("--pages-per-split", type=int, default=0, help="decode split size (0 = planner's choice)")
     ap.add_argument("--skip-e2e", action="store_true", help="skip the host-buffer leg (profiling)")
     ap.add_argument("--skip-cpu", action="store_true", help="skip the CPU oracle leg (profiling)")
     args = ap.parse_args()

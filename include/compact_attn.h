@@ -65,7 +65,7 @@ typedef struct cpa_config {
     int32_t page_size;       /* 16 */
     float   scale;           /* softmax scale, normally 1/sqrt(head_dim) */
     int32_t q_tile_rows;     /* query rows per prefill work item; 0 = default (128) */
-    int32_t pages_per_split; /* KV pages per decode work item (<= 128); 0 = chosen from the batch */
+    int32_t pages_per_split; /* KV pages per decode work item (<= 1024); 0 = chosen per block from the batch */
     int32_t num_sms;         /* SM count the split heuristic aims at; 0 = 148 */
 } cpa_config;
 
@@ -80,7 +80,8 @@ enum {
     CPA_ARR_SLOT_MAPPING = 4,  /* [tokens] pool slot (page*P + offset) of every prefill token */
     CPA_ARR_PREFILL_ITEMS = 5, /* [n,2] (block, q_tile) in launch order */
     CPA_ARR_DECODE_ITEMS = 6,  /* [n,3] (block, kv_head, split) in launch order */
-    CPA_ARR_SPLIT_INDPTR = 7   /* [B+1] prefix sums of decode splits per block */
+    CPA_ARR_SPLIT_INDPTR = 7,  /* [B+1] prefix sums of decode splits per block */
+    CPA_ARR_SPLIT_PAGES = 8    /* [B] pages per decode split of each block (the last split may be shorter) */
 };
 
 /* Scalars of a plan, for cpa_plan_param. */
@@ -88,7 +89,7 @@ enum {
     CPA_PARAM_NUM_BLOCKS = 0,
     CPA_PARAM_TOTAL_TOKENS = 1,
     CPA_PARAM_Q_TILE_ROWS = 2,
-    CPA_PARAM_PAGES_PER_SPLIT = 3,
+    CPA_PARAM_PAGES_PER_SPLIT = 3,       /* largest split size over the blocks */
     CPA_PARAM_PAGES_USED = 4,            /* page_indptr[B] */
     CPA_PARAM_INDEX_BYTES = 5,           /* size of the device index buffer for cpa_plan_upload */
     CPA_PARAM_DECODE_WORKSPACE_BYTES = 6,/* size of cpa_decode's device workspace */
@@ -104,8 +105,11 @@ enum {
  *   the slot of every prefill token; the prefill work list of (block, q_tile)
  *   ordered by descending cost (keys seen by the tile's last row), ties by
  *   ascending block then tile; the decode work list of (block, kv_head, split),
- *   split s = pages [s*C, (s+1)*C) of the block, ordered by descending page
- *   count, ties by ascending block, kv head, split.
+ *   split s = pages [s*C_b, (s+1)*C_b) of the block, ordered by descending page
+ *   count, ties by ascending block, kv head, split.  C_b is cfg->pages_per_split, or
+ *   with 0 it is chosen per block so that all items fill one wave of CTAs (two per
+ *   SM): splits start at one per block and the block with the largest splits is
+ *   split further while kv_heads more items still fit (never below 4 pages).
  * block_lens, free_pages: host int32 arrays (copied; caller keeps ownership).
  * Page ids must be >= 0 and distinct (distinctness is the caller's contract).
  * Errors: CPA_EINVAL (null pointer, num_blocks < 1, a length < 1,

@@ -15,10 +15,11 @@ stated in full):
 * prefill items   (block, q_tile) for q_tile < ceil(L_b / q_tile_rows); cost is
                   the number of keys its last row sees; order: descending cost,
                   ties by ascending block, then tile
-* decode items    (block, kv_head, split): split s covers pages
-                  [s*C, min((s+1)*C, pages_b)); order: descending page count,
-                  ties by ascending block, kv head, split
-* split_indptr    prefix sums of ceil(pages_b / C)
+* decode items    (block, kv_head, split): split s of block b covers pages
+                  [s*C_b, min((s+1)*C_b, pages_b)); order: descending page count,
+                  ties by ascending block, kv head, split.  C_b (pages per split)
+                  is an input: one number for all blocks or one per block
+* split_indptr    prefix sums of ceil(pages_b / C_b)
 """
 from __future__ import annotations
 
@@ -37,13 +38,17 @@ def partition(history_len: int, block_size: int):
 
 def build_plan(block_lens: Sequence[int], max_new_tokens: int, page_size: int,
                free_pages: Sequence[int], num_kv_heads: int,
-               q_tile_rows: int, pages_per_split: int) -> Dict[str, list]:
+               q_tile_rows: int, pages_per_split) -> Dict[str, list]:
     B = len(block_lens)
     if B < 1:
         raise ValueError("need at least one block")
     if any(int(L) < 1 for L in block_lens):
         raise ValueError("block lengths must be >= 1")
-    if max_new_tokens < 0 or page_size < 1 or q_tile_rows < 1 or pages_per_split < 1:
+    if isinstance(pages_per_split, int):
+        pages_per_split = [pages_per_split] * B
+    if len(pages_per_split) != B:
+        raise ValueError("one split size per block")
+    if max_new_tokens < 0 or page_size < 1 or q_tile_rows < 1 or min(pages_per_split) < 1:
         raise ValueError("bad parameter")
 
     cu = [0]
@@ -79,11 +84,12 @@ def build_plan(block_lens: Sequence[int], max_new_tokens: int, page_size: int,
     split_indptr = [0]
     decode = []
     for b, n in enumerate(pages_per_block):
-        n_splits = (n + pages_per_split - 1) // pages_per_split
+        c_b = int(pages_per_split[b])
+        n_splits = (n + c_b - 1) // c_b
         split_indptr.append(split_indptr[-1] + n_splits)
         for g in range(num_kv_heads):
             for s in range(n_splits):
-                size = min(pages_per_split, n - s * pages_per_split)
+                size = min(c_b, n - s * c_b)
                 decode.append((-size, b, g, s))
     decode.sort()
     decode_items = [[b, g, s] for (_, b, g, s) in decode]

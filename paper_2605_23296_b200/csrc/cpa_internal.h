@@ -16,9 +16,9 @@ struct cpa_dev_index {
     int32_t* append_indptr;        // [B+1] source-row offsets of a general append
     const int32_t* page_indices;   // [pages_used]
     const int32_t* prefill_items;  // [n_prefill, 2]
-    const int32_t* decode_items;   // [n_decode, item_stride]: (block, kv_head, split, pages) + the split's page ids
+    const int32_t* decode_items;   // [n_decode, item_stride]: (block, kv_head, split, pages, split size, 0, 0, 0) + page ids
     int32_t* merge_tickets;        // [B * Hkv] arrival counters of the fused split merge (zero between launches)
-    int32_t item_stride;           // int32 words per decode item: 4 + pages_per_split rounded up to 4
+    int32_t item_stride;           // int32 words per decode item: 8 + largest split size rounded up to 4
 };
 
 struct cpa_plan {
@@ -26,10 +26,10 @@ struct cpa_plan {
     int32_t B = 0;
     int32_t T = 0;          // max_new_tokens
     int32_t q_tile = 0;     // query rows per prefill item
-    int32_t C = 0;          // pages per decode split
+    int32_t C = 0;          // largest pages-per-split over the blocks
     int64_t total_tokens = 0;
     std::vector<int32_t> block_lens, cu_seqlens, page_indptr, page_indices, seq_lens, slot_mapping,
-        prefill_items, decode_items, split_indptr;
+        prefill_items, decode_items, split_indptr, split_pages;
     int32_t n_prefill = 0, n_decode = 0;
 
     // packed image of the device index buffer (int32 words) and offsets into it

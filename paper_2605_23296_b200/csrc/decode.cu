@@ -1,17 +1,22 @@
 // Batched paged-KV decode attention: one query token per block over that block's
 // pages, split over the KV length, then a log-sum-exp merge of the split partials.
 //
-// The step is a streaming scan of the KV pool and is bound by HBM bandwidth: every
-// K and V element is read once per kv head, with 128-bit loads straight into
-// registers; the G query heads of a kv-head group share those registers.  The
-// per-key arithmetic runs on the legacy warp-level MMA (m16n8k16, bf16 in, fp32
-// accumulate), which costs nothing next to the memory stream and keeps the fp32
-// ALU free at G = 8:
+// The step is a streaming scan of the KV pool and is bound by HBM bandwidth: every K
+// and V element is read once per kv head.  A (page, kv head) chunk of the pool is
+// contiguous (16 keys x head_dim bf16), so it moves with ONE bulk asynchronous copy
+// (cp.async.bulk, global -> shared, completion counted on an mbarrier).  Each warp
+// owns a ring of stages in shared memory and keeps several pages in flight without
+// spending registers or L1 miss slots on them; that depth, not arithmetic, decides
+// the bandwidth reached.
+//
+// The per-key arithmetic runs on the warp-level MMA (m16n8k16, bf16 in, fp32
+// accumulate), which costs nothing next to the memory stream and keeps the fp32 ALU
+// free at G = 8; the G query heads of a kv-head group share every byte read:
 //   S  [heads(16, G used) x keys(8)]   = Q [heads x dims] . K^T      (A = Q, B = K rows)
 //   O^T[dims(16) x heads(8, G used)]  += V^T[dims x keys(16)] . P^T  (A = V^T, B = P)
-// Both contractions are invariant under a permutation of the contracted index, so
-// a thread loads whole 16-byte chunks and pairs registers up as the MMA fragments
-// need them; no shared-memory staging, no transposes.
+// Both contractions are invariant under a permutation of the contracted index, so a
+// thread reads whole 16-byte chunks from the staged page and pairs registers up as
+// the MMA fragments need them; no transposes, no ldmatrix.
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 
@@ -21,6 +26,9 @@ namespace {
 
 constexpr int kDecodeWarps = 4;
 constexpr int kDecodeThreads = kDecodeWarps * 32;
+constexpr int kDecodeSmemBytes = 96 * 1024;          // stage rings of the four warps (two CTAs per SM)
+constexpr int kMaxSplitPages = 1024;                 // planner's cap on pages per split
+constexpr uint32_t kSpinLimit = 1u << 18;            // bounded mbarrier wait (each try suspends briefly)
 
 __device__ __forceinline__ void mma_bf16_16816(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
                                                uint32_t b0, uint32_t b1) {
@@ -35,11 +43,9 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
     return *reinterpret_cast<uint32_t*>(&t);
 }
 
-__device__ __forceinline__ uint4 ldg128(const void* p) {
+__device__ __forceinline__ uint4 lds128(uint32_t addr) {
     uint4 r;
-    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];\n"
-                 : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w)
-                 : "l"(p));
+    asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];\n" : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w) : "r"(addr));
     return r;
 }
 
@@ -47,62 +53,93 @@ __device__ __forceinline__ uint32_t sel(const uint4& v, int i) {
     return i == 0 ? v.x : i == 1 ? v.y : i == 2 ? v.z : v.w;
 }
 
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;\n" :: "r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;\n" :: "r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}\n"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok;
+}
+// Contiguous global -> shared copy; both addresses 16-byte aligned, size a multiple of 16.
+__device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];\n"
+                 :: "r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
+
 // One work item = (block, kv head, split of up to C pages); the item record carries the
-// split's page ids, so the first K/V load waits for one earlier load only and is issued
-// before the cached length is known (every page of the record belongs to the block, so the
-// speculative read is in bounds; what lies beyond the length is masked by index).  Four
-// warps take the split's pages round-robin, each keeps its own running (max, sum, acc); the
-// CTA merges them in shared memory.  A block with a single active split is normalised and
-// stored directly; otherwise the CTA writes one partial per query head and takes a ticket:
-// the last CTA of a (block, kv head) to arrive merges all partials
+// split's page ids.  Four warps take the split's pages round-robin; each streams its pages
+// through its own ring of STAGES shared-memory stages (K chunk + V chunk per stage) and
+// keeps its own running (max, sum, acc).  The CTA then merges the four warps in shared
+// memory.  A block with a single active split is normalised and stored directly; otherwise
+// the CTA writes one partial per query head and takes a ticket: the last CTA of a
+// (block, kv head) to arrive merges all partials
 //     m = max_s m_s,  l = sum_s l_s 2^(m_s - m),  O = sum_s acc_s 2^(m_s - m) / l
 // and resets the ticket counter for the next launch.
 //   part_ml : [total_splits, Hq, 2]  (max in log2 units, sum), fp32
 //   part_o  : [total_splits, Hq, D]  unnormalised accumulators, fp32
 template <int D>
-__global__ void __launch_bounds__(kDecodeThreads, 4)
+__global__ void __launch_bounds__(kDecodeThreads, 2)
 decode_split_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ k_pool,
                     const __nv_bfloat16* __restrict__ v_pool, float* __restrict__ part_ml,
                     float* __restrict__ part_o, __nv_bfloat16* __restrict__ out, cpa_dev_index ix, int Hq,
-                    int Hkv, int G, int C, float scale_log2) {
+                    int Hkv, int G, float scale_log2) {
     constexpr int P = 16;
     constexpr int KC = D / 32;  // 16-byte K chunks per thread per 8-key group
     constexpr int VC = D / 64;  // 16-byte V chunks per thread per key row
-    const int32_t* item = ix.decode_items + (int64_t)blockIdx.x * ix.item_stride;
-    const int4 hdr = *reinterpret_cast<const int4*>(item);
-    const int b = hdr.x, g = hdr.y, s = hdr.z, n_reserved = hdr.w;
+    constexpr uint32_t kChunkBytes = P * D * 2;                  // one (page, head) chunk of K or of V
+    constexpr uint32_t kStageBytes = 2 * kChunkBytes;
+    constexpr int STAGES = kDecodeSmemBytes / kDecodeWarps / kStageBytes;   // 3 at d=128, 6 at d=64
+    extern __shared__ __align__(128) unsigned char dsm[];
+    __shared__ __align__(8) uint64_t sm_bar[kDecodeWarps][STAGES];
+    __shared__ float sm_m[kDecodeWarps][8];
+    __shared__ float sm_l[kDecodeWarps][8];
+    __shared__ int sm_last;
+    __shared__ int sm_pages[kDecodeWarps][kMaxSplitPages / kDecodeWarps];  // page ids of each warp's pages
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int gid = lane >> 2, tig = lane & 3;
-
-    // lane i keeps the id of this warp's i-th page (pages warp, warp+4, ... of the split)
-    int my_page = 0;
-    if (warp + kDecodeWarps * lane < n_reserved) my_page = item[4 + warp + kDecodeWarps * lane];
-    const int len = ix.seq_lens[b];
-
-    uint4 kreg[2][KC];
-    uint4 vreg[4][VC];
-    auto load_k = [&](int page) {
-        const __nv_bfloat16* base = k_pool + ((int64_t)page * Hkv + g) * (P * D);
+    const uint32_t ring = (uint32_t)__cvta_generic_to_shared(dsm) + warp * (STAGES * kStageBytes);
+    const uint32_t bar0 = (uint32_t)__cvta_generic_to_shared(&sm_bar[warp][0]);
+    if (lane == 0) {
 #pragma unroll
-        for (int t = 0; t < 2; ++t)
-#pragma unroll
-            for (int c = 0; c < KC; ++c) kreg[t][c] = ldg128(base + (gid + 8 * t) * D + (c * 4 + tig) * 8);
-    };
-    auto load_v = [&](int page) {
-        const __nv_bfloat16* base = v_pool + ((int64_t)page * Hkv + g) * (P * D);
-#pragma unroll
-        for (int r = 0; r < 4; ++r) {
-            const int row = 2 * tig + (r & 1) + 8 * (r >> 1);
-#pragma unroll
-            for (int c = 0; c < VC; ++c) vreg[r][c] = ldg128(base + row * D + (c * 8 + gid) * 8);
-        }
-    };
-    if (warp < n_reserved) {  // speculative: the page is the block's own even if still empty
-        const int page = __shfl_sync(0xffffffffu, my_page, 0);
-        load_k(page);
-        load_v(page);
+        for (int st = 0; st < STAGES; ++st) mbar_init(bar0 + 8 * st, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory");
     }
+    __syncwarp();
+
+    const int32_t* item = ix.decode_items + (int64_t)blockIdx.x * ix.item_stride;
+    const int4 hdr = *reinterpret_cast<const int4*>(item);
+    const int b = hdr.x, g = hdr.y, s = hdr.z, n_reserved = hdr.w;
+    const int C = item[4];  // pages per split of this block
+    // this warp's pages are warp, warp+4, ... of the split: park their ids in shared memory
+    for (int j = lane; warp + kDecodeWarps * j < n_reserved; j += 32)
+        sm_pages[warp][j] = item[8 + warp + kDecodeWarps * j];
+    const int len = ix.seq_lens[b];
+    __syncwarp();
+    const int pages_active = (len + P - 1) / P;
+    const int first = s * C;
+    const int n_active = min(n_reserved, pages_active - first);  // pages of this split that hold keys
+    if (n_active <= 0) return;  // split lies beyond the cached length (uniform per CTA)
+    const int n_mine = (n_active - warp + kDecodeWarps - 1) / kDecodeWarps;  // pages of this warp (may be <= 0)
+
+    auto issue = [&](int st, int page) {  // lane 0 only
+        const uint32_t bar = bar0 + 8 * st;
+        const uint32_t dst = ring + st * kStageBytes;
+        const int64_t chunk = ((int64_t)page * Hkv + g) * (P * D);
+        mbar_expect_tx(bar, kStageBytes);
+        bulk_load(dst, k_pool + chunk, kChunkBytes, bar);
+        bulk_load(dst + kChunkBytes, v_pool + chunk, kChunkBytes, bar);
+    };
+#pragma unroll
+    for (int st = 0; st < STAGES; ++st)
+        if (st < n_mine && lane == 0) issue(st, sm_pages[warp][st]);
 
     // Q fragments: row gid of the A tile is query head g*G + gid (zero rows beyond G)
     uint4 qf[KC];
@@ -114,11 +151,6 @@ decode_split_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __
         for (int c = 0; c < KC; ++c) qf[c] = *reinterpret_cast<const uint4*>(qrow + (c * 4 + tig) * 8);
     }
 
-    const int pages_active = (len + P - 1) / P;
-    const int first = s * C;
-    const int n_active = min(n_reserved, pages_active - first);  // pages of this split that hold keys
-    if (n_active <= 0) return;  // split lies beyond the cached length (uniform per CTA)
-
     float acc[VC][4][4];
 #pragma unroll
     for (int c = 0; c < VC; ++c)
@@ -128,11 +160,20 @@ decode_split_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __
             for (int e = 0; e < 4; ++e) acc[c][i][e] = 0.f;
     float m_run = -INFINITY;  // running max of raw scores, row gid
     float l_run = 0.f;        // this thread's share of the running sum, row gid
+    bool gave_up = false;     // a bounded wait ran out: stop waiting, results are void, status says so
 
-    for (int i = 0; warp + kDecodeWarps * i < n_active; ++i) {
+    for (int i = 0; i < n_mine; ++i) {
+        const int st = i % STAGES;
+        const uint32_t parity = (uint32_t)(i / STAGES) & 1u;
         const int pg = first + warp + kDecodeWarps * i;  // page index inside the block
-        const bool has_next = warp + kDecodeWarps * (i + 1) < n_active;
-        const int next_page = __shfl_sync(0xffffffffu, my_page, (i + 1) & 31);
+        if (!gave_up) {
+            uint32_t spins = 0;
+            while (!mbar_try_wait(bar0 + 8 * st, parity)) {
+                if (++spins > kSpinLimit) { gave_up = true; atomicCAS(ix.status, 0, 1); break; }
+            }
+        }
+        const uint32_t ks = ring + st * kStageBytes;
+        const uint32_t vs = ks + kChunkBytes;
         // ---- S = Q K^T for the 16 keys of this page
         float sc[2][4];
 #pragma unroll
@@ -140,12 +181,11 @@ decode_split_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __
             sc[t][0] = sc[t][1] = sc[t][2] = sc[t][3] = 0.f;
 #pragma unroll
             for (int c = 0; c < KC; ++c) {
-                mma_bf16_16816(sc[t], qf[c].x, 0u, qf[c].y, 0u, kreg[t][c].x, kreg[t][c].y);
-                mma_bf16_16816(sc[t], qf[c].z, 0u, qf[c].w, 0u, kreg[t][c].z, kreg[t][c].w);
+                const uint4 kr = lds128(ks + (gid + 8 * t) * (D * 2) + (c * 4 + tig) * 16);
+                mma_bf16_16816(sc[t], qf[c].x, 0u, qf[c].y, 0u, kr.x, kr.y);
+                mma_bf16_16816(sc[t], qf[c].z, 0u, qf[c].w, 0u, kr.z, kr.w);
             }
         }
-        if (has_next) load_k(next_page);
-
         // ---- mask the tail of the last page by index, then online softmax (row gid)
         const int key0 = pg * P + tig * 2;
         const bool partial = (pg + 1) * P > len;
@@ -178,37 +218,37 @@ decode_split_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __
         const float a0 = __shfl_sync(0xffffffffu, alpha, (2 * tig) * 4);
         const float a1 = __shfl_sync(0xffffffffu, alpha, (2 * tig + 1) * 4);
 
-        if (partial) {  // unused slots may hold anything (even NaN): select them away
+        // ---- O^T += V^T P^T
+#pragma unroll
+        for (int c = 0; c < VC; ++c) {
+            uint4 vr[4];
 #pragma unroll
             for (int r = 0; r < 4; ++r) {
                 const int row = 2 * tig + (r & 1) + 8 * (r >> 1);
-                if (pg * P + row >= len) {
-#pragma unroll
-                    for (int c = 0; c < VC; ++c) vreg[r][c] = make_uint4(0, 0, 0, 0);
-                }
+                vr[r] = lds128(vs + row * (D * 2) + (c * 8 + gid) * 16);
+                // unused slots may hold anything (even NaN): select them away
+                if (partial && pg * P + row >= len) vr[r] = make_uint4(0, 0, 0, 0);
             }
-        }
-        // ---- O^T += V^T P^T
-#pragma unroll
-        for (int c = 0; c < VC; ++c)
 #pragma unroll
             for (int i2 = 0; i2 < 4; ++i2) {
                 acc[c][i2][0] *= a0; acc[c][i2][1] *= a1; acc[c][i2][2] *= a0; acc[c][i2][3] *= a1;
-                const uint32_t r0 = sel(vreg[0][c], i2), r1 = sel(vreg[1][c], i2);
-                const uint32_t r2 = sel(vreg[2][c], i2), r3 = sel(vreg[3][c], i2);
+                const uint32_t r0 = sel(vr[0], i2), r1 = sel(vr[1], i2);
+                const uint32_t r2 = sel(vr[2], i2), r3 = sel(vr[3], i2);
                 mma_bf16_16816(acc[c][i2], __byte_perm(r0, r1, 0x5410), __byte_perm(r0, r1, 0x7632),
                                __byte_perm(r2, r3, 0x5410), __byte_perm(r2, r3, 0x7632), pb0, pb1);
             }
-        if (has_next) load_v(next_page);
+        }
+        // every lane has taken what it needs from this stage: refill it
+        __syncwarp();
+        const int nxt = i + STAGES;
+        if (nxt < n_mine && lane == 0) issue(st, sm_pages[warp][nxt]);
     }
     l_run += __shfl_xor_sync(0xffffffffu, l_run, 1);
     l_run += __shfl_xor_sync(0xffffffffu, l_run, 2);
 
-    // ---- merge the four warps
-    __shared__ float sm_m[kDecodeWarps][8];
-    __shared__ float sm_l[kDecodeWarps][8];
-    __shared__ __align__(8) float sm_o[kDecodeWarps][8][D + 4];
-    __shared__ int sm_last;
+    // ---- merge the four warps; the stage rings are idle now (every issued copy was consumed)
+    __syncthreads();
+    float (*sm_o)[8][D + 4] = reinterpret_cast<float (*)[8][D + 4]>(dsm);
     if (tig == 0) { sm_m[warp][gid] = m_run * scale_log2; sm_l[warp][gid] = l_run; }
 #pragma unroll
     for (int c = 0; c < VC; ++c)
@@ -298,11 +338,20 @@ int launch_decode(const cpa_plan* plan, const void* q, const void* k_pool, const
     const float scale_log2 = c.scale * 1.4426950408889634f;
     bool any_empty = false;  // host mirror of the cached lengths
     for (int b = 0; b < plan->B; ++b) any_empty |= plan->seq_lens[b] == 0;
+    static bool configured = false;  // per instantiation; one device per process assumed for this cache
+    if (!configured) {
+        if (cudaFuncSetAttribute(decode_split_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 kDecodeSmemBytes) != cudaSuccess) {
+            (void)cudaGetLastError();
+            return CPA_ECUDA;
+        }
+        configured = true;
+    }
     if (any_empty)
         decode_empty_rows_kernel<<<plan->B, 128, 0, st>>>((__nv_bfloat16*)o, ix, plan->B, c.num_q_heads * D);
-    decode_split_kernel<D><<<plan->n_decode, kDecodeThreads, 0, st>>>(
+    decode_split_kernel<D><<<plan->n_decode, kDecodeThreads, kDecodeSmemBytes, st>>>(
         (const __nv_bfloat16*)q, (const __nv_bfloat16*)k_pool, (const __nv_bfloat16*)v_pool, part_ml, part_o,
-        (__nv_bfloat16*)o, ix, c.num_q_heads, c.num_kv_heads, G, plan->C, scale_log2);
+        (__nv_bfloat16*)o, ix, c.num_q_heads, c.num_kv_heads, G, scale_log2);
     return cudaGetLastError() == cudaSuccess ? CPA_OK : CPA_ECUDA;
 }
 

@@ -13,11 +13,7 @@ namespace {
 
 int64_t align4(int64_t words) { return (words + 3) / 4 * 4; }  // 16-byte alignment of every array
 
-int64_t decode_item_count(const std::vector<int32_t>& pages_per_block, int32_t hkv, int32_t C) {
-    int64_t n = 0;
-    for (int32_t p : pages_per_block) n += (int64_t)hkv * ((p + C - 1) / C);
-    return n;
-}
+constexpr int32_t kMaxSplitPages = 1024;  // page ids of one split the decode kernel keeps in shared memory
 
 }  // namespace
 
@@ -35,7 +31,7 @@ extern "C" int cpa_plan_create(const cpa_config* cfg, int32_t num_blocks, const 
         cfg->num_q_heads / cfg->num_kv_heads > 8)
         return CPA_EUNSUPPORTED;
     if (cfg->q_tile_rows != 0 && cfg->q_tile_rows != 128) return CPA_EUNSUPPORTED;
-    if (cfg->pages_per_split > 128) return CPA_EUNSUPPORTED;
+    if (cfg->pages_per_split > kMaxSplitPages) return CPA_EUNSUPPORTED;
 
     cpa_plan* p = new (std::nothrow) cpa_plan();
     if (!p) return CPA_ENOSPC;
@@ -93,26 +89,45 @@ extern "C" int cpa_plan_create(const cpa_config* cfg, int32_t num_blocks, const 
     p->prefill_items.reserve(pit.size() * 2);
     for (const PItem& it : pit) { p->prefill_items.push_back(it.block); p->prefill_items.push_back(it.tile); }
 
-    // pages per decode split: the largest power of two (<= 64) that still fills about one
-    // wave of resident CTAs (four per SM); never below 4 pages unless asked for.  Few large
-    // splits amortise each CTA's start-up latency and keep the merge short.
+    // Decode splits.  Every CTA pays a fixed start-up and merge cost, so the planner aims at
+    // ONE wave of resident CTAs (two per SM): starting from one split per block, it keeps
+    // splitting the block whose splits are largest while the item count (kv heads x splits)
+    // still fits.  split_pages[b] is the page count of block b's splits (the last may be
+    // shorter).  A fixed pages_per_split from the configuration overrides the search.
+    p->split_pages.assign(B, 0);
+    std::vector<int32_t> n_splits(B, 1);
     if (cfg->pages_per_split > 0) {
-        p->C = cfg->pages_per_split;
+        for (int32_t b = 0; b < B; ++b) p->split_pages[b] = cfg->pages_per_split;
     } else {
-        const int64_t target = 7LL * (cfg->num_sms ? cfg->num_sms : 148) / 2;
-        int32_t C = 64;
-        while (C > 4 && decode_item_count(pages_per_block, cfg->num_kv_heads, C) < target) C /= 2;
-        p->C = C;
+        const int64_t slots = 2LL * (cfg->num_sms ? cfg->num_sms : 148);
+        int64_t items = (int64_t)B * cfg->num_kv_heads;
+        while (items + cfg->num_kv_heads <= slots) {
+            int32_t best = -1;
+            int32_t best_size = 4;  // never split below 4 pages
+            for (int32_t b = 0; b < B; ++b) {
+                const int32_t size = (pages_per_block[b] + n_splits[b] - 1) / n_splits[b];
+                if (size > best_size) { best_size = size; best = b; }
+            }
+            if (best < 0) break;
+            ++n_splits[best];
+            items += cfg->num_kv_heads;
+        }
+        for (int32_t b = 0; b < B; ++b) {
+            int32_t size = (pages_per_block[b] + n_splits[b] - 1) / n_splits[b];
+            p->split_pages[b] = std::min(size, kMaxSplitPages);
+        }
     }
+    p->C = *std::max_element(p->split_pages.begin(), p->split_pages.end());
     struct DItem { int32_t pages, block, head, split; };
     std::vector<DItem> dit;
     p->split_indptr.assign(B + 1, 0);
     for (int32_t b = 0; b < B; ++b) {
-        int32_t n_splits = (pages_per_block[b] + p->C - 1) / p->C;
-        p->split_indptr[b + 1] = p->split_indptr[b] + n_splits;
+        const int32_t Cb = p->split_pages[b];
+        const int32_t ns = (pages_per_block[b] + Cb - 1) / Cb;
+        p->split_indptr[b + 1] = p->split_indptr[b] + ns;
         for (int32_t g = 0; g < cfg->num_kv_heads; ++g)
-            for (int32_t s = 0; s < n_splits; ++s)
-                dit.push_back({std::min(p->C, pages_per_block[b] - s * p->C), b, g, s});
+            for (int32_t s = 0; s < ns; ++s)
+                dit.push_back({std::min(Cb, pages_per_block[b] - s * Cb), b, g, s});
     }
     std::stable_sort(dit.begin(), dit.end(), [](const DItem& a, const DItem& c) {
         if (a.pages != c.pages) return a.pages > c.pages;
@@ -138,7 +153,7 @@ extern "C" int cpa_plan_create(const cpa_config* cfg, int32_t num_blocks, const 
     p->off_append = w;  w = align4(w + B + 1);
     p->off_pidx = w;    w = align4(w + pages_used);
     p->off_pitems = w;  w = align4(w + 2LL * p->n_prefill);
-    p->item_stride = 4 + (p->C + 3) / 4 * 4;
+    p->item_stride = 8 + (p->C + 3) / 4 * 4;
     p->off_ditems = w;  w = align4(w + (int64_t)p->item_stride * p->n_decode);
     p->off_tickets = w; w = align4(w + (int64_t)B * cfg->num_kv_heads);
     p->words = w;
@@ -157,8 +172,10 @@ extern "C" int cpa_plan_create(const cpa_config* cfg, int32_t num_blocks, const 
         it[1] = dit[i].head;
         it[2] = dit[i].split;
         it[3] = dit[i].pages;
-        const int32_t* src = p->page_indices.data() + p->page_indptr[dit[i].block] + dit[i].split * p->C;
-        for (int32_t j = 0; j < dit[i].pages; ++j) it[4 + j] = src[j];
+        it[4] = p->split_pages[dit[i].block];
+        const int32_t* src = p->page_indices.data() + p->page_indptr[dit[i].block] +
+                             dit[i].split * p->split_pages[dit[i].block];
+        for (int32_t j = 0; j < dit[i].pages; ++j) it[8 + j] = src[j];
     }
     p->append_stage.assign(B + 1, 0);
     *out = p;
@@ -178,6 +195,7 @@ extern "C" int cpa_plan_export(const cpa_plan* plan, int which, const int32_t** 
         case CPA_ARR_PREFILL_ITEMS: v = &plan->prefill_items; div = 2; break;
         case CPA_ARR_DECODE_ITEMS: v = &plan->decode_items; div = 3; break;
         case CPA_ARR_SPLIT_INDPTR: v = &plan->split_indptr; break;
+        case CPA_ARR_SPLIT_PAGES: v = &plan->split_pages; break;
         default: return CPA_EINVAL;
     }
     *ptr = v->data();
