@@ -156,6 +156,18 @@ CPA_API int cpa_prefill(const cpa_plan* plan, const void* q, const void* k, cons
                 void* d_workspace, void* stream);
 
 /*
+ * cpa_prefill_variant -- cpa_prefill with the kernel chosen by the caller; for
+ * cross-checking one kernel against the other on the device and for profiling.
+ * (The paper has no counterpart.)  Same arguments, layouts and errors as
+ * cpa_prefill; CPA_EINVAL for an unknown variant.
+ *   CPA_PREFILL_TENSOR_CORE  TMA-staged tiles, tcgen05 MMAs, accumulators in TMEM
+ *   CPA_PREFILL_WARP_MMA     warp-level mma.sync kernel (the earlier, slower design)
+ */
+enum { CPA_PREFILL_TENSOR_CORE = 0, CPA_PREFILL_WARP_MMA = 1 };
+CPA_API int cpa_prefill_variant(const cpa_plan* plan, const void* q, const void* k, const void* v, void* o,
+                                void* stream, int variant);
+
+/*
  * cpa_kv_append -- write new K/V rows into the blocks' pages and advance
  * seq_lens (the KV cache each sequence keeps while it decodes its summary).
  *   k_new, v_new : device bf16 [sum(new_lens), num_kv_heads, head_dim], block-major

@@ -63,6 +63,8 @@ _lib.cpa_plan_destroy.argtypes = [_vp]
 _lib.cpa_plan_destroy.restype = None
 _lib.cpa_prefill.argtypes = [_vp, _vp, _vp, _vp, _vp, _vp, _vp]
 _lib.cpa_prefill.restype = ctypes.c_int
+_lib.cpa_prefill_variant.argtypes = [_vp, _vp, _vp, _vp, _vp, _vp, ctypes.c_int]
+_lib.cpa_prefill_variant.restype = ctypes.c_int
 _lib.cpa_kv_append.argtypes = [_vp, _vp, _vp, _i32p, _vp, _vp, _vp]
 _lib.cpa_kv_append.restype = ctypes.c_int
 _lib.cpa_decode.argtypes = [_vp, _vp, _vp, _vp, _vp, _vp, _vp]
@@ -136,6 +138,13 @@ def cpa_plan_destroy(plan: int) -> None:
 
 def cpa_prefill(plan: int, q, k, v, o, d_workspace=None, stream: int = 0) -> int:
     return _lib.cpa_prefill(plan, _ptr(q), _ptr(k), _ptr(v), _ptr(o), _ptr(d_workspace), stream or None)
+
+
+PREFILL_TENSOR_CORE, PREFILL_WARP_MMA = 0, 1
+
+
+def cpa_prefill_variant(plan: int, q, k, v, o, stream: int = 0, variant: int = 0) -> int:
+    return _lib.cpa_prefill_variant(plan, _ptr(q), _ptr(k), _ptr(v), _ptr(o), stream or None, int(variant))
 
 
 def cpa_kv_append(plan: int, k_new, v_new, new_lens, k_pool, v_pool, stream: int = 0) -> int:

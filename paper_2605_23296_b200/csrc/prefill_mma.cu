@@ -262,12 +262,21 @@ int cpa_prefill_mma(const cpa_plan* plan, const void* q, const void* k, const vo
                                      : launch_prefill_mma<64>(plan, q, k, v, o, st);
 }
 
-extern "C" int cpa_prefill(const cpa_plan* plan, const void* q, const void* k, const void* v, void* o,
-                           void* d_workspace, void* stream) {
-    (void)d_workspace;
+int cpa_prefill_tc(const cpa_plan* plan, const void* q, const void* k, const void* v, void* o, void* stream);
+
+extern "C" int cpa_prefill_variant(const cpa_plan* plan, const void* q, const void* k, const void* v, void* o,
+                                   void* stream, int variant) {
     if (!plan || !q || !k || !v || !o) return CPA_EINVAL;
     if (!cpa_aligned16(q) || !cpa_aligned16(k) || !cpa_aligned16(v) || !cpa_aligned16(o)) return CPA_EINVAL;
     if (o == q || o == k || o == v) return CPA_EINVAL;
     if (!plan->d_base) return CPA_ESTATE;
-    return cpa_prefill_mma(plan, q, k, v, o, stream);
+    if (variant == CPA_PREFILL_TENSOR_CORE) return cpa_prefill_tc(plan, q, k, v, o, stream);
+    if (variant == CPA_PREFILL_WARP_MMA) return cpa_prefill_mma(plan, q, k, v, o, stream);
+    return CPA_EINVAL;
+}
+
+extern "C" int cpa_prefill(const cpa_plan* plan, const void* q, const void* k, const void* v, void* o,
+                           void* d_workspace, void* stream) {
+    (void)d_workspace;
+    return cpa_prefill_variant(plan, q, k, v, o, stream, CPA_PREFILL_TENSOR_CORE);
 }

@@ -78,11 +78,15 @@ class CompactionSession:
 
     # -- the hot path -------------------------------------------------------
     def prefill(self, q: torch.Tensor, k: torch.Tensor, v: torch.Tensor,
-                out: Optional[torch.Tensor] = None) -> torch.Tensor:
+                out: Optional[torch.Tensor] = None, variant: Optional[int] = None) -> torch.Tensor:
         """Causal attention of every block over itself; q/out [tokens,Hq,d], k/v [tokens,Hkv,d]."""
         if out is None:
             out = torch.empty_like(q)
-        self._check(B.cpa_prefill(self.plan, q, k, v, out, None, self._stream()), "cpa_prefill")
+        if variant is None:
+            self._check(B.cpa_prefill(self.plan, q, k, v, out, None, self._stream()), "cpa_prefill")
+        else:
+            self._check(B.cpa_prefill_variant(self.plan, q, k, v, out, self._stream(), variant),
+                        "cpa_prefill_variant")
         return out
 
     def append_prefill(self, k: torch.Tensor, v: torch.Tensor) -> None:

@@ -156,6 +156,21 @@ def test_prefill_does_not_write_outside_its_rows():
     s.close()
 
 
+def test_prefill_kernels_agree_with_each_other():
+    # the tensor-core (tcgen05/TMEM) kernel and the warp-MMA kernel, both against the oracle
+    from paper_2605_23296_b200 import binding as B
+    w = wl.custom([700, 129, 1, 384], 8, 2, 128, steps=0, seed=17).materialise()
+    s = _session(w)
+    q, k, v = _dev(w.q), _dev(w.k), _dev(w.v)
+    want = oa.prefill(w.q, w.k, w.v, _cu(w), w.scale)
+    for variant in (B.PREFILL_TENSOR_CORE, B.PREFILL_WARP_MMA):
+        o = s.prefill(q, k, v, variant=variant)
+        assert s.status() == 0
+        assert_attention_close(_bits(o), want, f"variant {variant}")
+    assert B.cpa_prefill_variant(s.plan, q, k, v, o, 0, 7) == B.CPA_EINVAL
+    s.close()
+
+
 def test_prefill_outlier_keys():
     w = wl.dense8b(seed=21, num_blocks=3, block_len=700, steps=0)
     _check_prefill(w, what="outlier")
