@@ -64,7 +64,7 @@ typedef struct cpa_config {
     int32_t head_dim;        /* 64 or 128 */
     int32_t page_size;       /* 16 */
     float   scale;           /* softmax scale, normally 1/sqrt(head_dim) */
-    int32_t q_tile_rows;     /* query rows per prefill work item; 0 = default (128) */
+    int32_t q_tile_rows;     /* query rows per prefill work item: 128 or 256; 0 = default (256) */
     int32_t pages_per_split; /* KV pages per decode work item (<= 1024); 0 = chosen per block from the batch */
     int32_t num_sms;         /* SM count the split heuristic aims at; 0 = 148 */
 } cpa_config;

@@ -30,7 +30,7 @@ extern "C" int cpa_plan_create(const cpa_config* cfg, int32_t num_blocks, const 
     if ((cfg->head_dim != 64 && cfg->head_dim != 128) || cfg->page_size != 16 ||
         cfg->num_q_heads / cfg->num_kv_heads > 8)
         return CPA_EUNSUPPORTED;
-    if (cfg->q_tile_rows != 0 && cfg->q_tile_rows != 128) return CPA_EUNSUPPORTED;
+    if (cfg->q_tile_rows != 0 && cfg->q_tile_rows != 128 && cfg->q_tile_rows != 256) return CPA_EUNSUPPORTED;
     if (cfg->pages_per_split > kMaxSplitPages) return CPA_EUNSUPPORTED;
 
     cpa_plan* p = new (std::nothrow) cpa_plan();
@@ -38,7 +38,7 @@ extern "C" int cpa_plan_create(const cpa_config* cfg, int32_t num_blocks, const 
     p->cfg = *cfg;
     p->B = num_blocks;
     p->T = max_new_tokens;
-    p->q_tile = cfg->q_tile_rows ? cfg->q_tile_rows : 128;
+    p->q_tile = cfg->q_tile_rows ? cfg->q_tile_rows : 256;
     const int32_t P = cfg->page_size;
     const int32_t B = num_blocks;
 

@@ -69,7 +69,7 @@ template <int D>
 __global__ void __launch_bounds__(kPrefillThreads, 1)
 prefill_mma_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ k,
                    const __nv_bfloat16* __restrict__ v, __nv_bfloat16* __restrict__ o, cpa_dev_index ix,
-                   int Hq, int Hkv, float scale_log2) {
+                   int Hq, int Hkv, int subs, float scale_log2) {
     extern __shared__ __align__(128) unsigned char smem_raw[];
     constexpr int KSTEPS = D / 16;   // k-steps of the QK^T contraction
     constexpr int NT_S = kKVTile / 8;  // 8-key n-tiles of S
@@ -78,11 +78,14 @@ prefill_mma_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __r
     const uint32_t s_k = s_q + kQTile * D * 2;
     const uint32_t s_v = s_k + 2 * kKVTile * D * 2;
 
-    const int b = ix.prefill_items[2 * blockIdx.x], tile = ix.prefill_items[2 * blockIdx.x + 1];
+    // a work item of subs*128 query rows is covered by `subs` CTAs of 128 rows each
+    const int item = blockIdx.x / subs;
+    const int b = ix.prefill_items[2 * item], tile = ix.prefill_items[2 * item + 1] * subs + (blockIdx.x - item * subs);
     const int h = blockIdx.y, g = h / (Hq / Hkv);
     const int tok0 = ix.cu_seqlens[b];
     const int L = ix.cu_seqlens[b + 1] - tok0;
     const int q0 = tile * kQTile;
+    if (q0 >= L) return;
     const int q_rows = min(kQTile, L - q0);
     const int kv_end = q0 + q_rows;  // keys visible to the tile's last row
     const int n_tiles = (kv_end + kKVTile - 1) / kKVTile;
@@ -247,10 +250,11 @@ int launch_prefill_mma(const cpa_plan* plan, const void* q, const void* k, const
         }
         configured = true;
     }
-    dim3 grid(plan->n_prefill, c.num_q_heads);
+    const int subs = plan->q_tile / kQTile;
+    dim3 grid(plan->n_prefill * subs, c.num_q_heads);
     prefill_mma_kernel<D><<<grid, kPrefillThreads, smem, st>>>(
         (const __nv_bfloat16*)q, (const __nv_bfloat16*)k, (const __nv_bfloat16*)v, (__nv_bfloat16*)o, plan->dev(),
-        c.num_q_heads, c.num_kv_heads, c.scale * 1.4426950408889634f);
+        c.num_q_heads, c.num_kv_heads, subs, c.scale * 1.4426950408889634f);
     return cudaGetLastError() == cudaSuccess ? CPA_OK : CPA_ECUDA;
 }
 

@@ -2,20 +2,22 @@
 // cores: TMA-staged tiles, tcgen05.mma with accumulators in tensor memory (TMEM), online
 // softmax in fp32 registers.
 //
-// One CTA = one (block, q_tile of 128 rows, query head) item; 6 warps with fixed roles:
-//   warps 0-3  softmax + epilogue: thread r owns query row r (TMEM lane r), so row max and
-//              row sum need no shuffles
-//   warp 4     TMA producer (one elected lane): Q once, then K and V tiles of 128 keys
-//              through two-stage rings
-//   warp 5     MMA issuer (one elected lane) and owner of the TMEM allocation
-// TMEM columns: S0 [0,128), S1 [128,256) (fp32 scores, double buffered), O [256,256+D).
-// Per KV tile j:   S[j&1] = Q K_j^T          (SS MMA, both operands K-major in smem)
-//                  P_j    = exp2(scale*S - m) (registers -> bf16 -> swizzled smem)
-//                  O     += P_j V_j           (A = P K-major, B = V MN-major)
-// The issuer runs QK(j+1) ahead of PV(j), so the tensor core works on the next scores while
-// the softmax warps work on the current ones.  O stays in TMEM across tiles; it is rescaled
-// only when a row's running max grows by more than 2^8 (the stale max is used meanwhile,
-// which is exact after the final division by the row sum).
+// One CTA = one (block, q item, query head); a q item is 256 query rows handled as two
+// 128-row sub-tiles that share every K/V tile.  Ten warps with fixed roles:
+//   warps 0-3  softmax + epilogue of sub-tile 0: thread r owns query row r (TMEM lane r), so
+//   warps 4-7  ... of sub-tile 1                 row max and row sum need no shuffles
+//   warp 8     TMA producer (one elected lane): both Q sub-tiles once, then K and V tiles of
+//              128 keys through two-stage rings
+//   warp 9     MMA issuer (one elected lane) and owner of the TMEM allocation
+// TMEM columns: S_u at u*128 (fp32 scores of sub-tile u), O_u at 256 + u*128.
+// Per KV tile j and sub-tile u:
+//                  S_u  = Q_u K_j^T            (both operands K-major in shared memory)
+//                  P_u  = exp2(scale*S_u - m)  (registers -> bf16 -> TMEM, over S_u's first 64 columns)
+//                  O_u += P_u V_j              (A = P_u from TMEM, B = V MN-major in shared memory)
+// The issuer alternates the sub-tiles: PV_0(j), QK_0(j+1), PV_1(j), QK_1(j+1), ... so while
+// one warpgroup does its softmax the tensor core runs the other sub-tile's MMAs.  O stays in
+// TMEM across tiles; it is rescaled only when a row's running max grows by more than 2^8
+// (the stale max is used meanwhile, which is exact after the final division by the row sum).
 //
 // Shared-memory tiles use the 128-byte swizzle that both TMA and the MMA descriptors
 // understand: a tile is a set of column blocks of 64 bf16 (128 B) x rows, rows 128 B apart,
@@ -33,7 +35,7 @@ namespace {
 
 constexpr int kTileM = 128;        // query rows per CTA
 constexpr int kTileN = 128;        // keys per KV tile
-constexpr int kThreads = 192;
+constexpr int kThreads = 320;
 constexpr uint32_t kSpinLimit = 1u << 20;
 constexpr uint32_t kBlockBytes = 128 * 128;   // one column block: 128 rows x 128 B
 
@@ -140,58 +142,88 @@ __host__ __device__ constexpr uint32_t instr_desc(int M, int N, bool b_mn_major)
            ((uint32_t)(M >> 4) << 24);
 }
 
+// D[tmem] (+)= A[tmem] * B[smem desc]: A is a 128-lane x 16-element bf16 slice held in TMEM
+// (two consecutive K elements per 32-bit column, row = lane).
+__device__ __forceinline__ void tc_mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n"
+        " tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n}\n"
+        :: "r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
+// 32 consecutive 32-bit columns of this thread's TMEM lane, no wait (pair with tc_wait_ld).
+__device__ __forceinline__ void tc_ld32_nowait(uint32_t taddr, uint32_t (&r)[32]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
+        "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];\n"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+          "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+          "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;\n" ::: "memory"); }
+__device__ __forceinline__ void tc_st16(uint32_t taddr, const uint32_t* v) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};\n"
+        :: "r"(taddr), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]),
+           "r"(v[8]), "r"(v[9]), "r"(v[10]), "r"(v[11]), "r"(v[12]), "r"(v[13]), "r"(v[14]), "r"(v[15])
+        : "memory");
+}
+__device__ __forceinline__ void wg_sync(int id) { asm volatile("bar.sync %0, 128;\n" :: "r"(id) : "memory"); }
+
 struct __align__(8) TcBarriers {
-    uint64_t q_full, k_full[2], k_empty[2], v_full[2], v_empty[2], s_full[2], s_empty[2], p_full, pv_done;
+    uint64_t q_full[2], k_full[2], k_empty[2], v_full[2], v_empty[2], s_full[2], p_full[2], pv_done[2];
     uint32_t tmem_base;
 };
 
+// One CTA = one (block, q item of `q_rows` = 128 or 256 rows, query head).  A 256-row item is
+// two 128-row sub-tiles u = 0, 1 that share every K/V tile; sub-tile u has its own softmax
+// warpgroup, its own S_u / O_u columns in TMEM, and sees KV tiles 0 .. t0+u (t0 = index of
+// sub-tile 0 in units of 128 rows; the last of them touches the diagonal).
 template <int D>
 __global__ void __launch_bounds__(kThreads, 1)
 prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                   const __grid_constant__ CUtensorMap tm_v, __nv_bfloat16* __restrict__ o, cpa_dev_index ix, int Hq,
-                  int Hkv, float scale_log2) {
+                  int Hkv, int q_rows, float scale_log2) {
     constexpr int NB = D / 64;                         // 64-wide column blocks of a Q/K/V tile
-    constexpr uint32_t kTileBytes = NB * kBlockBytes;  // one Q, K or V tile
+    constexpr uint32_t kTileBytes = NB * kBlockBytes;  // one Q sub-tile, K tile or V tile
     constexpr uint32_t kTmemCols = 512;
-    constexpr uint32_t kColS0 = 0, kColO = 256;
+    constexpr uint32_t kColO = 256;                    // S_u at u*128 (P_u aliases its first 64 columns), O_u at 256 + u*128
     extern __shared__ unsigned char dsm_raw[];
     __shared__ TcBarriers bars;
 
     const uint32_t base = (smem_u32(dsm_raw) + 1023u) & ~1023u;
-    const uint32_t s_q = base;
-    const uint32_t s_k = s_q + kTileBytes;           // two stages
+    const uint32_t s_q = base;                       // two sub-tiles
+    const uint32_t s_k = s_q + 2 * kTileBytes;       // two stages
     const uint32_t s_v = s_k + 2 * kTileBytes;       // two stages
-    const uint32_t s_p = s_v + 2 * kTileBytes;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int b = ix.prefill_items[2 * blockIdx.x], tile = ix.prefill_items[2 * blockIdx.x + 1];
+    const int b = ix.prefill_items[2 * blockIdx.x], item = ix.prefill_items[2 * blockIdx.x + 1];
     const int h = blockIdx.y, g = h / (Hq / Hkv);
     const int tok0 = ix.cu_seqlens[b];
     const int L = ix.cu_seqlens[b + 1] - tok0;
-    const int q0 = tile * kTileM;
-    const int n_tiles = tile + 1;  // KV tiles 0..tile; only the last one touches the diagonal
+    const int q0 = item * q_rows;
+    const int t0 = q0 / kTileM;
+    const int n_sub = (q_rows > kTileM && L - q0 > kTileM) ? 2 : 1;
+    const int n_total = t0 + n_sub;                  // KV tiles the CTA streams; sub-tile u uses the first t0+1+u
 
-    const uint32_t b_q_full = smem_u32(&bars.q_full), b_p_full = smem_u32(&bars.p_full), b_pv_done = smem_u32(&bars.pv_done);
-    const uint32_t b_k_full = smem_u32(&bars.k_full[0]), b_k_empty = smem_u32(&bars.k_empty[0]);
-    const uint32_t b_v_full = smem_u32(&bars.v_full[0]), b_v_empty = smem_u32(&bars.v_empty[0]);
-    const uint32_t b_s_full = smem_u32(&bars.s_full[0]), b_s_empty = smem_u32(&bars.s_empty[0]);
+    auto bar = [&](uint64_t* p) { return smem_u32(p); };
 
     if (threadIdx.x == 0) {
-        mbar_init(b_q_full, 1);
-        mbar_init(b_p_full, 128);
-        mbar_init(b_pv_done, 1);
-        for (int s = 0; s < 2; ++s) {
-            mbar_init(b_k_full + 8 * s, 1);
-            mbar_init(b_k_empty + 8 * s, 1);
-            mbar_init(b_v_full + 8 * s, 1);
-            mbar_init(b_v_empty + 8 * s, 1);
-            mbar_init(b_s_full + 8 * s, 1);
-            mbar_init(b_s_empty + 8 * s, 128);
+        for (int u = 0; u < 2; ++u) {
+            mbar_init(bar(&bars.q_full[u]), 1);
+            mbar_init(bar(&bars.k_full[u]), 1);
+            mbar_init(bar(&bars.k_empty[u]), 1);
+            mbar_init(bar(&bars.v_full[u]), 1);
+            mbar_init(bar(&bars.v_empty[u]), 1);
+            mbar_init(bar(&bars.s_full[u]), 1);
+            mbar_init(bar(&bars.p_full[u]), 128);
+            mbar_init(bar(&bars.pv_done[u]), 1);
         }
         asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory");
     }
-    if (warp == 5) {  // TMEM allocation is warp-wide
+    if (warp == 9) {  // TMEM allocation is warp-wide
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;\n"
                      :: "r"(smem_u32(&bars.tmem_base)), "r"(kTmemCols) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;\n" ::: "memory");
@@ -202,97 +234,118 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
     const uint32_t tmem = bars.tmem_base;
     bool dead = false;
 
-    if (warp == 4) {
+    if (warp == 8) {
         // ------------------------------------------------------------ TMA producer
         if (lane == 0) {
-            mbar_expect_tx(b_q_full, kTileBytes);
+            for (int u = 0; u < n_sub; ++u) {
+                mbar_expect_tx(bar(&bars.q_full[u]), kTileBytes);
 #pragma unroll
-            for (int c = 0; c < NB; ++c) tma_load_2d(s_q + c * kBlockBytes, &tm_q, h * D + 64 * c, tok0 + q0, b_q_full);
-            for (int j = 0; j < n_tiles; ++j) {
+                for (int c = 0; c < NB; ++c)
+                    tma_load_2d(s_q + u * kTileBytes + c * kBlockBytes, &tm_q, h * D + 64 * c, tok0 + q0 + u * kTileM,
+                                bar(&bars.q_full[u]));
+            }
+            for (int j = 0; j < n_total; ++j) {
                 const int s = j & 1;
                 const uint32_t par = (uint32_t)(j >> 1) & 1u;
                 const int row = tok0 + j * kTileN;
-                mbar_wait(b_k_empty + 8 * s, par ^ 1u, dead, ix.status);
-                mbar_expect_tx(b_k_full + 8 * s, kTileBytes);
+                mbar_wait(bar(&bars.k_empty[s]), par ^ 1u, dead, ix.status);
+                mbar_expect_tx(bar(&bars.k_full[s]), kTileBytes);
 #pragma unroll
                 for (int c = 0; c < NB; ++c)
-                    tma_load_2d(s_k + s * kTileBytes + c * kBlockBytes, &tm_k, g * D + 64 * c, row, b_k_full + 8 * s);
-                mbar_wait(b_v_empty + 8 * s, par ^ 1u, dead, ix.status);
-                mbar_expect_tx(b_v_full + 8 * s, kTileBytes);
+                    tma_load_2d(s_k + s * kTileBytes + c * kBlockBytes, &tm_k, g * D + 64 * c, row, bar(&bars.k_full[s]));
+                mbar_wait(bar(&bars.v_empty[s]), par ^ 1u, dead, ix.status);
+                mbar_expect_tx(bar(&bars.v_full[s]), kTileBytes);
 #pragma unroll
                 for (int c = 0; c < NB; ++c)
-                    tma_load_2d(s_v + s * kTileBytes + c * kBlockBytes, &tm_v, g * D + 64 * c, row, b_v_full + 8 * s);
+                    tma_load_2d(s_v + s * kTileBytes + c * kBlockBytes, &tm_v, g * D + 64 * c, row, bar(&bars.v_full[s]));
             }
         }
-    } else if (warp == 5) {
+    } else if (warp == 9) {
         // ------------------------------------------------------------ MMA issuer
         if (lane == 0) {
             constexpr uint32_t idesc_qk = instr_desc(kTileM, kTileN, false);
             constexpr uint32_t idesc_pv = instr_desc(kTileM, D, true);
-            auto issue_qk = [&](int j) {
+            auto issue_qk = [&](int u, int j) {   // S_u = Q_u K_j^T
                 const int s = j & 1;
-                const uint32_t par = (uint32_t)(j >> 1) & 1u;
-                mbar_wait(b_k_full + 8 * s, par, dead, ix.status);
-                mbar_wait(b_s_empty + 8 * s, par ^ 1u, dead, ix.status);
-                tc_fence_after();
 #pragma unroll
                 for (int k = 0; k < D / 16; ++k) {
                     // 16 head dims per instruction: 32 B inside the 128-B swizzled row, next block after 4 steps
                     const uint32_t off = (k >> 2) * kBlockBytes + (k & 3) * 32;
-                    tc_mma_ss(tmem + kColS0 + s * 128, smem_desc(s_q + off, 16, 1024),
+                    tc_mma_ss(tmem + u * 128, smem_desc(s_q + u * kTileBytes + off, 16, 1024),
                               smem_desc(s_k + s * kTileBytes + off, 16, 1024), idesc_qk, k > 0);
                 }
-                tc_commit(b_k_empty + 8 * s);
-                tc_commit(b_s_full + 8 * s);
+                tc_commit(bar(&bars.s_full[u]));
             };
-            auto issue_pv = [&](int j) {
+            auto issue_pv = [&](int u, int j) {   // O_u += P_u V_j, P_u read from TMEM (aliases S_u)
                 const int s = j & 1;
-                mbar_wait(b_v_full + 8 * s, (uint32_t)(j >> 1) & 1u, dead, ix.status);
-                mbar_wait(b_p_full, (uint32_t)j & 1u, dead, ix.status);
-                tc_fence_after();
 #pragma unroll
-                for (int k = 0; k < kTileN / 16; ++k) {
-                    // A = P: 16 keys per step (32 B inside the row, next column block after 4 steps)
-                    // B = V: 16 keys per step = 16 rows of 128 B; column blocks kBlockBytes apart
-                    const uint32_t a_off = (k >> 2) * kBlockBytes + (k & 3) * 32;
-                    tc_mma_ss(tmem + kColO, smem_desc(s_p + a_off, 16, 1024),
+                for (int k = 0; k < kTileN / 16; ++k)
+                    // 16 keys per instruction: 8 TMEM columns of A; 16 rows of 128 B of V, column blocks kBlockBytes apart
+                    tc_mma_ts(tmem + kColO + u * 128, tmem + u * 128 + k * 8,
                               smem_desc(s_v + s * kTileBytes + k * 2048, kBlockBytes, 1024), idesc_pv, (j > 0 || k > 0));
-                }
-                tc_commit(b_v_empty + 8 * s);
-                tc_commit(b_pv_done);
             };
-            mbar_wait(b_q_full, 0, dead, ix.status);
-            for (int j = 0; j < n_tiles; ++j) {
-                issue_qk(j);
-                if (j > 0) issue_pv(j - 1);
+            // MMAs issued by this one thread execute in issue order, so QK_u(j+1) may be queued right
+            // behind PV_u(j) although it overwrites the columns PV_u(j) reads P_u from.
+            mbar_wait(bar(&bars.k_full[0]), 0, dead, ix.status);
+            for (int u = 0; u < n_sub; ++u) {
+                mbar_wait(bar(&bars.q_full[u]), 0, dead, ix.status);
+                tc_fence_after();
+                issue_qk(u, 0);
             }
-            issue_pv(n_tiles - 1);
+            tc_commit(bar(&bars.k_empty[0]));
+            for (int j = 0; j < n_total; ++j) {
+                const int s = j & 1;
+                bool have_v = false, have_k = false;
+                for (int u = 0; u < n_sub; ++u) {
+                    const int n_kv = t0 + 1 + u;
+                    if (j < n_kv) {
+                        if (!have_v) { mbar_wait(bar(&bars.v_full[s]), (uint32_t)(j >> 1) & 1u, dead, ix.status); have_v = true; }
+                        mbar_wait(bar(&bars.p_full[u]), (uint32_t)j & 1u, dead, ix.status);
+                        tc_fence_after();
+                        issue_pv(u, j);
+                        if (j == n_kv - 1) tc_commit(bar(&bars.pv_done[u]));
+                    }
+                    if (j + 1 < n_kv) {
+                        if (!have_k) {
+                            mbar_wait(bar(&bars.k_full[s ^ 1]), (uint32_t)((j + 1) >> 1) & 1u, dead, ix.status);
+                            tc_fence_after();
+                            have_k = true;
+                        }
+                        issue_qk(u, j + 1);
+                    }
+                }
+                tc_commit(bar(&bars.v_empty[s]));
+                if (j + 1 < n_total) tc_commit(bar(&bars.k_empty[s ^ 1]));
+            }
         }
-    } else {
-        // ------------------------------------------------------------ softmax + epilogue (128 threads)
-        const int r = threadIdx.x;                                   // query row inside the tile = TMEM lane
-        const uint32_t lane_addr = ((uint32_t)(warp * 32) << 16);    // this warp's 32 TMEM lanes
-        const uint32_t p_row = s_p + r * 128;
+    } else if (warp < 4 * n_sub) {
+        // ------------------------------------------------------------ softmax + epilogue (one warpgroup per sub-tile)
+        const int u = warp >> 2;
+        const int r = threadIdx.x & 127;                                  // query row inside the sub-tile = TMEM lane
+        const uint32_t lane_addr = ((uint32_t)((warp & 3) * 32) << 16);   // this warp's 32 TMEM lanes
+        const uint32_t t_s = tmem + lane_addr + u * 128;
+        const uint32_t t_o = tmem + lane_addr + kColO + u * 128;
+        const int n_kv = t0 + 1 + u;
         float m_used = -INFINITY;   // row max the weights are currently scaled with (log2 units)
         float l_run = 0.f;
-        for (int j = 0; j < n_tiles; ++j) {
-            const int s = j & 1;
-            mbar_wait(b_s_full + 8 * s, (uint32_t)(j >> 1) & 1u, dead, ix.status);
+        for (int j = 0; j < n_kv; ++j) {
+            // s_full(j) also means PV_u(j-1) has completed (the commit covers every earlier MMA):
+            // O_u is settled and the P_u columns may be overwritten
+            mbar_wait(bar(&bars.s_full[u]), (uint32_t)j & 1u, dead, ix.status);
             tc_fence_after();
-            const uint32_t t_s = tmem + lane_addr + kColS0 + s * 128;
-            const bool diag = (j == n_tiles - 1);
-            // pass 1: row max of this tile
+            const bool diag = (j == n_kv - 1);
+            uint32_t sv[4][32];
+#pragma unroll
+            for (int c = 0; c < 4; ++c) tc_ld32_nowait(t_s + c * 32, sv[c]);
+            tc_wait_ld();
             float mx = -INFINITY;
 #pragma unroll
-            for (int c = 0; c < 4; ++c) {
-                float v[32];
-                tc_ld32(t_s + c * 32, v);
+            for (int c = 0; c < 4; ++c)
 #pragma unroll
                 for (int i = 0; i < 32; ++i) {
-                    const bool masked = diag && (c * 32 + i > r);
-                    mx = fmaxf(mx, masked ? -INFINITY : v[i]);
+                    if (diag && (c * 32 + i > r)) sv[c][i] = 0xff800000u;   // -inf: key is in the row's future
+                    mx = fmaxf(mx, __uint_as_float(sv[c][i]));
                 }
-            }
             mx *= scale_log2;       // scale > 0, so the max commutes with the scaling
             // lazy rescale: keep the old reference max unless the new one is more than 2^8 above it
             float alpha = 1.f;
@@ -300,83 +353,79 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                 alpha = (m_used == -INFINITY) ? 0.f : exp2f(m_used - mx);
                 m_used = mx;
             }
-            // P of the previous tile must have been consumed (and O settled) before P is overwritten
-            if (j > 0) {
-                mbar_wait(b_pv_done, (uint32_t)(j - 1) & 1u, dead, ix.status);
-                tc_fence_after();
-            }
-            const bool rescale = __any_sync(0xffffffffu, alpha != 1.f) && j > 0;
-            if (rescale) {
+            if (j > 0 && __any_sync(0xffffffffu, alpha != 1.f)) {
 #pragma unroll
                 for (int c = 0; c < D / 32; ++c) {
                     float v[32];
-                    tc_ld32(tmem + lane_addr + kColO + c * 32, v);
+                    tc_ld32(t_o + c * 32, v);
 #pragma unroll
                     for (int i = 0; i < 32; ++i) v[i] *= alpha;
-                    tc_st32(tmem + lane_addr + kColO + c * 32, v);
+                    tc_st32(t_o + c * 32, v);
                 }
-                tc_wait_st();
             }
             l_run *= alpha;
-            // pass 2: weights, rounded to bf16, written K-major into the swizzled P tile
+            // weights, rounded to bf16, two keys per 32-bit TMEM column (P_u over the first 64 columns of S_u)
             float sum = 0.f;
 #pragma unroll
             for (int c = 0; c < 4; ++c) {
-                float v[32];
-                tc_ld32(t_s + c * 32, v);
                 uint32_t pk[16];
 #pragma unroll
                 for (int i = 0; i < 32; i += 2) {
-                    const bool m0 = diag && (c * 32 + i > r), m1 = diag && (c * 32 + i + 1 > r);
-                    const float p0 = m0 ? 0.f : exp2f(fmaf(v[i], scale_log2, -m_used));
-                    const float p1 = m1 ? 0.f : exp2f(fmaf(v[i + 1], scale_log2, -m_used));
+                    const float p0 = exp2f(fmaf(__uint_as_float(sv[c][i]), scale_log2, -m_used));
+                    const float p1 = exp2f(fmaf(__uint_as_float(sv[c][i + 1]), scale_log2, -m_used));
                     const uint32_t w = pack_bf16(p0, p1);
                     pk[i >> 1] = w;
                     // row sum over the rounded weights: numerator and denominator stay consistent
                     sum += __uint_as_float(w << 16) + __uint_as_float(w & 0xffff0000u);
                 }
-#pragma unroll
-                for (int q4 = 0; q4 < 4; ++q4) {
-                    const int chunk = c * 4 + q4;            // 16-byte chunk (8 keys) of this row: 0..15
-                    const uint32_t addr = p_row + (chunk >> 3) * kBlockBytes + (((chunk & 7) ^ (r & 7)) << 4);
-                    asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};\n"
-                                 :: "r"(addr), "r"(pk[4 * q4]), "r"(pk[4 * q4 + 1]), "r"(pk[4 * q4 + 2]), "r"(pk[4 * q4 + 3]) : "memory");
-                }
+                tc_st16(t_s + c * 16, pk);
             }
             l_run += sum;
-            // S[s] may be overwritten by QK(j+2); P is ready for PV(j)
+            tc_wait_st();
             tc_fence_before();
-            mbar_arrive(b_s_empty + 8 * s);
-            asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory");
-            mbar_arrive(b_p_full);
+            mbar_arrive(bar(&bars.p_full[u]));
         }
-        // ---- epilogue: O / l, rows past the end of the block are never stored
-        mbar_wait(b_pv_done, (uint32_t)(n_tiles - 1) & 1u, dead, ix.status);
+        // ---- epilogue: O / l -> bf16 -> this sub-tile's (now idle) Q buffer -> coalesced stores
+        mbar_wait(bar(&bars.pv_done[u]), 0, dead, ix.status);
         tc_fence_after();
         const float inv = 1.f / l_run;
-        const bool valid = (q0 + r < L) && !dead;
-        __nv_bfloat16* dst = o + ((int64_t)(tok0 + q0 + r) * Hq + h) * D;
+        constexpr int RB = D * 2;                 // bytes per output row
+        constexpr int CH = RB / 16;               // 16-byte chunks per row
+        const uint32_t stage = s_q + u * kTileBytes;
 #pragma unroll
         for (int c = 0; c < D / 32; ++c) {
             float v[32];
-            tc_ld32(tmem + lane_addr + kColO + c * 32, v);
-            if (valid) {
+            tc_ld32(t_o + c * 32, v);
 #pragma unroll
-                for (int i = 0; i < 32; i += 8) {
-                    uint4 w;
-                    w.x = pack_bf16(v[i] * inv, v[i + 1] * inv);
-                    w.y = pack_bf16(v[i + 2] * inv, v[i + 3] * inv);
-                    w.z = pack_bf16(v[i + 4] * inv, v[i + 5] * inv);
-                    w.w = pack_bf16(v[i + 6] * inv, v[i + 7] * inv);
-                    *reinterpret_cast<uint4*>(dst + c * 32 + i) = w;
-                }
+            for (int i = 0; i < 32; i += 8) {
+                const int chunk = c * 4 + (i >> 3);
+                const uint32_t addr = stage + r * RB + ((chunk ^ (r & 7)) << 4);
+                asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};\n"
+                             :: "r"(addr), "r"(pack_bf16(v[i] * inv, v[i + 1] * inv)), "r"(pack_bf16(v[i + 2] * inv, v[i + 3] * inv)),
+                                "r"(pack_bf16(v[i + 4] * inv, v[i + 5] * inv)), "r"(pack_bf16(v[i + 6] * inv, v[i + 7] * inv))
+                             : "memory");
+            }
+        }
+        wg_sync(1 + u);
+        // rows past the end of the block belong to the next block (or to nobody): never store them
+        const int rows_valid = dead ? 0 : min(kTileM, L - (q0 + u * kTileM));
+        __nv_bfloat16* dst0 = o + ((int64_t)(tok0 + q0 + u * kTileM) * Hq + h) * D;
+        const int tid = threadIdx.x & 127;
+        for (int idx = tid; idx < kTileM * CH; idx += 128) {
+            const int row = idx / CH, chunk = idx - row * CH;
+            if (row < rows_valid) {
+                uint4 w;
+                asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];\n"
+                             : "=r"(w.x), "=r"(w.y), "=r"(w.z), "=r"(w.w)
+                             : "r"(stage + row * RB + ((chunk ^ (row & 7)) << 4)));
+                *reinterpret_cast<uint4*>(dst0 + (int64_t)row * Hq * D + chunk * 8) = w;
             }
         }
     }
 
     tc_fence_before();
     __syncthreads();
-    if (warp == 5) {
+    if (warp == 9) {
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;\n" :: "r"(tmem), "r"(kTmemCols) : "memory");
     }
@@ -419,7 +468,7 @@ template <int D>
 int launch_prefill_tc(const cpa_plan* plan, const void* q, const void* k, const void* v, void* o, cudaStream_t st) {
     const cpa_config& c = plan->cfg;
     constexpr int NB = D / 64;
-    constexpr int smem = (5 * NB + 2) * (int)kBlockBytes + 1024;   // Q + 2K + 2V tiles, P tile, alignment slack
+    constexpr int smem = 6 * NB * (int)kBlockBytes + 1024;   // 2 Q sub-tiles + 2 K + 2 V tiles, alignment slack
     static bool configured = false;  // per instantiation; one device per process assumed for this cache
     if (!configured) {
         if (cudaFuncSetAttribute(prefill_tc_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) {
@@ -435,7 +484,7 @@ int launch_prefill_tc(const cpa_plan* plan, const void* q, const void* k, const 
         return CPA_ECUDA;
     dim3 grid(plan->n_prefill, c.num_q_heads);
     prefill_tc_kernel<D><<<grid, kThreads, smem, st>>>(tm_q, tm_k, tm_v, (__nv_bfloat16*)o, plan->dev(), c.num_q_heads,
-                                                      c.num_kv_heads, c.scale * 1.4426950408889634f);
+                                                      c.num_kv_heads, plan->q_tile, c.scale * 1.4426950408889634f);
     return cudaGetLastError() == cudaSuccess ? CPA_OK : CPA_ECUDA;
 }
 
