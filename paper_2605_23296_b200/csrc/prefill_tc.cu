@@ -162,12 +162,17 @@ __device__ __forceinline__ void tc_ld32_nowait(uint32_t taddr, uint32_t (&r)[32]
         : "r"(taddr) : "memory");
 }
 __device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;\n" ::: "memory"); }
-__device__ __forceinline__ void tc_st16(uint32_t taddr, const uint32_t* v) {
+__device__ __forceinline__ void tc_st16(uint32_t taddr, const uint32_t (&v)[16]) {
     asm volatile(
         "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};\n"
         :: "r"(taddr), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]),
            "r"(v[8]), "r"(v[9]), "r"(v[10]), "r"(v[11]), "r"(v[12]), "r"(v[13]), "r"(v[14]), "r"(v[15])
         : "memory");
+}
+__device__ __forceinline__ float max3(float a, float b, float c) {
+    float d;
+    asm("max.f32 %0, %1, %2, %3;\n" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+    return d;
 }
 __device__ __forceinline__ void wg_sync(int id) { asm volatile("bar.sync %0, 128;\n" :: "r"(id) : "memory"); }
 
@@ -338,14 +343,27 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
 #pragma unroll
             for (int c = 0; c < 4; ++c) tc_ld32_nowait(t_s + c * 32, sv[c]);
             tc_wait_ld();
-            float mx = -INFINITY;
+            if (diag) {   // only the last tile touches the diagonal: keys in the row's future become -inf
 #pragma unroll
-            for (int c = 0; c < 4; ++c)
+                for (int c = 0; c < 4; ++c)
 #pragma unroll
-                for (int i = 0; i < 32; ++i) {
-                    if (diag && (c * 32 + i > r)) sv[c][i] = 0xff800000u;   // -inf: key is in the row's future
-                    mx = fmaxf(mx, __uint_as_float(sv[c][i]));
+                    for (int i = 0; i < 32; ++i)
+                        if (c * 32 + i > r) sv[c][i] = 0xff800000u;
+            }
+            // row max as a tree of 3-input max over eight independent accumulators
+            float mxa[8];
+#pragma unroll
+            for (int a = 0; a < 8; ++a) mxa[a] = max3(__uint_as_float(sv[0][a]), __uint_as_float(sv[0][a + 8]), __uint_as_float(sv[0][a + 16]));
+#pragma unroll
+            for (int a = 0; a < 8; ++a) mxa[a] = fmaxf(mxa[a], __uint_as_float(sv[0][a + 24]));
+#pragma unroll
+            for (int c = 1; c < 4; ++c)
+#pragma unroll
+                for (int a = 0; a < 8; ++a) {
+                    mxa[a] = max3(mxa[a], __uint_as_float(sv[c][a]), __uint_as_float(sv[c][a + 8]));
+                    mxa[a] = max3(mxa[a], __uint_as_float(sv[c][a + 16]), __uint_as_float(sv[c][a + 24]));
                 }
+            float mx = max3(max3(mxa[0], mxa[1], mxa[2]), max3(mxa[3], mxa[4], mxa[5]), fmaxf(mxa[6], mxa[7]));
             mx *= scale_log2;       // scale > 0, so the max commutes with the scaling
             // lazy rescale: keep the old reference max unless the new one is more than 2^8 above it
             float alpha = 1.f;
@@ -365,7 +383,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
             }
             l_run *= alpha;
             // weights, rounded to bf16, two keys per 32-bit TMEM column (P_u over the first 64 columns of S_u)
-            float sum = 0.f;
+            float sum[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
             for (int c = 0; c < 4; ++c) {
                 uint32_t pk[16];
@@ -376,11 +394,11 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                     const uint32_t w = pack_bf16(p0, p1);
                     pk[i >> 1] = w;
                     // row sum over the rounded weights: numerator and denominator stay consistent
-                    sum += __uint_as_float(w << 16) + __uint_as_float(w & 0xffff0000u);
+                    sum[(i >> 1) & 3] += __uint_as_float(w << 16) + __uint_as_float(w & 0xffff0000u);
                 }
                 tc_st16(t_s + c * 16, pk);
             }
-            l_run += sum;
+            l_run += (sum[0] + sum[1]) + (sum[2] + sum[3]);
             tc_wait_st();
             tc_fence_before();
             mbar_arrive(bar(&bars.p_full[u]));
