@@ -9,6 +9,8 @@
 //   warp 8     TMA producer (one elected lane): both Q sub-tiles once, then K and V tiles of
 //              128 keys through two-stage rings
 //   warp 9     MMA issuer (one elected lane) and owner of the TMEM allocation
+//   warps 10-11 idle; they complete the third warpgroup so that its registers can be handed
+//              to the softmax warpgroups (setmaxnreg works on whole warpgroups)
 // TMEM columns: S_u at u*128 (fp32 scores of sub-tile u), O_u at 256 + u*128.
 // Per KV tile j and sub-tile u:
 //                  S_u  = Q_u K_j^T            (both operands K-major in shared memory)
@@ -35,7 +37,9 @@ namespace {
 
 constexpr int kTileM = 128;        // query rows per CTA
 constexpr int kTileN = 128;        // keys per KV tile
-constexpr int kThreads = 320;
+constexpr int kThreads = 384;        // 2 softmax warpgroups + 1 warpgroup holding the producer and issuer warps
+constexpr int kRegsSoftmax = 232;    // register split after launch (launch gives every thread 168):
+constexpr int kRegsControl = 40;     // 2*128*232 + 128*40 = 64512 = 384*168, exactly the launch total
 constexpr uint32_t kSpinLimit = 1u << 20;
 constexpr uint32_t kBlockBytes = 128 * 128;   // one column block: 128 rows x 128 B
 
@@ -239,6 +243,9 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
     const uint32_t tmem = bars.tmem_base;
     bool dead = false;
 
+    if (warp >= 8) {
+    // the control warpgroup hands most of its registers to the softmax warpgroups
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;\n" :: "n"(kRegsControl));
     if (warp == 8) {
         // ------------------------------------------------------------ TMA producer
         if (lane == 0) {
@@ -323,7 +330,10 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                 if (j + 1 < n_total) tc_commit(bar(&bars.k_empty[s ^ 1]));
             }
         }
-    } else if (warp < 4 * n_sub) {
+    }
+    } else {
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;\n" :: "n"(kRegsSoftmax));
+    if (warp < 4 * n_sub) {
         // ------------------------------------------------------------ softmax + epilogue (one warpgroup per sub-tile)
         const int u = warp >> 2;
         const int r = threadIdx.x & 127;                                  // query row inside the sub-tile = TMEM lane
@@ -440,6 +450,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
             }
         }
     }
+    }
 
     tc_fence_before();
     __syncthreads();
@@ -489,10 +500,15 @@ int launch_prefill_tc(const cpa_plan* plan, const void* q, const void* k, const 
     constexpr int smem = 6 * NB * (int)kBlockBytes + 1024;   // 2 Q sub-tiles + 2 K + 2 V tiles, alignment slack
     static bool configured = false;  // per instantiation; one device per process assumed for this cache
     if (!configured) {
-        if (cudaFuncSetAttribute(prefill_tc_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) {
+        cudaFuncAttributes attr;
+        if (cudaFuncGetAttributes(&attr, prefill_tc_kernel<D>) != cudaSuccess ||
+            cudaFuncSetAttribute(prefill_tc_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) {
             (void)cudaGetLastError();
             return CPA_ECUDA;
         }
+        // The in-kernel register split may only hand out what the launch allocates; a kernel
+        // that asked for more would wait for registers forever, so refuse to launch it.
+        if (attr.numRegs * kThreads < 2 * 128 * kRegsSoftmax + 128 * kRegsControl) return CPA_EUNSUPPORTED;
         configured = true;
     }
     CUtensorMap tm_q, tm_k, tm_v;
