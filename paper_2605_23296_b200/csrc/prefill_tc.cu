@@ -38,8 +38,8 @@ namespace {
 constexpr int kTileM = 128;        // query rows per CTA
 constexpr int kTileN = 128;        // keys per KV tile
 constexpr int kThreads = 384;        // 2 softmax warpgroups + 1 warpgroup holding the producer and issuer warps
-constexpr int kRegsSoftmax = 232;    // register split after launch (launch gives every thread 168):
-constexpr int kRegsControl = 40;     // 2*128*232 + 128*40 = 64512 = 384*168, exactly the launch total
+constexpr int kRegsSoftmax = 216;    // register split after launch (launch gives every thread 168):
+constexpr int kRegsControl = 72;     // 2*128*216 + 128*72 = 64512 = 384*168, exactly the launch total
 constexpr uint32_t kSpinLimit = 1u << 20;
 constexpr uint32_t kBlockBytes = 128 * 128;   // one column block: 128 rows x 128 B
 
@@ -277,24 +277,32 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
         if (lane == 0) {
             constexpr uint32_t idesc_qk = instr_desc(kTileM, kTileN, false);
             constexpr uint32_t idesc_pv = instr_desc(kTileM, D, true);
+            // Descriptors are built once; inside the loops an operand advances by adding a constant
+            // to the descriptor's address field (units of 16 bytes), which keeps the issuing thread's
+            // instruction count per MMA small: it shares its scheduler with softmax warps.
+            const uint64_t dq0 = smem_desc(s_q, 16, 1024), dk0 = smem_desc(s_k, 16, 1024);
+            const uint64_t dv0 = smem_desc(s_v, kBlockBytes, 1024);
             auto issue_qk = [&](int u, int j) {   // S_u = Q_u K_j^T
-                const int s = j & 1;
+                const uint64_t dq = dq0 + (uint64_t)((u * kTileBytes) >> 4);
+                const uint64_t dk = dk0 + (uint64_t)(((j & 1) * kTileBytes) >> 4);
+                const uint32_t d_tmem = tmem + u * 128;
 #pragma unroll
                 for (int k = 0; k < D / 16; ++k) {
                     // 16 head dims per instruction: 32 B inside the 128-B swizzled row, next block after 4 steps
-                    const uint32_t off = (k >> 2) * kBlockBytes + (k & 3) * 32;
-                    tc_mma_ss(tmem + u * 128, smem_desc(s_q + u * kTileBytes + off, 16, 1024),
-                              smem_desc(s_k + s * kTileBytes + off, 16, 1024), idesc_qk, k > 0);
+                    constexpr uint32_t kBlk = kBlockBytes >> 4;
+                    const uint32_t off = (k >> 2) * kBlk + (k & 3) * 2;
+                    tc_mma_ss(d_tmem, dq + off, dk + off, idesc_qk, k > 0);
                 }
                 tc_commit(bar(&bars.s_full[u]));
             };
             auto issue_pv = [&](int u, int j) {   // O_u += P_u V_j, P_u read from TMEM (aliases S_u)
-                const int s = j & 1;
+                const uint64_t dv = dv0 + (uint64_t)(((j & 1) * kTileBytes) >> 4);
+                const uint32_t d_tmem = tmem + kColO + u * 128, a_tmem = tmem + u * 128;
+                const uint32_t acc0 = j > 0;
 #pragma unroll
                 for (int k = 0; k < kTileN / 16; ++k)
                     // 16 keys per instruction: 8 TMEM columns of A; 16 rows of 128 B of V, column blocks kBlockBytes apart
-                    tc_mma_ts(tmem + kColO + u * 128, tmem + u * 128 + k * 8,
-                              smem_desc(s_v + s * kTileBytes + k * 2048, kBlockBytes, 1024), idesc_pv, (j > 0 || k > 0));
+                    tc_mma_ts(d_tmem, a_tmem + k * 8, dv + k * (2048 >> 4), idesc_pv, k > 0 ? 1u : acc0);
             };
             // MMAs issued by this one thread execute in issue order, so QK_u(j+1) may be queued right
             // behind PV_u(j) although it overwrites the columns PV_u(j) reads P_u from.
