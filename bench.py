@@ -259,7 +259,7 @@ def run_gpu(args) -> None:
                 dec_events.append((t, e0, e1))
             else:
                 s.decode(qd[t], out=od[t])
-        state["launches"] += 1 + 2 + 3 * T
+        state["launches"] += 1 + 2 + 2 * T     # prefill, bulk append + length advance, T x (append, decode)
         return s
 
     def barrier():
@@ -348,12 +348,15 @@ def run_gpu(args) -> None:
     samp_bytes = statistics.mean(decode_kv_bytes(w, t) for t, _ in dec_samples)
     samp_ms = statistics.mean(m for _, m in dec_samples)
     achieved = samp_bytes / (samp_ms * 1e-3) / 1e9
-    roofline = {"bound": "hbm", "kernel": "decode_split_kernel + decode_combine_kernel (one cpa_decode call)",
+    # DRAM bytes of one decode_split_kernel launch on this workload from the ncu capture summarised in
+    # profiles/decode_split_kernel_dense8b.md (valid only for the default dense8b shape)
+    traffic = 138.8e6 if (w.name == "dense8b" and w.num_blocks == 8 and int(w.block_lens[0]) == 4096) else None
+    roofline = {"bound": "hbm", "kernel": "decode_split_kernel (one cpa_decode call: split-K scan with the merge fused in)",
                 "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                 "frac": achieved / peaks["hbm_gbs"], "peak_kind": f"of {peak_kind}",
                 "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS,
                 "launch_us": samp_ms * 1e3, "bytes_per_launch": samp_bytes,
-                "launches_sampled": len(dec_samples), "traffic": None}
+                "launches_sampled": len(dec_samples), "traffic": traffic}
 
     if args.skip_cpu:
         cpu = {"estimated_step_s": float("nan"), "cores": 0, "sample": "skipped", "measured_s": 0.0}

@@ -3,7 +3,7 @@
 // softmax in fp32 registers.
 //
 // One CTA = one (block, q item, query head); a q item is 256 query rows handled as two
-// 128-row sub-tiles that share every K/V tile.  Ten warps with fixed roles:
+// 128-row sub-tiles that share every K/V tile.  Twelve warps with fixed roles:
 //   warps 0-3  softmax + epilogue of sub-tile 0: thread r owns query row r (TMEM lane r), so
 //   warps 4-7  ... of sub-tile 1                 row max and row sum need no shuffles
 //   warp 8     TMA producer (one elected lane): both Q sub-tiles once, then K and V tiles of
