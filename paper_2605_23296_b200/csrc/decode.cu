@@ -121,6 +121,10 @@ decode_split_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __
     // this warp's pages are warp, warp+4, ... of the split: park their ids in shared memory
     for (int j = lane; warp + kDecodeWarps * j < n_reserved; j += 32)
         sm_pages[warp][j] = item[8 + warp + kDecodeWarps * j];
+    // Everything above reads plan constants only.  The launch may have started while the
+    // previous kernel in the stream (normally the step's append) was still running; from here
+    // on its writes (cached length, the new K/V row) are needed, so wait for it to finish.
+    asm volatile("griddepcontrol.wait;\n" ::: "memory");
     const int len = ix.seq_lens[b];
     __syncwarp();
     const int pages_active = (len + P - 1) / P;
@@ -349,9 +353,23 @@ int launch_decode(const cpa_plan* plan, const void* q, const void* k_pool, const
     }
     if (any_empty)
         decode_empty_rows_kernel<<<plan->B, 128, 0, st>>>((__nv_bfloat16*)o, ix, plan->B, c.num_q_heads * D);
-    decode_split_kernel<D><<<plan->n_decode, kDecodeThreads, kDecodeSmemBytes, st>>>(
-        (const __nv_bfloat16*)q, (const __nv_bfloat16*)k_pool, (const __nv_bfloat16*)v_pool, part_ml, part_o,
-        (__nv_bfloat16*)o, ix, c.num_q_heads, c.num_kv_heads, G, scale_log2);
+    // Programmatic dependent launch: the grid may be scheduled while the previous kernel of the
+    // stream drains; the kernel itself waits (griddepcontrol.wait) before it reads anything
+    // that kernel wrote.
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(plan->n_decode);
+    cfg.blockDim = dim3(kDecodeThreads);
+    cfg.dynamicSmemBytes = kDecodeSmemBytes;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    cudaError_t e = cudaLaunchKernelEx(&cfg, decode_split_kernel<D>, (const __nv_bfloat16*)q,
+                                       (const __nv_bfloat16*)k_pool, (const __nv_bfloat16*)v_pool, part_ml, part_o,
+                                       (__nv_bfloat16*)o, ix, (int)c.num_q_heads, (int)c.num_kv_heads, G, scale_log2);
+    if (e != cudaSuccess) { (void)cudaGetLastError(); return CPA_ECUDA; }
     return cudaGetLastError() == cudaSuccess ? CPA_OK : CPA_ECUDA;
 }
 

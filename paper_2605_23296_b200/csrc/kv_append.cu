@@ -25,6 +25,9 @@ __device__ __forceinline__ void copy_row_chunks(const uint4* __restrict__ k_src,
 __global__ void kv_append_step_kernel(const uint4* __restrict__ k_new, const uint4* __restrict__ v_new,
                                       uint4* __restrict__ k_pool, uint4* __restrict__ v_pool,
                                       cpa_dev_index ix, int Hkv, int chunks_per_head, int P) {
+    // let a dependent launch (the step's decode) start its own set-up now; it waits for this
+    // grid to finish before it reads what is written here
+    asm volatile("griddepcontrol.launch_dependents;\n" ::: "memory");
     const int b = blockIdx.x;
     const int pos = ix.seq_lens[b];
     const int capacity = (ix.page_indptr[b + 1] - ix.page_indptr[b]) * P;
