@@ -38,6 +38,7 @@ struct cpa_plan {
             off_append = 0, off_pidx = 0, off_pitems = 0, off_ditems = 0, off_tickets = 0, words = 0;
     int32_t item_stride = 0;
     int32_t* d_base = nullptr;   // caller's device buffer after cpa_plan_upload
+    mutable uint32_t decode_calls = 0;  // decode launches so far; its parity picks the scan direction
     std::vector<int32_t> append_stage;  // host staging for general appends
 
     int64_t index_bytes() const { return words * 4; }

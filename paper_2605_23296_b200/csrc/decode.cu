@@ -88,7 +88,7 @@ __global__ void __launch_bounds__(kDecodeThreads, 2)
 decode_split_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ k_pool,
                     const __nv_bfloat16* __restrict__ v_pool, float* __restrict__ part_ml,
                     float* __restrict__ part_o, __nv_bfloat16* __restrict__ out, cpa_dev_index ix, int Hq,
-                    int Hkv, int G, float scale_log2) {
+                    int Hkv, int G, float scale_log2, int reverse) {
     constexpr int P = 16;
     constexpr int KC = D / 32;  // 16-byte K chunks per thread per 8-key group
     constexpr int VC = D / 64;  // 16-byte V chunks per thread per key row
@@ -141,9 +141,14 @@ decode_split_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __
         bulk_load(dst, k_pool + chunk, kChunkBytes, bar);
         bulk_load(dst + kChunkBytes, v_pool + chunk, kChunkBytes, bar);
     };
+    // Consecutive decode steps walk the pages in opposite directions: what the previous step
+    // read last is what this step reads first, so a pool of about the L2's size is served
+    // largely from L2 instead of being evicted just before its reuse.  The online softmax does
+    // not care about the order of the keys.
+    auto local_index = [&](int i) { return reverse ? n_mine - 1 - i : i; };
 #pragma unroll
     for (int st = 0; st < STAGES; ++st)
-        if (st < n_mine && lane == 0) issue(st, sm_pages[warp][st]);
+        if (st < n_mine && lane == 0) issue(st, sm_pages[warp][local_index(st)]);
 
     // Q fragments: row gid of the A tile is query head g*G + gid (zero rows beyond G)
     uint4 qf[KC];
@@ -169,7 +174,7 @@ decode_split_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __
     for (int i = 0; i < n_mine; ++i) {
         const int st = i % STAGES;
         const uint32_t parity = (uint32_t)(i / STAGES) & 1u;
-        const int pg = first + warp + kDecodeWarps * i;  // page index inside the block
+        const int pg = first + warp + kDecodeWarps * local_index(i);  // page index inside the block
         if (!gave_up) {
             uint32_t spins = 0;
             while (!mbar_try_wait(bar0 + 8 * st, parity)) {
@@ -245,7 +250,7 @@ decode_split_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __
         // every lane has taken what it needs from this stage: refill it
         __syncwarp();
         const int nxt = i + STAGES;
-        if (nxt < n_mine && lane == 0) issue(st, sm_pages[warp][nxt]);
+        if (nxt < n_mine && lane == 0) issue(st, sm_pages[warp][local_index(nxt)]);
     }
     l_run += __shfl_xor_sync(0xffffffffu, l_run, 1);
     l_run += __shfl_xor_sync(0xffffffffu, l_run, 2);
@@ -368,7 +373,8 @@ int launch_decode(const cpa_plan* plan, const void* q, const void* k_pool, const
     cfg.numAttrs = 1;
     cudaError_t e = cudaLaunchKernelEx(&cfg, decode_split_kernel<D>, (const __nv_bfloat16*)q,
                                        (const __nv_bfloat16*)k_pool, (const __nv_bfloat16*)v_pool, part_ml, part_o,
-                                       (__nv_bfloat16*)o, ix, (int)c.num_q_heads, (int)c.num_kv_heads, G, scale_log2);
+                                       (__nv_bfloat16*)o, ix, (int)c.num_q_heads, (int)c.num_kv_heads, G, scale_log2,
+                                       (int)(plan->decode_calls++ & 1));
     if (e != cudaSuccess) { (void)cudaGetLastError(); return CPA_ECUDA; }
     return cudaGetLastError() == cudaSuccess ? CPA_OK : CPA_ECUDA;
 }
