@@ -195,6 +195,23 @@ class ClockSampler:
         return out
 
 
+def max_over_ranks(x: float, world: int, device) -> float:
+    """The slowest rank's time: every multi-GPU number is the maximum over ranks."""
+    if world == 1:
+        return x
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([x], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_tokens(w, world: int) -> int:
+    """Summary tokens produced per step by all ranks: every rank runs its own event of the same
+    shape (weak scaling, blocks are independent, no data-path collective)."""
+    return world * w.num_blocks * w.decode_steps
+
+
 def run_gpu(args) -> None:
     import torch
     import torch.distributed as dist
@@ -306,6 +323,7 @@ def run_gpu(args) -> None:
 
     # ---- end to end: host buffers in, host buffers out, copies inside the timed region -----
     e2e_ms = []
+    side = torch.cuda.Stream(dev)
     h2d = sum(t.numel() * 2 for t in (h_q, h_k, h_v, h_qd, h_kd, h_vd))
     d2h = (h_o.numel() + h_od.numel()) * 2
     for i in range(0 if args.skip_e2e else 1 + args.steps):
@@ -315,9 +333,14 @@ def run_gpu(args) -> None:
         e0.record(stream)
         q, k, v = (t.to(dev, non_blocking=True) for t in (h_q, h_k, h_v))
         qd, kd, vd = (t.to(dev, non_blocking=True) for t in (h_qd, h_kd, h_vd))
-        s = one_pass(q, k, v, qd, kd, vd, d_o, d_od)
-        h_o.copy_(d_o, non_blocking=True)
+        ev_pre = {n: torch.cuda.Event() for n in ("planned", "prefilled", "appended")}
+        s = one_pass(q, k, v, qd, kd, vd, d_o, d_od, ev_pre)
+        # the prefill output goes home on a side stream while the decode steps run
+        side.wait_event(ev_pre["prefilled"])
+        with torch.cuda.stream(side):
+            h_o.copy_(d_o, non_blocking=True)
         h_od.copy_(d_od, non_blocking=True)
+        stream.wait_stream(side)
         e1.record(stream)
         torch.cuda.synchronize(dev)
         assert s.status() == 0
@@ -325,21 +348,14 @@ def run_gpu(args) -> None:
         if i > 0:
             e2e_ms.append(e0.elapsed_time(e1))
 
-    def max_over_ranks(x: float) -> float:
-        if world == 1:
-            return x
-        t = torch.tensor([x], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        return float(t.item())
-
-    ms = max_over_ranks(statistics.mean(step_ms))
-    e2e = max_over_ranks(statistics.mean(e2e_ms)) if e2e_ms else float("nan")
+    ms = max_over_ranks(statistics.mean(step_ms), world, dev)
+    e2e = max_over_ranks(statistics.mean(e2e_ms), world, dev) if e2e_ms else float("nan")
     if rank != 0:
         if world > 1:
             dist.destroy_process_group()
         return
 
-    tokens = world * Bn * T
+    tokens = whole_job_tokens(w, world)
     pf_ms, dc_ms = statistics.mean(prefill_ms), statistics.mean(decode_ms)
     pf_tflops = prefill_flops(w) / (pf_ms * 1e-3) / 1e12
     total_kv = sum(decode_kv_bytes(w, t) for t in range(T))
@@ -348,9 +364,9 @@ def run_gpu(args) -> None:
     samp_bytes = statistics.mean(decode_kv_bytes(w, t) for t, _ in dec_samples)
     samp_ms = statistics.mean(m for _, m in dec_samples)
     achieved = samp_bytes / (samp_ms * 1e-3) / 1e9
-    # DRAM bytes of one decode_split_kernel launch on this workload from the ncu capture summarised in
-    # profiles/decode_split_kernel_dense8b.md (valid only for the default dense8b shape)
-    traffic = 138.8e6 if (w.name == "dense8b" and w.num_blocks == 8 and int(w.block_lens[0]) == 4096) else None
+    # DRAM bytes per launch are not quoted here: consecutive launches share L2 contents (the scan
+    # direction alternates), so a per-launch figure depends on the profiler's cache control
+    traffic = None
     roofline = {"bound": "hbm", "kernel": "decode_split_kernel (one cpa_decode call: split-K scan with the merge fused in)",
                 "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                 "frac": achieved / peaks["hbm_gbs"], "peak_kind": f"of {peak_kind}",

@@ -37,14 +37,14 @@ class CompactionSession:
     def __init__(self, block_lens: Sequence[int], max_new_tokens: int, num_q_heads: int,
                  num_kv_heads: int, head_dim: int, free_pages: Sequence[int], num_pages: int,
                  scale: Optional[float] = None, device: str = "cuda:0", pages_per_split: int = 0,
-                 poison_pools: bool = False, page_size: int = 16):
+                 poison_pools: bool = False, page_size: int = 16, q_tile_rows: int = 0):
         self.device = torch.device(device)
         self.Hq, self.Hkv, self.d, self.P = num_q_heads, num_kv_heads, head_dim, page_size
         self.B = len(block_lens)
         self.block_lens = np.asarray(block_lens, dtype=np.int32)
         self.scale = float(scale if scale is not None else head_dim ** -0.5)
         props = torch.cuda.get_device_properties(self.device)
-        self.cfg = B.cpa_config(num_q_heads, num_kv_heads, head_dim, page_size, self.scale, 0,
+        self.cfg = B.cpa_config(num_q_heads, num_kv_heads, head_dim, page_size, self.scale, q_tile_rows,
                                 pages_per_split, props.multi_processor_count)
         self.plan = B.cpa_plan_create(self.cfg, self.block_lens, max_new_tokens, free_pages)
         self.total_tokens = B.cpa_plan_param(self.plan, B.PARAM_TOTAL_TOKENS)

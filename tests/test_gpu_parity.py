@@ -171,6 +171,21 @@ def test_prefill_kernels_agree_with_each_other():
     s.close()
 
 
+@pytest.mark.parametrize("q_tile_rows", [128, 256])
+def test_prefill_both_work_item_sizes(q_tile_rows):
+    from paper_2605_23296_b200.session import CompactionSession
+    w = wl.custom([1, 128, 129, 255, 256, 257, 640], 8, 2, 128, steps=0, seed=23).materialise()
+    s = CompactionSession(w.block_lens, 0, 8, 2, 128, w.free_pages, w.num_pages, scale=w.scale,
+                          q_tile_rows=q_tile_rows)
+    assert s.param(2) == q_tile_rows
+    want = oa.prefill(w.q, w.k, w.v, _cu(w), w.scale)
+    for variant in (0, 1):
+        o = s.prefill(_dev(w.q), _dev(w.k), _dev(w.v), variant=variant)
+        assert s.status() == 0
+        assert_attention_close(_bits(o), want, f"q_tile {q_tile_rows} variant {variant}")
+    s.close()
+
+
 def test_prefill_outlier_keys():
     w = wl.dense8b(seed=21, num_blocks=3, block_len=700, steps=0)
     _check_prefill(w, what="outlier")
