@@ -107,7 +107,7 @@ enum {
  *   ascending block then tile; the decode work list of (block, kv_head, split),
  *   split s = pages [s*C_b, (s+1)*C_b) of the block, ordered by descending page
  *   count, ties by ascending block, kv head, split.  C_b is cfg->pages_per_split, or
- *   with 0 it is chosen per block so that all items fill one wave of CTAs (two per
+ *   with 0 it is chosen per block so that all items fill one wave of CTAs (three per
  *   SM): splits start at one per block and the block with the largest splits is
  *   split further while kv_heads more items still fit (never below 4 pages).
  * block_lens, free_pages: host int32 arrays (copied; caller keeps ownership).

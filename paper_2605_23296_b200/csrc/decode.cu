@@ -26,7 +26,7 @@ namespace {
 
 constexpr int kDecodeWarps = 4;
 constexpr int kDecodeThreads = kDecodeWarps * 32;
-constexpr int kDecodeSmemBytes = 96 * 1024;          // stage rings of the four warps (two CTAs per SM)
+constexpr int kDecodeSmemBytes = 64 * 1024;          // stage rings of the four warps (three CTAs per SM)
 constexpr int kMaxSplitPages = 1024;                 // planner's cap on pages per split
 constexpr uint32_t kSpinLimit = 1u << 18;            // bounded mbarrier wait (each try suspends briefly)
 
@@ -74,7 +74,9 @@ __device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_
 
 // One work item = (block, kv head, split of up to C pages); the item record carries the
 // split's page ids.  Four warps take the split's pages round-robin; each streams its pages
-// through its own ring of STAGES shared-memory stages (K chunk + V chunk per stage) and
+// through its own ring of STAGES shared-memory stages (K chunk + V chunk per stage; two
+// stages at head_dim 128 so that three CTAs = twelve warps fit an SM: once the pool is partly
+// served from L2 the per-page arithmetic latency, not the copy depth, is what needs hiding) and
 // keeps its own running (max, sum, acc).  The CTA then merges the four warps in shared
 // memory.  A block with a single active split is normalised and stored directly; otherwise
 // the CTA writes one partial per query head and takes a ticket: the last CTA of a
@@ -84,7 +86,7 @@ __device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_
 //   part_ml : [total_splits, Hq, 2]  (max in log2 units, sum), fp32
 //   part_o  : [total_splits, Hq, D]  unnormalised accumulators, fp32
 template <int D>
-__global__ void __launch_bounds__(kDecodeThreads, 2)
+__global__ void __launch_bounds__(kDecodeThreads, 3)
 decode_split_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ k_pool,
                     const __nv_bfloat16* __restrict__ v_pool, float* __restrict__ part_ml,
                     float* __restrict__ part_o, __nv_bfloat16* __restrict__ out, cpa_dev_index ix, int Hq,
@@ -94,7 +96,7 @@ decode_split_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __
     constexpr int VC = D / 64;  // 16-byte V chunks per thread per key row
     constexpr uint32_t kChunkBytes = P * D * 2;                  // one (page, head) chunk of K or of V
     constexpr uint32_t kStageBytes = 2 * kChunkBytes;
-    constexpr int STAGES = kDecodeSmemBytes / kDecodeWarps / kStageBytes;   // 3 at d=128, 6 at d=64
+    constexpr int STAGES = kDecodeSmemBytes / kDecodeWarps / kStageBytes;   // 2 at d=128, 4 at d=64
     extern __shared__ __align__(128) unsigned char dsm[];
     __shared__ __align__(8) uint64_t sm_bar[kDecodeWarps][STAGES];
     __shared__ float sm_m[kDecodeWarps][8];
@@ -187,13 +189,16 @@ decode_split_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __
         float sc[2][4];
 #pragma unroll
         for (int t = 0; t < 2; ++t) {
-            sc[t][0] = sc[t][1] = sc[t][2] = sc[t][3] = 0.f;
+            // two accumulators per 8-key group halve the length of the dependent MMA chain
+            float sa[4] = {0.f, 0.f, 0.f, 0.f}, sb[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
             for (int c = 0; c < KC; ++c) {
                 const uint4 kr = lds128(ks + (gid + 8 * t) * (D * 2) + (c * 4 + tig) * 16);
-                mma_bf16_16816(sc[t], qf[c].x, 0u, qf[c].y, 0u, kr.x, kr.y);
-                mma_bf16_16816(sc[t], qf[c].z, 0u, qf[c].w, 0u, kr.z, kr.w);
+                mma_bf16_16816(sa, qf[c].x, 0u, qf[c].y, 0u, kr.x, kr.y);
+                mma_bf16_16816(sb, qf[c].z, 0u, qf[c].w, 0u, kr.z, kr.w);
             }
+#pragma unroll
+            for (int e = 0; e < 4; ++e) sc[t][e] = sa[e] + sb[e];
         }
         // ---- mask the tail of the last page by index, then online softmax (row gid)
         const int key0 = pg * P + tig * 2;

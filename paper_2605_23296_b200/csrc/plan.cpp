@@ -90,7 +90,7 @@ extern "C" int cpa_plan_create(const cpa_config* cfg, int32_t num_blocks, const 
     for (const PItem& it : pit) { p->prefill_items.push_back(it.block); p->prefill_items.push_back(it.tile); }
 
     // Decode splits.  Every CTA pays a fixed start-up and merge cost, so the planner aims at
-    // ONE wave of resident CTAs (two per SM): starting from one split per block, it keeps
+    // ONE wave of resident CTAs (three per SM): starting from one split per block, it keeps
     // splitting the block whose splits are largest while the item count (kv heads x splits)
     // still fits.  split_pages[b] is the page count of block b's splits (the last may be
     // shorter).  A fixed pages_per_split from the configuration overrides the search.
@@ -99,7 +99,7 @@ extern "C" int cpa_plan_create(const cpa_config* cfg, int32_t num_blocks, const 
     if (cfg->pages_per_split > 0) {
         for (int32_t b = 0; b < B; ++b) p->split_pages[b] = cfg->pages_per_split;
     } else {
-        const int64_t slots = 2LL * (cfg->num_sms ? cfg->num_sms : 148);
+        const int64_t slots = 3LL * (cfg->num_sms ? cfg->num_sms : 148);
         int64_t items = (int64_t)B * cfg->num_kv_heads;
         while (items + cfg->num_kv_heads <= slots) {
             int32_t best = -1;

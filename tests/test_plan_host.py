@@ -72,8 +72,8 @@ def test_plan_bit_exact_full_configs(name):
     C = check_against_oracle(w, 0, permute=(name == "ragged"))
     pages = (w.block_lens.astype(np.int64) + w.decode_steps + 15) // 16
     n_items = int((w.num_kv_heads * -(-pages // np.asarray(C))).sum())
-    assert n_items <= 2 * 148                       # one wave of two CTAs per SM
-    assert n_items + w.num_kv_heads > 2 * 148 or max(C) <= 4
+    assert n_items <= 3 * 148                       # one wave of three CTAs per SM
+    assert n_items + w.num_kv_heads > 3 * 148 or max(C) <= 4
     sizes = -(-pages // -(-pages // np.asarray(C)))
     # greedy rule: the largest split could not be halved any more within the wave, and every
     # split that was made is at least as large as half the largest remaining one
@@ -94,7 +94,7 @@ def test_auto_split_aims_at_the_sm_count():
         ca = B.cpa_plan_param(plan_a, B.PARAM_PAGES_PER_SPLIT)
         cb = B.cpa_plan_param(plan_b, B.PARAM_PAGES_PER_SPLIT)
         assert cb >= ca
-        assert B.cpa_plan_export(plan_a, B.ARR_DECODE_ITEMS).shape[0] <= 2 * 148
+        assert B.cpa_plan_export(plan_a, B.ARR_DECODE_ITEMS).shape[0] <= 3 * 148
         assert B.cpa_plan_export(plan_b, B.ARR_DECODE_ITEMS).shape[0] == 64      # one split per (block, head)
     finally:
         B.cpa_plan_destroy(plan_a)
