@@ -420,8 +420,10 @@ def main() -> None:
     ap.add_argument("--skip-cpu", action="store_true", help="skip the CPU oracle leg (profiling)")
     args = ap.parse_args()
     args.overrides = {"num_blocks": args.blocks, "block_len": args.block_len, "steps": args.decode_steps}
-    if args.config == "ragged" and args.block_len:
-        ap.error("--block-len does not apply to the ragged configuration")
+    if args.config in ("ragged", "split", "tiny") and args.block_len:
+        ap.error("--block-len does not apply to this configuration")
+    if args.config == "tiny":
+        args.overrides = {}
     if args.impl == "reference":
         run_reference(args)
     else:

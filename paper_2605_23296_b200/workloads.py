@@ -160,9 +160,15 @@ def custom(lens, hq, hkv, d, steps, seed=7, permute_pages=True, outlier_scale=0.
                permute_pages=permute_pages, outlier_scale=outlier_scale)
 
 
+def split(seed: int = 4, num_blocks: int = 8, steps: int = 256) -> Workload:
+    """One point of the split sweep, addressable by name (block count as a keyword)."""
+    return split_sweep(num_blocks, seed=seed, steps=steps)
+
+
 CONFIGS = {
     "tiny": tiny,
     "dense8b": dense8b,
     "ragged": ragged,
     "moe120b": moe120b,
+    "split": split,
 }
