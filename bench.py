@@ -319,7 +319,6 @@ def run_gpu(args) -> None:
         dec_samples += [(t, e0.elapsed_time(e1)) for t, e0, e1 in dec_events]
     barrier()
     launches = state["launches"]
-    clocks = sampler.stop() if rank == 0 else {}
 
     # ---- end to end: host buffers in, host buffers out, copies inside the timed region -----
     e2e_ms = []
@@ -348,6 +347,7 @@ def run_gpu(args) -> None:
         if i > 0:
             e2e_ms.append(e0.elapsed_time(e1))
 
+    clocks = sampler.stop() if rank == 0 else {}   # sampled over both timed legs (device-resident and end-to-end)
     ms = max_over_ranks(statistics.mean(step_ms), world, dev)
     e2e = max_over_ranks(statistics.mean(e2e_ms), world, dev) if e2e_ms else float("nan")
     if rank != 0:
