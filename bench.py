@@ -267,16 +267,21 @@ def run_gpu(args) -> None:
         if ev:
             ev["appended"].record(stream)
         for t in range(T):
-            s.append(kd[t], vd[t])
-            if dec_events is not None and t % sample_every == 0:
+            sampled = dec_events is not None and t % sample_every == 0
+            if args.separate_append:
+                s.append(kd[t], vd[t])
+            if sampled:
                 e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
                 e0.record(stream)
+            if args.separate_append:
                 s.decode(qd[t], out=od[t])
+            else:   # the step's append is fused into the decode launch
+                s.decode_append(qd[t], kd[t], vd[t], out=od[t])
+            if sampled:
                 e1.record(stream)
                 dec_events.append((t, e0, e1))
-            else:
-                s.decode(qd[t], out=od[t])
-        state["launches"] += 1 + 2 + 2 * T     # prefill, bulk append + length advance, T x (append, decode)
+        # prefill, bulk append + length advance, then per step one fused launch (or append + decode)
+        state["launches"] += 1 + 2 + (2 if args.separate_append else 1) * T
         return s
 
     def barrier():
@@ -367,7 +372,7 @@ def run_gpu(args) -> None:
     # DRAM bytes per launch are not quoted here: consecutive launches share L2 contents (the scan
     # direction alternates), so a per-launch figure depends on the profiler's cache control
     traffic = None
-    roofline = {"bound": "hbm", "kernel": "decode_split_kernel (one cpa_decode call: split-K scan with the merge fused in)",
+    roofline = {"bound": "hbm", "kernel": "decode_split_kernel (one launch per step: append, split-K scan and merge fused)",
                 "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                 "frac": achieved / peaks["hbm_gbs"], "peak_kind": f"of {peak_kind}",
                 "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS,
@@ -416,6 +421,8 @@ def main() -> None:
     ap.add_argument("--block-len", type=int, default=0, help="override the block length (profiling)")
     ap.add_argument("--decode-steps", type=int, default=0, help="override the decode steps (profiling)")
     ap.add_argument("--pages-per-split", type=int, default=0, help="decode split size (0 = planner's choice)")
+    ap.add_argument("--separate-append", action="store_true",
+                    help="per decode step call cpa_kv_append and cpa_decode instead of the fused cpa_decode_append")
     ap.add_argument("--skip-e2e", action="store_true", help="skip the host-buffer leg (profiling)")
     ap.add_argument("--skip-cpu", action="store_true", help="skip the CPU oracle leg (profiling)")
     args = ap.parse_args()

@@ -200,6 +200,24 @@ CPA_API int cpa_decode(const cpa_plan* plan, const void* q, const void* k_pool, 
                void* o, void* d_workspace, void* stream);
 
 /*
+ * cpa_decode_append -- one decode step with its append fused in: exactly
+ * cpa_kv_append(plan, k_new, v_new, NULL, ...) followed by cpa_decode(...), in one launch
+ * (the per-step work of a summarisation sequence, Section 4 "Dispatch": store the new
+ * token's key/value, then attend over the block's cache including it).
+ *   q, o          : device bf16 [B, num_q_heads, head_dim]
+ *   k_new, v_new  : device bf16 [B, num_kv_heads, head_dim], the new token of every block
+ *   k_pool/v_pool : device bf16 pools; the new rows are written into them
+ *   d_workspace   : as for cpa_decode
+ * The CTA that scans the page holding the new position stores the row and uses it from its
+ * staged copy; the device lengths are double buffered, so the call needs no separate kernel
+ * to advance them.  Results are those of the two separate calls.  Errors: CPA_EINVAL,
+ * CPA_ESTATE, CPA_ENOSPC (a block would outgrow L_b + max_new_tokens; nothing is launched),
+ * CPA_ECUDA.
+ */
+CPA_API int cpa_decode_append(cpa_plan* plan, const void* q, const void* k_new, const void* v_new, void* k_pool,
+                              void* v_pool, void* o, void* d_workspace, void* stream);
+
+/*
  * cpa_decode_static -- cpa_decode for callers that cannot hand over scratch memory.
  * (The paper has no counterpart; this is a packaging variant of cpa_decode.)
  *

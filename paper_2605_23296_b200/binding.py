@@ -69,6 +69,8 @@ _lib.cpa_kv_append.argtypes = [_vp, _vp, _vp, _i32p, _vp, _vp, _vp]
 _lib.cpa_kv_append.restype = ctypes.c_int
 _lib.cpa_decode.argtypes = [_vp, _vp, _vp, _vp, _vp, _vp, _vp]
 _lib.cpa_decode.restype = ctypes.c_int
+_lib.cpa_decode_append.argtypes = [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]
+_lib.cpa_decode_append.restype = ctypes.c_int
 _lib.cpa_decode_static.argtypes = [_vp, _vp, _vp, _vp, _vp, _vp]
 _lib.cpa_decode_static.restype = ctypes.c_int
 _lib.cpa_strerror.argtypes = [ctypes.c_int]
@@ -160,6 +162,11 @@ def cpa_kv_append(plan: int, k_new, v_new, new_lens, k_pool, v_pool, stream: int
 def cpa_decode(plan: int, q, k_pool, v_pool, o, d_workspace, stream: int = 0) -> int:
     return _lib.cpa_decode(plan, _ptr(q), _ptr(k_pool), _ptr(v_pool), _ptr(o), _ptr(d_workspace),
                            stream or None)
+
+
+def cpa_decode_append(plan: int, q, k_new, v_new, k_pool, v_pool, o, d_workspace, stream: int = 0) -> int:
+    return _lib.cpa_decode_append(plan, _ptr(q), _ptr(k_new), _ptr(v_new), _ptr(k_pool), _ptr(v_pool), _ptr(o),
+                                  _ptr(d_workspace), stream or None)
 
 
 STATIC_SCRATCH_BYTES = 16 << 20

@@ -13,6 +13,7 @@ struct cpa_dev_index {
     const int32_t* page_indptr;    // [B+1]
     const int32_t* split_indptr;   // [B+1]
     int32_t* seq_lens;             // [B]   tokens cached per block (advanced by the append kernels)
+    int32_t* seq_lens_next;        // [B]   the other length buffer: a fused decode+append writes the new lengths here
     int32_t* append_indptr;        // [B+1] source-row offsets of a general append
     const int32_t* page_indices;   // [pages_used]
     const int32_t* prefill_items;  // [n_prefill, 2]
@@ -35,7 +36,9 @@ struct cpa_plan {
     // packed image of the device index buffer (int32 words) and offsets into it
     std::vector<int32_t> image;
     int64_t off_status = 0, off_cu = 0, off_pindptr = 0, off_sindptr = 0, off_seqlens = 0,
-            off_append = 0, off_pidx = 0, off_pitems = 0, off_ditems = 0, off_tickets = 0, words = 0;
+            off_append = 0, off_pidx = 0, off_pitems = 0, off_ditems = 0, off_tickets = 0, off_seqlens2 = 0,
+            words = 0;
+    int cur_lens = 0;            // which of the two device length buffers is current
     int32_t item_stride = 0;
     int32_t* d_base = nullptr;   // caller's device buffer after cpa_plan_upload
     mutable uint32_t decode_calls = 0;  // decode launches so far; its parity picks the scan direction
@@ -54,7 +57,8 @@ struct cpa_plan {
         d.cu_seqlens = d_base + off_cu;
         d.page_indptr = d_base + off_pindptr;
         d.split_indptr = d_base + off_sindptr;
-        d.seq_lens = d_base + off_seqlens;
+        d.seq_lens = d_base + (cur_lens ? off_seqlens2 : off_seqlens);
+        d.seq_lens_next = d_base + (cur_lens ? off_seqlens : off_seqlens2);
         d.append_indptr = d_base + off_append;
         d.page_indices = d_base + off_pidx;
         d.prefill_items = d_base + off_pitems;

@@ -72,6 +72,14 @@ __device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_
                  :: "r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
 }
 
+// Optional fused append (cpa_decode_append): k_new == nullptr means plain decode.
+struct cpa_fused_append {
+    const __nv_bfloat16* k_new;   // [B, Hkv, D] the step's new key rows
+    const __nv_bfloat16* v_new;
+    __nv_bfloat16* k_pool;        // the pools again, writable
+    __nv_bfloat16* v_pool;
+};
+
 // One work item = (block, kv head, split of up to C pages); the item record carries the
 // split's page ids.  Four warps take the split's pages round-robin; each streams its pages
 // through its own ring of STAGES shared-memory stages (K chunk + V chunk per stage; two
@@ -90,7 +98,7 @@ __global__ void __launch_bounds__(kDecodeThreads, 3)
 decode_split_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ k_pool,
                     const __nv_bfloat16* __restrict__ v_pool, float* __restrict__ part_ml,
                     float* __restrict__ part_o, __nv_bfloat16* __restrict__ out, cpa_dev_index ix, int Hq,
-                    int Hkv, int G, float scale_log2, int reverse) {
+                    int Hkv, int G, float scale_log2, int reverse, cpa_fused_append fa) {
     constexpr int P = 16;
     constexpr int KC = D / 32;  // 16-byte K chunks per thread per 8-key group
     constexpr int VC = D / 64;  // 16-byte V chunks per thread per key row
@@ -127,10 +135,32 @@ decode_split_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __
     // previous kernel in the stream (normally the step's append) was still running; from here
     // on its writes (cached length, the new K/V row) are needed, so wait for it to finish.
     asm volatile("griddepcontrol.wait;\n" ::: "memory");
-    const int len = ix.seq_lens[b];
+    // Fused append: the block's newest token (position len_old) is not in the pool yet.  The
+    // CTA whose split holds that position stores the row (for later steps) and patches its own
+    // staged copy of the page; every CTA counts the token.  Lengths are double buffered: this
+    // launch reads one array and the owner CTA of kv head 0 writes the other, so no CTA can see
+    // a length that already moved.
+    const bool fused = fa.k_new != nullptr;
+    const int len_old = ix.seq_lens[b];
+    const int len = len_old + (fused ? 1 : 0);
     __syncwarp();
     const int pages_active = (len + P - 1) / P;
     const int first = s * C;
+    const int pg_new = fused ? len_old / P : -1;   // page (inside the block) of the new token
+    const bool owner = fused && pg_new >= first && pg_new < first + n_reserved;
+    uint4 new_chunk = make_uint4(0, 0, 0, 0);      // lanes 0-15: a 16-byte piece of the K row, 16-31: of the V row
+    if (owner && warp == (pg_new - first) % kDecodeWarps) {
+        const int piece = lane & 15;
+        if (piece < D / 8) {
+            const __nv_bfloat16* src = (lane < 16 ? fa.k_new : fa.v_new) + ((int64_t)b * Hkv + g) * D + piece * 8;
+            new_chunk = *reinterpret_cast<const uint4*>(src);
+            const int64_t page = sm_pages[warp][(pg_new - first) / kDecodeWarps];
+            __nv_bfloat16* dst = (lane < 16 ? fa.k_pool : fa.v_pool) +
+                                 (((page * Hkv + g) * P) + (len_old % P)) * D + piece * 8;
+            *reinterpret_cast<uint4*>(dst) = new_chunk;
+        }
+        if (g == 0 && lane == 0) ix.seq_lens_next[b] = len;
+    }
     const int n_active = min(n_reserved, pages_active - first);  // pages of this split that hold keys
     if (n_active <= 0) return;  // split lies beyond the cached length (uniform per CTA)
     const int n_mine = (n_active - warp + kDecodeWarps - 1) / kDecodeWarps;  // pages of this warp (may be <= 0)
@@ -185,6 +215,15 @@ decode_split_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __
         }
         const uint32_t ks = ring + st * kStageBytes;
         const uint32_t vs = ks + kChunkBytes;
+        if (pg == pg_new) {   // (only the owning warp ever sees this page) put the new row into the staged copy
+            const int piece = lane & 15;
+            if (piece < D / 8) {
+                const uint32_t addr = (lane < 16 ? ks : vs) + (len_old % P) * (D * 2) + piece * 16;
+                asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};\n"
+                             :: "r"(addr), "r"(new_chunk.x), "r"(new_chunk.y), "r"(new_chunk.z), "r"(new_chunk.w) : "memory");
+            }
+            __syncwarp();
+        }
         // ---- S = Q K^T for the 16 keys of this page
         float sc[2][4];
 #pragma unroll
@@ -343,7 +382,7 @@ __global__ void decode_empty_rows_kernel(__nv_bfloat16* __restrict__ out, cpa_de
 
 template <int D>
 int launch_decode(const cpa_plan* plan, const void* q, const void* k_pool, const void* v_pool, void* o,
-                  void* ws, cudaStream_t st) {
+                  void* ws, cudaStream_t st, cpa_fused_append fa = cpa_fused_append{nullptr, nullptr, nullptr, nullptr}) {
     const cpa_config& c = plan->cfg;
     const int G = c.num_q_heads / c.num_kv_heads;
     const cpa_dev_index ix = plan->dev();
@@ -379,7 +418,7 @@ int launch_decode(const cpa_plan* plan, const void* q, const void* k_pool, const
     cudaError_t e = cudaLaunchKernelEx(&cfg, decode_split_kernel<D>, (const __nv_bfloat16*)q,
                                        (const __nv_bfloat16*)k_pool, (const __nv_bfloat16*)v_pool, part_ml, part_o,
                                        (__nv_bfloat16*)o, ix, (int)c.num_q_heads, (int)c.num_kv_heads, G, scale_log2,
-                                       (int)(plan->decode_calls++ & 1));
+                                       (int)(plan->decode_calls++ & 1), fa);
     if (e != cudaSuccess) { (void)cudaGetLastError(); return CPA_ECUDA; }
     return cudaGetLastError() == cudaSuccess ? CPA_OK : CPA_ECUDA;
 }
@@ -430,4 +469,30 @@ extern "C" int cpa_decode_static(const cpa_plan* plan, const void* q, const void
     cudaStream_t st = (cudaStream_t)stream;
     return plan->cfg.head_dim == 128 ? launch_decode<128>(plan, q, k_pool, v_pool, o, scratch_addr[dev], st)
                                      : launch_decode<64>(plan, q, k_pool, v_pool, o, scratch_addr[dev], st);
+}
+
+extern "C" int cpa_decode_append(cpa_plan* plan, const void* q, const void* k_new, const void* v_new, void* k_pool,
+                                 void* v_pool, void* o, void* d_workspace, void* stream) {
+    if (!plan || !q || !k_new || !v_new || !k_pool || !v_pool || !o || !d_workspace) return CPA_EINVAL;
+    if (!cpa_aligned16(q) || !cpa_aligned16(k_new) || !cpa_aligned16(v_new) || !cpa_aligned16(k_pool) ||
+        !cpa_aligned16(v_pool) || !cpa_aligned16(o) || !cpa_aligned16(d_workspace))
+        return CPA_EINVAL;
+    if (!plan->d_base) return CPA_ESTATE;
+    for (int b = 0; b < plan->B; ++b)
+        if ((int64_t)plan->seq_lens[b] + 1 > (int64_t)plan->block_lens[b] + plan->T) return CPA_ENOSPC;
+    // the kernel counts the new token itself; the host mirror moves first so that the launcher
+    // sees non-empty caches, and moves back if the launch fails
+    for (int b = 0; b < plan->B; ++b) plan->seq_lens[b] += 1;
+    cpa_fused_append fa{(const __nv_bfloat16*)k_new, (const __nv_bfloat16*)v_new, (__nv_bfloat16*)k_pool,
+                        (__nv_bfloat16*)v_pool};
+    cudaStream_t st = (cudaStream_t)stream;
+    // the device still holds the old lengths in the current buffer; they are read there
+    const int rc = plan->cfg.head_dim == 128 ? launch_decode<128>(plan, q, k_pool, v_pool, o, d_workspace, st, fa)
+                                             : launch_decode<64>(plan, q, k_pool, v_pool, o, d_workspace, st, fa);
+    if (rc != CPA_OK) {
+        for (int b = 0; b < plan->B; ++b) plan->seq_lens[b] -= 1;
+        return rc;
+    }
+    plan->cur_lens ^= 1;   // the other buffer now holds the lengths
+    return CPA_OK;
 }

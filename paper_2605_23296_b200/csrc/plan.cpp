@@ -156,6 +156,7 @@ extern "C" int cpa_plan_create(const cpa_config* cfg, int32_t num_blocks, const 
     p->item_stride = 8 + (p->C + 3) / 4 * 4;
     p->off_ditems = w;  w = align4(w + (int64_t)p->item_stride * p->n_decode);
     p->off_tickets = w; w = align4(w + (int64_t)B * cfg->num_kv_heads);
+    p->off_seqlens2 = w; w = align4(w + B);
     p->words = w;
     p->image.assign((size_t)w, 0);
     int32_t* im = p->image.data();
@@ -224,6 +225,7 @@ extern "C" int cpa_plan_upload(cpa_plan* plan, void* d_index_buf, int64_t bytes,
     if (bytes < plan->index_bytes()) return CPA_ENOSPC;
     // the device copy starts from an empty cache, so the host mirror does too
     std::fill(plan->seq_lens.begin(), plan->seq_lens.end(), 0);
+    plan->cur_lens = 0;
     cudaError_t e = cudaMemcpyAsync(d_index_buf, plan->image.data(), (size_t)plan->index_bytes(),
                                     cudaMemcpyHostToDevice, (cudaStream_t)stream);
     if (e != cudaSuccess) { (void)cudaGetLastError(); return CPA_ECUDA; }

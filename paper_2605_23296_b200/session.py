@@ -107,6 +107,15 @@ class CompactionSession:
                                  self._stream()), "cpa_decode")
         return out
 
+    def decode_append(self, q: torch.Tensor, k_new: torch.Tensor, v_new: torch.Tensor,
+                      out: Optional[torch.Tensor] = None) -> torch.Tensor:
+        """One decode step with its append fused in (same result as append() then decode())."""
+        if out is None:
+            out = torch.empty_like(q)
+        self._check(B.cpa_decode_append(self.plan, q, k_new, v_new, self.k_pool, self.v_pool, out,
+                                        self.workspace, self._stream()), "cpa_decode_append")
+        return out
+
     def status(self) -> int:
         return B.cpa_plan_status(self.plan, self._stream())
 

@@ -231,6 +231,43 @@ def test_decode_edge_lengths_cross_page_boundaries(hq, hkv, d):
     _check_decode(wl.custom(lens, hq, hkv, d, steps=20, seed=hq + d), what=f"edge {hq}/{hkv}/{d}")
 
 
+@pytest.mark.parametrize("hq,hkv,d", [(8, 2, 128), (8, 1, 64), (4, 4, 128)])
+def test_fused_decode_append_matches_oracle_and_separate_calls(hq, hkv, d):
+    # lengths around page boundaries, so new tokens land at the end of a page, open a new page,
+    # and fall into first / middle / last splits; fused and separate steps are interleaved
+    lens = [1, 15, 16, 17, 31, 32, 250, 256, 1000]
+    w = wl.custom(lens, hq, hkv, d, steps=24, seed=hq * 7 + d).materialise()
+    cu = _cu(w)
+    fused = _session(w, poison=True, pages_per_split=3)
+    plain = _session(w, poison=True, pages_per_split=3)
+    for s in (fused, plain):
+        s.append_prefill(_dev(w.k), _dev(w.v))
+    st = oa.DecodeState(w.k, w.v, cu, w.decode_steps)
+    kd, vd, qd = _dev(w.k_dec), _dev(w.v_dec), _dev(w.q_dec)
+    for t in range(w.decode_steps):
+        if t % 5 == 3:      # an ordinary step in between: the two length buffers must stay in sync
+            fused.append(kd[t], vd[t])
+            got = fused.decode(qd[t])
+        else:
+            got = fused.decode_append(qd[t], kd[t], vd[t])
+        plain.append(kd[t], vd[t])
+        ref = plain.decode(qd[t])
+        st.append(w.k_dec[t], w.v_dec[t])
+        assert fused.status() == 0
+        assert_attention_close(_bits(got), st.decode(w.q_dec[t], w.scale), f"fused step {t}")
+        assert np.array_equal(_bits(got), _bits(ref)), f"fused != separate at step {t}"
+    assert np.array_equal(fused.export(3), w.block_lens + w.decode_steps)
+    # the pools hold the same bytes wherever a token was written
+    assert np.array_equal(_bits(fused.k_pool), _bits(plain.k_pool))
+    assert np.array_equal(_bits(fused.v_pool), _bits(plain.v_pool))
+    # one more token than reserved is refused on the host
+    from paper_2605_23296_b200 import binding as B
+    assert B.cpa_decode_append(fused.plan, qd[0], kd[0], vd[0], fused.k_pool, fused.v_pool, got,
+                               fused.workspace) == B.CPA_ENOSPC
+    fused.close()
+    plain.close()
+
+
 def test_decode_step_equals_prefill_last_row_on_gpu():
     # the same identity the oracle is pinned with, now across the two CUDA kernels
     w = wl.custom([200, 77], 8, 2, 128, steps=1, seed=12).materialise()
