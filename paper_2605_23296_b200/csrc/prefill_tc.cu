@@ -173,6 +173,11 @@ __device__ __forceinline__ void tc_st16(uint32_t taddr, const uint32_t (&v)[16])
            "r"(v[8]), "r"(v[9]), "r"(v[10]), "r"(v[11]), "r"(v[12]), "r"(v[13]), "r"(v[14]), "r"(v[15])
         : "memory");
 }
+// acc += lo(w) + hi(w), the two bf16 halves of w widened exactly (mixed-precision add)
+__device__ __forceinline__ void add_bf16x2(float& acc, uint32_t w) {
+    asm("{\n .reg .b16 lo, hi;\n mov.b32 {lo, hi}, %1;\n add.rn.f32.bf16 %0, lo, %0;\n add.rn.f32.bf16 %0, hi, %0;\n}\n"
+        : "+f"(acc) : "r"(w));
+}
 __device__ __forceinline__ float max3(float a, float b, float c) {
     float d;
     asm("max.f32 %0, %1, %2, %3;\n" : "=f"(d) : "f"(a), "f"(b), "f"(c));
@@ -401,7 +406,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
             }
             l_run *= alpha;
             // weights, rounded to bf16, two keys per 32-bit TMEM column (P_u over the first 64 columns of S_u)
-            float sum[4] = {0.f, 0.f, 0.f, 0.f};
+            float sum[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
 #pragma unroll
             for (int c = 0; c < 4; ++c) {
                 uint32_t pk[16];
@@ -411,12 +416,13 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                     const float p1 = exp2f(fmaf(__uint_as_float(sv[c][i + 1]), scale_log2, -m_used));
                     const uint32_t w = pack_bf16(p0, p1);
                     pk[i >> 1] = w;
-                    // row sum over the rounded weights: numerator and denominator stay consistent
-                    sum[(i >> 1) & 3] += __uint_as_float(w << 16) + __uint_as_float(w & 0xffff0000u);
+                    // row sum over the rounded weights (numerator and denominator stay consistent);
+                    // the bf16 halves are added to the fp32 sum directly
+                    add_bf16x2(sum[(i >> 1) & 7], w);
                 }
                 tc_st16(t_s + c * 16, pk);
             }
-            l_run += (sum[0] + sum[1]) + (sum[2] + sum[3]);
+            l_run += ((sum[0] + sum[1]) + (sum[2] + sum[3])) + ((sum[4] + sum[5]) + (sum[6] + sum[7]));
             tc_wait_st();
             tc_fence_before();
             mbar_arrive(bar(&bars.p_full[u]));
