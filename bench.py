@@ -368,6 +368,13 @@ def run_gpu(args) -> None:
     # dominant kernel: the decode launches (split + merge), per-launch event pairs on sampled steps
     samp_bytes = statistics.mean(decode_kv_bytes(w, t) for t, _ in dec_samples)
     samp_ms = statistics.mean(m for _, m in dec_samples)
+    pair_us = samp_ms * 1e3
+    if not args.separate_append:
+        # every decode step is exactly one launch (append fused in), so the average launch duration
+        # over the timed region is the decode phase's CUDA-event time / T; event pairs around single
+        # launches add their own cost and break the overlap of consecutive launches
+        samp_bytes = total_kv / T
+        samp_ms = dc_ms / T
     achieved = samp_bytes / (samp_ms * 1e-3) / 1e9
     # DRAM bytes per launch are not quoted here: consecutive launches share L2 contents (the scan
     # direction alternates), so a per-launch figure depends on the profiler's cache control
@@ -377,7 +384,8 @@ def run_gpu(args) -> None:
                 "frac": achieved / peaks["hbm_gbs"], "peak_kind": f"of {peak_kind}",
                 "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS,
                 "launch_us": samp_ms * 1e3, "bytes_per_launch": samp_bytes,
-                "launches_sampled": len(dec_samples), "traffic": traffic}
+                "launches_timed": (T * args.steps if not args.separate_append else len(dec_samples)),
+                "launch_us_event_pair_sampled": pair_us, "traffic": traffic}
 
     if args.skip_cpu:
         cpu = {"estimated_step_s": float("nan"), "cores": 0, "sample": "skipped", "measured_s": 0.0}

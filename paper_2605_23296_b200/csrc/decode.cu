@@ -391,7 +391,13 @@ int launch_decode(const cpa_plan* plan, const void* q, const void* k_pool, const
     const float scale_log2 = c.scale * 1.4426950408889634f;
     bool any_empty = false;  // host mirror of the cached lengths
     for (int b = 0; b < plan->B; ++b) any_empty |= plan->seq_lens[b] == 0;
-    static bool configured = false;  // per instantiation; one device per process assumed for this cache
+    static bool configured_dev[64] = {};  // the attribute is per device: remember which devices have it
+    int dev_id = 0;
+    if (cudaGetDevice(&dev_id) != cudaSuccess || dev_id < 0 || dev_id >= 64) {
+        (void)cudaGetLastError();
+        return CPA_ECUDA;
+    }
+    bool& configured = configured_dev[dev_id];
     if (!configured) {
         if (cudaFuncSetAttribute(decode_split_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  kDecodeSmemBytes) != cudaSuccess) {

@@ -242,7 +242,13 @@ template <int D>
 int launch_prefill_mma(const cpa_plan* plan, const void* q, const void* k, const void* v, void* o, cudaStream_t st) {
     const cpa_config& c = plan->cfg;
     constexpr int smem = (kQTile + 4 * kKVTile) * D * 2;
-    static bool configured = false;  // one device per process is assumed for this attribute cache
+    static bool configured_dev[64] = {};  // the attribute is per device: remember which devices have it
+    int dev_id = 0;
+    if (cudaGetDevice(&dev_id) != cudaSuccess || dev_id < 0 || dev_id >= 64) {
+        (void)cudaGetLastError();
+        return CPA_ECUDA;
+    }
+    bool& configured = configured_dev[dev_id];
     if (!configured) {
         if (cudaFuncSetAttribute(prefill_mma_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) {
             (void)cudaGetLastError();

@@ -512,7 +512,13 @@ int launch_prefill_tc(const cpa_plan* plan, const void* q, const void* k, const 
     const cpa_config& c = plan->cfg;
     constexpr int NB = D / 64;
     constexpr int smem = 6 * NB * (int)kBlockBytes + 1024;   // 2 Q sub-tiles + 2 K + 2 V tiles, alignment slack
-    static bool configured = false;  // per instantiation; one device per process assumed for this cache
+    static bool configured_dev[64] = {};  // the attribute is per device: remember which devices have it
+    int dev_id = 0;
+    if (cudaGetDevice(&dev_id) != cudaSuccess || dev_id < 0 || dev_id >= 64) {
+        (void)cudaGetLastError();
+        return CPA_ECUDA;
+    }
+    bool& configured = configured_dev[dev_id];
     if (!configured) {
         cudaFuncAttributes attr;
         if (cudaFuncGetAttributes(&attr, prefill_tc_kernel<D>) != cudaSuccess ||
