@@ -81,15 +81,20 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
 }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;\n" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory"); }
-__device__ __forceinline__ void tc_commit(uint32_t bar) {
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n" :: "r"(bar) : "memory");
+// The issuing warp runs its loops convergently (all lanes), which lets the compiler keep MMA
+// operands on the uniform datapath; only the instruction itself is predicated on `leader`.
+__device__ __forceinline__ void tc_commit(uint32_t bar, uint32_t leader) {
+    asm volatile("{\n .reg .pred q;\n setp.ne.b32 q, %1, 0;\n"
+                 " @q tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n}\n"
+                 :: "r"(bar), "r"(leader) : "memory");
 }
 // D[tmem] (+)= A[smem desc] * B[smem desc]; `accumulate` = 0 overwrites D.
-__device__ __forceinline__ void tc_mma_ss(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+__device__ __forceinline__ void tc_mma_ss(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate,
+                                          uint32_t leader) {
     asm volatile(
-        "{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n"
-        " tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}\n"
-        :: "r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+        "{\n .reg .pred p, q;\n setp.ne.b32 p, %4, 0;\n setp.ne.b32 q, %5, 0;\n"
+        " @q tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}\n"
+        :: "r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(leader) : "memory");
 }
 // 32 consecutive fp32 columns of this thread's TMEM lane.
 __device__ __forceinline__ void tc_ld32(uint32_t taddr, float (&v)[32]) {
@@ -148,11 +153,12 @@ __host__ __device__ constexpr uint32_t instr_desc(int M, int N, bool b_mn_major)
 
 // D[tmem] (+)= A[tmem] * B[smem desc]: A is a 128-lane x 16-element bf16 slice held in TMEM
 // (two consecutive K elements per 32-bit column, row = lane).
-__device__ __forceinline__ void tc_mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+__device__ __forceinline__ void tc_mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc, uint32_t accumulate,
+                                          uint32_t leader) {
     asm volatile(
-        "{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n"
-        " tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n}\n"
-        :: "r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+        "{\n .reg .pred p, q;\n setp.ne.b32 p, %4, 0;\n setp.ne.b32 q, %5, 0;\n"
+        " @q tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n}\n"
+        :: "r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(leader) : "memory");
 }
 // 32 consecutive 32-bit columns of this thread's TMEM lane, no wait (pair with tc_wait_ld).
 __device__ __forceinline__ void tc_ld32_nowait(uint32_t taddr, uint32_t (&r)[32]) {
@@ -278,8 +284,9 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
             }
         }
     } else if (warp == 9) {
-        // ------------------------------------------------------------ MMA issuer
-        if (lane == 0) {
+        // ------------------------------------------------------------ MMA issuer (whole warp, one lane issues)
+        {
+            const uint32_t leader = (lane == 0);
             constexpr uint32_t idesc_qk = instr_desc(kTileM, kTileN, false);
             constexpr uint32_t idesc_pv = instr_desc(kTileM, D, true);
             // Descriptors are built once; inside the loops an operand advances by adding a constant
@@ -296,9 +303,9 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                     // 16 head dims per instruction: 32 B inside the 128-B swizzled row, next block after 4 steps
                     constexpr uint32_t kBlk = kBlockBytes >> 4;
                     const uint32_t off = (k >> 2) * kBlk + (k & 3) * 2;
-                    tc_mma_ss(d_tmem, dq + off, dk + off, idesc_qk, k > 0);
+                    tc_mma_ss(d_tmem, dq + off, dk + off, idesc_qk, k > 0, leader);
                 }
-                tc_commit(bar(&bars.s_full[u]));
+                tc_commit(bar(&bars.s_full[u]), leader);
             };
             auto issue_pv = [&](int u, int j) {   // O_u += P_u V_j, P_u read from TMEM (aliases S_u)
                 const uint64_t dv = dv0 + (uint64_t)(((j & 1) * kTileBytes) >> 4);
@@ -307,7 +314,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
 #pragma unroll
                 for (int k = 0; k < kTileN / 16; ++k)
                     // 16 keys per instruction: 8 TMEM columns of A; 16 rows of 128 B of V, column blocks kBlockBytes apart
-                    tc_mma_ts(d_tmem, a_tmem + k * 8, dv + k * (2048 >> 4), idesc_pv, k > 0 ? 1u : acc0);
+                    tc_mma_ts(d_tmem, a_tmem + k * 8, dv + k * (2048 >> 4), idesc_pv, k > 0 ? 1u : acc0, leader);
             };
             // MMAs issued by this one thread execute in issue order, so QK_u(j+1) may be queued right
             // behind PV_u(j) although it overwrites the columns PV_u(j) reads P_u from.
@@ -317,7 +324,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                 tc_fence_after();
                 issue_qk(u, 0);
             }
-            tc_commit(bar(&bars.k_empty[0]));
+            tc_commit(bar(&bars.k_empty[0]), leader);
             for (int j = 0; j < n_total; ++j) {
                 const int s = j & 1;
                 bool have_v = false, have_k = false;
@@ -328,7 +335,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                         mbar_wait(bar(&bars.p_full[u]), (uint32_t)j & 1u, dead, ix.status);
                         tc_fence_after();
                         issue_pv(u, j);
-                        if (j == n_kv - 1) tc_commit(bar(&bars.pv_done[u]));
+                        if (j == n_kv - 1) tc_commit(bar(&bars.pv_done[u]), leader);
                     }
                     if (j + 1 < n_kv) {
                         if (!have_k) {
@@ -339,8 +346,8 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                         issue_qk(u, j + 1);
                     }
                 }
-                tc_commit(bar(&bars.v_empty[s]));
-                if (j + 1 < n_total) tc_commit(bar(&bars.k_empty[s ^ 1]));
+                tc_commit(bar(&bars.v_empty[s]), leader);
+                if (j + 1 < n_total) tc_commit(bar(&bars.k_empty[s ^ 1]), leader);
             }
         }
     }
