@@ -17,6 +17,8 @@
 // Both contractions are invariant under a permutation of the contracted index, so a
 // thread reads whole 16-byte chunks from the staged page and pairs registers up as
 // the MMA fragments need them; no transposes, no ldmatrix.
+#include <algorithm>
+
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 
@@ -98,7 +100,7 @@ __global__ void __launch_bounds__(kDecodeThreads, 3)
 decode_split_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ k_pool,
                     const __nv_bfloat16* __restrict__ v_pool, float* __restrict__ part_ml,
                     float* __restrict__ part_o, __nv_bfloat16* __restrict__ out, cpa_dev_index ix, int Hq,
-                    int Hkv, int G, float scale_log2, int reverse, cpa_fused_append fa) {
+                    int Hkv, int G, float scale_log2, int reverse, cpa_fused_append fa, int n_items) {
     constexpr int P = 16;
     constexpr int KC = D / 32;  // 16-byte K chunks per thread per 8-key group
     constexpr int VC = D / 64;  // 16-byte V chunks per thread per key row
@@ -124,7 +126,13 @@ decode_split_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __
     }
     __syncwarp();
 
-    const int32_t* item = ix.decode_items + (int64_t)blockIdx.x * ix.item_stride;
+    bool gave_up = false;  // a bounded wait ran out: stop waiting, results are void, status says so
+    int ring_pos = 0;      // pages this warp has pushed through its ring so far (stage and phase carry over)
+    // A CTA takes items blockIdx.x, blockIdx.x + gridDim.x, ...: the grid is at most one wave, so when
+    // there are more items than resident CTAs nobody waits for a second, half-empty wave.
+    for (int item_idx = blockIdx.x; item_idx < n_items; item_idx += gridDim.x) {
+    if (item_idx != (int)blockIdx.x) __syncthreads();  // the previous item's merge buffer aliases the rings
+    const int32_t* item = ix.decode_items + (int64_t)item_idx * ix.item_stride;
     const int4 hdr = *reinterpret_cast<const int4*>(item);
     const int b = hdr.x, g = hdr.y, s = hdr.z, n_reserved = hdr.w;
     const int C = item[4];  // pages per split of this block
@@ -162,7 +170,7 @@ decode_split_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __
         if (g == 0 && lane == 0) ix.seq_lens_next[b] = len;
     }
     const int n_active = min(n_reserved, pages_active - first);  // pages of this split that hold keys
-    if (n_active <= 0) return;  // split lies beyond the cached length (uniform per CTA)
+    if (n_active <= 0) continue;  // split lies beyond the cached length (uniform per CTA)
     const int n_mine = (n_active - warp + kDecodeWarps - 1) / kDecodeWarps;  // pages of this warp (may be <= 0)
 
     auto issue = [&](int st, int page) {  // lane 0 only
@@ -180,7 +188,7 @@ decode_split_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __
     auto local_index = [&](int i) { return reverse ? n_mine - 1 - i : i; };
 #pragma unroll
     for (int st = 0; st < STAGES; ++st)
-        if (st < n_mine && lane == 0) issue(st, sm_pages[warp][local_index(st)]);
+        if (st < n_mine && lane == 0) issue((ring_pos + st) % STAGES, sm_pages[warp][local_index(st)]);
 
     // Q fragments: row gid of the A tile is query head g*G + gid (zero rows beyond G)
     uint4 qf[KC];
@@ -201,11 +209,10 @@ decode_split_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __
             for (int e = 0; e < 4; ++e) acc[c][i][e] = 0.f;
     float m_run = -INFINITY;  // running max of raw scores, row gid
     float l_run = 0.f;        // this thread's share of the running sum, row gid
-    bool gave_up = false;     // a bounded wait ran out: stop waiting, results are void, status says so
 
     for (int i = 0; i < n_mine; ++i) {
-        const int st = i % STAGES;
-        const uint32_t parity = (uint32_t)(i / STAGES) & 1u;
+        const int st = (ring_pos + i) % STAGES;
+        const uint32_t parity = (uint32_t)((ring_pos + i) / STAGES) & 1u;
         const int pg = first + warp + kDecodeWarps * local_index(i);  // page index inside the block
         if (!gave_up) {
             uint32_t spins = 0;
@@ -296,6 +303,7 @@ decode_split_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __
         const int nxt = i + STAGES;
         if (nxt < n_mine && lane == 0) issue(st, sm_pages[warp][local_index(nxt)]);
     }
+    if (n_mine > 0) ring_pos += n_mine;
     l_run += __shfl_xor_sync(0xffffffffu, l_run, 1);
     l_run += __shfl_xor_sync(0xffffffffu, l_run, 2);
 
@@ -339,7 +347,7 @@ decode_split_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __
             if (dim == 0) *reinterpret_cast<float2*>(part_ml + (prow + h) * 2) = make_float2(m, l);
         }
     }
-    if (n_splits == 1) return;
+    if (n_splits == 1) continue;
 
     // ---- the last CTA of this (block, kv head) merges the splits
     __threadfence();
@@ -351,7 +359,7 @@ decode_split_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __
         if (sm_last) *ticket = 0;  // every other split has arrived; ready for the next launch
     }
     __syncthreads();
-    if (!sm_last) return;
+    if (!sm_last) continue;
     __threadfence();
     const int64_t base = (int64_t)ix.split_indptr[b] * Hq + g * G;
     for (int idx = threadIdx.x; idx < G * HP; idx += kDecodeThreads) {
@@ -371,6 +379,7 @@ decode_split_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __
         const float inv = 1.f / l;
         *reinterpret_cast<__nv_bfloat162*>(out + (out_row + h) * D + dim) = __floats2bfloat162_rn(o0 * inv, o1 * inv);
     }
+    }  // items
 }
 
 // A block whose cache is still empty has no active split and gets a zero output row.
@@ -412,7 +421,8 @@ int launch_decode(const cpa_plan* plan, const void* q, const void* k_pool, const
     // stream drains; the kernel itself waits (griddepcontrol.wait) before it reads anything
     // that kernel wrote.
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(plan->n_decode);
+    const int slots = 3 * (c.num_sms ? c.num_sms : 148);   // resident CTAs: three per SM
+    cfg.gridDim = dim3(std::min(plan->n_decode, slots));
     cfg.blockDim = dim3(kDecodeThreads);
     cfg.dynamicSmemBytes = kDecodeSmemBytes;
     cfg.stream = st;
@@ -424,7 +434,7 @@ int launch_decode(const cpa_plan* plan, const void* q, const void* k_pool, const
     cudaError_t e = cudaLaunchKernelEx(&cfg, decode_split_kernel<D>, (const __nv_bfloat16*)q,
                                        (const __nv_bfloat16*)k_pool, (const __nv_bfloat16*)v_pool, part_ml, part_o,
                                        (__nv_bfloat16*)o, ix, (int)c.num_q_heads, (int)c.num_kv_heads, G, scale_log2,
-                                       (int)(plan->decode_calls++ & 1), fa);
+                                       (int)(plan->decode_calls++ & 1), fa, (int)plan->n_decode);
     if (e != cudaSuccess) { (void)cudaGetLastError(); return CPA_ECUDA; }
     return cudaGetLastError() == cudaSuccess ? CPA_OK : CPA_ECUDA;
 }
