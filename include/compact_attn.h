@@ -176,7 +176,7 @@ CPA_API int cpa_prefill_variant(const cpa_plan* plan, const void* q, const void*
  * Token i of block b goes to position seq_lens[b] + i, i.e. pool slot
  * page_indices[page_indptr[b] + pos / P] * P + pos % P.  With new_lens == NULL,
  * or new_lens == block_lens on an empty cache, nothing is copied from the host,
- * so the call can be recorded in a CUDA graph; otherwise B+1 offsets are copied
+ * so the call enqueues device work only; otherwise B+1 offsets are copied
  * to the device first.  Errors: CPA_EINVAL, CPA_ESTATE, CPA_ENOSPC (a block would
  * outgrow L_b + max_new_tokens; nothing is launched), CPA_ECUDA.
  */
