@@ -268,6 +268,27 @@ def test_fused_decode_append_matches_oracle_and_separate_calls(hq, hkv, d):
     plain.close()
 
 
+def test_decode_with_some_blocks_still_empty():
+    # blocks 1 and 3 have nothing cached yet: their output rows are zero, the others are attended normally
+    import torch
+    w = wl.custom([40, 9, 70, 5], 8, 2, 128, steps=2, seed=51).materialise()
+    s = _session(w, poison=True)
+    cu = _cu(w)
+    lens = np.array([40, 0, 33, 0], dtype=np.int32)
+    rows = np.concatenate([np.arange(cu[b], cu[b] + lens[b]) for b in range(4)])
+    s.append(_dev(w.k[rows]), _dev(w.v[rows]), lens)
+    q = _dev(w.q_dec[0])
+    out = torch.full_like(q, 5.0)
+    s.decode(q, out=out)
+    assert s.status() == 0
+    got = _bits(out)
+    assert (got[1] == 0).all() and (got[3] == 0).all()
+    for b in (0, 2):
+        want = oa.attend_token(w.q_dec[0][b], w.k[cu[b]:cu[b] + lens[b]], w.v[cu[b]:cu[b] + lens[b]], w.scale)
+        assert_attention_close(got[b], want, f"block {b}")
+    s.close()
+
+
 def test_decode_step_equals_prefill_last_row_on_gpu():
     # the same identity the oracle is pinned with, now across the two CUDA kernels
     w = wl.custom([200, 77], 8, 2, 128, steps=1, seed=12).materialise()
