@@ -69,4 +69,7 @@ struct cpa_plan {
     }
 };
 
+// largest pages-per-split the planner produces: the decode kernel parks a split's page ids in shared memory
+constexpr int32_t kMaxSplitPages = 1024;
+
 static inline bool cpa_aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }

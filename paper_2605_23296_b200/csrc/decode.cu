@@ -29,7 +29,6 @@ namespace {
 constexpr int kDecodeWarps = 4;
 constexpr int kDecodeThreads = kDecodeWarps * 32;
 constexpr int kDecodeSmemBytes = 64 * 1024;          // stage rings of the four warps (three CTAs per SM)
-constexpr int kMaxSplitPages = 1024;                 // planner's cap on pages per split
 constexpr uint32_t kSpinLimit = 1u << 18;            // bounded mbarrier wait (each try suspends briefly)
 
 __device__ __forceinline__ void mma_bf16_16816(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,

@@ -13,7 +13,6 @@ namespace {
 
 int64_t align4(int64_t words) { return (words + 3) / 4 * 4; }  // 16-byte alignment of every array
 
-constexpr int32_t kMaxSplitPages = 1024;  // page ids of one split the decode kernel keeps in shared memory
 
 }  // namespace
 
