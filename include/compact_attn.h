@@ -25,7 +25,10 @@
  *   - Tensors are bf16.  Packed token-major layout [tokens, heads, head_dim] for
  *     Q/K/V/O, blocks back to back in block order (offsets = cu_seqlens).
  *     KV pools are [num_pages, num_kv_heads, page_size, head_dim], one pool for K
- *     and one for V; a (page, head) chunk is contiguous.
+ *     and one for V; a (page, head) chunk is contiguous.  Inside a row the 16-byte
+ *     pieces are permuted: piece j of the row in slot r is stored at position
+ *     (j & ~7) | ((j & 7) ^ (r & 7)), so that a chunk copied verbatim into shared
+ *     memory is read without bank conflicts.  Only this library reads the pools.
  *   - Every call returns 0 (CPA_OK) or a negative cpa_status.  Nothing throws,
  *     exits, or traps the device.  Device-side waits are bounded; if one gives up
  *     the kernel records it in the plan's device status word, which

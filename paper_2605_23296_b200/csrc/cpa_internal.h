@@ -72,4 +72,10 @@ struct cpa_plan {
 // largest pages-per-split the planner produces: the decode kernel parks a split's page ids in shared memory
 constexpr int32_t kMaxSplitPages = 1024;
 
+// Pool rows are stored with their 16-byte pieces permuted: piece j of the row in slot r sits at
+// position cpa_pool_piece(j, r) (an involution inside every group of 8 pieces = 128 bytes).  A
+// (page, head) chunk copied to shared memory as it is can then be read by the decode kernel's
+// fragment pattern without bank conflicts on the V side.
+__host__ __device__ static inline int cpa_pool_piece(int j, int slot) { return (j & ~7) | ((j & 7) ^ (slot & 7)); }
+
 static inline bool cpa_aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }

@@ -163,7 +163,7 @@ decode_split_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __
             new_chunk = *reinterpret_cast<const uint4*>(src);
             const int64_t page = sm_pages[warp][(pg_new - first) / kDecodeWarps];
             __nv_bfloat16* dst = (lane < 16 ? fa.k_pool : fa.v_pool) +
-                                 (((page * Hkv + g) * P) + (len_old % P)) * D + piece * 8;
+                                 (((page * Hkv + g) * P) + (len_old % P)) * D + cpa_pool_piece(piece, len_old % P) * 8;
             *reinterpret_cast<uint4*>(dst) = new_chunk;
         }
         if (g == 0 && lane == 0) ix.seq_lens_next[b] = len;
@@ -224,7 +224,7 @@ decode_split_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __
         if (pg == pg_new) {   // (only the owning warp ever sees this page) put the new row into the staged copy
             const int piece = lane & 15;
             if (piece < D / 8) {
-                const uint32_t addr = (lane < 16 ? ks : vs) + (len_old % P) * (D * 2) + piece * 16;
+                const uint32_t addr = (lane < 16 ? ks : vs) + (len_old % P) * (D * 2) + cpa_pool_piece(piece, len_old % P) * 16;
                 asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};\n"
                              :: "r"(addr), "r"(new_chunk.x), "r"(new_chunk.y), "r"(new_chunk.z), "r"(new_chunk.w) : "memory");
             }
@@ -238,7 +238,7 @@ decode_split_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __
             float sa[4] = {0.f, 0.f, 0.f, 0.f}, sb[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
             for (int c = 0; c < KC; ++c) {
-                const uint4 kr = lds128(ks + (gid + 8 * t) * (D * 2) + (c * 4 + tig) * 16);
+                const uint4 kr = lds128(ks + (gid + 8 * t) * (D * 2) + cpa_pool_piece(c * 4 + tig, gid) * 16);
                 mma_bf16_16816(sa, qf[c].x, 0u, qf[c].y, 0u, kr.x, kr.y);
                 mma_bf16_16816(sb, qf[c].z, 0u, qf[c].w, 0u, kr.z, kr.w);
             }
@@ -284,7 +284,7 @@ decode_split_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __
 #pragma unroll
             for (int r = 0; r < 4; ++r) {
                 const int row = 2 * tig + (r & 1) + 8 * (r >> 1);
-                vr[r] = lds128(vs + row * (D * 2) + (c * 8 + gid) * 16);
+                vr[r] = lds128(vs + row * (D * 2) + cpa_pool_piece(c * 8 + gid, row) * 16);
                 // unused slots may hold anything (even NaN): select them away
                 if (partial && pg * P + row >= len) vr[r] = make_uint4(0, 0, 0, 0);
             }

@@ -14,7 +14,7 @@ __device__ __forceinline__ void copy_row_chunks(const uint4* __restrict__ k_src,
     for (int c = threadIdx.x; c < chunks; c += blockDim.x) {
         const int g = c / chunks_per_head;
         const int j = c - g * chunks_per_head;
-        const int64_t dst = ((page * Hkv + g) * P + off) * chunks_per_head + j;
+        const int64_t dst = ((page * Hkv + g) * P + off) * chunks_per_head + cpa_pool_piece(j, off);
         k_pool[dst] = k_src[c];
         v_pool[dst] = v_src[c];
     }

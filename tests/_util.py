@@ -10,6 +10,18 @@ def bits_to_f64(bits: np.ndarray) -> np.ndarray:
     return u.view(np.float32).astype(np.float64)
 
 
+def pool_rows(pool_bits: np.ndarray) -> np.ndarray:
+    """Undo the documented row layout of a KV pool [pages, Hkv, P, d]: the library stores the
+    16-byte piece j of the row in slot r at position (j & ~7) | ((j & 7) ^ (r & 7))."""
+    pages, hkv, P, d = pool_bits.shape
+    pieces = pool_bits.reshape(pages, hkv, P, d // 8, 8)
+    out = np.empty_like(pieces)
+    for r in range(P):
+        j = np.arange(d // 8)
+        out[:, :, r, j] = pieces[:, :, r, (j & ~7) | ((j & 7) ^ (r & 7))]
+    return out.reshape(pages, hkv, P, d)
+
+
 def assert_attention_close(got_bits: np.ndarray, want: np.ndarray, what: str = "") -> None:
     """GPU bf16 output vs the unrounded fp64 oracle.
 

@@ -4,7 +4,7 @@ mean-abs 1e-3 of the unrounded fp64 result."""
 import numpy as np
 import pytest
 
-from _util import assert_attention_close
+from _util import assert_attention_close, pool_rows
 from oracle import attention as oa
 from oracle import plan as op
 from paper_2605_23296_b200 import workloads as wl
@@ -75,7 +75,7 @@ def test_append_bit_exact(make):
         ks.append(w.k_dec[t])
         vs.append(w.v_dec[t])
     kp, vp, written = oa.expected_pool(slots, np.concatenate(ks), np.concatenate(vs), w.num_pages, w.page_size)
-    got_k, got_v = _bits(s.k_pool), _bits(s.v_pool)
+    got_k, got_v = pool_rows(_bits(s.k_pool)), pool_rows(_bits(s.v_pool))
     mask = np.broadcast_to(written[:, None, :, None], got_k.shape)
     assert np.array_equal(got_k[mask], kp[mask]) and np.array_equal(got_v[mask], vp[mask])
     # slots nobody owns still hold the poison pattern
@@ -101,8 +101,8 @@ def test_append_general_lengths_and_capacity_error():
     plan = op.build_plan(w.block_lens.tolist(), 20, 16, w.free_pages.tolist(), 2, 128, 1)
     kp, vp, written = oa.expected_pool(plan["slot_mapping"], w.k, w.v, w.num_pages, 16)
     mask = np.broadcast_to(written[:, None, :, None], kp.shape)
-    assert np.array_equal(_bits(s.k_pool)[mask], kp[mask])
-    assert np.array_equal(_bits(s.v_pool)[mask], vp[mask])
+    assert np.array_equal(pool_rows(_bits(s.k_pool))[mask], kp[mask])
+    assert np.array_equal(pool_rows(_bits(s.v_pool))[mask], vp[mask])
     # growing a block past L_b + T is refused on the host, nothing is launched
     too_many = np.array([21, 0, 0], dtype=np.int32)
     junk = _dev(w.k[:21])
