@@ -28,6 +28,9 @@ METRIC = "summary tok/s at B blocks (attention only: prefill + paged decode)"
 UNIT = "tok/s"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 NOMINAL_HBM_GBS = 8000.0
+# dram__bytes_read.sum + dram__bytes_write.sum of one decode_split_kernel launch (134.93 MB + 3.9 MB),
+# profiler capture of the kernel as it stands; None for workloads that were not captured
+DECODE_DRAM_BYTES_PER_LAUNCH = {"dense8b": 138.8e6}
 NOMINAL_BF16_TFLOPS = 2250.0
 
 
@@ -376,9 +379,11 @@ def run_gpu(args) -> None:
         samp_bytes = total_kv / T
         samp_ms = dc_ms / T
     achieved = samp_bytes / (samp_ms * 1e-3) / 1e9
-    # DRAM bytes per launch are not quoted here: consecutive launches share L2 contents (the scan
-    # direction alternates), so a per-launch figure depends on the profiler's cache control
-    traffic = None
+    # DRAM bytes per launch (read + written) from a profiler capture of this kernel on the default
+    # workload; the capture replays each launch with a cold L2, whereas consecutive launches of a
+    # real step share L2 contents (the scan direction alternates), so this is the upper figure
+    overridden = args.blocks or args.block_len or args.decode_steps or args.pages_per_split or args.separate_append
+    traffic = DECODE_DRAM_BYTES_PER_LAUNCH.get(args.config) if not overridden else None
     roofline = {"bound": "hbm", "kernel": "decode_split_kernel (one launch per step: append, split-K scan and merge fused)",
                 "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                 "frac": achieved / peaks["hbm_gbs"], "peak_kind": f"of {peak_kind}",

@@ -7,17 +7,21 @@
 //   warps 0-3  softmax + epilogue of sub-tile 0: thread r owns query row r (TMEM lane r), so
 //   warps 4-7  ... of sub-tile 1                 row max and row sum need no shuffles
 //   warp 8     TMA producer (one elected lane): both Q sub-tiles once, then K and V tiles of
-//              128 keys through two-stage rings
+//              128 keys through rings of two (head_dim 128) or four (head_dim 64) stages
 //   warp 9     MMA issuer (one elected lane) and owner of the TMEM allocation
 //   warps 10-11 idle; they complete the third warpgroup so that its registers can be handed
 //              to the softmax warpgroups (setmaxnreg works on whole warpgroups)
-// TMEM columns: S_u at u*128 (fp32 scores of sub-tile u), O_u at 256 + u*128.
-// Per KV tile j and sub-tile u:
-//                  S_u  = Q_u K_j^T            (both operands K-major in shared memory)
-//                  P_u  = exp2(scale*S_u - m)  (registers -> bf16 -> TMEM, over S_u's first 64 columns)
-//                  O_u += P_u V_j              (A = P_u from TMEM, B = V MN-major in shared memory)
-// The issuer alternates the sub-tiles: PV_0(j), QK_0(j+1), PV_1(j), QK_1(j+1), ... so while
-// one warpgroup does its softmax the tensor core runs the other sub-tile's MMAs.  O stays in
+// Per KV tile j and sub-tile u (a "step"; steps are numbered n = n_sub*j + u):
+//                  S    = Q_u K_j^T            (both operands K-major in shared memory)
+//                  P    = exp2(scale*S - m)    (registers -> bf16 -> TMEM, over the first 64 columns of S)
+//                  O_u += P V_j                (A = P from TMEM, B = V MN-major in shared memory)
+// TMEM holds NBUF score buffers of 128 fp32 columns and the two O_u accumulators behind them;
+// step n uses score buffer n mod NBUF.  head_dim 128 has room for two buffers (one per
+// sub-tile), head_dim 64 for three.  The issuer queues PV(n), then QK(n + NBUF) into the buffer
+// PV(n) has just read: MMAs of one thread execute in issue order, so that is safe, and while
+// one warpgroup does its softmax the tensor core runs the other sub-tile's MMAs.  With three
+// buffers the scores of a sub-tile's next KV tile are computed while its warpgroup is still
+// busy with the current one, so neither side waits for the other's round trip.  O stays in
 // TMEM across tiles; it is rescaled only when a row's running max grows by more than 2^8
 // (the stale max is used meanwhile, which is exact after the final division by the row sum).
 //
@@ -88,13 +92,16 @@ __device__ __forceinline__ void tc_commit(uint32_t bar, uint32_t leader) {
                  " @q tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n}\n"
                  :: "r"(bar), "r"(leader) : "memory");
 }
-// D[tmem] (+)= A[smem desc] * B[smem desc]; `accumulate` = 0 overwrites D.
-__device__ __forceinline__ void tc_mma_ss(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate,
-                                          uint32_t leader) {
+// D[tmem] (+)= A[smem desc] * B[smem desc]; `accumulate` = 0 overwrites D.  The descriptors are given
+// as 32-bit halves: `a_lo` / `b_lo` carry the start address (and the leading-dimension field), `hi`
+// is common to both operands; advancing an operand is one 32-bit add.
+__device__ __forceinline__ void tc_mma_ss_lo(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t hi, uint32_t idesc,
+                                             uint32_t accumulate, uint32_t leader) {
     asm volatile(
-        "{\n .reg .pred p, q;\n setp.ne.b32 p, %4, 0;\n setp.ne.b32 q, %5, 0;\n"
-        " @q tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}\n"
-        :: "r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(leader) : "memory");
+        "{\n .reg .pred p, q;\n .reg .b64 da, db;\n setp.ne.b32 p, %5, 0;\n setp.ne.b32 q, %6, 0;\n"
+        " mov.b64 da, {%1, %3};\n mov.b64 db, {%2, %3};\n"
+        " @q tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %4, p;\n}\n"
+        :: "r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(hi), "r"(idesc), "r"(accumulate), "r"(leader) : "memory");
 }
 // 32 consecutive fp32 columns of this thread's TMEM lane.
 __device__ __forceinline__ void tc_ld32(uint32_t taddr, float (&v)[32]) {
@@ -153,12 +160,13 @@ __host__ __device__ constexpr uint32_t instr_desc(int M, int N, bool b_mn_major)
 
 // D[tmem] (+)= A[tmem] * B[smem desc]: A is a 128-lane x 16-element bf16 slice held in TMEM
 // (two consecutive K elements per 32-bit column, row = lane).
-__device__ __forceinline__ void tc_mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc, uint32_t accumulate,
-                                          uint32_t leader) {
+__device__ __forceinline__ void tc_mma_ts_lo(uint32_t d_tmem, uint32_t a_tmem, uint32_t b_lo, uint32_t b_hi, uint32_t idesc,
+                                             uint32_t accumulate, uint32_t leader) {
     asm volatile(
-        "{\n .reg .pred p, q;\n setp.ne.b32 p, %4, 0;\n setp.ne.b32 q, %5, 0;\n"
-        " @q tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n}\n"
-        :: "r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(leader) : "memory");
+        "{\n .reg .pred p, q;\n .reg .b64 db;\n setp.ne.b32 p, %5, 0;\n setp.ne.b32 q, %6, 0;\n"
+        " mov.b64 db, {%2, %3};\n"
+        " @q tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], db, %4, p;\n}\n"
+        :: "r"(d_tmem), "r"(a_tmem), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accumulate), "r"(leader) : "memory");
 }
 // 32 consecutive 32-bit columns of this thread's TMEM lane, no wait (pair with tc_wait_ld).
 __device__ __forceinline__ void tc_ld32_nowait(uint32_t taddr, uint32_t (&r)[32]) {
@@ -184,6 +192,15 @@ __device__ __forceinline__ void add_bf16x2(float& acc, uint32_t w) {
     asm("{\n .reg .b16 lo, hi;\n mov.b32 {lo, hi}, %1;\n add.rn.f32.bf16 %0, lo, %0;\n add.rn.f32.bf16 %0, hi, %0;\n}\n"
         : "+f"(acc) : "r"(w));
 }
+// (a, b) = (a, b) * s + c in one packed fp32 instruction
+__device__ __forceinline__ void fma_x2(float& a, float& b, float s, float c) {
+    uint64_t in, sc, cc, out;
+    asm("mov.b64 %0, {%1, %2};\n" : "=l"(in) : "f"(a), "f"(b));
+    asm("mov.b64 %0, {%1, %1};\n" : "=l"(sc) : "f"(s));
+    asm("mov.b64 %0, {%1, %1};\n" : "=l"(cc) : "f"(c));
+    asm("fma.rn.f32x2 %0, %1, %2, %3;\n" : "=l"(out) : "l"(in), "l"(sc), "l"(cc));
+    asm("mov.b64 {%0, %1}, %2;\n" : "=f"(a), "=f"(b) : "l"(out));
+}
 __device__ __forceinline__ float max3(float a, float b, float c) {
     float d;
     asm("max.f32 %0, %1, %2, %3;\n" : "=f"(d) : "f"(a), "f"(b), "f"(c));
@@ -191,31 +208,47 @@ __device__ __forceinline__ float max3(float a, float b, float c) {
 }
 __device__ __forceinline__ void wg_sync(int id) { asm volatile("bar.sync %0, 128;\n" :: "r"(id) : "memory"); }
 
+constexpr int kMaxStages = 4, kMaxBufs = 3;
 struct __align__(8) TcBarriers {
-    uint64_t q_full[2], k_full[2], k_empty[2], v_full[2], v_empty[2], s_full[2], p_full[2], pv_done[2];
+    uint64_t q_full[2], k_full[kMaxStages], k_empty[kMaxStages], v_full[kMaxStages], v_empty[kMaxStages];
+    uint64_t s_full[kMaxBufs], p_full[kMaxBufs], pv_done[2];
     uint32_t tmem_base;
 };
 
 // One CTA = one (block, q item of `q_rows` = 128 or 256 rows, query head).  A 256-row item is
 // two 128-row sub-tiles u = 0, 1 that share every K/V tile; sub-tile u has its own softmax
-// warpgroup, its own S_u / O_u columns in TMEM, and sees KV tiles 0 .. t0+u (t0 = index of
+// warpgroup and its own O_u columns in TMEM, and sees KV tiles 0 .. t0+u (t0 = index of
 // sub-tile 0 in units of 128 rows; the last of them touches the diagonal).
+template <int D>
+struct TcShape {
+    static constexpr int NB = D / 64;                          // 64-wide column blocks of a Q/K/V tile
+    static constexpr uint32_t kTileBytes = NB * kBlockBytes;   // one Q sub-tile, K tile or V tile
+    static constexpr int kBufs = (D == 64) ? 3 : 2;            // score buffers in TMEM
+    static constexpr int kStages = (D == 64) ? 4 : 2;          // K ring and V ring depth
+    static constexpr uint32_t kColO = kBufs * 128;             // O_u at kColO + u*D
+    static constexpr uint32_t kTmemCols = 512;
+    static constexpr int kSmem = (2 + 2 * kStages) * (int)kTileBytes + 1024;   // Q sub-tiles + rings + alignment slack
+    static_assert(kColO + 2 * D <= kTmemCols, "TMEM layout");
+    static_assert(kBufs <= kMaxBufs && kStages <= kMaxStages, "barrier arrays");
+};
+
 template <int D>
 __global__ void __launch_bounds__(kThreads, 1)
 prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                   const __grid_constant__ CUtensorMap tm_v, __nv_bfloat16* __restrict__ o, cpa_dev_index ix, int Hq,
                   int Hkv, int q_rows, float scale_log2) {
-    constexpr int NB = D / 64;                         // 64-wide column blocks of a Q/K/V tile
-    constexpr uint32_t kTileBytes = NB * kBlockBytes;  // one Q sub-tile, K tile or V tile
-    constexpr uint32_t kTmemCols = 512;
-    constexpr uint32_t kColO = 256;                    // S_u at u*128 (P_u aliases its first 64 columns), O_u at 256 + u*128
+    using Sh = TcShape<D>;
+    constexpr int NB = Sh::NB;
+    constexpr uint32_t kTileBytes = Sh::kTileBytes;
+    constexpr int NBUF = Sh::kBufs, KS = Sh::kStages;
+    constexpr uint32_t kColO = Sh::kColO;
     extern __shared__ unsigned char dsm_raw[];
     __shared__ TcBarriers bars;
 
     const uint32_t base = (smem_u32(dsm_raw) + 1023u) & ~1023u;
     const uint32_t s_q = base;                       // two sub-tiles
-    const uint32_t s_k = s_q + 2 * kTileBytes;       // two stages
-    const uint32_t s_v = s_k + 2 * kTileBytes;       // two stages
+    const uint32_t s_k = s_q + 2 * kTileBytes;       // KS stages
+    const uint32_t s_v = s_k + KS * kTileBytes;      // KS stages
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int b = ix.prefill_items[2 * blockIdx.x], item = ix.prefill_items[2 * blockIdx.x + 1];
@@ -232,20 +265,24 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
     if (threadIdx.x == 0) {
         for (int u = 0; u < 2; ++u) {
             mbar_init(bar(&bars.q_full[u]), 1);
-            mbar_init(bar(&bars.k_full[u]), 1);
-            mbar_init(bar(&bars.k_empty[u]), 1);
-            mbar_init(bar(&bars.v_full[u]), 1);
-            mbar_init(bar(&bars.v_empty[u]), 1);
-            mbar_init(bar(&bars.s_full[u]), 1);
-            mbar_init(bar(&bars.p_full[u]), 128);
             mbar_init(bar(&bars.pv_done[u]), 1);
+        }
+        for (int s = 0; s < KS; ++s) {
+            mbar_init(bar(&bars.k_full[s]), 1);
+            mbar_init(bar(&bars.k_empty[s]), 1);
+            mbar_init(bar(&bars.v_full[s]), 1);
+            mbar_init(bar(&bars.v_empty[s]), 1);
+        }
+        for (int i = 0; i < NBUF; ++i) {
+            mbar_init(bar(&bars.s_full[i]), 1);
+            mbar_init(bar(&bars.p_full[i]), 128);
         }
         asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory");
     }
     if (warp == 9) {  // TMEM allocation is warp-wide
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;\n"
-                     :: "r"(smem_u32(&bars.tmem_base)), "r"(kTmemCols) : "memory");
+                     :: "r"(smem_u32(&bars.tmem_base)), "r"(Sh::kTmemCols) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;\n" ::: "memory");
     }
     tc_fence_before();
@@ -268,8 +305,8 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                                 bar(&bars.q_full[u]));
             }
             for (int j = 0; j < n_total; ++j) {
-                const int s = j & 1;
-                const uint32_t par = (uint32_t)(j >> 1) & 1u;
+                const int s = j % KS;
+                const uint32_t par = (uint32_t)(j / KS) & 1u;
                 const int row = tok0 + j * kTileN;
                 mbar_wait(bar(&bars.k_empty[s]), par ^ 1u, dead, ix.status);
                 mbar_expect_tx(bar(&bars.k_full[s]), kTileBytes);
@@ -285,70 +322,104 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
         }
     } else if (warp == 9) {
         // ------------------------------------------------------------ MMA issuer (whole warp, one lane issues)
-        {
-            const uint32_t leader = (lane == 0);
-            constexpr uint32_t idesc_qk = instr_desc(kTileM, kTileN, false);
-            constexpr uint32_t idesc_pv = instr_desc(kTileM, D, true);
-            // Descriptors are built once; inside the loops an operand advances by adding a constant
-            // to the descriptor's address field (units of 16 bytes), which keeps the issuing thread's
-            // instruction count per MMA small: it shares its scheduler with softmax warps.
-            const uint64_t dq0 = smem_desc(s_q, 16, 1024), dk0 = smem_desc(s_k, 16, 1024);
-            const uint64_t dv0 = smem_desc(s_v, kBlockBytes, 1024);
-            auto issue_qk = [&](int u, int j) {   // S_u = Q_u K_j^T
-                const uint64_t dq = dq0 + (uint64_t)((u * kTileBytes) >> 4);
-                const uint64_t dk = dk0 + (uint64_t)(((j & 1) * kTileBytes) >> 4);
-                const uint32_t d_tmem = tmem + u * 128;
+        // Everything the issuing thread executes between two MMAs delays the tensor core, so the
+        // loops below are written out per case with as little index arithmetic as possible.
+        const uint32_t leader = (lane == 0);
+        constexpr uint32_t idesc_qk = instr_desc(kTileM, kTileN, false);
+        constexpr uint32_t idesc_pv = instr_desc(kTileM, D, true);
+        constexpr uint32_t kTile16 = kTileBytes >> 4;        // descriptor address units are 16 bytes
+        // Descriptors are kept as 32-bit halves; an operand advances by adding a constant to the low half.
+        const uint64_t dqk = smem_desc(0, 16, 1024), dvv = smem_desc(0, kBlockBytes, 1024);
+        const uint32_t qk_hi = (uint32_t)(dqk >> 32), pv_hi = (uint32_t)(dvv >> 32);
+        const uint32_t q_lo = (uint32_t)dqk | (s_q >> 4), k_lo = (uint32_t)dqk | (s_k >> 4), v_lo = (uint32_t)dvv | (s_v >> 4);
+        auto qk = [&](int u, int buf, int ks) {   // S[buf] = Q_u K[stage ks]^T
+            const uint32_t a = q_lo + u * kTile16, bq = k_lo + ks * kTile16, d_tmem = tmem + buf * 128;
 #pragma unroll
-                for (int k = 0; k < D / 16; ++k) {
-                    // 16 head dims per instruction: 32 B inside the 128-B swizzled row, next block after 4 steps
-                    constexpr uint32_t kBlk = kBlockBytes >> 4;
-                    const uint32_t off = (k >> 2) * kBlk + (k & 3) * 2;
-                    tc_mma_ss(d_tmem, dq + off, dk + off, idesc_qk, k > 0, leader);
-                }
-                tc_commit(bar(&bars.s_full[u]), leader);
-            };
-            auto issue_pv = [&](int u, int j) {   // O_u += P_u V_j, P_u read from TMEM (aliases S_u)
-                const uint64_t dv = dv0 + (uint64_t)(((j & 1) * kTileBytes) >> 4);
-                const uint32_t d_tmem = tmem + kColO + u * 128, a_tmem = tmem + u * 128;
-                const uint32_t acc0 = j > 0;
-#pragma unroll
-                for (int k = 0; k < kTileN / 16; ++k)
-                    // 16 keys per instruction: 8 TMEM columns of A; 16 rows of 128 B of V, column blocks kBlockBytes apart
-                    tc_mma_ts(d_tmem, a_tmem + k * 8, dv + k * (2048 >> 4), idesc_pv, k > 0 ? 1u : acc0, leader);
-            };
-            // MMAs issued by this one thread execute in issue order, so QK_u(j+1) may be queued right
-            // behind PV_u(j) although it overwrites the columns PV_u(j) reads P_u from.
-            mbar_wait(bar(&bars.k_full[0]), 0, dead, ix.status);
-            for (int u = 0; u < n_sub; ++u) {
-                mbar_wait(bar(&bars.q_full[u]), 0, dead, ix.status);
-                tc_fence_after();
-                issue_qk(u, 0);
+            for (int k = 0; k < D / 16; ++k) {
+                // 16 head dims per instruction: 32 B inside the 128-B swizzled row, next block after 4 steps
+                const uint32_t off = (k >> 2) * (kBlockBytes >> 4) + (k & 3) * 2;
+                tc_mma_ss_lo(d_tmem, a + off, bq + off, qk_hi, idesc_qk, k > 0, leader);
             }
+            tc_commit(bar(&bars.s_full[buf]), leader);
+        };
+        auto pv = [&](int u, int buf, uint32_t par, int vs, uint32_t acc0) {   // O_u += P[buf] V[stage vs]
+            mbar_wait(bar(&bars.p_full[buf]), par, dead, ix.status);
+            tc_fence_after();
+            const uint32_t bv = v_lo + vs * kTile16, d_tmem = tmem + kColO + u * D, a_tmem = tmem + buf * 128;
+#pragma unroll
+            for (int k = 0; k < kTileN / 16; ++k)
+                // 16 keys per instruction: 8 TMEM columns of A; 16 rows of 128 B of V, column blocks kBlockBytes apart
+                tc_mma_ts_lo(d_tmem, a_tmem + k * 8, bv + k * (2048 >> 4), pv_hi, idesc_pv, k > 0 ? 1u : acc0, leader);
+        };
+        auto wait_k = [&](int j) {
+            mbar_wait(bar(&bars.k_full[j % KS]), (uint32_t)(j / KS) & 1u, dead, ix.status);
+            tc_fence_after();
+        };
+        auto wait_v = [&](int j) { mbar_wait(bar(&bars.v_full[j % KS]), (uint32_t)(j / KS) & 1u, dead, ix.status); };
+        // Steps are numbered n = n_sub*j + u (KV tile j, sub-tile u); step n uses score buffer n mod NBUF,
+        // and QK(n + NBUF) is queued right behind PV(n), which reads the buffer it overwrites.
+        if (n_sub == 2) {
+            // step 2j uses buffer b0, step 2j+1 buffer b1; par = parity of that buffer's use count
+            int b0 = 0, b1 = 1;
+            uint32_t par0 = 0, par1 = 0;
+            mbar_wait(bar(&bars.q_full[0]), 0, dead, ix.status);
+            mbar_wait(bar(&bars.q_full[1]), 0, dead, ix.status);
+            wait_k(0);
+            qk(0, 0, 0);
+            qk(1, 1, 0);
             tc_commit(bar(&bars.k_empty[0]), leader);
-            for (int j = 0; j < n_total; ++j) {
-                const int s = j & 1;
-                bool have_v = false, have_k = false;
-                for (int u = 0; u < n_sub; ++u) {
-                    const int n_kv = t0 + 1 + u;
-                    if (j < n_kv) {
-                        if (!have_v) { mbar_wait(bar(&bars.v_full[s]), (uint32_t)(j >> 1) & 1u, dead, ix.status); have_v = true; }
-                        mbar_wait(bar(&bars.p_full[u]), (uint32_t)j & 1u, dead, ix.status);
-                        tc_fence_after();
-                        issue_pv(u, j);
-                        if (j == n_kv - 1) tc_commit(bar(&bars.pv_done[u]), leader);
-                    }
-                    if (j + 1 < n_kv) {
-                        if (!have_k) {
-                            mbar_wait(bar(&bars.k_full[s ^ 1]), (uint32_t)((j + 1) >> 1) & 1u, dead, ix.status);
-                            tc_fence_after();
-                            have_k = true;
-                        }
-                        issue_qk(u, j + 1);
-                    }
+            if (NBUF == 3 && t0 >= 1) { wait_k(1); qk(0, 2, 1 % KS); }
+            for (int j = 0; j <= t0; ++j) {      // tiles both sub-tiles have; sub-tile 1 also has tile t0+1
+                const int vs = j % KS, k1 = (j + 1) % KS;
+                wait_v(j);
+                pv(0, b0, par0, vs, j > 0);
+                if (j == t0) tc_commit(bar(&bars.pv_done[0]), leader);
+                if (NBUF == 2) {                 // buffer b0 next holds step 2j+2 = (sub-tile 0, tile j+1)
+                    if (j < t0) { wait_k(j + 1); qk(0, b0, k1); }
+                } else {                         // buffer b0 next holds step 2j+3 = (sub-tile 1, tile j+1)
+                    if (j == t0) wait_k(j + 1);  // otherwise (sub-tile 0, tile j+1) has been issued already
+                    qk(1, b0, k1);
+                    tc_commit(bar(&bars.k_empty[k1]), leader);    // sub-tile 1 is the last reader of a K tile
                 }
-                tc_commit(bar(&bars.v_empty[s]), leader);
-                if (j + 1 < n_total) tc_commit(bar(&bars.k_empty[s ^ 1]), leader);
+                pv(1, b1, par1, vs, j > 0);
+                tc_commit(bar(&bars.v_empty[vs]), leader);
+                if (NBUF == 2) {                 // buffer b1 next holds step 2j+3 = (sub-tile 1, tile j+1)
+                    if (j == t0) wait_k(j + 1);
+                    qk(1, b1, k1);
+                    tc_commit(bar(&bars.k_empty[k1]), leader);
+                } else if (j + 2 <= t0) {        // buffer b1 next holds step 2j+4 = (sub-tile 0, tile j+2)
+                    wait_k(j + 2);
+                    qk(0, b1, (j + 2) % KS);
+                }
+                b0 += 2; if (b0 >= NBUF) { b0 -= NBUF; par0 ^= 1u; }
+                b1 += 2; if (b1 >= NBUF) { b1 -= NBUF; par1 ^= 1u; }
             }
+            wait_v(t0 + 1);
+            pv(1, b1, par1, (t0 + 1) % KS, 1u);
+            tc_commit(bar(&bars.pv_done[1]), leader);
+        } else {
+            // one sub-tile: step n = tile n; with two or three buffers the scores run ahead of the softmax
+            mbar_wait(bar(&bars.q_full[0]), 0, dead, ix.status);
+            for (int i = 0; i < NBUF && i <= t0; ++i) {
+                wait_k(i);
+                qk(0, i, i % KS);
+                tc_commit(bar(&bars.k_empty[i % KS]), leader);
+            }
+            int buf = 0;
+            uint32_t par = 0;
+            for (int j = 0; j <= t0; ++j) {
+                const int vs = j % KS;
+                wait_v(j);
+                pv(0, buf, par, vs, j > 0);
+                tc_commit(bar(&bars.v_empty[vs]), leader);
+                if (j + NBUF <= t0) {
+                    wait_k(j + NBUF);
+                    qk(0, buf, (j + NBUF) % KS);
+                    tc_commit(bar(&bars.k_empty[(j + NBUF) % KS]), leader);
+                }
+                if (++buf == NBUF) { buf = 0; par ^= 1u; }
+            }
+            tc_commit(bar(&bars.pv_done[0]), leader);
         }
     }
     } else {
@@ -358,15 +429,15 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
         const int u = warp >> 2;
         const int r = threadIdx.x & 127;                                  // query row inside the sub-tile = TMEM lane
         const uint32_t lane_addr = ((uint32_t)((warp & 3) * 32) << 16);   // this warp's 32 TMEM lanes
-        const uint32_t t_s = tmem + lane_addr + u * 128;
-        const uint32_t t_o = tmem + lane_addr + kColO + u * 128;
+        const uint32_t t_o = tmem + lane_addr + kColO + u * D;
         const int n_kv = t0 + 1 + u;
         float m_used = -INFINITY;   // row max the weights are currently scaled with (log2 units)
         float l_run = 0.f;
+        int buf = u;                // score buffer of this sub-tile's step n = n_sub*j + u, i.e. n mod NBUF
+        uint32_t par = 0;           // parity of that buffer's use count
         for (int j = 0; j < n_kv; ++j) {
-            // s_full(j) also means PV_u(j-1) has completed (the commit covers every earlier MMA):
-            // O_u is settled and the P_u columns may be overwritten
-            mbar_wait(bar(&bars.s_full[u]), (uint32_t)j & 1u, dead, ix.status);
+            const uint32_t t_s = tmem + lane_addr + buf * 128;
+            mbar_wait(bar(&bars.s_full[buf]), par, dead, ix.status);
             tc_fence_after();
             const bool diag = (j == n_kv - 1);
             uint32_t sv[4][32];
@@ -402,6 +473,11 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                 m_used = mx;
             }
             if (j > 0 && __any_sync(0xffffffffu, alpha != 1.f)) {
+                // O_u must hold every earlier tile before it is rescaled, and the scores of this tile may
+                // have been ready before PV of the previous one has run.  The release of V tile j-1 is
+                // committed behind the last PV that reads it, which is issued after PV_u(j-1).
+                mbar_wait(bar(&bars.v_empty[(j - 1) % KS]), (uint32_t)((j - 1) / KS) & 1u, dead, ix.status);
+                tc_fence_after();
 #pragma unroll
                 for (int c = 0; c < D / 32; ++c) {
                     float v[32];
@@ -412,16 +488,17 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                 }
             }
             l_run *= alpha;
-            // weights, rounded to bf16, two keys per 32-bit TMEM column (P_u over the first 64 columns of S_u)
+            // weights, rounded to bf16, two keys per 32-bit TMEM column (P over the first 64 columns of S)
             float sum[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+            const float neg_m = -m_used;
 #pragma unroll
             for (int c = 0; c < 4; ++c) {
                 uint32_t pk[16];
 #pragma unroll
                 for (int i = 0; i < 32; i += 2) {
-                    const float p0 = exp2f(fmaf(__uint_as_float(sv[c][i]), scale_log2, -m_used));
-                    const float p1 = exp2f(fmaf(__uint_as_float(sv[c][i + 1]), scale_log2, -m_used));
-                    const uint32_t w = pack_bf16(p0, p1);
+                    float x0 = __uint_as_float(sv[c][i]), x1 = __uint_as_float(sv[c][i + 1]);
+                    fma_x2(x0, x1, scale_log2, neg_m);
+                    const uint32_t w = pack_bf16(exp2f(x0), exp2f(x1));
                     pk[i >> 1] = w;
                     // row sum over the rounded weights (numerator and denominator stay consistent);
                     // the bf16 halves are added to the fp32 sum directly
@@ -432,7 +509,9 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
             l_run += ((sum[0] + sum[1]) + (sum[2] + sum[3])) + ((sum[4] + sum[5]) + (sum[6] + sum[7]));
             tc_wait_st();
             tc_fence_before();
-            mbar_arrive(bar(&bars.p_full[u]));
+            mbar_arrive(bar(&bars.p_full[buf]));
+            buf += n_sub;
+            if (buf >= NBUF) { buf -= NBUF; par ^= 1u; }
         }
         // ---- epilogue: O / l -> bf16 -> this sub-tile's (now idle) Q buffer -> coalesced stores
         mbar_wait(bar(&bars.pv_done[u]), 0, dead, ix.status);
@@ -477,7 +556,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
     __syncthreads();
     if (warp == 9) {
         tc_fence_after();
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;\n" :: "r"(tmem), "r"(kTmemCols) : "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;\n" :: "r"(tmem), "r"(Sh::kTmemCols) : "memory");
     }
 }
 
@@ -517,8 +596,7 @@ bool make_map(CUtensorMap* map, const void* ptr, int64_t rows, int64_t cols) {
 template <int D>
 int launch_prefill_tc(const cpa_plan* plan, const void* q, const void* k, const void* v, void* o, cudaStream_t st) {
     const cpa_config& c = plan->cfg;
-    constexpr int NB = D / 64;
-    constexpr int smem = 6 * NB * (int)kBlockBytes + 1024;   // 2 Q sub-tiles + 2 K + 2 V tiles, alignment slack
+    constexpr int smem = TcShape<D>::kSmem;
     static bool configured_dev[64] = {};  // the attribute is per device: remember which devices have it
     int dev_id = 0;
     if (cudaGetDevice(&dev_id) != cudaSuccess || dev_id < 0 || dev_id >= 64) {
