@@ -16,7 +16,7 @@ struct cpa_dev_index {
     int32_t* seq_lens_next;        // [B]   the other length buffer: a fused decode+append writes the new lengths here
     int32_t* append_indptr;        // [B+1] source-row offsets of a general append
     const int32_t* page_indices;   // [pages_used]
-    const int32_t* prefill_items;  // [n_prefill, 2]
+    const int32_t* prefill_items;  // [n_prefill, 4]: (block, q item, first token of the block, block length), 16-byte aligned
     const int32_t* decode_items;   // [n_decode, item_stride]: (block, kv_head, split, pages, split size, 0, 0, 0) + page ids
     int32_t* merge_tickets;        // [B * Hkv] arrival counters of the fused split merge (zero between launches)
     int32_t item_stride;           // int32 words per decode item: 8 + largest split size rounded up to 4

@@ -151,7 +151,7 @@ extern "C" int cpa_plan_create(const cpa_config* cfg, int32_t num_blocks, const 
     p->off_seqlens = w; w = align4(w + B);
     p->off_append = w;  w = align4(w + B + 1);
     p->off_pidx = w;    w = align4(w + pages_used);
-    p->off_pitems = w;  w = align4(w + 2LL * p->n_prefill);
+    p->off_pitems = w;  w = align4(w + 4LL * p->n_prefill);
     p->item_stride = 8 + (p->C + 3) / 4 * 4;
     p->off_ditems = w;  w = align4(w + (int64_t)p->item_stride * p->n_decode);
     p->off_tickets = w; w = align4(w + (int64_t)B * cfg->num_kv_heads);
@@ -163,7 +163,15 @@ extern "C" int cpa_plan_create(const cpa_config* cfg, int32_t num_blocks, const 
     std::memcpy(im + p->off_pindptr, p->page_indptr.data(), sizeof(int32_t) * (B + 1));
     std::memcpy(im + p->off_sindptr, p->split_indptr.data(), sizeof(int32_t) * (B + 1));
     std::memcpy(im + p->off_pidx, p->page_indices.data(), sizeof(int32_t) * pages_used);
-    std::memcpy(im + p->off_pitems, p->prefill_items.data(), sizeof(int32_t) * 2 * p->n_prefill);
+    for (int32_t i = 0; i < p->n_prefill; ++i) {
+        // a prefill item carries its block's token range, so a kernel needs one load per item
+        const int32_t b = p->prefill_items[2 * i];
+        int32_t* it = im + p->off_pitems + 4LL * i;
+        it[0] = b;
+        it[1] = p->prefill_items[2 * i + 1];
+        it[2] = p->cu_seqlens[b];
+        it[3] = p->block_lens[b];
+    }
     for (int32_t i = 0; i < p->n_decode; ++i) {
         // a decode item carries its own page ids, so the kernel's first KV load depends on
         // one prior load only

@@ -80,7 +80,7 @@ prefill_mma_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __r
 
     // a work item of subs*128 query rows is covered by `subs` CTAs of 128 rows each
     const int item = blockIdx.x / subs;
-    const int b = ix.prefill_items[2 * item], tile = ix.prefill_items[2 * item + 1] * subs + (blockIdx.x - item * subs);
+    const int b = ix.prefill_items[4 * item], tile = ix.prefill_items[4 * item + 1] * subs + (blockIdx.x - item * subs);
     const int h = blockIdx.y, g = h / (Hq / Hkv);
     const int tok0 = ix.cu_seqlens[b];
     const int L = ix.cu_seqlens[b + 1] - tok0;

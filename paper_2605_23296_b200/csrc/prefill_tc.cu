@@ -2,8 +2,9 @@
 // cores: TMA-staged tiles, tcgen05.mma with accumulators in tensor memory (TMEM), online
 // softmax in fp32 registers.
 //
-// One CTA = one (block, q item, query head); a q item is 256 query rows handled as two
-// 128-row sub-tiles that share every K/V tile.  Twelve warps with fixed roles:
+// One unit of work = one (block, q item, query head); a q item is 256 query rows handled as two
+// 128-row sub-tiles that share every K/V tile.  The grid is persistent (one CTA per SM, each
+// walking its share of the units).  Twelve warps with fixed roles:
 //   warps 0-3  softmax + epilogue of sub-tile 0: thread r owns query row r (TMEM lane r), so
 //   warps 4-7  ... of sub-tile 1                 row max and row sum need no shuffles
 //   warp 8     TMA producer (one elected lane): both Q sub-tiles once, then K and V tiles of
@@ -206,19 +207,16 @@ __device__ __forceinline__ float max3(float a, float b, float c) {
     asm("max.f32 %0, %1, %2, %3;\n" : "=f"(d) : "f"(a), "f"(b), "f"(c));
     return d;
 }
-__device__ __forceinline__ void wg_sync(int id) { asm volatile("bar.sync %0, 128;\n" :: "r"(id) : "memory"); }
 
-constexpr int kMaxStages = 4, kMaxBufs = 3;
+constexpr int kMaxStages = 4;
 struct __align__(8) TcBarriers {
-    uint64_t q_full[2], k_full[kMaxStages], k_empty[kMaxStages], v_full[kMaxStages], v_empty[kMaxStages];
-    uint64_t s_full[kMaxBufs], p_full[kMaxBufs], pv_done[2];
+    uint64_t q_full[2], q_empty[2], k_full[kMaxStages], k_empty[kMaxStages], v_full[kMaxStages], v_empty[kMaxStages];
+    // [sub-tile][that sub-tile's step count mod 4]: at most three steps are ever ahead of a waiter, so a
+    // waiter can never meet the phase after the one it is waiting for
+    uint64_t s_full[2][4], p_full[2][4], pv_done[2];
     uint32_t tmem_base;
 };
 
-// One CTA = one (block, q item of `q_rows` = 128 or 256 rows, query head).  A 256-row item is
-// two 128-row sub-tiles u = 0, 1 that share every K/V tile; sub-tile u has its own softmax
-// warpgroup and its own O_u columns in TMEM, and sees KV tiles 0 .. t0+u (t0 = index of
-// sub-tile 0 in units of 128 rows; the last of them touches the diagonal).
 template <int D>
 struct TcShape {
     static constexpr int NB = D / 64;                          // 64-wide column blocks of a Q/K/V tile
@@ -229,14 +227,30 @@ struct TcShape {
     static constexpr uint32_t kTmemCols = 512;
     static constexpr int kSmem = (2 + 2 * kStages) * (int)kTileBytes + 1024;   // Q sub-tiles + rings + alignment slack
     static_assert(kColO + 2 * D <= kTmemCols, "TMEM layout");
-    static_assert(kBufs <= kMaxBufs && kStages <= kMaxStages, "barrier arrays");
+    static_assert(kBufs <= 3 && kStages <= kMaxStages, "barrier arrays");
 };
 
+// One unit of work = one (block, q item of `q_rows` = 128 or 256 rows, query head).  A 256-row item is
+// two 128-row sub-tiles u = 0, 1 that share every K/V tile; sub-tile u has its own softmax
+// warpgroup and its own O_u columns in TMEM, and sees KV tiles 0 .. t0+u (t0 = index of
+// sub-tile 0 in units of 128 rows; the last of them touches the diagonal).
+struct TcWork {
+    int h, g, tok0, L, q0, t0, n_sub, n_total;   // n_total: KV tiles streamed; sub-tile u uses the first t0+1+u
+    bool valid;                                  // false: this CTA has no unit in that round (last round only)
+};
+
+// The grid is persistent: CTA c takes units c, 2G-1-c, 2G+c, ... (G = grid size; the order of the
+// list is descending cost, so the back-and-forth deal keeps the CTAs' totals within one unit of
+// each other).  Unit w is (item w / Hq, head w % Hq): neighbouring CTAs work on the heads of one
+// item and find its K/V tiles in L2.  Every role walks the same list with its own running
+// counters, so the pipeline never drains between units: the producer is already loading the next
+// unit's Q and K/V, and the issuer its first scores, while a softmax warpgroup still writes the
+// previous unit's output.
 template <int D>
 __global__ void __launch_bounds__(kThreads, 1)
 prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                   const __grid_constant__ CUtensorMap tm_v, __nv_bfloat16* __restrict__ o, cpa_dev_index ix, int Hq,
-                  int Hkv, int q_rows, float scale_log2) {
+                  int Hkv, int q_rows, float scale_log2, int n_work) {
     using Sh = TcShape<D>;
     constexpr int NB = Sh::NB;
     constexpr uint32_t kTileBytes = Sh::kTileBytes;
@@ -251,31 +265,49 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
     const uint32_t s_v = s_k + KS * kTileBytes;      // KS stages
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int b = ix.prefill_items[2 * blockIdx.x], item = ix.prefill_items[2 * blockIdx.x + 1];
-    const int h = blockIdx.y, g = h / (Hq / Hkv);
-    const int tok0 = ix.cu_seqlens[b];
-    const int L = ix.cu_seqlens[b + 1] - tok0;
-    const int q0 = item * q_rows;
-    const int t0 = q0 / kTileM;
-    const int n_sub = (q_rows > kTileM && L - q0 > kTileM) ? 2 : 1;
-    const int n_total = t0 + n_sub;                  // KV tiles the CTA streams; sub-tile u uses the first t0+1+u
+    const int G = gridDim.x, n_rounds = (n_work + G - 1) / G;
+    const int group = Hq / Hkv;
+    // Unit of round k for this CTA.  Every role fetches the next round's item record (one 16-byte
+    // load) while it works on the current unit, so no global load sits between two units.
+    auto fetch = [&](int k, int4& rec, int& h) {
+        const int idx = k * G + ((k & 1) ? G - 1 - (int)blockIdx.x : (int)blockIdx.x);
+        rec = make_int4(0, 0, 0, 0);                  // block length 0: no unit in that round (last round only)
+        h = 0;
+        if (k < n_rounds && idx < n_work) {
+            const int it = idx / Hq;
+            h = idx - it * Hq;
+            rec = __ldg(reinterpret_cast<const int4*>(ix.prefill_items) + it);
+        }
+    };
+    auto decode = [&](const int4& rec, int h, TcWork& w) {
+        w.valid = rec.w > 0;
+        w.h = h;
+        w.g = h / group;
+        w.tok0 = rec.z;
+        w.L = rec.w;
+        w.q0 = rec.y * q_rows;
+        w.t0 = w.q0 / kTileM;
+        w.n_sub = (q_rows > kTileM && w.L - w.q0 > kTileM) ? 2 : 1;
+        w.n_total = w.t0 + w.n_sub;
+    };
 
     auto bar = [&](uint64_t* p) { return smem_u32(p); };
 
     if (threadIdx.x == 0) {
         for (int u = 0; u < 2; ++u) {
             mbar_init(bar(&bars.q_full[u]), 1);
+            mbar_init(bar(&bars.q_empty[u]), 1);
             mbar_init(bar(&bars.pv_done[u]), 1);
+            for (int i = 0; i < 4; ++i) {
+                mbar_init(bar(&bars.s_full[u][i]), 1);
+                mbar_init(bar(&bars.p_full[u][i]), 128);
+            }
         }
         for (int s = 0; s < KS; ++s) {
             mbar_init(bar(&bars.k_full[s]), 1);
             mbar_init(bar(&bars.k_empty[s]), 1);
             mbar_init(bar(&bars.v_full[s]), 1);
             mbar_init(bar(&bars.v_empty[s]), 1);
-        }
-        for (int i = 0; i < NBUF; ++i) {
-            mbar_init(bar(&bars.s_full[i]), 1);
-            mbar_init(bar(&bars.p_full[i]), 128);
         }
         asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory");
@@ -297,27 +329,41 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
     if (warp == 8) {
         // ------------------------------------------------------------ TMA producer
         if (lane == 0) {
-            for (int u = 0; u < n_sub; ++u) {
-                mbar_expect_tx(bar(&bars.q_full[u]), kTileBytes);
+            int kt = 0;                   // K/V tiles loaded so far: stage kt % KS, use count kt / KS
+            uint32_t q_loads[2] = {0, 0};   // loads of Q_u so far
+            TcWork w;
+            int4 rec;
+            int rec_h;
+            fetch(0, rec, rec_h);
+            for (int k = 0; k < n_rounds; ++k) {
+                decode(rec, rec_h, w);
+                fetch(k + 1, rec, rec_h);
+                if (!w.valid) continue;
+                for (int u = 0; u < w.n_sub; ++u) {
+                    // the buffer is free once the last score MMA of its previous unit has run
+                    mbar_wait(bar(&bars.q_empty[u]), (q_loads[u] & 1u) ^ 1u, dead, ix.status);
+                    ++q_loads[u];
+                    mbar_expect_tx(bar(&bars.q_full[u]), kTileBytes);
 #pragma unroll
-                for (int c = 0; c < NB; ++c)
-                    tma_load_2d(s_q + u * kTileBytes + c * kBlockBytes, &tm_q, h * D + 64 * c, tok0 + q0 + u * kTileM,
-                                bar(&bars.q_full[u]));
-            }
-            for (int j = 0; j < n_total; ++j) {
-                const int s = j % KS;
-                const uint32_t par = (uint32_t)(j / KS) & 1u;
-                const int row = tok0 + j * kTileN;
-                mbar_wait(bar(&bars.k_empty[s]), par ^ 1u, dead, ix.status);
-                mbar_expect_tx(bar(&bars.k_full[s]), kTileBytes);
+                    for (int c = 0; c < NB; ++c)
+                        tma_load_2d(s_q + u * kTileBytes + c * kBlockBytes, &tm_q, w.h * D + 64 * c,
+                                    w.tok0 + w.q0 + u * kTileM, bar(&bars.q_full[u]));
+                }
+                for (int j = 0; j < w.n_total; ++j, ++kt) {
+                    const int s = kt % KS;
+                    const uint32_t par = (uint32_t)(kt / KS) & 1u;
+                    const int row = w.tok0 + j * kTileN;
+                    mbar_wait(bar(&bars.k_empty[s]), par ^ 1u, dead, ix.status);
+                    mbar_expect_tx(bar(&bars.k_full[s]), kTileBytes);
 #pragma unroll
-                for (int c = 0; c < NB; ++c)
-                    tma_load_2d(s_k + s * kTileBytes + c * kBlockBytes, &tm_k, g * D + 64 * c, row, bar(&bars.k_full[s]));
-                mbar_wait(bar(&bars.v_empty[s]), par ^ 1u, dead, ix.status);
-                mbar_expect_tx(bar(&bars.v_full[s]), kTileBytes);
+                    for (int c = 0; c < NB; ++c)
+                        tma_load_2d(s_k + s * kTileBytes + c * kBlockBytes, &tm_k, w.g * D + 64 * c, row, bar(&bars.k_full[s]));
+                    mbar_wait(bar(&bars.v_empty[s]), par ^ 1u, dead, ix.status);
+                    mbar_expect_tx(bar(&bars.v_full[s]), kTileBytes);
 #pragma unroll
-                for (int c = 0; c < NB; ++c)
-                    tma_load_2d(s_v + s * kTileBytes + c * kBlockBytes, &tm_v, g * D + 64 * c, row, bar(&bars.v_full[s]));
+                    for (int c = 0; c < NB; ++c)
+                        tma_load_2d(s_v + s * kTileBytes + c * kBlockBytes, &tm_v, w.g * D + 64 * c, row, bar(&bars.v_full[s]));
+                }
             }
         }
     } else if (warp == 9) {
@@ -332,112 +378,151 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
         const uint64_t dqk = smem_desc(0, 16, 1024), dvv = smem_desc(0, kBlockBytes, 1024);
         const uint32_t qk_hi = (uint32_t)(dqk >> 32), pv_hi = (uint32_t)(dvv >> 32);
         const uint32_t q_lo = (uint32_t)dqk | (s_q >> 4), k_lo = (uint32_t)dqk | (s_k >> 4), v_lo = (uint32_t)dvv | (s_v >> 4);
-        auto qk = [&](int u, int buf, int ks) {   // S[buf] = Q_u K[stage ks]^T
-            const uint32_t a = q_lo + u * kTile16, bq = k_lo + ks * kTile16, d_tmem = tmem + buf * 128;
+        uint32_t n_qk[2] = {0, 0}, n_pv[2] = {0, 0};   // score / PV steps issued so far per sub-tile (they pick the barrier)
+        uint32_t q_uses[2] = {0, 0};                    // units that used Q_u so far
+        int kt0 = 0;                                    // K/V tiles of earlier units
+        auto qk = [&](int u, int buf, int kt) {   // S[buf] = Q_u K[tile kt]^T
+            const uint32_t a = q_lo + u * kTile16, bq = k_lo + (kt % KS) * kTile16, d_tmem = tmem + buf * 128;
 #pragma unroll
             for (int k = 0; k < D / 16; ++k) {
                 // 16 head dims per instruction: 32 B inside the 128-B swizzled row, next block after 4 steps
                 const uint32_t off = (k >> 2) * (kBlockBytes >> 4) + (k & 3) * 2;
                 tc_mma_ss_lo(d_tmem, a + off, bq + off, qk_hi, idesc_qk, k > 0, leader);
             }
-            tc_commit(bar(&bars.s_full[buf]), leader);
+            tc_commit(bar(&bars.s_full[u][n_qk[u] & 3u]), leader);
+            ++n_qk[u];
         };
-        auto pv = [&](int u, int buf, uint32_t par, int vs, uint32_t acc0) {   // O_u += P[buf] V[stage vs]
-            mbar_wait(bar(&bars.p_full[buf]), par, dead, ix.status);
+        auto pv = [&](int u, int buf, int kt, uint32_t acc0) {   // O_u += P[buf] V[tile kt]
+            mbar_wait(bar(&bars.p_full[u][n_pv[u] & 3u]), (n_pv[u] >> 2) & 1u, dead, ix.status);
+            ++n_pv[u];
             tc_fence_after();
-            const uint32_t bv = v_lo + vs * kTile16, d_tmem = tmem + kColO + u * D, a_tmem = tmem + buf * 128;
+            const uint32_t bv = v_lo + (kt % KS) * kTile16, d_tmem = tmem + kColO + u * D, a_tmem = tmem + buf * 128;
 #pragma unroll
             for (int k = 0; k < kTileN / 16; ++k)
                 // 16 keys per instruction: 8 TMEM columns of A; 16 rows of 128 B of V, column blocks kBlockBytes apart
                 tc_mma_ts_lo(d_tmem, a_tmem + k * 8, bv + k * (2048 >> 4), pv_hi, idesc_pv, k > 0 ? 1u : acc0, leader);
         };
-        auto wait_k = [&](int j) {
-            mbar_wait(bar(&bars.k_full[j % KS]), (uint32_t)(j / KS) & 1u, dead, ix.status);
+        auto wait_k = [&](int kt) {
+            mbar_wait(bar(&bars.k_full[kt % KS]), (uint32_t)(kt / KS) & 1u, dead, ix.status);
             tc_fence_after();
         };
-        auto wait_v = [&](int j) { mbar_wait(bar(&bars.v_full[j % KS]), (uint32_t)(j / KS) & 1u, dead, ix.status); };
-        // Steps are numbered n = n_sub*j + u (KV tile j, sub-tile u); step n uses score buffer n mod NBUF,
-        // and QK(n + NBUF) is queued right behind PV(n), which reads the buffer it overwrites.
-        if (n_sub == 2) {
-            // step 2j uses buffer b0, step 2j+1 buffer b1; par = parity of that buffer's use count
-            int b0 = 0, b1 = 1;
-            uint32_t par0 = 0, par1 = 0;
-            mbar_wait(bar(&bars.q_full[0]), 0, dead, ix.status);
-            mbar_wait(bar(&bars.q_full[1]), 0, dead, ix.status);
-            wait_k(0);
-            qk(0, 0, 0);
-            qk(1, 1, 0);
-            tc_commit(bar(&bars.k_empty[0]), leader);
-            if (NBUF == 3 && t0 >= 1) { wait_k(1); qk(0, 2, 1 % KS); }
-            for (int j = 0; j <= t0; ++j) {      // tiles both sub-tiles have; sub-tile 1 also has tile t0+1
-                const int vs = j % KS, k1 = (j + 1) % KS;
-                wait_v(j);
-                pv(0, b0, par0, vs, j > 0);
-                if (j == t0) tc_commit(bar(&bars.pv_done[0]), leader);
-                if (NBUF == 2) {                 // buffer b0 next holds step 2j+2 = (sub-tile 0, tile j+1)
-                    if (j < t0) { wait_k(j + 1); qk(0, b0, k1); }
-                } else {                         // buffer b0 next holds step 2j+3 = (sub-tile 1, tile j+1)
-                    if (j == t0) wait_k(j + 1);  // otherwise (sub-tile 0, tile j+1) has been issued already
-                    qk(1, b0, k1);
-                    tc_commit(bar(&bars.k_empty[k1]), leader);    // sub-tile 1 is the last reader of a K tile
+        auto wait_v = [&](int kt) { mbar_wait(bar(&bars.v_full[kt % KS]), (uint32_t)(kt / KS) & 1u, dead, ix.status); };
+        auto wait_q = [&](int u) {
+            mbar_wait(bar(&bars.q_full[u]), q_uses[u] & 1u, dead, ix.status);
+            ++q_uses[u];
+        };
+        // Within a unit, steps are numbered n = n_sub*j + u (KV tile j, sub-tile u); step n uses score
+        // buffer n mod NBUF, and QK(n + NBUF) is queued right behind PV(n), which reads the buffer it
+        // overwrites.  All buffers are free again once the last PV of a unit has been queued.
+        TcWork w;
+        int4 rec;
+        int rec_h;
+        fetch(0, rec, rec_h);
+        for (int r = 0; r < n_rounds; ++r) {
+            decode(rec, rec_h, w);
+            fetch(r + 1, rec, rec_h);
+            if (!w.valid) continue;
+            const int t0 = w.t0;
+            if (w.n_sub == 2) {
+                int b0 = 0, b1 = 1;       // step 2j uses buffer b0, step 2j+1 buffer b1
+                wait_q(0);
+                wait_q(1);
+                wait_k(kt0);
+                qk(0, 0, kt0);
+                qk(1, 1, kt0);
+                tc_commit(bar(&bars.k_empty[kt0 % KS]), leader);
+                if (NBUF == 3 && t0 >= 1) { wait_k(kt0 + 1); qk(0, 2, kt0 + 1); }
+                // Q_u may be overwritten once the last score MMA that reads it has run
+                const int last_q0 = (NBUF == 2) ? (t0 > 0 ? t0 - 1 : 0) : t0 - 2;   // iteration that queues QK_0(t0); < 0: done above
+                if (NBUF == 3 && last_q0 < 0) tc_commit(bar(&bars.q_empty[0]), leader);
+                for (int j = 0; j <= t0; ++j) {      // tiles both sub-tiles have; sub-tile 1 also has tile t0+1
+                    const int kt = kt0 + j;
+                    wait_v(kt);
+                    pv(0, b0, kt, j > 0);
+                    if (j == t0) tc_commit(bar(&bars.pv_done[0]), leader);
+                    if (NBUF == 2) {                 // buffer b0 next holds step 2j+2 = (sub-tile 0, tile j+1)
+                        if (j < t0) { wait_k(kt + 1); qk(0, b0, kt + 1); }
+                        if (j == last_q0) tc_commit(bar(&bars.q_empty[0]), leader);
+                    } else {                         // buffer b0 next holds step 2j+3 = (sub-tile 1, tile j+1)
+                        if (j == t0) wait_k(kt + 1);  // otherwise (sub-tile 0, tile j+1) has been issued already
+                        qk(1, b0, kt + 1);
+                        tc_commit(bar(&bars.k_empty[(kt + 1) % KS]), leader);    // sub-tile 1 is the last reader of a K tile
+                        if (j == t0) tc_commit(bar(&bars.q_empty[1]), leader);
+                    }
+                    pv(1, b1, kt, j > 0);
+                    tc_commit(bar(&bars.v_empty[kt % KS]), leader);
+                    if (NBUF == 2) {                 // buffer b1 next holds step 2j+3 = (sub-tile 1, tile j+1)
+                        if (j == t0) wait_k(kt + 1);
+                        qk(1, b1, kt + 1);
+                        tc_commit(bar(&bars.k_empty[(kt + 1) % KS]), leader);
+                        if (j == t0) tc_commit(bar(&bars.q_empty[1]), leader);
+                    } else if (j + 2 <= t0) {        // buffer b1 next holds step 2j+4 = (sub-tile 0, tile j+2)
+                        wait_k(kt + 2);
+                        qk(0, b1, kt + 2);
+                        if (j == last_q0) tc_commit(bar(&bars.q_empty[0]), leader);
+                    }
+                    b0 += 2; if (b0 >= NBUF) b0 -= NBUF;
+                    b1 += 2; if (b1 >= NBUF) b1 -= NBUF;
                 }
-                pv(1, b1, par1, vs, j > 0);
-                tc_commit(bar(&bars.v_empty[vs]), leader);
-                if (NBUF == 2) {                 // buffer b1 next holds step 2j+3 = (sub-tile 1, tile j+1)
-                    if (j == t0) wait_k(j + 1);
-                    qk(1, b1, k1);
-                    tc_commit(bar(&bars.k_empty[k1]), leader);
-                } else if (j + 2 <= t0) {        // buffer b1 next holds step 2j+4 = (sub-tile 0, tile j+2)
-                    wait_k(j + 2);
-                    qk(0, b1, (j + 2) % KS);
+                wait_v(kt0 + t0 + 1);
+                pv(1, b1, kt0 + t0 + 1, 1u);
+                tc_commit(bar(&bars.v_empty[(kt0 + t0 + 1) % KS]), leader);
+                tc_commit(bar(&bars.pv_done[1]), leader);
+            } else {
+                // one sub-tile: step n = tile n; with two or three buffers the scores run ahead of the softmax
+                wait_q(0);
+                for (int i = 0; i < NBUF && i <= t0; ++i) {
+                    wait_k(kt0 + i);
+                    qk(0, i, kt0 + i);
+                    tc_commit(bar(&bars.k_empty[(kt0 + i) % KS]), leader);
                 }
-                b0 += 2; if (b0 >= NBUF) { b0 -= NBUF; par0 ^= 1u; }
-                b1 += 2; if (b1 >= NBUF) { b1 -= NBUF; par1 ^= 1u; }
-            }
-            wait_v(t0 + 1);
-            pv(1, b1, par1, (t0 + 1) % KS, 1u);
-            tc_commit(bar(&bars.pv_done[1]), leader);
-        } else {
-            // one sub-tile: step n = tile n; with two or three buffers the scores run ahead of the softmax
-            mbar_wait(bar(&bars.q_full[0]), 0, dead, ix.status);
-            for (int i = 0; i < NBUF && i <= t0; ++i) {
-                wait_k(i);
-                qk(0, i, i % KS);
-                tc_commit(bar(&bars.k_empty[i % KS]), leader);
-            }
-            int buf = 0;
-            uint32_t par = 0;
-            for (int j = 0; j <= t0; ++j) {
-                const int vs = j % KS;
-                wait_v(j);
-                pv(0, buf, par, vs, j > 0);
-                tc_commit(bar(&bars.v_empty[vs]), leader);
-                if (j + NBUF <= t0) {
-                    wait_k(j + NBUF);
-                    qk(0, buf, (j + NBUF) % KS);
-                    tc_commit(bar(&bars.k_empty[(j + NBUF) % KS]), leader);
+                if (t0 < NBUF) tc_commit(bar(&bars.q_empty[0]), leader);
+                int buf = 0;
+                for (int j = 0; j <= t0; ++j) {
+                    const int kt = kt0 + j;
+                    wait_v(kt);
+                    pv(0, buf, kt, j > 0);
+                    tc_commit(bar(&bars.v_empty[kt % KS]), leader);
+                    if (j + NBUF <= t0) {
+                        wait_k(kt + NBUF);
+                        qk(0, buf, kt + NBUF);
+                        tc_commit(bar(&bars.k_empty[(kt + NBUF) % KS]), leader);
+                        if (j + NBUF == t0) tc_commit(bar(&bars.q_empty[0]), leader);
+                    }
+                    if (++buf == NBUF) buf = 0;
                 }
-                if (++buf == NBUF) { buf = 0; par ^= 1u; }
+                tc_commit(bar(&bars.pv_done[0]), leader);
             }
-            tc_commit(bar(&bars.pv_done[0]), leader);
+            kt0 += w.n_total;
         }
     }
     } else {
     asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;\n" :: "n"(kRegsSoftmax));
-    if (warp < 4 * n_sub) {
+    {
         // ------------------------------------------------------------ softmax + epilogue (one warpgroup per sub-tile)
         const int u = warp >> 2;
         const int r = threadIdx.x & 127;                                  // query row inside the sub-tile = TMEM lane
         const uint32_t lane_addr = ((uint32_t)((warp & 3) * 32) << 16);   // this warp's 32 TMEM lanes
         const uint32_t t_o = tmem + lane_addr + kColO + u * D;
-        const int n_kv = t0 + 1 + u;
+        uint32_t n_steps = 0;       // steps of this sub-tile so far (they pick the barrier)
+        uint32_t n_units = 0;       // units this sub-tile took part in
+        int kt0 = 0;                // K/V tiles of earlier units
+        TcWork w;
+        int4 rec;
+        int rec_h;
+        fetch(0, rec, rec_h);
+        for (int rd = 0; rd < n_rounds; ++rd) {
+        decode(rec, rec_h, w);
+        fetch(rd + 1, rec, rec_h);
+        if (!w.valid) continue;
+        if (u < w.n_sub) {
+        const int n_kv = w.t0 + 1 + u;
+        int buf = u;                // score buffer of this sub-tile's step n = n_sub*j + u, i.e. n mod NBUF
         float m_used = -INFINITY;   // row max the weights are currently scaled with (log2 units)
         float l_run = 0.f;
-        int buf = u;                // score buffer of this sub-tile's step n = n_sub*j + u, i.e. n mod NBUF
-        uint32_t par = 0;           // parity of that buffer's use count
-        for (int j = 0; j < n_kv; ++j) {
+        for (int j = 0; j < n_kv; ++j, ++n_steps) {
             const uint32_t t_s = tmem + lane_addr + buf * 128;
-            mbar_wait(bar(&bars.s_full[buf]), par, dead, ix.status);
+            mbar_wait(bar(&bars.s_full[u][n_steps & 3u]), (n_steps >> 2) & 1u, dead, ix.status);
             tc_fence_after();
             const bool diag = (j == n_kv - 1);
             uint32_t sv[4][32];
@@ -476,7 +561,8 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                 // O_u must hold every earlier tile before it is rescaled, and the scores of this tile may
                 // have been ready before PV of the previous one has run.  The release of V tile j-1 is
                 // committed behind the last PV that reads it, which is issued after PV_u(j-1).
-                mbar_wait(bar(&bars.v_empty[(j - 1) % KS]), (uint32_t)((j - 1) / KS) & 1u, dead, ix.status);
+                const int kt = kt0 + j - 1;
+                mbar_wait(bar(&bars.v_empty[kt % KS]), (uint32_t)(kt / KS) & 1u, dead, ix.status);
                 tc_fence_after();
 #pragma unroll
                 for (int c = 0; c < D / 32; ++c) {
@@ -498,56 +584,49 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                 for (int i = 0; i < 32; i += 2) {
                     float x0 = __uint_as_float(sv[c][i]), x1 = __uint_as_float(sv[c][i + 1]);
                     fma_x2(x0, x1, scale_log2, neg_m);
-                    const uint32_t w = pack_bf16(exp2f(x0), exp2f(x1));
-                    pk[i >> 1] = w;
+                    const uint32_t w2 = pack_bf16(exp2f(x0), exp2f(x1));
+                    pk[i >> 1] = w2;
                     // row sum over the rounded weights (numerator and denominator stay consistent);
                     // the bf16 halves are added to the fp32 sum directly
-                    add_bf16x2(sum[(i >> 1) & 7], w);
+                    add_bf16x2(sum[(i >> 1) & 7], w2);
                 }
                 tc_st16(t_s + c * 16, pk);
             }
             l_run += ((sum[0] + sum[1]) + (sum[2] + sum[3])) + ((sum[4] + sum[5]) + (sum[6] + sum[7]));
             tc_wait_st();
             tc_fence_before();
-            mbar_arrive(bar(&bars.p_full[buf]));
-            buf += n_sub;
-            if (buf >= NBUF) { buf -= NBUF; par ^= 1u; }
+            mbar_arrive(bar(&bars.p_full[u][n_steps & 3u]));
+            buf += w.n_sub;
+            if (buf >= NBUF) buf -= NBUF;
         }
-        // ---- epilogue: O / l -> bf16 -> this sub-tile's (now idle) Q buffer -> coalesced stores
-        mbar_wait(bar(&bars.pv_done[u]), 0, dead, ix.status);
+        // ---- epilogue: O / l -> bf16 -> global; thread r owns row r and writes it in 64-byte runs.
+        // O_u is overwritten by the next unit's first PV, which waits for this warpgroup's next weights.
+        mbar_wait(bar(&bars.pv_done[u]), n_units & 1u, dead, ix.status);
+        ++n_units;
         tc_fence_after();
         const float inv = 1.f / l_run;
-        constexpr int RB = D * 2;                 // bytes per output row
-        constexpr int CH = RB / 16;               // 16-byte chunks per row
-        const uint32_t stage = s_q + u * kTileBytes;
+        // rows past the end of the block belong to the next block (or to nobody): never store them
+        const bool row_ok = !dead && r < w.L - (w.q0 + u * kTileM);
+        __nv_bfloat16* dst = o + ((int64_t)(w.tok0 + w.q0 + u * kTileM + r) * Hq + w.h) * D;
 #pragma unroll
         for (int c = 0; c < D / 32; ++c) {
             float v[32];
             tc_ld32(t_o + c * 32, v);
+            if (row_ok) {
 #pragma unroll
-            for (int i = 0; i < 32; i += 8) {
-                const int chunk = c * 4 + (i >> 3);
-                const uint32_t addr = stage + r * RB + ((chunk ^ (r & 7)) << 4);
-                asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};\n"
-                             :: "r"(addr), "r"(pack_bf16(v[i] * inv, v[i + 1] * inv)), "r"(pack_bf16(v[i + 2] * inv, v[i + 3] * inv)),
-                                "r"(pack_bf16(v[i + 4] * inv, v[i + 5] * inv)), "r"(pack_bf16(v[i + 6] * inv, v[i + 7] * inv))
-                             : "memory");
+                for (int i = 0; i < 32; i += 8) {
+                    uint4 q4;
+                    q4.x = pack_bf16(v[i] * inv, v[i + 1] * inv);
+                    q4.y = pack_bf16(v[i + 2] * inv, v[i + 3] * inv);
+                    q4.z = pack_bf16(v[i + 4] * inv, v[i + 5] * inv);
+                    q4.w = pack_bf16(v[i + 6] * inv, v[i + 7] * inv);
+                    *reinterpret_cast<uint4*>(dst + c * 32 + i) = q4;
+                }
             }
         }
-        wg_sync(1 + u);
-        // rows past the end of the block belong to the next block (or to nobody): never store them
-        const int rows_valid = dead ? 0 : min(kTileM, L - (q0 + u * kTileM));
-        __nv_bfloat16* dst0 = o + ((int64_t)(tok0 + q0 + u * kTileM) * Hq + h) * D;
-        const int tid = threadIdx.x & 127;
-        for (int idx = tid; idx < kTileM * CH; idx += 128) {
-            const int row = idx / CH, chunk = idx - row * CH;
-            if (row < rows_valid) {
-                uint4 w;
-                asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];\n"
-                             : "=r"(w.x), "=r"(w.y), "=r"(w.z), "=r"(w.w)
-                             : "r"(stage + row * RB + ((chunk ^ (row & 7)) << 4)));
-                *reinterpret_cast<uint4*>(dst0 + (int64_t)row * Hq * D + chunk * 8) = w;
-            }
+        tc_fence_before();
+        }
+        kt0 += w.n_total;
         }
     }
     }
@@ -621,9 +700,17 @@ int launch_prefill_tc(const cpa_plan* plan, const void* q, const void* k, const 
         !make_map(&tm_k, k, plan->total_tokens, (int64_t)c.num_kv_heads * D) ||
         !make_map(&tm_v, v, plan->total_tokens, (int64_t)c.num_kv_heads * D))
         return CPA_ECUDA;
-    dim3 grid(plan->n_prefill, c.num_q_heads);
+    // persistent grid: one CTA per SM, each walks its share of the (item, head) units
+    int sms = c.num_sms;
+    if (sms <= 0 && cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev_id) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return CPA_ECUDA;
+    }
+    const int64_t n_work = (int64_t)plan->n_prefill * c.num_q_heads;
+    if (n_work > INT32_MAX) return CPA_EUNSUPPORTED;
+    const int grid = (int)(n_work < sms ? n_work : sms);
     prefill_tc_kernel<D><<<grid, kThreads, smem, st>>>(tm_q, tm_k, tm_v, (__nv_bfloat16*)o, plan->dev(), c.num_q_heads,
-                                                      c.num_kv_heads, plan->q_tile, c.scale * 1.4426950408889634f);
+                                                      c.num_kv_heads, plan->q_tile, c.scale * 1.4426950408889634f, (int)n_work);
     return cudaGetLastError() == cudaSuccess ? CPA_OK : CPA_ECUDA;
 }
 
