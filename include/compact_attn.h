@@ -84,7 +84,9 @@ enum {
     CPA_ARR_PREFILL_ITEMS = 5, /* [n,2] (block, q_tile) in launch order */
     CPA_ARR_DECODE_ITEMS = 6,  /* [n,3] (block, kv_head, split) in launch order */
     CPA_ARR_SPLIT_INDPTR = 7,  /* [B+1] prefix sums of decode splits per block */
-    CPA_ARR_SPLIT_PAGES = 8    /* [B] pages per decode split of each block (the last split may be shorter) */
+    CPA_ARR_SPLIT_PAGES = 8,   /* [B] pages per decode split of each block (the last split may be shorter) */
+    CPA_ARR_PREFILL_SCHED = 9  /* [rounds * CPA_PARAM_PREFILL_CTAS] prefill unit (item * num_q_heads + head) of CTA c
+                                  in round k at k * ctas + c, -1 = none; every unit appears exactly once */
 };
 
 /* Scalars of a plan, for cpa_plan_param. */
@@ -97,7 +99,8 @@ enum {
     CPA_PARAM_INDEX_BYTES = 5,           /* size of the device index buffer for cpa_plan_upload */
     CPA_PARAM_DECODE_WORKSPACE_BYTES = 6,/* size of cpa_decode's device workspace */
     CPA_PARAM_TOTAL_SPLITS = 7,          /* split_indptr[B] */
-    CPA_PARAM_MAX_NEW_TOKENS = 8
+    CPA_PARAM_MAX_NEW_TOKENS = 8,
+    CPA_PARAM_PREFILL_CTAS = 9           /* CTAs of the prefill launch = min(num_sms, prefill units) */
 };
 
 /*
@@ -107,7 +110,9 @@ enum {
  *   order from `free_pages` (block 0 first); seq_lens (0: nothing cached yet);
  *   the slot of every prefill token; the prefill work list of (block, q_tile)
  *   ordered by descending cost (keys seen by the tile's last row), ties by
- *   ascending block then tile; the decode work list of (block, kv_head, split),
+ *   ascending block then tile; the deal of the prefill units (item, query head) to
+ *   the CTAs of the persistent prefill kernel (kv head by kv head, greedy on the tile
+ *   count, see CPA_ARR_PREFILL_SCHED); the decode work list of (block, kv_head, split),
  *   split s = pages [s*C_b, (s+1)*C_b) of the block, ordered by descending page
  *   count, ties by ascending block, kv head, split.  C_b is cfg->pages_per_split, or
  *   with 0 it is chosen per block so that all items fill one wave of CTAs (three per
@@ -151,8 +156,9 @@ CPA_API void cpa_plan_destroy(cpa_plan* plan);
  * block-diagonal because of the independent-chunks layout).
  *   q, o : device bf16 [total_tokens, num_q_heads, head_dim]
  *   k, v : device bf16 [total_tokens, num_kv_heads, head_dim]
- * All four 16-byte aligned; o must not alias the inputs.  One launch covers all
- * (block, q_tile, head) work items.  d_workspace is unused (may be NULL).
+ * All four 16-byte aligned; o must not alias the inputs.  One launch of
+ * CPA_PARAM_PREFILL_CTAS persistent CTAs covers all (block, q_tile, head) units.
+ * d_workspace is unused (may be NULL).
  * Errors: CPA_EINVAL, CPA_ESTATE (plan not uploaded), CPA_ECUDA.
  */
 CPA_API int cpa_prefill(const cpa_plan* plan, const void* q, const void* k, const void* v, void* o,

@@ -20,6 +20,13 @@ stated in full):
                   ties by ascending block, kv head, split.  C_b (pages per split)
                   is an input: one number for all blocks or one per block
 * split_indptr    prefix sums of ceil(pages_b / C_b)
+* prefill schedule the deal of prefill units (item, query head) to the CTAs of a
+                  persistent kernel: units listed kv head by kv head, inside a kv
+                  head in prefill-item order, the G query heads of the group side by
+                  side; each unit goes to the CTA with the least cost so far (ties:
+                  lower CTA); a unit costs 10 * (its KV tiles of 128 keys) + 18,
+                  where an item of 256 query rows whose block has more than 128 rows
+                  left streams one tile more than its first 128-row half
 """
 from __future__ import annotations
 
@@ -104,6 +111,27 @@ def build_plan(block_lens: Sequence[int], max_new_tokens: int, page_size: int,
         "decode_items": decode_items,
         "split_indptr": split_indptr,
     }
+
+
+def prefill_schedule(block_lens: Sequence[int], prefill_items, q_tile_rows: int, num_q_heads: int,
+                     num_kv_heads: int, num_ctas: int):
+    """[rounds][num_ctas] unit codes (item * num_q_heads + head), -1 where a CTA has none."""
+    group = num_q_heads // num_kv_heads
+    n_units = len(prefill_items) * num_q_heads
+    ctas = min(num_ctas, n_units)
+    load = [0] * ctas
+    lists = [[] for _ in range(ctas)]
+    for g in range(num_kv_heads):
+        for i, (b, t) in enumerate(prefill_items):
+            first_row = t * q_tile_rows
+            halves = 2 if (q_tile_rows > 128 and int(block_lens[b]) - first_row > 128) else 1
+            cost = 10 * (first_row // 128 + halves) + 18
+            for h in range(group):
+                c = min(range(ctas), key=lambda x: (load[x], x))
+                lists[c].append(i * num_q_heads + g * group + h)
+                load[c] += cost
+    rounds = max(len(l) for l in lists)
+    return [[lists[c][k] if k < len(lists[c]) else -1 for c in range(ctas)] for k in range(rounds)]
 
 
 def slot_of(plan: Dict[str, list], page_size: int, block: int, pos: int) -> int:

@@ -21,11 +21,13 @@ CPA_OK, CPA_EINVAL, CPA_ENOSPC, CPA_EUNSUPPORTED, CPA_ECUDA, CPA_ETIMEOUT, CPA_E
 ARR_CU_SEQLENS, ARR_PAGE_INDPTR, ARR_PAGE_INDICES, ARR_SEQ_LENS = 0, 1, 2, 3
 ARR_SLOT_MAPPING, ARR_PREFILL_ITEMS, ARR_DECODE_ITEMS, ARR_SPLIT_INDPTR = 4, 5, 6, 7
 ARR_SPLIT_PAGES = 8
+ARR_PREFILL_SCHED = 9
 _ARR_WIDTH = {ARR_PREFILL_ITEMS: 2, ARR_DECODE_ITEMS: 3}
 
 PARAM_NUM_BLOCKS, PARAM_TOTAL_TOKENS, PARAM_Q_TILE_ROWS, PARAM_PAGES_PER_SPLIT = 0, 1, 2, 3
 PARAM_PAGES_USED, PARAM_INDEX_BYTES, PARAM_DECODE_WORKSPACE_BYTES, PARAM_TOTAL_SPLITS = 4, 5, 6, 7
 PARAM_MAX_NEW_TOKENS = 8
+PARAM_PREFILL_CTAS = 9
 
 
 class cpa_config(ctypes.Structure):

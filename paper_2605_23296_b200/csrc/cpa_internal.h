@@ -17,6 +17,7 @@ struct cpa_dev_index {
     int32_t* append_indptr;        // [B+1] source-row offsets of a general append
     const int32_t* page_indices;   // [pages_used]
     const int32_t* prefill_items;  // [n_prefill, 4]: (block, q item, first token of the block, block length), 16-byte aligned
+    const int32_t* prefill_sched;  // [prefill_rounds, prefill_ctas]: unit (item * Hq + head) of CTA c in round k, -1 = none
     const int32_t* decode_items;   // [n_decode, item_stride]: (block, kv_head, split, pages, split size, 0, 0, 0) + page ids
     int32_t* merge_tickets;        // [B * Hkv] arrival counters of the fused split merge (zero between launches)
     int32_t item_stride;           // int32 words per decode item: 8 + largest split size rounded up to 4
@@ -30,13 +31,14 @@ struct cpa_plan {
     int32_t C = 0;          // largest pages-per-split over the blocks
     int64_t total_tokens = 0;
     std::vector<int32_t> block_lens, cu_seqlens, page_indptr, page_indices, seq_lens, slot_mapping,
-        prefill_items, decode_items, split_indptr, split_pages;
+        prefill_items, prefill_sched, decode_items, split_indptr, split_pages;
     int32_t n_prefill = 0, n_decode = 0;
+    int32_t prefill_ctas = 0, prefill_rounds = 0;   // shape of prefill_sched
 
     // packed image of the device index buffer (int32 words) and offsets into it
     std::vector<int32_t> image;
     int64_t off_status = 0, off_cu = 0, off_pindptr = 0, off_sindptr = 0, off_seqlens = 0,
-            off_append = 0, off_pidx = 0, off_pitems = 0, off_ditems = 0, off_tickets = 0, off_seqlens2 = 0,
+            off_append = 0, off_pidx = 0, off_pitems = 0, off_psched = 0, off_ditems = 0, off_tickets = 0, off_seqlens2 = 0,
             words = 0;
     int cur_lens = 0;            // which of the two device length buffers is current
     int32_t item_stride = 0;
@@ -62,6 +64,7 @@ struct cpa_plan {
         d.append_indptr = d_base + off_append;
         d.page_indices = d_base + off_pidx;
         d.prefill_items = d_base + off_pitems;
+        d.prefill_sched = d_base + off_psched;
         d.decode_items = d_base + off_ditems;
         d.merge_tickets = d_base + off_tickets;
         d.item_stride = item_stride;

@@ -6,6 +6,9 @@
 #include <algorithm>
 #include <cstring>
 #include <new>
+#include <queue>
+#include <utility>
+#include <vector>
 
 #include "cpa_internal.h"
 
@@ -88,6 +91,44 @@ extern "C" int cpa_plan_create(const cpa_config* cfg, int32_t num_blocks, const 
     p->prefill_items.reserve(pit.size() * 2);
     for (const PItem& it : pit) { p->prefill_items.push_back(it.block); p->prefill_items.push_back(it.tile); }
 
+    // Prefill schedule for the persistent kernel (one CTA per SM).  A unit is (item, query head).  Units
+    // are listed kv head by kv head, inside a kv head in item order, the G query heads of the group
+    // side by side: CTAs that run at the same time then stream the same few K/V ranges, which stay in
+    // L2.  The list is dealt to the CTAs greedily (next unit to the CTA with the least work so far, ties
+    // to the lower CTA), with a unit's cost taken as its KV tile count plus a fixed part, which is what
+    // a hardware scheduler would do with these durations.
+    {
+        const int32_t Hq = cfg->num_q_heads, G = Hq / cfg->num_kv_heads;
+        const int64_t n_units = (int64_t)p->n_prefill * Hq;
+        if (n_units > INT32_MAX / 4) { delete p; return CPA_EUNSUPPORTED; }
+        const int32_t ctas = (int32_t)std::min<int64_t>(cfg->num_sms ? cfg->num_sms : 148, n_units);
+        std::vector<std::vector<int32_t>> per_cta((size_t)ctas);
+        typedef std::pair<int64_t, int32_t> Load;   // (work so far, CTA)
+        std::priority_queue<Load, std::vector<Load>, std::greater<Load>> heap;
+        for (int32_t c = 0; c < ctas; ++c) heap.push(Load(0, c));
+        const int32_t sub_per_item = p->q_tile / 128;
+        for (int32_t g = 0; g < cfg->num_kv_heads; ++g)
+            for (int32_t i = 0; i < p->n_prefill; ++i) {
+                const int32_t b = p->prefill_items[2 * i], t = p->prefill_items[2 * i + 1];
+                const int32_t q0 = t * p->q_tile;
+                const int32_t n_sub = (sub_per_item > 1 && block_lens[b] - q0 > 128) ? 2 : 1;
+                const int64_t cost = 10LL * (q0 / 128 + n_sub) + 18;
+                for (int32_t h = 0; h < G; ++h) {
+                    Load l = heap.top();
+                    heap.pop();
+                    per_cta[(size_t)l.second].push_back(i * Hq + g * G + h);
+                    heap.push(Load(l.first + cost, l.second));
+                }
+            }
+        size_t rounds = 0;
+        for (const auto& v : per_cta) rounds = std::max(rounds, v.size());
+        p->prefill_ctas = ctas;
+        p->prefill_rounds = (int32_t)rounds;
+        p->prefill_sched.assign(rounds * (size_t)ctas, -1);
+        for (int32_t c = 0; c < ctas; ++c)
+            for (size_t k = 0; k < per_cta[(size_t)c].size(); ++k) p->prefill_sched[k * (size_t)ctas + c] = per_cta[(size_t)c][k];
+    }
+
     // Decode splits.  Every CTA pays a fixed start-up and merge cost, so the planner aims at
     // ONE wave of resident CTAs (three per SM): starting from one split per block, it keeps
     // splitting the block whose splits are largest while the item count (kv heads x splits)
@@ -152,6 +193,7 @@ extern "C" int cpa_plan_create(const cpa_config* cfg, int32_t num_blocks, const 
     p->off_append = w;  w = align4(w + B + 1);
     p->off_pidx = w;    w = align4(w + pages_used);
     p->off_pitems = w;  w = align4(w + 4LL * p->n_prefill);
+    p->off_psched = w;  w = align4(w + (int64_t)p->prefill_sched.size());
     p->item_stride = 8 + (p->C + 3) / 4 * 4;
     p->off_ditems = w;  w = align4(w + (int64_t)p->item_stride * p->n_decode);
     p->off_tickets = w; w = align4(w + (int64_t)B * cfg->num_kv_heads);
@@ -172,6 +214,7 @@ extern "C" int cpa_plan_create(const cpa_config* cfg, int32_t num_blocks, const 
         it[2] = p->cu_seqlens[b];
         it[3] = p->block_lens[b];
     }
+    std::memcpy(im + p->off_psched, p->prefill_sched.data(), sizeof(int32_t) * p->prefill_sched.size());
     for (int32_t i = 0; i < p->n_decode; ++i) {
         // a decode item carries its own page ids, so the kernel's first KV load depends on
         // one prior load only
@@ -204,6 +247,7 @@ extern "C" int cpa_plan_export(const cpa_plan* plan, int which, const int32_t** 
         case CPA_ARR_DECODE_ITEMS: v = &plan->decode_items; div = 3; break;
         case CPA_ARR_SPLIT_INDPTR: v = &plan->split_indptr; break;
         case CPA_ARR_SPLIT_PAGES: v = &plan->split_pages; break;
+        case CPA_ARR_PREFILL_SCHED: v = &plan->prefill_sched; break;
         default: return CPA_EINVAL;
     }
     *ptr = v->data();
@@ -223,6 +267,7 @@ extern "C" int64_t cpa_plan_param(const cpa_plan* plan, int which) {
         case CPA_PARAM_DECODE_WORKSPACE_BYTES: return plan->decode_workspace_bytes();
         case CPA_PARAM_TOTAL_SPLITS: return plan->split_indptr[plan->B];
         case CPA_PARAM_MAX_NEW_TOKENS: return plan->T;
+        case CPA_PARAM_PREFILL_CTAS: return plan->prefill_ctas;
         default: return CPA_EINVAL;
     }
 }

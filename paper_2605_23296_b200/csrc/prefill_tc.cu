@@ -239,18 +239,17 @@ struct TcWork {
     bool valid;                                  // false: this CTA has no unit in that round (last round only)
 };
 
-// The grid is persistent: CTA c takes units c, 2G-1-c, 2G+c, ... (G = grid size; the order of the
-// list is descending cost, so the back-and-forth deal keeps the CTAs' totals within one unit of
-// each other).  Unit w is (item w / Hq, head w % Hq): neighbouring CTAs work on the heads of one
-// item and find its K/V tiles in L2.  Every role walks the same list with its own running
-// counters, so the pipeline never drains between units: the producer is already loading the next
-// unit's Q and K/V, and the issuer its first scores, while a softmax warpgroup still writes the
-// previous unit's output.
+// The grid is persistent: CTA c walks column c of the planner's schedule (units dealt greedily by
+// cost, listed kv head by kv head so that the CTAs running at one time stream the same few K/V
+// ranges out of L2).  Every role walks the same list with its own running counters, so the
+// pipeline never drains between units: the producer is already loading the next unit's Q and
+// K/V, and the issuer its first scores, while a softmax warpgroup still writes the previous
+// unit's output.
 template <int D>
 __global__ void __launch_bounds__(kThreads, 1)
 prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                   const __grid_constant__ CUtensorMap tm_v, __nv_bfloat16* __restrict__ o, cpa_dev_index ix, int Hq,
-                  int Hkv, int q_rows, float scale_log2, int n_work) {
+                  int Hkv, int q_rows, float scale_log2, int n_rounds) {
     using Sh = TcShape<D>;
     constexpr int NB = Sh::NB;
     constexpr uint32_t kTileBytes = Sh::kTileBytes;
@@ -265,17 +264,18 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
     const uint32_t s_v = s_k + KS * kTileBytes;      // KS stages
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int G = gridDim.x, n_rounds = (n_work + G - 1) / G;
+    const int G = gridDim.x;
     const int group = Hq / Hkv;
-    // Unit of round k for this CTA.  Every role fetches the next round's item record (one 16-byte
-    // load) while it works on the current unit, so no global load sits between two units.
-    auto fetch = [&](int k, int4& rec, int& h) {
-        const int idx = k * G + ((k & 1) ? G - 1 - (int)blockIdx.x : (int)blockIdx.x);
-        rec = make_int4(0, 0, 0, 0);                  // block length 0: no unit in that round (last round only)
+    // Unit of round k for this CTA, from the planner's schedule.  Every role keeps the schedule entry of
+    // round k+2 and the item record of round k+1 in flight while it works on round k, so neither of the
+    // two dependent global loads sits between two units.
+    auto fetch_code = [&](int k) { return k < n_rounds ? __ldg(ix.prefill_sched + (int64_t)k * G + blockIdx.x) : -1; };
+    auto fetch = [&](int code, int4& rec, int& h) {
+        rec = make_int4(0, 0, 0, 0);                  // block length 0: no unit in that round
         h = 0;
-        if (k < n_rounds && idx < n_work) {
-            const int it = idx / Hq;
-            h = idx - it * Hq;
+        if (code >= 0) {
+            const int it = code / Hq;
+            h = code - it * Hq;
             rec = __ldg(reinterpret_cast<const int4*>(ix.prefill_items) + it);
         }
     };
@@ -334,10 +334,12 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
             TcWork w;
             int4 rec;
             int rec_h;
-            fetch(0, rec, rec_h);
+            fetch(fetch_code(0), rec, rec_h);
+            int code = fetch_code(1);
             for (int k = 0; k < n_rounds; ++k) {
                 decode(rec, rec_h, w);
-                fetch(k + 1, rec, rec_h);
+                fetch(code, rec, rec_h);
+                code = fetch_code(k + 2);
                 if (!w.valid) continue;
                 for (int u = 0; u < w.n_sub; ++u) {
                     // the buffer is free once the last score MMA of its previous unit has run
@@ -417,10 +419,12 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
         TcWork w;
         int4 rec;
         int rec_h;
-        fetch(0, rec, rec_h);
+        fetch(fetch_code(0), rec, rec_h);
+        int code = fetch_code(1);
         for (int r = 0; r < n_rounds; ++r) {
             decode(rec, rec_h, w);
-            fetch(r + 1, rec, rec_h);
+            fetch(code, rec, rec_h);
+            code = fetch_code(r + 2);
             if (!w.valid) continue;
             const int t0 = w.t0;
             if (w.n_sub == 2) {
@@ -510,10 +514,12 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
         TcWork w;
         int4 rec;
         int rec_h;
-        fetch(0, rec, rec_h);
+        fetch(fetch_code(0), rec, rec_h);
+        int code = fetch_code(1);
         for (int rd = 0; rd < n_rounds; ++rd) {
         decode(rec, rec_h, w);
-        fetch(rd + 1, rec, rec_h);
+        fetch(code, rec, rec_h);
+        code = fetch_code(rd + 2);
         if (!w.valid) continue;
         if (u < w.n_sub) {
         const int n_kv = w.t0 + 1 + u;
@@ -700,17 +706,10 @@ int launch_prefill_tc(const cpa_plan* plan, const void* q, const void* k, const 
         !make_map(&tm_k, k, plan->total_tokens, (int64_t)c.num_kv_heads * D) ||
         !make_map(&tm_v, v, plan->total_tokens, (int64_t)c.num_kv_heads * D))
         return CPA_ECUDA;
-    // persistent grid: one CTA per SM, each walks its share of the (item, head) units
-    int sms = c.num_sms;
-    if (sms <= 0 && cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev_id) != cudaSuccess) {
-        (void)cudaGetLastError();
-        return CPA_ECUDA;
-    }
-    const int64_t n_work = (int64_t)plan->n_prefill * c.num_q_heads;
-    if (n_work > INT32_MAX) return CPA_EUNSUPPORTED;
-    const int grid = (int)(n_work < sms ? n_work : sms);
-    prefill_tc_kernel<D><<<grid, kThreads, smem, st>>>(tm_q, tm_k, tm_v, (__nv_bfloat16*)o, plan->dev(), c.num_q_heads,
-                                                      c.num_kv_heads, plan->q_tile, c.scale * 1.4426950408889634f, (int)n_work);
+    // persistent grid: one CTA per SM, each walks its column of the planner's schedule
+    prefill_tc_kernel<D><<<plan->prefill_ctas, kThreads, smem, st>>>(tm_q, tm_k, tm_v, (__nv_bfloat16*)o, plan->dev(),
+                                                                   c.num_q_heads, c.num_kv_heads, plan->q_tile,
+                                                                   c.scale * 1.4426950408889634f, plan->prefill_rounds);
     return cudaGetLastError() == cudaSuccess ? CPA_OK : CPA_ECUDA;
 }
 

@@ -42,6 +42,15 @@ def check_against_oracle(w, pages_per_split=0, permute=False):
             got = B.cpa_plan_export(plan, which)
             want = np.asarray(ref[key], dtype=np.int32).reshape(got.shape)
             assert np.array_equal(got, want), key
+        # the deal of prefill units to persistent CTAs: bit-exact with the restated rule, and a partition
+        ctas = B.cpa_plan_param(plan, B.PARAM_PREFILL_CTAS)
+        n_units = len(ref["prefill_items"]) * w.num_q_heads
+        assert ctas == min(148, n_units)
+        sched = B.cpa_plan_export(plan, B.ARR_PREFILL_SCHED)
+        want = op.prefill_schedule(w.block_lens.tolist(), ref["prefill_items"], M, w.num_q_heads,
+                                   w.num_kv_heads, 148)
+        assert np.array_equal(sched.reshape(-1, ctas), np.asarray(want, dtype=np.int32))
+        assert sorted(sched[sched >= 0].tolist()) == list(range(n_units))
         assert B.cpa_plan_param(plan, B.PARAM_NUM_BLOCKS) == w.num_blocks
         assert B.cpa_plan_param(plan, B.PARAM_TOTAL_TOKENS) == w.total_tokens
         assert B.cpa_plan_param(plan, B.PARAM_PAGES_USED) == w.pages_needed
