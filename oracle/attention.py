@@ -11,6 +11,12 @@ itself is the textbook causal softmax attention with grouped-query heads
 key/value first and then attends over all cached keys, the new one included,
 so step t of block b equals the last row of a causal prefill over the
 (L_b + t + 1)-token sequence.
+
+The paper's own layout (Section 4, "Prefix-aware target-at-end layout") is
+covered by ``prefill_prefix_aware`` / ``PrefixDecodeState``: the prompt of
+worker w is the history up to its block followed by its own (target) tokens, so
+a target token attends causally over that whole prompt; it is written here as
+exactly that, the plain causal attention over the concatenated prompt.
 """
 from __future__ import annotations
 
@@ -152,6 +158,60 @@ class DecodeState:
             n = self.len[b]
             out[b] = attend_token(q[b], self.k[b][:n], self.v[b][:n], scale)
         return out
+
+
+def prefill_prefix_aware(q: np.ndarray, k: np.ndarray, v: np.ndarray, cu_seqlens: Sequence[int],
+                         k_hist: np.ndarray, v_hist: np.ndarray, prefix_lens: Sequence[int],
+                         scale: float, rows: Optional[Sequence[int]] = None) -> np.ndarray:
+    """Attention of every worker's own tokens over its prompt (Section 4, "Dispatch").
+
+    Worker w's prompt is the first prefix_lens[w] tokens of the shared history
+    (k_hist/v_hist [hist_tokens,Hkv,d]) followed by its own tokens
+    k/v[cu[w]:cu[w+1]] (the target block with its markers).  Row i of worker w
+    sees the whole prefix and its own tokens 0..i: causal attention over the
+    concatenated prompt, evaluated for the rows of the own tokens only.
+    q [tokens,Hq,d] holds the own tokens' queries (the prefix needs none).
+    Returns float64 [tokens,Hq,d], or [len(rows),Hq,d] for `rows` (ids into q).
+    """
+    cu = [int(x) for x in cu_seqlens]
+    W = len(cu) - 1
+    tokens, Hq, d = q.shape
+    assert len(prefix_lens) == W and cu[-1] == tokens
+    wanted = None if rows is None else [int(r) for r in rows]
+    out = np.empty((tokens if wanted is None else len(wanted), Hq, d), dtype=np.float64)
+    for w in range(W):
+        n_pre, lo, hi = int(prefix_lens[w]), cu[w], cu[w + 1]
+        assert 0 <= n_pre <= k_hist.shape[0]
+        if wanted is None:
+            local, dest = list(range(hi - lo)), list(range(lo, hi))
+        else:
+            sel = [(i, r - lo) for i, r in enumerate(wanted) if lo <= r < hi]
+            if not sel:
+                continue
+            dest, local = [i for i, _ in sel], [r for _, r in sel]
+        prompt_k = np.concatenate([k_hist[:n_pre], k[lo:hi]])
+        prompt_v = np.concatenate([v_hist[:n_pre], v[lo:hi]])
+        prompt_q = np.concatenate([np.zeros((n_pre, Hq, d), dtype=np.uint16), q[lo:hi]])
+        res = prefill(prompt_q, prompt_k, prompt_v, [0, n_pre + hi - lo], scale,
+                      rows=[n_pre + r for r in local])
+        out[dest] = res
+    return out
+
+
+class PrefixDecodeState(DecodeState):
+    """Decode in the prefix-aware layout: worker w's cache is its prompt (history prefix, then its
+    own tokens), kept contiguously per worker and extended one token per step."""
+
+    def __init__(self, k: np.ndarray, v: np.ndarray, cu_seqlens: Sequence[int], k_hist: np.ndarray,
+                 v_hist: np.ndarray, prefix_lens: Sequence[int], max_new: int):
+        cu = [int(x) for x in cu_seqlens]
+        ks, vs, ccu = [], [], [0]
+        for w in range(len(cu) - 1):
+            n_pre = int(prefix_lens[w])
+            ks += [k_hist[:n_pre], k[cu[w]:cu[w + 1]]]
+            vs += [v_hist[:n_pre], v[cu[w]:cu[w + 1]]]
+            ccu.append(ccu[-1] + n_pre + cu[w + 1] - cu[w])
+        super().__init__(np.concatenate(ks), np.concatenate(vs), ccu, max_new)
 
 
 def expected_pool(slot_mapping: Sequence[int], k: np.ndarray, v: np.ndarray,

@@ -20,6 +20,10 @@ stated in full):
                   ties by ascending block, kv head, split.  C_b (pages per split)
                   is an input: one number for all blocks or one per block
 * split_indptr    prefix sums of ceil(pages_b / C_b)
+* prefix-aware    (Section 4, "Prefix-aware target-at-end layout") each sequence
+                  additionally starts with prefix_lens[b] cached history tokens in
+                  shared pages: they come first in its page list, count in seq_lens,
+                  in the cost of its prefill items and in its decode splits
 * prefill schedule the deal of prefill units (item, query head) to the CTAs of a
                   persistent kernel: units listed kv head by kv head, inside a kv
                   head in prefill-item order, the G query heads of the group side by
@@ -45,8 +49,19 @@ def partition(history_len: int, block_size: int):
 
 def build_plan(block_lens: Sequence[int], max_new_tokens: int, page_size: int,
                free_pages: Sequence[int], num_kv_heads: int,
-               q_tile_rows: int, pages_per_split) -> Dict[str, list]:
+               q_tile_rows: int, pages_per_split, prefix_lens: Sequence[int] = (),
+               shared_pages: Sequence[int] = ()) -> Dict[str, list]:
+    """Independent chunks (no prefix_lens), or the prefix-aware layout of Section 4: sequence b
+    (worker b) already has the first prefix_lens[b] tokens of the shared history cached in the first
+    prefix_lens[b] / P entries of `shared_pages` (same pages for every worker: the prefix cache), and
+    block_lens[b] are its own tokens (target block plus markers), stored after the prefix in pages of
+    its own taken from the free list."""
     B = len(block_lens)
+    prefix_lens = [int(x) for x in prefix_lens] if len(prefix_lens) else [0] * B
+    if len(prefix_lens) != B or any(x < 0 or x % page_size for x in prefix_lens):
+        raise ValueError("one page-aligned prefix length per block")
+    if max(prefix_lens) > len(shared_pages) * page_size:
+        raise ValueError("prefix longer than the shared pages")
     if B < 1:
         raise ValueError("need at least one block")
     if any(int(L) < 1 for L in block_lens):
@@ -62,20 +77,25 @@ def build_plan(block_lens: Sequence[int], max_new_tokens: int, page_size: int,
     for L in block_lens:
         cu.append(cu[-1] + int(L))
 
-    pages_per_block = []
-    for L in block_lens:
+    pages_per_block, own_pages = [], []
+    for b, L in enumerate(block_lens):
         tokens = int(L) + max_new_tokens
-        pages_per_block.append((tokens + page_size - 1) // page_size)
+        own_pages.append((tokens + page_size - 1) // page_size)
+        pages_per_block.append(prefix_lens[b] // page_size + own_pages[b])
     indptr = [0]
     for n in pages_per_block:
         indptr.append(indptr[-1] + n)
-    if indptr[-1] > len(free_pages):
+    if sum(own_pages) > len(free_pages):
         raise MemoryError("not enough free pages")
-    page_indices = [int(free_pages[i]) for i in range(indptr[-1])]
+    page_indices, taken = [], 0
+    for b in range(B):
+        page_indices += [int(x) for x in shared_pages[: prefix_lens[b] // page_size]]
+        page_indices += [int(free_pages[taken + i]) for i in range(own_pages[b])]
+        taken += own_pages[b]
 
     slot_mapping = []
     for b, L in enumerate(block_lens):
-        for p in range(int(L)):
+        for p in range(prefix_lens[b], prefix_lens[b] + int(L)):
             page = page_indices[indptr[b] + p // page_size]
             slot_mapping.append(page * page_size + p % page_size)
 
@@ -83,7 +103,7 @@ def build_plan(block_lens: Sequence[int], max_new_tokens: int, page_size: int,
     for b, L in enumerate(block_lens):
         n_tiles = (int(L) + q_tile_rows - 1) // q_tile_rows
         for t in range(n_tiles):
-            cost = min((t + 1) * q_tile_rows, int(L))
+            cost = prefix_lens[b] + min((t + 1) * q_tile_rows, int(L))
             prefill.append((-cost, b, t))
     prefill.sort()
     prefill_items = [[b, t] for (_, b, t) in prefill]
@@ -105,7 +125,7 @@ def build_plan(block_lens: Sequence[int], max_new_tokens: int, page_size: int,
         "cu_seqlens": cu,
         "page_indptr": indptr,
         "page_indices": page_indices,
-        "seq_lens": [0] * B,
+        "seq_lens": list(prefix_lens),
         "slot_mapping": slot_mapping,
         "prefill_items": prefill_items,
         "decode_items": decode_items,
@@ -114,7 +134,7 @@ def build_plan(block_lens: Sequence[int], max_new_tokens: int, page_size: int,
 
 
 def prefill_schedule(block_lens: Sequence[int], prefill_items, q_tile_rows: int, num_q_heads: int,
-                     num_kv_heads: int, num_ctas: int):
+                     num_kv_heads: int, num_ctas: int, prefix_lens: Sequence[int] = ()):
     """[rounds][num_ctas] unit codes (item * num_q_heads + head), -1 where a CTA has none."""
     group = num_q_heads // num_kv_heads
     n_units = len(prefill_items) * num_q_heads
@@ -125,7 +145,8 @@ def prefill_schedule(block_lens: Sequence[int], prefill_items, q_tile_rows: int,
         for i, (b, t) in enumerate(prefill_items):
             first_row = t * q_tile_rows
             halves = 2 if (q_tile_rows > 128 and int(block_lens[b]) - first_row > 128) else 1
-            cost = 10 * (first_row // 128 + halves) + 18
+            prefix_tiles = int(prefix_lens[b]) // 128 if len(prefix_lens) else 0
+            cost = 10 * (prefix_tiles + first_row // 128 + halves) + 18
             for h in range(group):
                 c = min(range(ctas), key=lambda x: (load[x], x))
                 lists[c].append(i * num_q_heads + g * group + h)

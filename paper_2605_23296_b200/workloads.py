@@ -165,6 +165,59 @@ def split(seed: int = 4, num_blocks: int = 8, steps: int = 256) -> Workload:
     return split_sweep(num_blocks, seed=seed, steps=steps)
 
 
+@dataclass
+class PrefixWorkload:
+    """Inputs for the paper's prefix-aware target-at-end layout (Section 4).
+
+    A history of `num_workers` blocks of `block_len` tokens is already cached (k_hist/v_hist, in
+    `shared_pages` of the pool).  Worker w re-reads blocks 0..w-1 from that cache (prefix_lens[w] =
+    w * block_len tokens) and runs its own tokens, block w wrapped in `marker_tokens` marker tokens:
+    `own` holds those per-worker tokens (block_lens = block_len + marker_tokens each), their
+    queries, the free pages for them and the decode-step inputs.  Page ids: the shared pages are
+    0 .. hist_pages-1 (permuted together with the free pages when `own.permute_pages`)."""
+
+    own: Workload
+    block_len: int
+    marker_tokens: int
+    prefix_lens: np.ndarray                   # int32 [W]
+    shared_pages: Optional[np.ndarray] = None  # int32 [hist_tokens / P]
+    k_hist: Optional[np.ndarray] = None        # uint16 [hist_tokens, Hkv, d]
+    v_hist: Optional[np.ndarray] = None
+
+    @property
+    def hist_tokens(self) -> int:
+        return int(self.prefix_lens.max())
+
+    @property
+    def num_pages(self) -> int:
+        return self.hist_tokens // self.own.page_size + self.own.num_pages
+
+    def materialise(self, with_decode: bool = True) -> "PrefixWorkload":
+        if self.k_hist is not None:
+            return self
+        o = self.own.materialise(with_decode)
+        rng = o._rng
+        hkv, d = o.num_kv_heads, o.head_dim
+        self.k_hist = f32_to_bf16_bits(rng.standard_normal((self.hist_tokens, hkv, d), dtype=np.float32))
+        self.v_hist = f32_to_bf16_bits(rng.standard_normal((self.hist_tokens, hkv, d), dtype=np.float32))
+        n_shared = self.hist_tokens // o.page_size
+        ids = rng.permutation(self.num_pages).astype(np.int32) if o.permute_pages else np.arange(self.num_pages, dtype=np.int32)
+        self.shared_pages = ids[:n_shared].copy()
+        o.free_pages = ids[n_shared:].copy()
+        return self
+
+
+def prefix_aware(num_workers: int, block_len: int, hq: int, hkv: int, d: int, steps: int, seed: int = 11,
+                 marker_tokens: int = 16, permute_pages: bool = True) -> PrefixWorkload:
+    """`num_workers` workers over a history of blocks of `block_len` tokens (a multiple of 128)."""
+    assert block_len % 128 == 0 and num_workers >= 1
+    rng = np.random.Generator(np.random.PCG64(seed))
+    own = _mk(f"prefix{num_workers}x{block_len}", hq, hkv, d, [block_len + marker_tokens] * num_workers, steps, seed,
+              rng, permute_pages=permute_pages)
+    pre = np.arange(num_workers, dtype=np.int32) * np.int32(block_len)
+    return PrefixWorkload(own=own, block_len=block_len, marker_tokens=marker_tokens, prefix_lens=pre)
+
+
 CONFIGS = {
     "tiny": tiny,
     "dense8b": dense8b,
