@@ -128,6 +128,34 @@ CPA_API int cpa_plan_create(const cpa_config* cfg, int32_t num_blocks, const int
                     int32_t max_new_tokens, const int32_t* free_pages, int32_t num_free,
                     cpa_plan** out);
 
+/*
+ * cpa_plan_create_prefix -- the plan for the paper's own layout (Section 4, "Dispatch" and
+ * "Prefix-aware target-at-end layout"): the prompt of worker w is blocks 1..w-1 of the history
+ * followed by block w wrapped in its markers, every worker's prefix extends the previous worker's,
+ * and that prefix is not recomputed but read from the KV cache the history already has.
+ *   own_lens[w]    : tokens worker w runs itself (its target block plus markers), >= 1
+ *   prefix_lens[w] : history tokens worker w reads from the cache; a multiple of 128 (the
+ *                    prefill kernel reads a cached prefix in whole KV tiles of 128 keys; a
+ *                    block boundary that is not a multiple of 128 is handled by the caller
+ *                    giving the remainder to own_lens, as a serving engine's block-granular
+ *                    prefix cache does with a partial block)
+ *   shared_pages   : host int32 [num_shared] pool pages that hold the history, page i = history
+ *                    tokens [16 i, 16 i + 16); they must be filled (cpa_kv_append through a plan
+ *                    that owns them) before cpa_prefill_prefix or a decode call reads them, and
+ *                    no call through this plan ever writes them
+ * Worker w's page list is shared_pages[0 .. prefix_lens[w]/16) followed by
+ * ceil((own_lens[w] + max_new_tokens) / 16) pages of its own from `free_pages`; its cached
+ * length (seq_lens) starts at prefix_lens[w]; positions, slots and the decode splits count from
+ * the start of the prompt; the cost of a prefill item includes the prefix.  Everything else is
+ * as for cpa_plan_create, which is the case prefix_lens == 0.  Errors as for cpa_plan_create,
+ * plus CPA_EINVAL for a prefix that is negative, not a multiple of 128, or longer than
+ * 16 * num_shared.
+ */
+CPA_API int cpa_plan_create_prefix(const cpa_config* cfg, int32_t num_workers, const int32_t* own_lens,
+                                   const int32_t* prefix_lens, const int32_t* shared_pages, int32_t num_shared,
+                                   int32_t max_new_tokens, const int32_t* free_pages, int32_t num_free,
+                                   cpa_plan** out);
+
 /* Borrow a host view of one index array (valid until the plan is destroyed or,
  * for CPA_ARR_SEQ_LENS, until the next cpa_kv_append).  Errors: CPA_EINVAL. */
 CPA_API int cpa_plan_export(const cpa_plan* plan, int which, const int32_t** ptr, int64_t* count);
@@ -163,6 +191,23 @@ CPA_API void cpa_plan_destroy(cpa_plan* plan);
  */
 CPA_API int cpa_prefill(const cpa_plan* plan, const void* q, const void* k, const void* v, void* o,
                 void* d_workspace, void* stream);
+
+/*
+ * cpa_prefill_prefix -- the prefill of the prefix-aware layout (Section 4, "Dispatch"; the
+ * per-worker cost the paper's Section 6 calls "each worker must additionally prefill its own
+ * unique block content"): row i of worker w attends over the prefix_lens[w] cached history
+ * tokens and over its own tokens 0..i,
+ *     O[i,h,:] = sum_{j < prefix or j-prefix <= i} softmax_j(scale * q[i,h,:].k[j,g,:]) v[j,g,:].
+ *   q, o   : device bf16 [sum(own_lens), num_q_heads, head_dim], the workers' own tokens
+ *   k, v   : device bf16 [sum(own_lens), num_kv_heads, head_dim], the same tokens' keys/values
+ *   k_pool, v_pool : the pools; only the shared pages of each worker's prefix are read
+ * The plan must come from cpa_plan_create_prefix (or cpa_plan_create: then nothing is read from
+ * the pools and the result is cpa_prefill's).  Prefix tiles are staged straight from the pool
+ * pages into the kernel's shared-memory tiles.  Follow with cpa_kv_append(own_lens) to cache the
+ * own tokens behind the prefix.  Errors: as cpa_prefill.
+ */
+CPA_API int cpa_prefill_prefix(const cpa_plan* plan, const void* q, const void* k, const void* v, const void* k_pool,
+                               const void* v_pool, void* o, void* stream);
 
 /*
  * cpa_prefill_variant -- cpa_prefill with the kernel chosen by the caller; for

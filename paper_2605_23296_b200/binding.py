@@ -53,6 +53,9 @@ _vp, _i32p = ctypes.c_void_p, ctypes.POINTER(ctypes.c_int32)
 _lib.cpa_plan_create.argtypes = [ctypes.POINTER(cpa_config), ctypes.c_int32, _i32p, ctypes.c_int32,
                                  _i32p, ctypes.c_int32, ctypes.POINTER(_vp)]
 _lib.cpa_plan_create.restype = ctypes.c_int
+_lib.cpa_plan_create_prefix.argtypes = [ctypes.POINTER(cpa_config), ctypes.c_int32, _i32p, _i32p, _i32p, ctypes.c_int32,
+                                        ctypes.c_int32, _i32p, ctypes.c_int32, ctypes.POINTER(_vp)]
+_lib.cpa_plan_create_prefix.restype = ctypes.c_int
 _lib.cpa_plan_export.argtypes = [_vp, ctypes.c_int, ctypes.POINTER(_i32p), ctypes.POINTER(ctypes.c_int64)]
 _lib.cpa_plan_export.restype = ctypes.c_int
 _lib.cpa_plan_param.argtypes = [_vp, ctypes.c_int]
@@ -65,6 +68,8 @@ _lib.cpa_plan_destroy.argtypes = [_vp]
 _lib.cpa_plan_destroy.restype = None
 _lib.cpa_prefill.argtypes = [_vp, _vp, _vp, _vp, _vp, _vp, _vp]
 _lib.cpa_prefill.restype = ctypes.c_int
+_lib.cpa_prefill_prefix.argtypes = [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]
+_lib.cpa_prefill_prefix.restype = ctypes.c_int
 _lib.cpa_prefill_variant.argtypes = [_vp, _vp, _vp, _vp, _vp, _vp, ctypes.c_int]
 _lib.cpa_prefill_variant.restype = ctypes.c_int
 _lib.cpa_kv_append.argtypes = [_vp, _vp, _vp, _i32p, _vp, _vp, _vp]
@@ -111,6 +116,23 @@ def cpa_plan_create(cfg: cpa_config, block_lens: Sequence[int], max_new_tokens: 
     return out.value
 
 
+def cpa_plan_create_prefix(cfg: cpa_config, own_lens: Sequence[int], prefix_lens: Sequence[int],
+                           shared_pages: Sequence[int], max_new_tokens: int, free_pages: Sequence[int],
+                           check: bool = True):
+    """Plan of the prefix-aware layout; returns the handle, or (status, handle) with check=False."""
+    lens, pre, shared, free = _i32(own_lens), _i32(prefix_lens), _i32(shared_pages), _i32(free_pages)
+    out = _vp()
+    rc = _lib.cpa_plan_create_prefix(ctypes.byref(cfg), lens.shape[0], lens.ctypes.data_as(_i32p),
+                                     pre.ctypes.data_as(_i32p), shared.ctypes.data_as(_i32p), shared.shape[0],
+                                     int(max_new_tokens), free.ctypes.data_as(_i32p), free.shape[0],
+                                     ctypes.byref(out))
+    if not check:
+        return rc, out.value
+    if rc != CPA_OK:
+        raise CpaError(rc, "cpa_plan_create_prefix")
+    return out.value
+
+
 def cpa_plan_export(plan: int, which: int) -> np.ndarray:
     """Copy of one host index array; item lists come back as [n, width]."""
     ptr, n = _i32p(), ctypes.c_int64()
@@ -145,6 +167,10 @@ def cpa_prefill(plan: int, q, k, v, o, d_workspace=None, stream: int = 0) -> int
 
 
 PREFILL_TENSOR_CORE, PREFILL_WARP_MMA = 0, 1
+
+
+def cpa_prefill_prefix(plan: int, q, k, v, k_pool, v_pool, o, stream: int = 0) -> int:
+    return _lib.cpa_prefill_prefix(plan, _ptr(q), _ptr(k), _ptr(v), _ptr(k_pool), _ptr(v_pool), _ptr(o), stream)
 
 
 def cpa_prefill_variant(plan: int, q, k, v, o, stream: int = 0, variant: int = 0) -> int:

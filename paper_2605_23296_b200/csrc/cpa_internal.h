@@ -16,7 +16,8 @@ struct cpa_dev_index {
     int32_t* seq_lens_next;        // [B]   the other length buffer: a fused decode+append writes the new lengths here
     int32_t* append_indptr;        // [B+1] source-row offsets of a general append
     const int32_t* page_indices;   // [pages_used]
-    const int32_t* prefill_items;  // [n_prefill, 4]: (block, q item, first token of the block, block length), 16-byte aligned
+    const int32_t* prefill_items;  // [n_prefill, 4]: (first token of the block, block length, q item | prefix KV tiles << 16,
+                                   //   first entry of the sequence in page_indices), 16-byte aligned
     const int32_t* prefill_sched;  // [prefill_rounds, prefill_ctas]: unit (item * Hq + head) of CTA c in round k, -1 = none
     const int32_t* decode_items;   // [n_decode, item_stride]: (block, kv_head, split, pages, split size, 0, 0, 0) + page ids
     int32_t* merge_tickets;        // [B * Hkv] arrival counters of the fused split merge (zero between launches)
@@ -30,6 +31,8 @@ struct cpa_plan {
     int32_t q_tile = 0;     // query rows per prefill item
     int32_t C = 0;          // largest pages-per-split over the blocks
     int64_t total_tokens = 0;
+    int32_t pool_pages = 0; // largest page id in the page table + 1 (extent of the pools the prefill reads a prefix from)
+    std::vector<int32_t> prefix_lens;   // [B] tokens of each sequence that are cached before the plan starts (0: none)
     std::vector<int32_t> block_lens, cu_seqlens, page_indptr, page_indices, seq_lens, slot_mapping,
         prefill_items, prefill_sched, decode_items, split_indptr, split_pages;
     int32_t n_prefill = 0, n_decode = 0;

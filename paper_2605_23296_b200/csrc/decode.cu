@@ -494,7 +494,7 @@ extern "C" int cpa_decode_append(cpa_plan* plan, const void* q, const void* k_ne
         return CPA_EINVAL;
     if (!plan->d_base) return CPA_ESTATE;
     for (int b = 0; b < plan->B; ++b)
-        if ((int64_t)plan->seq_lens[b] + 1 > (int64_t)plan->block_lens[b] + plan->T) return CPA_ENOSPC;
+        if ((int64_t)plan->seq_lens[b] + 1 > (int64_t)plan->prefix_lens[b] + plan->block_lens[b] + plan->T) return CPA_ENOSPC;
     // the kernel counts the new token itself; the host mirror moves first so that the launcher
     // sees non-empty caches, and moves back if the launch fails
     for (int b = 0; b < plan->B; ++b) plan->seq_lens[b] += 1;

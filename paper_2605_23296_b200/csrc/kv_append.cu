@@ -86,8 +86,8 @@ extern "C" int cpa_kv_append(cpa_plan* plan, const void* k_new, const void* v_ne
     for (int b = 0; b < B; ++b) {
         const int n = new_lens ? new_lens[b] : 1;
         if (n < 0) return CPA_EINVAL;
-        if ((int64_t)plan->seq_lens[b] + n > (int64_t)plan->block_lens[b] + plan->T) return CPA_ENOSPC;
-        if (new_lens && (plan->seq_lens[b] != 0 || n != plan->block_lens[b])) is_prefill_bulk = false;
+        if ((int64_t)plan->seq_lens[b] + n > (int64_t)plan->prefix_lens[b] + plan->block_lens[b] + plan->T) return CPA_ENOSPC;
+        if (new_lens && (plan->seq_lens[b] != plan->prefix_lens[b] || n != plan->block_lens[b])) is_prefill_bulk = false;
         rows += n;
     }
     if (rows == 0) return CPA_OK;

@@ -19,12 +19,14 @@ int64_t align4(int64_t words) { return (words + 3) / 4 * 4; }  // 16-byte alignm
 
 }  // namespace
 
-extern "C" int cpa_plan_create(const cpa_config* cfg, int32_t num_blocks, const int32_t* block_lens,
-                               int32_t max_new_tokens, const int32_t* free_pages, int32_t num_free,
-                               cpa_plan** out) {
+namespace {
+// Both layouts: `prefix_lens` == nullptr is the independent-chunks layout (no cached prefix).
+int plan_create(const cpa_config* cfg, int32_t num_blocks, const int32_t* block_lens, const int32_t* prefix_lens,
+                const int32_t* shared_pages, int32_t num_shared, int32_t max_new_tokens, const int32_t* free_pages,
+                int32_t num_free, cpa_plan** out) {
     if (out) *out = nullptr;
     if (!cfg || !block_lens || !out || num_blocks < 1 || max_new_tokens < 0 || num_free < 0 ||
-        (num_free > 0 && !free_pages))
+        (num_free > 0 && !free_pages) || num_shared < 0 || (num_shared > 0 && !shared_pages))
         return CPA_EINVAL;
     if (cfg->num_q_heads < 1 || cfg->num_kv_heads < 1 || cfg->num_q_heads % cfg->num_kv_heads != 0 ||
         cfg->q_tile_rows < 0 || cfg->pages_per_split < 0 || cfg->num_sms < 0 || !(cfg->scale > 0.f))
@@ -45,33 +47,61 @@ extern "C" int cpa_plan_create(const cpa_config* cfg, int32_t num_blocks, const 
     const int32_t B = num_blocks;
 
     p->block_lens.assign(block_lens, block_lens + B);
+    p->prefix_lens.assign(B, 0);
+    if (prefix_lens) p->prefix_lens.assign(prefix_lens, prefix_lens + B);
     p->cu_seqlens.assign(B + 1, 0);
     p->page_indptr.assign(B + 1, 0);
-    std::vector<int32_t> pages_per_block(B);
+    std::vector<int32_t> pages_per_block(B), own_pages(B);
+    int64_t own_total = 0;
     for (int32_t b = 0; b < B; ++b) {
         if (block_lens[b] < 1) { delete p; return CPA_EINVAL; }
+        const int32_t pre = p->prefix_lens[b];
+        // a cached prefix is read in whole KV tiles of 128 keys (so also in whole pages)
+        if (pre < 0 || pre % 128 != 0 || pre > (int64_t)num_shared * P) { delete p; return CPA_EINVAL; }
+        // the device item record packs the q item and the prefix tile count into 16 bits each
+        if (pre / 128 > 0x7FFF || (block_lens[b] + 127) / 128 > 0xFFFF) { delete p; return CPA_EUNSUPPORTED; }
         int64_t cu = (int64_t)p->cu_seqlens[b] + block_lens[b];
-        int64_t pages = ((int64_t)block_lens[b] + max_new_tokens + P - 1) / P;
-        int64_t ip = (int64_t)p->page_indptr[b] + pages;
-        if (cu > INT32_MAX / 2 || ip > INT32_MAX / 64) { delete p; return CPA_EUNSUPPORTED; }
+        int64_t own = ((int64_t)block_lens[b] + max_new_tokens + P - 1) / P;
+        int64_t ip = (int64_t)p->page_indptr[b] + pre / P + own;
+        if (cu > INT32_MAX / 2 || ip > INT32_MAX / 64 || (int64_t)pre + block_lens[b] + max_new_tokens > INT32_MAX / 2) {
+            delete p;
+            return CPA_EUNSUPPORTED;
+        }
         p->cu_seqlens[b + 1] = (int32_t)cu;
         p->page_indptr[b + 1] = (int32_t)ip;
-        pages_per_block[b] = (int32_t)pages;
+        own_pages[b] = (int32_t)own;
+        pages_per_block[b] = (int32_t)(pre / P + own);
+        own_total += own;
     }
     p->total_tokens = p->cu_seqlens[B];
     const int32_t pages_used = p->page_indptr[B];
-    if (pages_used > num_free) { delete p; return CPA_ENOSPC; }
-    p->page_indices.assign(free_pages, free_pages + pages_used);
-    for (int32_t id : p->page_indices)
+    if (own_total > num_free) { delete p; return CPA_ENOSPC; }
+    // a sequence's pages: the shared pages of its cached prefix first, then pages of its own, dealt
+    // in order from the free list
+    p->page_indices.reserve((size_t)pages_used);
+    int64_t taken = 0;
+    for (int32_t b = 0; b < B; ++b) {
+        p->page_indices.insert(p->page_indices.end(), shared_pages, shared_pages + p->prefix_lens[b] / P);
+        p->page_indices.insert(p->page_indices.end(), free_pages + taken, free_pages + taken + own_pages[b]);
+        taken += own_pages[b];
+    }
+    int32_t max_page = 0;
+    for (int32_t id : p->page_indices) {
         if (id < 0 || id > INT32_MAX / 64) { delete p; return CPA_EINVAL; }
-    p->seq_lens.assign(B, 0);
+        max_page = std::max(max_page, id);
+    }
+    p->pool_pages = max_page + 1;
+    p->seq_lens = p->prefix_lens;   // the prefix is cached already
 
-    // slot of every prefill token
+    // slot of every prefill token (positions count from the start of the sequence, prefix included)
     p->slot_mapping.resize((size_t)p->total_tokens);
     for (int32_t b = 0; b < B; ++b) {
         const int32_t* pages = p->page_indices.data() + p->page_indptr[b];
         int32_t* slots = p->slot_mapping.data() + p->cu_seqlens[b];
-        for (int32_t pos = 0; pos < block_lens[b]; ++pos) slots[pos] = pages[pos / P] * P + pos % P;
+        for (int32_t i = 0; i < block_lens[b]; ++i) {
+            const int32_t pos = p->prefix_lens[b] + i;
+            slots[i] = pages[pos / P] * P + pos % P;
+        }
     }
 
     // prefill work list: longest tiles first (later q tiles of a causal block see more keys)
@@ -80,7 +110,7 @@ extern "C" int cpa_plan_create(const cpa_config* cfg, int32_t num_blocks, const 
     for (int32_t b = 0; b < B; ++b) {
         int32_t n_tiles = (block_lens[b] + p->q_tile - 1) / p->q_tile;
         for (int32_t t = 0; t < n_tiles; ++t)
-            pit.push_back({std::min((t + 1) * p->q_tile, block_lens[b]), b, t});
+            pit.push_back({p->prefix_lens[b] + std::min((t + 1) * p->q_tile, block_lens[b]), b, t});
     }
     std::stable_sort(pit.begin(), pit.end(), [](const PItem& a, const PItem& c) {
         if (a.cost != c.cost) return a.cost > c.cost;
@@ -112,7 +142,7 @@ extern "C" int cpa_plan_create(const cpa_config* cfg, int32_t num_blocks, const 
                 const int32_t b = p->prefill_items[2 * i], t = p->prefill_items[2 * i + 1];
                 const int32_t q0 = t * p->q_tile;
                 const int32_t n_sub = (sub_per_item > 1 && block_lens[b] - q0 > 128) ? 2 : 1;
-                const int64_t cost = 10LL * (q0 / 128 + n_sub) + 18;
+                const int64_t cost = 10LL * (p->prefix_lens[b] / 128 + q0 / 128 + n_sub) + 18;
                 for (int32_t h = 0; h < G; ++h) {
                     Load l = heap.top();
                     heap.pop();
@@ -206,14 +236,16 @@ extern "C" int cpa_plan_create(const cpa_config* cfg, int32_t num_blocks, const 
     std::memcpy(im + p->off_sindptr, p->split_indptr.data(), sizeof(int32_t) * (B + 1));
     std::memcpy(im + p->off_pidx, p->page_indices.data(), sizeof(int32_t) * pages_used);
     for (int32_t i = 0; i < p->n_prefill; ++i) {
-        // a prefill item carries its block's token range, so a kernel needs one load per item
+        // a prefill item carries its block's token range and cached prefix (one 16-byte record), so a
+        // kernel needs no dependent loads per item
         const int32_t b = p->prefill_items[2 * i];
         int32_t* it = im + p->off_pitems + 4LL * i;
-        it[0] = b;
-        it[1] = p->prefill_items[2 * i + 1];
-        it[2] = p->cu_seqlens[b];
-        it[3] = p->block_lens[b];
+        it[0] = p->cu_seqlens[b];                                             // first token of the block
+        it[1] = p->block_lens[b];
+        it[2] = p->prefill_items[2 * i + 1] | ((p->prefix_lens[b] / 128) << 16);   // q item, KV tiles of the cached prefix
+        it[3] = p->page_indptr[b];                                            // where the sequence's page ids start
     }
+    for (int32_t b = 0; b < B; ++b) im[p->off_seqlens + b] = im[p->off_seqlens2 + b] = p->prefix_lens[b];
     std::memcpy(im + p->off_psched, p->prefill_sched.data(), sizeof(int32_t) * p->prefill_sched.size());
     for (int32_t i = 0; i < p->n_decode; ++i) {
         // a decode item carries its own page ids, so the kernel's first KV load depends on
@@ -231,6 +263,23 @@ extern "C" int cpa_plan_create(const cpa_config* cfg, int32_t num_blocks, const 
     p->append_stage.assign(B + 1, 0);
     *out = p;
     return CPA_OK;
+}
+}  // namespace
+
+extern "C" int cpa_plan_create(const cpa_config* cfg, int32_t num_blocks, const int32_t* block_lens,
+                               int32_t max_new_tokens, const int32_t* free_pages, int32_t num_free,
+                               cpa_plan** out) {
+    return plan_create(cfg, num_blocks, block_lens, nullptr, nullptr, 0, max_new_tokens, free_pages, num_free, out);
+}
+
+extern "C" int cpa_plan_create_prefix(const cpa_config* cfg, int32_t num_workers, const int32_t* own_lens,
+                                      const int32_t* prefix_lens, const int32_t* shared_pages, int32_t num_shared,
+                                      int32_t max_new_tokens, const int32_t* free_pages, int32_t num_free,
+                                      cpa_plan** out) {
+    if (out) *out = nullptr;
+    if (!prefix_lens) return CPA_EINVAL;
+    return plan_create(cfg, num_workers, own_lens, prefix_lens, shared_pages, num_shared, max_new_tokens, free_pages,
+                       num_free, out);
 }
 
 extern "C" int cpa_plan_export(const cpa_plan* plan, int which, const int32_t** ptr, int64_t* count) {
@@ -275,8 +324,8 @@ extern "C" int64_t cpa_plan_param(const cpa_plan* plan, int which) {
 extern "C" int cpa_plan_upload(cpa_plan* plan, void* d_index_buf, int64_t bytes, void* stream) {
     if (!plan || !d_index_buf || !cpa_aligned16(d_index_buf)) return CPA_EINVAL;
     if (bytes < plan->index_bytes()) return CPA_ENOSPC;
-    // the device copy starts from an empty cache, so the host mirror does too
-    std::fill(plan->seq_lens.begin(), plan->seq_lens.end(), 0);
+    // the device copy starts with nothing but the cached prefixes, so the host mirror does too
+    plan->seq_lens = plan->prefix_lens;
     plan->cur_lens = 0;
     cudaError_t e = cudaMemcpyAsync(d_index_buf, plan->image.data(), (size_t)plan->index_bytes(),
                                     cudaMemcpyHostToDevice, (cudaStream_t)stream);

@@ -80,10 +80,10 @@ prefill_mma_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __r
 
     // a work item of subs*128 query rows is covered by `subs` CTAs of 128 rows each
     const int item = blockIdx.x / subs;
-    const int b = ix.prefill_items[4 * item], tile = ix.prefill_items[4 * item + 1] * subs + (blockIdx.x - item * subs);
+    const int tile = (ix.prefill_items[4 * item + 2] & 0xFFFF) * subs + (blockIdx.x - item * subs);
     const int h = blockIdx.y, g = h / (Hq / Hkv);
-    const int tok0 = ix.cu_seqlens[b];
-    const int L = ix.cu_seqlens[b + 1] - tok0;
+    const int tok0 = ix.prefill_items[4 * item];
+    const int L = ix.prefill_items[4 * item + 1];
     const int q0 = tile * kQTile;
     if (q0 >= L) return;
     const int q_rows = min(kQTile, L - q0);
@@ -272,7 +272,16 @@ int cpa_prefill_mma(const cpa_plan* plan, const void* q, const void* k, const vo
                                      : launch_prefill_mma<64>(plan, q, k, v, o, st);
 }
 
-int cpa_prefill_tc(const cpa_plan* plan, const void* q, const void* k, const void* v, void* o, void* stream);
+int cpa_prefill_tc(const cpa_plan* plan, const void* q, const void* k, const void* v, void* o, const void* k_pool,
+                   const void* v_pool, void* stream);
+
+namespace {
+bool has_prefix(const cpa_plan* plan) {
+    for (int32_t n : plan->prefix_lens)
+        if (n > 0) return true;
+    return false;
+}
+}  // namespace
 
 extern "C" int cpa_prefill_variant(const cpa_plan* plan, const void* q, const void* k, const void* v, void* o,
                                    void* stream, int variant) {
@@ -280,7 +289,8 @@ extern "C" int cpa_prefill_variant(const cpa_plan* plan, const void* q, const vo
     if (!cpa_aligned16(q) || !cpa_aligned16(k) || !cpa_aligned16(v) || !cpa_aligned16(o)) return CPA_EINVAL;
     if (o == q || o == k || o == v) return CPA_EINVAL;
     if (!plan->d_base) return CPA_ESTATE;
-    if (variant == CPA_PREFILL_TENSOR_CORE) return cpa_prefill_tc(plan, q, k, v, o, stream);
+    if (has_prefix(plan)) return CPA_EINVAL;   // a cached prefix is read from the pools: cpa_prefill_prefix
+    if (variant == CPA_PREFILL_TENSOR_CORE) return cpa_prefill_tc(plan, q, k, v, o, nullptr, nullptr, stream);
     if (variant == CPA_PREFILL_WARP_MMA) return cpa_prefill_mma(plan, q, k, v, o, stream);
     return CPA_EINVAL;
 }
@@ -289,4 +299,15 @@ extern "C" int cpa_prefill(const cpa_plan* plan, const void* q, const void* k, c
                            void* d_workspace, void* stream) {
     (void)d_workspace;
     return cpa_prefill_variant(plan, q, k, v, o, stream, CPA_PREFILL_TENSOR_CORE);
+}
+
+extern "C" int cpa_prefill_prefix(const cpa_plan* plan, const void* q, const void* k, const void* v, const void* k_pool,
+                                  const void* v_pool, void* o, void* stream) {
+    if (!plan || !q || !k || !v || !o || !k_pool || !v_pool) return CPA_EINVAL;
+    if (!cpa_aligned16(q) || !cpa_aligned16(k) || !cpa_aligned16(v) || !cpa_aligned16(o) || !cpa_aligned16(k_pool) ||
+        !cpa_aligned16(v_pool))
+        return CPA_EINVAL;
+    if (o == q || o == k || o == v) return CPA_EINVAL;
+    if (!plan->d_base) return CPA_ESTATE;
+    return cpa_prefill_tc(plan, q, k, v, o, k_pool, v_pool, stream);
 }

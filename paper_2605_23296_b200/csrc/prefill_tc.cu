@@ -232,11 +232,15 @@ struct TcShape {
 
 // One unit of work = one (block, q item of `q_rows` = 128 or 256 rows, query head).  A 256-row item is
 // two 128-row sub-tiles u = 0, 1 that share every K/V tile; sub-tile u has its own softmax
-// warpgroup and its own O_u columns in TMEM, and sees KV tiles 0 .. t0+u (t0 = index of
-// sub-tile 0 in units of 128 rows; the last of them touches the diagonal).
+// warpgroup and its own O_u columns in TMEM, and sees KV tiles 0 .. t0+u; the last of them touches
+// the diagonal.  In the prefix-aware layout the sequence's cached prefix (whole tiles, every row sees
+// all of it) comes first and is staged from the paged pool; t0 = prefix tiles + index of sub-tile 0
+// among the sequence's own 128-row tiles.
 struct TcWork {
     int h, g, tok0, L, q0, t0, n_sub, n_total;   // n_total: KV tiles streamed; sub-tile u uses the first t0+1+u
-    bool valid;                                  // false: this CTA has no unit in that round (last round only)
+    int n_pre, page_base;                        // the first n_pre KV tiles are the sequence's cached prefix, read from
+                                                 // pool pages page_indices[page_base ...]; t0 counts them too
+    bool valid;                                  // false: this CTA has no unit in that round
 };
 
 // The grid is persistent: CTA c walks column c of the planner's schedule (units dealt greedily by
@@ -248,7 +252,8 @@ struct TcWork {
 template <int D>
 __global__ void __launch_bounds__(kThreads, 1)
 prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
-                  const __grid_constant__ CUtensorMap tm_v, __nv_bfloat16* __restrict__ o, cpa_dev_index ix, int Hq,
+                  const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_kpool,
+                  const __grid_constant__ CUtensorMap tm_vpool, __nv_bfloat16* __restrict__ o, cpa_dev_index ix, int Hq,
                   int Hkv, int q_rows, float scale_log2, int n_rounds) {
     using Sh = TcShape<D>;
     constexpr int NB = Sh::NB;
@@ -270,23 +275,26 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
     // round k+2 and the item record of round k+1 in flight while it works on round k, so neither of the
     // two dependent global loads sits between two units.
     auto fetch_code = [&](int k) { return k < n_rounds ? __ldg(ix.prefill_sched + (int64_t)k * G + blockIdx.x) : -1; };
-    auto fetch = [&](int code, int4& rec, int& h) {
-        rec = make_int4(0, 0, 0, 0);                  // block length 0: no unit in that round
-        h = 0;
+    struct Rec { int4 a; int h; };   // raw item record: (first token, length, q item | prefix tiles << 16, page base)
+    auto fetch = [&](int code, Rec& r) {
+        r.a = make_int4(0, 0, 0, 0);                  // block length 0: no unit in that round
+        r.h = 0;
         if (code >= 0) {
             const int it = code / Hq;
-            h = code - it * Hq;
-            rec = __ldg(reinterpret_cast<const int4*>(ix.prefill_items) + it);
+            r.h = code - it * Hq;
+            r.a = __ldg(reinterpret_cast<const int4*>(ix.prefill_items) + it);
         }
     };
-    auto decode = [&](const int4& rec, int h, TcWork& w) {
-        w.valid = rec.w > 0;
-        w.h = h;
-        w.g = h / group;
-        w.tok0 = rec.z;
-        w.L = rec.w;
-        w.q0 = rec.y * q_rows;
-        w.t0 = w.q0 / kTileM;
+    auto decode = [&](const Rec& r, TcWork& w) {
+        w.valid = r.a.y > 0;
+        w.h = r.h;
+        w.g = r.h / group;
+        w.tok0 = r.a.x;
+        w.L = r.a.y;
+        w.q0 = (r.a.z & 0xFFFF) * q_rows;
+        w.n_pre = r.a.z >> 16;
+        w.page_base = r.a.w;
+        w.t0 = w.n_pre + w.q0 / kTileM;
         w.n_sub = (q_rows > kTileM && w.L - w.q0 > kTileM) ? 2 : 1;
         w.n_total = w.t0 + w.n_sub;
     };
@@ -328,43 +336,101 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
     asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;\n" :: "n"(kRegsControl));
     if (warp == 8) {
         // ------------------------------------------------------------ TMA producer
-        if (lane == 0) {
+        // Lane 0 waits and issues the loads from the packed tensors.  A KV tile of a cached prefix is
+        // eight pool pages: lanes 0-7 take one page each.  A (page, head) chunk of the pool is 16 rows
+        // whose 128-byte groups are stored in the swizzled order already (see cpa_pool_piece), so a
+        // plain copy of 16 rows x 128 bytes lands as rows 16p .. 16p+15 of a swizzled column block.
+        {
             int kt = 0;                   // K/V tiles loaded so far: stage kt % KS, use count kt / KS
             uint32_t q_loads[2] = {0, 0};   // loads of Q_u so far
             TcWork w;
-            int4 rec;
-            int rec_h;
-            fetch(fetch_code(0), rec, rec_h);
+            Rec rec;
+            fetch(fetch_code(0), rec);
             int code = fetch_code(1);
             for (int k = 0; k < n_rounds; ++k) {
-                decode(rec, rec_h, w);
-                fetch(code, rec, rec_h);
+                decode(rec, w);
+                fetch(code, rec);
                 code = fetch_code(k + 2);
                 if (!w.valid) continue;
-                for (int u = 0; u < w.n_sub; ++u) {
-                    // the buffer is free once the last score MMA of its previous unit has run
-                    mbar_wait(bar(&bars.q_empty[u]), (q_loads[u] & 1u) ^ 1u, dead, ix.status);
-                    ++q_loads[u];
-                    mbar_expect_tx(bar(&bars.q_full[u]), kTileBytes);
+                if (lane == 0) {
+                    for (int u = 0; u < w.n_sub; ++u) {
+                        // the buffer is free once the last score MMA of its previous unit has run
+                        mbar_wait(bar(&bars.q_empty[u]), (q_loads[u] & 1u) ^ 1u, dead, ix.status);
+                        ++q_loads[u];
+                        mbar_expect_tx(bar(&bars.q_full[u]), kTileBytes);
 #pragma unroll
-                    for (int c = 0; c < NB; ++c)
-                        tma_load_2d(s_q + u * kTileBytes + c * kBlockBytes, &tm_q, w.h * D + 64 * c,
-                                    w.tok0 + w.q0 + u * kTileM, bar(&bars.q_full[u]));
+                        for (int c = 0; c < NB; ++c)
+                            tma_load_2d(s_q + u * kTileBytes + c * kBlockBytes, &tm_q, w.h * D + 64 * c,
+                                        w.tok0 + w.q0 + u * kTileM, bar(&bars.q_full[u]));
+                    }
                 }
+                if (w.n_pre == 0) {
+                    // no cached prefix: one lane streams the K/V tiles of the packed tensors
+                    if (lane == 0) {
+                        for (int j = 0; j < w.n_total; ++j, ++kt) {
+                            const int s = kt % KS;
+                            const uint32_t par = (uint32_t)(kt / KS) & 1u;
+                            const int row = w.tok0 + j * kTileN;
+                            mbar_wait(bar(&bars.k_empty[s]), par ^ 1u, dead, ix.status);
+                            mbar_expect_tx(bar(&bars.k_full[s]), kTileBytes);
+#pragma unroll
+                            for (int c = 0; c < NB; ++c)
+                                tma_load_2d(s_k + s * kTileBytes + c * kBlockBytes, &tm_k, w.g * D + 64 * c, row, bar(&bars.k_full[s]));
+                            mbar_wait(bar(&bars.v_empty[s]), par ^ 1u, dead, ix.status);
+                            mbar_expect_tx(bar(&bars.v_full[s]), kTileBytes);
+#pragma unroll
+                            for (int c = 0; c < NB; ++c)
+                                tma_load_2d(s_v + s * kTileBytes + c * kBlockBytes, &tm_v, w.g * D + 64 * c, row, bar(&bars.v_full[s]));
+                        }
+                    } else {
+                        kt += w.n_total;
+                    }
+                    __syncwarp();
+                    continue;
+                }
+                // page of this lane in the next prefix tile, fetched one tile ahead
+                int page = lane < 8 ? __ldg(ix.page_indices + w.page_base + lane) : 0;
                 for (int j = 0; j < w.n_total; ++j, ++kt) {
                     const int s = kt % KS;
                     const uint32_t par = (uint32_t)(kt / KS) & 1u;
-                    const int row = w.tok0 + j * kTileN;
-                    mbar_wait(bar(&bars.k_empty[s]), par ^ 1u, dead, ix.status);
-                    mbar_expect_tx(bar(&bars.k_full[s]), kTileBytes);
+                    const bool cached = j < w.n_pre;
+                    const int my_page = page;
+                    if (lane < 8 && j + 1 < w.n_pre) page = __ldg(ix.page_indices + w.page_base + 8 * (j + 1) + lane);
+                    const int row = cached ? (my_page * Hkv + w.g) * 16 : w.tok0 + (j - w.n_pre) * kTileN;
+                    if (lane == 0) {
+                        mbar_wait(bar(&bars.k_empty[s]), par ^ 1u, dead, ix.status);
+                        mbar_expect_tx(bar(&bars.k_full[s]), kTileBytes);
+                    }
+                    __syncwarp();
+                    if (cached) {
+                        if (lane < 8) {
 #pragma unroll
-                    for (int c = 0; c < NB; ++c)
-                        tma_load_2d(s_k + s * kTileBytes + c * kBlockBytes, &tm_k, w.g * D + 64 * c, row, bar(&bars.k_full[s]));
-                    mbar_wait(bar(&bars.v_empty[s]), par ^ 1u, dead, ix.status);
-                    mbar_expect_tx(bar(&bars.v_full[s]), kTileBytes);
+                            for (int c = 0; c < NB; ++c)
+                                tma_load_2d(s_k + s * kTileBytes + c * kBlockBytes + lane * 2048, &tm_kpool, 64 * c, row,
+                                            bar(&bars.k_full[s]));
+                        }
+                    } else if (lane == 0) {
 #pragma unroll
-                    for (int c = 0; c < NB; ++c)
-                        tma_load_2d(s_v + s * kTileBytes + c * kBlockBytes, &tm_v, w.g * D + 64 * c, row, bar(&bars.v_full[s]));
+                        for (int c = 0; c < NB; ++c)
+                            tma_load_2d(s_k + s * kTileBytes + c * kBlockBytes, &tm_k, w.g * D + 64 * c, row, bar(&bars.k_full[s]));
+                    }
+                    if (lane == 0) {
+                        mbar_wait(bar(&bars.v_empty[s]), par ^ 1u, dead, ix.status);
+                        mbar_expect_tx(bar(&bars.v_full[s]), kTileBytes);
+                    }
+                    __syncwarp();
+                    if (cached) {
+                        if (lane < 8) {
+#pragma unroll
+                            for (int c = 0; c < NB; ++c)
+                                tma_load_2d(s_v + s * kTileBytes + c * kBlockBytes + lane * 2048, &tm_vpool, 64 * c, row,
+                                            bar(&bars.v_full[s]));
+                        }
+                    } else if (lane == 0) {
+#pragma unroll
+                        for (int c = 0; c < NB; ++c)
+                            tma_load_2d(s_v + s * kTileBytes + c * kBlockBytes, &tm_v, w.g * D + 64 * c, row, bar(&bars.v_full[s]));
+                    }
                 }
             }
         }
@@ -417,13 +483,12 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
         // buffer n mod NBUF, and QK(n + NBUF) is queued right behind PV(n), which reads the buffer it
         // overwrites.  All buffers are free again once the last PV of a unit has been queued.
         TcWork w;
-        int4 rec;
-        int rec_h;
-        fetch(fetch_code(0), rec, rec_h);
+        Rec rec;
+        fetch(fetch_code(0), rec);
         int code = fetch_code(1);
         for (int r = 0; r < n_rounds; ++r) {
-            decode(rec, rec_h, w);
-            fetch(code, rec, rec_h);
+            decode(rec, w);
+            fetch(code, rec);
             code = fetch_code(r + 2);
             if (!w.valid) continue;
             const int t0 = w.t0;
@@ -512,13 +577,12 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
         uint32_t n_units = 0;       // units this sub-tile took part in
         int kt0 = 0;                // K/V tiles of earlier units
         TcWork w;
-        int4 rec;
-        int rec_h;
-        fetch(fetch_code(0), rec, rec_h);
+        Rec rec;
+        fetch(fetch_code(0), rec);
         int code = fetch_code(1);
         for (int rd = 0; rd < n_rounds; ++rd) {
-        decode(rec, rec_h, w);
-        fetch(code, rec, rec_h);
+        decode(rec, w);
+        fetch(code, rec);
         code = fetch_code(rd + 2);
         if (!w.valid) continue;
         if (u < w.n_sub) {
@@ -678,8 +742,23 @@ bool make_map(CUtensorMap* map, const void* ptr, int64_t rows, int64_t cols) {
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// 2-D view [rows = pages * kv_heads * 16 slots][cols = D] of a paged pool; box = 64 cols x 16 rows (one
+// 128-byte group of every slot of a (page, head) chunk), copied as stored.
+bool make_pool_map(CUtensorMap* map, const void* ptr, int64_t rows, int64_t cols) {
+    EncodeTiledFn fn = get_encode_fn();
+    if (!fn) return false;
+    const cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+    const cuuint64_t strides[1] = {(cuuint64_t)cols * 2};
+    const cuuint32_t box[2] = {64, 16};
+    const cuuint32_t elem[2] = {1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, elem,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 template <int D>
-int launch_prefill_tc(const cpa_plan* plan, const void* q, const void* k, const void* v, void* o, cudaStream_t st) {
+int launch_prefill_tc(const cpa_plan* plan, const void* q, const void* k, const void* v, void* o, const void* k_pool,
+                      const void* v_pool, cudaStream_t st) {
     const cpa_config& c = plan->cfg;
     constexpr int smem = TcShape<D>::kSmem;
     static bool configured_dev[64] = {};  // the attribute is per device: remember which devices have it
@@ -706,17 +785,26 @@ int launch_prefill_tc(const cpa_plan* plan, const void* q, const void* k, const 
         !make_map(&tm_k, k, plan->total_tokens, (int64_t)c.num_kv_heads * D) ||
         !make_map(&tm_v, v, plan->total_tokens, (int64_t)c.num_kv_heads * D))
         return CPA_ECUDA;
+    // pools are only read for sequences with a cached prefix; without pools the maps are never used
+    CUtensorMap tm_kpool = tm_k, tm_vpool = tm_v;
+    if (k_pool && v_pool) {
+        const int64_t pool_rows = (int64_t)plan->pool_pages * c.num_kv_heads * c.page_size;
+        if (!make_pool_map(&tm_kpool, k_pool, pool_rows, D) || !make_pool_map(&tm_vpool, v_pool, pool_rows, D))
+            return CPA_ECUDA;
+    }
     // persistent grid: one CTA per SM, each walks its column of the planner's schedule
-    prefill_tc_kernel<D><<<plan->prefill_ctas, kThreads, smem, st>>>(tm_q, tm_k, tm_v, (__nv_bfloat16*)o, plan->dev(),
-                                                                   c.num_q_heads, c.num_kv_heads, plan->q_tile,
+    prefill_tc_kernel<D><<<plan->prefill_ctas, kThreads, smem, st>>>(tm_q, tm_k, tm_v, tm_kpool, tm_vpool,
+                                                                   (__nv_bfloat16*)o, plan->dev(), c.num_q_heads,
+                                                                   c.num_kv_heads, plan->q_tile,
                                                                    c.scale * 1.4426950408889634f, plan->prefill_rounds);
     return cudaGetLastError() == cudaSuccess ? CPA_OK : CPA_ECUDA;
 }
 
 }  // namespace
 
-int cpa_prefill_tc(const cpa_plan* plan, const void* q, const void* k, const void* v, void* o, void* stream) {
+int cpa_prefill_tc(const cpa_plan* plan, const void* q, const void* k, const void* v, void* o, const void* k_pool,
+                   const void* v_pool, void* stream) {
     cudaStream_t st = (cudaStream_t)stream;
-    return plan->cfg.head_dim == 128 ? launch_prefill_tc<128>(plan, q, k, v, o, st)
-                                     : launch_prefill_tc<64>(plan, q, k, v, o, st);
+    return plan->cfg.head_dim == 128 ? launch_prefill_tc<128>(plan, q, k, v, o, k_pool, v_pool, st)
+                                     : launch_prefill_tc<64>(plan, q, k, v, o, k_pool, v_pool, st);
 }

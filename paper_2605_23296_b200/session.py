@@ -37,7 +37,9 @@ class CompactionSession:
     def __init__(self, block_lens: Sequence[int], max_new_tokens: int, num_q_heads: int,
                  num_kv_heads: int, head_dim: int, free_pages: Sequence[int], num_pages: int,
                  scale: Optional[float] = None, device: str = "cuda:0", pages_per_split: int = 0,
-                 poison_pools: bool = False, page_size: int = 16, q_tile_rows: int = 0):
+                 poison_pools: bool = False, page_size: int = 16, q_tile_rows: int = 0,
+                 prefix_lens: Optional[Sequence[int]] = None, shared_pages: Optional[Sequence[int]] = None,
+                 pools=None):
         self.device = torch.device(device)
         self.Hq, self.Hkv, self.d, self.P = num_q_heads, num_kv_heads, head_dim, page_size
         self.B = len(block_lens)
@@ -46,12 +48,20 @@ class CompactionSession:
         props = torch.cuda.get_device_properties(self.device)
         self.cfg = B.cpa_config(num_q_heads, num_kv_heads, head_dim, page_size, self.scale, q_tile_rows,
                                 pages_per_split, props.multi_processor_count)
-        self.plan = B.cpa_plan_create(self.cfg, self.block_lens, max_new_tokens, free_pages)
+        self.prefix_aware = prefix_lens is not None
+        if self.prefix_aware:   # the paper's layout: cached history prefix + own tokens per worker
+            self.plan = B.cpa_plan_create_prefix(self.cfg, self.block_lens, prefix_lens, shared_pages,
+                                                 max_new_tokens, free_pages)
+        else:
+            self.plan = B.cpa_plan_create(self.cfg, self.block_lens, max_new_tokens, free_pages)
         self.total_tokens = B.cpa_plan_param(self.plan, B.PARAM_TOTAL_TOKENS)
         nbytes = B.cpa_plan_param(self.plan, B.PARAM_INDEX_BYTES)
         self.index_buf = torch.empty(nbytes, dtype=torch.uint8, device=self.device)
         pool_shape = (num_pages, num_kv_heads, page_size, head_dim)
-        if poison_pools:   # unused slots hold NaN: the kernels must mask by index, not by value
+        if pools is not None:   # pools that already hold a cached history (shared with another session)
+            self.k_pool, self.v_pool = pools
+            assert tuple(self.k_pool.shape) == pool_shape and tuple(self.v_pool.shape) == pool_shape
+        elif poison_pools:   # unused slots hold NaN: the kernels must mask by index, not by value
             self.k_pool = torch.full(pool_shape, float("nan"), dtype=torch.bfloat16, device=self.device)
             self.v_pool = torch.full(pool_shape, float("nan"), dtype=torch.bfloat16, device=self.device)
         else:  # no initialisation needed: slots are masked by index until they are written
@@ -82,7 +92,10 @@ class CompactionSession:
         """Causal attention of every block over itself; q/out [tokens,Hq,d], k/v [tokens,Hkv,d]."""
         if out is None:
             out = torch.empty_like(q)
-        if variant is None:
+        if self.prefix_aware:
+            self._check(B.cpa_prefill_prefix(self.plan, q, k, v, self.k_pool, self.v_pool, out, self._stream()),
+                        "cpa_prefill_prefix")
+        elif variant is None:
             self._check(B.cpa_prefill(self.plan, q, k, v, out, None, self._stream()), "cpa_prefill")
         else:
             self._check(B.cpa_prefill_variant(self.plan, q, k, v, out, self._stream(), variant),

@@ -1,0 +1,151 @@
+"""Parity of the prefix-aware layout (paper, Section 4: a worker's prompt is the cached history up to
+its block, then its own tokens) on the CUDA path, through the C-ABI, against the CPU oracle: page
+table and pool bytes bit-exact, attention within max-abs 1e-2 / mean-abs 1e-3."""
+import numpy as np
+import pytest
+
+from _util import assert_attention_close, pool_rows
+from oracle import attention as oa
+from oracle import plan as op
+from paper_2605_23296_b200 import workloads as wl
+
+pytestmark = pytest.mark.gpu
+
+
+def _dev(bits):
+    from paper_2605_23296_b200.session import bits_to_tensor
+    return bits_to_tensor(bits, "cuda:0")
+
+
+def _bits(t):
+    from paper_2605_23296_b200.session import tensor_to_bits
+    return tensor_to_bits(t)
+
+
+def _sessions(w, poison=True, pages_per_split=0, q_tile_rows=0):
+    """(history session or None, workers' session): the history is cached first, through a plan of
+    its own that owns the shared pages; the workers' plan then reads those pages."""
+    import torch
+    from paper_2605_23296_b200.session import CompactionSession
+    o = w.own
+    shape = (w.num_pages, o.num_kv_heads, o.page_size, o.head_dim)
+    fill = float("nan") if poison else 0.0
+    pools = (torch.full(shape, fill, dtype=torch.bfloat16, device="cuda:0"),
+             torch.full(shape, fill, dtype=torch.bfloat16, device="cuda:0"))
+    hist = None
+    if w.hist_tokens:
+        hist = CompactionSession([w.hist_tokens], 0, o.num_q_heads, o.num_kv_heads, o.head_dim, w.shared_pages,
+                                 w.num_pages, scale=o.scale, pools=pools)
+        hist.append_prefill(_dev(w.k_hist), _dev(w.v_hist))
+    s = CompactionSession(o.block_lens, o.decode_steps, o.num_q_heads, o.num_kv_heads, o.head_dim, o.free_pages,
+                          w.num_pages, scale=o.scale, pages_per_split=pages_per_split, q_tile_rows=q_tile_rows,
+                          prefix_lens=w.prefix_lens, shared_pages=w.shared_pages, pools=pools)
+    return hist, s
+
+
+def _cu(o):
+    return np.concatenate([[0], np.cumsum(o.block_lens.astype(np.int64))])
+
+
+def run_event(w, pages_per_split=0, q_tile_rows=0, fused_every=2):
+    from paper_2605_23296_b200 import binding as B
+    o = w.own
+    cu = _cu(o)
+    hist, s = _sessions(w, pages_per_split=pages_per_split, q_tile_rows=q_tile_rows)
+    try:
+        # page table: bit-exact with the restated rules
+        C = s.export(B.ARR_SPLIT_PAGES).tolist()
+        ref = op.build_plan(o.block_lens.tolist(), o.decode_steps, o.page_size, o.free_pages.tolist(), o.num_kv_heads,
+                            s.param(B.PARAM_Q_TILE_ROWS), C, prefix_lens=w.prefix_lens.tolist(),
+                            shared_pages=w.shared_pages.tolist())
+        for which, key in [(B.ARR_PAGE_INDPTR, "page_indptr"), (B.ARR_PAGE_INDICES, "page_indices"),
+                           (B.ARR_SLOT_MAPPING, "slot_mapping"), (B.ARR_SEQ_LENS, "seq_lens")]:
+            assert np.array_equal(s.export(which), np.asarray(ref[key], dtype=np.int32)), key
+        # prefill of the own tokens over prefix + own tokens
+        k, v = _dev(o.k), _dev(o.v)
+        out = s.prefill(_dev(o.q), k, v)
+        want = oa.prefill_prefix_aware(o.q, o.k, o.v, cu, w.k_hist, w.v_hist, w.prefix_lens, o.scale)
+        assert s.status() == 0
+        assert_attention_close(_bits(out), want, f"{o.name} prefix-aware prefill")
+        # the own tokens go behind the prefix, the shared pages keep the history bit for bit
+        s.append_prefill(k, v)
+        kp, vp = pool_rows(_bits(s.k_pool)), pool_rows(_bits(s.v_pool))
+        P = o.page_size
+        for i, slot in enumerate(ref["slot_mapping"]):
+            assert np.array_equal(kp[slot // P, :, slot % P], o.k[i]) and np.array_equal(vp[slot // P, :, slot % P], o.v[i])
+        for t in range(w.hist_tokens):
+            page = int(w.shared_pages[t // P])
+            assert np.array_equal(kp[page, :, t % P], w.k_hist[t]) and np.array_equal(vp[page, :, t % P], w.v_hist[t])
+        # decode over shared prefix pages + own pages
+        st = oa.PrefixDecodeState(o.k, o.v, cu, w.k_hist, w.v_hist, w.prefix_lens, o.decode_steps)
+        for t in range(o.decode_steps):
+            st.append(o.k_dec[t], o.v_dec[t])
+            if fused_every and t % fused_every == 0:
+                got = s.decode_append(_dev(o.q_dec[t]), _dev(o.k_dec[t]), _dev(o.v_dec[t]))
+            else:
+                s.append(_dev(o.k_dec[t]), _dev(o.v_dec[t]))
+                got = s.decode(_dev(o.q_dec[t]))
+            assert_attention_close(_bits(got), st.decode(o.q_dec[t], o.scale), f"{o.name} prefix-aware decode step {t}")
+        assert s.status() == 0
+        assert np.array_equal(s.export(B.ARR_SEQ_LENS), w.prefix_lens + o.block_lens + o.decode_steps)
+    finally:
+        s.close()
+        if hist is not None:
+            hist.close()
+
+
+@pytest.mark.parametrize("workers,block_len,hq,hkv,d", [(3, 128, 4, 1, 64), (4, 256, 8, 2, 128), (3, 384, 8, 8, 128),
+                                                        (5, 128, 16, 2, 64)])
+def test_prefix_aware_event(workers, block_len, hq, hkv, d):
+    run_event(wl.prefix_aware(workers, block_len, hq, hkv, d, steps=5, seed=workers + d).materialise())
+
+
+def test_prefix_aware_markers_make_ragged_own_lengths():
+    # own lengths that are not multiples of anything: partial last q tile, partial last page
+    run_event(wl.prefix_aware(3, 256, 8, 2, 128, steps=3, seed=31, marker_tokens=37).materialise())
+
+
+@pytest.mark.parametrize("q_tile_rows", [128, 256])
+def test_prefix_aware_both_work_item_sizes(q_tile_rows):
+    run_event(wl.prefix_aware(3, 256, 4, 2, 64, steps=2, seed=17).materialise(), q_tile_rows=q_tile_rows)
+
+
+def test_prefix_aware_small_decode_splits():
+    run_event(wl.prefix_aware(3, 256, 8, 2, 128, steps=4, seed=23).materialise(), pages_per_split=3)
+
+
+def test_single_worker_has_no_prefix_and_equals_plain_prefill():
+    from paper_2605_23296_b200.session import CompactionSession
+    w = wl.prefix_aware(1, 256, 8, 2, 128, steps=0, seed=5).materialise()
+    o = w.own
+    _, s = _sessions(w)
+    plain = CompactionSession(o.block_lens, 0, o.num_q_heads, o.num_kv_heads, o.head_dim, o.free_pages, w.num_pages,
+                              scale=o.scale)
+    try:
+        a = s.prefill(_dev(o.q), _dev(o.k), _dev(o.v))
+        b = plain.prefill(_dev(o.q), _dev(o.k), _dev(o.v))
+        assert np.array_equal(_bits(a), _bits(b))
+    finally:
+        s.close()
+        plain.close()
+
+
+def test_long_prefix_sampled_rows():
+    # 8 workers x 2048-token blocks: prefixes up to 14336 tokens (112 tiles); rows sampled per worker
+    w = wl.prefix_aware(8, 2048, 32, 8, 128, steps=0, seed=41).materialise(with_decode=False)
+    o = w.own
+    cu = _cu(o)
+    hist, s = _sessions(w, poison=False)
+    try:
+        out = _bits(s.prefill(_dev(o.q), _dev(o.k), _dev(o.v)))
+        assert s.status() == 0
+        rng = np.random.default_rng(0)
+        rows = []
+        for b in range(o.num_blocks):
+            L = int(o.block_lens[b])
+            rows += [int(cu[b]) + r for r in sorted({0, 1, 127, 128, 129, 255, 256, L - 1} | set(rng.integers(0, L, 6).tolist()))]
+        want = oa.prefill_prefix_aware(o.q, o.k, o.v, cu, w.k_hist, w.v_hist, w.prefix_lens, o.scale, rows=rows)
+        assert_attention_close(out[rows], want, "long prefix, sampled rows")
+    finally:
+        s.close()
+        hist.close()

@@ -168,3 +168,52 @@ def test_library_exports_every_declared_symbol():
     lib = ctypes.CDLL(B.LIB_PATH)
     for n in sorted(names):
         assert hasattr(lib, n), n
+
+
+# ----------------------------------------------------------------------------
+# prefix-aware layout: shared prefix pages
+# ----------------------------------------------------------------------------
+
+def _prefix_plan(w, pages_per_split=0, check=True, prefix_lens=None, shared=None):
+    o = w.own
+    cfg = B.cpa_config(o.num_q_heads, o.num_kv_heads, o.head_dim, o.page_size, o.scale, 0, pages_per_split, 0)
+    return B.cpa_plan_create_prefix(cfg, o.block_lens, w.prefix_lens if prefix_lens is None else prefix_lens,
+                                    w.shared_pages if shared is None else shared, o.decode_steps, o.free_pages,
+                                    check=check)
+
+
+@pytest.mark.parametrize("pps", [0, 5])
+def test_prefix_plan_bit_exact(pps):
+    w = wl.prefix_aware(5, 384, 8, 2, 128, steps=7, seed=3, marker_tokens=21).materialise(with_decode=False)
+    o = w.own
+    plan = _prefix_plan(w, pps)
+    try:
+        C = B.cpa_plan_export(plan, B.ARR_SPLIT_PAGES).tolist()
+        M = B.cpa_plan_param(plan, B.PARAM_Q_TILE_ROWS)
+        ref = op.build_plan(o.block_lens.tolist(), o.decode_steps, o.page_size, o.free_pages.tolist(), o.num_kv_heads,
+                            M, C, prefix_lens=w.prefix_lens.tolist(), shared_pages=w.shared_pages.tolist())
+        for which, key in [(B.ARR_CU_SEQLENS, "cu_seqlens"), (B.ARR_PAGE_INDPTR, "page_indptr"),
+                           (B.ARR_PAGE_INDICES, "page_indices"), (B.ARR_SEQ_LENS, "seq_lens"),
+                           (B.ARR_SLOT_MAPPING, "slot_mapping"), (B.ARR_PREFILL_ITEMS, "prefill_items"),
+                           (B.ARR_DECODE_ITEMS, "decode_items"), (B.ARR_SPLIT_INDPTR, "split_indptr")]:
+            got = B.cpa_plan_export(plan, which)
+            assert np.array_equal(got, np.asarray(ref[key], dtype=np.int32).reshape(got.shape)), key
+        ctas = B.cpa_plan_param(plan, B.PARAM_PREFILL_CTAS)
+        want = op.prefill_schedule(o.block_lens.tolist(), ref["prefill_items"], M, o.num_q_heads, o.num_kv_heads, 148,
+                                   prefix_lens=w.prefix_lens.tolist())
+        assert np.array_equal(B.cpa_plan_export(plan, B.ARR_PREFILL_SCHED).reshape(-1, ctas), np.asarray(want, dtype=np.int32))
+        assert B.cpa_plan_param(plan, B.PARAM_PAGES_USED) == ref["page_indptr"][-1]
+    finally:
+        B.cpa_plan_destroy(plan)
+
+
+def test_prefix_plan_errors():
+    w = wl.prefix_aware(3, 128, 4, 1, 64, steps=2, seed=1).materialise(with_decode=False)
+    for bad in ([0, 128, 200], [0, -128, 256], [0, 128, 16]):       # not a multiple of 128 / negative
+        rc, h = _prefix_plan(w, check=False, prefix_lens=bad)
+        assert rc == B.CPA_EINVAL and not h
+    rc, h = _prefix_plan(w, check=False, shared=w.shared_pages[:-1])  # prefix longer than the shared pages
+    assert rc == B.CPA_EINVAL and not h
+    w.own.free_pages = w.own.free_pages[:2]                              # own pages do not fit
+    rc, h = _prefix_plan(w, check=False)
+    assert rc == B.CPA_ENOSPC and not h
