@@ -423,13 +423,118 @@ def run_gpu(args) -> None:
         dist.destroy_process_group()
 
 
+# ------------------------------------------------------------------------------------------
+# the paper's own layout (prefix-aware target-at-end): a separate, non-default workload
+# ------------------------------------------------------------------------------------------
+
+def run_prefix(args) -> None:
+    """`--config prefix8b`: W workers over one cached history (paper, Section 4): worker w prefills
+    its own block (+ markers) over the w cached blocks before it, then all W decode T tokens.  The
+    history's K/V are in the pool before the timed region (they are the conversation's KV cache)."""
+    import torch
+
+    from paper_2605_23296_b200.session import CompactionSession, bits_to_tensor
+
+    if int(os.environ.get("WORLD_SIZE", "1")) != 1:
+        raise SystemExit("--config prefix8b is a single-GPU measurement")
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    peaks, peak_kind = load_peaks()
+    W = args.blocks or 16
+    block_len = args.block_len or 8192
+    T = args.decode_steps or 256
+    w = wl.prefix_aware(W, block_len, 32, 8, 128, T, seed=11, permute_pages=False).materialise()
+    o = w.own
+    stream = torch.cuda.current_stream(dev)
+    d = lambda bits: bits_to_tensor(bits, dev)
+    shape = (w.num_pages, o.num_kv_heads, o.page_size, o.head_dim)
+    pools = (torch.empty(shape, dtype=torch.bfloat16, device=dev), torch.empty(shape, dtype=torch.bfloat16, device=dev))
+    hist = CompactionSession([w.hist_tokens], 0, o.num_q_heads, o.num_kv_heads, o.head_dim, w.shared_pages, w.num_pages,
+                             scale=o.scale, pools=pools)
+    hist.append_prefill(d(w.k_hist), d(w.v_hist))
+    q, k, v, qd, kd, vd = (d(x) for x in (o.q, o.k, o.v, o.q_dec, o.k_dec, o.v_dec))
+    out = torch.empty_like(q)
+    od = torch.empty((T, W, o.num_q_heads, o.head_dim), dtype=torch.bfloat16, device=dev)
+    flush = torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device=dev)
+
+    def one_pass(ev=None):
+        s = CompactionSession(o.block_lens, T, o.num_q_heads, o.num_kv_heads, o.head_dim, o.free_pages, w.num_pages,
+                              scale=o.scale, prefix_lens=w.prefix_lens, shared_pages=w.shared_pages, pools=pools)
+        if ev:
+            ev["planned"].record(stream)
+        s.prefill(q, k, v, out=out)
+        if ev:
+            ev["prefilled"].record(stream)
+        s.append_prefill(k, v)
+        if ev:
+            ev["appended"].record(stream)
+        for t in range(T):
+            s.decode_append(qd[t], kd[t], vd[t], out=od[t])
+        return s
+
+    for _ in range(args.warmup):
+        s = one_pass()
+        torch.cuda.synchronize(dev)
+        assert s.status() == 0
+        s.close()
+    sampler = ClockSampler(0)
+    sampler.start()
+    step_ms, prefill_ms, decode_ms = [], [], []
+    for _ in range(args.steps):
+        flush.fill_(1)
+        ev = {n: torch.cuda.Event(enable_timing=True) for n in ("start", "planned", "prefilled", "appended", "end")}
+        ev["start"].record(stream)
+        s = one_pass(ev)
+        ev["end"].record(stream)
+        torch.cuda.synchronize(dev)
+        assert s.status() == 0
+        s.close()
+        step_ms.append(ev["start"].elapsed_time(ev["end"]))
+        prefill_ms.append(ev["planned"].elapsed_time(ev["prefilled"]))
+        decode_ms.append(ev["appended"].elapsed_time(ev["end"]))
+    clocks = sampler.stop()
+    hist.close()
+
+    L = o.block_lens.astype(np.float64)
+    pre = w.prefix_lens.astype(np.float64)
+    # every own row sees the whole prefix, plus the causal half of the own tokens
+    flops = float((4.0 * o.num_q_heads * o.head_dim * (L * pre + L * (L + 1.0) / 2.0)).sum())
+    row_bytes = 2.0 * o.num_kv_heads * o.head_dim * 2.0
+    # what this decode reads: every worker streams its whole prompt (prefix included) every step;
+    # `unique` counts each cached history page once per step
+    read = sum(float((pre + L + t + 1).sum()) * row_bytes for t in range(T))
+    unique = sum((float(pre.max()) + float((L + t + 1).sum())) * row_bytes for t in range(T))
+    ms, pf_ms, dc_ms = (statistics.mean(x) for x in (step_ms, prefill_ms, decode_ms))
+    # algorithmic bytes: each cached K and V element once per step and kv head, however many workers
+    # share it; `read` is what the kernel asks for (part of it served from L2)
+    achieved = unique / (dc_ms * 1e-3) / 1e9
+    print(json.dumps({
+        "metric": METRIC, "value": W * T / (ms * 1e-3), "unit": UNIT, "n_gpus": 1, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": o.name, "layout": "prefix-aware target-at-end", "workers": W, "block_len": block_len,
+                   "marker_tokens": w.marker_tokens, "history_tokens_cached": w.hist_tokens, "q_heads": o.num_q_heads,
+                   "kv_heads": o.num_kv_heads, "head_dim": o.head_dim, "decode_steps": T, "page_size": o.page_size,
+                   "seed": o.seed, "l2": "256 MiB write between timed steps"},
+        "phases": {"prefill_ms": pf_ms, "decode_ms": dc_ms, "prefill_tflops": flops / (pf_ms * 1e-3) / 1e12,
+                   "prefill_frac_of_bf16_peak": flops / (pf_ms * 1e-3) / 1e12 / peaks["bf16_tflops"],
+                   "decode_gbs_unique_pages": achieved, "decode_gbs_requested": read / (dc_ms * 1e-3) / 1e9,
+                   "peaks": dict(peaks, kind=peak_kind)},
+        "roofline": {"bound": "hbm", "kernel": "decode_split_kernel over shared prefix pages + own pages",
+                     "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"],
+                     "peak_kind": f"of {peak_kind}", "launch_us": dc_ms * 1e3 / T, "bytes_per_launch": unique / T,
+                     "requested_bytes_per_launch": read / T, "traffic": None},
+        "gpu_launches": args.steps * (3 + T), "clocks": clocks,
+    }))
+
+
 def main() -> None:
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--config", default="dense8b", choices=sorted(wl.CONFIGS))
+    ap.add_argument("--config", default="dense8b", choices=sorted(wl.CONFIGS) + ["prefix8b"])
     ap.add_argument("--blocks", type=int, default=0, help="override the number of blocks (profiling)")
     ap.add_argument("--block-len", type=int, default=0, help="override the block length (profiling)")
     ap.add_argument("--decode-steps", type=int, default=0, help="override the decode steps (profiling)")
@@ -444,7 +549,11 @@ def main() -> None:
         ap.error("--block-len does not apply to this configuration")
     if args.config == "tiny":
         args.overrides = {}
-    if args.impl == "reference":
+    if args.config == "prefix8b":
+        if args.impl == "reference":
+            raise SystemExit("--impl reference times the default layout's workloads")
+        run_prefix(args)
+    elif args.impl == "reference":
         run_reference(args)
     else:
         run_gpu(args)
