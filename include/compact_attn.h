@@ -111,8 +111,9 @@ enum {
  *   the slot of every prefill token; the prefill work list of (block, q_tile)
  *   ordered by descending cost (keys seen by the tile's last row), ties by
  *   ascending block then tile; the deal of the prefill units (item, query head) to
- *   the CTAs of the persistent prefill kernel (kv head by kv head, greedy on the tile
- *   count, see CPA_ARR_PREFILL_SCHED); the decode work list of (block, kv_head, split),
+ *   the CTAs of the persistent prefill kernel (kv head by kv head, in rounds of one unit
+ *   per CTA, the most expensive unit of a round to the least loaded CTA, see
+ *   CPA_ARR_PREFILL_SCHED); the decode work list of (block, kv_head, split),
  *   split s = pages [s*C_b, (s+1)*C_b) of the block, ordered by descending page
  *   count, ties by ascending block, kv head, split.  C_b is cfg->pages_per_split, or
  *   with 0 it is chosen per block so that all items fill one wave of CTAs (three per

@@ -27,8 +27,10 @@ stated in full):
 * prefill schedule the deal of prefill units (item, query head) to the CTAs of a
                   persistent kernel: units listed kv head by kv head, inside a kv
                   head in prefill-item order, the G query heads of the group side by
-                  side; each unit goes to the CTA with the least cost so far (ties:
-                  lower CTA); a unit costs 10 * (its KV tiles of 128 keys) + 18,
+                  side; the list is dealt in rounds of one unit per CTA: CTAs ranked by
+                  cost so far (least first, ties: lower CTA), the round's units by cost
+                  (largest first, ties: list order), i-th unit to i-th CTA; a unit
+                  costs 10 * (its KV tiles of 128 keys) + 18,
                   where an item of 256 query rows whose block has more than 128 rows
                   left streams one tile more than its first 128-row half
 """
@@ -137,22 +139,26 @@ def prefill_schedule(block_lens: Sequence[int], prefill_items, q_tile_rows: int,
                      num_kv_heads: int, num_ctas: int, prefix_lens: Sequence[int] = ()):
     """[rounds][num_ctas] unit codes (item * num_q_heads + head), -1 where a CTA has none."""
     group = num_q_heads // num_kv_heads
-    n_units = len(prefill_items) * num_q_heads
-    ctas = min(num_ctas, n_units)
-    load = [0] * ctas
-    lists = [[] for _ in range(ctas)]
+    units = []                                      # (cost, code) in list order
     for g in range(num_kv_heads):
         for i, (b, t) in enumerate(prefill_items):
             first_row = t * q_tile_rows
             halves = 2 if (q_tile_rows > 128 and int(block_lens[b]) - first_row > 128) else 1
             prefix_tiles = int(prefix_lens[b]) // 128 if len(prefix_lens) else 0
             cost = 10 * (prefix_tiles + first_row // 128 + halves) + 18
-            for h in range(group):
-                c = min(range(ctas), key=lambda x: (load[x], x))
-                lists[c].append(i * num_q_heads + g * group + h)
-                load[c] += cost
-    rounds = max(len(l) for l in lists)
-    return [[lists[c][k] if k < len(lists[c]) else -1 for c in range(ctas)] for k in range(rounds)]
+            units += [(cost, i * num_q_heads + g * group + h) for h in range(group)]
+    ctas = min(num_ctas, len(units))
+    load = [0] * ctas
+    table = []
+    for start in range(0, len(units), ctas):
+        batch = sorted(units[start:start + ctas], key=lambda x: -x[0])      # stable: ties stay in list order
+        ranked = sorted(range(ctas), key=lambda c: (load[c], c))
+        row = [-1] * ctas
+        for (cost, code), c in zip(batch, ranked):
+            row[c] = code
+            load[c] += cost
+        table.append(row)
+    return table
 
 
 def slot_of(plan: Dict[str, list], page_size: int, block: int, pos: int) -> int:

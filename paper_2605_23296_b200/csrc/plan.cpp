@@ -6,7 +6,6 @@
 #include <algorithm>
 #include <cstring>
 #include <new>
-#include <queue>
 #include <utility>
 #include <vector>
 
@@ -58,7 +57,8 @@ int plan_create(const cpa_config* cfg, int32_t num_blocks, const int32_t* block_
         const int32_t pre = p->prefix_lens[b];
         // a cached prefix is read in whole KV tiles of 128 keys (so also in whole pages)
         if (pre < 0 || pre % 128 != 0 || pre > (int64_t)num_shared * P) { delete p; return CPA_EINVAL; }
-        // the device item record packs the q item and the prefix tile count into 16 bits each
+        // the device item record packs the q item and the prefix tile count into 16 bits each (which also
+        // keeps a unit's cost far below the 20 bits the schedule's sort key gives it)
         if (pre / 128 > 0x7FFF || (block_lens[b] + 127) / 128 > 0xFFFF) { delete p; return CPA_EUNSUPPORTED; }
         int64_t cu = (int64_t)p->cu_seqlens[b] + block_lens[b];
         int64_t own = ((int64_t)block_lens[b] + max_new_tokens + P - 1) / P;
@@ -124,39 +124,48 @@ int plan_create(const cpa_config* cfg, int32_t num_blocks, const int32_t* block_
     // Prefill schedule for the persistent kernel (one CTA per SM).  A unit is (item, query head).  Units
     // are listed kv head by kv head, inside a kv head in item order, the G query heads of the group
     // side by side: CTAs that run at the same time then stream the same few K/V ranges, which stay in
-    // L2.  The list is dealt to the CTAs greedily (next unit to the CTA with the least work so far, ties
-    // to the lower CTA), with a unit's cost taken as its KV tile count plus a fixed part, which is what
-    // a hardware scheduler would do with these durations.
+    // L2.  The list is dealt in rounds of one unit per CTA: in every round the CTAs are ranked by the
+    // work they have so far (least first, ties to the lower CTA), the round's units by cost (largest
+    // first, ties in list order), and the i-th unit goes to the i-th CTA.  A unit's cost is its KV
+    // tile count plus a fixed part.
     {
         const int32_t Hq = cfg->num_q_heads, G = Hq / cfg->num_kv_heads;
         const int64_t n_units = (int64_t)p->n_prefill * Hq;
         if (n_units > INT32_MAX / 4) { delete p; return CPA_EUNSUPPORTED; }
         const int32_t ctas = (int32_t)std::min<int64_t>(cfg->num_sms ? cfg->num_sms : 148, n_units);
-        std::vector<std::vector<int32_t>> per_cta((size_t)ctas);
-        typedef std::pair<int64_t, int32_t> Load;   // (work so far, CTA)
-        std::priority_queue<Load, std::vector<Load>, std::greater<Load>> heap;
-        for (int32_t c = 0; c < ctas; ++c) heap.push(Load(0, c));
-        const int32_t sub_per_item = p->q_tile / 128;
-        for (int32_t g = 0; g < cfg->num_kv_heads; ++g)
-            for (int32_t i = 0; i < p->n_prefill; ++i) {
-                const int32_t b = p->prefill_items[2 * i], t = p->prefill_items[2 * i + 1];
-                const int32_t q0 = t * p->q_tile;
-                const int32_t n_sub = (sub_per_item > 1 && block_lens[b] - q0 > 128) ? 2 : 1;
-                const int64_t cost = 10LL * (p->prefix_lens[b] / 128 + q0 / 128 + n_sub) + 18;
-                for (int32_t h = 0; h < G; ++h) {
-                    Load l = heap.top();
-                    heap.pop();
-                    per_cta[(size_t)l.second].push_back(i * Hq + g * G + h);
-                    heap.push(Load(l.first + cost, l.second));
-                }
-            }
-        size_t rounds = 0;
-        for (const auto& v : per_cta) rounds = std::max(rounds, v.size());
+        const int32_t rounds = (int32_t)((n_units + ctas - 1) / ctas);
         p->prefill_ctas = ctas;
-        p->prefill_rounds = (int32_t)rounds;
-        p->prefill_sched.assign(rounds * (size_t)ctas, -1);
-        for (int32_t c = 0; c < ctas; ++c)
-            for (size_t k = 0; k < per_cta[(size_t)c].size(); ++k) p->prefill_sched[k * (size_t)ctas + c] = per_cta[(size_t)c][k];
+        p->prefill_rounds = rounds;
+        p->prefill_sched.assign((size_t)rounds * (size_t)ctas, -1);
+        const int32_t sub_per_item = p->q_tile / 128;
+        std::vector<int32_t> item_cost((size_t)p->n_prefill);
+        for (int32_t i = 0; i < p->n_prefill; ++i) {
+            const int32_t b = p->prefill_items[2 * i], q0 = p->prefill_items[2 * i + 1] * p->q_tile;
+            const int32_t n_sub = (sub_per_item > 1 && block_lens[b] - q0 > 128) ? 2 : 1;
+            item_cost[(size_t)i] = 10 * (p->prefix_lens[b] / 128 + q0 / 128 + n_sub) + 18;
+        }
+        std::vector<int64_t> load((size_t)ctas, 0);
+        std::vector<uint64_t> rank((size_t)ctas), batch((size_t)ctas);   // packed sort keys
+        const int64_t per_head = (int64_t)p->n_prefill * G;            // units of one kv head
+        for (int32_t r = 0; r < rounds; ++r) {
+            const int64_t u0 = (int64_t)r * ctas, n = std::min<int64_t>(ctas, n_units - u0);
+            for (int64_t j = 0; j < n; ++j) {
+                // unit u0 + j of the list -> (kv head, item, head inside the group)
+                const int64_t u = u0 + j, g = u / per_head, rem = u - g * per_head;
+                const int32_t i = (int32_t)(rem / G), h = (int32_t)(rem - (int64_t)i * G);
+                // descending cost, then list order: the position j breaks ties
+                batch[(size_t)j] = ((uint64_t)(0xFFFFFu - (uint32_t)item_cost[(size_t)i]) << 44) | ((uint64_t)j << 32) |
+                                   (uint32_t)(i * Hq + (int32_t)g * G + h);
+            }
+            std::sort(batch.begin(), batch.begin() + n);
+            for (int32_t c = 0; c < ctas; ++c) rank[(size_t)c] = ((uint64_t)load[(size_t)c] << 16) | (uint32_t)c;
+            std::sort(rank.begin(), rank.end());
+            for (int64_t j = 0; j < n; ++j) {
+                const int32_t c = (int32_t)(rank[(size_t)j] & 0xFFFFu);
+                p->prefill_sched[(size_t)r * (size_t)ctas + (size_t)c] = (int32_t)(batch[(size_t)j] & 0xFFFFFFFFu);
+                load[(size_t)c] += 0xFFFFF - (int64_t)(batch[(size_t)j] >> 44);
+            }
+        }
     }
 
     // Decode splits.  Every CTA pays a fixed start-up and merge cost, so the planner aims at
