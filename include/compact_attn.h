@@ -100,7 +100,8 @@ enum {
     CPA_PARAM_DECODE_WORKSPACE_BYTES = 6,/* size of cpa_decode's device workspace */
     CPA_PARAM_TOTAL_SPLITS = 7,          /* split_indptr[B] */
     CPA_PARAM_MAX_NEW_TOKENS = 8,
-    CPA_PARAM_PREFILL_CTAS = 9           /* CTAs of the prefill launch = min(num_sms, prefill units) */
+    CPA_PARAM_PREFILL_CTAS = 9,          /* CTAs of the prefill launch = min(num_sms, prefill units) */
+    CPA_PARAM_SHARED_CHUNK_PAGES = 10    /* pages per chunk of the shared-prefix decode scan; 0 without cached prefixes */
 };
 
 /*

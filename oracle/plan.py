@@ -52,12 +52,14 @@ def partition(history_len: int, block_size: int):
 def build_plan(block_lens: Sequence[int], max_new_tokens: int, page_size: int,
                free_pages: Sequence[int], num_kv_heads: int,
                q_tile_rows: int, pages_per_split, prefix_lens: Sequence[int] = (),
-               shared_pages: Sequence[int] = ()) -> Dict[str, list]:
+               shared_pages: Sequence[int] = (), shared_chunk_pages: int = 0) -> Dict[str, list]:
     """Independent chunks (no prefix_lens), or the prefix-aware layout of Section 4: sequence b
     (worker b) already has the first prefix_lens[b] tokens of the shared history cached in the first
     prefix_lens[b] / P entries of `shared_pages` (same pages for every worker: the prefix cache), and
     block_lens[b] are its own tokens (target block plus markers), stored after the prefix in pages of
-    its own taken from the free list."""
+    its own taken from the free list.  With shared_chunk_pages > 0 the decode of the shared pages is a
+    scan of its own in chunks of that many pages: sequence b gets ceil(prefix pages / chunk) partial
+    slots for it in front of the slots of its splits, and its splits cover its own pages only."""
     B = len(block_lens)
     prefix_lens = [int(x) for x in prefix_lens] if len(prefix_lens) else [0] * B
     if len(prefix_lens) != B or any(x < 0 or x % page_size for x in prefix_lens):
@@ -114,8 +116,12 @@ def build_plan(block_lens: Sequence[int], max_new_tokens: int, page_size: int,
     decode = []
     for b, n in enumerate(pages_per_block):
         c_b = int(pages_per_split[b])
+        prefix_pages = prefix_lens[b] // page_size
+        fixed = -(-prefix_pages // shared_chunk_pages) if shared_chunk_pages else 0
+        if shared_chunk_pages:
+            n -= prefix_pages                     # the splits cover the own pages only
         n_splits = (n + c_b - 1) // c_b
-        split_indptr.append(split_indptr[-1] + n_splits)
+        split_indptr.append(split_indptr[-1] + fixed + n_splits)
         for g in range(num_kv_heads):
             for s in range(n_splits):
                 size = min(c_b, n - s * c_b)

@@ -28,6 +28,7 @@ PARAM_NUM_BLOCKS, PARAM_TOTAL_TOKENS, PARAM_Q_TILE_ROWS, PARAM_PAGES_PER_SPLIT =
 PARAM_PAGES_USED, PARAM_INDEX_BYTES, PARAM_DECODE_WORKSPACE_BYTES, PARAM_TOTAL_SPLITS = 4, 5, 6, 7
 PARAM_MAX_NEW_TOKENS = 8
 PARAM_PREFILL_CTAS = 9
+PARAM_SHARED_CHUNK_PAGES = 10
 
 
 class cpa_config(ctypes.Structure):

@@ -19,7 +19,12 @@ struct cpa_dev_index {
     const int32_t* prefill_items;  // [n_prefill, 4]: (first token of the block, block length, q item | prefix KV tiles << 16,
                                    //   first entry of the sequence in page_indices), 16-byte aligned
     const int32_t* prefill_sched;  // [prefill_rounds, prefill_ctas]: unit (item * Hq + head) of CTA c in round k, -1 = none
-    const int32_t* decode_items;   // [n_decode, item_stride]: (block, kv_head, split, pages, split size, 0, 0, 0) + page ids
+    const int32_t* decode_items;   // [n_decode, item_stride]: (block, kv_head, split, pages, split size, first page of the
+                                   //   split in the sequence's page list, partial slot, slots filled by the shared scan) + page ids
+    const int32_t* prefix_lens;    // [B] cached prefix tokens of each sequence
+    const int32_t* shared_items;   // [n_shared, 4]: (first worker | workers << 16, kv head, chunk, pages) of the shared-prefix scan
+    const int32_t* shared_page_ids;// [longest prefix in pages] pool pages of the shared history
+    int32_t shared_chunk;          // pages per chunk of the shared-prefix scan (0: no shared prefix)
     int32_t* merge_tickets;        // [B * Hkv] arrival counters of the fused split merge (zero between launches)
     int32_t item_stride;           // int32 words per decode item: 8 + largest split size rounded up to 4
 };
@@ -37,11 +42,15 @@ struct cpa_plan {
         prefill_items, prefill_sched, decode_items, split_indptr, split_pages;
     int32_t n_prefill = 0, n_decode = 0;
     int32_t prefill_ctas = 0, prefill_rounds = 0;   // shape of prefill_sched
+    // two-level decode of the prefix-aware layout: partial slots of each sequence that the shared-prefix
+    // scan fills, its chunk size in pages, its work items and the shared pages' ids
+    std::vector<int32_t> n_fixed, shared_items, shared_page_ids;
+    int32_t shared_chunk = 0, n_shared = 0;
 
     // packed image of the device index buffer (int32 words) and offsets into it
     std::vector<int32_t> image;
     int64_t off_status = 0, off_cu = 0, off_pindptr = 0, off_sindptr = 0, off_seqlens = 0,
-            off_append = 0, off_pidx = 0, off_pitems = 0, off_psched = 0, off_ditems = 0, off_tickets = 0, off_seqlens2 = 0,
+            off_append = 0, off_pidx = 0, off_pitems = 0, off_psched = 0, off_prefix = 0, off_shitems = 0, off_shpages = 0, off_ditems = 0, off_tickets = 0, off_seqlens2 = 0,
             words = 0;
     int cur_lens = 0;            // which of the two device length buffers is current
     int32_t item_stride = 0;
@@ -69,6 +78,10 @@ struct cpa_plan {
         d.prefill_items = d_base + off_pitems;
         d.prefill_sched = d_base + off_psched;
         d.decode_items = d_base + off_ditems;
+        d.prefix_lens = d_base + off_prefix;
+        d.shared_items = d_base + off_shitems;
+        d.shared_page_ids = d_base + off_shpages;
+        d.shared_chunk = shared_chunk;
         d.merge_tickets = d_base + off_tickets;
         d.item_stride = item_stride;
         return d;

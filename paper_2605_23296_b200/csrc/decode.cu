@@ -152,7 +152,9 @@ decode_split_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __
     const int len = len_old + (fused ? 1 : 0);
     __syncwarp();
     const int pages_active = (len + P - 1) / P;
-    const int first = s * C;
+    const int first = item[5];           // first page of the split inside the block's page list
+    const int slot = item[6];            // its partial slot among the block's slots
+    const int n_fixed = item[7];         // slots in front that the shared-prefix scan has filled
     const int pg_new = fused ? len_old / P : -1;   // page (inside the block) of the new token
     const bool owner = fused && pg_new >= first && pg_new < first + n_reserved;
     uint4 new_chunk = make_uint4(0, 0, 0, 0);      // lanes 0-15: a 16-byte piece of the K row, 16-31: of the V row
@@ -319,9 +321,10 @@ decode_split_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __
                 sm_o[warp][2 * tig + (e & 1)][8 * (8 * c + gid) + 2 * i + (e >> 1)] = acc[c][i][e];
     __syncthreads();
 
-    const int n_splits = (pages_active + C - 1) / C;  // active splits of this block
+    const int n_own = (pages_active - (first - s * C) + C - 1) / C;  // active splits of this block's own pages
+    const int n_splits = n_fixed + n_own;                            // partials to merge
     const int64_t out_row = (int64_t)b * Hq + g * G;
-    const int64_t prow = (int64_t)(ix.split_indptr[b] + s) * Hq + g * G;
+    const int64_t prow = (int64_t)(ix.split_indptr[b] + slot) * Hq + g * G;
     constexpr int HP = D / 2;  // dim pairs per head
     for (int idx = threadIdx.x; idx < G * HP; idx += kDecodeThreads) {
         const int h = idx / HP, dim = 2 * (idx - h * HP);
@@ -354,7 +357,7 @@ decode_split_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __
     if (threadIdx.x == 0) {
         int* ticket = ix.merge_tickets + b * Hkv + g;
         const int t = atomicAdd(ticket, 1);
-        sm_last = (t == n_splits - 1);
+        sm_last = (t == n_own - 1);
         if (sm_last) *ticket = 0;  // every other split has arrived; ready for the next launch
     }
     __syncthreads();
@@ -379,6 +382,230 @@ decode_split_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __
         *reinterpret_cast<__nv_bfloat162*>(out + (out_row + h) * D + dim) = __floats2bfloat162_rn(o0 * inv, o1 * inv);
     }
     }  // items
+}
+
+// Shared-prefix scan of the prefix-aware layout: one work item = (group of consecutive workers,
+// kv head, chunk of shared history pages).  Every page of the chunk is read ONCE, by a producer
+// warp, into a ring of stages that all four compute warps consume; compute warp w owns rows
+// 16w .. 16w+15 of the group's (worker, query head) rows (row = worker * G + head; up to 64 rows),
+// sixteen rows on the M side of S = Q K^T and two groups of eight on the N side of O^T += V^T P^T.
+// A row sees the keys below its worker's prefix length only (masked by index), so the workers
+// whose prefix ends inside or before the chunk are handled by the same pass.  Each row that sees
+// at least one key of the chunk leaves a partial (max, sum, acc) in slot `chunk` of its worker;
+// the per-worker kernel that follows in the stream merges them with the partials of the worker's
+// own pages.
+constexpr int kSharedThreads = 5 * 32;               // four compute warps + the producer warp
+constexpr int kSharedSmemBytes = 64 * 1024;          // the ring
+
+template <int D>
+__global__ void __launch_bounds__(kSharedThreads, 2)
+decode_shared_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ k_pool,
+                     const __nv_bfloat16* __restrict__ v_pool, float* __restrict__ part_ml,
+                     float* __restrict__ part_o, cpa_dev_index ix, int Hq, int Hkv, int G, float scale_log2) {
+    constexpr int P = 16;
+    constexpr int KC = D / 32;  // 16-byte K chunks per thread per 8-key group
+    constexpr int VC = D / 64;  // 16-byte V chunks per thread per key row
+    constexpr uint32_t kChunkBytes = P * D * 2;
+    constexpr uint32_t kStageBytes = 2 * kChunkBytes;
+    constexpr int STAGES = kSharedSmemBytes / kStageBytes;   // 8 at d=128, 16 at d=64
+    extern __shared__ __align__(128) unsigned char dsm[];
+    __shared__ __align__(8) uint64_t sm_full[STAGES], sm_empty[STAGES];
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int gid = lane >> 2, tig = lane & 3;
+    const uint32_t ring = (uint32_t)__cvta_generic_to_shared(dsm);
+    const uint32_t full0 = (uint32_t)__cvta_generic_to_shared(&sm_full[0]);
+    const uint32_t empty0 = (uint32_t)__cvta_generic_to_shared(&sm_empty[0]);
+    if (threadIdx.x == 0) {
+        for (int st = 0; st < STAGES; ++st) { mbar_init(full0 + 8 * st, 1); mbar_init(empty0 + 8 * st, 4); }
+        asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory");
+    }
+    __syncthreads();
+
+    const int4 hdr = *reinterpret_cast<const int4*>(ix.shared_items + 4 * (int64_t)blockIdx.x);
+    const int w0 = hdr.x & 0xFFFF, nw = hdr.x >> 16, g = hdr.y, chunk = hdr.z, n_pages = hdr.w;
+    const int first = chunk * ix.shared_chunk;      // first history page of the chunk
+    bool gave_up = false;
+
+    if (warp == 4) {
+        // ---------------------------------------------------------------- producer
+        // page ids are fetched 32 at a time by the whole warp; lane 0 issues the copies
+        for (int base = 0; base < n_pages; base += 32) {
+            const int my = base + lane < n_pages ? __ldg(ix.shared_page_ids + first + base + lane) : 0;
+            const int cnt = min(32, n_pages - base);
+            for (int j = 0; j < cnt; ++j) {
+                const int page = __shfl_sync(0xffffffffu, my, j);
+                if (lane == 0) {
+                    const int i = base + j, st = i % STAGES;
+                    const uint32_t parity = (uint32_t)(i / STAGES) & 1u;
+                    if (!gave_up) {
+                        uint32_t spins = 0;
+                        while (!mbar_try_wait(empty0 + 8 * st, parity ^ 1u)) {
+                            if (++spins > kSpinLimit) { gave_up = true; atomicCAS(ix.status, 0, 1); break; }
+                        }
+                    }
+                    const uint32_t dst = ring + st * kStageBytes;
+                    const int64_t src = ((int64_t)page * Hkv + g) * (P * D);
+                    mbar_expect_tx(full0 + 8 * st, kStageBytes);
+                    bulk_load(dst, k_pool + src, kChunkBytes, full0 + 8 * st);
+                    bulk_load(dst + kChunkBytes, v_pool + src, kChunkBytes, full0 + 8 * st);
+                }
+            }
+        }
+        return;
+    }
+
+    // -------------------------------------------------------------------- compute warps
+    // rows of this thread: A = 16*warp + gid, B = A + 8 (row = worker * G + head inside the group)
+    const int n_rows = nw * G;
+    int vis[2], wk[2], hd[2];          // visible prefix length (tokens), worker, head of rows A and B
+    uint4 qa[KC], qb[KC];
+#pragma unroll
+    for (int r = 0; r < 2; ++r) {
+        const int row = 16 * warp + gid + 8 * r;
+        const bool real = row < n_rows;
+        wk[r] = w0 + (real ? row / G : 0);
+        hd[r] = real ? row % G : 0;
+        vis[r] = real ? __ldg(ix.prefix_lens + wk[r]) : 0;
+        const __nv_bfloat16* qrow = q + ((int64_t)wk[r] * Hq + g * G + hd[r]) * D;
+#pragma unroll
+        for (int c = 0; c < KC; ++c) {
+            const uint4 v = real ? *reinterpret_cast<const uint4*>(qrow + (c * 4 + tig) * 8) : make_uint4(0, 0, 0, 0);
+            if (r == 0) qa[c] = v; else qb[c] = v;
+        }
+    }
+    float acc[2][VC][4][4];
+#pragma unroll
+    for (int n = 0; n < 2; ++n)
+#pragma unroll
+        for (int c = 0; c < VC; ++c)
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+#pragma unroll
+                for (int e = 0; e < 4; ++e) acc[n][c][i][e] = 0.f;
+    float m_run[2] = {-INFINITY, -INFINITY};   // running max of raw scores, rows A and B
+    float l_run[2] = {0.f, 0.f};               // this thread's share of the running sums
+
+    for (int i = 0; i < n_pages; ++i) {
+        const int st = i % STAGES;
+        const uint32_t parity = (uint32_t)(i / STAGES) & 1u;
+        if (!gave_up) {
+            uint32_t spins = 0;
+            while (!mbar_try_wait(full0 + 8 * st, parity)) {
+                if (++spins > kSpinLimit) { gave_up = true; atomicCAS(ix.status, 0, 1); break; }
+            }
+        }
+        const uint32_t ks = ring + st * kStageBytes;
+        const uint32_t vs = ks + kChunkBytes;
+        // ---- S = Q K^T: 16 rows x 16 keys
+        float sc[2][4];
+#pragma unroll
+        for (int t = 0; t < 2; ++t) {
+            float sa[4] = {0.f, 0.f, 0.f, 0.f}, sb[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+            for (int c = 0; c < KC; ++c) {
+                const uint4 kr = lds128(ks + (gid + 8 * t) * (D * 2) + cpa_pool_piece(c * 4 + tig, gid) * 16);
+                mma_bf16_16816(sa, qa[c].x, qb[c].x, qa[c].y, qb[c].y, kr.x, kr.y);
+                mma_bf16_16816(sb, qa[c].z, qb[c].z, qa[c].w, qb[c].w, kr.z, kr.w);
+            }
+#pragma unroll
+            for (int e = 0; e < 4; ++e) sc[t][e] = sa[e] + sb[e];
+        }
+        // ---- a row sees the keys below its worker's prefix length; then the online softmax per row
+        const int key0 = (first + i) * P + tig * 2;
+        uint32_t pk[2][2];     // bf16 weights of rows A / B for key groups t = 0 / 1
+        float alpha[2];
+#pragma unroll
+        for (int r = 0; r < 2; ++r) {
+            float s00 = sc[0][2 * r], s01 = sc[0][2 * r + 1], s10 = sc[1][2 * r], s11 = sc[1][2 * r + 1];
+            if (key0 + 9 >= vis[r]) {   // the page reaches beyond this row's prefix
+                if (key0 >= vis[r]) s00 = -INFINITY;
+                if (key0 + 1 >= vis[r]) s01 = -INFINITY;
+                if (key0 + 8 >= vis[r]) s10 = -INFINITY;
+                if (key0 + 9 >= vis[r]) s11 = -INFINITY;
+            }
+            float mx = fmaxf(fmaxf(s00, s01), fmaxf(s10, s11));
+            mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
+            mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
+            const float m_new = fmaxf(m_run[r], mx);                     // -inf while the row has seen no key
+            alpha[r] = (m_run[r] == -INFINITY) ? 0.f : exp2f((m_run[r] - m_new) * scale_log2);
+            const float mb = (m_new == -INFINITY) ? 0.f : m_new * scale_log2;
+            const float p00 = exp2f(fmaf(s00, scale_log2, -mb)), p01 = exp2f(fmaf(s01, scale_log2, -mb));
+            const float p10 = exp2f(fmaf(s10, scale_log2, -mb)), p11 = exp2f(fmaf(s11, scale_log2, -mb));
+            // the row sum is taken over the bf16-rounded weights the MMA will multiply with
+            pk[r][0] = pack_bf16x2(p00, p01);
+            pk[r][1] = pack_bf16x2(p10, p11);
+            l_run[r] = l_run[r] * alpha[r] + (__uint_as_float(pk[r][0] << 16) + __uint_as_float(pk[r][0] & 0xffff0000u)) +
+                       (__uint_as_float(pk[r][1] << 16) + __uint_as_float(pk[r][1] & 0xffff0000u));
+            m_run[r] = m_new;
+        }
+        // accumulator columns are rows 2*tig, 2*tig+1 of each group of eight; their factors live in
+        // the lanes whose gid is that row
+        float a0[2], a1[2];
+#pragma unroll
+        for (int r = 0; r < 2; ++r) {
+            a0[r] = __shfl_sync(0xffffffffu, alpha[r], (2 * tig) * 4);
+            a1[r] = __shfl_sync(0xffffffffu, alpha[r], (2 * tig + 1) * 4);
+        }
+        // ---- O^T += V^T P^T, the V fragments shared by both groups of eight rows
+#pragma unroll
+        for (int c = 0; c < VC; ++c) {
+            uint4 vr[4];
+#pragma unroll
+            for (int r = 0; r < 4; ++r) {
+                const int row = 2 * tig + (r & 1) + 8 * (r >> 1);
+                vr[r] = lds128(vs + row * (D * 2) + cpa_pool_piece(c * 8 + gid, row) * 16);
+            }
+#pragma unroll
+            for (int i2 = 0; i2 < 4; ++i2) {
+                const uint32_t r0 = sel(vr[0], i2), r1 = sel(vr[1], i2);
+                const uint32_t r2 = sel(vr[2], i2), r3 = sel(vr[3], i2);
+                const uint32_t f0 = __byte_perm(r0, r1, 0x5410), f1 = __byte_perm(r0, r1, 0x7632);
+                const uint32_t f2 = __byte_perm(r2, r3, 0x5410), f3 = __byte_perm(r2, r3, 0x7632);
+#pragma unroll
+                for (int n = 0; n < 2; ++n) {
+                    acc[n][c][i2][0] *= a0[n]; acc[n][c][i2][1] *= a1[n]; acc[n][c][i2][2] *= a0[n]; acc[n][c][i2][3] *= a1[n];
+                    mma_bf16_16816(acc[n][c][i2], f0, f1, f2, f3, pk[n][0], pk[n][1]);
+                }
+            }
+        }
+        // this warp is done with the stage
+        __syncwarp();
+        if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];\n" :: "r"(empty0 + 8 * st) : "memory");
+    }
+#pragma unroll
+    for (int r = 0; r < 2; ++r) {
+        l_run[r] += __shfl_xor_sync(0xffffffffu, l_run[r], 1);
+        l_run[r] += __shfl_xor_sync(0xffffffffu, l_run[r], 2);
+    }
+    // ---- partials: slot `chunk` of every worker whose prefix reaches into the chunk
+    if (gave_up) return;
+#pragma unroll
+    for (int r = 0; r < 2; ++r) {
+        const int row = 16 * warp + gid + 8 * r;
+        if (tig == 0 && row < n_rows && vis[r] > first * P) {
+            const int64_t prow = (int64_t)(ix.split_indptr[wk[r]] + chunk) * Hq + g * G + hd[r];
+            *reinterpret_cast<float2*>(part_ml + prow * 2) = make_float2(m_run[r] * scale_log2, l_run[r]);
+        }
+    }
+#pragma unroll
+    for (int n = 0; n < 2; ++n)
+#pragma unroll
+        for (int e01 = 0; e01 < 2; ++e01) {
+            // accumulator column 2*tig + e01 of group n = row 16*warp + 8n + 2*tig + e01
+            const int row = 16 * warp + 8 * n + 2 * tig + e01;
+            if (row >= n_rows) continue;
+            const int wrk = w0 + row / G, h = row % G;
+            if (__ldg(ix.prefix_lens + wrk) <= first * P) continue;
+            float* dst = part_o + ((int64_t)(ix.split_indptr[wrk] + chunk) * Hq + g * G + h) * D;
+#pragma unroll
+            for (int c = 0; c < VC; ++c)
+#pragma unroll
+                for (int i = 0; i < 4; ++i)
+                    *reinterpret_cast<float2*>(dst + 8 * (8 * c + gid) + 2 * i) =
+                        make_float2(acc[n][c][i][e01], acc[n][c][i][e01 + 2]);
+        }
 }
 
 // A block whose cache is still empty has no active split and gets a zero output row.
@@ -408,7 +635,9 @@ int launch_decode(const cpa_plan* plan, const void* q, const void* k_pool, const
     bool& configured = configured_dev[dev_id];
     if (!configured) {
         if (cudaFuncSetAttribute(decode_split_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 kDecodeSmemBytes) != cudaSuccess) {
+                                 kDecodeSmemBytes) != cudaSuccess ||
+            cudaFuncSetAttribute(decode_shared_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 kSharedSmemBytes) != cudaSuccess) {
             (void)cudaGetLastError();
             return CPA_ECUDA;
         }
@@ -416,6 +645,12 @@ int launch_decode(const cpa_plan* plan, const void* q, const void* k_pool, const
     }
     if (any_empty)
         decode_empty_rows_kernel<<<plan->B, 128, 0, st>>>((__nv_bfloat16*)o, ix, plan->B, c.num_q_heads * D);
+    // Prefix-aware layout: the shared history pages are scanned once for all workers; the partials go
+    // to the first slots of every worker and are merged by the launch below, which follows in the stream.
+    if (plan->n_shared > 0)
+        decode_shared_kernel<D><<<plan->n_shared, kSharedThreads, kSharedSmemBytes, st>>>(
+            (const __nv_bfloat16*)q, (const __nv_bfloat16*)k_pool, (const __nv_bfloat16*)v_pool, part_ml, part_o, ix,
+            (int)c.num_q_heads, (int)c.num_kv_heads, G, scale_log2);
     // Programmatic dependent launch: the grid may be scheduled while the previous kernel of the
     // stream drains; the kernel itself waits (griddepcontrol.wait) before it reads anything
     // that kernel wrote.

@@ -173,6 +173,49 @@ int plan_create(const cpa_config* cfg, int32_t num_blocks, const int32_t* block_
     // splitting the block whose splits are largest while the item count (kv heads x splits)
     // still fits.  split_pages[b] is the page count of block b's splits (the last may be
     // shorter).  A fixed pages_per_split from the configuration overrides the search.
+    //
+    // Prefix-aware layout: the cached prefixes are shared pages, and reading them once per worker
+    // would multiply the traffic by about half the worker count.  They are scanned by a kernel of
+    // their own instead: the shared pages are cut into chunks of `shared_chunk` pages, workers are
+    // grouped (as many consecutive workers as give 64 (worker, head) rows per kv head), and one
+    // item = (group, kv head, chunk) computes a partial for every worker of the group whose prefix
+    // reaches into the chunk.  Worker b gets ceil(prefix pages / shared_chunk) partial slots for
+    // them in front of the slots of its own splits, which cover its own pages only.
+    bool two_level = false;
+    int32_t max_pre_pages = 0;
+    for (int32_t b = 0; b < B; ++b) max_pre_pages = std::max(max_pre_pages, p->prefix_lens[b] / P);
+    two_level = max_pre_pages > 0;
+    std::vector<int32_t> dec_pages(pages_per_block);   // pages the per-block splits cover
+    p->n_fixed.assign(B, 0);
+    p->shared_chunk = 0;
+    if (two_level) {
+        const int32_t G = cfg->num_q_heads / cfg->num_kv_heads;
+        const int32_t per_group = 64 / G;                                   // workers per group
+        const int32_t n_groups = (B + per_group - 1) / per_group;
+        const int64_t sms = cfg->num_sms ? cfg->num_sms : 148;
+        const int64_t want = std::max<int64_t>(1, 2 * sms / ((int64_t)cfg->num_kv_heads * n_groups));   // chunks per (group, head)
+        int64_t ch = (max_pre_pages + want - 1) / want;
+        ch = std::max<int64_t>(8, (ch + 7) / 8 * 8);                        // whole 128-key tiles
+        p->shared_chunk = (int32_t)ch;
+        for (int32_t b = 0; b < B; ++b) {
+            dec_pages[b] = pages_per_block[b] - p->prefix_lens[b] / P;
+            p->n_fixed[b] = (p->prefix_lens[b] / P + p->shared_chunk - 1) / p->shared_chunk;
+        }
+        for (int32_t r = 0; r < n_groups; ++r) {
+            const int32_t w0 = r * per_group, nw = std::min(per_group, B - w0);
+            int32_t reach = 0;
+            for (int32_t b = w0; b < w0 + nw; ++b) reach = std::max(reach, p->prefix_lens[b] / P);
+            for (int32_t c = 0; c * p->shared_chunk < reach; ++c)
+                for (int32_t g = 0; g < cfg->num_kv_heads; ++g) {
+                    p->shared_items.push_back(w0 | (nw << 16));
+                    p->shared_items.push_back(g);
+                    p->shared_items.push_back(c);
+                    p->shared_items.push_back(std::min(p->shared_chunk, reach - c * p->shared_chunk));
+                }
+        }
+        p->shared_page_ids.assign(shared_pages, shared_pages + max_pre_pages);
+    }
+    p->n_shared = (int32_t)(p->shared_items.size() / 4);
     p->split_pages.assign(B, 0);
     std::vector<int32_t> n_splits(B, 1);
     if (cfg->pages_per_split > 0) {
@@ -184,7 +227,7 @@ int plan_create(const cpa_config* cfg, int32_t num_blocks, const int32_t* block_
             int32_t best = -1;
             int32_t best_size = 4;  // never split below 4 pages
             for (int32_t b = 0; b < B; ++b) {
-                const int32_t size = (pages_per_block[b] + n_splits[b] - 1) / n_splits[b];
+                const int32_t size = (dec_pages[b] + n_splits[b] - 1) / n_splits[b];
                 if (size > best_size) { best_size = size; best = b; }
             }
             if (best < 0) break;
@@ -192,7 +235,7 @@ int plan_create(const cpa_config* cfg, int32_t num_blocks, const int32_t* block_
             items += cfg->num_kv_heads;
         }
         for (int32_t b = 0; b < B; ++b) {
-            int32_t size = (pages_per_block[b] + n_splits[b] - 1) / n_splits[b];
+            int32_t size = (dec_pages[b] + n_splits[b] - 1) / n_splits[b];
             p->split_pages[b] = std::min(size, kMaxSplitPages);
         }
     }
@@ -202,11 +245,11 @@ int plan_create(const cpa_config* cfg, int32_t num_blocks, const int32_t* block_
     p->split_indptr.assign(B + 1, 0);
     for (int32_t b = 0; b < B; ++b) {
         const int32_t Cb = p->split_pages[b];
-        const int32_t ns = (pages_per_block[b] + Cb - 1) / Cb;
-        p->split_indptr[b + 1] = p->split_indptr[b] + ns;
+        const int32_t ns = (dec_pages[b] + Cb - 1) / Cb;
+        p->split_indptr[b + 1] = p->split_indptr[b] + p->n_fixed[b] + ns;
         for (int32_t g = 0; g < cfg->num_kv_heads; ++g)
             for (int32_t s = 0; s < ns; ++s)
-                dit.push_back({std::min(Cb, pages_per_block[b] - s * Cb), b, g, s});
+                dit.push_back({std::min(Cb, dec_pages[b] - s * Cb), b, g, s});
     }
     std::stable_sort(dit.begin(), dit.end(), [](const DItem& a, const DItem& c) {
         if (a.pages != c.pages) return a.pages > c.pages;
@@ -237,6 +280,9 @@ int plan_create(const cpa_config* cfg, int32_t num_blocks, const int32_t* block_
     p->off_ditems = w;  w = align4(w + (int64_t)p->item_stride * p->n_decode);
     p->off_tickets = w; w = align4(w + (int64_t)B * cfg->num_kv_heads);
     p->off_seqlens2 = w; w = align4(w + B);
+    p->off_prefix = w;  w = align4(w + B);
+    p->off_shitems = w; w = align4(w + (int64_t)p->shared_items.size());
+    p->off_shpages = w; w = align4(w + (int64_t)p->shared_page_ids.size());
     p->words = w;
     p->image.assign((size_t)w, 0);
     int32_t* im = p->image.data();
@@ -256,6 +302,11 @@ int plan_create(const cpa_config* cfg, int32_t num_blocks, const int32_t* block_
     }
     for (int32_t b = 0; b < B; ++b) im[p->off_seqlens + b] = im[p->off_seqlens2 + b] = p->prefix_lens[b];
     std::memcpy(im + p->off_psched, p->prefill_sched.data(), sizeof(int32_t) * p->prefill_sched.size());
+    std::memcpy(im + p->off_prefix, p->prefix_lens.data(), sizeof(int32_t) * B);
+    if (!p->shared_items.empty()) {
+        std::memcpy(im + p->off_shitems, p->shared_items.data(), sizeof(int32_t) * p->shared_items.size());
+        std::memcpy(im + p->off_shpages, p->shared_page_ids.data(), sizeof(int32_t) * p->shared_page_ids.size());
+    }
     for (int32_t i = 0; i < p->n_decode; ++i) {
         // a decode item carries its own page ids, so the kernel's first KV load depends on
         // one prior load only
@@ -265,8 +316,13 @@ int plan_create(const cpa_config* cfg, int32_t num_blocks, const int32_t* block_
         it[2] = dit[i].split;
         it[3] = dit[i].pages;
         it[4] = p->split_pages[dit[i].block];
-        const int32_t* src = p->page_indices.data() + p->page_indptr[dit[i].block] +
-                             dit[i].split * p->split_pages[dit[i].block];
+        // where the split starts inside the sequence's page list (behind the pages the shared scan
+        // covers), its partial slot among the sequence's slots, and how many slots come before
+        const int32_t skip = two_level ? p->prefix_lens[dit[i].block] / P : 0;
+        it[5] = skip + dit[i].split * p->split_pages[dit[i].block];
+        it[6] = p->n_fixed[dit[i].block] + dit[i].split;
+        it[7] = p->n_fixed[dit[i].block];
+        const int32_t* src = p->page_indices.data() + p->page_indptr[dit[i].block] + it[5];
         for (int32_t j = 0; j < dit[i].pages; ++j) it[8 + j] = src[j];
     }
     p->append_stage.assign(B + 1, 0);
@@ -326,6 +382,7 @@ extern "C" int64_t cpa_plan_param(const cpa_plan* plan, int which) {
         case CPA_PARAM_TOTAL_SPLITS: return plan->split_indptr[plan->B];
         case CPA_PARAM_MAX_NEW_TOKENS: return plan->T;
         case CPA_PARAM_PREFILL_CTAS: return plan->prefill_ctas;
+        case CPA_PARAM_SHARED_CHUNK_PAGES: return plan->shared_chunk;
         default: return CPA_EINVAL;
     }
 }

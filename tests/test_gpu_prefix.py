@@ -55,12 +55,15 @@ def run_event(w, pages_per_split=0, q_tile_rows=0, fused_every=2):
     try:
         # page table: bit-exact with the restated rules
         C = s.export(B.ARR_SPLIT_PAGES).tolist()
+        CH = s.param(B.PARAM_SHARED_CHUNK_PAGES)
         ref = op.build_plan(o.block_lens.tolist(), o.decode_steps, o.page_size, o.free_pages.tolist(), o.num_kv_heads,
                             s.param(B.PARAM_Q_TILE_ROWS), C, prefix_lens=w.prefix_lens.tolist(),
-                            shared_pages=w.shared_pages.tolist())
+                            shared_pages=w.shared_pages.tolist(), shared_chunk_pages=CH)
         for which, key in [(B.ARR_PAGE_INDPTR, "page_indptr"), (B.ARR_PAGE_INDICES, "page_indices"),
-                           (B.ARR_SLOT_MAPPING, "slot_mapping"), (B.ARR_SEQ_LENS, "seq_lens")]:
-            assert np.array_equal(s.export(which), np.asarray(ref[key], dtype=np.int32)), key
+                           (B.ARR_SLOT_MAPPING, "slot_mapping"), (B.ARR_SEQ_LENS, "seq_lens"),
+                           (B.ARR_SPLIT_INDPTR, "split_indptr"), (B.ARR_DECODE_ITEMS, "decode_items")]:
+            got = s.export(which)
+            assert np.array_equal(got, np.asarray(ref[key], dtype=np.int32).reshape(got.shape)), key
         # prefill of the own tokens over prefix + own tokens
         k, v = _dev(o.k), _dev(o.v)
         out = s.prefill(_dev(o.q), k, v)
@@ -112,6 +115,26 @@ def test_prefix_aware_both_work_item_sizes(q_tile_rows):
 
 def test_prefix_aware_small_decode_splits():
     run_event(wl.prefix_aware(3, 256, 8, 2, 128, steps=4, seed=23).materialise(), pages_per_split=3)
+
+
+def test_decode_with_two_worker_groups():
+    # G = 8: eight workers fill the 64 rows of a shared-scan item, twelve workers need two groups
+    run_event(wl.prefix_aware(12, 128, 16, 2, 128, steps=3, seed=29).materialise())
+
+
+def test_prefix_ends_inside_a_shared_chunk():
+    # 88-page blocks against 16-page chunks: the prefixes of workers 1 and 3 end in the middle of a chunk,
+    # so the rows of one shared-scan item see different numbers of its keys
+    w = wl.prefix_aware(5, 1408, 8, 8, 64, steps=2, seed=37).materialise()
+    from paper_2605_23296_b200 import binding as B
+    hist, s = _sessions(w)
+    try:
+        ch = s.param(B.PARAM_SHARED_CHUNK_PAGES)
+        assert ch >= 16 and any((int(x) // 16) % ch for x in w.prefix_lens)
+    finally:
+        s.close()
+        hist.close()
+    run_event(w)
 
 
 def test_single_worker_has_no_prefix_and_equals_plain_prefill():

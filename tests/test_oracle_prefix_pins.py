@@ -148,6 +148,12 @@ def test_prefix_plan_matches_hand_worked_fixture():
         assert plan[key] == g[key], key
     assert sum(plan["prefill_items"], []) == g["prefill_items"]
     assert sum(plan["decode_items"], []) == g["decode_items"]
+    two = op.build_plan([3, 2, 3], 1, 4, [8, 1, 5, 0, 9], 1, 2, 2, prefix_lens=[0, 4, 8], shared_pages=[6, 3],
+                        shared_chunk_pages=1)
+    assert two["split_indptr"] == g["two_level_split_indptr"]
+    assert sum(two["decode_items"], []) == g["two_level_decode_items"]
+    for key in ("page_indptr", "page_indices", "seq_lens", "slot_mapping", "prefill_items"):
+        assert two[key] == plan[key], key
 
 
 def test_prefix_plan_invariants():

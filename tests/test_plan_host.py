@@ -190,8 +190,11 @@ def test_prefix_plan_bit_exact(pps):
     try:
         C = B.cpa_plan_export(plan, B.ARR_SPLIT_PAGES).tolist()
         M = B.cpa_plan_param(plan, B.PARAM_Q_TILE_ROWS)
+        CH = B.cpa_plan_param(plan, B.PARAM_SHARED_CHUNK_PAGES)
+        assert CH >= 8 and CH % 8 == 0
         ref = op.build_plan(o.block_lens.tolist(), o.decode_steps, o.page_size, o.free_pages.tolist(), o.num_kv_heads,
-                            M, C, prefix_lens=w.prefix_lens.tolist(), shared_pages=w.shared_pages.tolist())
+                            M, C, prefix_lens=w.prefix_lens.tolist(), shared_pages=w.shared_pages.tolist(),
+                            shared_chunk_pages=CH)
         for which, key in [(B.ARR_CU_SEQLENS, "cu_seqlens"), (B.ARR_PAGE_INDPTR, "page_indptr"),
                            (B.ARR_PAGE_INDICES, "page_indices"), (B.ARR_SEQ_LENS, "seq_lens"),
                            (B.ARR_SLOT_MAPPING, "slot_mapping"), (B.ARR_PREFILL_ITEMS, "prefill_items"),
