@@ -90,6 +90,8 @@ struct cpa_plan {
 
 // largest pages-per-split the planner produces: the decode kernel parks a split's page ids in shared memory
 constexpr int32_t kMaxSplitPages = 1024;
+// largest chunk of the shared-prefix scan (its page ids are parked in shared memory too)
+constexpr int32_t kMaxSharedChunkPages = 1024;
 
 // Pool rows are stored with their 16-byte pieces permuted: piece j of the row in slot r sits at
 // position cpa_pool_piece(j, r) (an involution inside every group of 8 pieces = 128 bytes).  A

@@ -99,7 +99,7 @@ __global__ void __launch_bounds__(kDecodeThreads, 3)
 decode_split_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ k_pool,
                     const __nv_bfloat16* __restrict__ v_pool, float* __restrict__ part_ml,
                     float* __restrict__ part_o, __nv_bfloat16* __restrict__ out, cpa_dev_index ix, int Hq,
-                    int Hkv, int G, float scale_log2, int reverse, cpa_fused_append fa, int n_items) {
+                    int Hkv, int G, float scale_log2, int reverse, cpa_fused_append fa, int n_items, int late_wait) {
     constexpr int P = 16;
     constexpr int KC = D / 32;  // 16-byte K chunks per thread per 8-key group
     constexpr int VC = D / 64;  // 16-byte V chunks per thread per key row
@@ -141,7 +141,9 @@ decode_split_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __
     // Everything above reads plan constants only.  The launch may have started while the
     // previous kernel in the stream (normally the step's append) was still running; from here
     // on its writes (cached length, the new K/V row) are needed, so wait for it to finish.
-    asm volatile("griddepcontrol.wait;\n" ::: "memory");
+    // (When the launch follows the shared-prefix scan of the same step, that earlier kernel is the only
+    // one still running; its partials are needed for the merge only, so the wait moves down there.)
+    if (!late_wait) asm volatile("griddepcontrol.wait;\n" ::: "memory");
     // Fused append: the block's newest token (position len_old) is not in the pool yet.  The
     // CTA whose split holds that position stores the row (for later steps) and patches its own
     // staged copy of the page; every CTA counts the token.  Lengths are double buffered: this
@@ -352,6 +354,7 @@ decode_split_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __
     if (n_splits == 1) continue;
 
     // ---- the last CTA of this (block, kv head) merges the splits
+    if (late_wait) asm volatile("griddepcontrol.wait;\n" ::: "memory");   // the shared scan's partials are complete
     __threadfence();
     __syncthreads();
     if (threadIdx.x == 0) {
@@ -385,20 +388,22 @@ decode_split_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __
 }
 
 // Shared-prefix scan of the prefix-aware layout: one work item = (group of consecutive workers,
-// kv head, chunk of shared history pages).  Every page of the chunk is read ONCE, by a producer
-// warp, into a ring of stages that all four compute warps consume; compute warp w owns rows
-// 16w .. 16w+15 of the group's (worker, query head) rows (row = worker * G + head; up to 64 rows),
-// sixteen rows on the M side of S = Q K^T and two groups of eight on the N side of O^T += V^T P^T.
-// A row sees the keys below its worker's prefix length only (masked by index), so the workers
-// whose prefix ends inside or before the chunk are handled by the same pass.  Each row that sees
-// at least one key of the chunk leaves a partial (max, sum, acc) in slot `chunk` of its worker;
-// the per-worker kernel that follows in the stream merges them with the partials of the worker's
-// own pages.
-constexpr int kSharedThreads = 5 * 32;               // four compute warps + the producer warp
-constexpr int kSharedSmemBytes = 64 * 1024;          // the ring
+// kv head, chunk of shared history pages).  Every page of the chunk is read ONCE into a ring of
+// stages that all four warps consume; warp w owns rows 16w .. 16w+15 of the group's (worker, query
+// head) rows (row = worker * G + head; up to 64 rows), sixteen rows on the M side of S = Q K^T and
+// two groups of eight on the N side of O^T += V^T P^T.  A row sees the keys below its worker's
+// prefix length only (masked by index), so the workers whose prefix ends inside or before the
+// chunk are handled by the same pass, and a warp skips the pages none of its rows sees.  Each row
+// that sees at least one key of the chunk leaves a partial (max, sum, acc) in slot `chunk` of its
+// worker; the per-worker kernel that follows in the stream merges them with the partials of the
+// worker's own pages.  Lane 0 of warp 0 also feeds the ring, two pages behind its own position, so
+// that it rarely has to wait for the other warps to release a stage.
+constexpr int kSharedThreads = 4 * 32;
+constexpr int kSharedSmemBytes = 64 * 1024;          // the ring (three CTAs per SM)
+constexpr int kSharedLag = 2;
 
 template <int D>
-__global__ void __launch_bounds__(kSharedThreads, 2)
+__global__ void __launch_bounds__(kSharedThreads, 3)
 decode_shared_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ k_pool,
                      const __nv_bfloat16* __restrict__ v_pool, float* __restrict__ part_ml,
                      float* __restrict__ part_o, cpa_dev_index ix, int Hq, int Hkv, int G, float scale_log2) {
@@ -410,6 +415,7 @@ decode_shared_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* _
     constexpr int STAGES = kSharedSmemBytes / kStageBytes;   // 8 at d=128, 16 at d=64
     extern __shared__ __align__(128) unsigned char dsm[];
     __shared__ __align__(8) uint64_t sm_full[STAGES], sm_empty[STAGES];
+    __shared__ int sm_ids[kMaxSharedChunkPages];
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int gid = lane >> 2, tig = lane & 3;
@@ -421,40 +427,26 @@ decode_shared_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* _
         asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory");
     }
-    __syncthreads();
-
+    // The per-worker kernel of this step is next in the stream and does not need anything from this one
+    // before its merge: let it start as soon as there is room for its CTAs.
+    asm volatile("griddepcontrol.launch_dependents;\n" ::: "memory");
     const int4 hdr = *reinterpret_cast<const int4*>(ix.shared_items + 4 * (int64_t)blockIdx.x);
     const int w0 = hdr.x & 0xFFFF, nw = hdr.x >> 16, g = hdr.y, chunk = hdr.z, n_pages = hdr.w;
     const int first = chunk * ix.shared_chunk;      // first history page of the chunk
+    for (int i = threadIdx.x; i < n_pages; i += kSharedThreads) sm_ids[i] = __ldg(ix.shared_page_ids + first + i);
+    __syncthreads();
     bool gave_up = false;
 
-    if (warp == 4) {
-        // ---------------------------------------------------------------- producer
-        // page ids are fetched 32 at a time by the whole warp; lane 0 issues the copies
-        for (int base = 0; base < n_pages; base += 32) {
-            const int my = base + lane < n_pages ? __ldg(ix.shared_page_ids + first + base + lane) : 0;
-            const int cnt = min(32, n_pages - base);
-            for (int j = 0; j < cnt; ++j) {
-                const int page = __shfl_sync(0xffffffffu, my, j);
-                if (lane == 0) {
-                    const int i = base + j, st = i % STAGES;
-                    const uint32_t parity = (uint32_t)(i / STAGES) & 1u;
-                    if (!gave_up) {
-                        uint32_t spins = 0;
-                        while (!mbar_try_wait(empty0 + 8 * st, parity ^ 1u)) {
-                            if (++spins > kSpinLimit) { gave_up = true; atomicCAS(ix.status, 0, 1); break; }
-                        }
-                    }
-                    const uint32_t dst = ring + st * kStageBytes;
-                    const int64_t src = ((int64_t)page * Hkv + g) * (P * D);
-                    mbar_expect_tx(full0 + 8 * st, kStageBytes);
-                    bulk_load(dst, k_pool + src, kChunkBytes, full0 + 8 * st);
-                    bulk_load(dst + kChunkBytes, v_pool + src, kChunkBytes, full0 + 8 * st);
-                }
-            }
-        }
-        return;
-    }
+    auto issue = [&](int i) {   // lane 0 of warp 0: page i of the chunk into its stage
+        const int st = i % STAGES;
+        const uint32_t dst = ring + st * kStageBytes;
+        const int64_t src = ((int64_t)sm_ids[i] * Hkv + g) * (P * D);
+        mbar_expect_tx(full0 + 8 * st, kStageBytes);
+        bulk_load(dst, k_pool + src, kChunkBytes, full0 + 8 * st);
+        bulk_load(dst + kChunkBytes, v_pool + src, kChunkBytes, full0 + 8 * st);
+    };
+    if (threadIdx.x == 0)
+        for (int i = 0; i < STAGES && i < n_pages; ++i) issue(i);
 
     // -------------------------------------------------------------------- compute warps
     // rows of this thread: A = 16*warp + gid, B = A + 8 (row = worker * G + head inside the group)
@@ -486,15 +478,39 @@ decode_shared_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* _
                 for (int e = 0; e < 4; ++e) acc[n][c][i][e] = 0.f;
     float m_run[2] = {-INFINITY, -INFINITY};   // running max of raw scores, rows A and B
     float l_run[2] = {0.f, 0.f};               // this thread's share of the running sums
+    int vis_warp = max(vis[0], vis[1]);        // no row of this warp sees keys from here on
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) vis_warp = max(vis_warp, __shfl_xor_sync(0xffffffffu, vis_warp, o));
 
     for (int i = 0; i < n_pages; ++i) {
         const int st = i % STAGES;
         const uint32_t parity = (uint32_t)(i / STAGES) & 1u;
+        if (threadIdx.x == 0) {
+            // refill: page j takes the stage of page j - STAGES, which every warp must have released
+            const int j = i + STAGES - kSharedLag;
+            if (j >= STAGES && j < n_pages) {
+                if (!gave_up) {
+                    uint32_t spins = 0;
+                    while (!mbar_try_wait(empty0 + 8 * (j % STAGES), ((uint32_t)(j / STAGES) & 1u) ^ 1u)) {
+                        if (++spins > kSpinLimit) { gave_up = true; atomicCAS(ix.status, 0, 1); break; }
+                    }
+                }
+                if (!gave_up) issue(j);
+            }
+        }
+        gave_up = __shfl_sync(0xffffffffu, gave_up, 0) || gave_up;
         if (!gave_up) {
             uint32_t spins = 0;
             while (!mbar_try_wait(full0 + 8 * st, parity)) {
                 if (++spins > kSpinLimit) { gave_up = true; atomicCAS(ix.status, 0, 1); break; }
             }
+        }
+        if ((first + i) * P >= vis_warp) {
+            // Nothing on this page for this warp's rows.  It still waits for the page before it releases
+            // the stage: a warp that ran ahead would add its releases of later pages to the current
+            // phase of the stage's barrier.
+            if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];\n" :: "r"(empty0 + 8 * st) : "memory");
+            continue;
         }
         const uint32_t ks = ring + st * kStageBytes;
         const uint32_t vs = ks + kChunkBytes;
@@ -668,7 +684,8 @@ int launch_decode(const cpa_plan* plan, const void* q, const void* k_pool, const
     cudaError_t e = cudaLaunchKernelEx(&cfg, decode_split_kernel<D>, (const __nv_bfloat16*)q,
                                        (const __nv_bfloat16*)k_pool, (const __nv_bfloat16*)v_pool, part_ml, part_o,
                                        (__nv_bfloat16*)o, ix, (int)c.num_q_heads, (int)c.num_kv_heads, G, scale_log2,
-                                       (int)(plan->decode_calls++ & 1), fa, (int)plan->n_decode);
+                                       (int)(plan->decode_calls++ & 1), fa, (int)plan->n_decode,
+                                       (int)(plan->n_shared > 0));
     if (e != cudaSuccess) { (void)cudaGetLastError(); return CPA_ECUDA; }
     return cudaGetLastError() == cudaSuccess ? CPA_OK : CPA_ECUDA;
 }

@@ -193,9 +193,9 @@ int plan_create(const cpa_config* cfg, int32_t num_blocks, const int32_t* block_
         const int32_t per_group = 64 / G;                                   // workers per group
         const int32_t n_groups = (B + per_group - 1) / per_group;
         const int64_t sms = cfg->num_sms ? cfg->num_sms : 148;
-        const int64_t want = std::max<int64_t>(1, 2 * sms / ((int64_t)cfg->num_kv_heads * n_groups));   // chunks per (group, head)
+        const int64_t want = std::max<int64_t>(1, 3 * sms / ((int64_t)cfg->num_kv_heads * n_groups));   // chunks per (group, head)
         int64_t ch = (max_pre_pages + want - 1) / want;
-        ch = std::max<int64_t>(8, (ch + 7) / 8 * 8);                        // whole 128-key tiles
+        ch = std::min<int64_t>(kMaxSharedChunkPages, std::max<int64_t>(8, (ch + 7) / 8 * 8));   // whole 128-key tiles
         p->shared_chunk = (int32_t)ch;
         for (int32_t b = 0; b < B; ++b) {
             dec_pages[b] = pages_per_block[b] - p->prefix_lens[b] / P;

@@ -123,9 +123,10 @@ def test_decode_with_two_worker_groups():
 
 
 def test_prefix_ends_inside_a_shared_chunk():
-    # 88-page blocks against 16-page chunks: the prefixes of workers 1 and 3 end in the middle of a chunk,
-    # so the rows of one shared-scan item see different numbers of its keys
-    w = wl.prefix_aware(5, 1408, 8, 8, 64, steps=2, seed=37).materialise()
+    # 136-page blocks against 16-page chunks (more pages than the scan's ring has stages): the prefixes of
+    # workers 1 and 3 end in the middle of a chunk, so the rows of one shared-scan item see different
+    # numbers of its keys, and the ring of stages is refilled while the warps are at different pages
+    w = wl.prefix_aware(5, 2176, 8, 8, 64, steps=2, seed=37).materialise()
     from paper_2605_23296_b200 import binding as B
     hist, s = _sessions(w)
     try:
@@ -135,6 +136,27 @@ def test_prefix_ends_inside_a_shared_chunk():
         s.close()
         hist.close()
     run_event(w)
+
+
+def test_decode_long_shared_chunks_sampled_steps():
+    # 8 workers x 4096-token blocks, d = 128: chunks of 40 pages against a ring of 8 stages
+    w = wl.prefix_aware(8, 4096, 32, 8, 128, steps=3, seed=43).materialise()
+    o = w.own
+    cu = _cu(o)
+    hist, s = _sessions(w, poison=False)
+    try:
+        from paper_2605_23296_b200 import binding as B
+        assert s.param(B.PARAM_SHARED_CHUNK_PAGES) > 8
+        s.append_prefill(_dev(o.k), _dev(o.v))
+        st = oa.PrefixDecodeState(o.k, o.v, cu, w.k_hist, w.v_hist, w.prefix_lens, o.decode_steps)
+        for t in range(o.decode_steps):
+            st.append(o.k_dec[t], o.v_dec[t])
+            got = s.decode_append(_dev(o.q_dec[t]), _dev(o.k_dec[t]), _dev(o.v_dec[t]))
+            assert_attention_close(_bits(got), st.decode(o.q_dec[t], o.scale), f"long shared chunks, step {t}")
+        assert s.status() == 0
+    finally:
+        s.close()
+        hist.close()
 
 
 def test_single_worker_has_no_prefix_and_equals_plain_prefill():
