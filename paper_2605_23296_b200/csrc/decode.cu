@@ -556,13 +556,21 @@ decode_shared_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* _
                        (__uint_as_float(pk[r][1] << 16) + __uint_as_float(pk[r][1] & 0xffff0000u));
             m_run[r] = m_new;
         }
-        // accumulator columns are rows 2*tig, 2*tig+1 of each group of eight; their factors live in
-        // the lanes whose gid is that row
-        float a0[2], a1[2];
+        // Rescale the accumulators only when some row's max moved (after the first pages it rarely
+        // does).  Accumulator columns are rows 2*tig, 2*tig+1 of each group of eight; their factors
+        // live in the lanes whose gid is that row.
+        if (__any_sync(0xffffffffu, alpha[0] != 1.f || alpha[1] != 1.f)) {
 #pragma unroll
-        for (int r = 0; r < 2; ++r) {
-            a0[r] = __shfl_sync(0xffffffffu, alpha[r], (2 * tig) * 4);
-            a1[r] = __shfl_sync(0xffffffffu, alpha[r], (2 * tig + 1) * 4);
+            for (int n = 0; n < 2; ++n) {
+                const float a0 = __shfl_sync(0xffffffffu, alpha[n], (2 * tig) * 4);
+                const float a1 = __shfl_sync(0xffffffffu, alpha[n], (2 * tig + 1) * 4);
+#pragma unroll
+                for (int c = 0; c < VC; ++c)
+#pragma unroll
+                    for (int i2 = 0; i2 < 4; ++i2) {
+                        acc[n][c][i2][0] *= a0; acc[n][c][i2][1] *= a1; acc[n][c][i2][2] *= a0; acc[n][c][i2][3] *= a1;
+                    }
+            }
         }
         // ---- O^T += V^T P^T, the V fragments shared by both groups of eight rows
 #pragma unroll
@@ -580,10 +588,7 @@ decode_shared_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* _
                 const uint32_t f0 = __byte_perm(r0, r1, 0x5410), f1 = __byte_perm(r0, r1, 0x7632);
                 const uint32_t f2 = __byte_perm(r2, r3, 0x5410), f3 = __byte_perm(r2, r3, 0x7632);
 #pragma unroll
-                for (int n = 0; n < 2; ++n) {
-                    acc[n][c][i2][0] *= a0[n]; acc[n][c][i2][1] *= a1[n]; acc[n][c][i2][2] *= a0[n]; acc[n][c][i2][3] *= a1[n];
-                    mma_bf16_16816(acc[n][c][i2], f0, f1, f2, f3, pk[n][0], pk[n][1]);
-                }
+                for (int n = 0; n < 2; ++n) mma_bf16_16816(acc[n][c][i2], f0, f1, f2, f3, pk[n][0], pk[n][1]);
             }
         }
         // this warp is done with the stage
