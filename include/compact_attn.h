@@ -147,8 +147,12 @@ CPA_API int cpa_plan_create(const cpa_config* cfg, int32_t num_blocks, const int
  *                    no call through this plan ever writes them
  * Worker w's page list is shared_pages[0 .. prefix_lens[w]/16) followed by
  * ceil((own_lens[w] + max_new_tokens) / 16) pages of its own from `free_pages`; its cached
- * length (seq_lens) starts at prefix_lens[w]; positions, slots and the decode splits count from
- * the start of the prompt; the cost of a prefill item includes the prefix.  Everything else is
+ * length (seq_lens) starts at prefix_lens[w]; positions and slots count from the start of the
+ * prompt; the cost of a prefill item includes the prefix.  Decode runs in two levels: the shared
+ * pages are scanned once for all workers in chunks of CPA_PARAM_SHARED_CHUNK_PAGES pages (a kernel
+ * of its own inside cpa_decode / cpa_decode_append), worker w has
+ * ceil(prefix pages / chunk) partial slots for that scan in front of the slots of its splits, and
+ * its splits (CPA_ARR_DECODE_ITEMS, CPA_ARR_SPLIT_PAGES) cover its own pages only.  Everything else is
  * as for cpa_plan_create, which is the case prefix_lens == 0.  Errors as for cpa_plan_create,
  * plus CPA_EINVAL for a prefix that is negative, not a multiple of 128, or longer than
  * 16 * num_shared.
