@@ -194,3 +194,47 @@ def test_long_prefix_sampled_rows():
     finally:
         s.close()
         hist.close()
+
+
+def test_entry_points_and_layouts_do_not_mix():
+    from paper_2605_23296_b200 import binding as B
+    from paper_2605_23296_b200.session import CompactionSession
+    w = wl.prefix_aware(2, 128, 4, 2, 64, steps=1, seed=3).materialise()
+    o = w.own
+    hist, s = _sessions(w)
+    plain = CompactionSession(o.block_lens, 1, o.num_q_heads, o.num_kv_heads, o.head_dim, o.free_pages, w.num_pages,
+                              scale=o.scale, pools=(s.k_pool, s.v_pool))
+    try:
+        q, k, v = _dev(o.q), _dev(o.k), _dev(o.v)
+        out = _dev(np.zeros_like(o.q))
+        # a plan with cached prefixes needs the pools: the plain prefill calls refuse it
+        assert B.cpa_prefill(s.plan, q, k, v, out, None, 0) == B.CPA_EINVAL
+        assert B.cpa_prefill_variant(s.plan, q, k, v, out, 0, 1) == B.CPA_EINVAL
+        assert B.cpa_prefill_prefix(s.plan, q, k, v, None, s.v_pool, out, 0) == B.CPA_EINVAL
+        # a plan without prefixes through the prefix entry point reads nothing from the pools
+        a = plain.prefill(q, k, v)
+        b = _dev(np.zeros_like(o.q))
+        assert B.cpa_prefill_prefix(plain.plan, q, k, v, plain.k_pool, plain.v_pool, b, plain._stream()) == B.CPA_OK
+        assert plain.status() == 0
+        assert np.array_equal(_bits(a), _bits(b))
+        assert plain.param(B.PARAM_SHARED_CHUNK_PAGES) == 0 and s.param(B.PARAM_SHARED_CHUNK_PAGES) >= 8
+    finally:
+        s.close()
+        plain.close()
+        hist.close()
+
+
+def test_prefill_only_event_and_single_token_workers():
+    # T = 0 (no decode), and workers whose own part is a single token behind a long prefix
+    w = wl.prefix_aware(3, 256, 8, 2, 128, steps=0, seed=13, own_len=1).materialise(with_decode=False)
+    o = w.own
+    cu = _cu(o)
+    hist, s = _sessions(w)
+    try:
+        out = s.prefill(_dev(o.q), _dev(o.k), _dev(o.v))
+        want = oa.prefill_prefix_aware(o.q, o.k, o.v, cu, w.k_hist, w.v_hist, w.prefix_lens, o.scale)
+        assert s.status() == 0
+        assert_attention_close(_bits(out), want, "single own token behind a prefix")
+    finally:
+        s.close()
+        hist.close()

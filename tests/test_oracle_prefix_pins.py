@@ -174,3 +174,54 @@ def test_prefix_plan_invariants():
     # own tokens never land in a shared page
     assert not {s // P for s in plan["slot_mapping"]} & set(w.shared_pages.tolist())
     assert plan["seq_lens"] == w.prefix_lens.tolist()
+
+
+# ----------------------------------------------------------------------------
+# the pins above can fail: plausible mistakes planted in copies of the oracle function (CPU only)
+# ----------------------------------------------------------------------------
+
+def _mutant(kind):
+    """A copy of oracle.attention.prefill_prefix_aware's steps with one planted mistake."""
+    def fn(q, k, v, cu_seqlens, k_hist, v_hist, prefix_lens, scale, rows=None):
+        cu = [int(x) for x in cu_seqlens]
+        out = np.empty(q.shape, dtype=np.float64)
+        for w in range(len(cu) - 1):
+            n_pre, lo, hi = int(prefix_lens[w]), cu[w], cu[w + 1]
+            kh, vh = k_hist[:n_pre], v_hist[:n_pre]
+            if kind == "prefix_from_the_end":          # the last n_pre history tokens instead of the first
+                kh, vh = k_hist[k_hist.shape[0] - n_pre:], v_hist[v_hist.shape[0] - n_pre:]
+            if kind == "prefix_one_short" and n_pre:   # drops the last visible history token
+                kh, vh = kh[:-1], vh[:-1]
+            if kind == "prefix_of_previous_worker":    # worker w reads worker w-1's prefix
+                n_prev = int(prefix_lens[w - 1]) if w else 0
+                kh, vh = k_hist[:n_prev], v_hist[:n_prev]
+            if kind == "values_not_prefixed":          # keys see the prefix, values are shifted
+                vh = np.roll(vh, 1, axis=0)
+            m = kh.shape[0]
+            pk, pv = np.concatenate([kh, k[lo:hi]]), np.concatenate([vh, v[lo:hi]])
+            pq = np.concatenate([np.zeros((m,) + q.shape[1:], dtype=np.uint16), q[lo:hi]])
+            first = m - 1 if kind == "rows_not_offset" and m else m    # the own rows start one row early
+            out[lo:hi] = oa.prefill(pq, pk, pv, [0, m + hi - lo], scale, rows=list(range(first, first + hi - lo)))
+        return out
+    return fn
+
+
+def _prefix_pins_hold(fn) -> bool:
+    w = small(seed=5, workers=3, block_len=128, hq=4, hkv=2, d=64)
+    o, cu = w.own, cu_of(w)
+    got = fn(o.q, o.k, o.v, cu, w.k_hist, w.v_hist, w.prefix_lens, o.scale)
+    for b in range(o.num_blocks):
+        n_pre = int(w.prefix_lens[b])
+        want = brute_force_worker(o.q[cu[b]:cu[b + 1]], o.k[cu[b]:cu[b + 1]], o.v[cu[b]:cu[b + 1]],
+                                  w.k_hist[:n_pre], w.v_hist[:n_pre], o.scale)
+        if not np.allclose(got[cu[b]:cu[b + 1]], want, rtol=1e-11, atol=1e-13):
+            return False
+    return True
+
+
+def test_prefix_pins_reject_planted_mistakes():
+    assert _prefix_pins_hold(oa.prefill_prefix_aware)
+    for kind in ("prefix_from_the_end", "prefix_one_short", "prefix_of_previous_worker", "values_not_prefixed",
+                 "rows_not_offset"):
+        assert not _prefix_pins_hold(_mutant(kind)), kind
+    assert _prefix_pins_hold(_mutant("none"))     # the copy without a mistake passes, so the copies are faithful
