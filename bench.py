@@ -528,13 +528,121 @@ def run_prefix(args) -> None:
     }))
 
 
+# ------------------------------------------------------------------------------------------
+# compaction in the background of a decoding agent (paper, Section 7: asynchronous compaction)
+# ------------------------------------------------------------------------------------------
+
+def run_async(args) -> None:
+    """`--config async`: a foreground sequence keeps decoding over a 100k-token cache on a high-priority
+    stream while compaction events (the dense8b workload) run on a low-priority stream with an SM
+    budget.  Reports the foreground's step times and the event's time, alone and together."""
+    import torch
+
+    from paper_2605_23296_b200.session import CompactionSession, bits_to_tensor
+
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    sms = torch.cuda.get_device_properties(dev).multi_processor_count
+    fg_stream = torch.cuda.Stream(dev, priority=-1)
+    bg_stream = torch.cuda.Stream(dev, priority=0)
+    rng = np.random.default_rng(5)
+    Hq, Hkv, d, ctx, steps = 32, 8, 128, 100_000, args.decode_steps or 200
+    bits = lambda shape: wl.f32_to_bf16_bits(rng.standard_normal(shape, dtype=np.float32))
+    to = lambda b: bits_to_tensor(b, dev)
+    pages = (ctx + steps + 15) // 16 + 1
+    with torch.cuda.stream(fg_stream):
+        fg = CompactionSession([ctx], steps, Hq, Hkv, d, np.arange(pages, dtype=np.int32), pages)
+        hk, hv = to(bits((ctx, Hkv, d))), to(bits((ctx, Hkv, d)))
+        fq, fk, fv = to(bits((steps, 1, Hq, d))), to(bits((steps, 1, Hkv, d))), to(bits((steps, 1, Hkv, d)))
+        fo = torch.empty_like(fq)
+    w = make_workload("dense8b").materialise()
+    bq, bk, bv, bqd, bkd, bvd = (to(x) for x in (w.q, w.k, w.v, w.q_dec, w.k_dec, w.v_dec))
+    bo = torch.empty_like(bq)
+    bod = torch.empty((w.decode_steps, w.num_blocks, Hq, d), dtype=torch.bfloat16, device=dev)
+    torch.cuda.synchronize(dev)
+
+    def background(budget):
+        with torch.cuda.stream(bg_stream):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(bg_stream)
+            s = CompactionSession(w.block_lens, w.decode_steps, Hq, Hkv, d, w.free_pages, w.num_pages, scale=w.scale,
+                                  num_sms=budget)
+            s.prefill(bq, bk, bv, out=bo)
+            s.append_prefill(bk, bv)
+            for t in range(w.decode_steps):
+                s.decode_append(bqd[t], bkd[t], bvd[t], out=bod[t])
+            e1.record(bg_stream)
+        return s, e0, e1
+
+    def rewind():
+        # the foreground's cache goes back to the bare context (plan uploaded again, the context appended
+        # again), so that every measurement decodes the same steps over the same lengths
+        with torch.cuda.stream(fg_stream):
+            from paper_2605_23296_b200 import binding as B
+            fg._check(B.cpa_plan_upload(fg.plan, fg.index_buf, fg.index_buf.numel(), fg._stream()), "cpa_plan_upload")
+            fg.append_prefill(hk, hv)
+        fg_stream.synchronize()
+
+    def foreground(t0, t1):
+        evs = []
+        with torch.cuda.stream(fg_stream):
+            for t in range(t0, t1):
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record(fg_stream)
+                fg.decode_append(fq[t], fk[t], fv[t], out=fo[t])
+                e1.record(fg_stream)
+                evs.append((e0, e1))
+        return evs
+
+    def stats(evs):
+        ms = np.array([a.elapsed_time(b) for a, b in evs]) * 1e3
+        return {"p50_us": float(np.percentile(ms, 50)), "p95_us": float(np.percentile(ms, 95)), "max_us": float(ms.max())}
+
+    results = []
+    quarter = steps // 4
+    for _ in range(2):   # warm-up of both paths
+        rewind()
+        s, _, _ = background(sms)
+        foreground(0, steps)
+        torch.cuda.synchronize(dev)
+        s.close()
+    rewind()
+    evs = foreground(0, steps)
+    torch.cuda.synchronize(dev)
+    alone_fg = stats(evs)
+    for budget in [sms, (3 * sms) // 4, sms // 2, sms // 4]:
+        s, e0, e1 = background(budget)
+        torch.cuda.synchronize(dev)
+        alone_bg = e0.elapsed_time(e1)
+        s.close()
+        # four events in a row, a quarter of the foreground's steps enqueued behind each, so that both
+        # streams have work for the whole measurement
+        rewind()
+        evs, bgs = [], []
+        for i in range(4):
+            bgs.append(background(budget))
+            evs += foreground(i * quarter, (i + 1) * quarter)
+        torch.cuda.synchronize(dev)
+        assert all(x[0].status() == 0 for x in bgs) and fg.status() == 0
+        results.append({"sm_budget": budget, "event_ms_alone": alone_bg,
+                        "event_ms_shared": float(np.mean([x[1].elapsed_time(x[2]) for x in bgs])),
+                        "foreground_shared": stats(evs)})
+        for x in bgs:
+            x[0].close()
+    print(json.dumps({"metric": "foreground decode step time next to a background compaction event", "unit": "us",
+                      "config": {"workload": "async", "foreground": f"1 sequence, {ctx}-token cache, {steps} steps, 32/8/128",
+                                 "background": "dense8b event (8 x 4096, T=256) on a low-priority stream", "sms": sms},
+                      "foreground_alone": alone_fg, "budgets": results}))
+    fg.close()
+
+
 def main() -> None:
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--config", default="dense8b", choices=sorted(wl.CONFIGS) + ["prefix8b"])
+    ap.add_argument("--config", default="dense8b", choices=sorted(wl.CONFIGS) + ["prefix8b", "async"])
     ap.add_argument("--blocks", type=int, default=0, help="override the number of blocks (profiling)")
     ap.add_argument("--block-len", type=int, default=0, help="override the block length (profiling)")
     ap.add_argument("--decode-steps", type=int, default=0, help="override the decode steps (profiling)")
@@ -549,10 +657,10 @@ def main() -> None:
         ap.error("--block-len does not apply to this configuration")
     if args.config == "tiny":
         args.overrides = {}
-    if args.config == "prefix8b":
+    if args.config in ("prefix8b", "async"):
         if args.impl == "reference":
             raise SystemExit("--impl reference times the default layout's workloads")
-        run_prefix(args)
+        run_prefix(args) if args.config == "prefix8b" else run_async(args)
     elif args.impl == "reference":
         run_reference(args)
     else:

@@ -69,7 +69,10 @@ typedef struct cpa_config {
     float   scale;           /* softmax scale, normally 1/sqrt(head_dim) */
     int32_t q_tile_rows;     /* query rows per prefill work item: 128 or 256; 0 = default (256) */
     int32_t pages_per_split; /* KV pages per decode work item (<= 1024); 0 = chosen per block from the batch */
-    int32_t num_sms;         /* SM count the split heuristic aims at; 0 = 148 */
+    int32_t num_sms;         /* SMs this plan's kernels may fill: the persistent prefill launches min(num_sms, units)
+                                CTAs (one per SM) and the decode wave is sized for 3 * num_sms CTAs; 0 = 148.  A
+                                value below the device's SM count leaves SMs to other streams (a CTA of the
+                                prefill keeps its SM for the whole launch, stream priority does not preempt it) */
 } cpa_config;
 
 typedef struct cpa_plan cpa_plan; /* opaque; host memory owned by the library */

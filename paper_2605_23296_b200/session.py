@@ -39,15 +39,17 @@ class CompactionSession:
                  scale: Optional[float] = None, device: str = "cuda:0", pages_per_split: int = 0,
                  poison_pools: bool = False, page_size: int = 16, q_tile_rows: int = 0,
                  prefix_lens: Optional[Sequence[int]] = None, shared_pages: Optional[Sequence[int]] = None,
-                 pools=None):
+                 pools=None, num_sms: int = 0):
         self.device = torch.device(device)
         self.Hq, self.Hkv, self.d, self.P = num_q_heads, num_kv_heads, head_dim, page_size
         self.B = len(block_lens)
         self.block_lens = np.asarray(block_lens, dtype=np.int32)
         self.scale = float(scale if scale is not None else head_dim ** -0.5)
         props = torch.cuda.get_device_properties(self.device)
+        # num_sms is the SM budget of this event: the persistent prefill grid and the decode wave are sized
+        # from it (all SMs unless the caller wants to leave room for other work on the device)
         self.cfg = B.cpa_config(num_q_heads, num_kv_heads, head_dim, page_size, self.scale, q_tile_rows,
-                                pages_per_split, props.multi_processor_count)
+                                pages_per_split, num_sms or props.multi_processor_count)
         self.prefix_aware = prefix_lens is not None
         if self.prefix_aware:   # the paper's layout: cached history prefix + own tokens per worker
             self.plan = B.cpa_plan_create_prefix(self.cfg, self.block_lens, prefix_lens, shared_pages,
