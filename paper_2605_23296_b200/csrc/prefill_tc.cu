@@ -7,8 +7,9 @@
 // walking its share of the units).  Twelve warps with fixed roles:
 //   warps 0-3  softmax + epilogue of sub-tile 0: thread r owns query row r (TMEM lane r), so
 //   warps 4-7  ... of sub-tile 1                 row max and row sum need no shuffles
-//   warp 8     TMA producer (one elected lane): both Q sub-tiles once, then K and V tiles of
-//              128 keys through rings of two (head_dim 128) or four (head_dim 64) stages
+//   warp 8     TMA producer (one elected lane; eight lanes for tiles of a cached prefix, which are
+//              gathered from pool pages): both Q sub-tiles of a unit, then K and V tiles of 128
+//              keys through rings of two (head_dim 128) or four (head_dim 64) stages
 //   warp 9     MMA issuer (one elected lane) and owner of the TMEM allocation
 //   warps 10-11 idle; they complete the third warpgroup so that its registers can be handed
 //              to the softmax warpgroups (setmaxnreg works on whole warpgroups)
