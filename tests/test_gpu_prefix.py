@@ -238,3 +238,26 @@ def test_prefill_only_event_and_single_token_workers():
     finally:
         s.close()
         hist.close()
+
+
+def test_decode_entry_points_agree_on_a_prefix_plan():
+    # separate append + cpa_decode, the fused step and the static-scratch variant over shared prefix pages
+    import torch
+    from paper_2605_23296_b200 import binding as B
+    w = wl.prefix_aware(4, 256, 8, 2, 128, steps=2, seed=19).materialise()
+    o = w.own
+    hist, s = _sessions(w)
+    try:
+        s.append_prefill(_dev(o.k), _dev(o.v))
+        s.append(_dev(o.k_dec[0]), _dev(o.v_dec[0]))
+        q = _dev(o.q_dec[0])
+        want = s.decode(q)
+        again = s.decode(q)
+        assert np.array_equal(_bits(want), _bits(again))          # the merge tickets reset themselves
+        got = torch.full_like(want, 7.0)
+        assert B.cpa_decode_static(s.plan, q, s.k_pool, s.v_pool, got, s._stream()) == B.CPA_OK
+        assert s.status() == 0
+        assert np.array_equal(_bits(got), _bits(want))
+    finally:
+        s.close()
+        hist.close()
