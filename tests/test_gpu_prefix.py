@@ -261,3 +261,36 @@ def test_decode_entry_points_agree_on_a_prefix_plan():
     finally:
         s.close()
         hist.close()
+
+
+def test_full_prefix8b_sampled():
+    # the configuration `bench.py --config prefix8b` times, in its launch configuration: 16 workers x
+    # (8192 + 16) own tokens over a cached history of 15 x 8192 tokens; prefill rows and decode outputs
+    # are checked on samples the oracle computes one by one
+    w = wl.prefix_aware(16, 8192, 32, 8, 128, 2, seed=11, permute_pages=False).materialise()
+    o = w.own
+    cu = _cu(o)
+    hist, s = _sessions(w, poison=False)
+    try:
+        k, v = _dev(o.k), _dev(o.v)
+        out = _bits(s.prefill(_dev(o.q), k, v))
+        assert s.status() == 0
+        rng = np.random.default_rng(1)
+        rows = []
+        for b in (0, 1, 7, 15):
+            L = int(o.block_lens[b])
+            rows += [int(cu[b]) + r for r in sorted({0, 127, 128, 255, 256, L - 1} | set(rng.integers(0, L, 2).tolist()))]
+        want = oa.prefill_prefix_aware(o.q, o.k, o.v, cu, w.k_hist, w.v_hist, w.prefix_lens, o.scale, rows=rows)
+        assert_attention_close(out[rows], want, "prefix8b prefill, sampled rows")
+        s.append_prefill(k, v)
+        st = oa.PrefixDecodeState(o.k, o.v, cu, w.k_hist, w.v_hist, w.prefix_lens, o.decode_steps)
+        for t in range(o.decode_steps):
+            st.append(o.k_dec[t], o.v_dec[t])
+            got = _bits(s.decode_append(_dev(o.q_dec[t]), _dev(o.k_dec[t]), _dev(o.v_dec[t])))
+            blocks = [0, 1, 8, 15]
+            want = st.decode(o.q_dec[t], o.scale, blocks=blocks)
+            assert_attention_close(got[blocks], want[blocks], f"prefix8b decode step {t}, sampled workers")
+        assert s.status() == 0
+    finally:
+        s.close()
+        hist.close()
