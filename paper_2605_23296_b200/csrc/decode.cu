@@ -367,6 +367,51 @@ decode_split_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __
     if (!sm_last) continue;
     __threadfence();
     const int64_t base = (int64_t)ix.split_indptr[b] * Hq + g * G;
+    constexpr int kMergeTable = kDecodeSmemBytes / 64;   // splits whose (factor, sum) pairs fit the idle rings
+    if (n_splits <= kMergeTable) {
+        // The (max, sum) pairs are fetched once, in parallel, into the idle stage rings and turned into
+        // scale factors there; the accumulator loop then issues nothing but independent loads.
+        float* sm_f = reinterpret_cast<float*>(dsm);              // [n_splits][8] max, then factor
+        float* sm_s = sm_f + kMergeTable * 8;                     // [n_splits][8] sum
+        __shared__ float sm_tot[8];
+        for (int idx = threadIdx.x; idx < n_splits * G; idx += kDecodeThreads) {
+            const int sp = idx / G, h = idx - sp * G;
+            const float2 ml = __ldcg(reinterpret_cast<const float2*>(part_ml + (base + (int64_t)sp * Hq + h) * 2));
+            sm_f[sp * 8 + h] = ml.x;
+            sm_s[sp * 8 + h] = ml.y;
+        }
+        __syncthreads();
+        for (int h = warp; h < G; h += kDecodeWarps) {            // one warp per head: max, factors, total
+            float m = -INFINITY;
+            for (int sp = lane; sp < n_splits; sp += 32) m = fmaxf(m, sm_f[sp * 8 + h]);
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+            float l = 0.f;
+            for (int sp = lane; sp < n_splits; sp += 32) {
+                const float f = exp2f(sm_f[sp * 8 + h] - m);
+                sm_f[sp * 8 + h] = f;
+                l = fmaf(f, sm_s[sp * 8 + h], l);
+            }
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) l += __shfl_xor_sync(0xffffffffu, l, o);
+            if (lane == 0) sm_tot[h] = l;
+        }
+        __syncthreads();
+        for (int idx = threadIdx.x; idx < G * HP; idx += kDecodeThreads) {
+            const int h = idx / HP, dim = 2 * (idx - h * HP);
+            float o0 = 0.f, o1 = 0.f;
+#pragma unroll 8
+            for (int sp = 0; sp < n_splits; ++sp) {
+                const float2 t = __ldcg(reinterpret_cast<const float2*>(part_o + (base + (int64_t)sp * Hq + h) * D + dim));
+                const float f = sm_f[sp * 8 + h];
+                o0 = fmaf(f, t.x, o0);
+                o1 = fmaf(f, t.y, o1);
+            }
+            const float inv = 1.f / sm_tot[h];
+            *reinterpret_cast<__nv_bfloat162*>(out + (out_row + h) * D + dim) = __floats2bfloat162_rn(o0 * inv, o1 * inv);
+        }
+        continue;   // (the next item's first __syncthreads separates these reads from its ring writes)
+    }
     for (int idx = threadIdx.x; idx < G * HP; idx += kDecodeThreads) {
         const int h = idx / HP, dim = 2 * (idx - h * HP);
         float m = -INFINITY;
