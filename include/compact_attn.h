@@ -202,9 +202,9 @@ CPA_API int cpa_prefill(const cpa_plan* plan, const void* q, const void* k, cons
                 void* d_workspace, void* stream);
 
 /*
- * cpa_prefill_prefix -- the prefill of the prefix-aware layout (Section 4, "Dispatch"; the
- * per-worker cost the paper's Section 6 calls "each worker must additionally prefill its own
- * unique block content"): row i of worker w attends over the prefix_lens[w] cached history
+ * cpa_prefill_prefix -- the prefill of the prefix-aware layout (Section 4, "Dispatch"; Section 6
+ * observes that every worker still has to prefill its own block, which the prefix cache does not
+ * hold): row i of worker w attends over the prefix_lens[w] cached history
  * tokens and over its own tokens 0..i,
  *     O[i,h,:] = sum_{j < prefix or j-prefix <= i} softmax_j(scale * q[i,h,:].k[j,g,:]) v[j,g,:].
  *   q, o   : device bf16 [sum(own_lens), num_q_heads, head_dim], the workers' own tokens
