@@ -100,3 +100,8 @@ constexpr int32_t kMaxSharedChunkPages = 1024;
 __host__ __device__ static inline int cpa_pool_piece(int j, int slot) { return (j & ~7) | ((j & 7) ^ (slot & 7)); }
 
 static inline bool cpa_aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// Shared-prefix scan of the prefix-aware decode on the tensor-core path (prefill_tc.cu): partials of every
+// (worker, head) row for every chunk of shared pages go to part_ml / part_o.
+int cpa_scan_tc(const cpa_plan* plan, const void* q, const void* k_pool, const void* v_pool, float* part_ml,
+                float* part_o, void* stream);

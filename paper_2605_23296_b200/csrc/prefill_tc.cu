@@ -85,6 +85,11 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
         "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];\n"
         :: "r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar) : "memory");
 }
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, int x, int y, int z, uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];\n"
+        :: "r"(dst), "l"(map), "r"(x), "r"(y), "r"(z), "r"(bar) : "memory");
+}
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;\n" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory"); }
 // The issuing warp runs its loops convergently (all lanes), which lets the compiler keep MMA
@@ -710,6 +715,301 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
     }
 }
 
+// ---------------------------------------------------------------- shared-prefix scan (decode, prefix-aware layout)
+// The decode step of the prefix-aware layout reads the cached history once for all workers: one
+// unit = (group of consecutive workers, kv head, chunk of shared pages).  The group's (worker, query
+// head) rows (row = worker * G + head, at most 128) are the rows of ONE 128-row tile, the chunk's
+// pages are its KV tiles (eight pages each, gathered from the pool like a cached prefix in the
+// prefill kernel), and the loop is the prefill kernel's single-sub-tile loop without a diagonal:
+// a row sees a KV tile iff the tile lies below its worker's prefix (prefixes are whole tiles).
+// Instead of a normalised output every row that saw a tile leaves a partial
+// (reference max in log2 units, sum, unnormalised accumulator) in slot `chunk` of its worker;
+// the per-worker decode kernel that follows in the stream merges those with its own partials.
+// Eight warps: 0-3 softmax (thread r owns row r), 4 producer, 5 MMA issuer, 6-7 idle.
+constexpr int kScanThreads = 256;
+
+template <int D>
+struct ScanShape {
+    static constexpr int NB = D / 64;
+    static constexpr uint32_t kTileBytes = NB * kBlockBytes;
+    static constexpr int kBufs = 2;                            // score buffers in TMEM
+    static constexpr int kStages = (D == 64) ? 6 : 3;          // K ring and V ring depth
+    static constexpr uint32_t kColO = kBufs * 128;
+    static constexpr uint32_t kTmemCols = 512;
+    static constexpr int kSmem = (1 + 2 * kStages) * (int)kTileBytes + 1024;
+};
+
+struct __align__(8) ScanBarriers {
+    uint64_t q_full, q_empty, k_full[6], k_empty[6], v_full[6], v_empty[6], s_full[4], p_full[4], pv_done;
+    uint32_t tmem_base;
+};
+
+template <int D>
+__global__ void __launch_bounds__(kScanThreads, 1)
+scan_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_kpool,
+               const __grid_constant__ CUtensorMap tm_vpool, float* __restrict__ part_ml, float* __restrict__ part_o,
+               cpa_dev_index ix, int Hq, int Hkv, int G, float scale_log2, int n_units) {
+    using Sh = ScanShape<D>;
+    constexpr int NB = Sh::NB;
+    constexpr uint32_t kTileBytes = Sh::kTileBytes;
+    constexpr int NBUF = Sh::kBufs, KS = Sh::kStages;
+    constexpr uint32_t kColO = Sh::kColO;
+    extern __shared__ unsigned char dsm_raw[];
+    __shared__ ScanBarriers bars;
+
+    const uint32_t base = (smem_u32(dsm_raw) + 1023u) & ~1023u;
+    const uint32_t s_q = base;
+    const uint32_t s_k = s_q + kTileBytes;
+    const uint32_t s_v = s_k + KS * kTileBytes;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    auto bar = [&](uint64_t* p) { return smem_u32(p); };
+
+    if (threadIdx.x == 0) {
+        mbar_init(bar(&bars.q_full), 1);
+        mbar_init(bar(&bars.q_empty), 1);
+        mbar_init(bar(&bars.pv_done), 1);
+        for (int s = 0; s < KS; ++s) {
+            mbar_init(bar(&bars.k_full[s]), 1);
+            mbar_init(bar(&bars.k_empty[s]), 1);
+            mbar_init(bar(&bars.v_full[s]), 1);
+            mbar_init(bar(&bars.v_empty[s]), 1);
+        }
+        for (int i = 0; i < 4; ++i) {
+            mbar_init(bar(&bars.s_full[i]), 1);
+            mbar_init(bar(&bars.p_full[i]), 128);
+        }
+        asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory");
+    }
+    if (warp == 5) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;\n"
+                     :: "r"(smem_u32(&bars.tmem_base)), "r"(Sh::kTmemCols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;\n" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    // the per-worker kernel of this step is next in the stream and needs this one only for its merge
+    asm volatile("griddepcontrol.launch_dependents;\n" ::: "memory");
+    const uint32_t tmem = bars.tmem_base;
+    bool dead = false;
+    // unit u of this CTA: (first worker | workers << 16, kv head, chunk, pages)
+    auto unit = [&](int u) { return __ldg(reinterpret_cast<const int4*>(ix.shared_items) + u); };
+
+    if (warp == 4) {
+        // ------------------------------------------------------------ producer (whole warp)
+        int kt = 0;
+        uint32_t q_loads = 0;
+        for (int u = blockIdx.x; u < n_units; u += gridDim.x) {
+            const int4 it = unit(u);
+            const int w0 = it.x & 0xFFFF, nw = it.x >> 16, g = it.y, first = it.z * ix.shared_chunk, n_tiles = it.w / 8;
+            // The query rows come in boxes of eight tile rows = 8/G workers x G heads of this kv group (a whole
+            // swizzle atom each); a box that reaches past the last worker is filled with zeros.
+            const int per_box = 8 / G, n_boxes = (nw + per_box - 1) / per_box;
+            if (lane == 0) {
+                mbar_wait(bar(&bars.q_empty), (q_loads & 1u) ^ 1u, dead, ix.status);
+                mbar_expect_tx(bar(&bars.q_full), (uint32_t)(n_boxes * NB * 1024));
+            }
+            ++q_loads;
+            __syncwarp();
+            for (int bx = lane; bx < n_boxes; bx += 32) {
+#pragma unroll
+                for (int c = 0; c < NB; ++c)
+                    tma_load_3d(s_q + c * kBlockBytes + bx * 1024, &tm_q, 64 * c, g * G, w0 + bx * per_box, bar(&bars.q_full));
+            }
+            int page = lane < 8 ? __ldg(ix.shared_page_ids + first + lane) : 0;
+            for (int j = 0; j < n_tiles; ++j, ++kt) {
+                const int s = kt % KS;
+                const uint32_t par = (uint32_t)(kt / KS) & 1u;
+                const int row = (page * Hkv + g) * 16;
+                if (lane < 8 && j + 1 < n_tiles) page = __ldg(ix.shared_page_ids + first + 8 * (j + 1) + lane);
+                if (lane == 0) {
+                    mbar_wait(bar(&bars.k_empty[s]), par ^ 1u, dead, ix.status);
+                    mbar_expect_tx(bar(&bars.k_full[s]), kTileBytes);
+                }
+                __syncwarp();
+                if (lane < 8) {
+#pragma unroll
+                    for (int c = 0; c < NB; ++c)
+                        tma_load_2d(s_k + s * kTileBytes + c * kBlockBytes + lane * 2048, &tm_kpool, 64 * c, row, bar(&bars.k_full[s]));
+                }
+                if (lane == 0) {
+                    mbar_wait(bar(&bars.v_empty[s]), par ^ 1u, dead, ix.status);
+                    mbar_expect_tx(bar(&bars.v_full[s]), kTileBytes);
+                }
+                __syncwarp();
+                if (lane < 8) {
+#pragma unroll
+                    for (int c = 0; c < NB; ++c)
+                        tma_load_2d(s_v + s * kTileBytes + c * kBlockBytes + lane * 2048, &tm_vpool, 64 * c, row, bar(&bars.v_full[s]));
+                }
+            }
+        }
+    } else if (warp == 5) {
+        // ------------------------------------------------------------ MMA issuer (whole warp, one lane issues)
+        const uint32_t leader = (lane == 0);
+        constexpr uint32_t idesc_qk = instr_desc(kTileM, kTileN, false);
+        constexpr uint32_t idesc_pv = instr_desc(kTileM, D, true);
+        constexpr uint32_t kTile16 = kTileBytes >> 4;
+        const uint64_t dqk = smem_desc(0, 16, 1024), dvv = smem_desc(0, kBlockBytes, 1024);
+        const uint32_t qk_hi = (uint32_t)(dqk >> 32), pv_hi = (uint32_t)(dvv >> 32);
+        const uint32_t q_lo = (uint32_t)dqk | (s_q >> 4), k_lo = (uint32_t)dqk | (s_k >> 4), v_lo = (uint32_t)dvv | (s_v >> 4);
+        uint32_t n_qk = 0, n_pv = 0, q_uses = 0;
+        int kt0 = 0;
+        auto qk = [&](int buf, int kt) {
+            const uint32_t bq = k_lo + (kt % KS) * kTile16, d_tmem = tmem + buf * 128;
+#pragma unroll
+            for (int k = 0; k < D / 16; ++k) {
+                const uint32_t off = (k >> 2) * (kBlockBytes >> 4) + (k & 3) * 2;
+                tc_mma_ss_lo(d_tmem, q_lo + off, bq + off, qk_hi, idesc_qk, k > 0, leader);
+            }
+            tc_commit(bar(&bars.s_full[n_qk & 3u]), leader);
+            ++n_qk;
+            tc_commit(bar(&bars.k_empty[kt % KS]), leader);
+        };
+        for (int u = blockIdx.x; u < n_units; u += gridDim.x) {
+            const int t_last = unit(u).w / 8 - 1;      // tiles 0 .. t_last
+            mbar_wait(bar(&bars.q_full), q_uses & 1u, dead, ix.status);
+            ++q_uses;
+            for (int i = 0; i < NBUF && i <= t_last; ++i) {
+                mbar_wait(bar(&bars.k_full[(kt0 + i) % KS]), (uint32_t)((kt0 + i) / KS) & 1u, dead, ix.status);
+                tc_fence_after();
+                qk(i, kt0 + i);
+            }
+            if (t_last < NBUF) tc_commit(bar(&bars.q_empty), leader);
+            int buf = 0;
+            for (int j = 0; j <= t_last; ++j) {
+                const int kt = kt0 + j;
+                mbar_wait(bar(&bars.v_full[kt % KS]), (uint32_t)(kt / KS) & 1u, dead, ix.status);
+                mbar_wait(bar(&bars.p_full[n_pv & 3u]), (n_pv >> 2) & 1u, dead, ix.status);
+                ++n_pv;
+                tc_fence_after();
+                const uint32_t bv = v_lo + (kt % KS) * kTile16, d_tmem = tmem + kColO, a_tmem = tmem + buf * 128;
+#pragma unroll
+                for (int k = 0; k < kTileN / 16; ++k)
+                    tc_mma_ts_lo(d_tmem, a_tmem + k * 8, bv + k * (2048 >> 4), pv_hi, idesc_pv, k > 0 ? 1u : (uint32_t)(j > 0), leader);
+                tc_commit(bar(&bars.v_empty[kt % KS]), leader);
+                if (j + NBUF <= t_last) {
+                    mbar_wait(bar(&bars.k_full[(kt + NBUF) % KS]), (uint32_t)((kt + NBUF) / KS) & 1u, dead, ix.status);
+                    tc_fence_after();
+                    qk(buf, kt + NBUF);
+                    if (j + NBUF == t_last) tc_commit(bar(&bars.q_empty), leader);
+                }
+                if (++buf == NBUF) buf = 0;
+            }
+            tc_commit(bar(&bars.pv_done), leader);
+            kt0 += t_last + 1;
+        }
+    } else if (warp < 4) {
+        // ------------------------------------------------------------ softmax + partial write-out (thread r owns row r)
+        const int r = threadIdx.x;
+        const uint32_t lane_addr = ((uint32_t)(warp * 32) << 16);
+        const uint32_t t_o = tmem + lane_addr + kColO;
+        uint32_t n_steps = 0, n_units_done = 0;
+        int kt0 = 0;
+        for (int u = blockIdx.x; u < n_units; u += gridDim.x) {
+            const int4 it = unit(u);
+            const int w0 = it.x & 0xFFFF, nw = it.x >> 16, g = it.y, chunk = it.z, n_tiles = it.w / 8;
+            const int tile0 = chunk * ix.shared_chunk / 8;            // first KV tile of the chunk in the history
+            const bool real = r < nw * G;
+            const int wk = w0 + (real ? r / G : 0), hd = real ? r % G : 0;
+            const int vis_tiles = real ? __ldg(ix.prefix_lens + wk) / kTileN : 0;   // the row sees history tiles below this
+            float m_used = -INFINITY, l_run = 0.f;
+            int buf = 0;
+            for (int j = 0; j < n_tiles; ++j, ++n_steps) {
+                const uint32_t t_s = tmem + lane_addr + buf * 128;
+                mbar_wait(bar(&bars.s_full[n_steps & 3u]), (n_steps >> 2) & 1u, dead, ix.status);
+                tc_fence_after();
+                const bool visible = tile0 + j < vis_tiles;
+                uint32_t sv[4][32];
+#pragma unroll
+                for (int c = 0; c < 4; ++c) tc_ld32_nowait(t_s + c * 32, sv[c]);
+                tc_wait_ld();
+                float mxa[8];
+#pragma unroll
+                for (int a = 0; a < 8; ++a) mxa[a] = max3(__uint_as_float(sv[0][a]), __uint_as_float(sv[0][a + 8]), __uint_as_float(sv[0][a + 16]));
+#pragma unroll
+                for (int a = 0; a < 8; ++a) mxa[a] = fmaxf(mxa[a], __uint_as_float(sv[0][a + 24]));
+#pragma unroll
+                for (int c = 1; c < 4; ++c)
+#pragma unroll
+                    for (int a = 0; a < 8; ++a) {
+                        mxa[a] = max3(mxa[a], __uint_as_float(sv[c][a]), __uint_as_float(sv[c][a + 8]));
+                        mxa[a] = max3(mxa[a], __uint_as_float(sv[c][a + 16]), __uint_as_float(sv[c][a + 24]));
+                    }
+                float mx = max3(max3(mxa[0], mxa[1], mxa[2]), max3(mxa[3], mxa[4], mxa[5]), fmaxf(mxa[6], mxa[7])) * scale_log2;
+                // a row that does not see the tile (or is no row at all) contributes zeros and keeps its state;
+                // its scores may be anything, NaN included, so they are not looked at
+                float alpha = 1.f;
+                if (visible && mx > m_used + 8.f) {       // lazy reference max, as in the prefill kernel
+                    alpha = (m_used == -INFINITY) ? 0.f : exp2f(m_used - mx);
+                    m_used = mx;
+                }
+                if (j > 0 && __any_sync(0xffffffffu, alpha != 1.f)) {
+                    const int kt = kt0 + j - 1;   // O must hold every earlier tile: V tile j-1 is released behind PV(j-1)
+                    mbar_wait(bar(&bars.v_empty[kt % KS]), (uint32_t)(kt / KS) & 1u, dead, ix.status);
+                    tc_fence_after();
+#pragma unroll
+                    for (int c = 0; c < D / 32; ++c) {
+                        float v[32];
+                        tc_ld32(t_o + c * 32, v);
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) v[i] *= alpha;
+                        tc_st32(t_o + c * 32, v);
+                    }
+                }
+                l_run *= alpha;
+                float sum[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+                const float neg_m = -m_used;
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                    uint32_t pk[16];
+#pragma unroll
+                    for (int i = 0; i < 32; i += 2) {
+                        float x0 = __uint_as_float(sv[c][i]), x1 = __uint_as_float(sv[c][i + 1]);
+                        fma_x2(x0, x1, scale_log2, neg_m);
+                        const uint32_t w2 = visible ? pack_bf16(exp2f(x0), exp2f(x1)) : 0u;
+                        pk[i >> 1] = w2;
+                        add_bf16x2(sum[(i >> 1) & 7], w2);
+                    }
+                    tc_st16(t_s + c * 16, pk);
+                }
+                l_run += ((sum[0] + sum[1]) + (sum[2] + sum[3])) + ((sum[4] + sum[5]) + (sum[6] + sum[7]));
+                tc_wait_st();
+                tc_fence_before();
+                mbar_arrive(bar(&bars.p_full[n_steps & 3u]));
+                if (++buf == NBUF) buf = 0;
+            }
+            // ---- the row's partial: (reference max, sum) and the unnormalised accumulator
+            mbar_wait(bar(&bars.pv_done), n_units_done & 1u, dead, ix.status);
+            ++n_units_done;
+            tc_fence_after();
+            const bool write = real && !dead && m_used != -INFINITY;
+            const int64_t prow = write ? (int64_t)(__ldg(ix.split_indptr + wk) + chunk) * Hq + g * G + hd : 0;
+            if (write) *reinterpret_cast<float2*>(part_ml + prow * 2) = make_float2(m_used, l_run);
+#pragma unroll
+            for (int c = 0; c < D / 32; ++c) {
+                float v[32];
+                tc_ld32(t_o + c * 32, v);
+                if (write) {
+#pragma unroll
+                    for (int i = 0; i < 32; i += 4)
+                        *reinterpret_cast<float4*>(part_o + prow * D + c * 32 + i) = make_float4(v[i], v[i + 1], v[i + 2], v[i + 3]);
+                }
+            }
+            tc_fence_before();
+            kt0 += n_tiles;
+        }
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 5) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;\n" :: "r"(tmem), "r"(Sh::kTmemCols) : "memory");
+    }
+}
+
 // ---------------------------------------------------------------- host side
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
@@ -801,7 +1101,61 @@ int launch_prefill_tc(const cpa_plan* plan, const void* q, const void* k, const 
     return cudaGetLastError() == cudaSuccess ? CPA_OK : CPA_ECUDA;
 }
 
+// 3-D view [sequences][heads][D] of the decode queries; box = 64 cols x G heads (one kv group) x 8/G
+// sequences = eight rows of the scan's query tile.
+bool make_q_rows_map(CUtensorMap* map, const void* ptr, int64_t seqs, int64_t heads, int64_t cols, int group) {
+    EncodeTiledFn fn = get_encode_fn();
+    if (!fn) return false;
+    const cuuint64_t dims[3] = {(cuuint64_t)cols, (cuuint64_t)heads, (cuuint64_t)seqs};
+    const cuuint64_t strides[2] = {(cuuint64_t)cols * 2, (cuuint64_t)heads * cols * 2};
+    const cuuint32_t box[3] = {64, (cuuint32_t)group, (cuuint32_t)(8 / group)};
+    const cuuint32_t elem[3] = {1, 1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(ptr), dims, strides, box, elem,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+template <int D>
+int launch_scan_tc(const cpa_plan* plan, const void* q, const void* k_pool, const void* v_pool, float* part_ml,
+                   float* part_o, cudaStream_t st) {
+    const cpa_config& c = plan->cfg;
+    constexpr int smem = ScanShape<D>::kSmem;
+    static bool configured_dev[64] = {};
+    int dev_id = 0;
+    if (cudaGetDevice(&dev_id) != cudaSuccess || dev_id < 0 || dev_id >= 64) {
+        (void)cudaGetLastError();
+        return CPA_ECUDA;
+    }
+    if (!configured_dev[dev_id]) {
+        if (cudaFuncSetAttribute(scan_tc_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) {
+            (void)cudaGetLastError();
+            return CPA_ECUDA;
+        }
+        configured_dev[dev_id] = true;
+    }
+    const int G = c.num_q_heads / c.num_kv_heads;
+    if (8 % G != 0) return CPA_EUNSUPPORTED;   // the query tile is loaded in boxes of 8/G sequences
+    CUtensorMap tm_q, tm_kpool, tm_vpool;
+    const int64_t pool_rows = (int64_t)plan->pool_pages * c.num_kv_heads * c.page_size;
+    if (!make_q_rows_map(&tm_q, q, plan->B, c.num_q_heads, D, G) ||
+        !make_pool_map(&tm_kpool, k_pool, pool_rows, D) || !make_pool_map(&tm_vpool, v_pool, pool_rows, D))
+        return CPA_ECUDA;
+    const int sms = c.num_sms ? c.num_sms : 148;
+    const int grid = plan->n_shared < sms ? plan->n_shared : sms;
+    scan_tc_kernel<D><<<grid, kScanThreads, smem, st>>>(tm_q, tm_kpool, tm_vpool, part_ml, part_o, plan->dev(),
+                                                       c.num_q_heads, c.num_kv_heads, G, c.scale * 1.4426950408889634f,
+                                                       plan->n_shared);
+    return cudaGetLastError() == cudaSuccess ? CPA_OK : CPA_ECUDA;
+}
+
 }  // namespace
+
+int cpa_scan_tc(const cpa_plan* plan, const void* q, const void* k_pool, const void* v_pool, float* part_ml,
+                float* part_o, void* stream) {
+    cudaStream_t st = (cudaStream_t)stream;
+    return plan->cfg.head_dim == 128 ? launch_scan_tc<128>(plan, q, k_pool, v_pool, part_ml, part_o, st)
+                                     : launch_scan_tc<64>(plan, q, k_pool, v_pool, part_ml, part_o, st);
+}
 
 int cpa_prefill_tc(const cpa_plan* plan, const void* q, const void* k, const void* v, void* o, const void* k_pool,
                    const void* v_pool, void* stream) {
