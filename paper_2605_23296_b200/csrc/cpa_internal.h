@@ -90,6 +90,15 @@ struct cpa_plan {
 
 // largest pages-per-split the planner produces: the decode kernel parks a split's page ids in shared memory
 constexpr int32_t kMaxSplitPages = 1024;
+// Which kernel scans the shared pages in the decode of the prefix-aware layout: the tensor-core one takes
+// the rows of a worker group as one 128-row tile (it needs a head group size that divides 8); the
+// warp-MMA one takes 64 rows.
+#ifndef CPA_SCAN_ON_TENSOR_CORES
+#define CPA_SCAN_ON_TENSOR_CORES 1
+#endif
+constexpr bool kScanOnTensorCores = CPA_SCAN_ON_TENSOR_CORES != 0;
+static inline int32_t cpa_scan_rows(int32_t group) { return (kScanOnTensorCores && 8 % group == 0) ? 128 : 64; }
+
 // largest chunk of the shared-prefix scan (its page ids are parked in shared memory too)
 constexpr int32_t kMaxSharedChunkPages = 1024;
 

@@ -446,10 +446,6 @@ decode_split_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __
 constexpr int kSharedThreads = 4 * 32;
 constexpr int kSharedSmemBytes = 64 * 1024;          // the ring (three CTAs per SM)
 constexpr int kSharedLag = 2;
-#ifndef CPA_SCAN_ON_TENSOR_CORES
-#define CPA_SCAN_ON_TENSOR_CORES 1
-#endif
-constexpr bool kScanOnTensorCores = CPA_SCAN_ON_TENSOR_CORES != 0;   // which of the two scan kernels the decode calls launch
 
 template <int D>
 __global__ void __launch_bounds__(kSharedThreads, 3)
@@ -718,7 +714,7 @@ int launch_decode(const cpa_plan* plan, const void* q, const void* k_pool, const
     // Prefix-aware layout: the shared history pages are scanned once for all workers; the partials go
     // to the first slots of every worker and are merged by the launch below, which follows in the stream.
     if (plan->n_shared > 0) {
-        if (kScanOnTensorCores && 8 % G == 0) {   // the tensor-core scan loads its query tile in boxes of 8/G sequences
+        if (cpa_scan_rows(G) == 128) {   // the tensor-core scan (its query tile is loaded in boxes of 8/G sequences)
             const int rc = cpa_scan_tc(plan, q, k_pool, v_pool, part_ml, part_o, st);
             if (rc != CPA_OK) return rc;
         } else {

@@ -177,7 +177,7 @@ int plan_create(const cpa_config* cfg, int32_t num_blocks, const int32_t* block_
     // Prefix-aware layout: the cached prefixes are shared pages, and reading them once per worker
     // would multiply the traffic by about half the worker count.  They are scanned by a kernel of
     // their own instead: the shared pages are cut into chunks of `shared_chunk` pages, workers are
-    // grouped (as many consecutive workers as give 64 (worker, head) rows per kv head), and one
+    // grouped (as many consecutive workers as give 128 (worker, head) rows per kv head), and one
     // item = (group, kv head, chunk) computes a partial for every worker of the group whose prefix
     // reaches into the chunk.  Worker b gets ceil(prefix pages / shared_chunk) partial slots for
     // them in front of the slots of its own splits, which cover its own pages only.
@@ -190,7 +190,7 @@ int plan_create(const cpa_config* cfg, int32_t num_blocks, const int32_t* block_
     p->shared_chunk = 0;
     if (two_level) {
         const int32_t G = cfg->num_q_heads / cfg->num_kv_heads;
-        const int32_t per_group = 64 / G;                                   // workers per group
+        const int32_t per_group = cpa_scan_rows(G) / G;                     // workers per group
         const int32_t n_groups = (B + per_group - 1) / per_group;
         const int64_t sms = cfg->num_sms ? cfg->num_sms : 148;
         const int64_t want = std::max<int64_t>(1, 3 * sms / ((int64_t)cfg->num_kv_heads * n_groups));   // chunks per (group, head)

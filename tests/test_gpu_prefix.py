@@ -98,7 +98,7 @@ def run_event(w, pages_per_split=0, q_tile_rows=0, fused_every=2):
 
 
 @pytest.mark.parametrize("workers,block_len,hq,hkv,d", [(3, 128, 4, 1, 64), (4, 256, 8, 2, 128), (3, 384, 8, 8, 128),
-                                                        (5, 128, 16, 2, 64)])
+                                                        (5, 128, 16, 2, 64), (4, 128, 6, 2, 128)])
 def test_prefix_aware_event(workers, block_len, hq, hkv, d):
     run_event(wl.prefix_aware(workers, block_len, hq, hkv, d, steps=5, seed=workers + d).materialise())
 
@@ -118,8 +118,8 @@ def test_prefix_aware_small_decode_splits():
 
 
 def test_decode_with_two_worker_groups():
-    # G = 8: eight workers fill the 64 rows of a shared-scan item, twelve workers need two groups
-    run_event(wl.prefix_aware(12, 128, 16, 2, 128, steps=3, seed=29).materialise())
+    # G = 8: sixteen workers fill the 128 rows of a shared-scan item, twenty workers need two groups
+    run_event(wl.prefix_aware(20, 128, 16, 2, 128, steps=3, seed=29).materialise())
 
 
 def test_prefix_ends_inside_a_shared_chunk():
