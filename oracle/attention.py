@@ -122,6 +122,22 @@ def attend_token(q: np.ndarray, k: np.ndarray, v: np.ndarray, scale: float,
     return (out, p) if return_weights else out
 
 
+def prefill_chunk(q: np.ndarray, k: np.ndarray, v: np.ndarray, cu_seqlens: Sequence[int], scale: float,
+                  block: int, first_row: int, n_rows: int) -> np.ndarray:
+    """One chunk of a chunked prefill (Section 4.2: the engine prefills long prompts in chunks).
+
+    When rows [first_row, first_row + n_rows) of `block` are prefilled, the block's later tokens do
+    not exist yet: the chunk attends, causally, over the block's tokens [0, first_row + n_rows) and
+    nothing else.  Written as exactly that: the block is cut off behind the chunk and the plain
+    causal attention is evaluated for the chunk's rows.  Returns float64 [n_rows, Hq, d].
+    """
+    lo = int(cu_seqlens[block])
+    end = first_row + n_rows
+    assert 0 <= first_row and n_rows >= 1 and lo + end <= int(cu_seqlens[block + 1])
+    return prefill(q[lo:lo + end], k[lo:lo + end], v[lo:lo + end], [0, end], scale,
+                   rows=np.arange(first_row, end, dtype=np.int64))
+
+
 class DecodeState:
     """Per-block contiguous K/V (independent of any page table).
 
@@ -144,9 +160,10 @@ class DecodeState:
             self.k.append(kb)
             self.v.append(vb)
 
-    def append(self, k_new: np.ndarray, v_new: np.ndarray) -> None:
-        """k_new, v_new: [B,Hkv,d] bf16 bits, one token per block."""
-        for b in range(self.B):
+    def append(self, k_new: np.ndarray, v_new: np.ndarray, blocks: Optional[Sequence[int]] = None) -> None:
+        """k_new, v_new: [B,Hkv,d] bf16 bits, one token per block (only for `blocks` when given: the
+        others sit the step out)."""
+        for b in (range(self.B) if blocks is None else blocks):
             self.k[b][self.len[b]] = k_new[b]
             self.v[b][self.len[b]] = v_new[b]
             self.len[b] += 1

@@ -20,19 +20,15 @@ stated in full):
                   ties by ascending block, kv head, split.  C_b (pages per split)
                   is an input: one number for all blocks or one per block
 * split_indptr    prefix sums of ceil(pages_b / C_b)
+* chunked prefill (Section 4.2: the serving engine runs with chunked prefill enabled; the
+                  paper gives no rule, this one is the library's reading) a block of L_b
+                  tokens is prefilled in ceil(L_b / C) chunks of C tokens (the last one
+                  short), one chunk per step, and decodes its T summary tokens in the T
+                  steps right after its last chunk; see mixed_schedule
 * prefix-aware    (Section 4, "Prefix-aware target-at-end layout") each sequence
                   additionally starts with prefix_lens[b] cached history tokens in
                   shared pages: they come first in its page list, count in seq_lens,
                   in the cost of its prefill items and in its decode splits
-* prefill schedule the deal of prefill units (item, query head) to the CTAs of a
-                  persistent kernel: units listed kv head by kv head, inside a kv
-                  head in prefill-item order, the G query heads of the group side by
-                  side; the list is dealt in rounds of one unit per CTA: CTAs ranked by
-                  cost so far (least first, ties: lower CTA), the round's units by cost
-                  (largest first, ties: list order), i-th unit to i-th CTA; a unit
-                  costs 10 * (its KV tiles of 128 keys) + 18,
-                  where an item of 256 query rows whose block has more than 128 rows
-                  left streams one tile more than its first 128-row half
 """
 from __future__ import annotations
 
@@ -141,30 +137,29 @@ def build_plan(block_lens: Sequence[int], max_new_tokens: int, page_size: int,
     }
 
 
-def prefill_schedule(block_lens: Sequence[int], prefill_items, q_tile_rows: int, num_q_heads: int,
-                     num_kv_heads: int, num_ctas: int, prefix_lens: Sequence[int] = ()):
-    """[rounds][num_ctas] unit codes (item * num_q_heads + head), -1 where a CTA has none."""
-    group = num_q_heads // num_kv_heads
-    units = []                                      # (cost, code) in list order
-    for g in range(num_kv_heads):
-        for i, (b, t) in enumerate(prefill_items):
-            first_row = t * q_tile_rows
-            halves = 2 if (q_tile_rows > 128 and int(block_lens[b]) - first_row > 128) else 1
-            prefix_tiles = int(prefix_lens[b]) // 128 if len(prefix_lens) else 0
-            cost = 10 * (prefix_tiles + first_row // 128 + halves) + 18
-            units += [(cost, i * num_q_heads + g * group + h) for h in range(group)]
-    ctas = min(num_ctas, len(units))
-    load = [0] * ctas
-    table = []
-    for start in range(0, len(units), ctas):
-        batch = sorted(units[start:start + ctas], key=lambda x: -x[0])      # stable: ties stay in list order
-        ranked = sorted(range(ctas), key=lambda c: (load[c], c))
-        row = [-1] * ctas
-        for (cost, code), c in zip(batch, ranked):
-            row[c] = code
-            load[c] += cost
-        table.append(row)
-    return table
+def mixed_schedule(block_lens: Sequence[int], chunk_tokens: int, max_new_tokens: int):
+    """Steps of one event with chunked prefill (Section 4.2: chunked prefill is enabled in the paper's
+    serving engine, so a long block's prefill is cut into chunks that share steps with the decode of
+    blocks that are already past their prefill; Section 6 is why it matters: 16k blocks are
+    prefill-bound).  Rule, stated in full because the paper gives none:
+
+      step s prefills rows [s*C, min((s+1)*C, L_b)) of every block b with s < n_b = ceil(L_b / C);
+      block b decodes summary token t at step n_b + t, t = 0 .. T-1;
+      the event has max_b(n_b) + T steps.
+
+    Returns a list with one entry per step: {"prefill": [(block, first_row, rows)], "decode": [blocks]},
+    both in ascending block order.
+    """
+    if chunk_tokens < 1 or max_new_tokens < 0 or not len(block_lens) or any(int(L) < 1 for L in block_lens):
+        raise ValueError("bad parameter")
+    n_chunks = [-(-int(L) // chunk_tokens) for L in block_lens]
+    steps = []
+    for s in range(max(n_chunks) + max_new_tokens):
+        pre = [(b, s * chunk_tokens, min(chunk_tokens, int(L) - s * chunk_tokens))
+               for b, L in enumerate(block_lens) if s < n_chunks[b]]
+        dec = [b for b in range(len(block_lens)) if n_chunks[b] <= s < n_chunks[b] + max_new_tokens]
+        steps.append({"prefill": pre, "decode": dec})
+    return steps
 
 
 def slot_of(plan: Dict[str, list], page_size: int, block: int, pos: int) -> int:
