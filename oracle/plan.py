@@ -25,6 +25,11 @@ stated in full):
                   tokens is prefilled in ceil(L_b / C) chunks of C tokens (the last one
                   short), one chunk per step, and decodes its T summary tokens in the T
                   steps right after its last chunk; see mixed_schedule
+* pages on demand (Section 8, "Dynamic block size and prompt selection": summaries of unknown
+                  length) instead of reserving pages for T tokens per block, a block holds
+                  pages for the tokens it has plus the next one; the rest of the free list is
+                  a common reserve that any block draws from when it fills a page, and that a
+                  finished block's pages go back to; see DynamicPages
 * prefix-aware    (Section 4, "Prefix-aware target-at-end layout") each sequence
                   additionally starts with prefix_lens[b] cached history tokens in
                   shared pages: they come first in its page list, count in seq_lens,
@@ -160,6 +165,71 @@ def mixed_schedule(block_lens: Sequence[int], chunk_tokens: int, max_new_tokens:
         dec = [b for b in range(len(block_lens)) if n_chunks[b] <= s < n_chunks[b] + max_new_tokens]
         steps.append({"prefill": pre, "decode": dec})
     return steps
+
+
+class DynamicPages:
+    """Page bookkeeping when nothing is reserved for the summaries (the paper's Section 8 asks for
+    per-block sizes that are not known in advance; the rule is this library's).
+
+    A live block always holds exactly the pages for its cached tokens plus the next token:
+    len // P + 1 pages (never more than its table holds, ceil((L + T) / P)).  It starts with that many
+    from the front of the free list, block by block; the rest of the free list is the common reserve.
+    A block that fills a page takes one page from the reserve; a finished block gives all its pages
+    back.  WHICH page a block gets is free (concurrent blocks may draw in any order), so this class
+    tracks counts, and `check` states what any valid outcome satisfies.
+    """
+
+    def __init__(self, block_lens: Sequence[int], max_new_tokens: int, page_size: int, free_pages: Sequence[int]):
+        self.P = page_size
+        self.len = [int(L) for L in block_lens]
+        self.cap = [-(-(int(L) + max_new_tokens) // page_size) for L in block_lens]
+        self.pages = [min(L // page_size + 1, c) for L, c in zip(self.len, self.cap)]
+        if sum(self.pages) > len(free_pages):
+            raise MemoryError("not enough free pages")
+        self.all_pages = sorted(int(x) for x in free_pages)
+        self.initial, taken = [], 0
+        for n in self.pages:
+            self.initial.append([int(x) for x in free_pages[taken:taken + n]])
+            taken += n
+        self.reserve = len(free_pages) - taken
+        self.live = [True] * len(self.len)
+
+    def step(self, active: Sequence[bool]) -> None:
+        """One decode step: every active live block caches one token."""
+        for b, a in enumerate(active):
+            if not (a and self.live[b]):
+                continue
+            if self.len[b] // self.P >= self.pages[b]:
+                raise MemoryError(f"block {b} has no page for its next token")
+            self.len[b] += 1
+            want = min(self.len[b] // self.P + 1, self.cap[b])
+            if want > self.pages[b]:
+                if self.reserve == 0:
+                    continue            # stays short of a page; its next step fails
+                self.reserve -= 1
+                self.pages[b] += 1
+
+    def release(self, blocks: Sequence[int]) -> None:
+        for b in blocks:
+            if self.live[b]:
+                self.reserve += self.pages[b]
+                self.pages[b] = 0
+                self.live[b] = False
+
+    def check(self, table_rows: Sequence[Sequence[int]], assigned: Sequence[int], lens: Sequence[int],
+              ring: Sequence[int]) -> None:
+        """table_rows[b][:assigned[b]] are block b's pages, `ring` the reserve's pages.  Raises
+        AssertionError unless: counts and lengths are the model's; every page of the original free
+        list is in exactly one place; a block's first pages are still the ones it started with."""
+        assert list(lens) == self.len, ("lengths", list(lens), self.len)
+        assert list(assigned) == self.pages, ("pages per block", list(assigned), self.pages)
+        assert len(ring) == self.reserve, ("reserve", len(ring), self.reserve)
+        held = [int(x) for b, row in enumerate(table_rows) for x in row[:assigned[b]]] + [int(x) for x in ring]
+        assert sorted(held) == self.all_pages, "a page is lost, duplicated or foreign"
+        for b, row in enumerate(table_rows):
+            if self.live[b]:
+                n = len(self.initial[b])
+                assert [int(x) for x in row[:n]] == self.initial[b], f"block {b} lost its first pages"
 
 
 def slot_of(plan: Dict[str, list], page_size: int, block: int, pos: int) -> int:
