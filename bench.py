@@ -3,6 +3,9 @@
 
 One "step" is one whole compaction event on synthetic blocks: plan -> ragged
 causal prefill -> bulk KV append -> T x (one-token append + batched decode).
+The default workload is `ragged` (32 blocks of 1024..8192 tokens, 512 decode steps), the
+largest single-GPU configuration; the same JSON line carries `per_config` numbers for
+dense8b, moe120b and the one-block (sequential) split.
 Prints ONE JSON line (rank 0).  `--impl reference` times the CPU oracle instead.
 """
 from __future__ import annotations
@@ -28,10 +31,16 @@ METRIC = "summary tok/s at B blocks (attention only: prefill + paged decode)"
 UNIT = "tok/s"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 NOMINAL_HBM_GBS = 8000.0
-# dram__bytes_read.sum + dram__bytes_write.sum of one decode_split_kernel launch (134.93 MB + 3.9 MB),
-# profiler capture of the kernel as it stands; None for workloads that were not captured
-DECODE_DRAM_BYTES_PER_LAUNCH = {"dense8b": 138.8e6}
 NOMINAL_BF16_TFLOPS = 2250.0
+L2_MB = 126
+DEFAULT_CONFIG = "ragged"   # the largest single-GPU workload of the throughput configurations
+# The other single-GPU configurations, measured in the same run (three timed steps each) into `per_config`.
+PER_CONFIG = [("dense8b", {}), ("moe120b", {}), ("split", {"num_blocks": 1})]
+# Profiler captures of one decode_split_kernel launch per workload (profiles/decode_split_kernel_*.md), of the
+# kernel as it stands: DRAM bytes read + written per launch with the caches left alone between consecutive steps
+# ("warm", the timed condition) and with the L2 flushed before the launch ("cold"), the cold launch duration,
+# and the algorithmic KV bytes of the captured launches.  A workload without a capture has no entry.
+DECODE_CAPTURES = {}
 
 
 def load_peaks():
@@ -117,8 +126,7 @@ def oracle_sample_seconds(w, rows_per_block: int, decode_samples: int):
 
 
 def run_reference(args) -> None:
-    rank = int(os.environ.get("RANK", "0"))
-    if rank != 0:
+    if args.layout[1] != 0:    # rank 0 alone runs the reference arm
         return
     w = make_workload(args.config, overrides=args.overrides).materialise()
     tokens = w.num_blocks * w.decode_steps
@@ -215,42 +223,50 @@ def whole_job_tokens(w, world: int) -> int:
     return world * w.num_blocks * w.decode_steps
 
 
-def run_gpu(args) -> None:
+def rank_layout(gpus: int, env, impl: str = "ours"):
+    """What `--gpus N` means for this process.  ("run", rank, world, local_rank): run as that rank;
+    ("spawn", argv): no launcher started us, so start N ranks (one per GPU) with torch's launcher and
+    relay their exit code.  A launcher whose WORLD_SIZE disagrees with --gpus is an error: the JSON
+    line would claim a GPU count that did not run."""
+    if gpus < 1:
+        raise SystemExit("--gpus must be at least 1")
+    world = env.get("WORLD_SIZE")
+    if world is None:
+        if gpus == 1 or impl == "reference":      # the reference arm runs on rank 0's host cores only
+            return ("run", 0, 1, 0)
+        argv = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={gpus}",
+                "--master-addr", "127.0.0.1", "--master-port", str(29400 + os.getpid() % 500),
+                os.path.abspath(__file__)] + sys.argv[1:]
+        return ("spawn", argv)
+    if int(world) != gpus:
+        raise SystemExit(f"--gpus {gpus} disagrees with the launcher's WORLD_SIZE={world}")
+    return ("run", int(env.get("RANK", "0")), int(world), int(env.get("LOCAL_RANK", "0")))
+
+
+def measure_event(w, args, dev, steps: int, warmup: int, with_e2e: bool, world: int = 1, rank: int = 0,
+                  local_rank: int = 0, sample_clocks: bool = True) -> dict:
+    """Time `steps` whole compaction events of workload `w` (after `warmup` untimed ones) with inputs resident
+    on the device, and optionally the same event from pinned host buffers (copies inside the timed region).
+    Returns phase times (ms, mean over the steps; the step time is the maximum over ranks) and clocks."""
     import torch
     import torch.distributed as dist
 
-    from paper_2605_23296_b200 import binding as B
-    from paper_2605_23296_b200.session import CompactionSession, bits_to_tensor
+    from paper_2605_23296_b200.session import CompactionSession
 
-    rank = int(os.environ.get("RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
-    if not torch.cuda.is_available():
-        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
-    torch.cuda.set_device(local_rank)
-    dev = torch.device("cuda", local_rank)
-    if world > 1:
-        dist.init_process_group("nccl", device_id=dev)
-
-    peaks, peak_kind = load_peaks()
-    # weak scaling: every rank runs its own compaction event of the same shape (own seed);
-    # blocks are independent, so there is no data-path collective
-    w = make_workload(args.config, seed_offset=rank, overrides=args.overrides).materialise()
     T, Bn = w.decode_steps, w.num_blocks
     stream = torch.cuda.current_stream(dev)
 
-    # host-side inputs in pinned memory (for the end-to-end leg) and device-resident copies
     def pinned(bits):
         return torch.from_numpy(bits.view(np.int16)).view(torch.bfloat16).pin_memory()
 
-    h_q, h_k, h_v = pinned(w.q), pinned(w.k), pinned(w.v)
-    h_qd, h_kd, h_vd = pinned(w.q_dec), pinned(w.k_dec), pinned(w.v_dec)
-    d_q, d_k, d_v = h_q.to(dev), h_k.to(dev), h_v.to(dev)
-    d_qd, d_kd, d_vd = h_qd.to(dev), h_kd.to(dev), h_vd.to(dev)
+    def resident(bits):
+        return torch.from_numpy(bits.view(np.int16)).view(torch.bfloat16).to(dev)
+
+    hosts = [pinned(x) for x in (w.q, w.k, w.v, w.q_dec, w.k_dec, w.v_dec)] if with_e2e else None
+    d_q, d_k, d_v, d_qd, d_kd, d_vd = (h.to(dev) for h in hosts) if with_e2e else (
+        resident(x) for x in (w.q, w.k, w.v, w.q_dec, w.k_dec, w.v_dec))
     d_o = torch.empty_like(d_q)
     d_od = torch.empty((T, Bn, w.num_q_heads, w.head_dim), dtype=torch.bfloat16, device=dev)
-    h_o = torch.empty(d_o.shape, dtype=torch.bfloat16).pin_memory()
-    h_od = torch.empty(d_od.shape, dtype=torch.bfloat16).pin_memory()
     flush = torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device=dev)  # > 126 MB of L2
 
     sample_every = max(1, T // 32)   # decode launches that get their own event pair
@@ -294,7 +310,7 @@ def run_gpu(args) -> None:
 
     # ---- device-resident timing ----------------------------------------------------------
     sessions = []
-    for _ in range(args.warmup):
+    for _ in range(warmup):
         sessions.append(one_pass(d_q, d_k, d_v, d_qd, d_kd, d_vd, d_o, d_od))
         flush.fill_(1)
     torch.cuda.synchronize(dev)
@@ -304,12 +320,12 @@ def run_gpu(args) -> None:
     sessions.clear()
 
     sampler = ClockSampler(local_rank)
-    if rank == 0:
+    if rank == 0 and sample_clocks:
         sampler.start()
     barrier()
     state["launches"] = 0
     step_ms, prefill_ms, decode_ms, append_ms, plan_ms, dec_samples = [], [], [], [], [], []
-    for _ in range(args.steps):
+    for _ in range(steps):
         flush.fill_(1)   # L2 flush between timed steps (the step's own inputs, 400+ MB, exceed L2 anyway)
         ev = {n: torch.cuda.Event(enable_timing=True) for n in ("start", "planned", "prefilled", "appended", "end")}
         dec_events = []
@@ -329,94 +345,158 @@ def run_gpu(args) -> None:
     launches = state["launches"]
 
     # ---- end to end: host buffers in, host buffers out, copies inside the timed region -----
-    e2e_ms = []
-    side = torch.cuda.Stream(dev)
-    h2d = sum(t.numel() * 2 for t in (h_q, h_k, h_v, h_qd, h_kd, h_vd))
-    d2h = (h_o.numel() + h_od.numel()) * 2
-    for i in range(0 if args.skip_e2e else 1 + args.steps):
-        flush.fill_(1)
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        torch.cuda.synchronize(dev)
-        e0.record(stream)
-        q, k, v = (t.to(dev, non_blocking=True) for t in (h_q, h_k, h_v))
-        qd, kd, vd = (t.to(dev, non_blocking=True) for t in (h_qd, h_kd, h_vd))
-        ev_pre = {n: torch.cuda.Event() for n in ("planned", "prefilled", "appended")}
-        s = one_pass(q, k, v, qd, kd, vd, d_o, d_od, ev_pre)
-        # the prefill output goes home on a side stream while the decode steps run
-        side.wait_event(ev_pre["prefilled"])
-        with torch.cuda.stream(side):
-            h_o.copy_(d_o, non_blocking=True)
-        h_od.copy_(d_od, non_blocking=True)
-        stream.wait_stream(side)
-        e1.record(stream)
-        torch.cuda.synchronize(dev)
-        assert s.status() == 0
-        s.close()
-        if i > 0:
-            e2e_ms.append(e0.elapsed_time(e1))
+    e2e_ms, h2d, d2h = [], 0, 0
+    if with_e2e:
+        h_q, h_k, h_v, h_qd, h_kd, h_vd = hosts
+        h_o = torch.empty(d_o.shape, dtype=torch.bfloat16).pin_memory()
+        h_od = torch.empty(d_od.shape, dtype=torch.bfloat16).pin_memory()
+        side = torch.cuda.Stream(dev)
+        h2d = sum(t.numel() * 2 for t in hosts)
+        d2h = (h_o.numel() + h_od.numel()) * 2
+        for i in range(1 + steps):
+            flush.fill_(1)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            torch.cuda.synchronize(dev)
+            e0.record(stream)
+            q, k, v = (t.to(dev, non_blocking=True) for t in (h_q, h_k, h_v))
+            qd, kd, vd = (t.to(dev, non_blocking=True) for t in (h_qd, h_kd, h_vd))
+            ev_pre = {n: torch.cuda.Event() for n in ("planned", "prefilled", "appended")}
+            s = one_pass(q, k, v, qd, kd, vd, d_o, d_od, ev_pre)
+            # the prefill output goes home on a side stream while the decode steps run
+            side.wait_event(ev_pre["prefilled"])
+            with torch.cuda.stream(side):
+                h_o.copy_(d_o, non_blocking=True)
+            h_od.copy_(d_od, non_blocking=True)
+            stream.wait_stream(side)
+            e1.record(stream)
+            torch.cuda.synchronize(dev)
+            assert s.status() == 0
+            s.close()
+            if i > 0:
+                e2e_ms.append(e0.elapsed_time(e1))
 
-    clocks = sampler.stop() if rank == 0 else {}   # sampled over both timed legs (device-resident and end-to-end)
-    ms = max_over_ranks(statistics.mean(step_ms), world, dev)
-    e2e = max_over_ranks(statistics.mean(e2e_ms), world, dev) if e2e_ms else float("nan")
+    clocks = sampler.stop() if rank == 0 and sample_clocks else {}   # sampled over both timed legs
+    mean = statistics.mean
+    pair_us = mean(m for _, m in dec_samples) * 1e3 if dec_samples else float("nan")
+    return {"ms": max_over_ranks(mean(step_ms), world, dev),
+            "e2e_ms": max_over_ranks(mean(e2e_ms), world, dev) if e2e_ms else float("nan"),
+            "plan_ms": mean(plan_ms), "prefill_ms": mean(prefill_ms), "append_ms": mean(append_ms),
+            "decode_ms": mean(decode_ms), "pair_us": pair_us, "pair_bytes": (mean(decode_kv_bytes(w, t) for t, _ in dec_samples)
+                                                                            if dec_samples else float("nan")),
+            "n_pairs": len(dec_samples), "launches": launches, "h2d": h2d, "d2h": d2h, "clocks": clocks}
+
+
+def phase_numbers(w, m: dict, peaks: dict, separate_append: bool) -> dict:
+    """Prefill TFLOP/s and decode GB/s (with their fractions of the measured peaks) from phase times."""
+    T = w.decode_steps
+    pf_tflops = prefill_flops(w) / (m["prefill_ms"] * 1e-3) / 1e12
+    total_kv = sum(decode_kv_bytes(w, t) for t in range(T))
+    if separate_append:   # per-launch event pairs on sampled steps
+        launch_us, launch_bytes = m["pair_us"], m["pair_bytes"]
+    else:
+        # every decode step is exactly one launch (append fused in), so the average launch duration over
+        # the timed region is the decode phase's CUDA-event time / T; event pairs around single launches
+        # add their own cost and break the overlap of consecutive launches
+        launch_us, launch_bytes = m["decode_ms"] * 1e3 / T, total_kv / T
+    gbs = launch_bytes / (launch_us * 1e-6) / 1e9
+    return {"prefill_ms": m["prefill_ms"], "prefill_tflops": pf_tflops,
+            "prefill_frac_of_bf16_peak": pf_tflops / peaks["bf16_tflops"],
+            "prefill_frac_of_nominal_2250": pf_tflops / NOMINAL_BF16_TFLOPS,
+            "decode_ms": m["decode_ms"], "decode_launch_us": launch_us, "decode_bytes_per_launch": launch_bytes,
+            "decode_gbs": gbs, "decode_frac_of_hbm_peak": gbs / peaks["hbm_gbs"],
+            "decode_frac_of_nominal_8TBs": gbs / NOMINAL_HBM_GBS,
+            "decode_pool_vs_l2": ("pool of %.0f MB per step against %d MB of L2: %s" % (
+                launch_bytes / 1e6, L2_MB, "an effective (L2-assisted) rate, not an HBM fraction"
+                if launch_bytes < 2.5 * L2_MB * 1e6 else "HBM-bound, at most a fifth can come from L2"))}
+
+
+def run_gpu(args) -> None:
+    import gc
+
+    import torch
+    import torch.distributed as dist
+
+    _, rank, world, local_rank = args.layout
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+
+    peaks, peak_kind = load_peaks()
+    # weak scaling: every rank runs its own compaction event of the same shape (own seed);
+    # blocks are independent, so there is no data-path collective
+    w = make_workload(args.config, seed_offset=rank, overrides=args.overrides).materialise()
+    T, Bn = w.decode_steps, w.num_blocks
+    m = measure_event(w, args, dev, args.steps, args.warmup, not args.skip_e2e, world, rank, local_rank)
     if rank != 0:
         if world > 1:
             dist.destroy_process_group()
         return
 
     tokens = whole_job_tokens(w, world)
-    pf_ms, dc_ms = statistics.mean(prefill_ms), statistics.mean(decode_ms)
-    pf_tflops = prefill_flops(w) / (pf_ms * 1e-3) / 1e12
-    total_kv = sum(decode_kv_bytes(w, t) for t in range(T))
-    dec_gbs_phase = total_kv / (dc_ms * 1e-3) / 1e9           # includes the per-step appends
-    # dominant kernel: the decode launches (split + merge), per-launch event pairs on sampled steps
-    samp_bytes = statistics.mean(decode_kv_bytes(w, t) for t, _ in dec_samples)
-    samp_ms = statistics.mean(m for _, m in dec_samples)
-    pair_us = samp_ms * 1e3
-    if not args.separate_append:
-        # every decode step is exactly one launch (append fused in), so the average launch duration
-        # over the timed region is the decode phase's CUDA-event time / T; event pairs around single
-        # launches add their own cost and break the overlap of consecutive launches
-        samp_bytes = total_kv / T
-        samp_ms = dc_ms / T
-    achieved = samp_bytes / (samp_ms * 1e-3) / 1e9
-    # DRAM bytes per launch (read + written) from a profiler capture of this kernel on the default
-    # workload; the capture replays each launch with a cold L2, whereas consecutive launches of a
-    # real step share L2 contents (the scan direction alternates), so this is the upper figure
-    overridden = args.blocks or args.block_len or args.decode_steps or args.pages_per_split or args.separate_append
-    traffic = DECODE_DRAM_BYTES_PER_LAUNCH.get(args.config) if not overridden else None
+    ph = phase_numbers(w, m, peaks, args.separate_append)
+    overridden = bool(args.blocks or args.block_len or args.decode_steps or args.pages_per_split or args.separate_append)
+    cap = DECODE_CAPTURES.get(args.config) if not overridden else None
+    # dominant kernel: the decode launches (one per step: append, split-K scan and merge fused).  `achieved` divides the
+    # ALGORITHMIC KV bytes by the launch time: when a step's pool is not much larger than the L2 (dense8b), part of
+    # those bytes is served from L2, and the figure is an effective rate.  `traffic` is the DRAM traffic of a launch
+    # in the timed condition (back-to-back steps, caches left alone), `traffic_cold` with the L2 flushed before the
+    # launch, `frac_cold_l2` the fraction the kernel reaches from a cold L2; all three from profiler captures of this
+    # kernel on this workload (profiles/), null where there is no capture of the kernel as it stands.
     roofline = {"bound": "hbm", "kernel": "decode_split_kernel (one launch per step: append, split-K scan and merge fused)",
-                "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                "frac": achieved / peaks["hbm_gbs"], "peak_kind": f"of {peak_kind}",
-                "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS,
-                "launch_us": samp_ms * 1e3, "bytes_per_launch": samp_bytes,
-                "launches_timed": (T * args.steps if not args.separate_append else len(dec_samples)),
-                "launch_us_event_pair_sampled": pair_us, "traffic": traffic}
+                "achieved": ph["decode_gbs"], "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                "frac": ph["decode_frac_of_hbm_peak"], "peak_kind": f"of {peak_kind}",
+                "frac_of_nominal_8TBs": ph["decode_frac_of_nominal_8TBs"],
+                "launch_us": ph["decode_launch_us"], "bytes_per_launch": ph["decode_bytes_per_launch"],
+                "launches_timed": (T * args.steps if not args.separate_append else m["n_pairs"]),
+                "launch_us_event_pair_sampled": m["pair_us"],
+                "traffic": cap["traffic_warm"] if cap else None,
+                "traffic_cold": cap["traffic_cold"] if cap else None,
+                "frac_cold_l2": (cap["algorithmic"] / (cap["cold_us"] * 1e-6) / 1e9 / peaks["hbm_gbs"]) if cap else None,
+                "traffic_source": cap["source"] if cap else None,
+                "l2_note": ph["decode_pool_vs_l2"]}
+
+    # ---- the other single-GPU configurations, three timed steps each, device-resident only -----
+    per_config = {}
+    if args.per_config and world == 1 and not overridden:
+        del w.q, w.k, w.v
+        for name, kw in PER_CONFIG:
+            if name == args.config and not kw:
+                continue
+            gc.collect()
+            torch.cuda.empty_cache()
+            w2 = wl.CONFIGS[name](**kw).materialise()
+            m2 = measure_event(w2, args, dev, 3, 3, False)
+            p2 = phase_numbers(w2, m2, peaks, False)
+            label = name if not kw else f"{name}:B={kw['num_blocks']}"
+            per_config[label] = dict(p2, config=workload_desc(w2), ms_per_step=m2["ms"],
+                                     value=w2.num_blocks * w2.decode_steps / (m2["ms"] * 1e-3), steps=3, warmup=3,
+                                     clocks=m2["clocks"])
+            del w2
+        w = make_workload(args.config, seed_offset=rank, overrides=args.overrides).materialise()
 
     if args.skip_cpu:
         cpu = {"estimated_step_s": float("nan"), "cores": 0, "sample": "skipped", "measured_s": 0.0}
     else:
         cpu = oracle_sample_seconds(w, rows_per_block=32, decode_samples=8)
     out = {
-        "metric": METRIC, "value": tokens / (ms * 1e-3), "unit": UNIT, "n_gpus": world,
-        "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
+        "metric": METRIC, "value": tokens / (m["ms"] * 1e-3), "unit": UNIT, "n_gpus": world,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": m["ms"], "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-        "config": dict(workload_desc(w), l2="256 MiB write between timed steps; step inputs (>400 MB) exceed L2",
-                       parallelism=f"replicas x{world} (independent blocks, no collective)"),
-        "phases": {"plan_ms": statistics.mean(plan_ms), "prefill_ms": pf_ms,
-                   "bulk_append_ms": statistics.mean(append_ms), "decode_ms": dc_ms,
-                   "prefill_tflops": pf_tflops,
-                   "prefill_frac_of_bf16_peak": pf_tflops / peaks["bf16_tflops"],
-                   "prefill_frac_of_nominal_2250": pf_tflops / NOMINAL_BF16_TFLOPS,
-                   "decode_gbs_incl_append": dec_gbs_phase,
-                   "decode_frac_of_hbm_peak": dec_gbs_phase / peaks["hbm_gbs"],
-                   "peaks": dict(peaks, kind=peak_kind)},
+        "config": workload_desc(w),
+        "timing": {"l2": "256 MiB write between timed steps; step inputs (>400 MB) exceed L2",
+                   "parallelism": f"replicas x{world} (independent blocks, no collective)"},
+        "phases": dict(ph, plan_ms=m["plan_ms"], bulk_append_ms=m["append_ms"], peaks=dict(peaks, kind=peak_kind)),
         "roofline": roofline,
+        "per_config": per_config,
         "cpu_baseline": {"value": Bn * T / cpu["estimated_step_s"], "unit": UNIT, "cores": cpu["cores"],
                          "kind": "oracle", "sample": cpu["sample"], "measured_s": cpu["measured_s"]},
-        "e2e": {"value": tokens / (e2e * 1e-3), "unit": UNIT, "ms_per_step": e2e,
-                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
-        "gpu_launches": launches,
-        "clocks": clocks,
+        "e2e": {"value": tokens / (m["e2e_ms"] * 1e-3), "unit": UNIT, "ms_per_step": m["e2e_ms"],
+                "h2d_bytes_per_step": m["h2d"], "d2h_bytes_per_step": m["d2h"]},
+        "gpu_launches": m["launches"],
+        "clocks": m["clocks"],
     }
     print(json.dumps(out))
     if world > 1:
@@ -435,7 +515,7 @@ def run_prefix(args) -> None:
 
     from paper_2605_23296_b200.session import CompactionSession, bits_to_tensor
 
-    if int(os.environ.get("WORLD_SIZE", "1")) != 1:
+    if args.layout[2] != 1:
         raise SystemExit("--config prefix8b is a single-GPU measurement")
     dev = torch.device("cuda", 0)
     torch.cuda.set_device(dev)
@@ -529,7 +609,109 @@ def run_prefix(args) -> None:
 
 
 # ------------------------------------------------------------------------------------------
-# compaction in the background of a decoding agent (paper, Section 7: asynchronous compaction)
+# chunked prefill mixed with decode (paper, Section 4.2 and Section 6): a separate, non-default workload
+# ------------------------------------------------------------------------------------------
+
+def run_mixed(args) -> None:
+    """`--config mixed16k`: one 16k block beside four 2k blocks (8B-class heads), T summary tokens each.  Whole-block
+    calls (one prefill launch over all blocks, then T decode steps) against the chunked schedule (2048-token chunks;
+    the short blocks decode while the long block is still prefilling, cpa_step_mixed).  Reports when the short
+    blocks' first and last summary tokens are out and when the whole event is done, both ways."""
+    import torch
+
+    from paper_2605_23296_b200 import binding as B
+    from paper_2605_23296_b200.session import CompactionSession, bits_to_tensor
+
+    if args.layout[2] != 1:
+        raise SystemExit("--config mixed16k is a single-GPU measurement")
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    peaks, peak_kind = load_peaks()
+    T = args.decode_steps or 256
+    chunk = 2048
+    lens = [16384, 2048, 2048, 2048, 2048]
+    w = wl.custom(lens, 32, 8, 128, steps=T, seed=13, permute_pages=True).materialise()
+    Bn = w.num_blocks
+    stream = torch.cuda.current_stream(dev)
+    d = lambda bits: bits_to_tensor(bits, dev)
+    q, k, v, qd, kd, vd = (d(x) for x in (w.q, w.k, w.v, w.q_dec, w.k_dec, w.v_dec))
+    o = torch.empty_like(q)
+    od = torch.empty((T + 8, Bn, w.num_q_heads, w.head_dim), dtype=torch.bfloat16, device=dev)
+    flush = torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device=dev)
+    new_ev = lambda: torch.cuda.Event(enable_timing=True)
+
+    def whole_blocks():
+        ev = {n: new_ev() for n in ("start", "first", "end")}
+        s = CompactionSession(w.block_lens, T, w.num_q_heads, w.num_kv_heads, w.head_dim, w.free_pages, w.num_pages,
+                              scale=w.scale)
+        torch.cuda.synchronize(dev)
+        ev["start"].record(stream)      # (planning and the plan's upload are outside both measurements)
+        s.prefill(q, k, v, out=o)
+        s.append_prefill(k, v)
+        for t in range(T):
+            s.decode_append(qd[t], kd[t], vd[t], out=od[t])
+            if t == 0:
+                ev["first"].record(stream)
+        ev["end"].record(stream)
+        return s, ev
+
+    def chunked():
+        ev = {n: new_ev() for n in ("start", "first", "short_done", "long_prefilled", "end")}
+        s = CompactionSession(w.block_lens, T, w.num_q_heads, w.num_kv_heads, w.head_dim, w.free_pages, w.num_pages,
+                              scale=w.scale, chunk_tokens=chunk, decode_sms=args.decode_sms)
+        start = s.export(B.ARR_DEC_START)
+        n_steps = s.param(B.PARAM_NUM_STEPS)
+        n_long = int(start.max())
+        # a block's t-th token takes the inputs of row t whatever step produces it: the short blocks run one
+        # step ahead per chunk of the long one, so the decode inputs of a step are gathered per block
+        steps_in = []
+        for step in range(n_steps):
+            t_of = np.clip(step - start, 0, T - 1)
+            steps_in.append(torch.from_numpy(t_of.astype(np.int64)).to(dev))
+        ar = torch.arange(Bn, device=dev)
+        gathered = [(qd[t_of, ar], kd[t_of, ar], vd[t_of, ar]) for t_of in steps_in]   # staged before the timed calls
+        torch.cuda.synchronize(dev)
+        ev["start"].record(stream)
+        for step in range(n_steps):
+            qi, ki, vi = gathered[step]
+            s.step_mixed(step, q, k, v, o, qi, ki, vi, od[min(step, T + 7)])
+            if step == 1:
+                ev["first"].record(stream)
+            if step == int(start.min()) + T - 1:
+                ev["short_done"].record(stream)
+            if step == n_long - 1:
+                ev["long_prefilled"].record(stream)
+        ev["end"].record(stream)
+        return s, ev
+
+    res = {"whole_blocks": [], "chunked": []}
+    for i in range(args.warmup + args.steps):
+        for name, fn in (("whole_blocks", whole_blocks), ("chunked", chunked)):
+            flush.fill_(1)
+            s, ev = fn()
+            torch.cuda.synchronize(dev)
+            assert s.status() == 0
+            s.close()
+            if i >= args.warmup:
+                res[name].append({n: ev["start"].elapsed_time(e) for n, e in ev.items() if n != "start"})
+    mean = lambda name, key: statistics.mean(r[key] for r in res[name])
+    out = {
+        "metric": "time until the short blocks' summaries are out, whole-block prefill vs chunked prefill mixed with decode",
+        "unit": "ms", "n_gpus": 1, "steps": args.steps, "warmup": args.warmup, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": "mixed16k", "block_lens": lens, "q_heads": 32, "kv_heads": 8, "head_dim": 128,
+                   "decode_steps": T, "chunk_tokens": chunk, "decode_sms": args.decode_sms or "a quarter of the SMs",
+                   "seed": w.seed},
+        "whole_blocks": {"first_summary_token_ms": mean("whole_blocks", "first"),
+                         "short_blocks_done_ms": mean("whole_blocks", "end"), "event_ms": mean("whole_blocks", "end")},
+        "chunked": {"first_summary_token_ms": mean("chunked", "first"),
+                    "short_blocks_done_ms": mean("chunked", "short_done"),
+                    "long_block_prefilled_ms": mean("chunked", "long_prefilled"), "event_ms": mean("chunked", "end")},
+    }
+    print(json.dumps(out))
+
+
+# ------------------------------------------------------------------------------------------
+# compaction in the background of a decoding agent (paper, Section 8: asynchronous compaction)
 # ------------------------------------------------------------------------------------------
 
 def run_async(args) -> None:
@@ -642,11 +824,14 @@ def main() -> None:
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--config", default="dense8b", choices=sorted(wl.CONFIGS) + ["prefix8b", "async"])
+    ap.add_argument("--config", default=DEFAULT_CONFIG, choices=sorted(wl.CONFIGS) + ["prefix8b", "async", "mixed16k"])
+    ap.add_argument("--no-per-config", dest="per_config", action="store_false",
+                    help="skip the per_config measurements of the other configurations")
     ap.add_argument("--blocks", type=int, default=0, help="override the number of blocks (profiling)")
     ap.add_argument("--block-len", type=int, default=0, help="override the block length (profiling)")
     ap.add_argument("--decode-steps", type=int, default=0, help="override the decode steps (profiling)")
     ap.add_argument("--pages-per-split", type=int, default=0, help="decode split size (0 = planner's choice)")
+    ap.add_argument("--decode-sms", type=int, default=0, help="mixed16k: SMs left to the decode wave beside a prefill chunk")
     ap.add_argument("--separate-append", action="store_true",
                     help="per decode step call cpa_kv_append and cpa_decode instead of the fused cpa_decode_append")
     ap.add_argument("--skip-e2e", action="store_true", help="skip the host-buffer leg (profiling)")
@@ -657,10 +842,13 @@ def main() -> None:
         ap.error("--block-len does not apply to this configuration")
     if args.config == "tiny":
         args.overrides = {}
-    if args.config in ("prefix8b", "async"):
+    args.layout = rank_layout(args.gpus, os.environ, args.impl)
+    if args.layout[0] == "spawn":
+        raise SystemExit(subprocess.run(args.layout[1]).returncode)
+    if args.config in ("prefix8b", "async", "mixed16k"):
         if args.impl == "reference":
             raise SystemExit("--impl reference times the default layout's workloads")
-        run_prefix(args) if args.config == "prefix8b" else run_async(args)
+        {"prefix8b": run_prefix, "async": run_async, "mixed16k": run_mixed}[args.config](args)
     elif args.impl == "reference":
         run_reference(args)
     else:

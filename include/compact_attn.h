@@ -31,8 +31,18 @@
  *     memory is read without bank conflicts.  Only this library reads the pools.
  *   - Every call returns 0 (CPA_OK) or a negative cpa_status.  Nothing throws,
  *     exits, or traps the device.  Device-side waits are bounded; if one gives up
- *     the kernel records it in the plan's device status word, which
- *     cpa_plan_status reads back.
+ *     the kernel stops issuing work, lets the copies and MMAs it has in flight
+ *     finish (again with a bound), frees its tensor memory and returns, and the
+ *     plan's device status word (the first int32 of the index buffer) keeps the
+ *     first code recorded: 1 = a wait gave up, 2 = an append found no room.
+ *     cpa_plan_status reads it back.  After a non-zero status the results of that
+ *     launch are void and the plan must be uploaded again before further use.
+ *   - Thread safety: a plan is used by one host thread at a time.  Different
+ *     plans may be used from different threads; the library's only process-wide
+ *     state are per-device flags and addresses that every thread sets to the same
+ *     value (kept in relaxed atomics).
+ *   - Limits: group size G <= 8, num_sms <= 4095, block lengths and page counts
+ *     below 2^30, and at most 65535 workers in a plan with cached prefixes.
  *   - There is no CPU fallback: without a CUDA device the compute calls return
  *     CPA_ECUDA.
  */
@@ -70,9 +80,11 @@ typedef struct cpa_config {
     int32_t q_tile_rows;     /* query rows per prefill work item: 128 or 256; 0 = default (256) */
     int32_t pages_per_split; /* KV pages per decode work item (<= 1024); 0 = chosen per block from the batch */
     int32_t num_sms;         /* SMs this plan's kernels may fill: the persistent prefill launches min(num_sms, units)
-                                CTAs (one per SM) and the decode wave is sized for 3 * num_sms CTAs; 0 = 148.  A
-                                value below the device's SM count leaves SMs to other streams (a CTA of the
-                                prefill keeps its SM for the whole launch, stream priority does not preempt it) */
+                                CTAs (one per SM) and the decode wave is sized for 3 * num_sms CTAs; 0 = the SM
+                                count of the device that is current when the plan is created (148 if there is
+                                none); at most 4095.  A value below the device's SM count leaves SMs to other
+                                streams (a CTA of the prefill keeps its SM for the whole launch, stream priority
+                                does not preempt it) */
 } cpa_config;
 
 typedef struct cpa_plan cpa_plan; /* opaque; host memory owned by the library */
@@ -88,8 +100,13 @@ enum {
     CPA_ARR_DECODE_ITEMS = 6,  /* [n,3] (block, kv_head, split) in launch order */
     CPA_ARR_SPLIT_INDPTR = 7,  /* [B+1] prefix sums of decode splits per block */
     CPA_ARR_SPLIT_PAGES = 8,   /* [B] pages per decode split of each block (the last split may be shorter) */
-    CPA_ARR_PREFILL_SCHED = 9  /* [rounds * CPA_PARAM_PREFILL_CTAS] prefill unit (item * num_q_heads + head) of CTA c
+    CPA_ARR_PREFILL_SCHED = 9, /* [rounds * CPA_PARAM_PREFILL_CTAS] prefill unit (item * num_q_heads + head) of CTA c
                                   in round k at k * ctas + c, -1 = none; every unit appears exactly once */
+    CPA_ARR_DEC_START = 10,    /* [B] chunked plans: the step at which each block starts to decode (its chunk count) */
+    CPA_ARR_CHUNK_ROWS = 11,   /* [CPA_PARAM_CHUNK_STEPS * (B+1)] chunked plans: per step, prefix sums of the rows
+                                  each block prefills in it */
+    CPA_ARR_PAGES_ASSIGNED = 12, /* [B] plans with pages on demand: pages each block holds (as of creation or the last cpa_plan_sync) */
+    CPA_ARR_FREE_RING = 13     /* plans with pages on demand: the pages of the common reserve, in the order they will be handed out */
 };
 
 /* Scalars of a plan, for cpa_plan_param. */
@@ -104,7 +121,12 @@ enum {
     CPA_PARAM_TOTAL_SPLITS = 7,          /* split_indptr[B] */
     CPA_PARAM_MAX_NEW_TOKENS = 8,
     CPA_PARAM_PREFILL_CTAS = 9,          /* CTAs of the prefill launch = min(num_sms, prefill units) */
-    CPA_PARAM_SHARED_CHUNK_PAGES = 10    /* pages per chunk of the shared-prefix decode scan; 0 without cached prefixes */
+    CPA_PARAM_SHARED_CHUNK_PAGES = 10,   /* pages per chunk of the shared-prefix decode scan; 0 without cached prefixes */
+    CPA_PARAM_CHUNK_TOKENS = 11,         /* tokens per prefill chunk; 0 = not a chunked plan */
+    CPA_PARAM_NUM_STEPS = 12,            /* steps of a chunked plan's schedule: most chunks of any block + max_new_tokens */
+    CPA_PARAM_CHUNK_STEPS = 13,          /* steps that prefill a chunk (the most chunks of any block) */
+    CPA_PARAM_DECODE_SMS = 14,           /* SMs a chunked plan leaves to the decode wave while a chunk is prefilled */
+    CPA_PARAM_NUM_SMS = 15               /* the plan's SM budget (cfg.num_sms, or the device's SM count for 0) */
 };
 
 /*
@@ -165,6 +187,54 @@ CPA_API int cpa_plan_create_prefix(const cpa_config* cfg, int32_t num_workers, c
                                    int32_t max_new_tokens, const int32_t* free_pages, int32_t num_free,
                                    cpa_plan** out);
 
+/*
+ * cpa_plan_create_chunked -- the plan for an event whose prefill runs in chunks.  The paper's serving
+ * engine runs with chunked prefill enabled (Section 4.2, "Hardware and Serving Infrastructure"), and its
+ * finding that 16k blocks are prefill-bound (Section 6, "Prefill cost limits parallelism") is the case
+ * this is for: a long block's prompt is cut into chunks, and the blocks that are past their prompt
+ * decode in the same steps instead of waiting behind it.  The paper gives no rule; this library's is:
+ *   a block of L_b tokens has n_b = ceil(L_b / chunk_tokens) chunks and prefills chunk s, rows
+ *   [s * chunk_tokens, min((s + 1) * chunk_tokens, L_b)), in step s < n_b; it decodes summary token t
+ *   in step n_b + t, t < max_new_tokens; the schedule has max_b(n_b) + max_new_tokens steps
+ *   (CPA_PARAM_NUM_STEPS), run one by one with cpa_step_mixed.
+ * chunk_tokens: a multiple of 128 (a later chunk reads the earlier ones from the block's pages in whole
+ * KV tiles of 128 keys).  decode_sms: SMs left to the decode wave in steps that also prefill a chunk
+ * (the chunk's persistent grid takes the other num_sms - decode_sms); 0 = a quarter of the plan's SMs.
+ * Everything else (pages, slots, whole-block prefill list, decode items) is as for cpa_plan_create, and
+ * the plan also works with the whole-block calls (cpa_prefill, cpa_kv_append, cpa_decode_append) as long
+ * as the two ways are not mixed within one event.  Errors as for cpa_plan_create, plus CPA_EINVAL for a
+ * chunk size below 128 or not a multiple of 128 and for decode_sms >= the plan's SMs.
+ */
+CPA_API int cpa_plan_create_chunked(const cpa_config* cfg, int32_t num_blocks, const int32_t* block_lens,
+                                    int32_t max_new_tokens, int32_t chunk_tokens, int32_t decode_sms,
+                                    const int32_t* free_pages, int32_t num_free, cpa_plan** out);
+
+/*
+ * cpa_plan_create_dynamic -- a plan that reserves no pages for the summaries.  The paper's outlook (Section 8,
+ * "Dynamic block size and prompt selection") wants block sizes and summary lengths that are not fixed in
+ * advance, and its second benchmark (Section 3.1: documents of about 0.7k tokens, six questions each) is many
+ * short sequences whose summaries stop at different lengths; reserving max_new_tokens for each wastes most of
+ * the pool.  The paper has no rule; this library's is:
+ *   a block starts with the pages for its tokens plus the next one, L_b / page_size + 1 of them (never more than
+ *   its row of the page table holds, ceil((L_b + max_new_tokens) / page_size): max_new_tokens only bounds growth),
+ *   dealt in order from `free_pages`; the rest of `free_pages` becomes a common reserve, a ring in the index
+ *   buffer; the decode launch that fills a block's page takes the next page for it from the ring; a block that
+ *   has stopped gives its pages back with cpa_release_blocks.
+ * CPA_ARR_PAGE_INDICES is then a table of B rows (row b = page_indptr[b] .. page_indptr[b+1]), valid up to
+ * CPA_ARR_PAGES_ASSIGNED[b] entries; the host copies are those of plan creation until cpa_plan_sync refreshes
+ * them.  Decode with cpa_decode_append or cpa_decode_append_dynamic (cpa_kv_append with new_lens == NULL
+ * returns CPA_EUNSUPPORTED: it takes no pages).  Errors as for cpa_plan_create (CPA_ENOSPC: the free list does
+ * not cover the first pages).
+ */
+CPA_API int cpa_plan_create_dynamic(const cpa_config* cfg, int32_t num_blocks, const int32_t* block_lens,
+                                    int32_t max_new_tokens, const int32_t* free_pages, int32_t num_free,
+                                    cpa_plan** out);
+
+/* Synchronise `stream` and read the device's lengths (CPA_ARR_SEQ_LENS) and, for a plan with pages on demand, its
+ * page table, pages per block and reserve back into the host copies that cpa_plan_export shows.  (The paper has
+ * no counterpart.)  Errors: CPA_EINVAL, CPA_ESTATE (not uploaded), CPA_ECUDA. */
+CPA_API int cpa_plan_sync(cpa_plan* plan, void* stream);
+
 /* Borrow a host view of one index array (valid until the plan is destroyed or,
  * for CPA_ARR_SEQ_LENS, until the next cpa_kv_append).  Errors: CPA_EINVAL. */
 CPA_API int cpa_plan_export(const cpa_plan* plan, int which, const int32_t** ptr, int64_t* count);
@@ -181,7 +251,8 @@ CPA_API int64_t cpa_plan_param(const cpa_plan* plan, int which);
  */
 CPA_API int cpa_plan_upload(cpa_plan* plan, void* d_index_buf, int64_t bytes, void* stream);
 
-/* Synchronise `stream`, read the device status word: CPA_OK, CPA_ETIMEOUT, or
+/* Synchronise `stream`, read the device status word: CPA_OK, CPA_ETIMEOUT (a bounded
+ * device-side wait gave up), CPA_ENOSPC (an append found no page or slot left), or
  * CPA_ECUDA if the stream reports an error.  CPA_ESTATE before upload. */
 CPA_API int cpa_plan_status(cpa_plan* plan, void* stream);
 
@@ -233,6 +304,9 @@ CPA_API int cpa_prefill_variant(const cpa_plan* plan, const void* q, const void*
 /*
  * cpa_kv_append -- write new K/V rows into the blocks' pages and advance
  * seq_lens (the KV cache each sequence keeps while it decodes its summary).
+ * The paper has no counterpart: Section 4.2 names the serving engine whose paged
+ * cache does this underneath and says nothing about it; the slot rule below is
+ * this library's own.
  *   k_new, v_new : device bf16 [sum(new_lens), num_kv_heads, head_dim], block-major
  *   new_lens     : host int32 [B] tokens to add per block, or NULL = one token
  *                  per block (a decode step; then k_new is [B, kv_heads, head_dim]).
@@ -247,7 +321,10 @@ CPA_API int cpa_kv_append(cpa_plan* plan, const void* k_new, const void* v_new, 
                   void* k_pool, void* v_pool, void* stream);
 
 /*
- * cpa_decode -- one batched decode step: the newest token of every block
+ * cpa_decode -- one batched decode step (Section 4, "Dispatch": the N summarisation
+ * sequences run concurrently, so every step produces one token of every block's
+ * summary; Section 2.1 notes that the per-token cost of this step grows with the
+ * context length): the newest token of every block
  * attends over that block's whole cache, the token itself included (call
  * cpa_kv_append for the step first).  Split-K over the block's pages, then a
  * log-sum-exp merge of the split partials
@@ -257,7 +334,8 @@ CPA_API int cpa_kv_append(cpa_plan* plan, const void* k_new, const void* v_new, 
  *   d_workspace : device scratch, >= CPA_PARAM_DECODE_WORKSPACE_BYTES, 16-byte aligned;
  *                 contents are overwritten; calls sharing one workspace must not overlap.
  * Lengths are read from the device seq_lens, so T steps can be enqueued back to
- * back without host synchronisation.  Errors: CPA_EINVAL, CPA_ESTATE, CPA_ECUDA.
+ * back without host synchronisation.  Errors: CPA_EINVAL, CPA_ESTATE (also: a worker
+ * of a prefix-aware plan has none of its own tokens cached yet), CPA_ECUDA.
  */
 CPA_API int cpa_decode(const cpa_plan* plan, const void* q, const void* k_pool, const void* v_pool,
                void* o, void* d_workspace, void* stream);
@@ -279,6 +357,54 @@ CPA_API int cpa_decode(const cpa_plan* plan, const void* q, const void* k_pool, 
  */
 CPA_API int cpa_decode_append(cpa_plan* plan, const void* q, const void* k_new, const void* v_new, void* k_pool,
                               void* v_pool, void* o, void* d_workspace, void* stream);
+
+/*
+ * cpa_decode_append_dynamic -- cpa_decode_append for a plan with pages on demand (cpa_plan_create_dynamic;
+ * Section 8, "Dynamic block size and prompt selection"), with per-block stop flags that live on the device, so
+ * that summaries of different, unknown lengths need neither a new plan nor a host round trip per step.
+ *   d_active : device int32 [B], or NULL = every block takes part.  Block b decodes in this step iff
+ *              d_active[b] != 0; a block that sits out keeps its length, and its rows of o are not written.
+ * A block whose new token fills a page takes the page for the next one from the reserve inside the launch.  If
+ * the reserve is empty the block stops growing: in its next step it sits out and the status word reads back as
+ * CPA_ENOSPC (cpa_plan_status); nothing is written outside the block's pages.  The host's CPA_ARR_SEQ_LENS counts
+ * a token per call for every block (an upper bound; cpa_plan_sync reads the true lengths), and the call returns
+ * CPA_ENOSPC without launching once that bound would pass L_b + max_new_tokens.  Other arguments, layouts and
+ * errors as for cpa_decode_append; CPA_ESTATE for a plan of another kind.
+ */
+CPA_API int cpa_decode_append_dynamic(cpa_plan* plan, const void* q, const void* k_new, const void* v_new,
+                                      const int32_t* d_active, void* k_pool, void* v_pool, void* o,
+                                      void* d_workspace, void* stream);
+
+/*
+ * cpa_release_blocks -- pages on demand: every block with d_active[b] == 0 that still holds pages gives them back
+ * to the reserve (device int32 [B] flags, as for cpa_decode_append_dynamic; Section 8 as cited there).  A
+ * released block takes part in no later step.  Enqueued on `stream`, ordered against the decode launches of the
+ * same stream.  Errors: CPA_EINVAL, CPA_ESTATE (not uploaded, or a plan of another kind), CPA_ECUDA.
+ */
+CPA_API int cpa_release_blocks(cpa_plan* plan, const int32_t* d_active, void* stream);
+
+/*
+ * cpa_step_mixed -- step `step` of a chunked plan's schedule (cpa_plan_create_chunked; Section 4.2 and
+ * Section 6 of the paper as cited there): the blocks that still have prompt left prefill their next
+ * chunk and cache it, and the blocks whose turn it is decode one token (append fused in), in one call.
+ * The two halves touch different blocks and run side by side: the chunk on a second stream the plan
+ * owns (created at the first such step; no device memory is allocated), the decode on `stream`; the
+ * call's work is complete on `stream` when both are.
+ *   q, k, v, o : the packed tensors of the whole event ([total_tokens, heads, head_dim]); the step reads
+ *                and writes only the rows of its chunks, rows cu_seqlens[b] + [s * chunk, ...) of every
+ *                block that has a chunk s, so later rows need not exist yet.  Row i of a chunk attends
+ *                over the block's cached tokens [0, s * chunk) and the chunk's tokens up to itself:
+ *                exactly the rows cpa_prefill gives.  May be NULL in steps without a chunk.
+ *   q_dec, o_dec       : device bf16 [B, num_q_heads, head_dim]; only the rows of the decoding blocks are
+ *                        read / written.  k_new, v_new: [B, num_kv_heads, head_dim] likewise.  May be
+ *                        NULL in steps in which no block decodes.
+ *   k_pool, v_pool, d_workspace : as for cpa_decode_append
+ * Steps run in order: `step` must be the number of steps run since cpa_plan_upload (CPA_ESTATE
+ * otherwise, and for a plan that is not chunked).  Errors: CPA_EINVAL, CPA_ESTATE, CPA_ECUDA.
+ */
+CPA_API int cpa_step_mixed(cpa_plan* plan, int32_t step, const void* q, const void* k, const void* v, void* o,
+                           const void* q_dec, const void* k_new, const void* v_new, void* o_dec, void* k_pool,
+                           void* v_pool, void* d_workspace, void* stream);
 
 /*
  * cpa_decode_static -- cpa_decode for callers that cannot hand over scratch memory.

@@ -22,6 +22,8 @@ ARR_CU_SEQLENS, ARR_PAGE_INDPTR, ARR_PAGE_INDICES, ARR_SEQ_LENS = 0, 1, 2, 3
 ARR_SLOT_MAPPING, ARR_PREFILL_ITEMS, ARR_DECODE_ITEMS, ARR_SPLIT_INDPTR = 4, 5, 6, 7
 ARR_SPLIT_PAGES = 8
 ARR_PREFILL_SCHED = 9
+ARR_DEC_START, ARR_CHUNK_ROWS = 10, 11
+ARR_PAGES_ASSIGNED, ARR_FREE_RING = 12, 13
 _ARR_WIDTH = {ARR_PREFILL_ITEMS: 2, ARR_DECODE_ITEMS: 3}
 
 PARAM_NUM_BLOCKS, PARAM_TOTAL_TOKENS, PARAM_Q_TILE_ROWS, PARAM_PAGES_PER_SPLIT = 0, 1, 2, 3
@@ -29,6 +31,7 @@ PARAM_PAGES_USED, PARAM_INDEX_BYTES, PARAM_DECODE_WORKSPACE_BYTES, PARAM_TOTAL_S
 PARAM_MAX_NEW_TOKENS = 8
 PARAM_PREFILL_CTAS = 9
 PARAM_SHARED_CHUNK_PAGES = 10
+PARAM_CHUNK_TOKENS, PARAM_NUM_STEPS, PARAM_CHUNK_STEPS, PARAM_DECODE_SMS, PARAM_NUM_SMS = 11, 12, 13, 14, 15
 
 
 class cpa_config(ctypes.Structure):
@@ -57,6 +60,20 @@ _lib.cpa_plan_create.restype = ctypes.c_int
 _lib.cpa_plan_create_prefix.argtypes = [ctypes.POINTER(cpa_config), ctypes.c_int32, _i32p, _i32p, _i32p, ctypes.c_int32,
                                         ctypes.c_int32, _i32p, ctypes.c_int32, ctypes.POINTER(_vp)]
 _lib.cpa_plan_create_prefix.restype = ctypes.c_int
+_lib.cpa_plan_create_chunked.argtypes = [ctypes.POINTER(cpa_config), ctypes.c_int32, _i32p, ctypes.c_int32, ctypes.c_int32,
+                                         ctypes.c_int32, _i32p, ctypes.c_int32, ctypes.POINTER(_vp)]
+_lib.cpa_plan_create_chunked.restype = ctypes.c_int
+_lib.cpa_plan_create_dynamic.argtypes = [ctypes.POINTER(cpa_config), ctypes.c_int32, _i32p, ctypes.c_int32, _i32p,
+                                         ctypes.c_int32, ctypes.POINTER(_vp)]
+_lib.cpa_plan_create_dynamic.restype = ctypes.c_int
+_lib.cpa_plan_sync.argtypes = [_vp, _vp]
+_lib.cpa_plan_sync.restype = ctypes.c_int
+_lib.cpa_decode_append_dynamic.argtypes = [_vp] * 10
+_lib.cpa_decode_append_dynamic.restype = ctypes.c_int
+_lib.cpa_release_blocks.argtypes = [_vp, _vp, _vp]
+_lib.cpa_release_blocks.restype = ctypes.c_int
+_lib.cpa_step_mixed.argtypes = [_vp, ctypes.c_int32] + [_vp] * 12
+_lib.cpa_step_mixed.restype = ctypes.c_int
 _lib.cpa_plan_export.argtypes = [_vp, ctypes.c_int, ctypes.POINTER(_i32p), ctypes.POINTER(ctypes.c_int64)]
 _lib.cpa_plan_export.restype = ctypes.c_int
 _lib.cpa_plan_param.argtypes = [_vp, ctypes.c_int]
@@ -134,6 +151,48 @@ def cpa_plan_create_prefix(cfg: cpa_config, own_lens: Sequence[int], prefix_lens
     return out.value
 
 
+def cpa_plan_create_chunked(cfg: cpa_config, block_lens: Sequence[int], max_new_tokens: int, chunk_tokens: int,
+                            free_pages: Sequence[int], decode_sms: int = 0, check: bool = True):
+    """Plan of an event with chunked prefill; returns the handle, or (status, handle) with check=False."""
+    lens, free = _i32(block_lens), _i32(free_pages)
+    out = _vp()
+    rc = _lib.cpa_plan_create_chunked(ctypes.byref(cfg), lens.shape[0], lens.ctypes.data_as(_i32p), int(max_new_tokens),
+                                      int(chunk_tokens), int(decode_sms), free.ctypes.data_as(_i32p), free.shape[0],
+                                      ctypes.byref(out))
+    if not check:
+        return rc, out.value
+    if rc != CPA_OK:
+        raise CpaError(rc, "cpa_plan_create_chunked")
+    return out.value
+
+
+def cpa_plan_create_dynamic(cfg: cpa_config, block_lens: Sequence[int], max_new_tokens: int,
+                            free_pages: Sequence[int], check: bool = True):
+    """Plan with pages on demand; returns the handle, or (status, handle) with check=False."""
+    lens, free = _i32(block_lens), _i32(free_pages)
+    out = _vp()
+    rc = _lib.cpa_plan_create_dynamic(ctypes.byref(cfg), lens.shape[0], lens.ctypes.data_as(_i32p), int(max_new_tokens),
+                                      free.ctypes.data_as(_i32p), free.shape[0], ctypes.byref(out))
+    if not check:
+        return rc, out.value
+    if rc != CPA_OK:
+        raise CpaError(rc, "cpa_plan_create_dynamic")
+    return out.value
+
+
+def cpa_plan_sync(plan: int, stream: int = 0) -> int:
+    return _lib.cpa_plan_sync(plan, stream or None)
+
+
+def cpa_decode_append_dynamic(plan: int, q, k_new, v_new, d_active, k_pool, v_pool, o, d_workspace, stream: int = 0) -> int:
+    return _lib.cpa_decode_append_dynamic(plan, _ptr(q), _ptr(k_new), _ptr(v_new), _ptr(d_active), _ptr(k_pool),
+                                          _ptr(v_pool), _ptr(o), _ptr(d_workspace), stream or None)
+
+
+def cpa_release_blocks(plan: int, d_active, stream: int = 0) -> int:
+    return _lib.cpa_release_blocks(plan, _ptr(d_active), stream or None)
+
+
 def cpa_plan_export(plan: int, which: int) -> np.ndarray:
     """Copy of one host index array; item lists come back as [n, width]."""
     ptr, n = _i32p(), ctypes.c_int64()
@@ -196,6 +255,12 @@ def cpa_decode(plan: int, q, k_pool, v_pool, o, d_workspace, stream: int = 0) ->
 def cpa_decode_append(plan: int, q, k_new, v_new, k_pool, v_pool, o, d_workspace, stream: int = 0) -> int:
     return _lib.cpa_decode_append(plan, _ptr(q), _ptr(k_new), _ptr(v_new), _ptr(k_pool), _ptr(v_pool), _ptr(o),
                                   _ptr(d_workspace), stream or None)
+
+
+def cpa_step_mixed(plan: int, step: int, q, k, v, o, q_dec, k_new, v_new, o_dec, k_pool, v_pool, d_workspace,
+                   stream: int = 0) -> int:
+    return _lib.cpa_step_mixed(plan, int(step), _ptr(q), _ptr(k), _ptr(v), _ptr(o), _ptr(q_dec), _ptr(k_new),
+                               _ptr(v_new), _ptr(o_dec), _ptr(k_pool), _ptr(v_pool), _ptr(d_workspace), stream or None)
 
 
 STATIC_SCRATCH_BYTES = 16 << 20

@@ -10,6 +10,9 @@ PKG = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(PKG)
 CSRC = os.path.join(PKG, "csrc")
 LIB = os.path.join(PKG, "libcompact_attn.so")
+# test-only probe kernels (the bounded wait running out); a library of its own, never part of the product
+PROBE_SRC = os.path.join(CSRC, "testing", "wait_probe.cu")
+PROBE_LIB = os.path.join(PKG, "libcpa_testprobe.so")
 
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
@@ -23,10 +26,11 @@ def sources():
 
 
 def is_stale() -> bool:
-    if not os.path.exists(LIB):
+    if not os.path.exists(LIB) or not os.path.exists(PROBE_LIB):
         return True
     t = os.path.getmtime(LIB)
-    deps = sources() + glob.glob(os.path.join(CSRC, "*.h")) + glob.glob(os.path.join(ROOT, "include", "*.h"))
+    deps = (sources() + glob.glob(os.path.join(CSRC, "*.h")) + glob.glob(os.path.join(CSRC, "*.cuh")) +
+            glob.glob(os.path.join(ROOT, "include", "*.h")))
     return any(os.path.getmtime(d) > t for d in deps)
 
 
@@ -42,7 +46,20 @@ def build(force: bool = False, verbose: bool = False) -> str:
     cmd += ["-o", tmp] + sources()
     subprocess.run(cmd, check=True)
     os.replace(tmp, LIB)
+    build_probe(force=True)
     return LIB
+
+
+def build_probe(force: bool = False) -> str:
+    """Compile the test-only wait probe into its own shared library."""
+    deps = [PROBE_SRC, os.path.join(CSRC, "cpa_device.cuh")]
+    if not force and os.path.exists(PROBE_LIB) and all(os.path.getmtime(d) <= os.path.getmtime(PROBE_LIB) for d in deps):
+        return PROBE_LIB
+    nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
+    tmp = PROBE_LIB + f".tmp{os.getpid()}"
+    subprocess.run([nvcc] + NVCC_FLAGS + ["-I", CSRC, "-o", tmp, PROBE_SRC], check=True)
+    os.replace(tmp, PROBE_LIB)
+    return PROBE_LIB
 
 
 if __name__ == "__main__":

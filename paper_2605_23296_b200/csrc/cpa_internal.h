@@ -1,6 +1,8 @@
 // Internal definitions shared by the host planner and the kernel launchers.
 #pragma once
 
+#include <cuda_runtime.h>
+
 #include <cstdint>
 #include <vector>
 
@@ -27,12 +29,37 @@ struct cpa_dev_index {
     int32_t shared_chunk;          // pages per chunk of the shared-prefix scan (0: no shared prefix)
     int32_t* merge_tickets;        // [B * Hkv] arrival counters of the fused split merge (zero between launches)
     int32_t item_stride;           // int32 words per decode item: 8 + largest split size rounded up to 4
+    const int32_t* dec_start;      // [B] chunked plans: the step at which a block starts to decode (= its chunk count)
+    // plans with pages on demand: page_indices is a table of B rows (row b holds page_indptr[b+1] - page_indptr[b]
+    // entries, the first pages_assigned[b] of them valid) that the decode kernel extends from the reserve
+    int32_t* page_table;           // page_indices again, writable
+    int32_t* pages_assigned;       // [B]
+    int32_t* ring_ctrl;            // [4]: pops so far (head), pushes so far (tail), ring size
+    int32_t* ring;                 // [ring size] page ids of the reserve; entry i of the sequence of pushes sits at i % size
+};
+
+// Which blocks take part in a decode launch.
+struct cpa_decode_mode {
+    int32_t step;             // >= 0: a step of a chunked plan's schedule, block b decodes iff 0 <= step - dec_start[b] < T;
+                              // -1: every block decodes
+    int32_t T;                // decode steps per block (chunked plans)
+    int32_t dynamic;          // pages on demand: page ids come from the table, a block that fills a page takes the next
+    const int32_t* d_active;  // dynamic plans: device flags [B], block b takes part iff d_active[b] != 0; nullptr: all do
+};
+
+// One step of a chunked plan's prefill: its items, their deal to CTAs, and the rows it appends.
+struct cpa_chunk_step {
+    int64_t off_items = 0;    // [n_items, 4] item records of the step (same format as prefill_items)
+    int64_t off_sched = 0;    // [rounds, ctas]
+    int64_t off_rows = 0;     // [B+1] prefix sums of the rows each block prefills in this step
+    int32_t n_items = 0, ctas = 0, rounds = 0, rows = 0;
 };
 
 struct cpa_plan {
     cpa_config cfg;
     int32_t B = 0;
     int32_t T = 0;          // max_new_tokens
+    int32_t num_sms = 0;    // SM budget of the plan's kernels: cfg.num_sms, or the device's SM count for 0
     int32_t q_tile = 0;     // query rows per prefill item
     int32_t C = 0;          // largest pages-per-split over the blocks
     int64_t total_tokens = 0;
@@ -46,6 +73,21 @@ struct cpa_plan {
     // scan fills, its chunk size in pages, its work items and the shared pages' ids
     std::vector<int32_t> n_fixed, shared_items, shared_page_ids;
     int32_t shared_chunk = 0, n_shared = 0;
+    // chunked prefill: tokens per chunk (0: none), SMs left to the decode wave while a chunk is prefilled,
+    // the step at which each block starts to decode, the per-step prefill work, and the schedule's position
+    int32_t chunk = 0, decode_sms = 0, n_steps = 0, next_step = 0;
+    std::vector<int32_t> dec_start, chunk_rows;   // chunk_rows: [chunk steps][B+1] prefix sums of the rows a step prefills
+    std::vector<cpa_chunk_step> chunk_steps;
+    int64_t off_decstart = 0;
+    // pages on demand: no pages are reserved for the summaries; the reserve lives in a ring in the index buffer
+    bool dynamic = false;
+    std::vector<int32_t> pages_assigned, free_ring;   // host mirrors (as of plan creation or the last cpa_plan_sync)
+    int32_t ring_size = 0;
+    int64_t off_assigned = 0, off_ringctrl = 0, off_ring = 0;
+    // a mixed step runs its prefill chunk beside its decode launch: a second stream and two events, created
+    // at the first mixed step on the device that is current then, destroyed with the plan
+    cudaStream_t side_stream = nullptr;
+    cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
 
     // packed image of the device index buffer (int32 words) and offsets into it
     std::vector<int32_t> image;
@@ -84,10 +126,17 @@ struct cpa_plan {
         d.shared_chunk = shared_chunk;
         d.merge_tickets = d_base + off_tickets;
         d.item_stride = item_stride;
+        d.dec_start = d_base + off_decstart;
+        d.page_table = d_base + off_pidx;
+        d.pages_assigned = d_base + off_assigned;
+        d.ring_ctrl = d_base + off_ringctrl;
+        d.ring = d_base + off_ring;
         return d;
     }
 };
 
+// largest SM budget a plan takes (the schedule's sort keys hold a CTA id in 12 bits)
+constexpr int32_t kMaxPlanSms = 4095;
 // largest pages-per-split the planner produces: the decode kernel parks a split's page ids in shared memory
 constexpr int32_t kMaxSplitPages = 1024;
 // Which kernel scans the shared pages in the decode of the prefix-aware layout: the tensor-core one takes
@@ -114,3 +163,14 @@ static inline bool cpa_aligned16(const void* p) { return (reinterpret_cast<uintp
 // (worker, head) row for every chunk of shared pages go to part_ml / part_o.
 int cpa_scan_tc(const cpa_plan* plan, const void* q, const void* k_pool, const void* v_pool, float* part_ml,
                 float* part_o, void* stream);
+
+// The tensor-core prefill over an explicit work list (a chunk step's items and deal); `items`, `sched` are device
+// pointers into the index buffer.  cpa_prefill_tc runs the plan's whole-block list.
+int cpa_prefill_tc_list(const cpa_plan* plan, const void* q, const void* k, const void* v, void* o, const void* k_pool,
+                        const void* v_pool, const int32_t* items, const int32_t* sched, int ctas, int rounds, void* stream);
+// One chunk step's append: rows [step * chunk, ...) of every block that has them go to the pools; every block that
+// does not decode in this step gets its length carried into the other length buffer.
+int cpa_append_chunk(cpa_plan* plan, int step, const void* k, const void* v, void* k_pool, void* v_pool, void* stream);
+// One decode launch (append fused in when k_new is given) over the blocks `mode` selects.
+int cpa_decode_launch(const cpa_plan* plan, const void* q, const void* k_new, const void* v_new, void* k_pool,
+                      void* v_pool, void* o, void* ws, cpa_decode_mode mode, int wave_sms, void* stream);

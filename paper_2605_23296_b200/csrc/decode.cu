@@ -18,10 +18,12 @@
 // thread reads whole 16-byte chunks from the staged page and pairs registers up as
 // the MMA fragments need them; no transposes, no ldmatrix.
 #include <algorithm>
+#include <atomic>
 
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 
+#include "cpa_device.cuh"
 #include "cpa_internal.h"
 
 namespace {
@@ -30,6 +32,7 @@ constexpr int kDecodeWarps = 4;
 constexpr int kDecodeThreads = kDecodeWarps * 32;
 constexpr int kDecodeSmemBytes = 64 * 1024;          // stage rings of the four warps (three CTAs per SM)
 constexpr uint32_t kSpinLimit = 1u << 18;            // bounded mbarrier wait (each try suspends briefly)
+constexpr uint32_t kDrainLimit = 1u << 12;           // last look at a copy in flight after a wait gave up
 
 __device__ __forceinline__ void mma_bf16_16816(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
                                                uint32_t b0, uint32_t b1) {
@@ -54,19 +57,6 @@ __device__ __forceinline__ uint32_t sel(const uint4& v, int i) {
     return i == 0 ? v.x : i == 1 ? v.y : i == 2 ? v.z : v.w;
 }
 
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;\n" :: "r"(bar), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;\n" :: "r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity) {
-    uint32_t ok;
-    asm volatile(
-        "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}\n"
-        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-    return ok;
-}
 // Contiguous global -> shared copy; both addresses 16-byte aligned, size a multiple of 16.
 __device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];\n"
@@ -99,7 +89,8 @@ __global__ void __launch_bounds__(kDecodeThreads, 3)
 decode_split_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ k_pool,
                     const __nv_bfloat16* __restrict__ v_pool, float* __restrict__ part_ml,
                     float* __restrict__ part_o, __nv_bfloat16* __restrict__ out, cpa_dev_index ix, int Hq,
-                    int Hkv, int G, float scale_log2, int reverse, cpa_fused_append fa, int n_items, int late_wait) {
+                    int Hkv, int G, float scale_log2, int reverse, cpa_fused_append fa, int n_items, int late_wait,
+                    cpa_decode_mode mode) {
     constexpr int P = 16;
     constexpr int KC = D / 32;  // 16-byte K chunks per thread per 8-key group
     constexpr int VC = D / 64;  // 16-byte V chunks per thread per key row
@@ -134,10 +125,18 @@ decode_split_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __
     const int32_t* item = ix.decode_items + (int64_t)item_idx * ix.item_stride;
     const int4 hdr = *reinterpret_cast<const int4*>(item);
     const int b = hdr.x, g = hdr.y, s = hdr.z, n_reserved = hdr.w;
+    // A step of a chunked plan: only the blocks whose turn it is decode; the others sit the step out (their
+    // lengths are carried over by the step's length kernel, their output rows are not touched).
+    if (mode.step >= 0 && (unsigned)(mode.step - __ldg(ix.dec_start + b)) >= (unsigned)mode.T) continue;
     const int C = item[4];  // pages per split of this block
-    // this warp's pages are warp, warp+4, ... of the split: park their ids in shared memory
-    for (int j = lane; warp + kDecodeWarps * j < n_reserved; j += 32)
-        sm_pages[warp][j] = item[8 + warp + kDecodeWarps * j];
+    const int first = item[5];           // first page of the split inside the block's page list
+    const int slot = item[6];            // its partial slot among the block's slots
+    const int n_fixed = item[7];         // slots in front that the shared-prefix scan has filled
+    // this warp's pages are warp, warp+4, ... of the split: park their ids in shared memory (the item record
+    // carries them; a plan with pages on demand reads them from the page table further down)
+    if (!mode.dynamic)
+        for (int j = lane; warp + kDecodeWarps * j < n_reserved; j += 32)
+            sm_pages[warp][j] = item[8 + warp + kDecodeWarps * j];
     // Everything above reads plan constants only.  The launch may have started while the
     // previous kernel in the stream (normally the step's append) was still running; from here
     // on its writes (cached length, the new K/V row) are needed, so wait for it to finish.
@@ -151,12 +150,30 @@ decode_split_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __
     // a length that already moved.
     const bool fused = fa.k_new != nullptr;
     const int len_old = ix.seq_lens[b];
+    if (mode.dynamic) {
+        // Pages on demand.  A block takes part unless the caller's flag says it has stopped.  The page its new
+        // token goes to was taken from the reserve when the page before it filled up; if the reserve was empty
+        // then, the block cannot grow: it sits the step out and the status word says why.  The first CTA of a
+        // block that sits out carries its length over.
+        const bool idle = mode.d_active != nullptr && mode.d_active[b] == 0;
+        const bool no_room = !idle && fused && len_old / P >= ix.pages_assigned[b];
+        if (idle || no_room) {
+            if (fused && g == 0 && s == 0 && threadIdx.x == 0) {
+                ix.seq_lens_next[b] = len_old;
+                if (no_room) atomicCAS(ix.status, 0, kStatusNoSpace);
+            }
+            continue;
+        }
+    }
     const int len = len_old + (fused ? 1 : 0);
     __syncwarp();
     const int pages_active = (len + P - 1) / P;
-    const int first = item[5];           // first page of the split inside the block's page list
-    const int slot = item[6];            // its partial slot among the block's slots
-    const int n_fixed = item[7];         // slots in front that the shared-prefix scan has filled
+    if (mode.dynamic) {   // the ids of the pages that hold keys, from the block's row of the page table
+        const int32_t* row = ix.page_indices + ix.page_indptr[b] + first;
+        for (int j = lane; warp + kDecodeWarps * j < n_reserved && first + warp + kDecodeWarps * j < pages_active; j += 32)
+            sm_pages[warp][j] = row[warp + kDecodeWarps * j];
+        __syncwarp();
+    }
     const int pg_new = fused ? len_old / P : -1;   // page (inside the block) of the new token
     const bool owner = fused && pg_new >= first && pg_new < first + n_reserved;
     uint4 new_chunk = make_uint4(0, 0, 0, 0);      // lanes 0-15: a 16-byte piece of the K row, 16-31: of the V row
@@ -170,7 +187,24 @@ decode_split_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __
                                  (((page * Hkv + g) * P) + (len_old % P)) * D + cpa_pool_piece(piece, len_old % P) * 8;
             *reinterpret_cast<uint4*>(dst) = new_chunk;
         }
-        if (g == 0 && lane == 0) ix.seq_lens_next[b] = len;
+        if (g == 0 && lane == 0) {
+            ix.seq_lens_next[b] = len;
+            if (mode.dynamic && len % P == 0) {
+                // this token filled its page: take the page of the next one from the reserve now, so that every
+                // CTA of the next launch finds it in the table (pushes happen in other launches only, so the
+                // count of pushes is a constant here)
+                const int next_pg = len / P, cap = ix.page_indptr[b + 1] - ix.page_indptr[b];
+                if (next_pg < cap) {
+                    const int h = atomicAdd(ix.ring_ctrl, 1);
+                    if (h < ix.ring_ctrl[1]) {
+                        ix.page_table[ix.page_indptr[b] + next_pg] = ix.ring[h % ix.ring_ctrl[2]];
+                        ix.pages_assigned[b] = next_pg + 1;
+                    } else {
+                        atomicSub(ix.ring_ctrl, 1);   // the reserve is empty: the block's next step will say so
+                    }
+                }
+            }
+        }
     }
     const int n_active = min(n_reserved, pages_active - first);  // pages of this split that hold keys
     if (n_active <= 0) continue;  // split lies beyond the cached length (uniform per CTA)
@@ -217,11 +251,16 @@ decode_split_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __
         const int st = (ring_pos + i) % STAGES;
         const uint32_t parity = (uint32_t)((ring_pos + i) / STAGES) & 1u;
         const int pg = first + warp + kDecodeWarps * local_index(i);  // page index inside the block
-        if (!gave_up) {
-            uint32_t spins = 0;
-            while (!mbar_try_wait(bar0 + 8 * st, parity)) {
-                if (++spins > kSpinLimit) { gave_up = true; atomicCAS(ix.status, 0, 1); break; }
-            }
+        mbar_wait(bar0 + 8 * st, parity, gave_up, ix.status, kSpinLimit);
+        if (__any_sync(0xffffffffu, gave_up)) {
+            // The page never arrived: nothing more is issued, and the copies still on their way into
+            // this warp's stages (pages i .. i + STAGES - 1) get one last bounded look, so that the CTA
+            // does not end under a copy in flight.  The CTA returns below; the status word says why.
+            gave_up = true;
+            if (lane == 0)
+                for (int k2 = i; k2 < n_mine && k2 < i + STAGES; ++k2)
+                    mbar_drain(bar0 + 8 * ((ring_pos + k2) % STAGES), (uint32_t)((ring_pos + k2) / STAGES) & 1u, kDrainLimit);
+            break;
         }
         const uint32_t ks = ring + st * kStageBytes;
         const uint32_t vs = ks + kChunkBytes;
@@ -311,7 +350,7 @@ decode_split_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __
     l_run += __shfl_xor_sync(0xffffffffu, l_run, 2);
 
     // ---- merge the four warps; the stage rings are idle now (every issued copy was consumed)
-    __syncthreads();
+    if (__syncthreads_or((int)gave_up)) return;   // a wait gave up: no copy is in flight any more, results are void
     float (*sm_o)[8][D + 4] = reinterpret_cast<float (*)[8][D + 4]>(dsm);
     if (tig == 0) { sm_m[warp][gid] = m_run * scale_log2; sm_l[warp][gid] = l_run; }
 #pragma unroll
@@ -490,8 +529,9 @@ decode_shared_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* _
         bulk_load(dst, k_pool + src, kChunkBytes, full0 + 8 * st);
         bulk_load(dst + kChunkBytes, v_pool + src, kChunkBytes, full0 + 8 * st);
     };
+    int n_issued = 0;   // pages handed to the copy engine so far (thread 0)
     if (threadIdx.x == 0)
-        for (int i = 0; i < STAGES && i < n_pages; ++i) issue(i);
+        for (int i = 0; i < STAGES && i < n_pages; ++i) { issue(i); n_issued = i + 1; }
 
     // -------------------------------------------------------------------- compute warps
     // rows of this thread: A = 16*warp + gid, B = A + 8 (row = worker * G + head inside the group)
@@ -534,22 +574,13 @@ decode_shared_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* _
             // refill: page j takes the stage of page j - STAGES, which every warp must have released
             const int j = i + STAGES - kSharedLag;
             if (j >= STAGES && j < n_pages) {
-                if (!gave_up) {
-                    uint32_t spins = 0;
-                    while (!mbar_try_wait(empty0 + 8 * (j % STAGES), ((uint32_t)(j / STAGES) & 1u) ^ 1u)) {
-                        if (++spins > kSpinLimit) { gave_up = true; atomicCAS(ix.status, 0, 1); break; }
-                    }
-                }
-                if (!gave_up) issue(j);
+                mbar_wait(empty0 + 8 * (j % STAGES), ((uint32_t)(j / STAGES) & 1u) ^ 1u, gave_up, ix.status, kSpinLimit);
+                if (!gave_up) { issue(j); n_issued = j + 1; }
             }
         }
         gave_up = __shfl_sync(0xffffffffu, gave_up, 0) || gave_up;
-        if (!gave_up) {
-            uint32_t spins = 0;
-            while (!mbar_try_wait(full0 + 8 * st, parity)) {
-                if (++spins > kSpinLimit) { gave_up = true; atomicCAS(ix.status, 0, 1); break; }
-            }
-        }
+        mbar_wait(full0 + 8 * st, parity, gave_up, ix.status, kSpinLimit);
+        if (__any_sync(0xffffffffu, gave_up)) { gave_up = true; break; }   // stop consuming; the CTA drains and returns below
         if ((first + i) * P >= vis_warp) {
             // Nothing on this page for this warp's rows.  It still waits for the page before it releases
             // the stage: a warp that ran ahead would add its releases of later pages to the current
@@ -646,7 +677,14 @@ decode_shared_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* _
         l_run[r] += __shfl_xor_sync(0xffffffffu, l_run[r], 2);
     }
     // ---- partials: slot `chunk` of every worker whose prefix reaches into the chunk
-    if (gave_up) return;
+    if (__syncthreads_or((int)gave_up)) {
+        // a wait gave up: the copies of the last pages issued may still be on their way into the ring;
+        // thread 0 gives each one last bounded look, so that no copy is in flight when the CTA ends
+        if (threadIdx.x == 0)
+            for (int j = max(0, n_issued - STAGES); j < n_issued; ++j)
+                mbar_drain(full0 + 8 * (j % STAGES), (uint32_t)(j / STAGES) & 1u, kDrainLimit);
+        return;
+    }
 #pragma unroll
     for (int r = 0; r < 2; ++r) {
         const int row = 16 * warp + gid + 8 * r;
@@ -683,7 +721,9 @@ __global__ void decode_empty_rows_kernel(__nv_bfloat16* __restrict__ out, cpa_de
 
 template <int D>
 int launch_decode(const cpa_plan* plan, const void* q, const void* k_pool, const void* v_pool, void* o,
-                  void* ws, cudaStream_t st, cpa_fused_append fa = cpa_fused_append{nullptr, nullptr, nullptr, nullptr}) {
+                  void* ws, cudaStream_t st, cpa_fused_append fa = cpa_fused_append{nullptr, nullptr, nullptr, nullptr},
+                  cpa_decode_mode mode = cpa_decode_mode{-1, 0, 0, nullptr}, int wave_sms = 0) {
+    if (plan->dynamic) mode.dynamic = 1;
     const cpa_config& c = plan->cfg;
     const int G = c.num_q_heads / c.num_kv_heads;
     const cpa_dev_index ix = plan->dev();
@@ -691,15 +731,22 @@ int launch_decode(const cpa_plan* plan, const void* q, const void* k_pool, const
     float* part_o = part_ml + ((int64_t)plan->split_indptr[plan->B] * c.num_q_heads * 2 + 3) / 4 * 4;
     const float scale_log2 = c.scale * 1.4426950408889634f;
     bool any_empty = false;  // host mirror of the cached lengths
-    for (int b = 0; b < plan->B; ++b) any_empty |= plan->seq_lens[b] == 0;
-    static bool configured_dev[64] = {};  // the attribute is per device: remember which devices have it
+    for (int b = 0; b < plan->B && mode.step < 0; ++b) {   // (in a chunked plan's step the schedule says who decodes)
+        any_empty |= plan->seq_lens[b] == 0;
+        // A worker of the prefix-aware layout that has cached none of its own tokens yet has no own split to
+        // run the merge of the shared scan's partials: the own tokens are appended before the first decode.
+        if (plan->prefix_lens[b] > 0 && plan->seq_lens[b] == plan->prefix_lens[b]) return CPA_ESTATE;
+    }
+    // the attribute is per device: remember which devices have it (setting it twice is harmless, so a
+    // relaxed flag is enough when several host threads arrive together)
+    static std::atomic<bool> configured_dev[64];
     int dev_id = 0;
     if (cudaGetDevice(&dev_id) != cudaSuccess || dev_id < 0 || dev_id >= 64) {
         (void)cudaGetLastError();
         return CPA_ECUDA;
     }
-    bool& configured = configured_dev[dev_id];
-    if (!configured) {
+    std::atomic<bool>& configured = configured_dev[dev_id];
+    if (!configured.load(std::memory_order_relaxed)) {
         if (cudaFuncSetAttribute(decode_split_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  kDecodeSmemBytes) != cudaSuccess ||
             cudaFuncSetAttribute(decode_shared_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -707,7 +754,7 @@ int launch_decode(const cpa_plan* plan, const void* q, const void* k_pool, const
             (void)cudaGetLastError();
             return CPA_ECUDA;
         }
-        configured = true;
+        configured.store(true, std::memory_order_relaxed);
     }
     if (any_empty)
         decode_empty_rows_kernel<<<plan->B, 128, 0, st>>>((__nv_bfloat16*)o, ix, plan->B, c.num_q_heads * D);
@@ -727,7 +774,7 @@ int launch_decode(const cpa_plan* plan, const void* q, const void* k_pool, const
     // stream drains; the kernel itself waits (griddepcontrol.wait) before it reads anything
     // that kernel wrote.
     cudaLaunchConfig_t cfg = {};
-    const int slots = 3 * (c.num_sms ? c.num_sms : 148);   // resident CTAs: three per SM
+    const int slots = 3 * (wave_sms > 0 ? wave_sms : plan->num_sms);   // resident CTAs: three per SM
     cfg.gridDim = dim3(std::min(plan->n_decode, slots));
     cfg.blockDim = dim3(kDecodeThreads);
     cfg.dynamicSmemBytes = kDecodeSmemBytes;
@@ -741,7 +788,7 @@ int launch_decode(const cpa_plan* plan, const void* q, const void* k_pool, const
                                        (const __nv_bfloat16*)k_pool, (const __nv_bfloat16*)v_pool, part_ml, part_o,
                                        (__nv_bfloat16*)o, ix, (int)c.num_q_heads, (int)c.num_kv_heads, G, scale_log2,
                                        (int)(plan->decode_calls++ & 1), fa, (int)plan->n_decode,
-                                       (int)(plan->n_shared > 0));
+                                       (int)(plan->n_shared > 0), mode);
     if (e != cudaSuccess) { (void)cudaGetLastError(); return CPA_ECUDA; }
     return cudaGetLastError() == cudaSuccess ? CPA_OK : CPA_ECUDA;
 }
@@ -749,9 +796,19 @@ int launch_decode(const cpa_plan* plan, const void* q, const void* k_pool, const
 // Scratch for cpa_decode_static: lives in the library image, so every GPU that loads the
 // library holds these bytes until the process exits.
 constexpr int64_t kStaticScratchBytes = 16ll << 20;
+static_assert(kStaticScratchBytes == CPA_STATIC_SCRATCH_BYTES, "the header promises this size");
 static __device__ __align__(256) unsigned char g_static_decode_scratch[kStaticScratchBytes];
 
 }  // namespace
+
+int cpa_decode_launch(const cpa_plan* plan, const void* q, const void* k_new, const void* v_new, void* k_pool,
+                      void* v_pool, void* o, void* ws, cpa_decode_mode mode, int wave_sms, void* stream) {
+    cpa_fused_append fa{(const __nv_bfloat16*)k_new, (const __nv_bfloat16*)v_new, (__nv_bfloat16*)k_pool,
+                        (__nv_bfloat16*)v_pool};
+    cudaStream_t st = (cudaStream_t)stream;
+    return plan->cfg.head_dim == 128 ? launch_decode<128>(plan, q, k_pool, v_pool, o, ws, st, fa, mode, wave_sms)
+                                     : launch_decode<64>(plan, q, k_pool, v_pool, o, ws, st, fa, mode, wave_sms);
+}
 
 extern "C" int cpa_decode(const cpa_plan* plan, const void* q, const void* k_pool, const void* v_pool, void* o,
                           void* d_workspace, void* stream) {
@@ -775,23 +832,24 @@ extern "C" int cpa_decode_static(const cpa_plan* plan, const void* q, const void
     // In host code the array's name is only a handle; its device address has to be asked for,
     // once per device, with that device current.
     constexpr int kMaxDevices = 64;
-    static void* scratch_addr[kMaxDevices] = {};
+    // the address is the same for every thread that looks it up, so a relaxed atomic slot per device is enough
+    static std::atomic<void*> scratch_addr[kMaxDevices];
     int dev = -1;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) {
         (void)cudaGetLastError();
         return CPA_ECUDA;
     }
-    if (!scratch_addr[dev]) {
-        void* p = nullptr;
-        if (cudaGetSymbolAddress(&p, g_static_decode_scratch) != cudaSuccess || !p) {
+    void* scratch = scratch_addr[dev].load(std::memory_order_relaxed);
+    if (!scratch) {
+        if (cudaGetSymbolAddress(&scratch, g_static_decode_scratch) != cudaSuccess || !scratch) {
             (void)cudaGetLastError();
             return CPA_ECUDA;
         }
-        scratch_addr[dev] = p;
+        scratch_addr[dev].store(scratch, std::memory_order_relaxed);
     }
     cudaStream_t st = (cudaStream_t)stream;
-    return plan->cfg.head_dim == 128 ? launch_decode<128>(plan, q, k_pool, v_pool, o, scratch_addr[dev], st)
-                                     : launch_decode<64>(plan, q, k_pool, v_pool, o, scratch_addr[dev], st);
+    return plan->cfg.head_dim == 128 ? launch_decode<128>(plan, q, k_pool, v_pool, o, scratch, st)
+                                     : launch_decode<64>(plan, q, k_pool, v_pool, o, scratch, st);
 }
 
 extern "C" int cpa_decode_append(cpa_plan* plan, const void* q, const void* k_new, const void* v_new, void* k_pool,
@@ -817,5 +875,28 @@ extern "C" int cpa_decode_append(cpa_plan* plan, const void* q, const void* k_ne
         return rc;
     }
     plan->cur_lens ^= 1;   // the other buffer now holds the lengths
+    return CPA_OK;
+}
+
+extern "C" int cpa_decode_append_dynamic(cpa_plan* plan, const void* q, const void* k_new, const void* v_new,
+                                         const int32_t* d_active, void* k_pool, void* v_pool, void* o,
+                                         void* d_workspace, void* stream) {
+    if (!plan || !q || !k_new || !v_new || !k_pool || !v_pool || !o || !d_workspace) return CPA_EINVAL;
+    if (!cpa_aligned16(q) || !cpa_aligned16(k_new) || !cpa_aligned16(v_new) || !cpa_aligned16(k_pool) ||
+        !cpa_aligned16(v_pool) || !cpa_aligned16(o) || !cpa_aligned16(d_workspace) || (reinterpret_cast<uintptr_t>(d_active) & 3u))
+        return CPA_EINVAL;
+    if (!plan->d_base || !plan->dynamic) return CPA_ESTATE;
+    // The host mirror counts a token for every block, stopped or not (the flags live on the device): it is an upper
+    // bound of the true lengths, which is what the capacity check needs.  cpa_plan_sync reads the true ones back.
+    for (int b = 0; b < plan->B; ++b)
+        if ((int64_t)plan->seq_lens[b] + 1 > (int64_t)plan->block_lens[b] + plan->T) return CPA_ENOSPC;
+    for (int b = 0; b < plan->B; ++b) plan->seq_lens[b] += 1;
+    const int rc = cpa_decode_launch(plan, q, k_new, v_new, k_pool, v_pool, o, d_workspace,
+                                     cpa_decode_mode{-1, 0, 1, d_active}, 0, stream);
+    if (rc != CPA_OK) {
+        for (int b = 0; b < plan->B; ++b) plan->seq_lens[b] -= 1;
+        return rc;
+    }
+    plan->cur_lens ^= 1;
     return CPA_OK;
 }

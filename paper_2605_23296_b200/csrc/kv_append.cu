@@ -2,6 +2,7 @@
 // the per-block cached length.  Pure data movement (bit-exact), bound by HBM.
 #include <cuda_runtime.h>
 
+#include "cpa_device.cuh"
 #include "cpa_internal.h"
 
 namespace {
@@ -33,7 +34,7 @@ __global__ void kv_append_step_kernel(const uint4* __restrict__ k_new, const uin
     const int capacity = (ix.page_indptr[b + 1] - ix.page_indptr[b]) * P;
     __syncthreads();  // every thread has read the length before thread 0 advances it
     if (pos >= capacity) {  // host checks make this unreachable; never write outside the block's pages
-        if (threadIdx.x == 0) atomicCAS(ix.status, 0, 2);
+        if (threadIdx.x == 0) atomicCAS(ix.status, 0, kStatusNoSpace);
         return;
     }
     const int64_t page = ix.page_indices[ix.page_indptr[b] + pos / P];
@@ -60,6 +61,55 @@ __global__ void kv_append_bulk_kernel(const uint4* __restrict__ k_new, const uin
         const int64_t row = r * Hkv * chunks_per_head;
         copy_row_chunks(k_new + row, v_new + row, k_pool, v_pool, page, pos % P, Hkv, chunks_per_head, P);
     }
+}
+
+// Chunk step of a chunked prefill: `rows` tokens, block-major; rows_indptr[b] is the first row of block b's
+// chunk, whose tokens are positions first_pos .. of the block (its earlier chunks are cached already), read
+// from rows cu_seqlens[b] + first_pos .. of the packed tensors.
+__global__ void kv_append_chunk_kernel(const uint4* __restrict__ k, const uint4* __restrict__ v,
+                                       uint4* __restrict__ k_pool, uint4* __restrict__ v_pool, cpa_dev_index ix,
+                                       const int32_t* __restrict__ rows_indptr, int B, int rows, int first_pos,
+                                       int Hkv, int chunks_per_head, int P) {
+    for (int r = blockIdx.x; r < rows; r += gridDim.x) {
+        int lo = 0, hi = B - 1;   // block that owns row r: last b with rows_indptr[b] <= r
+        while (lo < hi) {
+            const int mid = (lo + hi + 1) >> 1;
+            if (rows_indptr[mid] <= r) lo = mid; else hi = mid - 1;
+        }
+        const int b = lo;
+        const int pos = first_pos + (r - rows_indptr[b]);
+        const int64_t page = ix.page_indices[ix.page_indptr[b] + pos / P];
+        const int64_t row = ((int64_t)ix.cu_seqlens[b] + pos) * Hkv * chunks_per_head;
+        copy_row_chunks(k + row, v + row, k_pool, v_pool, page, pos % P, Hkv, chunks_per_head, P);
+    }
+}
+
+// Lengths after a step of a chunked plan, for every block that does not decode in it (the decode launch
+// writes the others): a block with a chunk in this step has cached it, the rest keep their length.  Reads
+// the current length buffer, writes the other one.
+__global__ void chunk_lengths_kernel(cpa_dev_index ix, const int32_t* __restrict__ rows_indptr, int B, int step, int T) {
+    const int b = blockIdx.x * blockDim.x + threadIdx.x;
+    if (b >= B) return;
+    const int d = step - ix.dec_start[b];
+    if (d >= 0 && d < T) return;   // decodes in this step
+    ix.seq_lens_next[b] = ix.seq_lens[b] + (rows_indptr ? rows_indptr[b + 1] - rows_indptr[b] : 0);
+}
+
+// Pages on demand: a block whose flag says it has stopped gives its pages back to the reserve.  One CTA per
+// block; pops happen in decode launches only, which are ordered against this one by the stream.
+__global__ void release_pages_kernel(cpa_dev_index ix, const int32_t* __restrict__ d_active, int B) {
+    __shared__ int base;
+    const int b = blockIdx.x;
+    if (b >= B || d_active[b] != 0) return;
+    const int n = ix.pages_assigned[b];
+    if (n == 0) return;
+    if (threadIdx.x == 0) base = atomicAdd(ix.ring_ctrl + 1, n);
+    __syncthreads();
+    const int size = ix.ring_ctrl[2];
+    const int32_t* row = ix.page_indices + ix.page_indptr[b];
+    for (int i = threadIdx.x; i < n; i += blockDim.x) ix.ring[(base + i) % size] = row[i];
+    __syncthreads();
+    if (threadIdx.x == 0) ix.pages_assigned[b] = 0;
 }
 
 __global__ void seq_lens_advance_kernel(cpa_dev_index ix, const int32_t* __restrict__ src_indptr, int B) {
@@ -91,6 +141,9 @@ extern "C" int cpa_kv_append(cpa_plan* plan, const void* k_new, const void* v_ne
         rows += n;
     }
     if (rows == 0) return CPA_OK;
+    // a single-token append does not take pages from the reserve: plans with pages on demand append inside the
+    // decode launch (cpa_decode_append, cpa_decode_append_dynamic)
+    if (plan->dynamic && !new_lens) return CPA_EUNSUPPORTED;
 
     const int threads = std::min(256, std::max(32, (Hkv * chunks_per_head + 31) / 32 * 32));
     if (!new_lens) {
@@ -108,7 +161,7 @@ extern "C" int cpa_kv_append(cpa_plan* plan, const void* k_new, const void* v_ne
             }
             src_indptr = ix.append_indptr;
         }
-        const int grid = (int)std::min<int64_t>(rows, 148 * 32);
+        const int grid = (int)std::min<int64_t>(rows, (int64_t)plan->num_sms * 32);
         kv_append_bulk_kernel<<<grid, threads, 0, st>>>((const uint4*)k_new, (const uint4*)v_new, (uint4*)k_pool,
                                                         (uint4*)v_pool, ix, src_indptr, B, rows, Hkv,
                                                         chunks_per_head, P);
@@ -117,4 +170,30 @@ extern "C" int cpa_kv_append(cpa_plan* plan, const void* k_new, const void* v_ne
     if (cudaGetLastError() != cudaSuccess) return CPA_ECUDA;
     for (int b = 0; b < B; ++b) plan->seq_lens[b] += new_lens ? new_lens[b] : 1;
     return CPA_OK;
+}
+
+int cpa_append_chunk(cpa_plan* plan, int step, const void* k, const void* v, void* k_pool, void* v_pool, void* stream) {
+    const int B = plan->B, P = plan->cfg.page_size, Hkv = plan->cfg.num_kv_heads;
+    const int chunks_per_head = plan->cfg.head_dim / 8;
+    cudaStream_t st = (cudaStream_t)stream;
+    const cpa_dev_index ix = plan->dev();
+    const int32_t* rows_indptr = nullptr;
+    if (step < (int)plan->chunk_steps.size()) {
+        const cpa_chunk_step& cs = plan->chunk_steps[(size_t)step];
+        rows_indptr = plan->d_base + cs.off_rows;
+        const int threads = std::min(256, std::max(32, (Hkv * chunks_per_head + 31) / 32 * 32));
+        const int grid = (int)std::min<int64_t>(cs.rows, (int64_t)plan->num_sms * 32);
+        kv_append_chunk_kernel<<<grid, threads, 0, st>>>((const uint4*)k, (const uint4*)v, (uint4*)k_pool, (uint4*)v_pool,
+                                                         ix, rows_indptr, B, cs.rows, step * plan->chunk, Hkv,
+                                                         chunks_per_head, P);
+    }
+    chunk_lengths_kernel<<<(B + 127) / 128, 128, 0, st>>>(ix, rows_indptr, B, step, plan->T);
+    return cudaGetLastError() == cudaSuccess ? CPA_OK : CPA_ECUDA;
+}
+
+extern "C" int cpa_release_blocks(cpa_plan* plan, const int32_t* d_active, void* stream) {
+    if (!plan || !d_active || (reinterpret_cast<uintptr_t>(d_active) & 3u)) return CPA_EINVAL;
+    if (!plan->d_base || !plan->dynamic) return CPA_ESTATE;
+    release_pages_kernel<<<plan->B, 128, 0, (cudaStream_t)stream>>>(plan->dev(), d_active, plan->B);
+    return cudaGetLastError() == cudaSuccess ? CPA_OK : CPA_ECUDA;
 }

@@ -15,6 +15,58 @@ namespace {
 
 int64_t align4(int64_t words) { return (words + 3) / 4 * 4; }  // 16-byte alignment of every array
 
+// SM count of the current device; 148 (a B200) when no device can be asked, so that plans can be
+// built and compared on a host without one.
+int32_t device_sm_count() {
+    int dev = 0, sms = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms < 1) {
+        (void)cudaGetLastError();
+        return 148;
+    }
+    return sms;
+}
+
+// Deal of prefill units to the CTAs of the persistent kernel (one CTA per SM).  A unit is (item, query
+// head).  Units are listed kv head by kv head, inside a kv head in item order, the G query heads of
+// the group side by side: CTAs that run at the same time then stream the same few K/V ranges, which
+// stay in L2.  The list is dealt in rounds of one unit per CTA: in every round the CTAs are ranked by
+// the work they have so far (least first, ties to the lower CTA), the round's units by cost (largest
+// first, ties in list order), and the i-th unit goes to the i-th CTA.  `item_cost[i]` is the cost of
+// every unit of item i.  Returns the table [rounds][ctas] (-1 = none) and sets ctas / rounds.
+std::vector<int32_t> deal_prefill_units(const std::vector<int32_t>& item_cost, int32_t Hq, int32_t G, int32_t max_ctas,
+                                        int32_t* ctas_out, int32_t* rounds_out) {
+    const int32_t n_items = (int32_t)item_cost.size();
+    const int64_t n_units = (int64_t)n_items * Hq;
+    const int32_t ctas = (int32_t)std::max<int64_t>(1, std::min<int64_t>(max_ctas, n_units));
+    const int32_t rounds = (int32_t)((n_units + ctas - 1) / ctas);
+    *ctas_out = ctas;
+    *rounds_out = rounds;
+    std::vector<int32_t> sched((size_t)rounds * (size_t)ctas, -1);
+    std::vector<int64_t> load((size_t)ctas, 0);
+    std::vector<uint64_t> rank((size_t)ctas), batch((size_t)ctas);   // packed sort keys
+    const int64_t per_head = (int64_t)n_items * G;                    // units of one kv head
+    for (int32_t r = 0; r < rounds; ++r) {
+        const int64_t u0 = (int64_t)r * ctas, n = std::min<int64_t>(ctas, n_units - u0);
+        for (int64_t j = 0; j < n; ++j) {
+            // unit u0 + j of the list -> (kv head, item, head inside the group)
+            const int64_t u = u0 + j, g = u / per_head, rem = u - g * per_head;
+            const int32_t i = (int32_t)(rem / G), h = (int32_t)(rem - (int64_t)i * G);
+            // descending cost, then list order: the position j breaks ties
+            batch[(size_t)j] = ((uint64_t)(0xFFFFFu - (uint32_t)item_cost[(size_t)i]) << 44) | ((uint64_t)j << 32) |
+                               (uint32_t)(i * Hq + (int32_t)g * G + h);
+        }
+        std::sort(batch.begin(), batch.begin() + n);
+        for (int32_t c = 0; c < ctas; ++c) rank[(size_t)c] = ((uint64_t)load[(size_t)c] << 16) | (uint32_t)c;
+        std::sort(rank.begin(), rank.end());
+        for (int64_t j = 0; j < n; ++j) {
+            const int32_t c = (int32_t)(rank[(size_t)j] & 0xFFFFu);
+            sched[(size_t)r * (size_t)ctas + (size_t)c] = (int32_t)(batch[(size_t)j] & 0xFFFFFFFFu);
+            load[(size_t)c] += 0xFFFFF - (int64_t)(batch[(size_t)j] >> 44);
+        }
+    }
+    return sched;
+}
 
 }  // namespace
 
@@ -22,7 +74,7 @@ namespace {
 // Both layouts: `prefix_lens` == nullptr is the independent-chunks layout (no cached prefix).
 int plan_create(const cpa_config* cfg, int32_t num_blocks, const int32_t* block_lens, const int32_t* prefix_lens,
                 const int32_t* shared_pages, int32_t num_shared, int32_t max_new_tokens, const int32_t* free_pages,
-                int32_t num_free, cpa_plan** out) {
+                int32_t num_free, int32_t chunk_tokens, int32_t decode_sms, bool dynamic, cpa_plan** out) {
     if (out) *out = nullptr;
     if (!cfg || !block_lens || !out || num_blocks < 1 || max_new_tokens < 0 || num_free < 0 ||
         (num_free > 0 && !free_pages) || num_shared < 0 || (num_shared > 0 && !shared_pages))
@@ -35,10 +87,18 @@ int plan_create(const cpa_config* cfg, int32_t num_blocks, const int32_t* block_
         return CPA_EUNSUPPORTED;
     if (cfg->q_tile_rows != 0 && cfg->q_tile_rows != 128 && cfg->q_tile_rows != 256) return CPA_EUNSUPPORTED;
     if (cfg->pages_per_split > kMaxSplitPages) return CPA_EUNSUPPORTED;
+    // the schedule's sort keys hold a CTA id in 12 bits; the shared-scan items pack worker ranges in 16
+    if (cfg->num_sms > kMaxPlanSms) return CPA_EUNSUPPORTED;
+    if (prefix_lens && num_blocks > 0xFFFF) return CPA_EUNSUPPORTED;
+    // a chunk is read back as a cached prefix of whole 128-key tiles
+    if (chunk_tokens < 0 || chunk_tokens % 128 != 0 || decode_sms < 0) return CPA_EINVAL;
+    if (chunk_tokens > 0 && prefix_lens) return CPA_EUNSUPPORTED;
+    if (dynamic && (chunk_tokens > 0 || prefix_lens)) return CPA_EUNSUPPORTED;
 
     cpa_plan* p = new (std::nothrow) cpa_plan();
     if (!p) return CPA_ENOSPC;
     p->cfg = *cfg;
+    p->num_sms = cfg->num_sms ? cfg->num_sms : std::min(device_sm_count(), kMaxPlanSms);
     p->B = num_blocks;
     p->T = max_new_tokens;
     p->q_tile = cfg->q_tile_rows ? cfg->q_tile_rows : 256;
@@ -75,6 +135,18 @@ int plan_create(const cpa_config* cfg, int32_t num_blocks, const int32_t* block_
     }
     p->total_tokens = p->cu_seqlens[B];
     const int32_t pages_used = p->page_indptr[B];
+    // Pages on demand: a block starts with the pages for its tokens plus the next one (never more than its row of
+    // the table holds); the rest of the free list is the common reserve.
+    p->dynamic = dynamic;
+    std::vector<int32_t> first_pages(own_pages);
+    if (dynamic) {
+        own_total = 0;
+        for (int32_t b = 0; b < B; ++b) {
+            first_pages[b] = std::min(block_lens[b] / P + 1, own_pages[b]);
+            own_total += first_pages[b];
+        }
+        p->pages_assigned = first_pages;
+    }
     if (own_total > num_free) { delete p; return CPA_ENOSPC; }
     // a sequence's pages: the shared pages of its cached prefix first, then pages of its own, dealt
     // in order from the free list
@@ -82,8 +154,15 @@ int plan_create(const cpa_config* cfg, int32_t num_blocks, const int32_t* block_
     int64_t taken = 0;
     for (int32_t b = 0; b < B; ++b) {
         p->page_indices.insert(p->page_indices.end(), shared_pages, shared_pages + p->prefix_lens[b] / P);
-        p->page_indices.insert(p->page_indices.end(), free_pages + taken, free_pages + taken + own_pages[b]);
-        taken += own_pages[b];
+        p->page_indices.insert(p->page_indices.end(), free_pages + taken, free_pages + taken + first_pages[b]);
+        p->page_indices.insert(p->page_indices.end(), (size_t)(own_pages[b] - first_pages[b]), 0);   // not assigned yet
+        taken += first_pages[b];
+    }
+    if (dynamic) {
+        p->free_ring.assign(free_pages + taken, free_pages + num_free);
+        p->ring_size = std::max(1, num_free);
+        for (int32_t id : p->free_ring)
+            if (id < 0 || id > INT32_MAX / 64) { delete p; return CPA_EINVAL; }
     }
     int32_t max_page = 0;
     for (int32_t id : p->page_indices) {
@@ -121,22 +200,12 @@ int plan_create(const cpa_config* cfg, int32_t num_blocks, const int32_t* block_
     p->prefill_items.reserve(pit.size() * 2);
     for (const PItem& it : pit) { p->prefill_items.push_back(it.block); p->prefill_items.push_back(it.tile); }
 
-    // Prefill schedule for the persistent kernel (one CTA per SM).  A unit is (item, query head).  Units
-    // are listed kv head by kv head, inside a kv head in item order, the G query heads of the group
-    // side by side: CTAs that run at the same time then stream the same few K/V ranges, which stay in
-    // L2.  The list is dealt in rounds of one unit per CTA: in every round the CTAs are ranked by the
-    // work they have so far (least first, ties to the lower CTA), the round's units by cost (largest
-    // first, ties in list order), and the i-th unit goes to the i-th CTA.  A unit's cost is its KV
-    // tile count plus a fixed part.
+    // Prefill schedule for the persistent kernel: see deal_prefill_units.  A unit's cost is its KV tile
+    // count plus a fixed part.
     {
         const int32_t Hq = cfg->num_q_heads, G = Hq / cfg->num_kv_heads;
         const int64_t n_units = (int64_t)p->n_prefill * Hq;
         if (n_units > INT32_MAX / 4) { delete p; return CPA_EUNSUPPORTED; }
-        const int32_t ctas = (int32_t)std::min<int64_t>(cfg->num_sms ? cfg->num_sms : 148, n_units);
-        const int32_t rounds = (int32_t)((n_units + ctas - 1) / ctas);
-        p->prefill_ctas = ctas;
-        p->prefill_rounds = rounds;
-        p->prefill_sched.assign((size_t)rounds * (size_t)ctas, -1);
         const int32_t sub_per_item = p->q_tile / 128;
         std::vector<int32_t> item_cost((size_t)p->n_prefill);
         for (int32_t i = 0; i < p->n_prefill; ++i) {
@@ -144,28 +213,7 @@ int plan_create(const cpa_config* cfg, int32_t num_blocks, const int32_t* block_
             const int32_t n_sub = (sub_per_item > 1 && block_lens[b] - q0 > 128) ? 2 : 1;
             item_cost[(size_t)i] = 10 * (p->prefix_lens[b] / 128 + q0 / 128 + n_sub) + 18;
         }
-        std::vector<int64_t> load((size_t)ctas, 0);
-        std::vector<uint64_t> rank((size_t)ctas), batch((size_t)ctas);   // packed sort keys
-        const int64_t per_head = (int64_t)p->n_prefill * G;            // units of one kv head
-        for (int32_t r = 0; r < rounds; ++r) {
-            const int64_t u0 = (int64_t)r * ctas, n = std::min<int64_t>(ctas, n_units - u0);
-            for (int64_t j = 0; j < n; ++j) {
-                // unit u0 + j of the list -> (kv head, item, head inside the group)
-                const int64_t u = u0 + j, g = u / per_head, rem = u - g * per_head;
-                const int32_t i = (int32_t)(rem / G), h = (int32_t)(rem - (int64_t)i * G);
-                // descending cost, then list order: the position j breaks ties
-                batch[(size_t)j] = ((uint64_t)(0xFFFFFu - (uint32_t)item_cost[(size_t)i]) << 44) | ((uint64_t)j << 32) |
-                                   (uint32_t)(i * Hq + (int32_t)g * G + h);
-            }
-            std::sort(batch.begin(), batch.begin() + n);
-            for (int32_t c = 0; c < ctas; ++c) rank[(size_t)c] = ((uint64_t)load[(size_t)c] << 16) | (uint32_t)c;
-            std::sort(rank.begin(), rank.end());
-            for (int64_t j = 0; j < n; ++j) {
-                const int32_t c = (int32_t)(rank[(size_t)j] & 0xFFFFu);
-                p->prefill_sched[(size_t)r * (size_t)ctas + (size_t)c] = (int32_t)(batch[(size_t)j] & 0xFFFFFFFFu);
-                load[(size_t)c] += 0xFFFFF - (int64_t)(batch[(size_t)j] >> 44);
-            }
-        }
+        p->prefill_sched = deal_prefill_units(item_cost, Hq, G, p->num_sms, &p->prefill_ctas, &p->prefill_rounds);
     }
 
     // Decode splits.  Every CTA pays a fixed start-up and merge cost, so the planner aims at
@@ -192,7 +240,7 @@ int plan_create(const cpa_config* cfg, int32_t num_blocks, const int32_t* block_
         const int32_t G = cfg->num_q_heads / cfg->num_kv_heads;
         const int32_t per_group = cpa_scan_rows(G) / G;                     // workers per group
         const int32_t n_groups = (B + per_group - 1) / per_group;
-        const int64_t sms = cfg->num_sms ? cfg->num_sms : 148;
+        const int64_t sms = p->num_sms;
         const int64_t want = std::max<int64_t>(1, 3 * sms / ((int64_t)cfg->num_kv_heads * n_groups));   // chunks per (group, head)
         int64_t ch = (max_pre_pages + want - 1) / want;
         ch = std::min<int64_t>(kMaxSharedChunkPages, std::max<int64_t>(8, (ch + 7) / 8 * 8));   // whole 128-key tiles
@@ -221,7 +269,7 @@ int plan_create(const cpa_config* cfg, int32_t num_blocks, const int32_t* block_
     if (cfg->pages_per_split > 0) {
         for (int32_t b = 0; b < B; ++b) p->split_pages[b] = cfg->pages_per_split;
     } else {
-        const int64_t slots = 3LL * (cfg->num_sms ? cfg->num_sms : 148);
+        const int64_t slots = 3LL * p->num_sms;
         int64_t items = (int64_t)B * cfg->num_kv_heads;
         while (items + cfg->num_kv_heads <= slots) {
             int32_t best = -1;
@@ -265,6 +313,68 @@ int plan_create(const cpa_config* cfg, int32_t num_blocks, const int32_t* block_
         p->decode_items.push_back(it.split);
     }
 
+    // Chunked prefill: step s prefills rows [s*C, min((s+1)*C, L_b)) of every block that has them, reading the
+    // block's earlier chunks from its pages exactly like a cached prefix; a block decodes in the T steps after
+    // its last chunk.  Every step gets its own item list and deal.  While some block decodes, the chunk's
+    // persistent grid leaves `decode_sms` SMs to the decode wave that runs beside it.
+    std::vector<int32_t> chunk_items, chunk_sched, chunk_rows;
+    if (chunk_tokens > 0) {
+        const int32_t Cc = chunk_tokens, Hq = cfg->num_q_heads, G = Hq / cfg->num_kv_heads;
+        p->chunk = Cc;
+        p->decode_sms = decode_sms ? decode_sms : std::max(1, p->num_sms / 4);
+        if (p->decode_sms >= p->num_sms) { delete p; return CPA_EINVAL; }
+        p->dec_start.assign(B, 0);
+        int32_t n_chunk_steps = 0;
+        for (int32_t b = 0; b < B; ++b) {
+            p->dec_start[b] = (block_lens[b] + Cc - 1) / Cc;
+            n_chunk_steps = std::max(n_chunk_steps, p->dec_start[b]);
+        }
+        p->n_steps = n_chunk_steps + max_new_tokens;
+        p->chunk_steps.resize((size_t)n_chunk_steps);
+        for (int32_t st = 0; st < n_chunk_steps; ++st) {
+            cpa_chunk_step& cs = p->chunk_steps[(size_t)st];
+            bool any_decode = false;
+            for (int32_t b = 0; b < B; ++b) any_decode |= p->dec_start[b] <= st && st < p->dec_start[b] + max_new_tokens;
+            std::vector<PItem> cit;
+            cs.off_rows = (int64_t)chunk_rows.size();
+            int32_t rows = 0;
+            for (int32_t b = 0; b < B; ++b) {
+                chunk_rows.push_back(rows);
+                if (st >= p->dec_start[b]) continue;
+                const int32_t len = std::min(Cc, block_lens[b] - st * Cc);
+                rows += len;
+                for (int32_t t = 0; t * p->q_tile < len; ++t)
+                    cit.push_back({st * Cc + std::min((t + 1) * p->q_tile, len), b, t});
+            }
+            chunk_rows.push_back(rows);
+            cs.rows = rows;
+            std::stable_sort(cit.begin(), cit.end(), [](const PItem& a, const PItem& c) {
+                if (a.cost != c.cost) return a.cost > c.cost;
+                if (a.block != c.block) return a.block < c.block;
+                return a.tile < c.tile;
+            });
+            cs.n_items = (int32_t)cit.size();
+            cs.off_items = (int64_t)chunk_items.size();
+            std::vector<int32_t> item_cost(cit.size());
+            for (size_t i = 0; i < cit.size(); ++i) {
+                const int32_t b = cit[i].block, q0 = cit[i].tile * p->q_tile;
+                const int32_t len = std::min(Cc, block_lens[b] - st * Cc);
+                const int32_t n_sub = (p->q_tile > 128 && len - q0 > 128) ? 2 : 1;
+                item_cost[i] = 10 * (st * Cc / 128 + q0 / 128 + n_sub) + 18;
+                // the chunk is a "block" of its own whose cached prefix is the block's earlier chunks
+                chunk_items.push_back(p->cu_seqlens[b] + st * Cc);
+                chunk_items.push_back(len);
+                chunk_items.push_back(cit[i].tile | ((st * Cc / 128) << 16));
+                chunk_items.push_back(p->page_indptr[b]);
+            }
+            if ((int64_t)st * Cc / 128 > 0x7FFF) { delete p; return CPA_EUNSUPPORTED; }
+            const int32_t budget = any_decode ? p->num_sms - p->decode_sms : p->num_sms;
+            std::vector<int32_t> sched = deal_prefill_units(item_cost, Hq, G, budget, &cs.ctas, &cs.rounds);
+            cs.off_sched = (int64_t)chunk_sched.size();
+            chunk_sched.insert(chunk_sched.end(), sched.begin(), sched.end());
+        }
+    }
+
     // device image
     int64_t w = 0;
     p->off_status = w;  w = align4(w + 4);
@@ -283,6 +393,15 @@ int plan_create(const cpa_config* cfg, int32_t num_blocks, const int32_t* block_
     p->off_prefix = w;  w = align4(w + B);
     p->off_shitems = w; w = align4(w + (int64_t)p->shared_items.size());
     p->off_shpages = w; w = align4(w + (int64_t)p->shared_page_ids.size());
+    p->off_decstart = w; w = align4(w + (int64_t)p->dec_start.size());
+    p->off_assigned = w; w = align4(w + (int64_t)p->pages_assigned.size());
+    p->off_ringctrl = w; w = align4(w + (dynamic ? 4 : 0));
+    p->off_ring = w;     w = align4(w + (dynamic ? p->ring_size : 0));
+    const int64_t off_citems = w; w = align4(w + (int64_t)chunk_items.size());
+    const int64_t off_csched = w; w = align4(w + (int64_t)chunk_sched.size());
+    const int64_t off_crows = w;  w = align4(w + (int64_t)chunk_rows.size());
+    for (cpa_chunk_step& cs : p->chunk_steps) { cs.off_items += off_citems; cs.off_sched += off_csched; cs.off_rows += off_crows; }
+    p->chunk_rows = chunk_rows;
     p->words = w;
     p->image.assign((size_t)w, 0);
     int32_t* im = p->image.data();
@@ -303,6 +422,20 @@ int plan_create(const cpa_config* cfg, int32_t num_blocks, const int32_t* block_
     for (int32_t b = 0; b < B; ++b) im[p->off_seqlens + b] = im[p->off_seqlens2 + b] = p->prefix_lens[b];
     std::memcpy(im + p->off_psched, p->prefill_sched.data(), sizeof(int32_t) * p->prefill_sched.size());
     std::memcpy(im + p->off_prefix, p->prefix_lens.data(), sizeof(int32_t) * B);
+    if (dynamic) {
+        std::memcpy(im + p->off_assigned, p->pages_assigned.data(), sizeof(int32_t) * B);
+        im[p->off_ringctrl + 0] = 0;                                 // pops so far
+        im[p->off_ringctrl + 1] = (int32_t)p->free_ring.size();      // pushes so far
+        im[p->off_ringctrl + 2] = p->ring_size;
+        if (!p->free_ring.empty())
+            std::memcpy(im + p->off_ring, p->free_ring.data(), sizeof(int32_t) * p->free_ring.size());
+    }
+    if (!p->dec_start.empty()) {
+        std::memcpy(im + p->off_decstart, p->dec_start.data(), sizeof(int32_t) * p->dec_start.size());
+        std::memcpy(im + off_citems, chunk_items.data(), sizeof(int32_t) * chunk_items.size());
+        std::memcpy(im + off_csched, chunk_sched.data(), sizeof(int32_t) * chunk_sched.size());
+        std::memcpy(im + off_crows, chunk_rows.data(), sizeof(int32_t) * chunk_rows.size());
+    }
     if (!p->shared_items.empty()) {
         std::memcpy(im + p->off_shitems, p->shared_items.data(), sizeof(int32_t) * p->shared_items.size());
         std::memcpy(im + p->off_shpages, p->shared_page_ids.data(), sizeof(int32_t) * p->shared_page_ids.size());
@@ -334,7 +467,50 @@ int plan_create(const cpa_config* cfg, int32_t num_blocks, const int32_t* block_
 extern "C" int cpa_plan_create(const cpa_config* cfg, int32_t num_blocks, const int32_t* block_lens,
                                int32_t max_new_tokens, const int32_t* free_pages, int32_t num_free,
                                cpa_plan** out) {
-    return plan_create(cfg, num_blocks, block_lens, nullptr, nullptr, 0, max_new_tokens, free_pages, num_free, out);
+    return plan_create(cfg, num_blocks, block_lens, nullptr, nullptr, 0, max_new_tokens, free_pages, num_free, 0, 0, false, out);
+}
+
+extern "C" int cpa_plan_create_dynamic(const cpa_config* cfg, int32_t num_blocks, const int32_t* block_lens,
+                                       int32_t max_new_tokens, const int32_t* free_pages, int32_t num_free,
+                                       cpa_plan** out) {
+    return plan_create(cfg, num_blocks, block_lens, nullptr, nullptr, 0, max_new_tokens, free_pages, num_free, 0, 0, true,
+                       out);
+}
+
+extern "C" int cpa_plan_sync(cpa_plan* plan, void* stream) {
+    if (!plan) return CPA_EINVAL;
+    if (!plan->d_base) return CPA_ESTATE;
+    cudaStream_t st = (cudaStream_t)stream;
+    const int B = plan->B;
+    std::vector<int32_t> ctrl(4, 0), ring((size_t)plan->ring_size, 0);
+    bool ok = cudaMemcpyAsync(plan->seq_lens.data(), plan->d_base + (plan->cur_lens ? plan->off_seqlens2 : plan->off_seqlens),
+                              sizeof(int32_t) * B, cudaMemcpyDeviceToHost, st) == cudaSuccess;
+    if (ok && plan->dynamic) {
+        ok = cudaMemcpyAsync(plan->page_indices.data(), plan->d_base + plan->off_pidx,
+                             sizeof(int32_t) * plan->page_indices.size(), cudaMemcpyDeviceToHost, st) == cudaSuccess &&
+             cudaMemcpyAsync(plan->pages_assigned.data(), plan->d_base + plan->off_assigned, sizeof(int32_t) * B,
+                             cudaMemcpyDeviceToHost, st) == cudaSuccess &&
+             cudaMemcpyAsync(ctrl.data(), plan->d_base + plan->off_ringctrl, sizeof(int32_t) * 4, cudaMemcpyDeviceToHost,
+                             st) == cudaSuccess &&
+             cudaMemcpyAsync(ring.data(), plan->d_base + plan->off_ring, sizeof(int32_t) * ring.size(),
+                             cudaMemcpyDeviceToHost, st) == cudaSuccess;
+    }
+    if (ok) ok = cudaStreamSynchronize(st) == cudaSuccess;
+    if (!ok) { (void)cudaGetLastError(); return CPA_ECUDA; }
+    if (plan->dynamic) {
+        plan->free_ring.clear();
+        for (int32_t i = ctrl[0]; i < ctrl[1]; ++i) plan->free_ring.push_back(ring[(size_t)(i % plan->ring_size)]);
+    }
+    return CPA_OK;
+}
+
+extern "C" int cpa_plan_create_chunked(const cpa_config* cfg, int32_t num_blocks, const int32_t* block_lens,
+                                       int32_t max_new_tokens, int32_t chunk_tokens, int32_t decode_sms,
+                                       const int32_t* free_pages, int32_t num_free, cpa_plan** out) {
+    if (out) *out = nullptr;
+    if (chunk_tokens < 128) return CPA_EINVAL;
+    return plan_create(cfg, num_blocks, block_lens, nullptr, nullptr, 0, max_new_tokens, free_pages, num_free,
+                       chunk_tokens, decode_sms, false, out);
 }
 
 extern "C" int cpa_plan_create_prefix(const cpa_config* cfg, int32_t num_workers, const int32_t* own_lens,
@@ -344,7 +520,7 @@ extern "C" int cpa_plan_create_prefix(const cpa_config* cfg, int32_t num_workers
     if (out) *out = nullptr;
     if (!prefix_lens) return CPA_EINVAL;
     return plan_create(cfg, num_workers, own_lens, prefix_lens, shared_pages, num_shared, max_new_tokens, free_pages,
-                       num_free, out);
+                       num_free, 0, 0, false, out);
 }
 
 extern "C" int cpa_plan_export(const cpa_plan* plan, int which, const int32_t** ptr, int64_t* count) {
@@ -362,6 +538,10 @@ extern "C" int cpa_plan_export(const cpa_plan* plan, int which, const int32_t** 
         case CPA_ARR_SPLIT_INDPTR: v = &plan->split_indptr; break;
         case CPA_ARR_SPLIT_PAGES: v = &plan->split_pages; break;
         case CPA_ARR_PREFILL_SCHED: v = &plan->prefill_sched; break;
+        case CPA_ARR_DEC_START: v = &plan->dec_start; break;
+        case CPA_ARR_CHUNK_ROWS: v = &plan->chunk_rows; break;
+        case CPA_ARR_PAGES_ASSIGNED: v = &plan->pages_assigned; break;
+        case CPA_ARR_FREE_RING: v = &plan->free_ring; break;
         default: return CPA_EINVAL;
     }
     *ptr = v->data();
@@ -376,13 +556,23 @@ extern "C" int64_t cpa_plan_param(const cpa_plan* plan, int which) {
         case CPA_PARAM_TOTAL_TOKENS: return plan->total_tokens;
         case CPA_PARAM_Q_TILE_ROWS: return plan->q_tile;
         case CPA_PARAM_PAGES_PER_SPLIT: return plan->C;
-        case CPA_PARAM_PAGES_USED: return plan->page_indptr[plan->B];
+        case CPA_PARAM_PAGES_USED: {
+            if (!plan->dynamic) return plan->page_indptr[plan->B];
+            int64_t n = 0;
+            for (int32_t a : plan->pages_assigned) n += a;
+            return n;
+        }
         case CPA_PARAM_INDEX_BYTES: return plan->index_bytes();
         case CPA_PARAM_DECODE_WORKSPACE_BYTES: return plan->decode_workspace_bytes();
         case CPA_PARAM_TOTAL_SPLITS: return plan->split_indptr[plan->B];
         case CPA_PARAM_MAX_NEW_TOKENS: return plan->T;
         case CPA_PARAM_PREFILL_CTAS: return plan->prefill_ctas;
         case CPA_PARAM_SHARED_CHUNK_PAGES: return plan->shared_chunk;
+        case CPA_PARAM_CHUNK_TOKENS: return plan->chunk;
+        case CPA_PARAM_NUM_STEPS: return plan->n_steps;
+        case CPA_PARAM_CHUNK_STEPS: return (int64_t)plan->chunk_steps.size();
+        case CPA_PARAM_DECODE_SMS: return plan->decode_sms;
+        case CPA_PARAM_NUM_SMS: return plan->num_sms;
         default: return CPA_EINVAL;
     }
 }
@@ -393,6 +583,13 @@ extern "C" int cpa_plan_upload(cpa_plan* plan, void* d_index_buf, int64_t bytes,
     // the device copy starts with nothing but the cached prefixes, so the host mirror does too
     plan->seq_lens = plan->prefix_lens;
     plan->cur_lens = 0;
+    plan->next_step = 0;
+    if (plan->dynamic) {   // the device starts from the plan's first assignment again, and so do the host mirrors
+        const int32_t* im = plan->image.data();
+        plan->page_indices.assign(im + plan->off_pidx, im + plan->off_pidx + plan->page_indices.size());
+        plan->pages_assigned.assign(im + plan->off_assigned, im + plan->off_assigned + plan->B);
+        plan->free_ring.assign(im + plan->off_ring, im + plan->off_ring + im[plan->off_ringctrl + 1]);
+    }
     cudaError_t e = cudaMemcpyAsync(d_index_buf, plan->image.data(), (size_t)plan->index_bytes(),
                                     cudaMemcpyHostToDevice, (cudaStream_t)stream);
     if (e != cudaSuccess) { (void)cudaGetLastError(); return CPA_ECUDA; }
@@ -408,10 +605,18 @@ extern "C" int cpa_plan_status(cpa_plan* plan, void* stream) {
                                     cudaMemcpyDeviceToHost, (cudaStream_t)stream);
     if (e == cudaSuccess) e = cudaStreamSynchronize((cudaStream_t)stream);
     if (e != cudaSuccess) { (void)cudaGetLastError(); return CPA_ECUDA; }
-    return word == 0 ? CPA_OK : CPA_ETIMEOUT;
+    // the first code a kernel recorded: 1 = a bounded wait gave up, 2 = an append found no room
+    return word == 0 ? CPA_OK : word == 2 ? CPA_ENOSPC : CPA_ETIMEOUT;
 }
 
-extern "C" void cpa_plan_destroy(cpa_plan* plan) { delete plan; }
+extern "C" void cpa_plan_destroy(cpa_plan* plan) {
+    if (!plan) return;
+    if (plan->ev_fork) cudaEventDestroy(plan->ev_fork);
+    if (plan->ev_join) cudaEventDestroy(plan->ev_join);
+    if (plan->side_stream) cudaStreamDestroy(plan->side_stream);
+    (void)cudaGetLastError();
+    delete plan;
+}
 
 extern "C" const char* cpa_strerror(int status) {
     switch (status) {

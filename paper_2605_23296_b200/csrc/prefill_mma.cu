@@ -6,6 +6,8 @@
 // registers (fp32).  Only tiles at or below the diagonal are visited; keys are
 // restricted to the query's own block by construction (tile ranges come from
 // cu_seqlens), rows past the block's end are never stored.
+#include <atomic>
+
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 
@@ -242,19 +244,19 @@ template <int D>
 int launch_prefill_mma(const cpa_plan* plan, const void* q, const void* k, const void* v, void* o, cudaStream_t st) {
     const cpa_config& c = plan->cfg;
     constexpr int smem = (kQTile + 4 * kKVTile) * D * 2;
-    static bool configured_dev[64] = {};  // the attribute is per device: remember which devices have it
+    static std::atomic<bool> configured_dev[64];  // the attribute is per device: remember which devices have it
     int dev_id = 0;
     if (cudaGetDevice(&dev_id) != cudaSuccess || dev_id < 0 || dev_id >= 64) {
         (void)cudaGetLastError();
         return CPA_ECUDA;
     }
-    bool& configured = configured_dev[dev_id];
-    if (!configured) {
+    std::atomic<bool>& configured = configured_dev[dev_id];
+    if (!configured.load(std::memory_order_relaxed)) {
         if (cudaFuncSetAttribute(prefill_mma_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) {
             (void)cudaGetLastError();
             return CPA_ECUDA;
         }
-        configured = true;
+        configured.store(true, std::memory_order_relaxed);
     }
     const int subs = plan->q_tile / kQTile;
     dim3 grid(plan->n_prefill * subs, c.num_q_heads);

@@ -33,10 +33,13 @@
 //
 // Every mbarrier wait is bounded: when one gives up the CTA records it in the status word,
 // stops waiting, still frees its TMEM and returns.
+#include <atomic>
+
 #include <cuda.h>
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 
+#include "cpa_device.cuh"
 #include "cpa_internal.h"
 
 namespace {
@@ -47,38 +50,15 @@ constexpr int kThreads = 384;        // 2 softmax warpgroups + 1 warpgroup holdi
 constexpr int kRegsSoftmax = 216;    // register split after launch (launch gives every thread 168):
 constexpr int kRegsControl = 72;     // 2*128*216 + 128*72 = 64512 = 384*168, exactly the launch total
 constexpr uint32_t kSpinLimit = 1u << 20;
+constexpr uint32_t kDrainLimit = 1u << 12;   // last look at work in flight after a wait gave up
 constexpr uint32_t kBlockBytes = 128 * 128;   // one column block: 128 rows x 128 B
 
 // ---------------------------------------------------------------- PTX wrappers
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;\n" :: "r"(bar), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;\n" :: "r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];\n" :: "r"(bar) : "memory");
-}
-__device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity) {
-    uint32_t ok;
-    asm volatile(
-        "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}\n"
-        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-    return ok;
-}
-// Bounded wait.  Returns false (and records it) when the limit is hit; `dead` makes all later waits no-ops.
-__device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, bool& dead, int32_t* status) {
-    if (dead) return;
-    uint32_t spins = 0;
-    while (!mbar_try_wait(bar, parity)) {
-        if (++spins > kSpinLimit) {
-            dead = true;
-            atomicCAS(status, 0, 1);
-            return;
-        }
-    }
+// Bounded wait with this file's limit (see mbar_wait): after it gave up once, `dead` turns every later wait into a no-op.
+__device__ __forceinline__ void tc_wait(uint32_t bar, uint32_t parity, bool& dead, int32_t* status) {
+    mbar_wait(bar, parity, dead, status, kSpinLimit);
 }
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
     asm volatile(
@@ -220,6 +200,7 @@ struct __align__(8) TcBarriers {
     // [sub-tile][that sub-tile's step count mod 4]: at most three steps are ever ahead of a waiter, so a
     // waiter can never meet the phase after the one it is waiting for
     uint64_t s_full[2][4], p_full[2][4], pv_done[2];
+    uint64_t drain;   // only used after a wait gave up: tracks the MMAs still queued, so that TMEM is not freed under them
     uint32_t tmem_base;
 };
 
@@ -317,6 +298,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                 mbar_init(bar(&bars.p_full[u][i]), 128);
             }
         }
+        mbar_init(bar(&bars.drain), 1);
         for (int s = 0; s < KS; ++s) {
             mbar_init(bar(&bars.k_full[s]), 1);
             mbar_init(bar(&bars.k_empty[s]), 1);
@@ -348,12 +330,16 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
         // plain copy of 16 rows x 128 bytes lands as rows 16p .. 16p+15 of a swizzled column block.
         {
             int kt = 0;                   // K/V tiles loaded so far: stage kt % KS, use count kt / KS
+            int k_issued = 0, v_issued = 0; // K / V tiles handed to the copy engine (they differ only after a wait gave up)
             uint32_t q_loads[2] = {0, 0};   // loads of Q_u so far
             TcWork w;
             Rec rec;
             fetch(fetch_code(0), rec);
             int code = fetch_code(1);
             for (int k = 0; k < n_rounds; ++k) {
+                // once a wait has given up nothing more is issued (lane 0 does the waiting: its verdict counts)
+                dead = __shfl_sync(0xffffffffu, (int)dead, 0) != 0;
+                if (dead) break;
                 decode(rec, w);
                 fetch(code, rec);
                 code = fetch_code(k + 2);
@@ -361,7 +347,8 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                 if (lane == 0) {
                     for (int u = 0; u < w.n_sub; ++u) {
                         // the buffer is free once the last score MMA of its previous unit has run
-                        mbar_wait(bar(&bars.q_empty[u]), (q_loads[u] & 1u) ^ 1u, dead, ix.status);
+                        tc_wait(bar(&bars.q_empty[u]), (q_loads[u] & 1u) ^ 1u, dead, ix.status);
+                        if (dead) break;
                         ++q_loads[u];
                         mbar_expect_tx(bar(&bars.q_full[u]), kTileBytes);
 #pragma unroll
@@ -377,16 +364,20 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                             const int s = kt % KS;
                             const uint32_t par = (uint32_t)(kt / KS) & 1u;
                             const int row = w.tok0 + j * kTileN;
-                            mbar_wait(bar(&bars.k_empty[s]), par ^ 1u, dead, ix.status);
+                            tc_wait(bar(&bars.k_empty[s]), par ^ 1u, dead, ix.status);
+                            if (dead) break;
                             mbar_expect_tx(bar(&bars.k_full[s]), kTileBytes);
 #pragma unroll
                             for (int c = 0; c < NB; ++c)
                                 tma_load_2d(s_k + s * kTileBytes + c * kBlockBytes, &tm_k, w.g * D + 64 * c, row, bar(&bars.k_full[s]));
-                            mbar_wait(bar(&bars.v_empty[s]), par ^ 1u, dead, ix.status);
+                            ++k_issued;
+                            tc_wait(bar(&bars.v_empty[s]), par ^ 1u, dead, ix.status);
+                            if (dead) break;
                             mbar_expect_tx(bar(&bars.v_full[s]), kTileBytes);
 #pragma unroll
                             for (int c = 0; c < NB; ++c)
                                 tma_load_2d(s_v + s * kTileBytes + c * kBlockBytes, &tm_v, w.g * D + 64 * c, row, bar(&bars.v_full[s]));
+                            ++v_issued;
                         }
                     } else {
                         kt += w.n_total;
@@ -404,10 +395,11 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                     if (lane < 8 && j + 1 < w.n_pre) page = __ldg(ix.page_indices + w.page_base + 8 * (j + 1) + lane);
                     const int row = cached ? (my_page * Hkv + w.g) * 16 : w.tok0 + (j - w.n_pre) * kTileN;
                     if (lane == 0) {
-                        mbar_wait(bar(&bars.k_empty[s]), par ^ 1u, dead, ix.status);
-                        mbar_expect_tx(bar(&bars.k_full[s]), kTileBytes);
+                        tc_wait(bar(&bars.k_empty[s]), par ^ 1u, dead, ix.status);
+                        if (!dead) mbar_expect_tx(bar(&bars.k_full[s]), kTileBytes);
                     }
-                    __syncwarp();
+                    dead = __shfl_sync(0xffffffffu, (int)dead, 0) != 0;
+                    if (dead) break;
                     if (cached) {
                         if (lane < 8) {
 #pragma unroll
@@ -420,11 +412,13 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                         for (int c = 0; c < NB; ++c)
                             tma_load_2d(s_k + s * kTileBytes + c * kBlockBytes, &tm_k, w.g * D + 64 * c, row, bar(&bars.k_full[s]));
                     }
+                    ++k_issued;
                     if (lane == 0) {
-                        mbar_wait(bar(&bars.v_empty[s]), par ^ 1u, dead, ix.status);
-                        mbar_expect_tx(bar(&bars.v_full[s]), kTileBytes);
+                        tc_wait(bar(&bars.v_empty[s]), par ^ 1u, dead, ix.status);
+                        if (!dead) mbar_expect_tx(bar(&bars.v_full[s]), kTileBytes);
                     }
-                    __syncwarp();
+                    dead = __shfl_sync(0xffffffffu, (int)dead, 0) != 0;
+                    if (dead) break;
                     if (cached) {
                         if (lane < 8) {
 #pragma unroll
@@ -437,14 +431,26 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                         for (int c = 0; c < NB; ++c)
                             tma_load_2d(s_v + s * kTileBytes + c * kBlockBytes, &tm_v, w.g * D + 64 * c, row, bar(&bars.v_full[s]));
                     }
+                    ++v_issued;
                 }
+            }
+            // After a wait gave up: the copies issued last may still be on their way into this CTA's
+            // shared memory.  Lane 0 gives the latest phase of every barrier that had a copy one more
+            // bounded look before the CTA goes on to its end.
+            if (__shfl_sync(0xffffffffu, (int)dead, 0) != 0 && lane == 0) {
+                for (int u = 0; u < 2; ++u)
+                    if (q_loads[u] > 0) mbar_drain(bar(&bars.q_full[u]), (q_loads[u] - 1u) & 1u, kDrainLimit);
+                for (int t = max(0, k_issued - KS); t < k_issued; ++t)
+                    mbar_drain(bar(&bars.k_full[t % KS]), (uint32_t)(t / KS) & 1u, kDrainLimit);
+                for (int t = max(0, v_issued - KS); t < v_issued; ++t)
+                    mbar_drain(bar(&bars.v_full[t % KS]), (uint32_t)(t / KS) & 1u, kDrainLimit);
             }
         }
     } else if (warp == 9) {
         // ------------------------------------------------------------ MMA issuer (whole warp, one lane issues)
         // Everything the issuing thread executes between two MMAs delays the tensor core, so the
         // loops below are written out per case with as little index arithmetic as possible.
-        const uint32_t leader = (lane == 0);
+        uint32_t leader = (lane == 0);   // cleared once a wait has given up: nothing more is issued then
         constexpr uint32_t idesc_qk = instr_desc(kTileM, kTileN, false);
         constexpr uint32_t idesc_pv = instr_desc(kTileM, D, true);
         constexpr uint32_t kTile16 = kTileBytes >> 4;        // descriptor address units are 16 bytes
@@ -467,7 +473,8 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
             ++n_qk[u];
         };
         auto pv = [&](int u, int buf, int kt, uint32_t acc0) {   // O_u += P[buf] V[tile kt]
-            mbar_wait(bar(&bars.p_full[u][n_pv[u] & 3u]), (n_pv[u] >> 2) & 1u, dead, ix.status);
+            tc_wait(bar(&bars.p_full[u][n_pv[u] & 3u]), (n_pv[u] >> 2) & 1u, dead, ix.status);
+            if (dead) leader = 0u;
             ++n_pv[u];
             tc_fence_after();
             const uint32_t bv = v_lo + (kt % KS) * kTile16, d_tmem = tmem + kColO + u * D, a_tmem = tmem + buf * 128;
@@ -477,12 +484,17 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                 tc_mma_ts_lo(d_tmem, a_tmem + k * 8, bv + k * (2048 >> 4), pv_hi, idesc_pv, k > 0 ? 1u : acc0, leader);
         };
         auto wait_k = [&](int kt) {
-            mbar_wait(bar(&bars.k_full[kt % KS]), (uint32_t)(kt / KS) & 1u, dead, ix.status);
+            tc_wait(bar(&bars.k_full[kt % KS]), (uint32_t)(kt / KS) & 1u, dead, ix.status);
+            if (dead) leader = 0u;
             tc_fence_after();
         };
-        auto wait_v = [&](int kt) { mbar_wait(bar(&bars.v_full[kt % KS]), (uint32_t)(kt / KS) & 1u, dead, ix.status); };
+        auto wait_v = [&](int kt) {
+            tc_wait(bar(&bars.v_full[kt % KS]), (uint32_t)(kt / KS) & 1u, dead, ix.status);
+            if (dead) leader = 0u;
+        };
         auto wait_q = [&](int u) {
-            mbar_wait(bar(&bars.q_full[u]), q_uses[u] & 1u, dead, ix.status);
+            tc_wait(bar(&bars.q_full[u]), q_uses[u] & 1u, dead, ix.status);
+            if (dead) leader = 0u;
             ++q_uses[u];
         };
         // Within a unit, steps are numbered n = n_sub*j + u (KV tile j, sub-tile u); step n uses score
@@ -570,6 +582,13 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
             }
             kt0 += w.n_total;
         }
+        // After a wait gave up: MMAs queued before that may still be running.  A last commit tracks them
+        // and gets a bounded look, so that the tensor memory is not freed under them.
+        if (__shfl_sync(0xffffffffu, (int)dead, 0) != 0) {
+            tc_commit(bar(&bars.drain), (uint32_t)(lane == 0));
+            if (lane == 0) mbar_drain(bar(&bars.drain), 0u, kDrainLimit);
+            __syncwarp();
+        }
     }
     } else {
     asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;\n" :: "n"(kRegsSoftmax));
@@ -598,7 +617,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
         float l_run = 0.f;
         for (int j = 0; j < n_kv; ++j, ++n_steps) {
             const uint32_t t_s = tmem + lane_addr + buf * 128;
-            mbar_wait(bar(&bars.s_full[u][n_steps & 3u]), (n_steps >> 2) & 1u, dead, ix.status);
+            tc_wait(bar(&bars.s_full[u][n_steps & 3u]), (n_steps >> 2) & 1u, dead, ix.status);
             tc_fence_after();
             const bool diag = (j == n_kv - 1);
             uint32_t sv[4][32];
@@ -638,7 +657,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                 // have been ready before PV of the previous one has run.  The release of V tile j-1 is
                 // committed behind the last PV that reads it, which is issued after PV_u(j-1).
                 const int kt = kt0 + j - 1;
-                mbar_wait(bar(&bars.v_empty[kt % KS]), (uint32_t)(kt / KS) & 1u, dead, ix.status);
+                tc_wait(bar(&bars.v_empty[kt % KS]), (uint32_t)(kt / KS) & 1u, dead, ix.status);
                 tc_fence_after();
 #pragma unroll
                 for (int c = 0; c < D / 32; ++c) {
@@ -677,7 +696,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
         }
         // ---- epilogue: O / l -> bf16 -> global; thread r owns row r and writes it in 64-byte runs.
         // O_u is overwritten by the next unit's first PV, which waits for this warpgroup's next weights.
-        mbar_wait(bar(&bars.pv_done[u]), n_units & 1u, dead, ix.status);
+        tc_wait(bar(&bars.pv_done[u]), n_units & 1u, dead, ix.status);
         ++n_units;
         tc_fence_after();
         const float inv = 1.f / l_run;
@@ -741,6 +760,7 @@ struct ScanShape {
 
 struct __align__(8) ScanBarriers {
     uint64_t q_full, q_empty, k_full[6], k_empty[6], v_full[6], v_empty[6], s_full[4], p_full[4], pv_done;
+    uint64_t drain;   // only used after a wait gave up (see TcBarriers)
     uint32_t tmem_base;
 };
 
@@ -768,6 +788,7 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
         mbar_init(bar(&bars.q_full), 1);
         mbar_init(bar(&bars.q_empty), 1);
         mbar_init(bar(&bars.pv_done), 1);
+        mbar_init(bar(&bars.drain), 1);
         for (int s = 0; s < KS; ++s) {
             mbar_init(bar(&bars.k_full[s]), 1);
             mbar_init(bar(&bars.k_empty[s]), 1);
@@ -798,7 +819,7 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
 
     if (warp == 4) {
         // ------------------------------------------------------------ producer (whole warp)
-        int kt = 0;
+        int kt = 0, k_issued = 0, v_issued = 0;
         uint32_t q_loads = 0;
         for (int u = blockIdx.x; u < n_units; u += gridDim.x) {
             const int4 it = unit(u);
@@ -807,11 +828,13 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
             // swizzle atom each); a box that reaches past the last worker is filled with zeros.
             const int per_box = 8 / G, n_boxes = (nw + per_box - 1) / per_box;
             if (lane == 0) {
-                mbar_wait(bar(&bars.q_empty), (q_loads & 1u) ^ 1u, dead, ix.status);
-                mbar_expect_tx(bar(&bars.q_full), (uint32_t)(n_boxes * NB * 1024));
+                tc_wait(bar(&bars.q_empty), (q_loads & 1u) ^ 1u, dead, ix.status);
+                if (!dead) mbar_expect_tx(bar(&bars.q_full), (uint32_t)(n_boxes * NB * 1024));
             }
+            // once a wait has given up nothing more is issued (lane 0 does the waiting: its verdict counts)
+            dead = __shfl_sync(0xffffffffu, (int)dead, 0) != 0;
+            if (dead) break;
             ++q_loads;
-            __syncwarp();
             for (int bx = lane; bx < n_boxes; bx += 32) {
 #pragma unroll
                 for (int c = 0; c < NB; ++c)
@@ -824,30 +847,43 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                 const int row = (page * Hkv + g) * 16;
                 if (lane < 8 && j + 1 < n_tiles) page = __ldg(ix.shared_page_ids + first + 8 * (j + 1) + lane);
                 if (lane == 0) {
-                    mbar_wait(bar(&bars.k_empty[s]), par ^ 1u, dead, ix.status);
-                    mbar_expect_tx(bar(&bars.k_full[s]), kTileBytes);
+                    tc_wait(bar(&bars.k_empty[s]), par ^ 1u, dead, ix.status);
+                    if (!dead) mbar_expect_tx(bar(&bars.k_full[s]), kTileBytes);
                 }
-                __syncwarp();
+                dead = __shfl_sync(0xffffffffu, (int)dead, 0) != 0;
+                if (dead) break;
                 if (lane < 8) {
 #pragma unroll
                     for (int c = 0; c < NB; ++c)
                         tma_load_2d(s_k + s * kTileBytes + c * kBlockBytes + lane * 2048, &tm_kpool, 64 * c, row, bar(&bars.k_full[s]));
                 }
+                ++k_issued;
                 if (lane == 0) {
-                    mbar_wait(bar(&bars.v_empty[s]), par ^ 1u, dead, ix.status);
-                    mbar_expect_tx(bar(&bars.v_full[s]), kTileBytes);
+                    tc_wait(bar(&bars.v_empty[s]), par ^ 1u, dead, ix.status);
+                    if (!dead) mbar_expect_tx(bar(&bars.v_full[s]), kTileBytes);
                 }
-                __syncwarp();
+                dead = __shfl_sync(0xffffffffu, (int)dead, 0) != 0;
+                if (dead) break;
                 if (lane < 8) {
 #pragma unroll
                     for (int c = 0; c < NB; ++c)
                         tma_load_2d(s_v + s * kTileBytes + c * kBlockBytes + lane * 2048, &tm_vpool, 64 * c, row, bar(&bars.v_full[s]));
                 }
+                ++v_issued;
             }
+            if (dead) break;
+        }
+        // after a wait gave up: one last bounded look at the copies that may still be in flight (see the prefill kernel)
+        if (dead && lane == 0) {
+            if (q_loads > 0) mbar_drain(bar(&bars.q_full), (q_loads - 1u) & 1u, kDrainLimit);
+            for (int t = max(0, k_issued - KS); t < k_issued; ++t)
+                mbar_drain(bar(&bars.k_full[t % KS]), (uint32_t)(t / KS) & 1u, kDrainLimit);
+            for (int t = max(0, v_issued - KS); t < v_issued; ++t)
+                mbar_drain(bar(&bars.v_full[t % KS]), (uint32_t)(t / KS) & 1u, kDrainLimit);
         }
     } else if (warp == 5) {
         // ------------------------------------------------------------ MMA issuer (whole warp, one lane issues)
-        const uint32_t leader = (lane == 0);
+        uint32_t leader = (lane == 0);   // cleared once a wait has given up
         constexpr uint32_t idesc_qk = instr_desc(kTileM, kTileN, false);
         constexpr uint32_t idesc_pv = instr_desc(kTileM, D, true);
         constexpr uint32_t kTile16 = kTileBytes >> 4;
@@ -869,10 +905,12 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
         };
         for (int u = blockIdx.x; u < n_units; u += gridDim.x) {
             const int t_last = unit(u).w / 8 - 1;      // tiles 0 .. t_last
-            mbar_wait(bar(&bars.q_full), q_uses & 1u, dead, ix.status);
+            tc_wait(bar(&bars.q_full), q_uses & 1u, dead, ix.status);
+            if (dead) leader = 0u;
             ++q_uses;
             for (int i = 0; i < NBUF && i <= t_last; ++i) {
-                mbar_wait(bar(&bars.k_full[(kt0 + i) % KS]), (uint32_t)((kt0 + i) / KS) & 1u, dead, ix.status);
+                tc_wait(bar(&bars.k_full[(kt0 + i) % KS]), (uint32_t)((kt0 + i) / KS) & 1u, dead, ix.status);
+                if (dead) leader = 0u;
                 tc_fence_after();
                 qk(i, kt0 + i);
             }
@@ -880,8 +918,9 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
             int buf = 0;
             for (int j = 0; j <= t_last; ++j) {
                 const int kt = kt0 + j;
-                mbar_wait(bar(&bars.v_full[kt % KS]), (uint32_t)(kt / KS) & 1u, dead, ix.status);
-                mbar_wait(bar(&bars.p_full[n_pv & 3u]), (n_pv >> 2) & 1u, dead, ix.status);
+                tc_wait(bar(&bars.v_full[kt % KS]), (uint32_t)(kt / KS) & 1u, dead, ix.status);
+                tc_wait(bar(&bars.p_full[n_pv & 3u]), (n_pv >> 2) & 1u, dead, ix.status);
+                if (dead) leader = 0u;
                 ++n_pv;
                 tc_fence_after();
                 const uint32_t bv = v_lo + (kt % KS) * kTile16, d_tmem = tmem + kColO, a_tmem = tmem + buf * 128;
@@ -890,7 +929,8 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                     tc_mma_ts_lo(d_tmem, a_tmem + k * 8, bv + k * (2048 >> 4), pv_hi, idesc_pv, k > 0 ? 1u : (uint32_t)(j > 0), leader);
                 tc_commit(bar(&bars.v_empty[kt % KS]), leader);
                 if (j + NBUF <= t_last) {
-                    mbar_wait(bar(&bars.k_full[(kt + NBUF) % KS]), (uint32_t)((kt + NBUF) / KS) & 1u, dead, ix.status);
+                    tc_wait(bar(&bars.k_full[(kt + NBUF) % KS]), (uint32_t)((kt + NBUF) / KS) & 1u, dead, ix.status);
+                    if (dead) leader = 0u;
                     tc_fence_after();
                     qk(buf, kt + NBUF);
                     if (j + NBUF == t_last) tc_commit(bar(&bars.q_empty), leader);
@@ -899,6 +939,12 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
             }
             tc_commit(bar(&bars.pv_done), leader);
             kt0 += t_last + 1;
+        }
+        // after a wait gave up: track the MMAs still queued, so that the tensor memory is not freed under them
+        if (__shfl_sync(0xffffffffu, (int)dead, 0) != 0) {
+            tc_commit(bar(&bars.drain), (uint32_t)(lane == 0));
+            if (lane == 0) mbar_drain(bar(&bars.drain), 0u, kDrainLimit);
+            __syncwarp();
         }
     } else if (warp < 4) {
         // ------------------------------------------------------------ softmax + partial write-out (thread r owns row r)
@@ -918,7 +964,7 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
             int buf = 0;
             for (int j = 0; j < n_tiles; ++j, ++n_steps) {
                 const uint32_t t_s = tmem + lane_addr + buf * 128;
-                mbar_wait(bar(&bars.s_full[n_steps & 3u]), (n_steps >> 2) & 1u, dead, ix.status);
+                tc_wait(bar(&bars.s_full[n_steps & 3u]), (n_steps >> 2) & 1u, dead, ix.status);
                 tc_fence_after();
                 const bool visible = tile0 + j < vis_tiles;
                 uint32_t sv[4][32];
@@ -947,7 +993,7 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                 }
                 if (j > 0 && __any_sync(0xffffffffu, alpha != 1.f)) {
                     const int kt = kt0 + j - 1;   // O must hold every earlier tile: V tile j-1 is released behind PV(j-1)
-                    mbar_wait(bar(&bars.v_empty[kt % KS]), (uint32_t)(kt / KS) & 1u, dead, ix.status);
+                    tc_wait(bar(&bars.v_empty[kt % KS]), (uint32_t)(kt / KS) & 1u, dead, ix.status);
                     tc_fence_after();
 #pragma unroll
                     for (int c = 0; c < D / 32; ++c) {
@@ -981,7 +1027,7 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                 if (++buf == NBUF) buf = 0;
             }
             // ---- the row's partial: (reference max, sum) and the unnormalised accumulator
-            mbar_wait(bar(&bars.pv_done), n_units_done & 1u, dead, ix.status);
+            tc_wait(bar(&bars.pv_done), n_units_done & 1u, dead, ix.status);
             ++n_units_done;
             tc_fence_after();
             const bool write = real && !dead && m_used != -INFINITY;
@@ -1059,17 +1105,19 @@ bool make_pool_map(CUtensorMap* map, const void* ptr, int64_t rows, int64_t cols
 
 template <int D>
 int launch_prefill_tc(const cpa_plan* plan, const void* q, const void* k, const void* v, void* o, const void* k_pool,
-                      const void* v_pool, cudaStream_t st) {
+                      const void* v_pool, const int32_t* items, const int32_t* sched, int ctas, int rounds,
+                      cudaStream_t st) {
     const cpa_config& c = plan->cfg;
     constexpr int smem = TcShape<D>::kSmem;
-    static bool configured_dev[64] = {};  // the attribute is per device: remember which devices have it
+    // the attribute is per device: remember which devices have it (relaxed flags: setting it twice is harmless)
+    static std::atomic<bool> configured_dev[64];
     int dev_id = 0;
     if (cudaGetDevice(&dev_id) != cudaSuccess || dev_id < 0 || dev_id >= 64) {
         (void)cudaGetLastError();
         return CPA_ECUDA;
     }
-    bool& configured = configured_dev[dev_id];
-    if (!configured) {
+    std::atomic<bool>& configured = configured_dev[dev_id];
+    if (!configured.load(std::memory_order_relaxed)) {
         cudaFuncAttributes attr;
         if (cudaFuncGetAttributes(&attr, prefill_tc_kernel<D>) != cudaSuccess ||
             cudaFuncSetAttribute(prefill_tc_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) {
@@ -1079,7 +1127,7 @@ int launch_prefill_tc(const cpa_plan* plan, const void* q, const void* k, const 
         // The in-kernel register split may only hand out what the launch allocates; a kernel
         // that asked for more would wait for registers forever, so refuse to launch it.
         if (attr.numRegs * kThreads < 2 * 128 * kRegsSoftmax + 128 * kRegsControl) return CPA_EUNSUPPORTED;
-        configured = true;
+        configured.store(true, std::memory_order_relaxed);
     }
     CUtensorMap tm_q, tm_k, tm_v;
     if (!make_map(&tm_q, q, plan->total_tokens, (int64_t)c.num_q_heads * D) ||
@@ -1093,11 +1141,20 @@ int launch_prefill_tc(const cpa_plan* plan, const void* q, const void* k, const 
         if (!make_pool_map(&tm_kpool, k_pool, pool_rows, D) || !make_pool_map(&tm_vpool, v_pool, pool_rows, D))
             return CPA_ECUDA;
     }
-    // persistent grid: one CTA per SM, each walks its column of the planner's schedule
-    prefill_tc_kernel<D><<<plan->prefill_ctas, kThreads, smem, st>>>(tm_q, tm_k, tm_v, tm_kpool, tm_vpool,
-                                                                   (__nv_bfloat16*)o, plan->dev(), c.num_q_heads,
-                                                                   c.num_kv_heads, plan->q_tile,
-                                                                   c.scale * 1.4426950408889634f, plan->prefill_rounds);
+    // persistent grid: one CTA per SM, each walks its column of the planner's schedule (the plan's whole-block
+    // list, or the list of one chunk step)
+    cpa_dev_index ix = plan->dev();
+    if (items) {
+        ix.prefill_items = items;
+        ix.prefill_sched = sched;
+    } else {
+        ctas = plan->prefill_ctas;
+        rounds = plan->prefill_rounds;
+    }
+    if (ctas < 1) return CPA_OK;   // nothing to prefill
+    prefill_tc_kernel<D><<<ctas, kThreads, smem, st>>>(tm_q, tm_k, tm_v, tm_kpool, tm_vpool, (__nv_bfloat16*)o, ix,
+                                                     c.num_q_heads, c.num_kv_heads, plan->q_tile,
+                                                     c.scale * 1.4426950408889634f, rounds);
     return cudaGetLastError() == cudaSuccess ? CPA_OK : CPA_ECUDA;
 }
 
@@ -1120,18 +1177,18 @@ int launch_scan_tc(const cpa_plan* plan, const void* q, const void* k_pool, cons
                    float* part_o, cudaStream_t st) {
     const cpa_config& c = plan->cfg;
     constexpr int smem = ScanShape<D>::kSmem;
-    static bool configured_dev[64] = {};
+    static std::atomic<bool> configured_dev[64];
     int dev_id = 0;
     if (cudaGetDevice(&dev_id) != cudaSuccess || dev_id < 0 || dev_id >= 64) {
         (void)cudaGetLastError();
         return CPA_ECUDA;
     }
-    if (!configured_dev[dev_id]) {
+    if (!configured_dev[dev_id].load(std::memory_order_relaxed)) {
         if (cudaFuncSetAttribute(scan_tc_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) {
             (void)cudaGetLastError();
             return CPA_ECUDA;
         }
-        configured_dev[dev_id] = true;
+        configured_dev[dev_id].store(true, std::memory_order_relaxed);
     }
     const int G = c.num_q_heads / c.num_kv_heads;
     if (8 % G != 0) return CPA_EUNSUPPORTED;   // the query tile is loaded in boxes of 8/G sequences
@@ -1140,7 +1197,7 @@ int launch_scan_tc(const cpa_plan* plan, const void* q, const void* k_pool, cons
     if (!make_q_rows_map(&tm_q, q, plan->B, c.num_q_heads, D, G) ||
         !make_pool_map(&tm_kpool, k_pool, pool_rows, D) || !make_pool_map(&tm_vpool, v_pool, pool_rows, D))
         return CPA_ECUDA;
-    const int sms = c.num_sms ? c.num_sms : 148;
+    const int sms = plan->num_sms;
     const int grid = plan->n_shared < sms ? plan->n_shared : sms;
     scan_tc_kernel<D><<<grid, kScanThreads, smem, st>>>(tm_q, tm_kpool, tm_vpool, part_ml, part_o, plan->dev(),
                                                        c.num_q_heads, c.num_kv_heads, G, c.scale * 1.4426950408889634f,
@@ -1157,9 +1214,15 @@ int cpa_scan_tc(const cpa_plan* plan, const void* q, const void* k_pool, const v
                                      : launch_scan_tc<64>(plan, q, k_pool, v_pool, part_ml, part_o, st);
 }
 
+int cpa_prefill_tc_list(const cpa_plan* plan, const void* q, const void* k, const void* v, void* o, const void* k_pool,
+                        const void* v_pool, const int32_t* items, const int32_t* sched, int ctas, int rounds, void* stream) {
+    cudaStream_t st = (cudaStream_t)stream;
+    return plan->cfg.head_dim == 128
+               ? launch_prefill_tc<128>(plan, q, k, v, o, k_pool, v_pool, items, sched, ctas, rounds, st)
+               : launch_prefill_tc<64>(plan, q, k, v, o, k_pool, v_pool, items, sched, ctas, rounds, st);
+}
+
 int cpa_prefill_tc(const cpa_plan* plan, const void* q, const void* k, const void* v, void* o, const void* k_pool,
                    const void* v_pool, void* stream) {
-    cudaStream_t st = (cudaStream_t)stream;
-    return plan->cfg.head_dim == 128 ? launch_prefill_tc<128>(plan, q, k, v, o, k_pool, v_pool, st)
-                                     : launch_prefill_tc<64>(plan, q, k, v, o, k_pool, v_pool, st);
+    return cpa_prefill_tc_list(plan, q, k, v, o, k_pool, v_pool, nullptr, nullptr, 0, 0, stream);
 }

@@ -39,7 +39,7 @@ class CompactionSession:
                  scale: Optional[float] = None, device: str = "cuda:0", pages_per_split: int = 0,
                  poison_pools: bool = False, page_size: int = 16, q_tile_rows: int = 0,
                  prefix_lens: Optional[Sequence[int]] = None, shared_pages: Optional[Sequence[int]] = None,
-                 pools=None, num_sms: int = 0):
+                 pools=None, num_sms: int = 0, chunk_tokens: int = 0, decode_sms: int = 0, dynamic_pages: bool = False):
         self.device = torch.device(device)
         self.Hq, self.Hkv, self.d, self.P = num_q_heads, num_kv_heads, head_dim, page_size
         self.B = len(block_lens)
@@ -51,7 +51,16 @@ class CompactionSession:
         self.cfg = B.cpa_config(num_q_heads, num_kv_heads, head_dim, page_size, self.scale, q_tile_rows,
                                 pages_per_split, num_sms or props.multi_processor_count)
         self.prefix_aware = prefix_lens is not None
-        if self.prefix_aware:   # the paper's layout: cached history prefix + own tokens per worker
+        self.chunk_tokens = chunk_tokens
+        self.dynamic_pages = dynamic_pages
+        if dynamic_pages:       # no pages reserved for the summaries: blocks draw from a common reserve as they grow
+            assert prefix_lens is None and not chunk_tokens
+            self.plan = B.cpa_plan_create_dynamic(self.cfg, self.block_lens, max_new_tokens, free_pages)
+        elif chunk_tokens:      # prefill in chunks, mixed with the decode of blocks that are past their prompt
+            assert prefix_lens is None
+            self.plan = B.cpa_plan_create_chunked(self.cfg, self.block_lens, max_new_tokens, chunk_tokens, free_pages,
+                                                  decode_sms)
+        elif self.prefix_aware:   # the paper's layout: cached history prefix + own tokens per worker
             self.plan = B.cpa_plan_create_prefix(self.cfg, self.block_lens, prefix_lens, shared_pages,
                                                  max_new_tokens, free_pages)
         else:
@@ -130,6 +139,28 @@ class CompactionSession:
         self._check(B.cpa_decode_append(self.plan, q, k_new, v_new, self.k_pool, self.v_pool, out,
                                         self.workspace, self._stream()), "cpa_decode_append")
         return out
+
+    def step_mixed(self, step: int, q, k, v, out, q_dec=None, k_new=None, v_new=None, out_dec=None) -> None:
+        """Step `step` of a chunked plan: the next prefill chunk of the blocks that have one (rows of the
+        whole-event tensors q/k/v/out) beside one decode token of the blocks whose turn it is."""
+        self._check(B.cpa_step_mixed(self.plan, step, q, k, v, out, q_dec, k_new, v_new, out_dec, self.k_pool,
+                                     self.v_pool, self.workspace, self._stream()), "cpa_step_mixed")
+
+    def decode_append_dynamic(self, q, k_new, v_new, active=None, out=None):
+        """One decode step of a plan with pages on demand; `active` is a device int32 [B] tensor of stop flags."""
+        if out is None:
+            out = torch.empty_like(q)
+        self._check(B.cpa_decode_append_dynamic(self.plan, q, k_new, v_new, active, self.k_pool, self.v_pool, out,
+                                                self.workspace, self._stream()), "cpa_decode_append_dynamic")
+        return out
+
+    def release(self, active) -> None:
+        """Blocks whose flag is 0 give their pages back to the reserve."""
+        self._check(B.cpa_release_blocks(self.plan, active, self._stream()), "cpa_release_blocks")
+
+    def sync(self) -> None:
+        """Read the device's lengths, page table and reserve back into the plan's host copies."""
+        self._check(B.cpa_plan_sync(self.plan, self._stream()), "cpa_plan_sync")
 
     def status(self) -> int:
         return B.cpa_plan_status(self.plan, self._stream())

@@ -58,6 +58,7 @@ class Workload:
     k: Optional[np.ndarray] = None            # uint16 [tokens, Hkv, d]
     v: Optional[np.ndarray] = None
     outlier_pos: Optional[np.ndarray] = None  # int64 [B] position inside each block
+    stop_lens: Optional[np.ndarray] = None    # int32 [B] tokens each sequence decodes before it stops (None: all T)
     q_dec: Optional[np.ndarray] = None        # uint16 [T, B, Hq, d]
     k_dec: Optional[np.ndarray] = None        # uint16 [T, B, Hkv, d]
     v_dec: Optional[np.ndarray] = None
@@ -153,6 +154,19 @@ def split_sweep(num_blocks: int, seed: int = 4, history: int = 131072, steps: in
     return _mk(f"split{num_blocks}", 32, 8, 128, [history // num_blocks] * num_blocks, steps, seed, rng)
 
 
+def locomo_like(seed: int = 6, num_docs: int = 32, questions: int = 6, lo: int = 512, hi: int = 1024,
+                steps: int = 256, min_stop: int = 32) -> Workload:
+    """Many short sequences (the paper's second benchmark feeds documents of about 0.7k tokens with six
+    questions each): num_docs x questions sequences of lo..hi tokens, 32q/8kv, d=128, whose summaries
+    stop at different lengths.  `stop_lens[b]` (drawn last) is the number of tokens sequence b decodes."""
+    rng = np.random.Generator(np.random.PCG64(seed))
+    n = num_docs * questions
+    lens = rng.integers(lo, hi + 1, size=n).astype(np.int32)
+    w = _mk("locomo_like", 32, 8, 128, lens, steps, seed, rng, permute_pages=True)
+    w.stop_lens = np.random.Generator(np.random.PCG64(seed + 7919)).integers(min(min_stop, steps), steps + 1, size=n).astype(np.int32)
+    return w
+
+
 def custom(lens, hq, hkv, d, steps, seed=7, permute_pages=True, outlier_scale=0.0) -> Workload:
     """Arbitrary small shapes for edge-case tests."""
     rng = np.random.Generator(np.random.PCG64(seed))
@@ -225,4 +239,5 @@ CONFIGS = {
     "ragged": ragged,
     "moe120b": moe120b,
     "split": split,
+    "locomo_like": locomo_like,
 }

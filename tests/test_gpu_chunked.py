@@ -1,0 +1,141 @@
+"""Chunked prefill and mixed steps on the CUDA path against the CPU oracle (paper, Section 4.2: the
+serving engine runs with chunked prefill enabled; Section 6: 16k blocks are prefill-bound).  Every step
+prefills the next chunk of the blocks that have one and decodes one token of the blocks whose turn it
+is; the prefill rows must be the rows of the unchunked prefill, the decode outputs those of the
+per-block contiguous cache, the pools bit-exact."""
+import numpy as np
+import pytest
+
+from _util import assert_attention_close, pool_rows
+from oracle import attention as oa
+from oracle import plan as op
+from paper_2605_23296_b200 import workloads as wl
+
+pytestmark = pytest.mark.gpu
+
+
+def _dev(bits):
+    from paper_2605_23296_b200.session import bits_to_tensor
+    return bits_to_tensor(bits, "cuda:0")
+
+
+def _bits(t):
+    from paper_2605_23296_b200.session import tensor_to_bits
+    return tensor_to_bits(t)
+
+
+def _cu(w):
+    return np.concatenate([[0], np.cumsum(w.block_lens.astype(np.int64))])
+
+
+def run_chunked_event(w, chunk, decode_sms=0, rows=None, what=""):
+    """All steps of the schedule through cpa_step_mixed.  Inputs of decode step t of a block are row t of
+    w.*_dec (so a block's t-th summary token has the same inputs whatever step it is produced in)."""
+    import torch
+    from paper_2605_23296_b200 import binding as B
+    from paper_2605_23296_b200.session import CompactionSession
+    w.materialise()
+    T, Bn = w.decode_steps, w.num_blocks
+    s = CompactionSession(w.block_lens, T, w.num_q_heads, w.num_kv_heads, w.head_dim, w.free_pages, w.num_pages,
+                          scale=w.scale, poison_pools=True, chunk_tokens=chunk, decode_sms=decode_sms)
+    sched = op.mixed_schedule(w.block_lens.tolist(), chunk, T)
+    assert s.param(B.PARAM_NUM_STEPS) == len(sched)
+    start = s.export(B.ARR_DEC_START)
+    q, k, v = _dev(w.q), _dev(w.k), _dev(w.v)
+    o = torch.full_like(q, 7.0)
+    qd, kd, vd = (_dev(w.q_dec), _dev(w.k_dec), _dev(w.v_dec)) if T else (None, None, None)
+    dec_out = {}
+    cu = _cu(w)
+    for step, st in enumerate(sched):
+        # this step's decode inputs: block b is at its token t = step - start[b]
+        act = st["decode"]
+        q_in = torch.zeros((Bn, w.num_q_heads, w.head_dim), dtype=torch.bfloat16, device="cuda:0")
+        k_in = torch.zeros((Bn, w.num_kv_heads, w.head_dim), dtype=torch.bfloat16, device="cuda:0")
+        v_in = torch.zeros_like(k_in)
+        for b in act:
+            t = step - int(start[b])
+            q_in[b], k_in[b], v_in[b] = qd[t, b], kd[t, b], vd[t, b]
+        out = torch.full_like(q_in, 5.0)
+        s.step_mixed(step, q, k, v, o, q_in, k_in, v_in, out)
+        got = _bits(out)
+        for b in range(Bn):
+            if b in act:
+                dec_out[(step, b)] = got[b]
+            else:
+                assert (out[b] == 5.0).all(), f"{what}: step {step} wrote the output row of idle block {b}"
+    assert s.status() == 0
+    from paper_2605_23296_b200 import binding as B2
+    # out of order: the schedule is over
+    assert B2.cpa_step_mixed(s.plan, 0, q, k, v, o, q_in, k_in, v_in, out, s.k_pool, s.v_pool, s.workspace) == B2.CPA_ESTATE
+
+    # ---- prefill rows = the rows of the unchunked prefill
+    if rows is None:
+        assert_attention_close(_bits(o), oa.prefill(w.q, w.k, w.v, cu, w.scale), f"{what} chunked prefill")
+    else:
+        got = _bits(o[torch.from_numpy(rows).to("cuda:0")])
+        assert_attention_close(got, oa.prefill(w.q, w.k, w.v, cu, w.scale, rows=rows), f"{what} chunked prefill (sampled rows)")
+    # ---- decode: block b's token t over its contiguous cache
+    state = oa.DecodeState(w.k, w.v, cu, T)
+    for t in range(T):
+        state.append(w.k_dec[t], w.v_dec[t])
+        want = state.decode(w.q_dec[t], w.scale)
+        for b in range(Bn):
+            assert_attention_close(dec_out[(int(start[b]) + t, b)], want[b], f"{what} block {b} token {t}")
+    # ---- pools: every token in its slot, bit for bit; lengths
+    plan = op.build_plan(w.block_lens.tolist(), T, w.page_size, w.free_pages.tolist(), w.num_kv_heads, 128, 1)
+    slots = list(plan["slot_mapping"])
+    ks, vs = [w.k], [w.v]
+    for t in range(T):
+        slots += [op.slot_of(plan, w.page_size, b, int(w.block_lens[b]) + t) for b in range(Bn)]
+        ks.append(w.k_dec[t])
+        vs.append(w.v_dec[t])
+    if T or rows is None:
+        kp, vp, written = oa.expected_pool(slots, np.concatenate(ks), np.concatenate(vs), w.num_pages, w.page_size)
+        mask = np.broadcast_to(written[:, None, :, None], kp.shape)
+        assert np.array_equal(pool_rows(_bits(s.k_pool))[mask], kp[mask])
+        assert np.array_equal(pool_rows(_bits(s.v_pool))[mask], vp[mask])
+    assert np.array_equal(s.export(B.ARR_SEQ_LENS), w.block_lens + T)
+    s.close()
+
+
+@pytest.mark.parametrize("hq,hkv,d", [(8, 2, 64), (8, 2, 128), (4, 4, 128)])
+def test_chunks_of_one_tile(hq, hkv, d):
+    # the hand-worked shape plus a block that ends one token into its second chunk
+    run_chunked_event(wl.custom([300, 100, 50, 129], hq, hkv, d, steps=3, seed=hq + d), 128, what=f"chunk 128 {hq}/{hkv}/{d}")
+
+
+def test_chunks_of_three_tiles_and_a_small_decode_share():
+    # 384-token chunks: a 256-row item and a 128-row item per chunk; one SM for the decode wave
+    run_chunked_event(wl.custom([1000, 400, 385, 7], 8, 2, 128, steps=4, seed=77), 384, decode_sms=1, what="chunk 384")
+
+
+def test_one_chunk_covers_every_block():
+    # chunk longer than every block: step 0 is the whole prefill, then plain decode steps
+    run_chunked_event(wl.tiny(4), 512, what="tiny, one chunk")
+
+
+def test_no_decode_steps():
+    run_chunked_event(wl.custom([700, 130], 8, 2, 128, steps=0, seed=78), 256, what="T = 0")
+
+
+def test_long_block_beside_short_ones_sampled_rows():
+    # the case chunking is for: a 16k block next to four 2k blocks (8B-class heads), 2048-token chunks;
+    # the short blocks decode while the long one is still prefilling
+    w = wl.custom([16384, 2048, 2048, 2048, 2048], 32, 8, 128, steps=10, seed=79, permute_pages=True).materialise()
+    rng = np.random.default_rng(79)
+    cu = _cu(w)
+    rows = []
+    for b, L in enumerate(int(x) for x in w.block_lens):
+        cand = {0, 1, L - 1} | {c for t in range(2048, L, 2048) for c in (t - 1, t, t + 1)} | set(int(x) for x in rng.integers(0, L, 10))
+        rows += [cu[b] + r for r in sorted(cand) if 0 <= r < L]
+    run_chunked_event(w, 2048, rows=np.asarray(rows, dtype=np.int64), what="16k + 4 x 2k")
+
+
+def test_mixed_step_needs_a_chunked_plan():
+    from paper_2605_23296_b200 import binding as B
+    from paper_2605_23296_b200.session import CompactionSession
+    w = wl.tiny(2).materialise()
+    s = CompactionSession(w.block_lens, 2, w.num_q_heads, w.num_kv_heads, w.head_dim, w.free_pages, w.num_pages)
+    q = _dev(w.q)
+    assert B.cpa_step_mixed(s.plan, 0, q, q, q, q, None, None, None, None, s.k_pool, s.v_pool, s.workspace) == B.CPA_ESTATE
+    s.close()

@@ -49,10 +49,35 @@ def test_single_rank_needs_no_process_group():
     assert bench.max_over_ranks(3.5, 1, "cpu") == 3.5
 
 
+def test_gpus_flag_means_that_many_ranks():
+    sys.path.insert(0, ROOT)
+    import bench
+    # started by a launcher: --gpus must agree with it
+    assert bench.rank_layout(2, {"WORLD_SIZE": "2", "RANK": "1", "LOCAL_RANK": "1"}) == ("run", 1, 2, 1)
+    with pytest.raises(SystemExit):
+        bench.rank_layout(8, {"WORLD_SIZE": "2", "RANK": "0", "LOCAL_RANK": "0"})
+    with pytest.raises(SystemExit):
+        bench.rank_layout(1, {"WORLD_SIZE": "2", "RANK": "0", "LOCAL_RANK": "0"})
+    # started bare: one GPU runs in place, more GPUs start one rank each through torch's launcher
+    assert bench.rank_layout(1, {}) == ("run", 0, 1, 0)
+    kind, argv = bench.rank_layout(4, {})
+    assert kind == "spawn" and "--nproc-per-node=4" in argv and "127.0.0.1" in argv
+    assert argv[argv.index("-m") + 1] == "torch.distributed.run"
+    # the reference arm is rank 0's host cores whatever --gpus says
+    assert bench.rank_layout(8, {}, impl="reference") == ("run", 0, 1, 0)
+
+
+def test_bare_launch_with_a_mismatching_world_size_fails_loudly():
+    env = dict(os.environ, RANK="0", WORLD_SIZE="2", LOCAL_RANK="0")
+    r = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "4", "--config", "tiny"],
+                       env=env, capture_output=True, text=True, timeout=300)
+    assert r.returncode != 0 and "WORLD_SIZE" in (r.stderr + r.stdout)
+
+
 def test_reference_arm_runs_on_rank_zero_only():
     env = dict(os.environ, RANK="1", WORLD_SIZE="2")
     cmd = [sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--config", "tiny",
-           "--steps", "1", "--warmup", "0"]
+           "--gpus", "2", "--steps", "1", "--warmup", "0"]
     r = subprocess.run(cmd, env=env, capture_output=True, text=True, timeout=300)
     assert r.returncode == 0 and r.stdout.strip() == ""
     env["RANK"] = "0"

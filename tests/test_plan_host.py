@@ -196,6 +196,101 @@ def test_library_exports_every_declared_symbol():
         assert hasattr(lib, n), n
 
 
+# ----------------------------------------------------------------------------
+# chunked prefill: the steps of the schedule
+# ----------------------------------------------------------------------------
+
+@pytest.mark.parametrize("lens,C,T", [([300, 100, 50], 128, 2), ([16384, 2048, 2048, 2048, 2048], 2048, 256),
+                                       ([1, 129, 128, 1000], 128, 3), ([700], 256, 0)])
+def test_chunked_plan_steps_bit_exact(lens, C, T):
+    cfg = B.cpa_config(8, 2, 128, 16, 0.088, 0, 0, 0)
+    pages = sum(-(-(L + T) // 16) for L in lens)
+    plan = B.cpa_plan_create_chunked(cfg, lens, T, C, np.arange(pages, dtype=np.int32))
+    try:
+        ref = op.mixed_schedule(lens, C, T)
+        assert B.cpa_plan_param(plan, B.PARAM_NUM_STEPS) == len(ref)
+        assert B.cpa_plan_param(plan, B.PARAM_CHUNK_TOKENS) == C
+        n_chunk_steps = B.cpa_plan_param(plan, B.PARAM_CHUNK_STEPS)
+        assert n_chunk_steps == sum(1 for st in ref if st["prefill"])
+        start = B.cpa_plan_export(plan, B.ARR_DEC_START).tolist()
+        rows = B.cpa_plan_export(plan, B.ARR_CHUNK_ROWS).reshape(n_chunk_steps, len(lens) + 1)
+        for s, st in enumerate(ref):
+            assert [b for b in range(len(lens)) if 0 <= s - start[b] < T] == st["decode"]
+            if s < n_chunk_steps:
+                per_block = np.diff(rows[s]).tolist()
+                want = [0] * len(lens)
+                for b, first, n in st["prefill"]:
+                    assert first == s * C
+                    want[b] = n
+                assert per_block == want and rows[s][0] == 0
+        # everything the whole-block calls use is the ordinary plan's
+        plain = B.cpa_plan_create(cfg, lens, T, np.arange(pages, dtype=np.int32))
+        for which in (B.ARR_CU_SEQLENS, B.ARR_PAGE_INDICES, B.ARR_SLOT_MAPPING, B.ARR_PREFILL_ITEMS, B.ARR_DECODE_ITEMS):
+            assert np.array_equal(B.cpa_plan_export(plan, which), B.cpa_plan_export(plain, which))
+        B.cpa_plan_destroy(plain)
+        sms = B.cpa_plan_param(plan, B.PARAM_NUM_SMS)
+        assert 1 <= B.cpa_plan_param(plan, B.PARAM_DECODE_SMS) < sms
+    finally:
+        B.cpa_plan_destroy(plan)
+
+
+def test_chunked_plan_errors():
+    cfg = B.cpa_config(8, 2, 64, 16, 0.125, 0, 0, 0)
+    free = np.arange(100, dtype=np.int32)
+    for chunk in (0, 64, 200, -128):
+        rc, h = B.cpa_plan_create_chunked(cfg, (300, 50), 2, chunk, free, check=False)
+        assert rc == B.CPA_EINVAL and not h
+    rc, h = B.cpa_plan_create_chunked(cfg, (300, 50), 2, 128, free, decode_sms=4096, check=False)
+    assert rc == B.CPA_EINVAL and not h
+    rc, h = B.cpa_plan_create_chunked(cfg, (300, 0), 2, 128, free, check=False)
+    assert rc == B.CPA_EINVAL and not h
+    fake = 4096
+    plan = B.cpa_plan_create_chunked(cfg, (300, 50), 2, 128, free)
+    assert B.cpa_step_mixed(plan, 0, fake, fake, fake, fake + 16, fake, fake, fake, fake, fake, fake, fake) == B.CPA_ESTATE  # not uploaded
+    B.cpa_plan_destroy(plan)
+
+
+# ----------------------------------------------------------------------------
+# pages on demand: the first assignment
+# ----------------------------------------------------------------------------
+
+def test_dynamic_plan_first_assignment_matches_the_model():
+    lens = [5, 16, 17, 300, 31, 32]
+    T, P = 40, 16
+    free = np.random.default_rng(3).permutation(80).astype(np.int32)
+    cfg = B.cpa_config(8, 2, 128, P, 0.088, 0, 0, 0)
+    plan = B.cpa_plan_create_dynamic(cfg, lens, T, free)
+    try:
+        m = op.DynamicPages(lens, T, P, free.tolist())
+        assert B.cpa_plan_export(plan, B.ARR_PAGES_ASSIGNED).tolist() == m.pages
+        indptr, idx = B.cpa_plan_export(plan, B.ARR_PAGE_INDPTR), B.cpa_plan_export(plan, B.ARR_PAGE_INDICES)
+        assert np.diff(indptr).tolist() == m.cap                       # a row per block, as long as the block may grow
+        assert [idx[indptr[b]:indptr[b] + m.pages[b]].tolist() for b in range(len(lens))] == m.initial
+        ring = B.cpa_plan_export(plan, B.ARR_FREE_RING).tolist()
+        assert ring == free[sum(m.pages):].tolist()                    # the rest, in free-list order
+        assert B.cpa_plan_param(plan, B.PARAM_PAGES_USED) == sum(m.pages)
+        # the prefill tokens' slots are those of an ordinary plan over the same first pages
+        slots = B.cpa_plan_export(plan, B.ARR_SLOT_MAPPING)
+        cu = np.concatenate([[0], np.cumsum(lens)])
+        for b, L in enumerate(lens):
+            for i in (0, L // 2, L - 1):
+                assert slots[cu[b] + i] == m.initial[b][i // P] * P + i % P
+        m.check([idx[indptr[b]:indptr[b + 1]].tolist() for b in range(len(lens))], m.pages, lens, ring)
+    finally:
+        B.cpa_plan_destroy(plan)
+    # the free list must cover the first pages; nothing beyond them is needed up front
+    need = sum(L // P + 1 for L in lens)
+    rc, h = B.cpa_plan_create_dynamic(cfg, lens, T, free[:need - 1], check=False)
+    assert rc == B.CPA_ENOSPC and not h
+    plan = B.cpa_plan_create_dynamic(cfg, lens, T, free[:need])
+    assert len(B.cpa_plan_export(plan, B.ARR_FREE_RING)) == 0
+    fake = 4096
+    assert B.cpa_decode_append_dynamic(plan, fake, fake, fake, None, fake, fake, fake, fake) == B.CPA_ESTATE   # not uploaded
+    assert B.cpa_release_blocks(plan, fake) == B.CPA_ESTATE
+    assert B.cpa_plan_sync(plan) == B.CPA_ESTATE
+    B.cpa_plan_destroy(plan)
+
+
 def test_probe_library_is_separate_and_exports_its_entry_point():
     import ctypes
     from paper_2605_23296_b200 import build
