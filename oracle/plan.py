@@ -23,8 +23,8 @@ stated in full):
 * chunked prefill (Section 4.2: the serving engine runs with chunked prefill enabled; the
                   paper gives no rule, this one is the library's reading) a block of L_b
                   tokens is prefilled in ceil(L_b / C) chunks of C tokens (the last one
-                  short), one chunk per step, and decodes its T summary tokens in the T
-                  steps right after its last chunk; see mixed_schedule
+                  short), a chunk every r steps, and decodes its T summary tokens in the T
+                  steps after its last chunk's r steps; see mixed_schedule
 * pages on demand (Section 8, "Dynamic block size and prompt selection": summaries of unknown
                   length) instead of reserving pages for T tokens per block, a block holds
                   pages for the tokens it has plus the next one; the rest of the free list is
@@ -142,27 +142,33 @@ def build_plan(block_lens: Sequence[int], max_new_tokens: int, page_size: int,
     }
 
 
-def mixed_schedule(block_lens: Sequence[int], chunk_tokens: int, max_new_tokens: int):
+def mixed_schedule(block_lens: Sequence[int], chunk_tokens: int, max_new_tokens: int, decode_steps_per_chunk: int = 1):
     """Steps of one event with chunked prefill (Section 4.2: chunked prefill is enabled in the paper's
     serving engine, so a long block's prefill is cut into chunks that share steps with the decode of
     blocks that are already past their prefill; Section 6 is why it matters: 16k blocks are
-    prefill-bound).  Rule, stated in full because the paper gives none:
+    prefill-bound).  Rule, stated in full because the paper gives none (C = chunk_tokens,
+    r = decode_steps_per_chunk: a chunk costs about as much as r decode steps, so the blocks that
+    decode take r tokens while a chunk is prefilled beside them):
 
-      step s prefills rows [s*C, min((s+1)*C, L_b)) of every block b with s < n_b = ceil(L_b / C);
-      block b decodes summary token t at step n_b + t, t = 0 .. T-1;
-      the event has max_b(n_b) + T steps.
+      chunk c of block b, rows [c*C, min((c+1)*C, L_b)), starts at step c*r, for c < n_b = ceil(L_b / C);
+      block b decodes summary token t at step n_b*r + t, t = 0 .. T-1;
+      the event has max_b(n_b)*r + T steps.
 
     Returns a list with one entry per step: {"prefill": [(block, first_row, rows)], "decode": [blocks]},
-    both in ascending block order.
+    both in ascending block order ("prefill" is empty in steps that start no chunk).
     """
-    if chunk_tokens < 1 or max_new_tokens < 0 or not len(block_lens) or any(int(L) < 1 for L in block_lens):
+    r = decode_steps_per_chunk
+    if chunk_tokens < 1 or max_new_tokens < 0 or r < 1 or not len(block_lens) or any(int(L) < 1 for L in block_lens):
         raise ValueError("bad parameter")
     n_chunks = [-(-int(L) // chunk_tokens) for L in block_lens]
     steps = []
-    for s in range(max(n_chunks) + max_new_tokens):
-        pre = [(b, s * chunk_tokens, min(chunk_tokens, int(L) - s * chunk_tokens))
-               for b, L in enumerate(block_lens) if s < n_chunks[b]]
-        dec = [b for b in range(len(block_lens)) if n_chunks[b] <= s < n_chunks[b] + max_new_tokens]
+    for s in range(max(n_chunks) * r + max_new_tokens):
+        pre = []
+        if s % r == 0:
+            c = s // r
+            pre = [(b, c * chunk_tokens, min(chunk_tokens, int(L) - c * chunk_tokens))
+                   for b, L in enumerate(block_lens) if c < n_chunks[b]]
+        dec = [b for b in range(len(block_lens)) if n_chunks[b] * r <= s < n_chunks[b] * r + max_new_tokens]
         steps.append({"prefill": pre, "decode": dec})
     return steps
 

@@ -32,30 +32,40 @@ def _read_golden():
 
 def test_mixed_schedule_matches_the_hand_worked_table():
     head, steps = _read_golden()
-    got = op.mixed_schedule(head["block_lens"], head["chunk_tokens"][0], head["max_new_tokens"][0])
+    got = op.mixed_schedule(head["block_lens"], head["chunk_tokens"][0], head["max_new_tokens"][0],
+                            head["decode_steps_per_chunk"][0])
     assert got == steps
+    # one decode step per chunk: the same chunks and decoders without the steps in between
+    lock = op.mixed_schedule(head["block_lens"], head["chunk_tokens"][0], 2, 1)
+    assert lock == [{"prefill": [(0, 0, 128), (1, 0, 100), (2, 0, 50)], "decode": []},
+                    {"prefill": [(0, 128, 128)], "decode": [1, 2]}, {"prefill": [(0, 256, 44)], "decode": [1, 2]},
+                    {"prefill": [], "decode": [0]}, {"prefill": [], "decode": [0]}]
 
 
-@pytest.mark.parametrize("lens,C,T", [([16384, 2048, 2048, 2048, 2048], 2048, 256), ([1, 129, 128, 1000], 128, 3),
-                                       ([700], 256, 0), ([5, 5, 5], 1024, 4)])
-def test_mixed_schedule_invariants(lens, C, T):
-    steps = op.mixed_schedule(lens, C, T)
+@pytest.mark.parametrize("lens,C,T,r", [([16384, 2048, 2048, 2048, 2048], 2048, 256, 1), ([1, 129, 128, 1000], 128, 3, 1),
+                                         ([700], 256, 0, 1), ([5, 5, 5], 1024, 4, 1), ([16384, 2048, 2048], 2048, 40, 16),
+                                         ([300, 100, 50], 128, 2, 3)])
+def test_mixed_schedule_invariants(lens, C, T, r):
+    steps = op.mixed_schedule(lens, C, T, r)
     rows_done = [0] * len(lens)
+    last_chunk_step = [None] * len(lens)
     decoded = [[] for _ in lens]
     for s, st in enumerate(steps):
+        assert not st["prefill"] or s % r == 0                    # a chunk starts every r steps
         for b, first, n in st["prefill"]:
             assert first == rows_done[b] and 1 <= n <= C          # chunks in order, nothing skipped or repeated
             assert n == C or first + n == lens[b]                 # only a block's last chunk is short
             rows_done[b] += n
+            last_chunk_step[b] = s
         for b in st["decode"]:
-            assert rows_done[b] == lens[b]                        # a block decodes only after its whole prefill
-            assert b not in [x[0] for x in st["prefill"]]
+            assert rows_done[b] == lens[b]                        # a block decodes only after its whole prefill ...
+            assert s >= last_chunk_step[b] + r                    # ... has had its r steps
             decoded[b].append(s)
     assert rows_done == list(lens)
     for b, d in enumerate(decoded):
-        assert len(d) == T and d == list(range(-(-lens[b] // C), -(-lens[b] // C) + T))   # T steps in a row, at once
-    assert len(steps) == max(-(-L // C) for L in lens) + T
-    assert steps[-1]["prefill"] or steps[-1]["decode"]            # no empty step at the end
+        n_b = -(-lens[b] // C)
+        assert len(d) == T and d == list(range(n_b * r, n_b * r + T))   # T steps in a row, at once
+    assert len(steps) == max(-(-L // C) for L in lens) * r + T
 
 
 def test_mixed_schedule_with_one_chunk_is_prefill_then_decode():
@@ -66,7 +76,7 @@ def test_mixed_schedule_with_one_chunk_is_prefill_then_decode():
 
 
 def test_mixed_schedule_rejects_bad_input():
-    for args in [([10], 0, 1), ([10], 8, -1), ([], 8, 1), ([0], 8, 1)]:
+    for args in [([10], 0, 1), ([10], 8, -1), ([], 8, 1), ([0], 8, 1), ([10], 8, 1, 0)]:
         with pytest.raises(ValueError):
             op.mixed_schedule(*args)
 
