@@ -658,7 +658,8 @@ def run_mixed(args) -> None:
     def chunked():
         ev = {n: new_ev() for n in ("start", "first", "short_done", "long_prefilled", "end")}
         s = CompactionSession(w.block_lens, T, w.num_q_heads, w.num_kv_heads, w.head_dim, w.free_pages, w.num_pages,
-                              scale=w.scale, chunk_tokens=chunk, decode_sms=args.decode_sms)
+                              scale=w.scale, chunk_tokens=chunk, decode_sms=args.decode_sms,
+                              decode_steps_per_chunk=args.steps_per_chunk)
         start = s.export(B.ARR_DEC_START)
         n_steps = s.param(B.PARAM_NUM_STEPS)
         n_long = int(start.max())
@@ -674,8 +675,8 @@ def run_mixed(args) -> None:
         ev["start"].record(stream)
         for step in range(n_steps):
             qi, ki, vi = gathered[step]
-            s.step_mixed(step, q, k, v, o, qi, ki, vi, od[min(step, T + 7)])
-            if step == 1:
+            s.step_mixed(step, q, k, v, o, qi, ki, vi, od[step % (T + 8)])
+            if step == int(start.min()):
                 ev["first"].record(stream)
             if step == int(start.min()) + T - 1:
                 ev["short_done"].record(stream)
@@ -700,6 +701,7 @@ def run_mixed(args) -> None:
         "unit": "ms", "n_gpus": 1, "steps": args.steps, "warmup": args.warmup, "dtype": "bf16", "data": "synthetic",
         "config": {"workload": "mixed16k", "block_lens": lens, "q_heads": 32, "kv_heads": 8, "head_dim": 128,
                    "decode_steps": T, "chunk_tokens": chunk, "decode_sms": args.decode_sms or "a quarter of the SMs",
+                   "decode_steps_per_chunk": args.steps_per_chunk,
                    "seed": w.seed},
         "whole_blocks": {"first_summary_token_ms": mean("whole_blocks", "first"),
                          "short_blocks_done_ms": mean("whole_blocks", "end"), "event_ms": mean("whole_blocks", "end")},
@@ -707,6 +709,106 @@ def run_mixed(args) -> None:
                     "short_blocks_done_ms": mean("chunked", "short_done"),
                     "long_block_prefilled_ms": mean("chunked", "long_prefilled"), "event_ms": mean("chunked", "end")},
     }
+    print(json.dumps(out))
+
+
+# ------------------------------------------------------------------------------------------
+# many short sequences with summaries of unknown length (paper, Section 3.1 and Section 8): non-default
+# ------------------------------------------------------------------------------------------
+
+def run_locomo(args) -> None:
+    """`--config locomo`: 192 sequences of 512..1024 tokens (the shape of the paper's second benchmark: short
+    documents, six questions each) whose summaries stop after 32..T tokens.  The plan with pages on demand
+    (stop flags on the device, pages drawn from a common reserve as blocks grow, given back when they stop)
+    against the ordinary plan, which reserves T tokens for every sequence and decodes all of them to the end."""
+    import torch
+
+    from paper_2605_23296_b200 import binding as B
+    from paper_2605_23296_b200.session import CompactionSession, bits_to_tensor
+
+    if args.layout[2] != 1:
+        raise SystemExit("--config locomo is a single-GPU measurement")
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    peaks, peak_kind = load_peaks()
+    w = wl.locomo_like(steps=args.decode_steps or 256).materialise()
+    T, Bn, P = w.decode_steps, w.num_blocks, w.page_size
+    stop = w.stop_lens
+    stream = torch.cuda.current_stream(dev)
+    d = lambda bits: bits_to_tensor(bits, dev)
+    q, k, v, qd, kd, vd = (d(x) for x in (w.q, w.k, w.v, w.q_dec, w.k_dec, w.v_dec))
+    o = torch.empty_like(q)
+    od = torch.empty((T, Bn, w.num_q_heads, w.head_dim), dtype=torch.bfloat16, device=dev)
+    flush = torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device=dev)
+    # stop flags of every step, and of every release point, staged on the device before the timed region
+    steps_idx = np.arange(T)[:, None]
+    flags = torch.from_numpy((steps_idx < stop[None, :]).astype(np.int32)).to(dev)
+    release_every = 32
+    first_pages = int((w.block_lens // P + 1).sum())
+    # the pool: first pages + what the summaries really need (+ a margin), instead of T tokens for everybody
+    need = int((-(-(w.block_lens.astype(np.int64) + stop) // P)).sum())
+    free = w.free_pages[:max(first_pages, need) + 64]
+    new_ev = lambda: torch.cuda.Event(enable_timing=True)
+
+    def reserved():
+        s = CompactionSession(w.block_lens, T, w.num_q_heads, w.num_kv_heads, w.head_dim, w.free_pages, w.num_pages,
+                              scale=w.scale)
+        ev = [new_ev() for _ in range(3)]
+        ev[0].record(stream)
+        s.prefill(q, k, v, out=o)
+        s.append_prefill(k, v)
+        ev[1].record(stream)
+        for t in range(T):
+            s.decode_append(qd[t], kd[t], vd[t], out=od[t])
+        ev[2].record(stream)
+        return s, ev
+
+    def on_demand():
+        s = CompactionSession(w.block_lens, T, w.num_q_heads, w.num_kv_heads, w.head_dim, free, w.num_pages,
+                              scale=w.scale, dynamic_pages=True)
+        ev = [new_ev() for _ in range(3)]
+        ev[0].record(stream)
+        s.prefill(q, k, v, out=o)
+        s.append_prefill(k, v)
+        ev[1].record(stream)
+        for t in range(T):
+            s.decode_append_dynamic(qd[t], kd[t], vd[t], flags[t], out=od[t])
+            if t % release_every == release_every - 1 and t + 1 < T:
+                s.release(flags[t + 1])
+        ev[2].record(stream)
+        return s, ev
+
+    res = {"reserved": [], "on_demand": []}
+    pages_end = None
+    for i in range(args.warmup + args.steps):
+        for name, fn in (("reserved", reserved), ("on_demand", on_demand)):
+            flush.fill_(1)
+            s, ev = fn()
+            torch.cuda.synchronize(dev)
+            assert s.status() == 0
+            if name == "on_demand":
+                s.sync()
+                pages_end = int(s.export(B.ARR_PAGES_ASSIGNED).sum())
+            s.close()
+            if i >= args.warmup:
+                res[name].append((ev[0].elapsed_time(ev[1]), ev[1].elapsed_time(ev[2])))
+    row = 2.0 * w.num_kv_heads * w.head_dim * 2.0
+    L = w.block_lens.astype(np.float64)
+    bytes_all = sum(float((L + t + 1).sum()) for t in range(T)) * row
+    bytes_live = sum(float(((L + t + 1) * (t < stop)).sum()) for t in range(T)) * row
+    out = {"metric": "decode of many short sequences whose summaries stop at different lengths", "unit": "ms", "n_gpus": 1,
+           "steps": args.steps, "warmup": args.warmup, "dtype": "bf16", "data": "synthetic",
+           "config": {"workload": "locomo", "sequences": Bn, "block_lens": f"{int(w.block_lens.min())}..{int(w.block_lens.max())}",
+                      "q_heads": w.num_q_heads, "kv_heads": w.num_kv_heads, "head_dim": w.head_dim, "decode_steps": T,
+                      "stop_lens": f"{int(stop.min())}..{int(stop.max())}", "summary_tokens": int(stop.sum()), "seed": w.seed},
+           "peaks": dict(peaks, kind=peak_kind)}
+    for name, nbytes, tokens, pages in (("reserved", bytes_all, Bn * T, w.pages_needed), ("on_demand", bytes_live, int(stop.sum()), len(free))):
+        pf, dc = (statistics.mean(x[j] for x in res[name]) for j in (0, 1))
+        out[name] = {"prefill_and_append_ms": pf, "decode_ms": dc, "decode_us_per_step": dc * 1e3 / T,
+                     "kv_bytes_read": nbytes, "decode_gbs": nbytes / (dc * 1e-3) / 1e9,
+                     "decode_frac_of_hbm_peak": nbytes / (dc * 1e-3) / 1e9 / peaks["hbm_gbs"],
+                     "tokens_decoded": tokens, "pool_pages": pages}
+    out["on_demand"]["pages_held_at_end"] = pages_end
     print(json.dumps(out))
 
 
@@ -824,7 +926,7 @@ def main() -> None:
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--config", default=DEFAULT_CONFIG, choices=sorted(wl.CONFIGS) + ["prefix8b", "async", "mixed16k"])
+    ap.add_argument("--config", default=DEFAULT_CONFIG, choices=sorted(wl.CONFIGS) + ["prefix8b", "async", "mixed16k", "locomo"])
     ap.add_argument("--no-per-config", dest="per_config", action="store_false",
                     help="skip the per_config measurements of the other configurations")
     ap.add_argument("--blocks", type=int, default=0, help="override the number of blocks (profiling)")
@@ -832,6 +934,7 @@ def main() -> None:
     ap.add_argument("--decode-steps", type=int, default=0, help="override the decode steps (profiling)")
     ap.add_argument("--pages-per-split", type=int, default=0, help="decode split size (0 = planner's choice)")
     ap.add_argument("--decode-sms", type=int, default=0, help="mixed16k: SMs left to the decode wave beside a prefill chunk")
+    ap.add_argument("--steps-per-chunk", type=int, default=16, help="mixed16k: decode steps the schedule gives one chunk")
     ap.add_argument("--separate-append", action="store_true",
                     help="per decode step call cpa_kv_append and cpa_decode instead of the fused cpa_decode_append")
     ap.add_argument("--skip-e2e", action="store_true", help="skip the host-buffer leg (profiling)")
@@ -845,10 +948,10 @@ def main() -> None:
     args.layout = rank_layout(args.gpus, os.environ, args.impl)
     if args.layout[0] == "spawn":
         raise SystemExit(subprocess.run(args.layout[1]).returncode)
-    if args.config in ("prefix8b", "async", "mixed16k"):
+    if args.config in ("prefix8b", "async", "mixed16k", "locomo"):
         if args.impl == "reference":
             raise SystemExit("--impl reference times the default layout's workloads")
-        {"prefix8b": run_prefix, "async": run_async, "mixed16k": run_mixed}[args.config](args)
+        {"prefix8b": run_prefix, "async": run_async, "mixed16k": run_mixed, "locomo": run_locomo}[args.config](args)
     elif args.impl == "reference":
         run_reference(args)
     else:

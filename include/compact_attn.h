@@ -102,9 +102,9 @@ enum {
     CPA_ARR_SPLIT_PAGES = 8,   /* [B] pages per decode split of each block (the last split may be shorter) */
     CPA_ARR_PREFILL_SCHED = 9, /* [rounds * CPA_PARAM_PREFILL_CTAS] prefill unit (item * num_q_heads + head) of CTA c
                                   in round k at k * ctas + c, -1 = none; every unit appears exactly once */
-    CPA_ARR_DEC_START = 10,    /* [B] chunked plans: the step at which each block starts to decode (its chunk count) */
-    CPA_ARR_CHUNK_ROWS = 11,   /* [CPA_PARAM_CHUNK_STEPS * (B+1)] chunked plans: per step, prefix sums of the rows
-                                  each block prefills in it */
+    CPA_ARR_DEC_START = 10,    /* [B] chunked plans: the step at which each block starts to decode */
+    CPA_ARR_CHUNK_ROWS = 11,   /* [CPA_PARAM_CHUNK_STEPS * (B+1)] chunked plans: per chunk index, prefix sums of the
+                                  rows each block prefills in it */
     CPA_ARR_PAGES_ASSIGNED = 12, /* [B] plans with pages on demand: pages each block holds (as of creation or the last cpa_plan_sync) */
     CPA_ARR_FREE_RING = 13     /* plans with pages on demand: the pages of the common reserve, in the order they will be handed out */
 };
@@ -123,10 +123,11 @@ enum {
     CPA_PARAM_PREFILL_CTAS = 9,          /* CTAs of the prefill launch = min(num_sms, prefill units) */
     CPA_PARAM_SHARED_CHUNK_PAGES = 10,   /* pages per chunk of the shared-prefix decode scan; 0 without cached prefixes */
     CPA_PARAM_CHUNK_TOKENS = 11,         /* tokens per prefill chunk; 0 = not a chunked plan */
-    CPA_PARAM_NUM_STEPS = 12,            /* steps of a chunked plan's schedule: most chunks of any block + max_new_tokens */
-    CPA_PARAM_CHUNK_STEPS = 13,          /* steps that prefill a chunk (the most chunks of any block) */
+    CPA_PARAM_NUM_STEPS = 12,            /* steps of a chunked plan's schedule */
+    CPA_PARAM_CHUNK_STEPS = 13,          /* chunk indices of the schedule (the most chunks of any block) */
     CPA_PARAM_DECODE_SMS = 14,           /* SMs a chunked plan leaves to the decode wave while a chunk is prefilled */
-    CPA_PARAM_NUM_SMS = 15               /* the plan's SM budget (cfg.num_sms, or the device's SM count for 0) */
+    CPA_PARAM_NUM_SMS = 15,              /* the plan's SM budget (cfg.num_sms, or the device's SM count for 0) */
+    CPA_PARAM_DECODE_STEPS_PER_CHUNK = 16 /* decode steps a chunked plan's schedule gives a chunk */
 };
 
 /*
@@ -192,22 +193,26 @@ CPA_API int cpa_plan_create_prefix(const cpa_config* cfg, int32_t num_workers, c
  * engine runs with chunked prefill enabled (Section 4.2, "Hardware and Serving Infrastructure"), and its
  * finding that 16k blocks are prefill-bound (Section 6, "Prefill cost limits parallelism") is the case
  * this is for: a long block's prompt is cut into chunks, and the blocks that are past their prompt
- * decode in the same steps instead of waiting behind it.  The paper gives no rule; this library's is:
- *   a block of L_b tokens has n_b = ceil(L_b / chunk_tokens) chunks and prefills chunk s, rows
- *   [s * chunk_tokens, min((s + 1) * chunk_tokens, L_b)), in step s < n_b; it decodes summary token t
- *   in step n_b + t, t < max_new_tokens; the schedule has max_b(n_b) + max_new_tokens steps
- *   (CPA_PARAM_NUM_STEPS), run one by one with cpa_step_mixed.
+ * decode meanwhile instead of waiting behind it.  The paper gives no rule; this library's is
+ * (C = chunk_tokens, r = decode_steps_per_chunk):
+ *   a block of L_b tokens has n_b = ceil(L_b / C) chunks; chunk c, rows [c * C, min((c + 1) * C, L_b)),
+ *   starts at step c * r; the block decodes summary token t at step n_b * r + t, t < max_new_tokens;
+ *   the schedule has max_b(n_b) * r + max_new_tokens steps (CPA_PARAM_NUM_STEPS), run one by one with
+ *   cpa_step_mixed.
  * chunk_tokens: a multiple of 128 (a later chunk reads the earlier ones from the block's pages in whole
- * KV tiles of 128 keys).  decode_sms: SMs left to the decode wave in steps that also prefill a chunk
- * (the chunk's persistent grid takes the other num_sms - decode_sms); 0 = a quarter of the plan's SMs.
+ * KV tiles of 128 keys).  decode_steps_per_chunk >= 1: how many decode steps a chunk is given; a chunk
+ * costs far more than a decode step, so with r = 1 the decoding blocks produce tokens at the chunks' pace,
+ * and with r near (chunk time / decode step time) both sides stay busy.  decode_sms: SMs left to the
+ * decode wave while a chunk is under way (the chunk's persistent grid takes the other num_sms -
+ * decode_sms); 0 = a quarter of the plan's SMs.
  * Everything else (pages, slots, whole-block prefill list, decode items) is as for cpa_plan_create, and
  * the plan also works with the whole-block calls (cpa_prefill, cpa_kv_append, cpa_decode_append) as long
  * as the two ways are not mixed within one event.  Errors as for cpa_plan_create, plus CPA_EINVAL for a
- * chunk size below 128 or not a multiple of 128 and for decode_sms >= the plan's SMs.
+ * chunk size below 128 or not a multiple of 128, decode_steps_per_chunk < 1 and decode_sms >= the plan's SMs.
  */
 CPA_API int cpa_plan_create_chunked(const cpa_config* cfg, int32_t num_blocks, const int32_t* block_lens,
-                                    int32_t max_new_tokens, int32_t chunk_tokens, int32_t decode_sms,
-                                    const int32_t* free_pages, int32_t num_free, cpa_plan** out);
+                                    int32_t max_new_tokens, int32_t chunk_tokens, int32_t decode_steps_per_chunk,
+                                    int32_t decode_sms, const int32_t* free_pages, int32_t num_free, cpa_plan** out);
 
 /*
  * cpa_plan_create_dynamic -- a plan that reserves no pages for the summaries.  The paper's outlook (Section 8,
@@ -385,16 +390,19 @@ CPA_API int cpa_release_blocks(cpa_plan* plan, const int32_t* d_active, void* st
 
 /*
  * cpa_step_mixed -- step `step` of a chunked plan's schedule (cpa_plan_create_chunked; Section 4.2 and
- * Section 6 of the paper as cited there): the blocks that still have prompt left prefill their next
- * chunk and cache it, and the blocks whose turn it is decode one token (append fused in), in one call.
- * The two halves touch different blocks and run side by side: the chunk on a second stream the plan
- * owns (created at the first such step; no device memory is allocated), the decode on `stream`; the
- * call's work is complete on `stream` when both are.
- *   q, k, v, o : the packed tensors of the whole event ([total_tokens, heads, head_dim]); the step reads
- *                and writes only the rows of its chunks, rows cu_seqlens[b] + [s * chunk, ...) of every
- *                block that has a chunk s, so later rows need not exist yet.  Row i of a chunk attends
- *                over the block's cached tokens [0, s * chunk) and the chunk's tokens up to itself:
- *                exactly the rows cpa_prefill gives.  May be NULL in steps without a chunk.
+ * Section 6 of the paper as cited there).  If a chunk starts at this step (step = c * r), the blocks that
+ * have a chunk c prefill it and cache it; the blocks whose turn it is decode one token (append fused in).
+ * The two touch different blocks and run side by side: chunks one after the other on a second stream the
+ * plan owns (created at the first chunk; no device memory is allocated), decode launches on `stream`.
+ * `stream` waits for the chunks started so far when a block decodes its first token, and at the last
+ * step of the schedule: the prefill rows of a chunk are complete on `stream` from the step in which one
+ * of its blocks starts to decode, and all of them after the last step.  A chunk is ordered behind what
+ * `stream` held when its step was called (its rows may just have been copied in there).
+ *   q, k, v, o : the packed tensors of the whole event ([total_tokens, heads, head_dim]); a chunk reads
+ *                and writes only its rows, rows cu_seqlens[b] + [c * C, ...) of every block that has a
+ *                chunk c, so later rows need not exist yet.  Row i of a chunk attends over the block's
+ *                cached tokens [0, c * C) and the chunk's tokens up to itself: exactly the rows
+ *                cpa_prefill gives.  May be NULL in steps that start no chunk.
  *   q_dec, o_dec       : device bf16 [B, num_q_heads, head_dim]; only the rows of the decoding blocks are
  *                        read / written.  k_new, v_new: [B, num_kv_heads, head_dim] likewise.  May be
  *                        NULL in steps in which no block decodes.

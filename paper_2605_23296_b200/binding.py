@@ -14,7 +14,8 @@ from typing import Optional, Sequence
 import numpy as np
 
 _PKG = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_PKG, "libcompact_attn.so")
+# CPA_LIB_PATH points at another build of the library (same ABI), e.g. one made with other compile-time options
+LIB_PATH = os.environ.get("CPA_LIB_PATH") or os.path.join(_PKG, "libcompact_attn.so")
 
 CPA_OK, CPA_EINVAL, CPA_ENOSPC, CPA_EUNSUPPORTED, CPA_ECUDA, CPA_ETIMEOUT, CPA_ESTATE = 0, -1, -2, -3, -4, -5, -6
 
@@ -32,6 +33,7 @@ PARAM_MAX_NEW_TOKENS = 8
 PARAM_PREFILL_CTAS = 9
 PARAM_SHARED_CHUNK_PAGES = 10
 PARAM_CHUNK_TOKENS, PARAM_NUM_STEPS, PARAM_CHUNK_STEPS, PARAM_DECODE_SMS, PARAM_NUM_SMS = 11, 12, 13, 14, 15
+PARAM_DECODE_STEPS_PER_CHUNK = 16
 
 
 class cpa_config(ctypes.Structure):
@@ -61,7 +63,7 @@ _lib.cpa_plan_create_prefix.argtypes = [ctypes.POINTER(cpa_config), ctypes.c_int
                                         ctypes.c_int32, _i32p, ctypes.c_int32, ctypes.POINTER(_vp)]
 _lib.cpa_plan_create_prefix.restype = ctypes.c_int
 _lib.cpa_plan_create_chunked.argtypes = [ctypes.POINTER(cpa_config), ctypes.c_int32, _i32p, ctypes.c_int32, ctypes.c_int32,
-                                         ctypes.c_int32, _i32p, ctypes.c_int32, ctypes.POINTER(_vp)]
+                                         ctypes.c_int32, ctypes.c_int32, _i32p, ctypes.c_int32, ctypes.POINTER(_vp)]
 _lib.cpa_plan_create_chunked.restype = ctypes.c_int
 _lib.cpa_plan_create_dynamic.argtypes = [ctypes.POINTER(cpa_config), ctypes.c_int32, _i32p, ctypes.c_int32, _i32p,
                                          ctypes.c_int32, ctypes.POINTER(_vp)]
@@ -152,12 +154,14 @@ def cpa_plan_create_prefix(cfg: cpa_config, own_lens: Sequence[int], prefix_lens
 
 
 def cpa_plan_create_chunked(cfg: cpa_config, block_lens: Sequence[int], max_new_tokens: int, chunk_tokens: int,
-                            free_pages: Sequence[int], decode_sms: int = 0, check: bool = True):
+                            free_pages: Sequence[int], decode_sms: int = 0, decode_steps_per_chunk: int = 1,
+                            check: bool = True):
     """Plan of an event with chunked prefill; returns the handle, or (status, handle) with check=False."""
     lens, free = _i32(block_lens), _i32(free_pages)
     out = _vp()
     rc = _lib.cpa_plan_create_chunked(ctypes.byref(cfg), lens.shape[0], lens.ctypes.data_as(_i32p), int(max_new_tokens),
-                                      int(chunk_tokens), int(decode_sms), free.ctypes.data_as(_i32p), free.shape[0],
+                                      int(chunk_tokens), int(decode_steps_per_chunk), int(decode_sms),
+                                      free.ctypes.data_as(_i32p), free.shape[0],
                                       ctypes.byref(out))
     if not check:
         return rc, out.value

@@ -29,7 +29,7 @@ struct cpa_dev_index {
     int32_t shared_chunk;          // pages per chunk of the shared-prefix scan (0: no shared prefix)
     int32_t* merge_tickets;        // [B * Hkv] arrival counters of the fused split merge (zero between launches)
     int32_t item_stride;           // int32 words per decode item: 8 + largest split size rounded up to 4
-    const int32_t* dec_start;      // [B] chunked plans: the step at which a block starts to decode (= its chunk count)
+    const int32_t* dec_start;      // [B] chunked plans: the step at which a block starts to decode
     // plans with pages on demand: page_indices is a table of B rows (row b holds page_indptr[b+1] - page_indptr[b]
     // entries, the first pages_assigned[b] of them valid) that the decode kernel extends from the reserve
     int32_t* page_table;           // page_indices again, writable
@@ -47,7 +47,8 @@ struct cpa_decode_mode {
     const int32_t* d_active;  // dynamic plans: device flags [B], block b takes part iff d_active[b] != 0; nullptr: all do
 };
 
-// One step of a chunked plan's prefill: its items, their deal to CTAs, and the rows it appends.
+// One chunk of a chunked plan's prefill (chunk c of every block that has one): its items, their deal to CTAs, and
+// the rows it appends.
 struct cpa_chunk_step {
     int64_t off_items = 0;    // [n_items, 4] item records of the step (same format as prefill_items)
     int64_t off_sched = 0;    // [rounds, ctas]
@@ -76,6 +77,8 @@ struct cpa_plan {
     // chunked prefill: tokens per chunk (0: none), SMs left to the decode wave while a chunk is prefilled,
     // the step at which each block starts to decode, the per-step prefill work, and the schedule's position
     int32_t chunk = 0, decode_sms = 0, n_steps = 0, next_step = 0;
+    int32_t steps_per_chunk = 1;      // decode steps the schedule gives a chunk (chunk c starts at step c * steps_per_chunk)
+    bool chunk_pending = false;       // a chunk has been started on the second stream and not been joined yet
     std::vector<int32_t> dec_start, chunk_rows;   // chunk_rows: [chunk steps][B+1] prefix sums of the rows a step prefills
     std::vector<cpa_chunk_step> chunk_steps;
     int64_t off_decstart = 0;
@@ -168,9 +171,8 @@ int cpa_scan_tc(const cpa_plan* plan, const void* q, const void* k_pool, const v
 // pointers into the index buffer.  cpa_prefill_tc runs the plan's whole-block list.
 int cpa_prefill_tc_list(const cpa_plan* plan, const void* q, const void* k, const void* v, void* o, const void* k_pool,
                         const void* v_pool, const int32_t* items, const int32_t* sched, int ctas, int rounds, void* stream);
-// One chunk step's append: rows [step * chunk, ...) of every block that has them go to the pools; every block that
-// does not decode in this step gets its length carried into the other length buffer.
-int cpa_append_chunk(cpa_plan* plan, int step, const void* k, const void* v, void* k_pool, void* v_pool, void* stream);
+// Chunk c's append: rows [c * chunk, ...) of every block that has them go to the block's pages.
+int cpa_append_chunk(cpa_plan* plan, int chunk, const void* k, const void* v, void* k_pool, void* v_pool, void* stream);
 // One decode launch (append fused in when k_new is given) over the blocks `mode` selects.
 int cpa_decode_launch(const cpa_plan* plan, const void* q, const void* k_new, const void* v_new, void* k_pool,
                       void* v_pool, void* o, void* ws, cpa_decode_mode mode, int wave_sms, void* stream);

@@ -125,9 +125,21 @@ decode_split_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __
     const int32_t* item = ix.decode_items + (int64_t)item_idx * ix.item_stride;
     const int4 hdr = *reinterpret_cast<const int4*>(item);
     const int b = hdr.x, g = hdr.y, s = hdr.z, n_reserved = hdr.w;
-    // A step of a chunked plan: only the blocks whose turn it is decode; the others sit the step out (their
-    // lengths are carried over by the step's length kernel, their output rows are not touched).
-    if (mode.step >= 0 && (unsigned)(mode.step - __ldg(ix.dec_start + b)) >= (unsigned)mode.T) continue;
+    // A step of a chunked plan: only the blocks whose turn it is decode; the others sit the step out and their
+    // output rows are not touched.  A block that is through with its tokens has its length carried into the
+    // other length buffer by its first CTA (below); one that is still being prefilled has no length yet.
+    int sched_pos = 0;   // chunked plans: the block's token number in this step
+    if (mode.step >= 0) {
+        sched_pos = mode.step - __ldg(ix.dec_start + b);
+        if (sched_pos < 0) continue;
+        if (sched_pos >= mode.T) {
+            if (fa.k_new != nullptr && g == 0 && s == 0 && threadIdx.x == 0) {
+                asm volatile("griddepcontrol.wait;\n" ::: "memory");   // the previous launch wrote the length read here
+                ix.seq_lens_next[b] = ix.seq_lens[b];
+            }
+            continue;
+        }
+    }
     const int C = item[4];  // pages per split of this block
     const int first = item[5];           // first page of the split inside the block's page list
     const int slot = item[6];            // its partial slot among the block's slots
@@ -149,7 +161,9 @@ decode_split_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __
     // launch reads one array and the owner CTA of kv head 0 writes the other, so no CTA can see
     // a length that already moved.
     const bool fused = fa.k_new != nullptr;
-    const int len_old = ix.seq_lens[b];
+    // (a block of a chunked plan enters its first decode step with its whole prompt cached, whatever the
+    // length buffers hold: the chunks that cached it ran beside earlier decode launches)
+    const int len_old = (mode.step >= 0 && sched_pos == 0) ? ix.cu_seqlens[b + 1] - ix.cu_seqlens[b] : ix.seq_lens[b];
     if (mode.dynamic) {
         // Pages on demand.  A block takes part unless the caller's flag says it has stopped.  The page its new
         // token goes to was taken from the reserve when the page before it filled up; if the reserve was empty

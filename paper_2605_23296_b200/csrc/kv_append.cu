@@ -84,17 +84,6 @@ __global__ void kv_append_chunk_kernel(const uint4* __restrict__ k, const uint4*
     }
 }
 
-// Lengths after a step of a chunked plan, for every block that does not decode in it (the decode launch
-// writes the others): a block with a chunk in this step has cached it, the rest keep their length.  Reads
-// the current length buffer, writes the other one.
-__global__ void chunk_lengths_kernel(cpa_dev_index ix, const int32_t* __restrict__ rows_indptr, int B, int step, int T) {
-    const int b = blockIdx.x * blockDim.x + threadIdx.x;
-    if (b >= B) return;
-    const int d = step - ix.dec_start[b];
-    if (d >= 0 && d < T) return;   // decodes in this step
-    ix.seq_lens_next[b] = ix.seq_lens[b] + (rows_indptr ? rows_indptr[b + 1] - rows_indptr[b] : 0);
-}
-
 // Pages on demand: a block whose flag says it has stopped gives its pages back to the reserve.  One CTA per
 // block; pops happen in decode launches only, which are ordered against this one by the stream.
 __global__ void release_pages_kernel(cpa_dev_index ix, const int32_t* __restrict__ d_active, int B) {
@@ -172,22 +161,16 @@ extern "C" int cpa_kv_append(cpa_plan* plan, const void* k_new, const void* v_ne
     return CPA_OK;
 }
 
-int cpa_append_chunk(cpa_plan* plan, int step, const void* k, const void* v, void* k_pool, void* v_pool, void* stream) {
+int cpa_append_chunk(cpa_plan* plan, int chunk, const void* k, const void* v, void* k_pool, void* v_pool, void* stream) {
     const int B = plan->B, P = plan->cfg.page_size, Hkv = plan->cfg.num_kv_heads;
     const int chunks_per_head = plan->cfg.head_dim / 8;
     cudaStream_t st = (cudaStream_t)stream;
-    const cpa_dev_index ix = plan->dev();
-    const int32_t* rows_indptr = nullptr;
-    if (step < (int)plan->chunk_steps.size()) {
-        const cpa_chunk_step& cs = plan->chunk_steps[(size_t)step];
-        rows_indptr = plan->d_base + cs.off_rows;
-        const int threads = std::min(256, std::max(32, (Hkv * chunks_per_head + 31) / 32 * 32));
-        const int grid = (int)std::min<int64_t>(cs.rows, (int64_t)plan->num_sms * 32);
-        kv_append_chunk_kernel<<<grid, threads, 0, st>>>((const uint4*)k, (const uint4*)v, (uint4*)k_pool, (uint4*)v_pool,
-                                                         ix, rows_indptr, B, cs.rows, step * plan->chunk, Hkv,
-                                                         chunks_per_head, P);
-    }
-    chunk_lengths_kernel<<<(B + 127) / 128, 128, 0, st>>>(ix, rows_indptr, B, step, plan->T);
+    const cpa_chunk_step& cs = plan->chunk_steps[(size_t)chunk];
+    const int threads = std::min(256, std::max(32, (Hkv * chunks_per_head + 31) / 32 * 32));
+    const int grid = (int)std::min<int64_t>(cs.rows, (int64_t)plan->num_sms * 32);
+    kv_append_chunk_kernel<<<grid, threads, 0, st>>>((const uint4*)k, (const uint4*)v, (uint4*)k_pool, (uint4*)v_pool,
+                                                     plan->dev(), plan->d_base + cs.off_rows, B, cs.rows,
+                                                     chunk * plan->chunk, Hkv, chunks_per_head, P);
     return cudaGetLastError() == cudaSuccess ? CPA_OK : CPA_ECUDA;
 }
 

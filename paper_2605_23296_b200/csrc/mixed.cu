@@ -1,10 +1,13 @@
 // Steps of an event with chunked prefill (the serving engine of the paper's Section 4.2 runs with chunked
-// prefill enabled; Section 6 finds that 16k blocks are prefill-bound): in one step the blocks that still have
-// prompt left prefill their next chunk, and the blocks that are past their prompt decode one token.  The two
-// halves touch different blocks, so they run side by side: the chunk's persistent prefill grid on most SMs
-// (second stream), the decode wave on the SMs the plan keeps free for it (caller's stream), joined by an
-// event before the call's work counts as done on the caller's stream.
+// prefill enabled; Section 6 finds that 16k blocks are prefill-bound): the blocks that still have prompt left
+// prefill it chunk by chunk, and the blocks that are past their prompt decode meanwhile.  The two touch
+// different blocks, so they run side by side: the chunks one after the other on a second stream the plan owns,
+// each on most SMs; the decode launches on the caller's stream, on the SMs the plan keeps free for them.  A
+// chunk is given the time of `steps_per_chunk` decode steps; the caller's stream waits for the chunks only when
+// a block goes from its last chunk to its first decode step, and at the end of the schedule.
 #include <cuda_runtime.h>
+
+#include <algorithm>
 
 #include "cpa_internal.h"
 
@@ -31,55 +34,69 @@ extern "C" int cpa_step_mixed(cpa_plan* plan, int32_t step, const void* q, const
     if (plan->chunk == 0) return CPA_ESTATE;                 // not a chunked plan
     if (!plan->d_base || step != plan->next_step) return CPA_ESTATE;
     if (step < 0 || step >= plan->n_steps) return CPA_EINVAL;
-    const int B = plan->B, T = plan->T;
-    const bool has_prefill = step < (int)plan->chunk_steps.size();
-    bool has_decode = false;
-    for (int b = 0; b < B; ++b) has_decode |= plan->dec_start[b] <= step && step < plan->dec_start[b] + T;
-    if (has_prefill && (!q || !k || !v || !o || o == q || o == k || o == v)) return CPA_EINVAL;
+    const int B = plan->B, T = plan->T, r = plan->steps_per_chunk;
+    const int n_chunks = (int)plan->chunk_steps.size();
+    const int chunk = step / r;
+    const bool starts_chunk = step % r == 0 && chunk < n_chunks;
+    const bool beside_chunk = chunk < n_chunks;              // by the schedule a chunk is under way during this step
+    bool has_decode = false, first_decode = false;
+    for (int b = 0; b < B; ++b) {
+        const int pos = step - plan->dec_start[b];
+        has_decode |= pos >= 0 && pos < T;
+        first_decode |= pos == 0 && T > 0;
+    }
+    const bool last = step == plan->n_steps - 1;
+    if (starts_chunk && (!q || !k || !v || !o || o == q || o == k || o == v)) return CPA_EINVAL;
     if (has_decode && (!q_dec || !k_new || !v_new || !o_dec || !d_workspace)) return CPA_EINVAL;
     const void* ptrs[] = {q, k, v, o, q_dec, k_new, v_new, o_dec, k_pool, v_pool, d_workspace};
     for (const void* ptr : ptrs)
         if (ptr && !cpa_aligned16(ptr)) return CPA_EINVAL;
 
     cudaStream_t main_st = (cudaStream_t)stream;
-    cudaStream_t pre_st = main_st;
-    const bool side_by_side = has_prefill && has_decode;
-    if (side_by_side) {
-        if (int rc = ensure_side_stream(plan)) return rc;
-        pre_st = plan->side_stream;
-        if (cudaEventRecord(plan->ev_fork, main_st) != cudaSuccess ||
-            cudaStreamWaitEvent(pre_st, plan->ev_fork, 0) != cudaSuccess) {
-            (void)cudaGetLastError();
-            return CPA_ECUDA;
-        }
-    }
+    auto join = [&]() -> int {   // the caller's stream waits for every chunk started so far
+        if (!plan->chunk_pending) return CPA_OK;
+        if (cudaStreamWaitEvent(main_st, plan->ev_join, 0) != cudaSuccess) { (void)cudaGetLastError(); return CPA_ECUDA; }
+        plan->chunk_pending = false;
+        return CPA_OK;
+    };
+    // a block that decodes its first token now needs its last chunk, which is the one started most recently
+    if (first_decode)
+        if (int rc = join()) return rc;
     int rc = CPA_OK;
-    if (has_prefill) {
-        // the chunk's rows attend over the block's earlier chunks (cached pages) and over the chunk itself
-        const cpa_chunk_step& cs = plan->chunk_steps[(size_t)step];
-        rc = cpa_prefill_tc_list(plan, q, k, v, o, k_pool, v_pool, plan->d_base + cs.off_items, plan->d_base + cs.off_sched,
-                                 cs.ctas, cs.rounds, pre_st);
-    }
-    // the chunk's K/V go to the pages, and every block that does not decode gets its next length
-    if (rc == CPA_OK) rc = cpa_append_chunk(plan, step, k, v, k_pool, v_pool, pre_st);
-    if (rc == CPA_OK && has_decode)
-        rc = cpa_decode_launch(plan, q_dec, k_new, v_new, k_pool, v_pool, o_dec, d_workspace, cpa_decode_mode{step, T, 0, nullptr},
-                               has_prefill ? plan->decode_sms : 0, main_st);
-    if (side_by_side) {
-        // joined even after a failed launch, so that the caller's stream never runs ahead of the second one
-        if (cudaEventRecord(plan->ev_join, pre_st) != cudaSuccess ||
-            cudaStreamWaitEvent(main_st, plan->ev_join, 0) != cudaSuccess) {
+    if (starts_chunk) {
+        if ((rc = ensure_side_stream(plan)) != CPA_OK) return rc;
+        // the chunk follows whatever the caller has enqueued on `stream` so far (its rows may just have been copied in)
+        if (cudaEventRecord(plan->ev_fork, main_st) != cudaSuccess ||
+            cudaStreamWaitEvent(plan->side_stream, plan->ev_fork, 0) != cudaSuccess) {
             (void)cudaGetLastError();
             return CPA_ECUDA;
         }
+        // the chunk's rows attend over the block's earlier chunks (cached pages) and over the chunk itself; then
+        // its K/V go to the block's pages, where the next chunk and the decode steps find them
+        const cpa_chunk_step& cs = plan->chunk_steps[(size_t)chunk];
+        rc = cpa_prefill_tc_list(plan, q, k, v, o, k_pool, v_pool, plan->d_base + cs.off_items, plan->d_base + cs.off_sched,
+                                 cs.ctas, cs.rounds, plan->side_stream);
+        if (rc == CPA_OK) rc = cpa_append_chunk(plan, chunk, k, v, k_pool, v_pool, plan->side_stream);
+        if (cudaEventRecord(plan->ev_join, plan->side_stream) != cudaSuccess) { (void)cudaGetLastError(); return CPA_ECUDA; }
+        plan->chunk_pending = true;
+        if (rc != CPA_OK) return rc;
     }
-    if (rc != CPA_OK) return rc;
-    // host mirror of the lengths, and the other length buffer is now the current one
-    for (int b = 0; b < B; ++b) {
-        if (plan->dec_start[b] <= step && step < plan->dec_start[b] + T) plan->seq_lens[b] += 1;
-        else if (step < plan->dec_start[b]) plan->seq_lens[b] = std::min(plan->block_lens[b], (step + 1) * plan->chunk);
+    if (has_decode) {
+        rc = cpa_decode_launch(plan, q_dec, k_new, v_new, k_pool, v_pool, o_dec, d_workspace,
+                               cpa_decode_mode{step, T, 0, nullptr}, beside_chunk ? plan->decode_sms : 0, main_st);
+        if (rc != CPA_OK) return rc;
+        // host mirror of the lengths; the other length buffer is now the current one
+        for (int b = 0; b < B; ++b) {
+            const int pos = step - plan->dec_start[b];
+            if (pos >= 0 && pos < T) plan->seq_lens[b] = plan->block_lens[b] + pos + 1;
+        }
+        plan->cur_lens ^= 1;
     }
-    plan->cur_lens ^= 1;
+    for (int b = 0; b < B; ++b)   // (mirror: a block's prompt counts as cached once its last chunk has been started)
+        if (starts_chunk && step < plan->dec_start[b])
+            plan->seq_lens[b] = std::min(plan->block_lens[b], (chunk + 1) * plan->chunk);
+    if (last)
+        if ((rc = join()) != CPA_OK) return rc;
     plan->next_step = step + 1;
     return CPA_OK;
 }

@@ -74,7 +74,8 @@ namespace {
 // Both layouts: `prefix_lens` == nullptr is the independent-chunks layout (no cached prefix).
 int plan_create(const cpa_config* cfg, int32_t num_blocks, const int32_t* block_lens, const int32_t* prefix_lens,
                 const int32_t* shared_pages, int32_t num_shared, int32_t max_new_tokens, const int32_t* free_pages,
-                int32_t num_free, int32_t chunk_tokens, int32_t decode_sms, bool dynamic, cpa_plan** out) {
+                int32_t num_free, int32_t chunk_tokens, int32_t decode_sms, int32_t steps_per_chunk, bool dynamic,
+                cpa_plan** out) {
     if (out) *out = nullptr;
     if (!cfg || !block_lens || !out || num_blocks < 1 || max_new_tokens < 0 || num_free < 0 ||
         (num_free > 0 && !free_pages) || num_shared < 0 || (num_shared > 0 && !shared_pages))
@@ -91,7 +92,7 @@ int plan_create(const cpa_config* cfg, int32_t num_blocks, const int32_t* block_
     if (cfg->num_sms > kMaxPlanSms) return CPA_EUNSUPPORTED;
     if (prefix_lens && num_blocks > 0xFFFF) return CPA_EUNSUPPORTED;
     // a chunk is read back as a cached prefix of whole 128-key tiles
-    if (chunk_tokens < 0 || chunk_tokens % 128 != 0 || decode_sms < 0) return CPA_EINVAL;
+    if (chunk_tokens < 0 || chunk_tokens % 128 != 0 || decode_sms < 0 || steps_per_chunk < 1) return CPA_EINVAL;
     if (chunk_tokens > 0 && prefix_lens) return CPA_EUNSUPPORTED;
     if (dynamic && (chunk_tokens > 0 || prefix_lens)) return CPA_EUNSUPPORTED;
 
@@ -313,34 +314,40 @@ int plan_create(const cpa_config* cfg, int32_t num_blocks, const int32_t* block_
         p->decode_items.push_back(it.split);
     }
 
-    // Chunked prefill: step s prefills rows [s*C, min((s+1)*C, L_b)) of every block that has them, reading the
-    // block's earlier chunks from its pages exactly like a cached prefix; a block decodes in the T steps after
-    // its last chunk.  Every step gets its own item list and deal.  While some block decodes, the chunk's
-    // persistent grid leaves `decode_sms` SMs to the decode wave that runs beside it.
+    // Chunked prefill: chunk c of a block, rows [c*C, min((c+1)*C, L_b)), starts at step c*r (r = steps_per_chunk: a
+    // chunk is given the time of r decode steps) and reads the block's earlier chunks from its pages exactly like a
+    // cached prefix; a block decodes in the T steps from step n_b*r on.  Every chunk index gets its own item list
+    // and deal.  While some block decodes during a chunk's r steps, the chunk's persistent grid leaves
+    // `decode_sms` SMs to the decode wave that runs beside it.
     std::vector<int32_t> chunk_items, chunk_sched, chunk_rows;
     if (chunk_tokens > 0) {
-        const int32_t Cc = chunk_tokens, Hq = cfg->num_q_heads, G = Hq / cfg->num_kv_heads;
+        const int32_t Cc = chunk_tokens, Hq = cfg->num_q_heads, G = Hq / cfg->num_kv_heads, r = steps_per_chunk;
         p->chunk = Cc;
+        p->steps_per_chunk = r;
         p->decode_sms = decode_sms ? decode_sms : std::max(1, p->num_sms / 4);
         if (p->decode_sms >= p->num_sms) { delete p; return CPA_EINVAL; }
         p->dec_start.assign(B, 0);
         int32_t n_chunk_steps = 0;
+        std::vector<int32_t> n_chunks(B);
         for (int32_t b = 0; b < B; ++b) {
-            p->dec_start[b] = (block_lens[b] + Cc - 1) / Cc;
-            n_chunk_steps = std::max(n_chunk_steps, p->dec_start[b]);
+            n_chunks[b] = (block_lens[b] + Cc - 1) / Cc;
+            if ((int64_t)n_chunks[b] * r + max_new_tokens > INT32_MAX / 2) { delete p; return CPA_EUNSUPPORTED; }
+            p->dec_start[b] = n_chunks[b] * r;
+            n_chunk_steps = std::max(n_chunk_steps, n_chunks[b]);
         }
-        p->n_steps = n_chunk_steps + max_new_tokens;
+        p->n_steps = n_chunk_steps * r + max_new_tokens;
         p->chunk_steps.resize((size_t)n_chunk_steps);
         for (int32_t st = 0; st < n_chunk_steps; ++st) {
             cpa_chunk_step& cs = p->chunk_steps[(size_t)st];
-            bool any_decode = false;
-            for (int32_t b = 0; b < B; ++b) any_decode |= p->dec_start[b] <= st && st < p->dec_start[b] + max_new_tokens;
+            bool any_decode = false;   // does some block decode during the r steps of this chunk?
+            for (int32_t b = 0; b < B; ++b)
+                any_decode |= p->dec_start[b] < (st + 1) * r && st * r < p->dec_start[b] + max_new_tokens;
             std::vector<PItem> cit;
             cs.off_rows = (int64_t)chunk_rows.size();
             int32_t rows = 0;
             for (int32_t b = 0; b < B; ++b) {
                 chunk_rows.push_back(rows);
-                if (st >= p->dec_start[b]) continue;
+                if (st >= n_chunks[b]) continue;
                 const int32_t len = std::min(Cc, block_lens[b] - st * Cc);
                 rows += len;
                 for (int32_t t = 0; t * p->q_tile < len; ++t)
@@ -467,13 +474,13 @@ int plan_create(const cpa_config* cfg, int32_t num_blocks, const int32_t* block_
 extern "C" int cpa_plan_create(const cpa_config* cfg, int32_t num_blocks, const int32_t* block_lens,
                                int32_t max_new_tokens, const int32_t* free_pages, int32_t num_free,
                                cpa_plan** out) {
-    return plan_create(cfg, num_blocks, block_lens, nullptr, nullptr, 0, max_new_tokens, free_pages, num_free, 0, 0, false, out);
+    return plan_create(cfg, num_blocks, block_lens, nullptr, nullptr, 0, max_new_tokens, free_pages, num_free, 0, 0, 1, false, out);
 }
 
 extern "C" int cpa_plan_create_dynamic(const cpa_config* cfg, int32_t num_blocks, const int32_t* block_lens,
                                        int32_t max_new_tokens, const int32_t* free_pages, int32_t num_free,
                                        cpa_plan** out) {
-    return plan_create(cfg, num_blocks, block_lens, nullptr, nullptr, 0, max_new_tokens, free_pages, num_free, 0, 0, true,
+    return plan_create(cfg, num_blocks, block_lens, nullptr, nullptr, 0, max_new_tokens, free_pages, num_free, 0, 0, 1, true,
                        out);
 }
 
@@ -505,12 +512,13 @@ extern "C" int cpa_plan_sync(cpa_plan* plan, void* stream) {
 }
 
 extern "C" int cpa_plan_create_chunked(const cpa_config* cfg, int32_t num_blocks, const int32_t* block_lens,
-                                       int32_t max_new_tokens, int32_t chunk_tokens, int32_t decode_sms,
-                                       const int32_t* free_pages, int32_t num_free, cpa_plan** out) {
+                                       int32_t max_new_tokens, int32_t chunk_tokens, int32_t decode_steps_per_chunk,
+                                       int32_t decode_sms, const int32_t* free_pages, int32_t num_free,
+                                       cpa_plan** out) {
     if (out) *out = nullptr;
     if (chunk_tokens < 128) return CPA_EINVAL;
     return plan_create(cfg, num_blocks, block_lens, nullptr, nullptr, 0, max_new_tokens, free_pages, num_free,
-                       chunk_tokens, decode_sms, false, out);
+                       chunk_tokens, decode_sms, decode_steps_per_chunk, false, out);
 }
 
 extern "C" int cpa_plan_create_prefix(const cpa_config* cfg, int32_t num_workers, const int32_t* own_lens,
@@ -520,7 +528,7 @@ extern "C" int cpa_plan_create_prefix(const cpa_config* cfg, int32_t num_workers
     if (out) *out = nullptr;
     if (!prefix_lens) return CPA_EINVAL;
     return plan_create(cfg, num_workers, own_lens, prefix_lens, shared_pages, num_shared, max_new_tokens, free_pages,
-                       num_free, 0, 0, false, out);
+                       num_free, 0, 0, 1, false, out);
 }
 
 extern "C" int cpa_plan_export(const cpa_plan* plan, int which, const int32_t** ptr, int64_t* count) {
@@ -573,6 +581,7 @@ extern "C" int64_t cpa_plan_param(const cpa_plan* plan, int which) {
         case CPA_PARAM_CHUNK_STEPS: return (int64_t)plan->chunk_steps.size();
         case CPA_PARAM_DECODE_SMS: return plan->decode_sms;
         case CPA_PARAM_NUM_SMS: return plan->num_sms;
+        case CPA_PARAM_DECODE_STEPS_PER_CHUNK: return plan->steps_per_chunk;
         default: return CPA_EINVAL;
     }
 }
@@ -584,6 +593,7 @@ extern "C" int cpa_plan_upload(cpa_plan* plan, void* d_index_buf, int64_t bytes,
     plan->seq_lens = plan->prefix_lens;
     plan->cur_lens = 0;
     plan->next_step = 0;
+    plan->chunk_pending = false;
     if (plan->dynamic) {   // the device starts from the plan's first assignment again, and so do the host mirrors
         const int32_t* im = plan->image.data();
         plan->page_indices.assign(im + plan->off_pidx, im + plan->off_pidx + plan->page_indices.size());

@@ -39,7 +39,8 @@ class CompactionSession:
                  scale: Optional[float] = None, device: str = "cuda:0", pages_per_split: int = 0,
                  poison_pools: bool = False, page_size: int = 16, q_tile_rows: int = 0,
                  prefix_lens: Optional[Sequence[int]] = None, shared_pages: Optional[Sequence[int]] = None,
-                 pools=None, num_sms: int = 0, chunk_tokens: int = 0, decode_sms: int = 0, dynamic_pages: bool = False):
+                 pools=None, num_sms: int = 0, chunk_tokens: int = 0, decode_sms: int = 0, dynamic_pages: bool = False,
+                 decode_steps_per_chunk: int = 1):
         self.device = torch.device(device)
         self.Hq, self.Hkv, self.d, self.P = num_q_heads, num_kv_heads, head_dim, page_size
         self.B = len(block_lens)
@@ -59,7 +60,7 @@ class CompactionSession:
         elif chunk_tokens:      # prefill in chunks, mixed with the decode of blocks that are past their prompt
             assert prefix_lens is None
             self.plan = B.cpa_plan_create_chunked(self.cfg, self.block_lens, max_new_tokens, chunk_tokens, free_pages,
-                                                  decode_sms)
+                                                  decode_sms, decode_steps_per_chunk)
         elif self.prefix_aware:   # the paper's layout: cached history prefix + own tokens per worker
             self.plan = B.cpa_plan_create_prefix(self.cfg, self.block_lens, prefix_lens, shared_pages,
                                                  max_new_tokens, free_pages)
@@ -141,8 +142,8 @@ class CompactionSession:
         return out
 
     def step_mixed(self, step: int, q, k, v, out, q_dec=None, k_new=None, v_new=None, out_dec=None) -> None:
-        """Step `step` of a chunked plan: the next prefill chunk of the blocks that have one (rows of the
-        whole-event tensors q/k/v/out) beside one decode token of the blocks whose turn it is."""
+        """Step `step` of a chunked plan: the chunk that starts at this step, if any (rows of the whole-event
+        tensors q/k/v/out), beside one decode token of the blocks whose turn it is."""
         self._check(B.cpa_step_mixed(self.plan, step, q, k, v, out, q_dec, k_new, v_new, out_dec, self.k_pool,
                                      self.v_pool, self.workspace, self._stream()), "cpa_step_mixed")
 

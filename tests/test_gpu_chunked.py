@@ -28,7 +28,7 @@ def _cu(w):
     return np.concatenate([[0], np.cumsum(w.block_lens.astype(np.int64))])
 
 
-def run_chunked_event(w, chunk, decode_sms=0, rows=None, what=""):
+def run_chunked_event(w, chunk, decode_sms=0, rows=None, what="", r=1):
     """All steps of the schedule through cpa_step_mixed.  Inputs of decode step t of a block are row t of
     w.*_dec (so a block's t-th summary token has the same inputs whatever step it is produced in)."""
     import torch
@@ -37,8 +37,9 @@ def run_chunked_event(w, chunk, decode_sms=0, rows=None, what=""):
     w.materialise()
     T, Bn = w.decode_steps, w.num_blocks
     s = CompactionSession(w.block_lens, T, w.num_q_heads, w.num_kv_heads, w.head_dim, w.free_pages, w.num_pages,
-                          scale=w.scale, poison_pools=True, chunk_tokens=chunk, decode_sms=decode_sms)
-    sched = op.mixed_schedule(w.block_lens.tolist(), chunk, T)
+                          scale=w.scale, poison_pools=True, chunk_tokens=chunk, decode_sms=decode_sms,
+                          decode_steps_per_chunk=r)
+    sched = op.mixed_schedule(w.block_lens.tolist(), chunk, T, r)
     assert s.param(B.PARAM_NUM_STEPS) == len(sched)
     start = s.export(B.ARR_DEC_START)
     q, k, v = _dev(w.q), _dev(w.k), _dev(w.v)
@@ -109,6 +110,13 @@ def test_chunks_of_three_tiles_and_a_small_decode_share():
     run_chunked_event(wl.custom([1000, 400, 385, 7], 8, 2, 128, steps=4, seed=77), 384, decode_sms=1, what="chunk 384")
 
 
+@pytest.mark.parametrize("r", [2, 5])
+def test_several_decode_steps_beside_one_chunk(r):
+    # the short blocks finish their summaries (6 tokens) while the long block is still on its second and third
+    # chunk, sit out until the schedule ends, and the long block starts to decode right after its last chunk
+    run_chunked_event(wl.custom([700, 100, 50, 129], 8, 2, 128, steps=6, seed=80 + r), 256, what=f"r = {r}", r=r)
+
+
 def test_one_chunk_covers_every_block():
     # chunk longer than every block: step 0 is the whole prefill, then plain decode steps
     run_chunked_event(wl.tiny(4), 512, what="tiny, one chunk")
@@ -128,7 +136,7 @@ def test_long_block_beside_short_ones_sampled_rows():
     for b, L in enumerate(int(x) for x in w.block_lens):
         cand = {0, 1, L - 1} | {c for t in range(2048, L, 2048) for c in (t - 1, t, t + 1)} | set(int(x) for x in rng.integers(0, L, 10))
         rows += [cu[b] + r for r in sorted(cand) if 0 <= r < L]
-    run_chunked_event(w, 2048, rows=np.asarray(rows, dtype=np.int64), what="16k + 4 x 2k")
+    run_chunked_event(w, 2048, rows=np.asarray(rows, dtype=np.int64), what="16k + 4 x 2k", r=3)
 
 
 def test_mixed_step_needs_a_chunked_plan():

@@ -200,29 +200,34 @@ def test_library_exports_every_declared_symbol():
 # chunked prefill: the steps of the schedule
 # ----------------------------------------------------------------------------
 
-@pytest.mark.parametrize("lens,C,T", [([300, 100, 50], 128, 2), ([16384, 2048, 2048, 2048, 2048], 2048, 256),
-                                       ([1, 129, 128, 1000], 128, 3), ([700], 256, 0)])
-def test_chunked_plan_steps_bit_exact(lens, C, T):
+@pytest.mark.parametrize("lens,C,T,r", [([300, 100, 50], 128, 2, 1), ([300, 100, 50], 128, 3, 2),
+                                         ([16384, 2048, 2048, 2048, 2048], 2048, 256, 16),
+                                         ([1, 129, 128, 1000], 128, 3, 1), ([700], 256, 0, 4)])
+def test_chunked_plan_steps_bit_exact(lens, C, T, r):
     cfg = B.cpa_config(8, 2, 128, 16, 0.088, 0, 0, 0)
     pages = sum(-(-(L + T) // 16) for L in lens)
-    plan = B.cpa_plan_create_chunked(cfg, lens, T, C, np.arange(pages, dtype=np.int32))
+    plan = B.cpa_plan_create_chunked(cfg, lens, T, C, np.arange(pages, dtype=np.int32), decode_steps_per_chunk=r)
     try:
-        ref = op.mixed_schedule(lens, C, T)
+        ref = op.mixed_schedule(lens, C, T, r)
         assert B.cpa_plan_param(plan, B.PARAM_NUM_STEPS) == len(ref)
         assert B.cpa_plan_param(plan, B.PARAM_CHUNK_TOKENS) == C
-        n_chunk_steps = B.cpa_plan_param(plan, B.PARAM_CHUNK_STEPS)
-        assert n_chunk_steps == sum(1 for st in ref if st["prefill"])
+        assert B.cpa_plan_param(plan, B.PARAM_DECODE_STEPS_PER_CHUNK) == r
+        n_chunks = B.cpa_plan_param(plan, B.PARAM_CHUNK_STEPS)
+        assert n_chunks == sum(1 for st in ref if st["prefill"])
         start = B.cpa_plan_export(plan, B.ARR_DEC_START).tolist()
-        rows = B.cpa_plan_export(plan, B.ARR_CHUNK_ROWS).reshape(n_chunk_steps, len(lens) + 1)
+        rows = B.cpa_plan_export(plan, B.ARR_CHUNK_ROWS).reshape(n_chunks, len(lens) + 1)
         for s, st in enumerate(ref):
             assert [b for b in range(len(lens)) if 0 <= s - start[b] < T] == st["decode"]
-            if s < n_chunk_steps:
-                per_block = np.diff(rows[s]).tolist()
+            if s % r == 0 and s // r < n_chunks:
+                c = s // r
+                per_block = np.diff(rows[c]).tolist()
                 want = [0] * len(lens)
                 for b, first, n in st["prefill"]:
-                    assert first == s * C
+                    assert first == c * C
                     want[b] = n
-                assert per_block == want and rows[s][0] == 0
+                assert per_block == want and rows[c][0] == 0
+            else:
+                assert not st["prefill"]
         # everything the whole-block calls use is the ordinary plan's
         plain = B.cpa_plan_create(cfg, lens, T, np.arange(pages, dtype=np.int32))
         for which in (B.ARR_CU_SEQLENS, B.ARR_PAGE_INDICES, B.ARR_SLOT_MAPPING, B.ARR_PREFILL_ITEMS, B.ARR_DECODE_ITEMS):
@@ -243,6 +248,8 @@ def test_chunked_plan_errors():
     rc, h = B.cpa_plan_create_chunked(cfg, (300, 50), 2, 128, free, decode_sms=4096, check=False)
     assert rc == B.CPA_EINVAL and not h
     rc, h = B.cpa_plan_create_chunked(cfg, (300, 0), 2, 128, free, check=False)
+    assert rc == B.CPA_EINVAL and not h
+    rc, h = B.cpa_plan_create_chunked(cfg, (300, 50), 2, 128, free, decode_steps_per_chunk=0, check=False)
     assert rc == B.CPA_EINVAL and not h
     fake = 4096
     plan = B.cpa_plan_create_chunked(cfg, (300, 50), 2, 128, free)
