@@ -34,8 +34,9 @@ NOMINAL_HBM_GBS = 8000.0
 NOMINAL_BF16_TFLOPS = 2250.0
 L2_MB = 126
 DEFAULT_CONFIG = "ragged"   # the largest single-GPU workload of the throughput configurations
-# The other single-GPU configurations, measured in the same run (three timed steps each) into `per_config`.
-PER_CONFIG = [("dense8b", {}), ("moe120b", {}), ("split", {"num_blocks": 1})]
+# The other single-GPU configurations, measured in the same run into `per_config`: (name, overrides, timed steps).
+# The step counts make each timed region last a few hundred milliseconds, long enough for the clock sampler.
+PER_CONFIG = [("dense8b", {}, 40), ("moe120b", {}, 8), ("split", {"num_blocks": 1}, 3)]
 # Profiler captures of one decode_split_kernel launch per workload (profiles/decode_split_kernel_*.md), of the
 # kernel as it stands: DRAM bytes read + written per launch with the caches left alone between consecutive steps
 # ("warm", the timed condition) and with the L2 flushed before the launch ("cold"), the cold launch duration,
@@ -462,17 +463,17 @@ def run_gpu(args) -> None:
     per_config = {}
     if args.per_config and world == 1 and not overridden:
         del w.q, w.k, w.v
-        for name, kw in PER_CONFIG:
+        for name, kw, n_timed in PER_CONFIG:
             if name == args.config and not kw:
                 continue
             gc.collect()
             torch.cuda.empty_cache()
             w2 = wl.CONFIGS[name](**kw).materialise()
-            m2 = measure_event(w2, args, dev, 3, 3, False)
+            m2 = measure_event(w2, args, dev, n_timed, 3, False)
             p2 = phase_numbers(w2, m2, peaks, False)
             label = name if not kw else f"{name}:B={kw['num_blocks']}"
             per_config[label] = dict(p2, config=workload_desc(w2), ms_per_step=m2["ms"],
-                                     value=w2.num_blocks * w2.decode_steps / (m2["ms"] * 1e-3), steps=3, warmup=3,
+                                     value=w2.num_blocks * w2.decode_steps / (m2["ms"] * 1e-3), steps=n_timed, warmup=3,
                                      clocks=m2["clocks"])
             del w2
         w = make_workload(args.config, seed_offset=rank, overrides=args.overrides).materialise()

@@ -200,6 +200,7 @@ struct __align__(8) TcBarriers {
     // [sub-tile][that sub-tile's step count mod 4]: at most three steps are ever ahead of a waiter, so a
     // waiter can never meet the phase after the one it is waiting for
     uint64_t s_full[2][4], p_full[2][4], pv_done[2];
+    uint64_t p_half[2][4];   // the first 64 keys' weights of a step are in TMEM (the PV MMAs over them start while the rest is computed)
     uint64_t drain;   // only used after a wait gave up: tracks the MMAs still queued, so that TMEM is not freed under them
     uint32_t tmem_base;
 };
@@ -210,6 +211,7 @@ struct TcShape {
     static constexpr uint32_t kTileBytes = NB * kBlockBytes;   // one Q sub-tile, K tile or V tile
     static constexpr int kBufs = (D == 64) ? 3 : 2;            // score buffers in TMEM
     static constexpr int kStages = (D == 64) ? 4 : 2;          // K ring and V ring depth
+    static constexpr bool kSplitP = (D == 128);                // the weights of a step are handed to the issuer in two halves
     static constexpr uint32_t kColO = kBufs * 128;             // O_u at kColO + u*D
     static constexpr uint32_t kTmemCols = 512;
     static constexpr int kSmem = (2 + 2 * kStages) * (int)kTileBytes + 1024;   // Q sub-tiles + rings + alignment slack
@@ -246,6 +248,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
     constexpr int NB = Sh::NB;
     constexpr uint32_t kTileBytes = Sh::kTileBytes;
     constexpr int NBUF = Sh::kBufs, KS = Sh::kStages;
+    constexpr bool kSplitP = Sh::kSplitP;
     constexpr uint32_t kColO = Sh::kColO;
     extern __shared__ unsigned char dsm_raw[];
     __shared__ TcBarriers bars;
@@ -296,6 +299,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
             for (int i = 0; i < 4; ++i) {
                 mbar_init(bar(&bars.s_full[u][i]), 1);
                 mbar_init(bar(&bars.p_full[u][i]), 128);
+                mbar_init(bar(&bars.p_half[u][i]), 128);
             }
         }
         mbar_init(bar(&bars.drain), 1);
@@ -473,14 +477,26 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
             ++n_qk[u];
         };
         auto pv = [&](int u, int buf, int kt, uint32_t acc0) {   // O_u += P[buf] V[tile kt]
+            const uint32_t bv = v_lo + (kt % KS) * kTile16, d_tmem = tmem + kColO + u * D, a_tmem = tmem + buf * 128;
+            // With kSplitP the weights arrive in two halves of 64 keys, and the MMAs over the first half run while the
+            // softmax warpgroup is still computing the second (head_dim 128, where a sub-tile's steps form one chain
+            // softmax -> PV -> QK; at head_dim 64 the third score buffer has cut that chain already and the extra
+            // barrier round only costs).
+            if (kSplitP) {
+                tc_wait(bar(&bars.p_half[u][n_pv[u] & 3u]), (n_pv[u] >> 2) & 1u, dead, ix.status);
+                if (dead) leader = 0u;
+                tc_fence_after();
+#pragma unroll
+                for (int k = 0; k < kTileN / 32; ++k)
+                    // 16 keys per instruction: 8 TMEM columns of A; 16 rows of 128 B of V, column blocks kBlockBytes apart
+                    tc_mma_ts_lo(d_tmem, a_tmem + k * 8, bv + k * (2048 >> 4), pv_hi, idesc_pv, k > 0 ? 1u : acc0, leader);
+            }
             tc_wait(bar(&bars.p_full[u][n_pv[u] & 3u]), (n_pv[u] >> 2) & 1u, dead, ix.status);
             if (dead) leader = 0u;
             ++n_pv[u];
             tc_fence_after();
-            const uint32_t bv = v_lo + (kt % KS) * kTile16, d_tmem = tmem + kColO + u * D, a_tmem = tmem + buf * 128;
 #pragma unroll
-            for (int k = 0; k < kTileN / 16; ++k)
-                // 16 keys per instruction: 8 TMEM columns of A; 16 rows of 128 B of V, column blocks kBlockBytes apart
+            for (int k = kSplitP ? kTileN / 32 : 0; k < kTileN / 16; ++k)
                 tc_mma_ts_lo(d_tmem, a_tmem + k * 8, bv + k * (2048 >> 4), pv_hi, idesc_pv, k > 0 ? 1u : acc0, leader);
         };
         auto wait_k = [&](int kt) {
@@ -686,6 +702,11 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                     add_bf16x2(sum[(i >> 1) & 7], w2);
                 }
                 tc_st16(t_s + c * 16, pk);
+                if (kSplitP && c == 1) {   // the first 64 keys' weights are in place: let their MMAs start
+                    tc_wait_st();
+                    tc_fence_before();
+                    mbar_arrive(bar(&bars.p_half[u][n_steps & 3u]));
+                }
             }
             l_run += ((sum[0] + sum[1]) + (sum[2] + sum[3])) + ((sum[4] + sum[5]) + (sum[6] + sum[7]));
             tc_wait_st();
