@@ -37,11 +37,21 @@ DEFAULT_CONFIG = "ragged"   # the largest single-GPU workload of the throughput 
 # The other single-GPU configurations, measured in the same run into `per_config`: (name, overrides, timed steps).
 # The step counts make each timed region last a few hundred milliseconds, long enough for the clock sampler.
 PER_CONFIG = [("dense8b", {}, 40), ("moe120b", {}, 8), ("split", {"num_blocks": 1}, 3)]
-# Profiler captures of one decode_split_kernel launch per workload (profiles/decode_split_kernel_*.md), of the
-# kernel as it stands: DRAM bytes read + written per launch with the caches left alone between consecutive steps
-# ("warm", the timed condition) and with the L2 flushed before the launch ("cold"), the cold launch duration,
-# and the algorithmic KV bytes of the captured launches.  A workload without a capture has no entry.
-DECODE_CAPTURES = {}
+# Profiler captures of decode_split_kernel launches per workload (profiles/decode_split_kernel_*.md), of the
+# kernel as it stands, on the workload with 24 instead of its full number of decode steps (eight launches,
+# steps 6..13): DRAM bytes read + written per launch divided by the algorithmic KV bytes of those launches, with
+# the caches left alone between consecutive steps ("warm", the timed condition) and with the L2 flushed before
+# the launch ("cold"), and the algorithmic bytes per second of the cold launches.  A step's traffic grows in
+# proportion to its KV bytes, so the ratios carry over to the average step of the full run.  A workload without
+# a capture has no entry.
+DECODE_CAPTURES = {
+    "ragged": {"warm_ratio": 0.9307, "cold_ratio": 1.0042, "cold_gbs": 6051.1,
+               "source": "profiles/decode_split_kernel_ragged.md"},
+    "dense8b": {"warm_ratio": 0.3516, "cold_ratio": 1.0085, "cold_gbs": 4022.1,
+                "source": "profiles/decode_split_kernel_dense8b.md"},
+    "moe120b": {"warm_ratio": 0.7622, "cold_ratio": 1.0052, "cold_gbs": 5046.6,
+                "source": "profiles/decode_split_kernel_moe120b.md"},
+}
 
 
 def load_peaks():
@@ -411,6 +421,14 @@ def phase_numbers(w, m: dict, peaks: dict, separate_append: bool) -> dict:
                 if launch_bytes < 2.5 * L2_MB * 1e6 else "HBM-bound, at most a fifth can come from L2"))}
 
 
+def capture_fields(cap, bytes_per_launch: float, peaks: dict) -> dict:
+    """DRAM traffic of one decode launch from the profiler captures (see DECODE_CAPTURES); nulls without one."""
+    if not cap:
+        return {"traffic": None, "traffic_cold": None, "frac_cold_l2": None, "traffic_source": None}
+    return {"traffic": cap["warm_ratio"] * bytes_per_launch, "traffic_cold": cap["cold_ratio"] * bytes_per_launch,
+            "frac_cold_l2": cap["cold_gbs"] / peaks["hbm_gbs"], "traffic_source": cap["source"]}
+
+
 def run_gpu(args) -> None:
     import gc
 
@@ -453,10 +471,7 @@ def run_gpu(args) -> None:
                 "launch_us": ph["decode_launch_us"], "bytes_per_launch": ph["decode_bytes_per_launch"],
                 "launches_timed": (T * args.steps if not args.separate_append else m["n_pairs"]),
                 "launch_us_event_pair_sampled": m["pair_us"],
-                "traffic": cap["traffic_warm"] if cap else None,
-                "traffic_cold": cap["traffic_cold"] if cap else None,
-                "frac_cold_l2": (cap["algorithmic"] / (cap["cold_us"] * 1e-6) / 1e9 / peaks["hbm_gbs"]) if cap else None,
-                "traffic_source": cap["source"] if cap else None,
+                **capture_fields(cap, ph["decode_bytes_per_launch"], peaks),
                 "l2_note": ph["decode_pool_vs_l2"]}
 
     # ---- the other single-GPU configurations, three timed steps each, device-resident only -----
@@ -472,7 +487,8 @@ def run_gpu(args) -> None:
             m2 = measure_event(w2, args, dev, n_timed, 3, False)
             p2 = phase_numbers(w2, m2, peaks, False)
             label = name if not kw else f"{name}:B={kw['num_blocks']}"
-            per_config[label] = dict(p2, config=workload_desc(w2), ms_per_step=m2["ms"],
+            per_config[label] = dict(p2, **capture_fields(DECODE_CAPTURES.get(label), p2["decode_bytes_per_launch"], peaks),
+                                     config=workload_desc(w2), ms_per_step=m2["ms"],
                                      value=w2.num_blocks * w2.decode_steps / (m2["ms"] * 1e-3), steps=n_timed, warmup=3,
                                      clocks=m2["clocks"])
             del w2
