@@ -77,7 +77,9 @@ typedef struct cpa_config {
     int32_t head_dim;        /* 64 or 128 */
     int32_t page_size;       /* 16 */
     float   scale;           /* softmax scale, normally 1/sqrt(head_dim) */
-    int32_t q_tile_rows;     /* query rows per prefill work item: 128 or 256; 0 = default (256) */
+    int32_t q_tile_rows;     /* query rows per prefill work item: 128, 256, or 512 (items of 512 rows run on pairs of
+                                CTAs, cta_group::2: head_dim 128, plans without cached prefixes or chunks only;
+                                measured no faster than 256, kept as an option); 0 = default (256) */
     int32_t pages_per_split; /* KV pages per decode work item (<= 1024); 0 = chosen per block from the batch */
     int32_t num_sms;         /* SMs this plan's kernels may fill: the persistent prefill launches min(num_sms, units)
                                 CTAs (one per SM) and the decode wave is sized for 3 * num_sms CTAs; 0 = the SM
@@ -120,7 +122,9 @@ enum {
     CPA_PARAM_DECODE_WORKSPACE_BYTES = 6,/* size of cpa_decode's device workspace */
     CPA_PARAM_TOTAL_SPLITS = 7,          /* split_indptr[B] */
     CPA_PARAM_MAX_NEW_TOKENS = 8,
-    CPA_PARAM_PREFILL_CTAS = 9,          /* CTAs of the prefill launch = min(num_sms, prefill units) */
+    CPA_PARAM_PREFILL_CTAS = 9,          /* columns of CPA_ARR_PREFILL_SCHED: the CTAs of the prefill launch,
+                                            min(num_sms, prefill units), or for 512-row items its PAIRS of CTAs,
+                                            min(num_sms / 2 (at most what the device holds at a time), units) */
     CPA_PARAM_SHARED_CHUNK_PAGES = 10,   /* pages per chunk of the shared-prefix decode scan; 0 without cached prefixes */
     CPA_PARAM_CHUNK_TOKENS = 11,         /* tokens per prefill chunk; 0 = not a chunked plan */
     CPA_PARAM_NUM_STEPS = 12,            /* steps of a chunked plan's schedule */

@@ -167,6 +167,11 @@ static inline bool cpa_aligned16(const void* p) { return (reinterpret_cast<uintp
 int cpa_scan_tc(const cpa_plan* plan, const void* q, const void* k_pool, const void* v_pool, float* part_ml,
                 float* part_o, void* stream);
 
+// The prefill on pairs of CTAs (prefill_tc2.cu): plans whose q items have 512 rows (head_dim 128, no cached prefix).
+int cpa_prefill_pairs(const cpa_plan* plan, const void* q, const void* k, const void* v, void* o, void* stream);
+// Pairs of that kernel's CTAs the current device holds at a time; 0 without a device.
+int cpa_prefill_pair_capacity();
+
 // The tensor-core prefill over an explicit work list (a chunk step's items and deal); `items`, `sched` are device
 // pointers into the index buffer.  cpa_prefill_tc runs the plan's whole-block list.
 int cpa_prefill_tc_list(const cpa_plan* plan, const void* q, const void* k, const void* v, void* o, const void* k_pool,

@@ -86,7 +86,12 @@ int plan_create(const cpa_config* cfg, int32_t num_blocks, const int32_t* block_
     if ((cfg->head_dim != 64 && cfg->head_dim != 128) || cfg->page_size != 16 ||
         cfg->num_q_heads / cfg->num_kv_heads > 8)
         return CPA_EUNSUPPORTED;
-    if (cfg->q_tile_rows != 0 && cfg->q_tile_rows != 128 && cfg->q_tile_rows != 256) return CPA_EUNSUPPORTED;
+    if (cfg->q_tile_rows != 0 && cfg->q_tile_rows != 128 && cfg->q_tile_rows != 256 && cfg->q_tile_rows != 512)
+        return CPA_EUNSUPPORTED;
+    // 512-row items run on pairs of CTAs: head_dim 128, whole blocks without cached prefix or chunks
+    const bool pairs_possible = cfg->head_dim == 128 && !prefix_lens && chunk_tokens == 0 &&
+                                (cfg->num_sms == 0 || cfg->num_sms >= 2);
+    if (cfg->q_tile_rows == 512 && !pairs_possible) return CPA_EUNSUPPORTED;
     if (cfg->pages_per_split > kMaxSplitPages) return CPA_EUNSUPPORTED;
     // the schedule's sort keys hold a CTA id in 12 bits; the shared-scan items pack worker ranges in 16
     if (cfg->num_sms > kMaxPlanSms) return CPA_EUNSUPPORTED;
@@ -211,10 +216,26 @@ int plan_create(const cpa_config* cfg, int32_t num_blocks, const int32_t* block_
         std::vector<int32_t> item_cost((size_t)p->n_prefill);
         for (int32_t i = 0; i < p->n_prefill; ++i) {
             const int32_t b = p->prefill_items[2 * i], q0 = p->prefill_items[2 * i + 1] * p->q_tile;
+            if (p->q_tile == 512) {
+                // a pair of CTAs runs the item: slot s covers sub-tiles 2s and 2s+1 and streams tiles 0 .. t0+2s+1
+                const int32_t n_sub = std::min(4, (block_lens[b] - q0 + 127) / 128);
+                int32_t steps = q0 / 128 + (n_sub > 1 ? 2 : 1);
+                if (n_sub > 2) steps += q0 / 128 + (n_sub > 3 ? 4 : 3);
+                item_cost[(size_t)i] = 10 * steps + 18;
+                continue;
+            }
             const int32_t n_sub = (sub_per_item > 1 && block_lens[b] - q0 > 128) ? 2 : 1;
             item_cost[(size_t)i] = 10 * (p->prefix_lens[b] / 128 + q0 / 128 + n_sub) + 18;
         }
-        p->prefill_sched = deal_prefill_units(item_cost, Hq, G, p->num_sms, &p->prefill_ctas, &p->prefill_rounds);
+        // one schedule column per CTA, or per pair of CTAs for 512-row items (as many pairs as the device holds at
+        // a time, when there is a device to ask)
+        int32_t workers = p->num_sms;
+        if (p->q_tile == 512) {
+            workers = p->num_sms / 2;
+            const int32_t cap = cpa_prefill_pair_capacity();
+            if (cap > 0 && cfg->num_sms == 0) workers = std::min(workers, cap);
+        }
+        p->prefill_sched = deal_prefill_units(item_cost, Hq, G, workers, &p->prefill_ctas, &p->prefill_rounds);
     }
 
     // Decode splits.  Every CTA pays a fixed start-up and merge cost, so the planner aims at

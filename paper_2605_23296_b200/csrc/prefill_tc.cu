@@ -39,160 +39,10 @@
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 
-#include "cpa_device.cuh"
 #include "cpa_internal.h"
+#include "cpa_tcgen05.cuh"
 
 namespace {
-
-constexpr int kTileM = 128;        // query rows per CTA
-constexpr int kTileN = 128;        // keys per KV tile
-constexpr int kThreads = 384;        // 2 softmax warpgroups + 1 warpgroup holding the producer and issuer warps
-constexpr int kRegsSoftmax = 216;    // register split after launch (launch gives every thread 168):
-constexpr int kRegsControl = 72;     // 2*128*216 + 128*72 = 64512 = 384*168, exactly the launch total
-constexpr uint32_t kSpinLimit = 1u << 20;
-constexpr uint32_t kDrainLimit = 1u << 12;   // last look at work in flight after a wait gave up
-constexpr uint32_t kBlockBytes = 128 * 128;   // one column block: 128 rows x 128 B
-
-// ---------------------------------------------------------------- PTX wrappers
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-// Bounded wait with this file's limit (see mbar_wait): after it gave up once, `dead` turns every later wait into a no-op.
-__device__ __forceinline__ void tc_wait(uint32_t bar, uint32_t parity, bool& dead, int32_t* status) {
-    mbar_wait(bar, parity, dead, status, kSpinLimit);
-}
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
-    asm volatile(
-        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];\n"
-        :: "r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar) : "memory");
-}
-__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, int x, int y, int z, uint32_t bar) {
-    asm volatile(
-        "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];\n"
-        :: "r"(dst), "l"(map), "r"(x), "r"(y), "r"(z), "r"(bar) : "memory");
-}
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;\n" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory"); }
-// The issuing warp runs its loops convergently (all lanes), which lets the compiler keep MMA
-// operands on the uniform datapath; only the instruction itself is predicated on `leader`.
-__device__ __forceinline__ void tc_commit(uint32_t bar, uint32_t leader) {
-    asm volatile("{\n .reg .pred q;\n setp.ne.b32 q, %1, 0;\n"
-                 " @q tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n}\n"
-                 :: "r"(bar), "r"(leader) : "memory");
-}
-// D[tmem] (+)= A[smem desc] * B[smem desc]; `accumulate` = 0 overwrites D.  The descriptors are given
-// as 32-bit halves: `a_lo` / `b_lo` carry the start address (and the leading-dimension field), `hi`
-// is common to both operands; advancing an operand is one 32-bit add.
-__device__ __forceinline__ void tc_mma_ss_lo(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t hi, uint32_t idesc,
-                                             uint32_t accumulate, uint32_t leader) {
-    asm volatile(
-        "{\n .reg .pred p, q;\n .reg .b64 da, db;\n setp.ne.b32 p, %5, 0;\n setp.ne.b32 q, %6, 0;\n"
-        " mov.b64 da, {%1, %3};\n mov.b64 db, {%2, %3};\n"
-        " @q tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %4, p;\n}\n"
-        :: "r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(hi), "r"(idesc), "r"(accumulate), "r"(leader) : "memory");
-}
-// 32 consecutive fp32 columns of this thread's TMEM lane.
-__device__ __forceinline__ void tc_ld32(uint32_t taddr, float (&v)[32]) {
-    uint32_t r[32];
-    asm volatile(
-        "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
-        "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];\n"
-        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
-          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
-          "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
-          "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
-        : "r"(taddr) : "memory");
-    asm volatile("tcgen05.wait::ld.sync.aligned;\n" ::: "memory");
-#pragma unroll
-    for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
-}
-__device__ __forceinline__ void tc_st32(uint32_t taddr, const float (&v)[32]) {
-    asm volatile(
-        "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,"
-        "%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31,%32};\n"
-        :: "r"(taddr),
-           "r"(__float_as_uint(v[0])), "r"(__float_as_uint(v[1])), "r"(__float_as_uint(v[2])), "r"(__float_as_uint(v[3])),
-           "r"(__float_as_uint(v[4])), "r"(__float_as_uint(v[5])), "r"(__float_as_uint(v[6])), "r"(__float_as_uint(v[7])),
-           "r"(__float_as_uint(v[8])), "r"(__float_as_uint(v[9])), "r"(__float_as_uint(v[10])), "r"(__float_as_uint(v[11])),
-           "r"(__float_as_uint(v[12])), "r"(__float_as_uint(v[13])), "r"(__float_as_uint(v[14])), "r"(__float_as_uint(v[15])),
-           "r"(__float_as_uint(v[16])), "r"(__float_as_uint(v[17])), "r"(__float_as_uint(v[18])), "r"(__float_as_uint(v[19])),
-           "r"(__float_as_uint(v[20])), "r"(__float_as_uint(v[21])), "r"(__float_as_uint(v[22])), "r"(__float_as_uint(v[23])),
-           "r"(__float_as_uint(v[24])), "r"(__float_as_uint(v[25])), "r"(__float_as_uint(v[26])), "r"(__float_as_uint(v[27])),
-           "r"(__float_as_uint(v[28])), "r"(__float_as_uint(v[29])), "r"(__float_as_uint(v[30])), "r"(__float_as_uint(v[31]))
-        : "memory");
-}
-__device__ __forceinline__ void tc_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;\n" ::: "memory"); }
-
-__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
-    __nv_bfloat162 t = __floats2bfloat162_rn(lo, hi);
-    return *reinterpret_cast<uint32_t*>(&t);
-}
-
-// Shared-memory matrix descriptor, 128-byte swizzle, descriptor version 1 (sm_100).
-//   K-major operand  : rows 128 B apart, 8-row groups `sbo` bytes apart (1024); lbo unused (1 unit)
-//   MN-major operand : 64-element column blocks `lbo` bytes apart, 8-row (k) groups `sbo` bytes apart
-__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
-    uint64_t d = 0;
-    d |= (uint64_t)((addr >> 4) & 0x3FFF);
-    d |= (uint64_t)((lbo_bytes >> 4) & 0x3FFF) << 16;
-    d |= (uint64_t)((sbo_bytes >> 4) & 0x3FFF) << 32;
-    d |= (uint64_t)1 << 46;   // descriptor version
-    d |= (uint64_t)2 << 61;   // SWIZZLE_128B
-    return d;
-}
-// Instruction descriptor for kind::f16: bf16 x bf16 -> fp32, M x N, optional MN-major B.
-__host__ __device__ constexpr uint32_t instr_desc(int M, int N, bool b_mn_major) {
-    return (1u << 4) | (1u << 7) | (1u << 10) | ((b_mn_major ? 1u : 0u) << 16) | ((uint32_t)(N >> 3) << 17) |
-           ((uint32_t)(M >> 4) << 24);
-}
-
-// D[tmem] (+)= A[tmem] * B[smem desc]: A is a 128-lane x 16-element bf16 slice held in TMEM
-// (two consecutive K elements per 32-bit column, row = lane).
-__device__ __forceinline__ void tc_mma_ts_lo(uint32_t d_tmem, uint32_t a_tmem, uint32_t b_lo, uint32_t b_hi, uint32_t idesc,
-                                             uint32_t accumulate, uint32_t leader) {
-    asm volatile(
-        "{\n .reg .pred p, q;\n .reg .b64 db;\n setp.ne.b32 p, %5, 0;\n setp.ne.b32 q, %6, 0;\n"
-        " mov.b64 db, {%2, %3};\n"
-        " @q tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], db, %4, p;\n}\n"
-        :: "r"(d_tmem), "r"(a_tmem), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accumulate), "r"(leader) : "memory");
-}
-// 32 consecutive 32-bit columns of this thread's TMEM lane, no wait (pair with tc_wait_ld).
-__device__ __forceinline__ void tc_ld32_nowait(uint32_t taddr, uint32_t (&r)[32]) {
-    asm volatile(
-        "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
-        "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];\n"
-        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
-          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
-          "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
-          "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
-        : "r"(taddr) : "memory");
-}
-__device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;\n" ::: "memory"); }
-__device__ __forceinline__ void tc_st16(uint32_t taddr, const uint32_t (&v)[16]) {
-    asm volatile(
-        "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};\n"
-        :: "r"(taddr), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]),
-           "r"(v[8]), "r"(v[9]), "r"(v[10]), "r"(v[11]), "r"(v[12]), "r"(v[13]), "r"(v[14]), "r"(v[15])
-        : "memory");
-}
-// acc += lo(w) + hi(w), the two bf16 halves of w widened exactly (mixed-precision add)
-__device__ __forceinline__ void add_bf16x2(float& acc, uint32_t w) {
-    asm("{\n .reg .b16 lo, hi;\n mov.b32 {lo, hi}, %1;\n add.rn.f32.bf16 %0, lo, %0;\n add.rn.f32.bf16 %0, hi, %0;\n}\n"
-        : "+f"(acc) : "r"(w));
-}
-// (a, b) = (a, b) * s + c in one packed fp32 instruction
-__device__ __forceinline__ void fma_x2(float& a, float& b, float s, float c) {
-    uint64_t in, sc, cc, out;
-    asm("mov.b64 %0, {%1, %2};\n" : "=l"(in) : "f"(a), "f"(b));
-    asm("mov.b64 %0, {%1, %1};\n" : "=l"(sc) : "f"(s));
-    asm("mov.b64 %0, {%1, %1};\n" : "=l"(cc) : "f"(c));
-    asm("fma.rn.f32x2 %0, %1, %2, %3;\n" : "=l"(out) : "l"(in), "l"(sc), "l"(cc));
-    asm("mov.b64 {%0, %1}, %2;\n" : "=f"(a), "=f"(b) : "l"(out));
-}
-__device__ __forceinline__ float max3(float a, float b, float c) {
-    float d;
-    asm("max.f32 %0, %1, %2, %3;\n" : "=f"(d) : "f"(a), "f"(b), "f"(c));
-    return d;
-}
 
 constexpr int kMaxStages = 4;
 struct __align__(8) TcBarriers {
@@ -1078,25 +928,6 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
 }
 
 // ---------------------------------------------------------------- host side
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-EncodeTiledFn get_encode_fn() {
-    static EncodeTiledFn fn = nullptr;
-    if (!fn) {
-        void* p = nullptr;
-        cudaDriverEntryPointQueryResult qres;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) != cudaSuccess ||
-            qres != cudaDriverEntryPointSuccess) {
-            (void)cudaGetLastError();
-            return nullptr;
-        }
-        fn = reinterpret_cast<EncodeTiledFn>(p);
-    }
-    return fn;
-}
-
 // 2-D view [rows = tokens][cols = heads*D] of a packed token-major tensor; box = 64 cols x 128 rows.
 bool make_map(CUtensorMap* map, const void* ptr, int64_t rows, int64_t cols) {
     EncodeTiledFn fn = get_encode_fn();
@@ -1245,5 +1076,6 @@ int cpa_prefill_tc_list(const cpa_plan* plan, const void* q, const void* k, cons
 
 int cpa_prefill_tc(const cpa_plan* plan, const void* q, const void* k, const void* v, void* o, const void* k_pool,
                    const void* v_pool, void* stream) {
+    if (plan->q_tile == 512) return cpa_prefill_pairs(plan, q, k, v, o, stream);   // 512-row items run on pairs of CTAs
     return cpa_prefill_tc_list(plan, q, k, v, o, k_pool, v_pool, nullptr, nullptr, 0, 0, stream);
 }

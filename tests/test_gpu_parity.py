@@ -171,10 +171,11 @@ def test_prefill_kernels_agree_with_each_other():
     s.close()
 
 
-@pytest.mark.parametrize("q_tile_rows", [128, 256])
+@pytest.mark.parametrize("q_tile_rows", [128, 256, 512])
 def test_prefill_both_work_item_sizes(q_tile_rows):
+    # 128 / 256 rows per item: the one-CTA kernel; 512: the kernel on pairs of CTAs
     from paper_2605_23296_b200.session import CompactionSession
-    w = wl.custom([1, 128, 129, 255, 256, 257, 640], 8, 2, 128, steps=0, seed=23).materialise()
+    w = wl.custom([1, 128, 129, 255, 256, 257, 640, 385, 511, 512, 513, 1100], 8, 2, 128, steps=0, seed=23).materialise()
     s = CompactionSession(w.block_lens, 0, 8, 2, 128, w.free_pages, w.num_pages, scale=w.scale,
                           q_tile_rows=q_tile_rows)
     assert s.param(2) == q_tile_rows
