@@ -108,7 +108,10 @@ enum {
     CPA_ARR_CHUNK_ROWS = 11,   /* [CPA_PARAM_CHUNK_STEPS * (B+1)] chunked plans: per chunk index, prefix sums of the
                                   rows each block prefills in it */
     CPA_ARR_PAGES_ASSIGNED = 12, /* [B] plans with pages on demand: pages each block holds (as of creation or the last cpa_plan_sync) */
-    CPA_ARR_FREE_RING = 13     /* plans with pages on demand: the pages of the common reserve, in the order they will be handed out */
+    CPA_ARR_FREE_RING = 13,    /* plans with pages on demand: the pages of the common reserve, in the order they will be handed out */
+    CPA_ARR_SPLIT_RANGES = 14  /* [own splits, 2] (first own page, pages) of every decode split of a block's own pages,
+                                  block-major (the splits of block b are entries split_indptr[b] + slots of the shared
+                                  scan .. split_indptr[b+1]) */
 };
 
 /* Scalars of a plan, for cpa_plan_param. */
@@ -131,7 +134,9 @@ enum {
     CPA_PARAM_CHUNK_STEPS = 13,          /* chunk indices of the schedule (the most chunks of any block) */
     CPA_PARAM_DECODE_SMS = 14,           /* SMs a chunked plan leaves to the decode wave while a chunk is prefilled */
     CPA_PARAM_NUM_SMS = 15,              /* the plan's SM budget (cfg.num_sms, or the device's SM count for 0) */
-    CPA_PARAM_DECODE_STEPS_PER_CHUNK = 16 /* decode steps a chunked plan's schedule gives a chunk */
+    CPA_PARAM_DECODE_STEPS_PER_CHUNK = 16, /* decode steps a chunked plan's schedule gives a chunk */
+    CPA_PARAM_DECODE_EVEN_CUT = 17,      /* 1: the decode splits come from the even cut (see cpa_plan_create), 0: uniform per block */
+    CPA_PARAM_DECODE_CTAS = 18           /* CTAs of a decode launch */
 };
 
 /*
@@ -149,7 +154,14 @@ enum {
  *   count, ties by ascending block, kv head, split.  C_b is cfg->pages_per_split, or
  *   with 0 it is chosen per block so that all items fill one wave of CTAs (three per
  *   SM): splits start at one per block and the block with the largest splits is
- *   split further while kv_heads more items still fit (never below 4 pages).
+ *   split further while kv_heads more items still fit (never below 4 pages).  With 0 the
+ *   planner also tries the EVEN CUT: all blocks' pages laid end to end are cut into equal
+ *   ranges, one per group of kv_heads CTAs of the wave, so that every CTA streams the same
+ *   number of pages; block b then has a first split that ends at the next cut, full splits
+ *   of C pages and a remainder (CPA_ARR_SPLIT_RANGES lists them), and a CTA whose range
+ *   crosses a block boundary has two items.  It is taken when it loads the busiest SM at
+ *   least 5 % less than the uniform cut, a second item in a CTA counted as 16 pages (CPA_PARAM_DECODE_EVEN_CUT); CPA_ARR_DECODE_ITEMS
+ *   is then in launch order (CTA-major rounds) instead of descending size.
  * block_lens, free_pages: host int32 arrays (copied; caller keeps ownership).
  * Page ids must be >= 0 and distinct (distinctness is the caller's contract).
  * Errors: CPA_EINVAL (null pointer, num_blocks < 1, a length < 1,

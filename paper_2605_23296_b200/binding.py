@@ -25,7 +25,8 @@ ARR_SPLIT_PAGES = 8
 ARR_PREFILL_SCHED = 9
 ARR_DEC_START, ARR_CHUNK_ROWS = 10, 11
 ARR_PAGES_ASSIGNED, ARR_FREE_RING = 12, 13
-_ARR_WIDTH = {ARR_PREFILL_ITEMS: 2, ARR_DECODE_ITEMS: 3}
+ARR_SPLIT_RANGES = 14
+_ARR_WIDTH = {ARR_PREFILL_ITEMS: 2, ARR_DECODE_ITEMS: 3, 14: 2}
 
 PARAM_NUM_BLOCKS, PARAM_TOTAL_TOKENS, PARAM_Q_TILE_ROWS, PARAM_PAGES_PER_SPLIT = 0, 1, 2, 3
 PARAM_PAGES_USED, PARAM_INDEX_BYTES, PARAM_DECODE_WORKSPACE_BYTES, PARAM_TOTAL_SPLITS = 4, 5, 6, 7
@@ -34,6 +35,7 @@ PARAM_PREFILL_CTAS = 9
 PARAM_SHARED_CHUNK_PAGES = 10
 PARAM_CHUNK_TOKENS, PARAM_NUM_STEPS, PARAM_CHUNK_STEPS, PARAM_DECODE_SMS, PARAM_NUM_SMS = 11, 12, 13, 14, 15
 PARAM_DECODE_STEPS_PER_CHUNK = 16
+PARAM_DECODE_EVEN_CUT, PARAM_DECODE_CTAS = 17, 18
 
 
 class cpa_config(ctypes.Structure):

@@ -68,7 +68,10 @@ struct cpa_plan {
     std::vector<int32_t> prefix_lens;   // [B] tokens of each sequence that are cached before the plan starts (0: none)
     std::vector<int32_t> block_lens, cu_seqlens, page_indptr, page_indices, seq_lens, slot_mapping,
         prefill_items, prefill_sched, decode_items, split_indptr, split_pages;
-    int32_t n_prefill = 0, n_decode = 0;
+    std::vector<int32_t> split_ranges;   // [own splits, 2] (first own page, pages) of every own split, block-major
+    bool even_cut = false;               // the decode items come from the even cut of all own pages (see plan.cpp)
+    int32_t decode_grid = 0;             // CTAs of a decode launch (one wave at most; the even cut fixes it exactly)
+    int32_t n_prefill = 0, n_decode = 0; // n_decode: device items, fillers of the even cut included
     int32_t prefill_ctas = 0, prefill_rounds = 0;   // shape of prefill_sched
     // two-level decode of the prefix-aware layout: partial slots of each sequence that the shared-prefix
     // scan fills, its chunk size in pages, its work items and the shared pages' ids

@@ -125,6 +125,7 @@ decode_split_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __
     const int32_t* item = ix.decode_items + (int64_t)item_idx * ix.item_stride;
     const int4 hdr = *reinterpret_cast<const int4*>(item);
     const int b = hdr.x, g = hdr.y, s = hdr.z, n_reserved = hdr.w;
+    if (n_reserved == 0) continue;   // a filler of the even cut: this CTA has nothing in this round
     // A step of a chunked plan: only the blocks whose turn it is decode; the others sit the step out and their
     // output rows are not touched.  A block that is through with its tokens has its length carried into the
     // other length buffer by its first CTA (below); one that is still being prefilled has no length yet.
@@ -376,7 +377,13 @@ decode_split_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __
                 sm_o[warp][2 * tig + (e & 1)][8 * (8 * c + gid) + 2 * i + (e >> 1)] = acc[c][i][e];
     __syncthreads();
 
-    const int n_own = (pages_active - (first - s * C) + C - 1) / C;  // active splits of this block's own pages
+    // Active splits of this block's own pages.  The own pages (behind `skip` pages the shared scan covers) are cut
+    // into a first split of `head` pages and splits of C pages behind it (uniform cut: head = C; even cut: the first
+    // split ends where the cut through all blocks' pages falls).
+    const int skip = late_wait ? __ldg(ix.prefix_lens + b) / P : 0;
+    const int head = s == 0 ? n_reserved : (first - skip) - (s - 1) * C;
+    const int own_active = pages_active - skip;
+    const int n_own = own_active <= head ? 1 : 1 + (own_active - head + C - 1) / C;
     const int n_splits = n_fixed + n_own;                            // partials to merge
     const int64_t out_row = (int64_t)b * Hq + g * G;
     const int64_t prow = (int64_t)(ix.split_indptr[b] + slot) * Hq + g * G;
@@ -788,8 +795,9 @@ int launch_decode(const cpa_plan* plan, const void* q, const void* k_pool, const
     // stream drains; the kernel itself waits (griddepcontrol.wait) before it reads anything
     // that kernel wrote.
     cudaLaunchConfig_t cfg = {};
-    const int slots = 3 * (wave_sms > 0 ? wave_sms : plan->num_sms);   // resident CTAs: three per SM
-    cfg.gridDim = dim3(std::min(plan->n_decode, slots));
+    // one wave at most: the plan's grid (three CTAs per SM of its budget; with the even cut exactly the CTAs the cut
+    // was made for), or what fits beside a prefill chunk; CTAs loop over the items when there are more
+    cfg.gridDim = dim3(wave_sms > 0 ? std::min(plan->decode_grid, 3 * wave_sms) : plan->decode_grid);
     cfg.blockDim = dim3(kDecodeThreads);
     cfg.dynamicSmemBytes = kDecodeSmemBytes;
     cfg.stream = st;

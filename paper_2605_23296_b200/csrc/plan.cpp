@@ -309,27 +309,115 @@ int plan_create(const cpa_config* cfg, int32_t num_blocks, const int32_t* block_
             p->split_pages[b] = std::min(size, kMaxSplitPages);
         }
     }
-    p->C = *std::max_element(p->split_pages.begin(), p->split_pages.end());
-    struct DItem { int32_t pages, block, head, split; };
-    std::vector<DItem> dit;
-    p->split_indptr.assign(B + 1, 0);
-    for (int32_t b = 0; b < B; ++b) {
-        const int32_t Cb = p->split_pages[b];
-        const int32_t ns = (dec_pages[b] + Cb - 1) / Cb;
-        p->split_indptr[b + 1] = p->split_indptr[b] + p->n_fixed[b] + ns;
-        for (int32_t g = 0; g < cfg->num_kv_heads; ++g)
-            for (int32_t s = 0; s < ns; ++s)
-                dit.push_back({std::min(Cb, dec_pages[b] - s * Cb), b, g, s});
+    // The uniform cut: block b in splits of split_pages[b] pages, one item per (block, kv head, split), largest first.
+    struct DItem { int32_t pages, block, head, split, first; };   // first: first own page of the split; block < 0: filler
+    auto uniform_items = [&]() {
+        std::vector<DItem> v;
+        for (int32_t b = 0; b < B; ++b) {
+            const int32_t Cb = p->split_pages[b];
+            const int32_t ns = (dec_pages[b] + Cb - 1) / Cb;
+            for (int32_t g = 0; g < cfg->num_kv_heads; ++g)
+                for (int32_t s2 = 0; s2 < ns; ++s2)
+                    v.push_back({std::min(Cb, dec_pages[b] - s2 * Cb), b, g, s2, s2 * Cb});
+        }
+        std::stable_sort(v.begin(), v.end(), [](const DItem& x, const DItem& y) {
+            if (x.pages != y.pages) return x.pages > y.pages;
+            if (x.block != y.block) return x.block < y.block;
+            if (x.head != y.head) return x.head < y.head;
+            return x.split < y.split;
+        });
+        return v;
+    };
+    // What a launch costs with a given item list: CTA c takes items c, c + grid, ...; CTA c runs on SM c mod num_sms
+    // (three to an SM), which shares its bandwidth between them; every item also pays a fixed cost, the CTA's ring of
+    // stages running empty and filling again plus the merge, worth about sixteen pages of streaming (measured: a
+    // second item in a CTA costs about 9 us where a CTA streams 1.8 pages per us).  The figure is the load of the
+    // busiest SM.
+    auto busiest_sm = [&](const std::vector<DItem>& v, int64_t grid) {
+        std::vector<int64_t> load((size_t)p->num_sms, 0);
+        for (size_t i = 0; i < v.size(); ++i)
+            if (v[i].block >= 0) load[(size_t)(((int64_t)i % grid) % p->num_sms)] += v[i].pages + 16;
+        return *std::max_element(load.begin(), load.end());
+    };
+    std::vector<DItem> dit = uniform_items();
+    // The even cut (only when the split size is the planner's choice): all own pages of all blocks, laid end to end,
+    // are cut into equal ranges of `cut` pages, one range per group of kv_heads CTAs, so that every CTA of the wave
+    // streams the same number of pages whatever the blocks' lengths; a range that crosses a block boundary becomes
+    // two items of its CTAs.  Block b then has a first split that ends at the next cut, full splits behind it and a
+    // remainder.  Taken when the busiest SM gets at least 5 % less than with the uniform cut, which happens when
+    // there are more (block, kv head) pairs than CTAs in a wave, so that some CTAs would run two whole items.
+    p->even_cut = false;
+    if (cfg->pages_per_split == 0) {
+        int64_t total = 0;
+        for (int32_t b = 0; b < B; ++b) total += dec_pages[b];
+        const int64_t groups = std::max<int64_t>(1, 3LL * p->num_sms / cfg->num_kv_heads);
+        const int64_t cut = std::min<int64_t>(kMaxSplitPages, std::max<int64_t>(4, (total + groups - 1) / groups));
+        const int64_t n_ranges = (total + cut - 1) / cut;
+        const int64_t workers = std::min(groups, n_ranges);          // groups of kv_heads CTAs
+        std::vector<std::vector<DItem>> per_worker((size_t)workers);
+        // a block's first split is not left shorter than `least` pages: it takes the following range's pages along
+        // (that range's CTAs then stream up to `least` pages more than the others)
+        const int32_t least = cut + cut / 16 + 2 <= kMaxSplitPages ? (int32_t)std::max<int64_t>(2, cut / 16) : 0;
+        int64_t off = 0;
+        for (int32_t b = 0; b < B; ++b) {
+            int32_t pos = 0, s2 = 0;
+            while (pos < dec_pages[b]) {
+                int64_t range = (off + pos) / cut;
+                int32_t len = (int32_t)std::min<int64_t>(dec_pages[b] - pos, (range + 1) * cut - (off + pos));
+                if (s2 == 0 && len < least && dec_pages[b] > len) {
+                    ++range;
+                    len = (int32_t)std::min<int64_t>(dec_pages[b], (range + 1) * cut - off);
+                }
+                per_worker[(size_t)(range % workers)].push_back({len, b, 0, s2, pos});
+                pos += len;
+                ++s2;
+            }
+            off += dec_pages[b];
+        }
+        size_t rounds = 0;
+        for (const auto& w : per_worker) rounds = std::max(rounds, w.size());
+        std::vector<DItem> even;
+        even.reserve(rounds * (size_t)workers * (size_t)cfg->num_kv_heads);
+        for (size_t k = 0; k < rounds; ++k)
+            for (int64_t w = 0; w < workers; ++w)
+                for (int32_t g = 0; g < cfg->num_kv_heads; ++g) {
+                    if (k < per_worker[(size_t)w].size()) {
+                        DItem it = per_worker[(size_t)w][k];
+                        it.head = g;
+                        even.push_back(it);
+                    } else {
+                        even.push_back({0, -1, g, -1, 0});     // this CTA has nothing in this round
+                    }
+                }
+        p->decode_grid = (int32_t)std::min<int64_t>((int64_t)dit.size(), 3LL * p->num_sms);
+        if (busiest_sm(even, workers * cfg->num_kv_heads) * 100 < busiest_sm(dit, p->decode_grid) * 95) {
+            p->even_cut = true;
+            p->decode_grid = (int32_t)(workers * cfg->num_kv_heads);
+            dit.swap(even);
+            for (int32_t b = 0; b < B; ++b) p->split_pages[b] = (int32_t)cut;
+        }
     }
-    std::stable_sort(dit.begin(), dit.end(), [](const DItem& a, const DItem& c) {
-        if (a.pages != c.pages) return a.pages > c.pages;
-        if (a.block != c.block) return a.block < c.block;
-        if (a.head != c.head) return a.head < c.head;
-        return a.split < c.split;
-    });
+    if (!p->even_cut) p->decode_grid = (int32_t)std::min<int64_t>((int64_t)dit.size(), 3LL * p->num_sms);
+    p->C = *std::max_element(p->split_pages.begin(), p->split_pages.end());
+    p->split_indptr.assign(B + 1, 0);
+    {
+        std::vector<int32_t> n_own_splits(B, 0);
+        for (const DItem& it : dit)
+            if (it.block >= 0 && it.head == 0) n_own_splits[it.block] = std::max(n_own_splits[it.block], it.split + 1);
+        for (int32_t b = 0; b < B; ++b) p->split_indptr[b + 1] = p->split_indptr[b] + p->n_fixed[b] + n_own_splits[b];
+        // (first own page, pages) of every own split, block-major
+        p->split_ranges.assign((size_t)2 * (size_t)(p->split_indptr[B]), 0);
+        for (const DItem& it : dit)
+            if (it.block >= 0 && it.head == 0) {
+                const size_t at = (size_t)2 * (size_t)(p->split_indptr[it.block] + p->n_fixed[it.block] + it.split);
+                p->split_ranges[at] = it.first;
+                p->split_ranges[at + 1] = it.pages;
+            }
+    }
     p->n_decode = (int32_t)dit.size();
     p->decode_items.reserve(dit.size() * 3);
     for (const DItem& it : dit) {
+        if (it.block < 0) continue;      // the host's list names the real items, in launch order
         p->decode_items.push_back(it.block);
         p->decode_items.push_back(it.head);
         p->decode_items.push_back(it.split);
@@ -414,7 +502,9 @@ int plan_create(const cpa_config* cfg, int32_t num_blocks, const int32_t* block_
     p->off_pidx = w;    w = align4(w + pages_used);
     p->off_pitems = w;  w = align4(w + 4LL * p->n_prefill);
     p->off_psched = w;  w = align4(w + (int64_t)p->prefill_sched.size());
-    p->item_stride = 8 + (p->C + 3) / 4 * 4;
+    int32_t most_pages = p->C;      // (a first split of the even cut may be a little longer than the cut)
+    for (const DItem& it : dit) most_pages = std::max(most_pages, it.pages);
+    p->item_stride = 8 + (most_pages + 3) / 4 * 4;
     p->off_ditems = w;  w = align4(w + (int64_t)p->item_stride * p->n_decode);
     p->off_tickets = w; w = align4(w + (int64_t)B * cfg->num_kv_heads);
     p->off_seqlens2 = w; w = align4(w + B);
@@ -472,6 +562,10 @@ int plan_create(const cpa_config* cfg, int32_t num_blocks, const int32_t* block_
         // a decode item carries its own page ids, so the kernel's first KV load depends on
         // one prior load only
         int32_t* it = im + p->off_ditems + (int64_t)p->item_stride * i;
+        if (dit[i].block < 0) {          // filler: no pages, belongs to nobody (split -1 never takes a block's chores)
+            it[0] = 0; it[1] = dit[i].head; it[2] = -1; it[3] = 0; it[4] = 1; it[5] = 0; it[6] = 0; it[7] = 0;
+            continue;
+        }
         it[0] = dit[i].block;
         it[1] = dit[i].head;
         it[2] = dit[i].split;
@@ -480,7 +574,7 @@ int plan_create(const cpa_config* cfg, int32_t num_blocks, const int32_t* block_
         // where the split starts inside the sequence's page list (behind the pages the shared scan
         // covers), its partial slot among the sequence's slots, and how many slots come before
         const int32_t skip = two_level ? p->prefix_lens[dit[i].block] / P : 0;
-        it[5] = skip + dit[i].split * p->split_pages[dit[i].block];
+        it[5] = skip + dit[i].first;
         it[6] = p->n_fixed[dit[i].block] + dit[i].split;
         it[7] = p->n_fixed[dit[i].block];
         const int32_t* src = p->page_indices.data() + p->page_indptr[dit[i].block] + it[5];
@@ -571,6 +665,7 @@ extern "C" int cpa_plan_export(const cpa_plan* plan, int which, const int32_t** 
         case CPA_ARR_CHUNK_ROWS: v = &plan->chunk_rows; break;
         case CPA_ARR_PAGES_ASSIGNED: v = &plan->pages_assigned; break;
         case CPA_ARR_FREE_RING: v = &plan->free_ring; break;
+        case CPA_ARR_SPLIT_RANGES: v = &plan->split_ranges; div = 2; break;
         default: return CPA_EINVAL;
     }
     *ptr = v->data();
@@ -603,6 +698,8 @@ extern "C" int64_t cpa_plan_param(const cpa_plan* plan, int which) {
         case CPA_PARAM_DECODE_SMS: return plan->decode_sms;
         case CPA_PARAM_NUM_SMS: return plan->num_sms;
         case CPA_PARAM_DECODE_STEPS_PER_CHUNK: return plan->steps_per_chunk;
+        case CPA_PARAM_DECODE_EVEN_CUT: return plan->even_cut ? 1 : 0;
+        case CPA_PARAM_DECODE_CTAS: return plan->decode_grid;
         default: return CPA_EINVAL;
     }
 }

@@ -269,6 +269,38 @@ def test_fused_decode_append_matches_oracle_and_separate_calls(hq, hkv, d):
     plain.close()
 
 
+@pytest.mark.parametrize("nb,L,hq,hkv,d,sms", [(27, 1500, 8, 2, 128, 16), (25, 1000, 4, 1, 64, 8)])
+def test_decode_with_the_even_cut(nb, L, hq, hkv, d, sms):
+    # equal blocks whose count does not divide the wave: the planner cuts all pages, laid end to end, into equal
+    # ranges, so splits start and end inside blocks at odd places, CTAs have two items, and some items are fillers
+    from paper_2605_23296_b200 import binding as B
+    from paper_2605_23296_b200.session import CompactionSession
+    w = wl.custom([L] * nb, hq, hkv, d, steps=20, seed=nb + d).materialise()
+    sessions = [CompactionSession(w.block_lens, 20, hq, hkv, d, w.free_pages, w.num_pages, scale=w.scale,
+                                  poison_pools=True, num_sms=sms, pages_per_split=pps) for pps in (0, 37)]
+    assert sessions[0].param(B.PARAM_DECODE_EVEN_CUT) == 1 and sessions[1].param(B.PARAM_DECODE_EVEN_CUT) == 0
+    st = oa.DecodeState(w.k, w.v, _cu(w), 20)
+    for s in sessions:
+        s.append_prefill(_dev(w.k), _dev(w.v))
+    kd, vd, qd = _dev(w.k_dec), _dev(w.v_dec), _dev(w.q_dec)
+    for t in range(20):
+        st.append(w.k_dec[t], w.v_dec[t])
+        want = st.decode(w.q_dec[t], w.scale)
+        if t % 3 == 2:          # the separate calls now and then
+            sessions[0].append(kd[t], vd[t])
+            got = sessions[0].decode(qd[t])
+        else:
+            got = sessions[0].decode_append(qd[t], kd[t], vd[t])
+        assert_attention_close(_bits(got), want, f"even cut step {t}")
+        assert_attention_close(_bits(sessions[1].decode_append(qd[t], kd[t], vd[t])), want, f"uniform cut step {t}")
+    for s in sessions:
+        assert s.status() == 0
+        assert np.array_equal(s.export(3), w.block_lens + 20)
+    assert np.array_equal(_bits(sessions[0].k_pool), _bits(sessions[1].k_pool))
+    for s in sessions:
+        s.close()
+
+
 def test_decode_with_some_blocks_still_empty():
     # blocks 1 and 3 have nothing cached yet: their output rows are zero, the others are attended normally
     import torch

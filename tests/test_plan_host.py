@@ -50,6 +50,35 @@ def check_schedule(sched, ctas, prefill_items, block_lens, q_rows, num_q_heads, 
         assert load.max() <= balance * load.mean(), (load.max(), load.mean())
 
 
+def check_decode_cut(plan, own_pages, num_kv_heads, n_fixed=None):
+    """The decode splits, whichever way the planner cut them: the splits of a block tile its own pages in order
+    without gaps, all but the first and the last have the block's split size, every (block, kv head, split) is an
+    item exactly once, and the launch is one wave at most."""
+    B_ = len(own_pages)
+    n_fixed = n_fixed or [0] * B_
+    indptr = B.cpa_plan_export(plan, B.ARR_SPLIT_INDPTR)
+    ranges = B.cpa_plan_export(plan, B.ARR_SPLIT_RANGES)
+    C = B.cpa_plan_export(plan, B.ARR_SPLIT_PAGES)
+    want_items = set()
+    for b in range(B_):
+        rows = ranges[indptr[b] + n_fixed[b]:indptr[b + 1]]
+        assert len(rows) >= 1 and rows[0][0] == 0
+        pos = 0
+        for s, (first, pages) in enumerate(rows.tolist()):
+            assert first == pos and pages >= 1
+            if 0 < s < len(rows) - 1:
+                assert pages == C[b]
+            if s == len(rows) - 1 and s > 0:
+                assert pages <= C[b]
+            pos += pages
+            want_items |= {(b, g, s) for g in range(num_kv_heads)}
+        assert pos == own_pages[b]
+    items = [tuple(x) for x in B.cpa_plan_export(plan, B.ARR_DECODE_ITEMS).tolist()]
+    assert len(items) == len(set(items)) and set(items) == want_items
+    sms = B.cpa_plan_param(plan, B.PARAM_NUM_SMS)
+    assert 1 <= B.cpa_plan_param(plan, B.PARAM_DECODE_CTAS) <= 3 * sms
+
+
 def check_against_oracle(w, pages_per_split=0, permute=False, balance=None):
     free = None
     if permute:
@@ -67,10 +96,16 @@ def check_against_oracle(w, pages_per_split=0, permute=False, balance=None):
                  (B.ARR_PAGE_INDICES, "page_indices"), (B.ARR_SEQ_LENS, "seq_lens"),
                  (B.ARR_SLOT_MAPPING, "slot_mapping"), (B.ARR_PREFILL_ITEMS, "prefill_items"),
                  (B.ARR_DECODE_ITEMS, "decode_items"), (B.ARR_SPLIT_INDPTR, "split_indptr")]
+        even = B.cpa_plan_param(plan, B.PARAM_DECODE_EVEN_CUT)
+        assert not (even and pages_per_split)               # a given split size is kept
         for which, key in pairs:
+            if even and key in ("decode_items", "split_indptr"):
+                continue    # the even cut is a free choice of the planner: checked by what is fixed (below)
             got = B.cpa_plan_export(plan, which)
             want = np.asarray(ref[key], dtype=np.int32).reshape(got.shape)
             assert np.array_equal(got, want), key
+        own_pages = (-(-(w.block_lens.astype(np.int64) + w.decode_steps) // w.page_size)).tolist()
+        check_decode_cut(plan, own_pages, w.num_kv_heads)
         # the deal of prefill units to persistent CTAs: a free choice, checked by its invariants
         ctas = B.cpa_plan_param(plan, B.PARAM_PREFILL_CTAS)
         n_units = len(ref["prefill_items"]) * w.num_q_heads
@@ -80,11 +115,11 @@ def check_against_oracle(w, pages_per_split=0, permute=False, balance=None):
         assert B.cpa_plan_param(plan, B.PARAM_NUM_BLOCKS) == w.num_blocks
         assert B.cpa_plan_param(plan, B.PARAM_TOTAL_TOKENS) == w.total_tokens
         assert B.cpa_plan_param(plan, B.PARAM_PAGES_USED) == w.pages_needed
-        assert B.cpa_plan_param(plan, B.PARAM_TOTAL_SPLITS) == ref["split_indptr"][-1]
+        assert even or B.cpa_plan_param(plan, B.PARAM_TOTAL_SPLITS) == ref["split_indptr"][-1]
         assert B.cpa_plan_param(plan, B.PARAM_MAX_NEW_TOKENS) == w.decode_steps
-        rows = ref["split_indptr"][-1] * w.num_q_heads
+        rows = B.cpa_plan_param(plan, B.PARAM_TOTAL_SPLITS) * w.num_q_heads
         assert B.cpa_plan_param(plan, B.PARAM_DECODE_WORKSPACE_BYTES) >= rows * (w.head_dim + 2) * 4
-        return C
+        return C, even
     finally:
         B.cpa_plan_destroy(plan)
 
@@ -104,7 +139,9 @@ def test_plan_bit_exact_edge_lengths():
 @pytest.mark.parametrize("name", ["dense8b", "ragged", "moe120b"])
 def test_plan_bit_exact_full_configs(name):
     w = wl.CONFIGS[name]()
-    C = check_against_oracle(w, 0, permute=(name == "ragged"), balance=1.05)
+    C, even = check_against_oracle(w, 0, permute=(name == "ragged"), balance=1.05)
+    if even:
+        return      # the even cut has its own invariants (check_decode_cut)
     pages = (w.block_lens.astype(np.int64) + w.decode_steps + 15) // 16
     n_items = int((w.num_kv_heads * -(-pages // np.asarray(C))).sum())
     assert n_items <= 3 * 148                       # one wave of three CTAs per SM
@@ -119,6 +156,29 @@ def test_plan_bit_exact_full_configs(name):
 @pytest.mark.parametrize("nb", [1, 2, 8, 64])
 def test_plan_bit_exact_split_sweep(nb):
     check_against_oracle(wl.split_sweep(nb), 0)
+
+
+def test_even_cut_for_equal_blocks_that_do_not_divide_the_wave():
+    # 64 x 2048 tokens, 8 kv heads: 512 (block, head) pairs against 444 CTAs of a wave.  One split per block leaves 68
+    # CTAs with two items; the even cut gives every CTA the same pages.
+    w = wl.split_sweep(64)
+    plan, _ = make_plan(w, 0)
+    try:
+        assert B.cpa_plan_param(plan, B.PARAM_DECODE_EVEN_CUT) == 1
+        pages = (-(-(w.block_lens.astype(np.int64) + w.decode_steps) // 16)).tolist()
+        check_decode_cut(plan, pages, w.num_kv_heads)
+        ctas = B.cpa_plan_param(plan, B.PARAM_DECODE_CTAS)
+        C = B.cpa_plan_param(plan, B.PARAM_PAGES_PER_SPLIT)
+        assert ctas % w.num_kv_heads == 0 and ctas <= 444
+        assert C == -(-sum(pages) // (ctas // w.num_kv_heads))          # equal ranges over all pages laid end to end
+        ranges = B.cpa_plan_export(plan, B.ARR_SPLIT_RANGES)
+        assert ranges[:, 1].max() <= C + C // 16 + 2
+    finally:
+        B.cpa_plan_destroy(plan)
+    # a split size given by the caller is kept as it is
+    plan, _ = make_plan(w, 100)
+    assert B.cpa_plan_param(plan, B.PARAM_DECODE_EVEN_CUT) == 0
+    B.cpa_plan_destroy(plan)
 
 
 def test_auto_split_aims_at_the_sm_count():
@@ -332,12 +392,17 @@ def test_prefix_plan_bit_exact(pps):
         ref = op.build_plan(o.block_lens.tolist(), o.decode_steps, o.page_size, o.free_pages.tolist(), o.num_kv_heads,
                             M, C, prefix_lens=w.prefix_lens.tolist(), shared_pages=w.shared_pages.tolist(),
                             shared_chunk_pages=CH)
+        even = B.cpa_plan_param(plan, B.PARAM_DECODE_EVEN_CUT)
         for which, key in [(B.ARR_CU_SEQLENS, "cu_seqlens"), (B.ARR_PAGE_INDPTR, "page_indptr"),
                            (B.ARR_PAGE_INDICES, "page_indices"), (B.ARR_SEQ_LENS, "seq_lens"),
                            (B.ARR_SLOT_MAPPING, "slot_mapping"), (B.ARR_PREFILL_ITEMS, "prefill_items"),
                            (B.ARR_DECODE_ITEMS, "decode_items"), (B.ARR_SPLIT_INDPTR, "split_indptr")]:
+            if even and key in ("decode_items", "split_indptr"):
+                continue
             got = B.cpa_plan_export(plan, which)
             assert np.array_equal(got, np.asarray(ref[key], dtype=np.int32).reshape(got.shape)), key
+        own = (-(-(o.block_lens.astype(np.int64) + o.decode_steps) // o.page_size)).tolist()
+        check_decode_cut(plan, own, o.num_kv_heads, n_fixed=[-(-(int(x) // o.page_size) // CH) for x in w.prefix_lens])
         ctas = B.cpa_plan_param(plan, B.PARAM_PREFILL_CTAS)
         check_schedule(B.cpa_plan_export(plan, B.ARR_PREFILL_SCHED), ctas, ref["prefill_items"], o.block_lens, M,
                        o.num_q_heads, o.num_kv_heads, prefix_lens=w.prefix_lens)
