@@ -215,6 +215,28 @@ def prefill_prefix_aware(q: np.ndarray, k: np.ndarray, v: np.ndarray, cu_seqlens
     return out
 
 
+def prefill_chunk_prefix_aware(q: np.ndarray, k: np.ndarray, v: np.ndarray, cu_seqlens: Sequence[int],
+                               k_hist: np.ndarray, v_hist: np.ndarray, prefix_lens: Sequence[int], scale: float,
+                               worker: int, first_row: int, n_rows: int) -> np.ndarray:
+    """One chunk of a worker's chunked prefill in the prefix-aware layout (Section 4 "Dispatch" for the prompt,
+    Section 4.2 for prefix caching and chunked prefill being on together in the paper's serving engine).
+
+    Worker w's prompt is its history prefix followed by its own tokens.  When rows [first_row, first_row + n_rows)
+    of the own tokens are prefilled, the later own tokens do not exist yet: the chunk attends, causally, over the
+    prefix and the own tokens [0, first_row + n_rows).  Written as that: the prompt is cut off behind the chunk and
+    plain causal attention is evaluated for the chunk's rows.  Returns float64 [n_rows, Hq, d].
+    """
+    lo, n_pre = int(cu_seqlens[worker]), int(prefix_lens[worker])
+    end = first_row + n_rows
+    assert 0 <= first_row and n_rows >= 1 and lo + end <= int(cu_seqlens[worker + 1])
+    Hq, d = q.shape[1], q.shape[2]
+    prompt_k = np.concatenate([k_hist[:n_pre], k[lo:lo + end]])
+    prompt_v = np.concatenate([v_hist[:n_pre], v[lo:lo + end]])
+    prompt_q = np.concatenate([np.zeros((n_pre, Hq, d), dtype=np.uint16), q[lo:lo + end]])
+    return prefill(prompt_q, prompt_k, prompt_v, [0, n_pre + end], scale,
+                   rows=np.arange(n_pre + first_row, n_pre + end, dtype=np.int64))
+
+
 class PrefixDecodeState(DecodeState):
     """Decode in the prefix-aware layout: worker w's cache is its prompt (history prefix, then its
     own tokens), kept contiguously per worker and extended one token per step."""

@@ -122,3 +122,24 @@ def test_decode_state_lets_blocks_sit_a_step_out():
     want = oa.attend_token(w.q_dec[0][1], np.concatenate([w.k[20:50], w.k_dec[0][1:2]]),
                            np.concatenate([w.v[20:50], w.v_dec[0][1:2]]), w.scale)
     assert np.array_equal(out[1], want) and np.isnan(out[0]).all()
+
+
+def test_prefix_aware_chunk_rows_equal_the_unchunked_prefix_aware_rows_bitwise():
+    # the same identity with a cached history in front: chunking a worker's own tokens changes none of its rows
+    pw = wl.prefix_aware(3, 128, 4, 2, 64, steps=0, seed=12, marker_tokens=45).materialise(with_decode=False)
+    o = pw.own
+    cu = np.concatenate([[0], np.cumsum(o.block_lens.astype(np.int64))])
+    full = oa.prefill_prefix_aware(o.q, o.k, o.v, cu, pw.k_hist, pw.v_hist, pw.prefix_lens, o.scale)
+    for st in op.mixed_schedule(o.block_lens.tolist(), 128, 0):
+        for w, first, n in st["prefill"]:
+            got = oa.prefill_chunk_prefix_aware(o.q, o.k, o.v, cu, pw.k_hist, pw.v_hist, pw.prefix_lens, o.scale, w, first, n)
+            assert np.array_equal(got, full[cu[w] + first: cu[w] + first + n])
+    # worker 0 has no prefix: its chunks are the independent-chunks ones
+    got = oa.prefill_chunk_prefix_aware(o.q, o.k, o.v, cu, pw.k_hist, pw.v_hist, pw.prefix_lens, o.scale, 0, 128, 45)
+    assert np.array_equal(got, oa.prefill_chunk(o.q, o.k, o.v, cu, o.scale, 0, 128, 45))
+    # a chunk of worker 2 sees the history inside its prefix and not the history beyond it
+    base = oa.prefill_chunk_prefix_aware(o.q, o.k, o.v, cu, pw.k_hist, pw.v_hist, pw.prefix_lens, o.scale, 2, 128, 45)
+    kh = pw.k_hist.copy()
+    kh[3] ^= 0x0100
+    moved = oa.prefill_chunk_prefix_aware(o.q, o.k, o.v, cu, kh, pw.v_hist, pw.prefix_lens, o.scale, 2, 128, 45)
+    assert (np.abs(moved - base).max(axis=(1, 2)) > 0).all()
