@@ -231,6 +231,24 @@ CPA_API int cpa_plan_create_chunked(const cpa_config* cfg, int32_t num_blocks, c
                                     int32_t decode_sms, const int32_t* free_pages, int32_t num_free, cpa_plan** out);
 
 /*
+ * cpa_plan_create_prefix_chunked -- the prefix-aware layout and chunked prefill together, which is how the
+ * paper's serving engine runs (Section 4.2: automatic prefix caching and chunked prefill both enabled;
+ * Section 4, "Dispatch": every worker's prompt extends the previous worker's).  Worker w reads prefix_lens[w]
+ * cached history tokens from `shared_pages` (as for cpa_plan_create_prefix) and runs its own_lens[w] tokens
+ * in chunks of chunk_tokens (as for cpa_plan_create_chunked): chunk c of worker w attends the cached history,
+ * then the worker's earlier chunks (already in its own pages), then causally itself; its keys and values land
+ * at sequence positions prefix_lens[w] + c * chunk_tokens + i; the worker's first decode step starts from the
+ * length prefix_lens[w] + own_lens[w].  The schedule (chunk c at step c * r, summary token t at step
+ * n_w * r + t), the arguments and cpa_step_mixed are those of cpa_plan_create_chunked; decode runs in the
+ * two levels of cpa_plan_create_prefix.  Errors: the union of the two creators'.
+ */
+CPA_API int cpa_plan_create_prefix_chunked(const cpa_config* cfg, int32_t num_workers, const int32_t* own_lens,
+                                           const int32_t* prefix_lens, const int32_t* shared_pages,
+                                           int32_t num_shared, int32_t max_new_tokens, int32_t chunk_tokens,
+                                           int32_t decode_steps_per_chunk, int32_t decode_sms,
+                                           const int32_t* free_pages, int32_t num_free, cpa_plan** out);
+
+/*
  * cpa_plan_create_dynamic -- a plan that reserves no pages for the summaries.  The paper's outlook (Section 8,
  * "Dynamic block size and prompt selection") wants block sizes and summary lengths that are not fixed in
  * advance, and its second benchmark (Section 3.1: documents of about 0.7k tokens, six questions each) is many

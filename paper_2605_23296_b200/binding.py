@@ -67,6 +67,10 @@ _lib.cpa_plan_create_prefix.restype = ctypes.c_int
 _lib.cpa_plan_create_chunked.argtypes = [ctypes.POINTER(cpa_config), ctypes.c_int32, _i32p, ctypes.c_int32, ctypes.c_int32,
                                          ctypes.c_int32, ctypes.c_int32, _i32p, ctypes.c_int32, ctypes.POINTER(_vp)]
 _lib.cpa_plan_create_chunked.restype = ctypes.c_int
+_lib.cpa_plan_create_prefix_chunked.argtypes = [ctypes.POINTER(cpa_config), ctypes.c_int32, _i32p, _i32p, _i32p,
+                                                ctypes.c_int32, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32,
+                                                ctypes.c_int32, _i32p, ctypes.c_int32, ctypes.POINTER(_vp)]
+_lib.cpa_plan_create_prefix_chunked.restype = ctypes.c_int
 _lib.cpa_plan_create_dynamic.argtypes = [ctypes.POINTER(cpa_config), ctypes.c_int32, _i32p, ctypes.c_int32, _i32p,
                                          ctypes.c_int32, ctypes.POINTER(_vp)]
 _lib.cpa_plan_create_dynamic.restype = ctypes.c_int
@@ -169,6 +173,25 @@ def cpa_plan_create_chunked(cfg: cpa_config, block_lens: Sequence[int], max_new_
         return rc, out.value
     if rc != CPA_OK:
         raise CpaError(rc, "cpa_plan_create_chunked")
+    return out.value
+
+
+def cpa_plan_create_prefix_chunked(cfg: cpa_config, own_lens: Sequence[int], prefix_lens: Sequence[int],
+                                   shared_pages: Sequence[int], max_new_tokens: int, chunk_tokens: int,
+                                   free_pages: Sequence[int], decode_sms: int = 0, decode_steps_per_chunk: int = 1,
+                                   check: bool = True):
+    """Plan of the prefix-aware layout with chunked prefill; the handle, or (status, handle) with check=False."""
+    lens, pre, shared, free = _i32(own_lens), _i32(prefix_lens), _i32(shared_pages), _i32(free_pages)
+    out = _vp()
+    rc = _lib.cpa_plan_create_prefix_chunked(ctypes.byref(cfg), lens.shape[0], lens.ctypes.data_as(_i32p),
+                                             pre.ctypes.data_as(_i32p), shared.ctypes.data_as(_i32p), shared.shape[0],
+                                             int(max_new_tokens), int(chunk_tokens), int(decode_steps_per_chunk),
+                                             int(decode_sms), free.ctypes.data_as(_i32p), free.shape[0],
+                                             ctypes.byref(out))
+    if not check:
+        return rc, out.value
+    if rc != CPA_OK:
+        raise CpaError(rc, "cpa_plan_create_prefix_chunked")
     return out.value
 
 

@@ -168,7 +168,7 @@ static inline bool cpa_aligned16(const void* p) { return (reinterpret_cast<uintp
 // Shared-prefix scan of the prefix-aware decode on the tensor-core path (prefill_tc.cu): partials of every
 // (worker, head) row for every chunk of shared pages go to part_ml / part_o.
 int cpa_scan_tc(const cpa_plan* plan, const void* q, const void* k_pool, const void* v_pool, float* part_ml,
-                float* part_o, void* stream);
+                float* part_o, int wave_sms, void* stream);
 
 // The prefill on pairs of CTAs (prefill_tc2.cu): plans whose q items have 512 rows (head_dim 128, no cached prefix).
 int cpa_prefill_pairs(const cpa_plan* plan, const void* q, const void* k, const void* v, void* o, void* stream);

@@ -164,7 +164,8 @@ decode_split_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __
     const bool fused = fa.k_new != nullptr;
     // (a block of a chunked plan enters its first decode step with its whole prompt cached, whatever the
     // length buffers hold: the chunks that cached it ran beside earlier decode launches)
-    const int len_old = (mode.step >= 0 && sched_pos == 0) ? ix.cu_seqlens[b + 1] - ix.cu_seqlens[b] : ix.seq_lens[b];
+    const int len_old = (mode.step >= 0 && sched_pos == 0)
+                            ? ix.prefix_lens[b] + ix.cu_seqlens[b + 1] - ix.cu_seqlens[b] : ix.seq_lens[b];
     if (mode.dynamic) {
         // Pages on demand.  A block takes part unless the caller's flag says it has stopped.  The page its new
         // token goes to was taken from the reserve when the page before it filled up; if the reserve was empty
@@ -783,7 +784,7 @@ int launch_decode(const cpa_plan* plan, const void* q, const void* k_pool, const
     // to the first slots of every worker and are merged by the launch below, which follows in the stream.
     if (plan->n_shared > 0) {
         if (cpa_scan_rows(G) == 128) {   // the tensor-core scan (its query tile is loaded in boxes of 8/G sequences)
-            const int rc = cpa_scan_tc(plan, q, k_pool, v_pool, part_ml, part_o, st);
+            const int rc = cpa_scan_tc(plan, q, k_pool, v_pool, part_ml, part_o, wave_sms, st);
             if (rc != CPA_OK) return rc;
         } else {
             decode_shared_kernel<D><<<plan->n_shared, kSharedThreads, kSharedSmemBytes, st>>>(

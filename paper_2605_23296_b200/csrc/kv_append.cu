@@ -77,9 +77,10 @@ __global__ void kv_append_chunk_kernel(const uint4* __restrict__ k, const uint4*
             if (rows_indptr[mid] <= r) lo = mid; else hi = mid - 1;
         }
         const int b = lo;
-        const int pos = first_pos + (r - rows_indptr[b]);
+        const int own = first_pos + (r - rows_indptr[b]);       // position among the block's own tokens
+        const int pos = ix.prefix_lens[b] + own;                 // position in the sequence (behind a cached prefix)
         const int64_t page = ix.page_indices[ix.page_indptr[b] + pos / P];
-        const int64_t row = ((int64_t)ix.cu_seqlens[b] + pos) * Hkv * chunks_per_head;
+        const int64_t row = ((int64_t)ix.cu_seqlens[b] + own) * Hkv * chunks_per_head;
         copy_row_chunks(k + row, v + row, k_pool, v_pool, page, pos % P, Hkv, chunks_per_head, P);
     }
 }

@@ -88,13 +88,13 @@ extern "C" int cpa_step_mixed(cpa_plan* plan, int32_t step, const void* q, const
         // host mirror of the lengths; the other length buffer is now the current one
         for (int b = 0; b < B; ++b) {
             const int pos = step - plan->dec_start[b];
-            if (pos >= 0 && pos < T) plan->seq_lens[b] = plan->block_lens[b] + pos + 1;
+            if (pos >= 0 && pos < T) plan->seq_lens[b] = plan->prefix_lens[b] + plan->block_lens[b] + pos + 1;
         }
         plan->cur_lens ^= 1;
     }
     for (int b = 0; b < B; ++b)   // (mirror: a block's prompt counts as cached once its last chunk has been started)
         if (starts_chunk && step < plan->dec_start[b])
-            plan->seq_lens[b] = std::min(plan->block_lens[b], (chunk + 1) * plan->chunk);
+            plan->seq_lens[b] = plan->prefix_lens[b] + std::min(plan->block_lens[b], (chunk + 1) * plan->chunk);
     if (last)
         if ((rc = join()) != CPA_OK) return rc;
     plan->next_step = step + 1;

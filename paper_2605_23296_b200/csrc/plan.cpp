@@ -98,7 +98,6 @@ int plan_create(const cpa_config* cfg, int32_t num_blocks, const int32_t* block_
     if (prefix_lens && num_blocks > 0xFFFF) return CPA_EUNSUPPORTED;
     // a chunk is read back as a cached prefix of whole 128-key tiles
     if (chunk_tokens < 0 || chunk_tokens % 128 != 0 || decode_sms < 0 || steps_per_chunk < 1) return CPA_EINVAL;
-    if (chunk_tokens > 0 && prefix_lens) return CPA_EUNSUPPORTED;
     if (dynamic && (chunk_tokens > 0 || prefix_lens)) return CPA_EUNSUPPORTED;
 
     cpa_plan* p = new (std::nothrow) cpa_plan();
@@ -460,7 +459,7 @@ int plan_create(const cpa_config* cfg, int32_t num_blocks, const int32_t* block_
                 const int32_t len = std::min(Cc, block_lens[b] - st * Cc);
                 rows += len;
                 for (int32_t t = 0; t * p->q_tile < len; ++t)
-                    cit.push_back({st * Cc + std::min((t + 1) * p->q_tile, len), b, t});
+                    cit.push_back({p->prefix_lens[b] + st * Cc + std::min((t + 1) * p->q_tile, len), b, t});
             }
             chunk_rows.push_back(rows);
             cs.rows = rows;
@@ -476,14 +475,16 @@ int plan_create(const cpa_config* cfg, int32_t num_blocks, const int32_t* block_
                 const int32_t b = cit[i].block, q0 = cit[i].tile * p->q_tile;
                 const int32_t len = std::min(Cc, block_lens[b] - st * Cc);
                 const int32_t n_sub = (p->q_tile > 128 && len - q0 > 128) ? 2 : 1;
-                item_cost[i] = 10 * (st * Cc / 128 + q0 / 128 + n_sub) + 18;
-                // the chunk is a "block" of its own whose cached prefix is the block's earlier chunks
+                // the chunk is a "block" of its own whose cached prefix is the sequence's cached history (prefix-aware
+                // layout) followed by the block's earlier chunks
+                const int32_t pre_tiles = (p->prefix_lens[b] + st * Cc) / 128;
+                if (pre_tiles > 0x7FFF) { delete p; return CPA_EUNSUPPORTED; }
+                item_cost[i] = 10 * (pre_tiles + q0 / 128 + n_sub) + 18;
                 chunk_items.push_back(p->cu_seqlens[b] + st * Cc);
                 chunk_items.push_back(len);
-                chunk_items.push_back(cit[i].tile | ((st * Cc / 128) << 16));
+                chunk_items.push_back(cit[i].tile | (pre_tiles << 16));
                 chunk_items.push_back(p->page_indptr[b]);
             }
-            if ((int64_t)st * Cc / 128 > 0x7FFF) { delete p; return CPA_EUNSUPPORTED; }
             const int32_t budget = any_decode ? p->num_sms - p->decode_sms : p->num_sms;
             std::vector<int32_t> sched = deal_prefill_units(item_cost, Hq, G, budget, &cs.ctas, &cs.rounds);
             cs.off_sched = (int64_t)chunk_sched.size();
@@ -644,6 +645,17 @@ extern "C" int cpa_plan_create_prefix(const cpa_config* cfg, int32_t num_workers
     if (!prefix_lens) return CPA_EINVAL;
     return plan_create(cfg, num_workers, own_lens, prefix_lens, shared_pages, num_shared, max_new_tokens, free_pages,
                        num_free, 0, 0, 1, false, out);
+}
+
+extern "C" int cpa_plan_create_prefix_chunked(const cpa_config* cfg, int32_t num_workers, const int32_t* own_lens,
+                                              const int32_t* prefix_lens, const int32_t* shared_pages, int32_t num_shared,
+                                              int32_t max_new_tokens, int32_t chunk_tokens, int32_t decode_steps_per_chunk,
+                                              int32_t decode_sms, const int32_t* free_pages, int32_t num_free,
+                                              cpa_plan** out) {
+    if (out) *out = nullptr;
+    if (!prefix_lens || chunk_tokens < 128) return CPA_EINVAL;
+    return plan_create(cfg, num_workers, own_lens, prefix_lens, shared_pages, num_shared, max_new_tokens, free_pages,
+                       num_free, chunk_tokens, decode_sms, decode_steps_per_chunk, false, out);
 }
 
 extern "C" int cpa_plan_export(const cpa_plan* plan, int which, const int32_t** ptr, int64_t* count) {

@@ -1026,7 +1026,7 @@ bool make_q_rows_map(CUtensorMap* map, const void* ptr, int64_t seqs, int64_t he
 
 template <int D>
 int launch_scan_tc(const cpa_plan* plan, const void* q, const void* k_pool, const void* v_pool, float* part_ml,
-                   float* part_o, cudaStream_t st) {
+                   float* part_o, int wave_sms, cudaStream_t st) {
     const cpa_config& c = plan->cfg;
     constexpr int smem = ScanShape<D>::kSmem;
     static std::atomic<bool> configured_dev[64];
@@ -1049,7 +1049,7 @@ int launch_scan_tc(const cpa_plan* plan, const void* q, const void* k_pool, cons
     if (!make_q_rows_map(&tm_q, q, plan->B, c.num_q_heads, D, G) ||
         !make_pool_map(&tm_kpool, k_pool, pool_rows, D) || !make_pool_map(&tm_vpool, v_pool, pool_rows, D))
         return CPA_ECUDA;
-    const int sms = plan->num_sms;
+    const int sms = wave_sms > 0 ? wave_sms : plan->num_sms;   // (beside a prefill chunk: the SMs left to the decode)
     const int grid = plan->n_shared < sms ? plan->n_shared : sms;
     scan_tc_kernel<D><<<grid, kScanThreads, smem, st>>>(tm_q, tm_kpool, tm_vpool, part_ml, part_o, plan->dev(),
                                                        c.num_q_heads, c.num_kv_heads, G, c.scale * 1.4426950408889634f,
@@ -1060,10 +1060,10 @@ int launch_scan_tc(const cpa_plan* plan, const void* q, const void* k_pool, cons
 }  // namespace
 
 int cpa_scan_tc(const cpa_plan* plan, const void* q, const void* k_pool, const void* v_pool, float* part_ml,
-                float* part_o, void* stream) {
+                float* part_o, int wave_sms, void* stream) {
     cudaStream_t st = (cudaStream_t)stream;
-    return plan->cfg.head_dim == 128 ? launch_scan_tc<128>(plan, q, k_pool, v_pool, part_ml, part_o, st)
-                                     : launch_scan_tc<64>(plan, q, k_pool, v_pool, part_ml, part_o, st);
+    return plan->cfg.head_dim == 128 ? launch_scan_tc<128>(plan, q, k_pool, v_pool, part_ml, part_o, wave_sms, st)
+                                     : launch_scan_tc<64>(plan, q, k_pool, v_pool, part_ml, part_o, wave_sms, st);
 }
 
 int cpa_prefill_tc_list(const cpa_plan* plan, const void* q, const void* k, const void* v, void* o, const void* k_pool,

@@ -57,8 +57,11 @@ class CompactionSession:
         if dynamic_pages:       # no pages reserved for the summaries: blocks draw from a common reserve as they grow
             assert prefix_lens is None and not chunk_tokens
             self.plan = B.cpa_plan_create_dynamic(self.cfg, self.block_lens, max_new_tokens, free_pages)
+        elif chunk_tokens and self.prefix_aware:   # both: cached history prefix, own tokens in chunks
+            self.plan = B.cpa_plan_create_prefix_chunked(self.cfg, self.block_lens, prefix_lens, shared_pages,
+                                                         max_new_tokens, chunk_tokens, free_pages, decode_sms,
+                                                         decode_steps_per_chunk)
         elif chunk_tokens:      # prefill in chunks, mixed with the decode of blocks that are past their prompt
-            assert prefix_lens is None
             self.plan = B.cpa_plan_create_chunked(self.cfg, self.block_lens, max_new_tokens, chunk_tokens, free_pages,
                                                   decode_sms, decode_steps_per_chunk)
         elif self.prefix_aware:   # the paper's layout: cached history prefix + own tokens per worker

@@ -18,7 +18,7 @@ block lengths, page permutation, Q, K, V, outlier positions, decode q/k/v.
 from __future__ import annotations
 
 from dataclasses import dataclass, field
-from typing import Optional
+from typing import Optional, Sequence
 
 import numpy as np
 
@@ -222,13 +222,16 @@ class PrefixWorkload:
 
 
 def prefix_aware(num_workers: int, block_len: int, hq: int, hkv: int, d: int, steps: int, seed: int = 11,
-                 marker_tokens: int = 16, permute_pages: bool = True, own_len: int = 0) -> PrefixWorkload:
+                 marker_tokens: int = 16, permute_pages: bool = True, own_len: int = 0,
+                 own_lens: Optional[Sequence[int]] = None) -> PrefixWorkload:
     """`num_workers` workers over a history of blocks of `block_len` tokens (a multiple of 128);
-    `own_len` > 0 replaces the workers' own length (block + markers), for edge cases."""
+    `own_len` > 0 replaces the workers' own length (block + markers), `own_lens` gives every worker
+    its own, for edge cases."""
     assert block_len % 128 == 0 and num_workers >= 1
     rng = np.random.Generator(np.random.PCG64(seed))
-    own = _mk(f"prefix{num_workers}x{block_len}", hq, hkv, d, [own_len or block_len + marker_tokens] * num_workers,
-              steps, seed, rng, permute_pages=permute_pages)
+    lens = list(own_lens) if own_lens is not None else [own_len or block_len + marker_tokens] * num_workers
+    assert len(lens) == num_workers
+    own = _mk(f"prefix{num_workers}x{block_len}", hq, hkv, d, lens, steps, seed, rng, permute_pages=permute_pages)
     pre = np.arange(num_workers, dtype=np.int32) * np.int32(block_len)
     return PrefixWorkload(own=own, block_len=block_len, marker_tokens=marker_tokens, prefix_lens=pre)
 

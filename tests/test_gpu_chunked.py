@@ -139,6 +139,98 @@ def test_long_block_beside_short_ones_sampled_rows():
     run_chunked_event(w, 2048, rows=np.asarray(rows, dtype=np.int64), what="16k + 4 x 2k", r=3)
 
 
+def run_prefix_chunked_event(w, chunk, r=1, decode_sms=0, what=""):
+    """The prefix-aware layout with chunked prefill (Section 4.2: prefix caching and chunked prefill both on):
+    the history is cached first through a plan of its own; worker b then runs its own tokens chunk by chunk
+    over history prefix + earlier chunks, and decodes over prefix + own tokens + its summary so far."""
+    import torch
+    from paper_2605_23296_b200 import binding as B
+    from paper_2605_23296_b200.session import CompactionSession
+    w.materialise()
+    o = w.own
+    T, Bn, P = o.decode_steps, o.num_blocks, o.page_size
+    shape = (w.num_pages, o.num_kv_heads, P, o.head_dim)
+    pools = (torch.full(shape, float("nan"), dtype=torch.bfloat16, device="cuda:0"),
+             torch.full(shape, float("nan"), dtype=torch.bfloat16, device="cuda:0"))
+    hist = CompactionSession([w.hist_tokens], 0, o.num_q_heads, o.num_kv_heads, o.head_dim, w.shared_pages,
+                             w.num_pages, scale=o.scale, pools=pools)
+    hist.append_prefill(_dev(w.k_hist), _dev(w.v_hist))
+    s = CompactionSession(o.block_lens, T, o.num_q_heads, o.num_kv_heads, o.head_dim, o.free_pages, w.num_pages,
+                          scale=o.scale, prefix_lens=w.prefix_lens, shared_pages=w.shared_pages, pools=pools,
+                          chunk_tokens=chunk, decode_sms=decode_sms, decode_steps_per_chunk=r)
+    sched = op.mixed_schedule(o.block_lens.tolist(), chunk, T, r)    # the schedule does not depend on the prefix
+    assert s.param(B.PARAM_NUM_STEPS) == len(sched)
+    start = s.export(B.ARR_DEC_START)
+    q, k, v = _dev(o.q), _dev(o.k), _dev(o.v)
+    out_pre = torch.full_like(q, 7.0)
+    qd, kd, vd = _dev(o.q_dec), _dev(o.k_dec), _dev(o.v_dec)
+    dec_out = {}
+    cu = np.concatenate([[0], np.cumsum(o.block_lens.astype(np.int64))])
+    for step, st in enumerate(sched):
+        act = st["decode"]
+        q_in = torch.zeros((Bn, o.num_q_heads, o.head_dim), dtype=torch.bfloat16, device="cuda:0")
+        k_in = torch.zeros((Bn, o.num_kv_heads, o.head_dim), dtype=torch.bfloat16, device="cuda:0")
+        v_in = torch.zeros_like(k_in)
+        for b in act:
+            t = step - int(start[b])
+            q_in[b], k_in[b], v_in[b] = qd[t, b], kd[t, b], vd[t, b]
+        out = torch.full_like(q_in, 5.0)
+        s.step_mixed(step, q, k, v, out_pre, q_in, k_in, v_in, out)
+        got = _bits(out)
+        for b in range(Bn):
+            if b in act:
+                dec_out[(step, b)] = got[b]
+            else:
+                assert (out[b] == 5.0).all(), f"{what}: step {step} wrote the output row of idle worker {b}"
+    assert s.status() == 0
+    # ---- prefill rows: those of the unchunked prefix-aware prefill; one chunk also by its own definition
+    got_pre = _bits(out_pre)
+    assert_attention_close(got_pre, oa.prefill_prefix_aware(o.q, o.k, o.v, cu, w.k_hist, w.v_hist, w.prefix_lens, o.scale),
+                           f"{what} chunked prefix-aware prefill")
+    wk = Bn - 1
+    first = (int(o.block_lens[wk]) - 1) // chunk * chunk        # the worker's last chunk
+    n = int(o.block_lens[wk]) - first
+    want = oa.prefill_chunk_prefix_aware(o.q, o.k, o.v, cu, w.k_hist, w.v_hist, w.prefix_lens, o.scale, wk, first, n)
+    assert_attention_close(got_pre[cu[wk] + first: cu[wk] + first + n], want, f"{what} last chunk of worker {wk}")
+    # ---- decode over shared prefix pages + own pages
+    state = oa.PrefixDecodeState(o.k, o.v, cu, w.k_hist, w.v_hist, w.prefix_lens, T)
+    for t in range(T):
+        state.append(o.k_dec[t], o.v_dec[t])
+        want = state.decode(o.q_dec[t], o.scale)
+        for b in range(Bn):
+            assert_attention_close(dec_out[(int(start[b]) + t, b)], want[b], f"{what} worker {b} token {t}")
+    # ---- pools: own tokens and summary tokens behind the prefix, the history untouched, bit for bit
+    ref = op.build_plan(o.block_lens.tolist(), T, P, o.free_pages.tolist(), o.num_kv_heads, 128, 1,
+                        prefix_lens=w.prefix_lens.tolist(), shared_pages=w.shared_pages.tolist(), shared_chunk_pages=16)
+    assert np.array_equal(s.export(B.ARR_PAGE_INDICES), np.asarray(ref["page_indices"], dtype=np.int32))
+    kp, vp = pool_rows(_bits(s.k_pool)), pool_rows(_bits(s.v_pool))
+    for i, slot in enumerate(ref["slot_mapping"]):
+        assert np.array_equal(kp[slot // P, :, slot % P], o.k[i]) and np.array_equal(vp[slot // P, :, slot % P], o.v[i])
+    for t in range(T):
+        for b in range(Bn):
+            slot = op.slot_of(ref, P, b, int(w.prefix_lens[b]) + int(o.block_lens[b]) + t)
+            assert np.array_equal(kp[slot // P, :, slot % P], o.k_dec[t][b])
+            assert np.array_equal(vp[slot // P, :, slot % P], o.v_dec[t][b])
+    for t in range(w.hist_tokens):
+        page = int(w.shared_pages[t // P])
+        assert np.array_equal(kp[page, :, t % P], w.k_hist[t]) and np.array_equal(vp[page, :, t % P], w.v_hist[t])
+    assert np.array_equal(s.export(B.ARR_SEQ_LENS), w.prefix_lens + o.block_lens + T)
+    s.close()
+    hist.close()
+
+
+@pytest.mark.parametrize("hq,hkv,d", [(8, 2, 128), (4, 1, 64)])
+def test_prefix_aware_workers_in_chunks(hq, hkv, d):
+    # four workers over a history of 256-token blocks; own lengths from one tile to three chunks, ragged ends
+    w = wl.prefix_aware(4, 256, hq, hkv, d, steps=4, seed=90 + d, own_lens=[272, 700, 129, 50])
+    run_prefix_chunked_event(w, 256, r=2, what=f"prefix + chunks {hq}/{hkv}/{d}")
+
+
+def test_prefix_aware_chunks_of_one_tile_with_one_decode_sm():
+    w = wl.prefix_aware(3, 384, 8, 8, 128, steps=3, seed=93, own_lens=[400, 130, 385])
+    run_prefix_chunked_event(w, 128, r=1, decode_sms=1, what="prefix + 128-token chunks")
+
+
 def test_mixed_step_needs_a_chunked_plan():
     from paper_2605_23296_b200 import binding as B
     from paper_2605_23296_b200.session import CompactionSession

@@ -300,6 +300,45 @@ def test_chunked_plan_steps_bit_exact(lens, C, T, r):
         B.cpa_plan_destroy(plan)
 
 
+def test_prefix_chunked_plan_is_the_prefix_plan_with_the_chunk_schedule():
+    # Section 4.2 runs prefix caching and chunked prefill together: pages, slots, lengths and the two-level
+    # decode cut are the prefix plan's, the steps are those of the chunk schedule over the own lengths
+    cfg = B.cpa_config(8, 2, 128, 16, 0.088, 0, 0, 0)
+    own, pre, T, C, r = [272, 700, 129, 50], [0, 256, 512, 768], 3, 256, 2
+    shared = np.arange(100, 100 + 48, dtype=np.int32)
+    free = np.arange(sum(-(-(L + T) // 16) for L in own), dtype=np.int32)
+    plan = B.cpa_plan_create_prefix_chunked(cfg, own, pre, shared, T, C, free, decode_steps_per_chunk=r)
+    try:
+        ref = op.mixed_schedule(own, C, T, r)
+        assert B.cpa_plan_param(plan, B.PARAM_NUM_STEPS) == len(ref)
+        n_chunks = B.cpa_plan_param(plan, B.PARAM_CHUNK_STEPS)
+        rows = B.cpa_plan_export(plan, B.ARR_CHUNK_ROWS).reshape(n_chunks, len(own) + 1)
+        for c in range(n_chunks):
+            want = [0] * len(own)
+            for b, first, n in ref[c * r]["prefill"]:
+                want[b] = n
+            assert np.diff(rows[c]).tolist() == want
+        assert B.cpa_plan_export(plan, B.ARR_DEC_START).tolist() == [-(-L // C) * r for L in own]
+        cfgq = B.cpa_config(8, 2, 128, 16, 0.088, B.cpa_plan_param(plan, B.PARAM_Q_TILE_ROWS), 0, 0)
+        plain = B.cpa_plan_create_prefix(cfgq, own, pre, shared, T, free)
+        for which in (B.ARR_CU_SEQLENS, B.ARR_PAGE_INDPTR, B.ARR_PAGE_INDICES, B.ARR_SLOT_MAPPING, B.ARR_SEQ_LENS,
+                      B.ARR_PREFILL_ITEMS, B.ARR_SPLIT_INDPTR, B.ARR_DECODE_ITEMS):
+            assert np.array_equal(B.cpa_plan_export(plan, which), B.cpa_plan_export(plain, which)), which
+        assert B.cpa_plan_export(plan, B.ARR_SEQ_LENS).tolist() == pre
+        B.cpa_plan_destroy(plain)
+    finally:
+        B.cpa_plan_destroy(plan)
+    # errors: the union of the two creators'
+    for kw, args in [({}, (own, [0, 200, 512, 768], shared, T, C, free)),           # prefix not whole KV tiles
+                     ({}, (own, pre, shared[:10], T, C, free)),                     # prefix longer than the cache
+                     ({}, (own, pre, shared, T, 200, free)),                        # chunk not a multiple of 128
+                     ({"decode_steps_per_chunk": 0}, (own, pre, shared, T, C, free))]:
+        rc, h = B.cpa_plan_create_prefix_chunked(cfg, *args, check=False, **kw)
+        assert rc == B.CPA_EINVAL and not h
+    rc, h = B.cpa_plan_create_prefix_chunked(cfg, own, pre, shared, T, C, free[:5], check=False)
+    assert rc == B.CPA_ENOSPC and not h
+
+
 def test_chunked_plan_errors():
     cfg = B.cpa_config(8, 2, 64, 16, 0.125, 0, 0, 0)
     free = np.arange(100, dtype=np.int32)
