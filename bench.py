@@ -361,24 +361,21 @@ def measure_event(w, args, dev, steps: int, warmup: int, with_e2e: bool, world: 
         h_q, h_k, h_v, h_qd, h_kd, h_vd = hosts
         h_o = torch.empty(d_o.shape, dtype=torch.bfloat16).pin_memory()
         h_od = torch.empty(d_od.shape, dtype=torch.bfloat16).pin_memory()
-        side = torch.cuda.Stream(dev)
         h2d = sum(t.numel() * 2 for t in hosts)
         d2h = (h_o.numel() + h_od.numel()) * 2
+        stage = None
         for i in range(1 + steps):
             flush.fill_(1)
             e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             torch.cuda.synchronize(dev)
             e0.record(stream)
-            q, k, v = (t.to(dev, non_blocking=True) for t in (h_q, h_k, h_v))
-            qd, kd, vd = (t.to(dev, non_blocking=True) for t in (h_qd, h_kd, h_vd))
-            ev_pre = {n: torch.cuda.Event() for n in ("planned", "prefilled", "appended")}
-            s = one_pass(q, k, v, qd, kd, vd, d_o, d_od, ev_pre)
-            # the prefill output goes home on a side stream while the decode steps run
-            side.wait_event(ev_pre["prefilled"])
-            with torch.cuda.stream(side):
-                h_o.copy_(d_o, non_blocking=True)
-            h_od.copy_(d_od, non_blocking=True)
-            stream.wait_stream(side)
+            # one C-ABI call with host pointers: plan (chunked, so that the copies overlap the kernels), prompts up
+            # chunk by chunk, prefill per chunk, outputs home behind the kernels, then the T decode steps
+            s = CompactionSession(w.block_lens, T, w.num_q_heads, w.num_kv_heads, w.head_dim,
+                                  w.free_pages, w.num_pages, scale=w.scale, device=str(dev),
+                                  pages_per_split=args.pages_per_split, chunk_tokens=args.e2e_chunk,
+                                  decode_sms=1 if args.e2e_chunk else 0)
+            stage = s.event_from_host(h_q, h_k, h_v, h_o, h_qd, h_kd, h_vd, h_od, stage=stage)
             e1.record(stream)
             torch.cuda.synchronize(dev)
             assert s.status() == 0
@@ -511,7 +508,8 @@ def run_gpu(args) -> None:
         "cpu_baseline": {"value": Bn * T / cpu["estimated_step_s"], "unit": UNIT, "cores": cpu["cores"],
                          "kind": "oracle", "sample": cpu["sample"], "measured_s": cpu["measured_s"]},
         "e2e": {"value": tokens / (m["e2e_ms"] * 1e-3), "unit": UNIT, "ms_per_step": m["e2e_ms"],
-                "h2d_bytes_per_step": m["h2d"], "d2h_bytes_per_step": m["d2h"]},
+                "h2d_bytes_per_step": m["h2d"], "d2h_bytes_per_step": m["d2h"],
+                "call": "cpa_event_host", "chunk_tokens": args.e2e_chunk},
         "gpu_launches": m["launches"],
         "clocks": m["clocks"],
     }
@@ -955,6 +953,8 @@ def main() -> None:
     ap.add_argument("--separate-append", action="store_true",
                     help="per decode step call cpa_kv_append and cpa_decode instead of the fused cpa_decode_append")
     ap.add_argument("--skip-e2e", action="store_true", help="skip the host-buffer leg (profiling)")
+    ap.add_argument("--e2e-chunk", type=int, default=4096,
+                    help="tokens per prefill chunk of the host-buffer leg (copies overlap the kernels); 0 = whole blocks, no overlap")
     ap.add_argument("--skip-cpu", action="store_true", help="skip the CPU oracle leg (profiling)")
     args = ap.parse_args()
     args.overrides = {"num_blocks": args.blocks, "block_len": args.block_len, "steps": args.decode_steps}

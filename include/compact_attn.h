@@ -136,7 +136,8 @@ enum {
     CPA_PARAM_NUM_SMS = 15,              /* the plan's SM budget (cfg.num_sms, or the device's SM count for 0) */
     CPA_PARAM_DECODE_STEPS_PER_CHUNK = 16, /* decode steps a chunked plan's schedule gives a chunk */
     CPA_PARAM_DECODE_EVEN_CUT = 17,      /* 1: the decode splits come from the even cut (see cpa_plan_create), 0: uniform per block */
-    CPA_PARAM_DECODE_CTAS = 18           /* CTAs of a decode launch */
+    CPA_PARAM_DECODE_CTAS = 18,          /* CTAs of a decode launch */
+    CPA_PARAM_HOST_STAGE_BYTES = 19      /* size of cpa_event_host's device staging buffer */
 };
 
 /*
@@ -447,6 +448,34 @@ CPA_API int cpa_release_blocks(cpa_plan* plan, const int32_t* d_active, void* st
 CPA_API int cpa_step_mixed(cpa_plan* plan, int32_t step, const void* q, const void* k, const void* v, void* o,
                            const void* q_dec, const void* k_new, const void* v_new, void* o_dec, void* k_pool,
                            void* v_pool, void* d_workspace, void* stream);
+
+/*
+ * cpa_event_host -- a whole compaction event with inputs and outputs in HOST memory: the prefill of every
+ * block (Section 4, "Dispatch": each worker runs its prompt), the append of the prompts' K/V, and
+ * max_new_tokens decode steps over all blocks, each with its append (the workers' summaries, Section 4).  The
+ * paper has no counterpart for the copy order; it is this library's way of hiding the PCIe transfers.
+ *   h_q, h_o            : host bf16 [total_tokens, num_q_heads, head_dim]  (h_o is written)
+ *   h_k, h_v            : host bf16 [total_tokens, num_kv_heads, head_dim]
+ *   h_q_dec, h_o_dec    : host bf16 [max_new_tokens, B, num_q_heads, head_dim]  (step t's row of every block;
+ *                         h_o_dec is written); h_k_dec, h_v_dec likewise with num_kv_heads.  May be NULL when
+ *                         max_new_tokens == 0.
+ *   d_stage             : device scratch, >= CPA_PARAM_HOST_STAGE_BYTES, 256-byte aligned; holds the device
+ *                         copies of all eight arrays (the caller may read them there after the call)
+ *   k_pool, v_pool, d_workspace : as for cpa_decode_append
+ * Host buffers should be page-locked (cudaHostAlloc / cudaHostRegister): with pageable memory the copies
+ * are still correct but do not overlap the kernels.  On a chunked plan (cpa_plan_create_chunked or
+ * cpa_plan_create_prefix_chunked; decode_sms = 1 leaves the chunks all SMs but one) the prompts go up chunk by
+ * chunk on a copy stream of the plan, chunk c of all blocks is prefilled in one launch as soon as its rows
+ * have landed, and the output rows go home on another stream once the last input is up (behind the remaining
+ * chunks and the decode steps); the decode steps then run for all blocks together (not the schedule of cpa_step_mixed, which this call uses up).
+ * On any other plan the same steps run without overlap.  Everything is enqueued; the results are in place
+ * when `stream` has been synchronised, and cpa_plan_status tells whether a kernel gave up.
+ * Errors: CPA_EINVAL (null or misaligned pointer), CPA_ESTATE (plan not uploaded, or something was
+ * already appended or stepped since the upload), CPA_EUNSUPPORTED (a plan with pages on demand), CPA_ECUDA.
+ */
+CPA_API int cpa_event_host(cpa_plan* plan, const void* h_q, const void* h_k, const void* h_v, void* h_o,
+                           const void* h_q_dec, const void* h_k_dec, const void* h_v_dec, void* h_o_dec,
+                           void* d_stage, void* k_pool, void* v_pool, void* d_workspace, void* stream);
 
 /*
  * cpa_decode_static -- cpa_decode for callers that cannot hand over scratch memory.

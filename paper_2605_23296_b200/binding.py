@@ -35,7 +35,7 @@ PARAM_PREFILL_CTAS = 9
 PARAM_SHARED_CHUNK_PAGES = 10
 PARAM_CHUNK_TOKENS, PARAM_NUM_STEPS, PARAM_CHUNK_STEPS, PARAM_DECODE_SMS, PARAM_NUM_SMS = 11, 12, 13, 14, 15
 PARAM_DECODE_STEPS_PER_CHUNK = 16
-PARAM_DECODE_EVEN_CUT, PARAM_DECODE_CTAS = 17, 18
+PARAM_DECODE_EVEN_CUT, PARAM_DECODE_CTAS, PARAM_HOST_STAGE_BYTES = 17, 18, 19
 
 
 class cpa_config(ctypes.Structure):
@@ -82,6 +82,8 @@ _lib.cpa_release_blocks.argtypes = [_vp, _vp, _vp]
 _lib.cpa_release_blocks.restype = ctypes.c_int
 _lib.cpa_step_mixed.argtypes = [_vp, ctypes.c_int32] + [_vp] * 12
 _lib.cpa_step_mixed.restype = ctypes.c_int
+_lib.cpa_event_host.argtypes = [_vp] * 14
+_lib.cpa_event_host.restype = ctypes.c_int
 _lib.cpa_plan_export.argtypes = [_vp, ctypes.c_int, ctypes.POINTER(_i32p), ctypes.POINTER(ctypes.c_int64)]
 _lib.cpa_plan_export.restype = ctypes.c_int
 _lib.cpa_plan_param.argtypes = [_vp, ctypes.c_int]
@@ -290,6 +292,14 @@ def cpa_step_mixed(plan: int, step: int, q, k, v, o, q_dec, k_new, v_new, o_dec,
                    stream: int = 0) -> int:
     return _lib.cpa_step_mixed(plan, int(step), _ptr(q), _ptr(k), _ptr(v), _ptr(o), _ptr(q_dec), _ptr(k_new),
                                _ptr(v_new), _ptr(o_dec), _ptr(k_pool), _ptr(v_pool), _ptr(d_workspace), stream or None)
+
+
+def cpa_event_host(plan: int, h_q, h_k, h_v, h_o, h_q_dec, h_k_dec, h_v_dec, h_o_dec, d_stage, k_pool, v_pool,
+                   d_workspace, stream: int = 0) -> int:
+    """A whole event from host tensors (page-locked for overlap); the results are in place after a stream sync."""
+    return _lib.cpa_event_host(plan, _ptr(h_q), _ptr(h_k), _ptr(h_v), _ptr(h_o), _ptr(h_q_dec), _ptr(h_k_dec),
+                               _ptr(h_v_dec), _ptr(h_o_dec), _ptr(d_stage), _ptr(k_pool), _ptr(v_pool),
+                               _ptr(d_workspace), stream or None)
 
 
 STATIC_SCRATCH_BYTES = 16 << 20

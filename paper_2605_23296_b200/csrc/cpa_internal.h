@@ -94,6 +94,10 @@ struct cpa_plan {
     // at the first mixed step on the device that is current then, destroyed with the plan
     cudaStream_t side_stream = nullptr;
     cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
+    // an event from host memory copies in and out on two streams of its own, ordered by events; made at the
+    // first such event on the device that is current then, destroyed with the plan
+    cudaStream_t in_stream = nullptr, out_stream = nullptr;
+    std::vector<cudaEvent_t> host_events;
 
     // packed image of the device index buffer (int32 words) and offsets into it
     std::vector<int32_t> image;
@@ -180,6 +184,8 @@ int cpa_prefill_pair_capacity();
 int cpa_prefill_tc_list(const cpa_plan* plan, const void* q, const void* k, const void* v, void* o, const void* k_pool,
                         const void* v_pool, const int32_t* items, const int32_t* sched, int ctas, int rounds, void* stream);
 // Chunk c's append: rows [c * chunk, ...) of every block that has them go to the block's pages.
+// device staging an event from host memory needs: q, k, v, o, then the decode steps' q, k, v, o (256-byte aligned each)
+int64_t cpa_host_stage_bytes(const cpa_plan* plan);
 int cpa_append_chunk(cpa_plan* plan, int chunk, const void* k, const void* v, void* k_pool, void* v_pool, void* stream);
 // One decode launch (append fused in when k_new is given) over the blocks `mode` selects.
 int cpa_decode_launch(const cpa_plan* plan, const void* q, const void* k_new, const void* v_new, void* k_pool,

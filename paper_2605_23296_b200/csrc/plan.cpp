@@ -712,6 +712,7 @@ extern "C" int64_t cpa_plan_param(const cpa_plan* plan, int which) {
         case CPA_PARAM_DECODE_STEPS_PER_CHUNK: return plan->steps_per_chunk;
         case CPA_PARAM_DECODE_EVEN_CUT: return plan->even_cut ? 1 : 0;
         case CPA_PARAM_DECODE_CTAS: return plan->decode_grid;
+        case CPA_PARAM_HOST_STAGE_BYTES: return cpa_host_stage_bytes(plan);
         default: return CPA_EINVAL;
     }
 }
@@ -754,6 +755,9 @@ extern "C" void cpa_plan_destroy(cpa_plan* plan) {
     if (plan->ev_fork) cudaEventDestroy(plan->ev_fork);
     if (plan->ev_join) cudaEventDestroy(plan->ev_join);
     if (plan->side_stream) cudaStreamDestroy(plan->side_stream);
+    for (cudaEvent_t e : plan->host_events) cudaEventDestroy(e);
+    if (plan->in_stream) cudaStreamDestroy(plan->in_stream);
+    if (plan->out_stream) cudaStreamDestroy(plan->out_stream);
     (void)cudaGetLastError();
     delete plan;
 }

@@ -150,6 +150,20 @@ class CompactionSession:
         self._check(B.cpa_step_mixed(self.plan, step, q, k, v, out, q_dec, k_new, v_new, out_dec, self.k_pool,
                                      self.v_pool, self.workspace, self._stream()), "cpa_step_mixed")
 
+    def event_from_host(self, h_q, h_k, h_v, h_out, h_q_dec=None, h_k_dec=None, h_v_dec=None, h_out_dec=None,
+                        stage: Optional[torch.Tensor] = None) -> torch.Tensor:
+        """The whole event from host tensors (page-locked ones overlap with the kernels): prompts [tokens,H,d],
+        decode steps' inputs [T,B,H,d]; h_out / h_out_dec are written.  Everything is enqueued on the current
+        stream; synchronise it before reading the outputs.  Returns the device staging buffer (uint8,
+        PARAM_HOST_STAGE_BYTES), which a later event of the same shape may be given again."""
+        need = self.param(B.PARAM_HOST_STAGE_BYTES)
+        if stage is None:
+            stage = torch.empty(max(need, 256), dtype=torch.uint8, device=self.device)
+        assert stage.numel() >= need and stage.device == self.device
+        self._check(B.cpa_event_host(self.plan, h_q, h_k, h_v, h_out, h_q_dec, h_k_dec, h_v_dec, h_out_dec, stage,
+                                     self.k_pool, self.v_pool, self.workspace, self._stream()), "cpa_event_host")
+        return stage
+
     def decode_append_dynamic(self, q, k_new, v_new, active=None, out=None):
         """One decode step of a plan with pages on demand; `active` is a device int32 [B] tensor of stop flags."""
         if out is None:

@@ -339,6 +339,25 @@ def test_prefix_chunked_plan_is_the_prefix_plan_with_the_chunk_schedule():
     assert rc == B.CPA_ENOSPC and not h
 
 
+def test_event_from_host_argument_checks_and_stage_size():
+    cfg = B.cpa_config(8, 2, 128, 16, 0.088, 0, 0, 0)
+    lens, T = (300, 50), 3
+    plan = B.cpa_plan_create_chunked(cfg, lens, T, 128, np.arange(100, dtype=np.int32))
+    tokens, rows = sum(lens), T * len(lens)
+    a = lambda n: -(-n // 256) * 256
+    want = 2 * a(tokens * 8 * 128 * 2) + 2 * a(tokens * 2 * 128 * 2) + 2 * a(rows * 8 * 128 * 2) + 2 * a(rows * 2 * 128 * 2)
+    assert B.cpa_plan_param(plan, B.PARAM_HOST_STAGE_BYTES) == want
+    f = 4096
+    assert B.cpa_event_host(plan, f, f, f, f, f, f, f, f, f, f, f, f) == B.CPA_ESTATE          # not uploaded
+    assert B.cpa_event_host(plan, None, f, f, f, f, f, f, f, f, f, f, f) == B.CPA_EINVAL
+    assert B.cpa_event_host(plan, f, f, f, f, None, f, f, f, f, f, f, f) == B.CPA_EINVAL       # T > 0 needs decode inputs
+    assert B.cpa_event_host(plan, f, f, f, f, f, f, f, f, f + 16, f, f, f) == B.CPA_EINVAL     # stage not 256-aligned
+    B.cpa_plan_destroy(plan)
+    dyn = B.cpa_plan_create_dynamic(cfg, lens, T, np.arange(100, dtype=np.int32))
+    assert B.cpa_plan_param(dyn, B.PARAM_HOST_STAGE_BYTES) == want
+    B.cpa_plan_destroy(dyn)
+
+
 def test_chunked_plan_errors():
     cfg = B.cpa_config(8, 2, 64, 16, 0.125, 0, 0, 0)
     free = np.arange(100, dtype=np.int32)
