@@ -108,7 +108,9 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
     const uint32_t s_k = s_q + 2 * kTileBytes;       // KS stages
     const uint32_t s_v = s_k + KS * kTileBytes;      // KS stages
 
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    // (the broadcast tells the compiler that the warp index, and every role, address and counter that follows from
+    // it, is the same in all lanes, so that it can keep them out of the per-thread registers)
+    const int warp = __shfl_sync(0xffffffffu, (int)(threadIdx.x >> 5), 0), lane = threadIdx.x & 31;
     const int G = gridDim.x;
     const int group = Hq / Hkv;
     // Unit of round k for this CTA, from the planner's schedule.  Every role keeps the schedule entry of
@@ -125,6 +127,8 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
             r.a = __ldg(reinterpret_cast<const int4*>(ix.prefill_items) + it);
         }
     };
+    // a value that is the same in all lanes of a warp by construction; said so to the compiler (see `warp`)
+    auto uniform = [&](int x) { return __shfl_sync(0xffffffffu, x, 0); };
     auto decode = [&](const Rec& r, TcWork& w) {
         w.valid = r.a.y > 0;
         w.h = r.h;
@@ -472,9 +476,10 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
         fetch(fetch_code(0), rec);
         int code = fetch_code(1);
         for (int rd = 0; rd < n_rounds; ++rd) {
+        rec.a.x = uniform(rec.a.x); rec.a.y = uniform(rec.a.y); rec.a.z = uniform(rec.a.z); rec.h = uniform(rec.h);
         decode(rec, w);
         fetch(code, rec);
-        code = fetch_code(rd + 2);
+        code = uniform(fetch_code(rd + 2));
         if (!w.valid) continue;
         if (u < w.n_sub) {
         const int n_kv = w.t0 + 1 + u;
@@ -525,13 +530,15 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                 const int kt = kt0 + j - 1;
                 tc_wait(bar(&bars.v_empty[kt % KS]), (uint32_t)(kt / KS) & 1u, dead, ix.status);
                 tc_fence_after();
+                // (rare, and the tile's scores are live in registers meanwhile: eight columns at a time, so that this
+                // path does not make the compiler spill in the loop around it)
+#pragma unroll 1
+                for (int c = 0; c < D / 8; ++c) {
+                    float v[8];
+                    tc_ld8(t_o + c * 8, v);
 #pragma unroll
-                for (int c = 0; c < D / 32; ++c) {
-                    float v[32];
-                    tc_ld32(t_o + c * 32, v);
-#pragma unroll
-                    for (int i = 0; i < 32; ++i) v[i] *= alpha;
-                    tc_st32(t_o + c * 32, v);
+                    for (int i = 0; i < 8; ++i) v[i] *= alpha;
+                    tc_st8(t_o + c * 8, v);
                 }
             }
             l_run *= alpha;
