@@ -431,11 +431,13 @@ CPA_API int cpa_release_blocks(cpa_plan* plan, const int32_t* d_active, void* st
  * plan owns (created at the first chunk; no device memory is allocated), decode launches on `stream`.
  * `stream` waits for the chunks started so far when a block decodes its first token, and at the last
  * step of the schedule: the prefill rows of a chunk are complete on `stream` from the step in which one
- * of its blocks starts to decode, and all of them after the last step.  A chunk is ordered behind what
- * `stream` held when its step was called (its rows may just have been copied in there).
+ * of its blocks starts to decode, and all of them after the last step.  The first chunk is ordered behind
+ * what `stream` held when step 0 was called, every later chunk behind the chunk before it and nothing else
+ * (so the chunks run back to back whatever the decode steps between them take): the inputs of all chunks
+ * must be complete on `stream` when step 0 is called, and must be the same buffers in every step.
  *   q, k, v, o : the packed tensors of the whole event ([total_tokens, heads, head_dim]); a chunk reads
  *                and writes only its rows, rows cu_seqlens[b] + [c * C, ...) of every block that has a
- *                chunk c, so later rows need not exist yet.  Row i of a chunk attends over the block's
+ *                chunk c.  Row i of a chunk attends over the block's
  *                cached tokens [0, c * C) and the chunk's tokens up to itself: exactly the rows
  *                cpa_prefill gives.  May be NULL in steps that start no chunk.
  *   q_dec, o_dec       : device bf16 [B, num_q_heads, head_dim]; only the rows of the decoding blocks are

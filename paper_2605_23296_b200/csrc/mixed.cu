@@ -3,8 +3,9 @@
 // prefill it chunk by chunk, and the blocks that are past their prompt decode meanwhile.  The two touch
 // different blocks, so they run side by side: the chunks one after the other on a second stream the plan owns,
 // each on most SMs; the decode launches on the caller's stream, on the SMs the plan keeps free for them.  A
-// chunk is given the time of `steps_per_chunk` decode steps; the caller's stream waits for the chunks only when
-// a block goes from its last chunk to its first decode step, and at the end of the schedule.
+// chunk is given the time of `steps_per_chunk` decode steps by the schedule (which fixes when a block may start
+// to decode), but the chunks themselves run back to back; the caller's stream waits for them only when a block
+// goes from its last chunk to its first decode step, and at the end of the schedule.
 #include <cuda_runtime.h>
 
 #include <algorithm>
@@ -65,9 +66,11 @@ extern "C" int cpa_step_mixed(cpa_plan* plan, int32_t step, const void* q, const
     int rc = CPA_OK;
     if (starts_chunk) {
         if ((rc = ensure_side_stream(plan)) != CPA_OK) return rc;
-        // the chunk follows whatever the caller has enqueued on `stream` so far (its rows may just have been copied in)
-        if (cudaEventRecord(plan->ev_fork, main_st) != cudaSuccess ||
-            cudaStreamWaitEvent(plan->side_stream, plan->ev_fork, 0) != cudaSuccess) {
+        // The first chunk follows whatever the caller has enqueued on `stream` so far (the inputs of all chunks);
+        // later chunks follow only the chunk before them, so that they run back to back instead of at the pace
+        // of the decode steps in between.
+        if (chunk == 0 && (cudaEventRecord(plan->ev_fork, main_st) != cudaSuccess ||
+                           cudaStreamWaitEvent(plan->side_stream, plan->ev_fork, 0) != cudaSuccess)) {
             (void)cudaGetLastError();
             return CPA_ECUDA;
         }
