@@ -126,7 +126,7 @@ extern "C" int cpa_event_host(cpa_plan* plan, const void* h_q, const void* h_k, 
     // and the inputs are on the critical path while the outputs have the decode steps to hide behind
     CPA_CK(cudaStreamWaitEvent(out_st, ev_dec_in, 0));
 
-    // ---- prefill and append per chunk; the chunk's output rows go home behind it
+    // ---- prefill and append per chunk; the chunk's output rows are queued for the way home (behind the inputs)
     bool any_prefix = false;
     for (int b = 0; b < B; ++b) any_prefix |= plan->prefix_lens[b] > 0;
     for (int c = 0; c < n_chunks; ++c) {
