@@ -45,11 +45,11 @@ PER_CONFIG = [("dense8b", {}, 40), ("moe120b", {}, 8), ("split", {"num_blocks": 
 # proportion to its KV bytes, so the ratios carry over to the average step of the full run.  A workload without
 # a capture has no entry.
 DECODE_CAPTURES = {
-    "ragged": {"warm_ratio": 0.9318, "cold_ratio": 1.0044, "cold_gbs": 6072.7,
+    "ragged": {"warm_ratio": 0.9319, "cold_ratio": 1.0043, "cold_gbs": 6043.7,
                "source": "profiles/decode_split_kernel_ragged.md"},
-    "dense8b": {"warm_ratio": 0.3703, "cold_ratio": 1.0077, "cold_gbs": 4067.3,
+    "dense8b": {"warm_ratio": 0.3681, "cold_ratio": 1.0071, "cold_gbs": 4072.7,
                 "source": "profiles/decode_split_kernel_dense8b.md"},
-    "moe120b": {"warm_ratio": 0.7620, "cold_ratio": 1.0050, "cold_gbs": 5016.0,
+    "moe120b": {"warm_ratio": 0.7621, "cold_ratio": 1.0049, "cold_gbs": 4967.1,
                 "source": "profiles/decode_split_kernel_moe120b.md"},
 }
 
