@@ -407,9 +407,13 @@ def phase_numbers(w, m: dict, peaks: dict, separate_append: bool) -> dict:
         # add their own cost and break the overlap of consecutive launches
         launch_us, launch_bytes = m["decode_ms"] * 1e3 / T, total_kv / T
     gbs = launch_bytes / (launch_us * 1e-6) / 1e9
+    # the prefill's second limiter: one exponential per unmasked score, Hq * L(L+1)/2 per block = flops / (4 d);
+    # the special-function units make 16 per clock and SM (nominal: 148 SMs at the maximum clock)
+    gexp = prefill_flops(w) / (4.0 * w.head_dim) / (m["prefill_ms"] * 1e-3) / 1e9
     return {"prefill_ms": m["prefill_ms"], "prefill_tflops": pf_tflops,
             "prefill_frac_of_bf16_peak": pf_tflops / peaks["bf16_tflops"],
             "prefill_frac_of_nominal_2250": pf_tflops / NOMINAL_BF16_TFLOPS,
+            "prefill_gexp_per_s": gexp, "prefill_frac_of_nominal_exp_rate": gexp / (16 * 148 * 1.965),
             "decode_ms": m["decode_ms"], "decode_launch_us": launch_us, "decode_bytes_per_launch": launch_bytes,
             "decode_gbs": gbs, "decode_frac_of_hbm_peak": gbs / peaks["hbm_gbs"],
             "decode_frac_of_nominal_8TBs": gbs / NOMINAL_HBM_GBS,
