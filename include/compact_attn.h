@@ -174,6 +174,18 @@ CPA_API int cpa_plan_create(const cpa_config* cfg, int32_t num_blocks, const int
                     cpa_plan** out);
 
 /*
+ * cpa_partition -- "Snapshot & partition" (Section 4): a history of |X| tokens is cut into N = ceil(|X| / B)
+ * contiguous blocks of B tokens, the last one possibly shorter (Section 5, "Threshold and block size
+ * interaction": 96k tokens at 16k per block are 6 workers, at 4k per block 24).  Writes the N block lengths
+ * to the host array `block_lens` (capacity `capacity` entries) and N to `num_blocks`; the lengths are what
+ * cpa_plan_create takes, and i * B what cpa_plan_create_prefix takes as worker i's prefix.  Host arithmetic
+ * only.  Errors: CPA_EINVAL (a length below 1, a null pointer), CPA_ENOSPC (more than `capacity` blocks;
+ * `num_blocks` still says how many), CPA_EUNSUPPORTED (more than 2^31 - 1 blocks).
+ */
+CPA_API int cpa_partition(int64_t history_tokens, int32_t block_tokens, int32_t* block_lens, int32_t capacity,
+                          int32_t* num_blocks);
+
+/*
  * cpa_plan_create_prefix -- the plan for the paper's own layout (Section 4, "Dispatch" and
  * "Prefix-aware target-at-end layout"): the prompt of worker w is blocks 1..w-1 of the history
  * followed by block w wrapped in its markers, every worker's prefix extends the previous worker's,

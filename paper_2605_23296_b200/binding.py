@@ -83,6 +83,8 @@ _lib.cpa_release_blocks.restype = ctypes.c_int
 _lib.cpa_step_mixed.argtypes = [_vp, ctypes.c_int32] + [_vp] * 12
 _lib.cpa_step_mixed.restype = ctypes.c_int
 _lib.cpa_event_host.argtypes = [_vp] * 14
+_lib.cpa_partition.argtypes = [ctypes.c_int64, ctypes.c_int32, _i32p, ctypes.c_int32, ctypes.POINTER(ctypes.c_int32)]
+_lib.cpa_partition.restype = ctypes.c_int
 _lib.cpa_event_host.restype = ctypes.c_int
 _lib.cpa_plan_export.argtypes = [_vp, ctypes.c_int, ctypes.POINTER(_i32p), ctypes.POINTER(ctypes.c_int64)]
 _lib.cpa_plan_export.restype = ctypes.c_int
@@ -142,6 +144,19 @@ def cpa_plan_create(cfg: cpa_config, block_lens: Sequence[int], max_new_tokens: 
     if rc != CPA_OK:
         raise CpaError(rc, "cpa_plan_create")
     return out.value
+
+
+def cpa_partition(history_tokens: int, block_tokens: int, capacity: int = 1 << 16, check: bool = True):
+    """Block lengths of a history cut into blocks of `block_tokens` (the last one may be short)."""
+    lens = np.zeros(max(capacity, 1), dtype=np.int32)
+    n = ctypes.c_int32(0)
+    rc = _lib.cpa_partition(int(history_tokens), int(block_tokens), lens.ctypes.data_as(_i32p), int(capacity),
+                            ctypes.byref(n))
+    if not check:
+        return rc, n.value
+    if rc != CPA_OK:
+        raise CpaError(rc, "cpa_partition")
+    return lens[:n.value].copy()
 
 
 def cpa_plan_create_prefix(cfg: cpa_config, own_lens: Sequence[int], prefix_lens: Sequence[int],

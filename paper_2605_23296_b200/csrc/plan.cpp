@@ -587,6 +587,19 @@ int plan_create(const cpa_config* cfg, int32_t num_blocks, const int32_t* block_
 }
 }  // namespace
 
+extern "C" int cpa_partition(int64_t history_tokens, int32_t block_tokens, int32_t* block_lens, int32_t capacity,
+                             int32_t* num_blocks) {
+    if (history_tokens < 1 || block_tokens < 1 || !num_blocks || capacity < 0 || (capacity > 0 && !block_lens))
+        return CPA_EINVAL;
+    const int64_t n = (history_tokens + block_tokens - 1) / block_tokens;
+    if (n > INT32_MAX) return CPA_EUNSUPPORTED;
+    *num_blocks = (int32_t)n;
+    if (n > capacity) return CPA_ENOSPC;
+    for (int64_t i = 0; i + 1 < n; ++i) block_lens[i] = block_tokens;
+    block_lens[n - 1] = (int32_t)(history_tokens - (n - 1) * block_tokens);   // the last block may be short
+    return CPA_OK;
+}
+
 extern "C" int cpa_plan_create(const cpa_config* cfg, int32_t num_blocks, const int32_t* block_lens,
                                int32_t max_new_tokens, const int32_t* free_pages, int32_t num_free,
                                cpa_plan** out) {

@@ -358,6 +358,24 @@ def test_event_from_host_argument_checks_and_stage_size():
     B.cpa_plan_destroy(dyn)
 
 
+def test_partition_is_the_papers_rule():
+    # Section 4 "Snapshot & partition", Section 5 "Threshold and block size interaction": the printed worker counts,
+    # the restated rule on odd sizes, and the creator's error cases
+    import os
+    with open(os.path.join(os.path.dirname(__file__), "golden", "worker_counts.txt")) as f:
+        rows = [tuple(int(x) for x in line.split()) for line in f if line.strip() and not line.startswith("#")]
+    assert rows
+    for tau, blk, workers in rows:
+        lens = B.cpa_partition(tau, blk)
+        assert len(lens) == workers and int(lens.sum()) == tau and (lens[:-1] == blk).all() and 1 <= lens[-1] <= blk
+    for tau, blk in [(1, 1), (1, 4096), (4096, 4096), (4097, 4096), (131072, 2048), (100000, 7777)]:
+        assert B.cpa_partition(tau, blk).tolist() == op.partition(tau, blk)
+    assert B.cpa_partition(0, 16, check=False)[0] == B.CPA_EINVAL
+    assert B.cpa_partition(16, 0, check=False)[0] == B.CPA_EINVAL
+    assert B.cpa_partition(100, 10, capacity=9, check=False) == (B.CPA_ENOSPC, 10)
+    assert B.cpa_partition(1 << 40, 1, capacity=4, check=False)[0] == B.CPA_EUNSUPPORTED
+
+
 def test_chunked_plan_errors():
     cfg = B.cpa_config(8, 2, 64, 16, 0.125, 0, 0, 0)
     free = np.arange(100, dtype=np.int32)
