@@ -28,7 +28,7 @@ def _cu(w):
     return np.concatenate([[0], np.cumsum(w.block_lens.astype(np.int64))])
 
 
-def run_chunked_event(w, chunk, decode_sms=0, rows=None, what="", r=1):
+def run_chunked_event(w, chunk, decode_sms=0, rows=None, what="", r=1, sparse_pool=False):
     """All steps of the schedule through cpa_step_mixed.  Inputs of decode step t of a block are row t of
     w.*_dec (so a block's t-th summary token has the same inputs whatever step it is produced in)."""
     import torch
@@ -37,7 +37,7 @@ def run_chunked_event(w, chunk, decode_sms=0, rows=None, what="", r=1):
     w.materialise()
     T, Bn = w.decode_steps, w.num_blocks
     s = CompactionSession(w.block_lens, T, w.num_q_heads, w.num_kv_heads, w.head_dim, w.free_pages, w.num_pages,
-                          scale=w.scale, poison_pools=True, chunk_tokens=chunk, decode_sms=decode_sms,
+                          scale=w.scale, poison_pools=not sparse_pool, chunk_tokens=chunk, decode_sms=decode_sms,
                           decode_steps_per_chunk=r)
     sched = op.mixed_schedule(w.block_lens.tolist(), chunk, T, r)
     assert s.param(B.PARAM_NUM_STEPS) == len(sched)
@@ -90,7 +90,17 @@ def run_chunked_event(w, chunk, decode_sms=0, rows=None, what="", r=1):
         slots += [op.slot_of(plan, w.page_size, b, int(w.block_lens[b]) + t) for b in range(Bn)]
         ks.append(w.k_dec[t])
         vs.append(w.v_dec[t])
-    if T or rows is None:
+    if sparse_pool:
+        # a pool of many gigabytes with a few pages in use: compare the written slots only, page by page
+        k_all, v_all = np.concatenate(ks), np.concatenate(vs)
+        for pool, want in ((s.k_pool, k_all), (s.v_pool, v_all)):
+            pages = {}
+            for i, slot in enumerate(slots):
+                page, off = slot // w.page_size, slot % w.page_size
+                if page not in pages:
+                    pages[page] = pool_rows(_bits(pool[page:page + 1]))[0]
+                assert np.array_equal(pages[page][:, off], want[i]), (i, slot)
+    elif T or rows is None:
         kp, vp, written = oa.expected_pool(slots, np.concatenate(ks), np.concatenate(vs), w.num_pages, w.page_size)
         mask = np.broadcast_to(written[:, None, :, None], kp.shape)
         assert np.array_equal(pool_rows(_bits(s.k_pool))[mask], kp[mask])
@@ -115,6 +125,20 @@ def test_several_decode_steps_beside_one_chunk(r):
     # the short blocks finish their summaries (6 tokens) while the long block is still on its second and third
     # chunk, sit out until the schedule ends, and the long block starts to decode right after its last chunk
     run_chunked_event(wl.custom([700, 100, 50, 129], 8, 2, 128, steps=6, seed=80 + r), 256, what=f"r = {r}", r=r)
+
+
+def test_page_ids_on_both_sides_of_the_four_gigabyte_line():
+    # 8 kv heads x 16 tokens x 128 dims x 2 bytes = 32 KiB per page and pool: page 131072 starts at byte 2^32.  The
+    # blocks' pages come from just below and well above that line, in a seeded shuffle, so every path that turns a
+    # page id into an address (chunk append, cached-prefix tiles of later chunks through tensor maps, decode's bulk
+    # copies, the fused append) has to do it in 64 bits.  The pools (9.2 GB together) are left uninitialised.
+    w = wl.custom([700, 130, 385], 32, 8, 128, steps=3, seed=111).materialise()
+    n = w.pages_needed
+    ids = np.concatenate([np.arange(131072 - n // 2, 131072), np.arange(147000, 147000 + n - n // 2)])
+    w.free_pages = np.random.default_rng(111).permutation(ids).astype(np.int32)
+    w.spare_pages = int(ids.max()) + 1 - n
+    assert w.num_pages * 32768 > 2 ** 32
+    run_chunked_event(w, 256, what="pages beyond 4 GB", r=2, sparse_pool=True)
 
 
 def test_one_chunk_covers_every_block():
