@@ -164,9 +164,10 @@ enum {
  *   least 5 % less than the uniform cut, a second item in a CTA counted as 16 pages (CPA_PARAM_DECODE_EVEN_CUT); CPA_ARR_DECODE_ITEMS
  *   is then in launch order (CTA-major rounds) instead of descending size.
  * block_lens, free_pages: host int32 arrays (copied; caller keeps ownership).
- * Page ids must be >= 0 and distinct (distinctness is the caller's contract).
+ * Page ids must be >= 0, at most (2^31 - 1) / max(64, 32 * num_kv_heads) (the pools' rows are addressed with
+ * 32-bit coordinates; far beyond what fits a device), and distinct (distinctness is the caller's contract).
  * Errors: CPA_EINVAL (null pointer, num_blocks < 1, a length < 1,
- * max_new_tokens < 0, negative page id, heads not divisible), CPA_EUNSUPPORTED,
+ * max_new_tokens < 0, page id out of range, heads not divisible), CPA_EUNSUPPORTED,
  * CPA_ENOSPC (num_free too small).  On error *out is NULL.
  */
 CPA_API int cpa_plan_create(const cpa_config* cfg, int32_t num_blocks, const int32_t* block_lens,

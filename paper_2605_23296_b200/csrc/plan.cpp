@@ -109,6 +109,8 @@ int plan_create(const cpa_config* cfg, int32_t num_blocks, const int32_t* block_
     p->q_tile = cfg->q_tile_rows ? cfg->q_tile_rows : 256;
     const int32_t P = cfg->page_size;
     const int32_t B = num_blocks;
+    // a pool's rows (page * Hkv + head) * P + slot are 32-bit tensor-map coordinates, and a slot is page * P + offset
+    const int32_t max_page_id = INT32_MAX / std::max(64, 2 * P * cfg->num_kv_heads);
 
     p->block_lens.assign(block_lens, block_lens + B);
     p->prefix_lens.assign(B, 0);
@@ -167,11 +169,11 @@ int plan_create(const cpa_config* cfg, int32_t num_blocks, const int32_t* block_
         p->free_ring.assign(free_pages + taken, free_pages + num_free);
         p->ring_size = std::max(1, num_free);
         for (int32_t id : p->free_ring)
-            if (id < 0 || id > INT32_MAX / 64) { delete p; return CPA_EINVAL; }
+            if (id < 0 || id > max_page_id) { delete p; return CPA_EINVAL; }
     }
     int32_t max_page = 0;
     for (int32_t id : p->page_indices) {
-        if (id < 0 || id > INT32_MAX / 64) { delete p; return CPA_EINVAL; }
+        if (id < 0 || id > max_page_id) { delete p; return CPA_EINVAL; }
         max_page = std::max(max_page, id);
     }
     p->pool_pages = max_page + 1;

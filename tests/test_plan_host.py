@@ -210,6 +210,16 @@ def test_plan_errors():
     assert rc(T=-1) == B.CPA_EINVAL
     assert rc(fr=np.arange(5, dtype=np.int32)) == B.CPA_ENOSPC   # too few pages
     assert rc(fr=np.array([0, 1, 2, -4, 5, 6, 7, 8], dtype=np.int32)) == B.CPA_EINVAL
+    # the largest page id: (2^31 - 1) / max(64, 32 * kv heads), so that a pool's rows keep 32-bit coordinates
+    top = (2 ** 31 - 1) // 64
+    assert rc(fr=np.array([0, 1, 2, top + 1, 5, 6, 7, 8], dtype=np.int32)) == B.CPA_EINVAL
+    handle = B.cpa_plan_create(ok, (40, 50), 4, np.array([0, 1, 2, top, 5, 6, 7, 8], dtype=np.int32))
+    B.cpa_plan_destroy(handle)
+    wide = B.cpa_config(32, 8, 64, 16, 0.125, 0, 0, 0)
+    top8 = (2 ** 31 - 1) // 256
+    assert rc(cfg=wide, fr=np.array([0, 1, 2, top8 + 1, 5, 6, 7, 8], dtype=np.int32)) == B.CPA_EINVAL
+    handle = B.cpa_plan_create(wide, (40, 50), 4, np.array([0, 1, 2, top8, 5, 6, 7, 8], dtype=np.int32))
+    B.cpa_plan_destroy(handle)
     assert rc(cfg=B.cpa_config(8, 3, 64, 16, 0.125, 0, 0, 0)) == B.CPA_EINVAL        # 8 % 3
     assert rc(cfg=B.cpa_config(8, 2, 96, 16, 0.125, 0, 0, 0)) == B.CPA_EUNSUPPORTED  # head_dim
     assert rc(cfg=B.cpa_config(8, 2, 64, 32, 0.125, 0, 0, 0)) == B.CPA_EUNSUPPORTED  # page size
