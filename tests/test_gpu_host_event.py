@@ -115,8 +115,10 @@ def test_a_second_event_reuses_stage_and_streams_after_a_new_upload():
     s.close()
 
 
-def test_prefix_aware_workers_from_host():
-    # both layouts' planner paths in one event: history cached first, workers' own tokens in chunks from the host
+@pytest.mark.parametrize("chunk", [256, 0])
+def test_prefix_aware_workers_from_host(chunk):
+    # both layouts' planner paths in one event: history cached first, workers' own tokens from the host, in chunks
+    # or (chunk 0: a plain prefix-aware plan) whole
     import torch
     from paper_2605_23296_b200 import binding as B
     from paper_2605_23296_b200.session import CompactionSession, bits_to_tensor
@@ -130,7 +132,7 @@ def test_prefix_aware_workers_from_host():
     hist.append_prefill(bits_to_tensor(w.k_hist, "cuda:0"), bits_to_tensor(w.v_hist, "cuda:0"))
     s = CompactionSession(o.block_lens, o.decode_steps, o.num_q_heads, o.num_kv_heads, o.head_dim, o.free_pages,
                           w.num_pages, scale=o.scale, prefix_lens=w.prefix_lens, shared_pages=w.shared_pages,
-                          pools=pools, chunk_tokens=256, decode_sms=1)
+                          pools=pools, chunk_tokens=chunk, decode_sms=1 if chunk else 0)
     h = [_pinned(x) for x in (o.q, o.k, o.v, o.q_dec, o.k_dec, o.v_dec)]
     h_o, h_od = torch.zeros_like(h[0]).pin_memory(), torch.zeros_like(h[3]).pin_memory()
     s.event_from_host(h[0], h[1], h[2], h_o, h[3], h[4], h[5], h_od)
