@@ -487,6 +487,8 @@ CPA_API int cpa_step_mixed(cpa_plan* plan, int32_t step, const void* q, const vo
  * when `stream` has been synchronised, and cpa_plan_status tells whether a kernel gave up.
  * Errors: CPA_EINVAL (null or misaligned pointer), CPA_ESTATE (plan not uploaded, or something was
  * already appended or stepped since the upload), CPA_EUNSUPPORTED (a plan with pages on demand), CPA_ECUDA.
+ * After CPA_ECUDA part of the event may have been enqueued: synchronise `stream` and upload the plan again
+ * before using it further.
  */
 CPA_API int cpa_event_host(cpa_plan* plan, const void* h_q, const void* h_k, const void* h_v, void* h_o,
                            const void* h_q_dec, const void* h_k_dec, const void* h_v_dec, void* h_o_dec,
