@@ -35,7 +35,9 @@ def _table_rows(s):
     return [idx[indptr[b]:indptr[b + 1]].tolist() for b in range(len(indptr) - 1)]
 
 
-def run_dynamic_event(w, stop_lens, spare_pages, release_every=0, what=""):
+def run_dynamic_event(w, stop_lens, spare_pages, release_every=0, what="", prefill_rows=None, check_steps=None):
+    """`prefill_rows` / `check_steps`: at full size the oracle sees a sample of the prefill rows and of the decode
+    steps (every live block at those steps); the page bookkeeping is checked at every step either way."""
     import torch
     from paper_2605_23296_b200 import binding as B
     from paper_2605_23296_b200.session import CompactionSession
@@ -54,7 +56,11 @@ def run_dynamic_event(w, stop_lens, spare_pages, release_every=0, what=""):
     cu = _cu(w)
     k, v = _dev(w.k), _dev(w.v)
     o = s.prefill(_dev(w.q), k, v)
-    assert_attention_close(_bits(o), oa.prefill(w.q, w.k, w.v, cu, w.scale), f"{what} prefill")
+    if prefill_rows is None:
+        assert_attention_close(_bits(o), oa.prefill(w.q, w.k, w.v, cu, w.scale), f"{what} prefill")
+    else:
+        got = _bits(o[torch.from_numpy(prefill_rows).to("cuda:0")])
+        assert_attention_close(got, oa.prefill(w.q, w.k, w.v, cu, w.scale, rows=prefill_rows), f"{what} prefill (sampled rows)")
     s.append_prefill(k, v)
     st = oa.DecodeState(w.k, w.v, cu, T)
     qd, kd, vd = _dev(w.q_dec), _dev(w.k_dec), _dev(w.v_dec)
@@ -67,10 +73,9 @@ def run_dynamic_event(w, stop_lens, spare_pages, release_every=0, what=""):
         model.step(active.tolist())
         live = np.flatnonzero(active).tolist()
         st.append(w.k_dec[t], w.v_dec[t], blocks=live)
-        want = st.decode(w.q_dec[t], w.scale, blocks=live)
-        got = _bits(out)
-        if live:
-            assert_attention_close(got[live], want[live], f"{what} step {t}")
+        if live and (check_steps is None or t in check_steps):
+            want = st.decode(w.q_dec[t], w.scale, blocks=live)
+            assert_attention_close(_bits(out)[live], want[live], f"{what} step {t}")
         idle = np.flatnonzero(~active)
         assert (out[torch.from_numpy(idle).to("cuda:0")] == 5.0).all(), f"{what}: step {t} wrote rows of idle blocks"
         if release_every and t % release_every == release_every - 1:
@@ -111,6 +116,25 @@ def test_stopped_blocks_give_their_pages_back():
     w = wl.custom(lens, 8, 2, 128, steps=48, seed=93, permute_pages=True)
     stop = np.where(np.arange(20) % 2 == 0, 8, 48).astype(np.int32)      # half of them stop after 8 tokens
     run_dynamic_event(w, stop, spare_pages=12, release_every=8, what="release")
+
+
+def test_many_short_sequences_at_full_size():
+    # the benchmark's second workload as it is timed (192 sequences of 514..1021 tokens, summaries that stop after
+    # 33..256 tokens, stopped sequences released every 32 steps): page bookkeeping at every step, the oracle on
+    # sampled prefill rows and on every live sequence at sampled steps (page boundaries of the summaries included)
+    w = wl.locomo_like().materialise()
+    rng = np.random.default_rng(6)
+    cu = _cu(w)
+    rows = []
+    for b, L in enumerate(int(x) for x in w.block_lens):
+        cand = {0, 1, 127, 128, 255, 256, 511, 512, L - 2, L - 1} | set(int(x) for x in rng.integers(0, L, 4))
+        rows += [cu[b] + r for r in sorted(cand) if 0 <= r < L]
+    steps = {0, 1, 15, 16, 17, 31, 32, 33, 63, 64, 127, 128, 200, 254, 255}
+    # the pool the benchmark gives it: the first pages plus what the summaries really need (+ 64), not T tokens each
+    first = int((w.block_lens // w.page_size + 1).sum())
+    need = int((-(-(w.block_lens.astype(np.int64) + w.stop_lens) // w.page_size)).sum())
+    run_dynamic_event(w, w.stop_lens, spare_pages=max(first, need) + 64 - first, release_every=32, what="192 short sequences",
+                      prefill_rows=np.asarray(rows, dtype=np.int64), check_steps=steps)
 
 
 def test_whole_batch_without_flags_equals_the_reserved_plan_bitwise():
