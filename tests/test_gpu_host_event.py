@@ -148,3 +148,41 @@ def test_prefix_aware_workers_from_host(chunk):
     assert np.array_equal(s.export(B.ARR_SEQ_LENS), w.prefix_lens + o.block_lens + o.decode_steps)
     s.close()
     hist.close()
+
+
+def test_ragged_at_full_size_through_the_host_call():
+    # the benchmark's end-to-end leg as it is timed: the default workload, chunks of 4096 tokens, pinned host
+    # buffers; prefill on sampled rows (block ends, tile and chunk boundaries, random rows), every block and head of
+    # the decode at sampled steps, lengths at the end
+    import torch
+    from paper_2605_23296_b200 import binding as B
+    from paper_2605_23296_b200.session import CompactionSession
+    w = wl.ragged().materialise()
+    T, chunk = w.decode_steps, 4096
+    s = CompactionSession(w.block_lens, T, w.num_q_heads, w.num_kv_heads, w.head_dim, w.free_pages, w.num_pages,
+                          scale=w.scale, chunk_tokens=chunk, decode_sms=1)
+    h = [_pinned(x) for x in (w.q, w.k, w.v, w.q_dec, w.k_dec, w.v_dec)]
+    h_o = torch.empty(h[0].shape, dtype=torch.bfloat16).pin_memory()
+    h_od = torch.empty(h[3].shape, dtype=torch.bfloat16).pin_memory()
+    s.event_from_host(h[0], h[1], h[2], h_o, h[3], h[4], h[5], h_od)
+    torch.cuda.synchronize()
+    assert s.status() == 0
+    cu = np.concatenate([[0], np.cumsum(w.block_lens.astype(np.int64))])
+    rng = np.random.default_rng(2)
+    rows = []
+    for b, L in enumerate(int(x) for x in w.block_lens):
+        cand = {0, 1, 127, 128, L - 2, L - 1} | {c + d for c in range(chunk, L, chunk) for d in (-1, 0, 1)}
+        cand |= set(int(x) for x in rng.integers(0, L, 4))
+        rows += [cu[b] + r for r in sorted(cand) if 0 <= r < L]
+    rows = np.asarray(rows, dtype=np.int64)
+    assert_attention_close(_host_bits(h_o)[rows], oa.prefill(w.q, w.k, w.v, cu, w.scale, rows=rows),
+                           "ragged prefill from host (sampled rows)", allow_big=False)
+    checks = {0, 1, 15, 16, 17, 300, T - 1}
+    st = oa.DecodeState(w.k, w.v, cu, T)
+    for t in range(T):
+        st.append(w.k_dec[t], w.v_dec[t])
+        if t in checks:
+            assert_attention_close(_host_bits(h_od[t]), st.decode(w.q_dec[t], w.scale), f"ragged decode step {t} from host",
+                                   allow_big=False)
+    assert np.array_equal(s.export(B.ARR_SEQ_LENS), w.block_lens + T)
+    s.close()
