@@ -296,7 +296,10 @@ def measure_event(w, args, dev, steps: int, warmup: int, with_e2e: bool, world: 
         s.append_prefill(k, v)
         if ev:
             ev["appended"].record(stream)
-        for t in range(T):
+        if not args.separate_append and dec_events is None and T > 0:
+            # all T fused steps enqueued by one call (their inputs are on the device already)
+            s.decode_append_steps(qd, kd, vd, out=od)
+        for t in (range(T) if args.separate_append or dec_events is not None else ()):
             sampled = dec_events is not None and t % sample_every == 0
             if args.separate_append:
                 s.append(kd[t], vd[t])
@@ -339,7 +342,8 @@ def measure_event(w, args, dev, steps: int, warmup: int, with_e2e: bool, world: 
     for _ in range(steps):
         flush.fill_(1)   # L2 flush between timed steps (the step's own inputs, 400+ MB, exceed L2 anyway)
         ev = {n: torch.cuda.Event(enable_timing=True) for n in ("start", "planned", "prefilled", "appended", "end")}
-        dec_events = []
+        # (with separate append and decode calls the launch time comes from event pairs around sampled launches)
+        dec_events = [] if args.separate_append else None
         ev["start"].record(stream)
         s = one_pass(d_q, d_k, d_v, d_qd, d_kd, d_vd, d_o, d_od, ev, dec_events)
         ev["end"].record(stream)
@@ -351,9 +355,19 @@ def measure_event(w, args, dev, steps: int, warmup: int, with_e2e: bool, world: 
         prefill_ms.append(ev["planned"].elapsed_time(ev["prefilled"]))
         append_ms.append(ev["prefilled"].elapsed_time(ev["appended"]))
         decode_ms.append(ev["appended"].elapsed_time(ev["end"]))
-        dec_samples += [(t, e0.elapsed_time(e1)) for t, e0, e1 in dec_events]
+        dec_samples += [(t, e0.elapsed_time(e1)) for t, e0, e1 in (dec_events or [])]
     barrier()
     launches = state["launches"]
+    if not args.separate_append:
+        # event pairs around single launches, for comparison with the phase time / T: one more pass, not timed as a
+        # step (the pairs add their own cost and break the overlap of consecutive launches)
+        flush.fill_(1)
+        dec_events = []
+        s = one_pass(d_q, d_k, d_v, d_qd, d_kd, d_vd, d_o, d_od, None, dec_events)
+        torch.cuda.synchronize(dev)
+        assert s.status() == 0
+        s.close()
+        dec_samples += [(t, e0.elapsed_time(e1)) for t, e0, e1 in dec_events]
 
     # ---- end to end: host buffers in, host buffers out, copies inside the timed region -----
     e2e_ms, h2d, d2h = [], 0, 0

@@ -412,6 +412,18 @@ CPA_API int cpa_decode_append(cpa_plan* plan, const void* q, const void* k_new, 
                               void* v_pool, void* o, void* d_workspace, void* stream);
 
 /*
+ * cpa_decode_append_steps -- `num_steps` consecutive cpa_decode_append calls enqueued by one call, for
+ * callers whose inputs of several steps are on the device already (a benchmark, a replay; in a model the next
+ * step's query depends on this step's output, so there it is one step per call).
+ *   q, o          : device bf16 [num_steps, B, num_q_heads, head_dim]; step t uses slice t
+ *   k_new, v_new  : device bf16 [num_steps, B, num_kv_heads, head_dim]
+ * Everything else, and the errors, as for cpa_decode_append; the capacity of every block is checked for all
+ * steps before the first launch (CPA_ENOSPC: nothing is launched).  num_steps < 0: CPA_EINVAL; 0: nothing to do.
+ */
+CPA_API int cpa_decode_append_steps(cpa_plan* plan, const void* q, const void* k_new, const void* v_new, void* k_pool,
+                                    void* v_pool, void* o, void* d_workspace, int32_t num_steps, void* stream);
+
+/*
  * cpa_decode_append_dynamic -- cpa_decode_append for a plan with pages on demand (cpa_plan_create_dynamic;
  * Section 8, "Dynamic block size and prompt selection"), with per-block stop flags that live on the device, so
  * that summaries of different, unknown lengths need neither a new plan nor a host round trip per step.

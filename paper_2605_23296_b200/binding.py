@@ -83,6 +83,8 @@ _lib.cpa_release_blocks.restype = ctypes.c_int
 _lib.cpa_step_mixed.argtypes = [_vp, ctypes.c_int32] + [_vp] * 12
 _lib.cpa_step_mixed.restype = ctypes.c_int
 _lib.cpa_event_host.argtypes = [_vp] * 14
+_lib.cpa_decode_append_steps.argtypes = [_vp] * 8 + [ctypes.c_int32, _vp]
+_lib.cpa_decode_append_steps.restype = ctypes.c_int
 _lib.cpa_partition.argtypes = [ctypes.c_int64, ctypes.c_int32, _i32p, ctypes.c_int32, ctypes.POINTER(ctypes.c_int32)]
 _lib.cpa_partition.restype = ctypes.c_int
 _lib.cpa_event_host.restype = ctypes.c_int
@@ -307,6 +309,12 @@ def cpa_step_mixed(plan: int, step: int, q, k, v, o, q_dec, k_new, v_new, o_dec,
                    stream: int = 0) -> int:
     return _lib.cpa_step_mixed(plan, int(step), _ptr(q), _ptr(k), _ptr(v), _ptr(o), _ptr(q_dec), _ptr(k_new),
                                _ptr(v_new), _ptr(o_dec), _ptr(k_pool), _ptr(v_pool), _ptr(d_workspace), stream or None)
+
+
+def cpa_decode_append_steps(plan: int, q, k_new, v_new, k_pool, v_pool, o, d_workspace, num_steps: int,
+                            stream: int = 0) -> int:
+    return _lib.cpa_decode_append_steps(plan, _ptr(q), _ptr(k_new), _ptr(v_new), _ptr(k_pool), _ptr(v_pool), _ptr(o),
+                                        _ptr(d_workspace), int(num_steps), stream or None)
 
 
 def cpa_event_host(plan: int, h_q, h_k, h_v, h_o, h_q_dec, h_k_dec, h_v_dec, h_o_dec, d_stage, k_pool, v_pool,

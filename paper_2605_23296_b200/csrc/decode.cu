@@ -901,6 +901,26 @@ extern "C" int cpa_decode_append(cpa_plan* plan, const void* q, const void* k_ne
     return CPA_OK;
 }
 
+extern "C" int cpa_decode_append_steps(cpa_plan* plan, const void* q, const void* k_new, const void* v_new, void* k_pool,
+                                       void* v_pool, void* o, void* d_workspace, int32_t num_steps, void* stream) {
+    if (!plan || num_steps < 0) return CPA_EINVAL;
+    if (num_steps == 0) return CPA_OK;
+    if (!plan->d_base) return CPA_ESTATE;
+    for (int b = 0; b < plan->B; ++b)
+        if ((int64_t)plan->seq_lens[b] + num_steps > (int64_t)plan->prefix_lens[b] + plan->block_lens[b] + plan->T)
+            return CPA_ENOSPC;
+    const int64_t q_step = (int64_t)plan->B * plan->cfg.num_q_heads * plan->cfg.head_dim * 2;     // bytes per step
+    const int64_t kv_step = (int64_t)plan->B * plan->cfg.num_kv_heads * plan->cfg.head_dim * 2;
+    for (int32_t t = 0; t < num_steps; ++t) {
+        const int rc = cpa_decode_append(plan, static_cast<const char*>(q) + t * q_step,
+                                         static_cast<const char*>(k_new) + t * kv_step,
+                                         static_cast<const char*>(v_new) + t * kv_step, k_pool, v_pool,
+                                         static_cast<char*>(o) + t * q_step, d_workspace, stream);
+        if (rc != CPA_OK) return rc;
+    }
+    return CPA_OK;
+}
+
 extern "C" int cpa_decode_append_dynamic(cpa_plan* plan, const void* q, const void* k_new, const void* v_new,
                                          const int32_t* d_active, void* k_pool, void* v_pool, void* o,
                                          void* d_workspace, void* stream) {

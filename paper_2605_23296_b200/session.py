@@ -144,6 +144,16 @@ class CompactionSession:
                                         self.workspace, self._stream()), "cpa_decode_append")
         return out
 
+    def decode_append_steps(self, q: torch.Tensor, k_new: torch.Tensor, v_new: torch.Tensor,
+                            out: Optional[torch.Tensor] = None) -> torch.Tensor:
+        """q/out [n,B,Hq,d], k_new/v_new [n,B,Hkv,d]: n consecutive fused decode steps enqueued by one call."""
+        if out is None:
+            out = torch.empty_like(q)
+        assert q.is_contiguous() and k_new.is_contiguous() and v_new.is_contiguous() and out.is_contiguous()
+        self._check(B.cpa_decode_append_steps(self.plan, q, k_new, v_new, self.k_pool, self.v_pool, out,
+                                              self.workspace, q.shape[0], self._stream()), "cpa_decode_append_steps")
+        return out
+
     def step_mixed(self, step: int, q, k, v, out, q_dec=None, k_new=None, v_new=None, out_dec=None) -> None:
         """Step `step` of a chunked plan: the chunk that starts at this step, if any (rows of the whole-event
         tensors q/k/v/out), beside one decode token of the blocks whose turn it is."""

@@ -269,6 +269,33 @@ def test_fused_decode_append_matches_oracle_and_separate_calls(hq, hkv, d):
     plain.close()
 
 
+def test_several_steps_in_one_call_are_the_single_steps():
+    # cpa_decode_append_steps is a loop over cpa_decode_append inside the library: same outputs, same pools, same
+    # lengths, bit for bit; a request beyond the reservation is refused before anything is launched
+    from paper_2605_23296_b200 import binding as B
+    w = wl.custom([1, 15, 16, 250, 1000], 8, 2, 128, steps=12, seed=41).materialise()
+    one, many = _session(w, poison=True), _session(w, poison=True)
+    for s in (one, many):
+        s.append_prefill(_dev(w.k), _dev(w.v))
+    kd, vd, qd = _dev(w.k_dec), _dev(w.v_dec), _dev(w.q_dec)
+    ref = np.stack([_bits(one.decode_append(qd[t], kd[t], vd[t])) for t in range(12)])
+    got = many.decode_append_steps(qd[:5], kd[:5], vd[:5])
+    got2 = many.decode_append_steps(qd[5:], kd[5:], vd[5:])
+    assert many.status() == 0
+    assert np.array_equal(np.concatenate([_bits(got), _bits(got2)]), ref)
+    assert np.array_equal(_bits(one.k_pool), _bits(many.k_pool)) and np.array_equal(_bits(one.v_pool), _bits(many.v_pool))
+    assert np.array_equal(many.export(3), w.block_lens + 12)
+    st = oa.DecodeState(w.k, w.v, _cu(w), 12)
+    for t in range(12):
+        st.append(w.k_dec[t], w.v_dec[t])
+    assert_attention_close(ref[11], st.decode(w.q_dec[11], w.scale), "last of twelve steps")
+    assert B.cpa_decode_append_steps(many.plan, qd, kd, vd, many.k_pool, many.v_pool, got, many.workspace, 1) == B.CPA_ENOSPC
+    assert B.cpa_decode_append_steps(many.plan, qd, kd, vd, many.k_pool, many.v_pool, got, many.workspace, -1) == B.CPA_EINVAL
+    assert B.cpa_decode_append_steps(many.plan, qd, kd, vd, many.k_pool, many.v_pool, got, many.workspace, 0) == B.CPA_OK
+    one.close()
+    many.close()
+
+
 @pytest.mark.parametrize("nb,L,hq,hkv,d,sms", [(27, 1500, 8, 2, 128, 16), (25, 1000, 4, 1, 64, 8)])
 def test_decode_with_the_even_cut(nb, L, hq, hkv, d, sms):
     # equal blocks whose count does not divide the wave: the planner cuts all pages, laid end to end, into equal

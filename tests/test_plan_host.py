@@ -359,6 +359,9 @@ def test_event_from_host_argument_checks_and_stage_size():
     assert B.cpa_plan_param(plan, B.PARAM_HOST_STAGE_BYTES) == want
     f = 4096
     assert B.cpa_event_host(plan, f, f, f, f, f, f, f, f, f, f, f, f) == B.CPA_ESTATE          # not uploaded
+    assert B.cpa_decode_append_steps(plan, f, f, f, f, f, f, f, 2) == B.CPA_ESTATE
+    assert B.cpa_decode_append_steps(plan, f, f, f, f, f, f, f, -2) == B.CPA_EINVAL
+    assert B.cpa_decode_append_steps(plan, f, f, f, f, f, f, f, 0) == B.CPA_OK
     assert B.cpa_event_host(plan, None, f, f, f, f, f, f, f, f, f, f, f) == B.CPA_EINVAL
     assert B.cpa_event_host(plan, f, f, f, f, None, f, f, f, f, f, f, f) == B.CPA_EINVAL       # T > 0 needs decode inputs
     assert B.cpa_event_host(plan, f, f, f, f, f, f, f, f, f + 16, f, f, f) == B.CPA_EINVAL     # stage not 256-aligned
