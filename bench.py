@@ -681,10 +681,10 @@ def run_mixed(args) -> None:
         ev["start"].record(stream)      # (planning and the plan's upload are outside both measurements)
         s.prefill(q, k, v, out=o)
         s.append_prefill(k, v)
-        for t in range(T):
-            s.decode_append(qd[t], kd[t], vd[t], out=od[t])
-            if t == 0:
-                ev["first"].record(stream)
+        s.decode_append_steps(qd[:1], kd[:1], vd[:1], out=od[:1])
+        ev["first"].record(stream)
+        if T > 1:      # the remaining steps enqueued by one call (inputs staged on the device)
+            s.decode_append_steps(qd[1:], kd[1:], vd[1:], out=od[1:T])
         ev["end"].record(stream)
         return s, ev
 
@@ -703,19 +703,28 @@ def run_mixed(args) -> None:
             t_of = np.clip(step - start, 0, T - 1)
             steps_in.append(torch.from_numpy(t_of.astype(np.int64)).to(dev))
         ar = torch.arange(Bn, device=dev)
-        gathered = [(qd[t_of, ar], kd[t_of, ar], vd[t_of, ar]) for t_of in steps_in]   # staged before the timed calls
+        # staged before the timed calls: [n_steps, B, H, d], slice i = the decode inputs of step i
+        q_in = torch.stack([qd[t_of, ar] for t_of in steps_in]).contiguous()
+        k_in = torch.stack([kd[t_of, ar] for t_of in steps_in]).contiguous()
+        v_in = torch.stack([vd[t_of, ar] for t_of in steps_in]).contiguous()
+        o_out = torch.empty_like(q_in)
         torch.cuda.synchronize(dev)
         ev["start"].record(stream)
-        for step in range(n_steps):
-            qi, ki, vi = gathered[step]
-            s.step_mixed(step, q, k, v, o, qi, ki, vi, od[step % (T + 8)])
-            if step == int(start.min()):
-                ev["first"].record(stream)
-            if step == int(start.min()) + T - 1:
-                ev["short_done"].record(stream)
-            if step == n_long - 1:
-                ev["long_prefilled"].record(stream)
-        ev["end"].record(stream)
+        # the steps between two time stamps are enqueued by one call each
+        marks = sorted({int(start.min()): "first", int(start.min()) + T - 1: "short_done", n_long - 1: "long_prefilled",
+                        n_steps - 1: "end"}.items())
+        done = 0
+        stamped = set()
+        for last, _ in marks:
+            if last + 1 > done:
+                s.step_mixed_range(done, last + 1 - done, q, k, v, o, q_in[done:last + 1], k_in[done:last + 1],
+                                   v_in[done:last + 1], o_out[done:last + 1])
+                done = last + 1
+            for step, name in ((int(start.min()), "first"), (int(start.min()) + T - 1, "short_done"),
+                               (n_long - 1, "long_prefilled"), (n_steps - 1, "end")):
+                if step == last and name not in stamped:
+                    ev[name].record(stream)
+                    stamped.add(name)
         return s, ev
 
     res = {"whole_blocks": [], "chunked": []}

@@ -477,6 +477,18 @@ CPA_API int cpa_step_mixed(cpa_plan* plan, int32_t step, const void* q, const vo
                            void* v_pool, void* d_workspace, void* stream);
 
 /*
+ * cpa_step_mixed_range -- steps first_step .. first_step + num_steps - 1 of the schedule enqueued by one call
+ * (cpa_step_mixed in a loop inside the library), for callers whose decode inputs of several steps are on the
+ * device already.  q_dec, o_dec: device bf16 [num_steps, B, num_q_heads, head_dim], slice i for step
+ * first_step + i (rows of the blocks that decode in that step, as for cpa_step_mixed); k_new, v_new likewise
+ * with num_kv_heads.  Everything else and the errors as for cpa_step_mixed; a step that fails ends the range
+ * (the steps before it have been enqueued).
+ */
+CPA_API int cpa_step_mixed_range(cpa_plan* plan, int32_t first_step, int32_t num_steps, const void* q, const void* k,
+                                 const void* v, void* o, const void* q_dec, const void* k_new, const void* v_new,
+                                 void* o_dec, void* k_pool, void* v_pool, void* d_workspace, void* stream);
+
+/*
  * cpa_event_host -- a whole compaction event with inputs and outputs in HOST memory: the prefill of every
  * block (Section 4, "Dispatch": each worker runs its prompt), the append of the prompts' K/V, and
  * max_new_tokens decode steps over all blocks, each with its append (the workers' summaries, Section 4).  The

@@ -83,6 +83,8 @@ _lib.cpa_release_blocks.restype = ctypes.c_int
 _lib.cpa_step_mixed.argtypes = [_vp, ctypes.c_int32] + [_vp] * 12
 _lib.cpa_step_mixed.restype = ctypes.c_int
 _lib.cpa_event_host.argtypes = [_vp] * 14
+_lib.cpa_step_mixed_range.argtypes = [_vp, ctypes.c_int32, ctypes.c_int32] + [_vp] * 12
+_lib.cpa_step_mixed_range.restype = ctypes.c_int
 _lib.cpa_decode_append_steps.argtypes = [_vp] * 8 + [ctypes.c_int32, _vp]
 _lib.cpa_decode_append_steps.restype = ctypes.c_int
 _lib.cpa_partition.argtypes = [ctypes.c_int64, ctypes.c_int32, _i32p, ctypes.c_int32, ctypes.POINTER(ctypes.c_int32)]
@@ -323,6 +325,13 @@ def cpa_event_host(plan: int, h_q, h_k, h_v, h_o, h_q_dec, h_k_dec, h_v_dec, h_o
     return _lib.cpa_event_host(plan, _ptr(h_q), _ptr(h_k), _ptr(h_v), _ptr(h_o), _ptr(h_q_dec), _ptr(h_k_dec),
                                _ptr(h_v_dec), _ptr(h_o_dec), _ptr(d_stage), _ptr(k_pool), _ptr(v_pool),
                                _ptr(d_workspace), stream or None)
+
+
+def cpa_step_mixed_range(plan: int, first_step: int, num_steps: int, q, k, v, o, q_dec, k_new, v_new, o_dec, k_pool,
+                         v_pool, d_workspace, stream: int = 0) -> int:
+    return _lib.cpa_step_mixed_range(plan, int(first_step), int(num_steps), _ptr(q), _ptr(k), _ptr(v), _ptr(o),
+                                     _ptr(q_dec), _ptr(k_new), _ptr(v_new), _ptr(o_dec), _ptr(k_pool), _ptr(v_pool),
+                                     _ptr(d_workspace), stream or None)
 
 
 STATIC_SCRATCH_BYTES = 16 << 20

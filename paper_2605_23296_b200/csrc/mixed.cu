@@ -103,3 +103,21 @@ extern "C" int cpa_step_mixed(cpa_plan* plan, int32_t step, const void* q, const
     plan->next_step = step + 1;
     return CPA_OK;
 }
+
+extern "C" int cpa_step_mixed_range(cpa_plan* plan, int32_t first_step, int32_t num_steps, const void* q, const void* k,
+                                    const void* v, void* o, const void* q_dec, const void* k_new, const void* v_new,
+                                    void* o_dec, void* k_pool, void* v_pool, void* d_workspace, void* stream) {
+    if (!plan || num_steps < 0) return CPA_EINVAL;
+    const int64_t q_step = (int64_t)plan->B * plan->cfg.num_q_heads * plan->cfg.head_dim * 2;     // bytes per step
+    const int64_t kv_step = (int64_t)plan->B * plan->cfg.num_kv_heads * plan->cfg.head_dim * 2;
+    auto at = [](const void* base, int64_t off) -> const void* {
+        return base ? static_cast<const char*>(base) + off : nullptr;
+    };
+    for (int32_t i = 0; i < num_steps; ++i) {
+        const int rc = cpa_step_mixed(plan, first_step + i, q, k, v, o, at(q_dec, i * q_step), at(k_new, i * kv_step),
+                                      at(v_new, i * kv_step), const_cast<void*>(at(o_dec, i * q_step)), k_pool, v_pool,
+                                      d_workspace, stream);
+        if (rc != CPA_OK) return rc;
+    }
+    return CPA_OK;
+}

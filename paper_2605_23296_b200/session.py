@@ -174,6 +174,14 @@ class CompactionSession:
                                      self.k_pool, self.v_pool, self.workspace, self._stream()), "cpa_event_host")
         return stage
 
+    def step_mixed_range(self, first_step: int, num_steps: int, q, k, v, out, q_dec=None, k_new=None, v_new=None,
+                         out_dec=None) -> None:
+        """Steps first_step .. first_step + num_steps - 1 of a chunked plan by one call; the decode tensors are
+        [num_steps, B, H, d], slice i for step first_step + i."""
+        self._check(B.cpa_step_mixed_range(self.plan, first_step, num_steps, q, k, v, out, q_dec, k_new, v_new,
+                                           out_dec, self.k_pool, self.v_pool, self.workspace, self._stream()),
+                    "cpa_step_mixed_range")
+
     def decode_append_dynamic(self, q, k_new, v_new, active=None, out=None):
         """One decode step of a plan with pages on demand; `active` is a device int32 [B] tensor of stop flags."""
         if out is None:

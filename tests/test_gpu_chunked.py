@@ -255,6 +255,41 @@ def test_prefix_aware_chunks_of_one_tile_with_one_decode_sm():
     run_prefix_chunked_event(w, 128, r=1, decode_sms=1, what="prefix + 128-token chunks")
 
 
+def test_a_range_of_steps_in_one_call_is_the_single_steps():
+    # cpa_step_mixed_range is cpa_step_mixed in a loop inside the library: outputs, pools and lengths bit for bit
+    import torch
+    from paper_2605_23296_b200 import binding as B
+    from paper_2605_23296_b200.session import CompactionSession
+    w = wl.custom([700, 100, 50, 129], 8, 2, 128, steps=5, seed=97).materialise()
+    T, Bn = 5, 4
+    q, k, v = _dev(w.q), _dev(w.k), _dev(w.v)
+    qd, kd, vd = _dev(w.q_dec), _dev(w.k_dec), _dev(w.v_dec)
+    res = []
+    for ranged in (False, True):
+        s = CompactionSession(w.block_lens, T, 8, 2, 128, w.free_pages, w.num_pages, scale=w.scale, poison_pools=True,
+                              chunk_tokens=256, decode_steps_per_chunk=2)
+        n = s.param(B.PARAM_NUM_STEPS)
+        start = torch.from_numpy(s.export(B.ARR_DEC_START).astype(np.int64)).to("cuda:0")
+        ar = torch.arange(Bn, device="cuda:0")
+        t_of = [torch.clamp(step - start, 0, T - 1) for step in range(n)]
+        q_in = torch.stack([qd[t, ar] for t in t_of]).contiguous()
+        k_in = torch.stack([kd[t, ar] for t in t_of]).contiguous()
+        v_in = torch.stack([vd[t, ar] for t in t_of]).contiguous()
+        o = torch.zeros_like(q)
+        out = torch.full_like(q_in, 5.0)
+        if ranged:
+            s.step_mixed_range(0, 3, q, k, v, o, q_in[:3], k_in[:3], v_in[:3], out[:3])
+            s.step_mixed_range(3, n - 3, q, k, v, o, q_in[3:], k_in[3:], v_in[3:], out[3:])
+        else:
+            for step in range(n):
+                s.step_mixed(step, q, k, v, o, q_in[step], k_in[step], v_in[step], out[step])
+        assert s.status() == 0
+        res.append((_bits(o), _bits(out), _bits(s.k_pool), _bits(s.v_pool), s.export(B.ARR_SEQ_LENS).copy()))
+        s.close()
+    for a, b in zip(res[0], res[1]):
+        assert np.array_equal(a, b)
+
+
 def test_mixed_step_needs_a_chunked_plan():
     from paper_2605_23296_b200 import binding as B
     from paper_2605_23296_b200.session import CompactionSession
