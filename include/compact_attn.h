@@ -9,7 +9,12 @@
  * library runs the attention of those N concurrent sequences in the
  * "independent chunks" layout of Section 4: a sequence sees its own block only,
  * so attention is block-diagonal and causal inside each block.  Sequential
- * compaction (Section 2.2, Eq. 1) is the N = 1 case of the same calls.
+ * compaction (Section 2.2, Eq. 1) is the N = 1 case of the same calls.  The same
+ * kernels serve the paper's own prefix-aware layout (cpa_plan_create_prefix: a
+ * worker reads the cached history up to its block, then runs its own tokens),
+ * prefill in chunks beside the decode of other blocks (cpa_plan_create_chunked,
+ * cpa_step_mixed), summaries of unknown length without reserved pages
+ * (cpa_plan_create_dynamic) and whole events from host memory (cpa_event_host).
  *
  * The paper does not spell out attention; it is the textbook operation
  *     O[i,h,:] = sum_{j<=i} softmax_j(scale * q[i,h,:].k[j,g,:]) v[j,g,:],  g = h div G,
